@@ -1,0 +1,272 @@
+"""Oracle prefetch policy "P0": roofline classification, residency (pin) selection and the
+ordered staging schedule.  Pure Python integers; no floating point anywhere.
+
+TEST INFRASTRUCTURE - see oracle/__init__.py.
+
+The paper describes the policy in prose only.  What it fixes, and where:
+* three kernel classes - CGI(link)-bound, GPU-memory-bound, compute-bound - from a roofline
+  with a compute roof, an HBM roof and a much lower CPU-GPU interconnect roof
+  (Section III-C; Section IV-C "UVM Analyzer");
+* prefetch exactly the tensors the upcoming kernel accesses, nothing else of the pool
+  (Section IV-B, IV-D "Prefetch Engine");
+* link-bound kernels trigger proactive prefetch; tensors reused across consecutive kernels
+  are held resident during their reuse window (Section IV-C look-ahead affinity, IV-D).
+Everything numeric below is this build's reading: the exact inequality, ties, the hold
+window W_AFF, the zero-copy ratio ZC_DEN, the ring minimum, the 512-byte alignment.
+
+Steps, in order (notation: P = peak flop/s, Bh = HBM bytes/s, Bl = host-link bytes/s):
+
+1. classify each op i with mig_i = sum of touched bytes of its pool accesses:
+     LINK    iff mig_i*P > flops_i*Bl and mig_i*Bh > hbm_i*Bl   (the link time exceeds both others)
+     COMPUTE iff not LINK and flops_i*Bh >= hbm_i*P
+     HBM     otherwise.                With the P bit off every op with mig_i > 0 is LINK.
+2. crit[t] iff a LINK op accesses t;  score[t] = sum of touched bytes over LINK-op accesses.
+3. zero-copy (ZC bit): a READONLY tensor whose every access touches < size/ZC_DEN bytes is read
+   in place over the link and never staged.
+4. residency episodes: consecutive accesses of t (same step, gap <= W_AFF ops) share one stay.
+   live_i = aligned bytes of all non-ZC episodes covering op i; ring_min = 2 * max_i live_i;
+   error if ring_min > budget.  pin_cap = budget - ring_min.
+5. pins (A bit): candidates score > 0, non-ZC, by density score/size descending (exact cross
+   products), tie -> lower id; greedy with skip while the aligned size fits in pin_cap.
+   Pins sit at [0, used); the ring is [used, budget).
+6. schedule: walk ops in order, accesses in list order.
+     pinned tensor, first access: LOAD (H2D into its slot), or ALLOC if MUTABLE and the access is W.
+     ring tensor, episode start: FIFO bump allocation (wrap to the ring base when the tail does
+       not fit), evicting the oldest stays it overlaps; wait_op = running max of the evicted stays'
+       last-use ops (and, for a MUTABLE tensor, of the op after which it was last written back);
+       kind H2D, or ALLOC when MUTABLE, never written and the access is W.
+       wait_op >= first_use -> error (ring too small).
+     ring tensor, episode end, written during the stay: D2H of the whole tensor after that op.
+"""
+from __future__ import annotations
+
+import struct
+from dataclasses import dataclass
+from typing import Dict, List, Tuple
+
+ALIGN = 512
+W_AFF = 4
+ZC_DEN = 2
+CLS_LINK, CLS_HBM, CLS_COMPUTE = 0, 1, 2
+CMD_H2D, CMD_ALLOC, CMD_D2H = 0, 1, 2
+BIT_A, BIT_P, BIT_ZC = 1, 2, 4
+MODE_R, MODE_W = 1, 2
+F_READONLY, F_MUTABLE = 1, 2
+
+
+class PlanError(Exception):
+    pass
+
+
+@dataclass
+class Machine:
+    peak_flops: int
+    hbm_Bps: int
+    h2d_Bps: int
+    d2h_Bps: int
+
+
+@dataclass
+class Cmd:
+    seq: int
+    kind: int
+    tensor: int
+    nbytes: int
+    pool_off: int
+    arena_off: int
+    wait_op: int
+    first_use: int
+    release_after: int
+
+    def pack(self) -> bytes:
+        return struct.pack("<IBIQQQiii", self.seq, self.kind, self.tensor, self.nbytes, self.pool_off,
+                           self.arena_off, self.wait_op, self.first_use, self.release_after)
+
+
+def alignup(x: int) -> int:
+    return (x + ALIGN - 1) // ALIGN * ALIGN
+
+
+def classify(flops: int, hbm: int, mig: int, m: Machine, bit_p: bool = True) -> int:
+    if mig > 0 and not bit_p:
+        return CLS_LINK
+    if mig * m.peak_flops > flops * m.h2d_Bps and mig * m.hbm_Bps > hbm * m.h2d_Bps:
+        return CLS_LINK
+    if flops * m.hbm_Bps >= hbm * m.peak_flops:
+        return CLS_COMPUTE
+    return CLS_HBM
+
+
+@dataclass
+class Plan:
+    cls: List[int]
+    crit: List[int]
+    score: List[int]
+    zc: List[int]
+    pins: List[Tuple[int, int]]
+    ring_base: int
+    ring_size: int
+    cmds: List[Cmd]
+    totals: List[Tuple[int, int, int, int]]       # per step (h2d bytes, d2h bytes, zc bytes, n cmds)
+    episodes: List[Tuple[int, int, int]]          # (tensor, first op, last op) of ring stays (diagnostic)
+
+    def blobs(self) -> Dict[str, bytes]:
+        return {
+            "classes": bytes(self.cls),
+            "tensors": b"".join(struct.pack("<BBQ", self.crit[t], self.zc[t], self.score[t]) for t in range(len(self.crit))),
+            "pins": b"".join(struct.pack("<IQ", t, o) for t, o in self.pins) + struct.pack("<QQ", self.ring_base, self.ring_size),
+            "commands": b"".join(c.pack() for c in self.cmds),
+            "totals": b"".join(struct.pack("<QQQQ", *x) for x in self.totals),
+        }
+
+
+def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A | BIT_P | BIT_ZC) -> Plan:
+    """tensors: list of objects with .size .pool_off .flags; ops: list with .step .flops .hbm .acc;
+    steps: [(kind, first op, count)]."""
+    T, N = len(tensors), len(ops)
+    # 1-2: classes, criticality, score
+    cls = []
+    crit = [0] * T
+    score = [0] * T
+    for op in ops:
+        mig = sum(a[2] for a in op.acc)
+        c = classify(op.flops, op.hbm, mig, machine, bool(bits & BIT_P))
+        cls.append(c)
+        if c == CLS_LINK:
+            for (t, _, touched) in op.acc:
+                crit[t] = 1
+                score[t] += touched
+    # 3: zero-copy
+    accessed = [0] * T
+    sparse = [1] * T
+    for op in ops:
+        for (t, _, touched) in op.acc:
+            accessed[t] = 1
+            if touched * ZC_DEN >= tensors[t].size:
+                sparse[t] = 0
+    zc = [1 if (bits & BIT_ZC) and accessed[t] and sparse[t] and tensors[t].flags == F_READONLY else 0 for t in range(T)]
+    # 4: episodes from the trace alone
+    step_of = [op.step for op in ops]
+    acc_ops: Dict[int, List[int]] = {}
+    for i, op in enumerate(ops):
+        for (t, _, _) in op.acc:
+            if not zc[t]:
+                lst = acc_ops.setdefault(t, [])
+                if not lst or lst[-1] != i:
+                    lst.append(i)
+    episodes_of: Dict[int, List[Tuple[int, int]]] = {}
+    for t, lst in acc_ops.items():
+        eps = []
+        first = last = lst[0]
+        for i in lst[1:]:
+            if i <= last + W_AFF and step_of[i] == step_of[last]:
+                last = i
+            else:
+                eps.append((first, last))
+                first = last = i
+        eps.append((first, last))
+        episodes_of[t] = eps
+    delta = [0] * (N + 1)
+    for t, eps in episodes_of.items():
+        a = alignup(tensors[t].size)
+        for (f, l) in eps:
+            delta[f] += a
+            delta[l + 1] -= a
+    wmax = live = 0
+    for i in range(N):
+        live += delta[i]
+        wmax = max(wmax, live)
+    ring_min = 2 * wmax
+    if ring_min > budget:
+        raise PlanError("budget smaller than the ring minimum")
+    pin_cap = budget - ring_min
+    # 5: pins
+    pinned_off: Dict[int, int] = {}
+    used = 0
+    if bits & BIT_A:
+        cands = [t for t in range(T) if score[t] > 0 and not zc[t]]
+        import functools
+
+        def cmp(a, b):
+            lhs, rhs = score[a] * tensors[b].size, score[b] * tensors[a].size
+            if lhs != rhs:
+                return -1 if lhs > rhs else 1
+            return -1 if a < b else (1 if a > b else 0)
+
+        for t in sorted(cands, key=functools.cmp_to_key(cmp)):
+            a = alignup(tensors[t].size)
+            if used + a <= pin_cap:
+                pinned_off[t] = used
+                used += a
+    ring_base, ring_size = used, budget - used
+    pins = sorted(pinned_off.items())
+    # 6: schedule
+    cmds: List[Cmd] = []
+    totals = [[0, 0, 0, 0] for _ in steps]
+    ep_index = {t: 0 for t in episodes_of}
+    open_stay: Dict[int, int] = {}            # ring tensor -> arena offset of its current stay
+    pin_loaded = set()
+    written_ever = set()
+    last_wb_op: Dict[int, int] = {}
+    fifo: List[Tuple[int, int, int]] = []     # (start, end, last-use op) of ring stays, oldest first
+    head = 0
+    run_wait = -1
+    ending: Dict[int, List[int]] = {}         # op -> ring tensors whose stay ends there
+    dirty_now = set()
+    ep_list = []
+
+    def emit(kind, t, arena_off, wait, first, release):
+        c = Cmd(len(cmds), kind, t, tensors[t].size, tensors[t].pool_off, arena_off, wait, first, release)
+        cmds.append(c)
+        tot = totals[step_of[first]]
+        tot[3] += 1
+        if kind == CMD_H2D:
+            tot[0] += c.nbytes
+        elif kind == CMD_D2H:
+            tot[1] += c.nbytes
+
+    for i, op in enumerate(ops):
+        for (t, mode, touched) in op.acc:
+            if zc[t]:
+                totals[op.step][2] += touched
+                continue
+            mutable = tensors[t].flags == F_MUTABLE
+            fresh_write = mutable and mode == MODE_W and t not in written_ever
+            if t in pinned_off:
+                if t not in pin_loaded:
+                    pin_loaded.add(t)
+                    emit(CMD_ALLOC if fresh_write else CMD_H2D, t, pinned_off[t], -1, i, N - 1)
+            elif t not in open_stay:
+                f, l = episodes_of[t][ep_index[t]]
+                assert f == i
+                a = alignup(tensors[t].size)
+                if a > ring_size:
+                    raise PlanError("tensor larger than the ring")
+                evicted = -1
+                if head + a > ring_size:                       # tail does not fit: skip it, wrap
+                    while fifo and fifo[0][0] >= head:
+                        evicted = max(evicted, fifo.pop(0)[2])
+                    head = 0
+                while fifo and fifo[0][0] < head + a and fifo[0][1] > head:
+                    evicted = max(evicted, fifo.pop(0)[2])
+                run_wait = max(run_wait, evicted, last_wb_op.get(t, -1))
+                if run_wait >= i:
+                    raise PlanError("ring too small: a stay would wait on its own op")
+                fifo.append((head, head + a, l))
+                open_stay[t] = ring_base + head
+                emit(CMD_ALLOC if fresh_write else CMD_H2D, t, ring_base + head, run_wait, i, l)
+                ending.setdefault(l, []).append(t)
+                ep_list.append((t, f, l))
+                head += a
+            if mode & MODE_W:
+                written_ever.add(t)
+                if t not in pinned_off:
+                    dirty_now.add(t)
+        for t in ending.pop(i, []):                            # stays that end at this op
+            off = open_stay.pop(t)
+            if t in dirty_now:
+                dirty_now.discard(t)
+                emit(CMD_D2H, t, off, i, i, i)
+                last_wb_op[t] = i
+            ep_index[t] += 1
+    return Plan(cls, crit, score, zc, pins, ring_base, ring_size, cmds, [tuple(x) for x in totals], ep_list)

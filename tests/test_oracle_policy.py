@@ -1,0 +1,237 @@
+"""Pins for the oracle trace and policy: hand-computed toy rooflines and op counts, an independent
+validator (with mutation tests proving it rejects broken plans), closed forms and a brute-force
+search over pin sets."""
+import itertools
+import os
+import struct
+from dataclasses import dataclass, replace
+
+import pytest
+
+import seeded_inputs as si
+from oracle import policy, trace, validate
+from conftest import MACHINE
+
+M = policy.Machine(**MACHINE)
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def test_toy_rooflines_from_fixture():
+    toy = policy.Machine(1000, 100, 10, 10)
+    names = {"LINK": policy.CLS_LINK, "HBM": policy.CLS_HBM, "COMPUTE": policy.CLS_COMPUTE}
+    n = 0
+    for line in open(os.path.join(GOLD, "toy_roofline.txt")):
+        line = line.split("#")[0].split()
+        if len(line) == 4:
+            f, h, g, want = int(line[0]), int(line[1]), int(line[2]), names[line[3]]
+            assert policy.classify(f, h, g, toy) == want, line
+            n += 1
+    assert n >= 8
+    assert policy.classify(20000, 300, 100, toy, bit_p=False) == policy.CLS_LINK      # selectivity off
+
+
+def test_gemm_ridge_on_the_measured_machine():
+    """A weight block streamed over the link is LINK-bound iff M < P/Bl (about 24.5k tokens here)."""
+    K = n = 8192
+    def cls(m):
+        return policy.classify(2 * m * K * n, 2 * m * K + 2 * K * n + 4 * m * n, 2 * K * n, M)
+    ridge = M.peak_flops // M.h2d_Bps
+    assert 24000 < ridge < 25000
+    assert cls(1) == policy.CLS_LINK and cls(16384) == policy.CLS_LINK
+    assert cls(ridge) == policy.CLS_LINK and cls(ridge + 1) == policy.CLS_COMPUTE and cls(32768) == policy.CLS_COMPUTE
+
+
+def test_trace_counts_by_hand_config_1():
+    lay = si.build_layout(si.CONFIGS[1])
+    ops, steps = trace.run_trace(lay)
+    assert len(steps) == 17 and steps[0][0] == trace.STEP_PREFILL and steps[1][0] == trace.STEP_DECODE
+    pre = ops[steps[0][1]: steps[0][1] + steps[0][2]]
+    dec = ops[steps[1][1]: steps[1][1] + steps[1][2]]
+    # embed gather, prefill: 32 tokens x 256 x (2 read + 4 written)
+    assert (pre[0].kind, pre[0].flops, pre[0].hbm, pre[0].acc[0][2]) == (trace.OP_EMBED, 0, 32 * 256 * 6, 32 * 256 * 2)
+    # decode wq block: M=1, K=256, n=256
+    g = [o for o in dec if o.kind == trace.OP_GEMM][0]
+    assert (g.flops, g.hbm, g.acc[0][2]) == (131072, 512 + 131072 + 1024, 131072)
+    # prefill attention: 4*B*Hq*Dh * S(S+1)/2 = 1024 * 528
+    a = [o for o in pre if o.kind == trace.OP_ATTN][0]
+    assert a.flops == 540672 and a.hbm == 4 * 32 * 4 * 64 + 4 * 1 * 4 * 32 * 64
+    assert [x[2] for x in a.acc] == [8192, 8192, 8192, 8192]          # 2 full K tiles then 2 full V tiles
+    # first decode step: position 32 opens tile 2 with one token; attention reads 3 K tiles then 3 V tiles
+    r = [o for o in dec if o.kind == trace.OP_ROPE_KV][0]
+    assert [(x[1], x[2]) for x in r.acc] == [(trace.MODE_W, 512), (trace.MODE_W, 512)]
+    a = [o for o in dec if o.kind == trace.OP_ATTN][0]
+    assert a.flops == 4 * 4 * 64 * 33 and [x[2] for x in a.acc] == [8192, 8192, 512] * 2
+    # ops per decode step: embed + L*(norm, q,k,v, rope, attn, o, norm, 4 gate, 4 up, swiglu, 4 down) + norm + 16 lm + argmax
+    assert len(dec) == 1 + 4 * (1 + 3 + 1 + 1 + 1 + 1 + 4 + 4 + 1 + 4) + 1 + 16 + 1
+    # down-projection block carries the residual read: K=1024, n=64
+    d = [o for o in dec if o.kind == trace.OP_GEMM and o.site == trace.site_of(trace.OP_GEMM, trace.K_WD)][0]
+    assert d.hbm == 2 * 1024 + 2 * 1024 * 64 + 4 * 64 + 4 * 64
+    # total flops of a decode step ~ 2 * (params without embed) + attention
+    params = (lay.weight_bytes // 2) - 4096 * 256 - 9 * 256
+    total = sum(o.flops for o in dec if o.kind == trace.OP_GEMM)
+    assert total == 2 * params
+
+
+def test_moe_trace_lists_only_routed_experts():
+    cfg = replace(si.CONFIGS[5], L=2, B=2, S=4, T=1, TK=4)
+    lay = si.build_layout(cfg, budget=8 << 30)
+    counts = [[[8, 0, 0, 8, 0, 0, 0, 0], [0, 16, 0, 0, 0, 0, 0, 0]], [[2, 2, 0, 0, 0, 0, 0, 0], [0, 0, 0, 0, 0, 0, 1, 3]]]
+    ops, steps = trace.run_trace(lay, expert_counts=counts)
+    experts = lambda k, l: sorted({o.expert for o in ops[steps[k][1]: steps[k][1] + steps[k][2]] if o.layer == l and o.expert >= 0})
+    assert experts(0, 0) == [0, 3] and experts(0, 1) == [1] and experts(1, 1) == [6, 7]
+    g = [o for o in ops if o.expert == 7 and o.kind == trace.OP_GEMM][0]
+    assert g.m == 3 and g.flops == 2 * 3 * g.acc[0][2] // 2
+
+
+@pytest.mark.parametrize("c", [1, 2, 3])
+def test_plan_invariants(c):
+    lay = si.build_layout(si.CONFIGS[c])
+    ops, steps = trace.run_trace(lay)
+    pl = policy.plan(lay.tensors, ops, steps, M, lay.budget)
+    r = validate.check(lay.tensors, ops, steps, lay.budget, pl.blobs())
+    assert r["n_cmds"] == len(pl.cmds) and r["n_pins"] == len(pl.pins)
+    # every decode op is link-bound or has no pool traffic; the embedding table is read in place
+    assert pl.zc[lay.blocks(si.K_EMBED)[0].tid] == 1
+    # steady decode step: bytes over the link = accessed non-ZC bytes - pinned accessed bytes
+    pinned = {t for t, _ in pl.pins}
+    k = len(steps) - 1
+    acc = {}
+    for o in ops[steps[k][1]: steps[k][1] + steps[k][2]]:
+        for (t, mode, touched) in o.acc:
+            acc[t] = 1
+    want = sum(lay.tensors[t].size for t in acc if t not in pinned and not pl.zc[t])
+    assert pl.totals[k][0] == want
+    # the policy's own lower bound: a step cannot move less than accessed - budget
+    assert pl.totals[k][0] >= sum(lay.tensors[t].size for t in acc if not pl.zc[t]) - lay.budget
+
+
+def _tamper(blobs, fn):
+    rec = struct.Struct("<IBIQQQiii")
+    cmds = [list(rec.unpack_from(blobs["commands"], k)) for k in range(0, len(blobs["commands"]), rec.size)]
+    fn(cmds)
+    out = dict(blobs)
+    out["commands"] = b"".join(rec.pack(*c) for c in cmds)
+    return out
+
+
+def test_validator_rejects_broken_plans():
+    lay = si.build_layout(si.CONFIGS[1])
+    ops, steps = trace.run_trace(lay)
+    pl = policy.plan(lay.tensors, ops, steps, M, lay.budget)
+    good = pl.blobs()
+    validate.check(lay.tensors, ops, steps, lay.budget, good)
+    ring = [k for k, c in enumerate(pl.cmds) if c.kind == policy.CMD_H2D and c.arena_off >= pl.ring_base]
+    late = ring[len(ring) // 2]
+
+    def drop(cmds):                      # a tensor never staged
+        del cmds[late]
+        for k, c in enumerate(cmds):
+            c[0] = k
+    def early(cmds):                     # reuse of ring space before its previous user is done
+        for k in ring[20:]:
+            cmds[k][6] = -1
+    def collide(cmds):                   # two live stays on the same bytes
+        cmds[late][5] = cmds[late - 1][5]
+    def swap(cmds):                      # order differs from first use
+        cmds[late], cmds[late + 8] = cmds[late + 8], cmds[late]
+        for k, c in enumerate(cmds):
+            c[0] = k
+    def outside(cmds):
+        cmds[late][5] = lay.budget
+    def no_writeback(cmds):
+        k = next(k for k, c in enumerate(cmds) if c[1] == policy.CMD_D2H)
+        del cmds[k]
+        for j, c in enumerate(cmds):
+            c[0] = j
+    for fn in (drop, early, collide, swap, outside):
+        with pytest.raises(validate.PlanInvalid):
+            validate.check(lay.tensors, ops, steps, lay.budget, _tamper(good, fn))
+    lay2 = si.build_layout(si.CONFIGS[2])
+    ops2, steps2 = trace.run_trace(lay2, n_decode=4)
+    pl2 = policy.plan(lay2.tensors, ops2, steps2, M, lay2.budget)
+    assert any(c.kind == policy.CMD_D2H for c in pl2.cmds)
+    validate.check(lay2.tensors, ops2, steps2, lay2.budget, pl2.blobs())
+    with pytest.raises(validate.PlanInvalid):
+        validate.check(lay2.tensors, ops2, steps2, lay2.budget, _tamper(pl2.blobs(), no_writeback))
+
+
+def test_closed_forms_large_and_minimal_budget():
+    lay = si.build_layout(si.CONFIGS[1])
+    ops, steps = trace.run_trace(lay)
+    accessed = {}
+    for o in ops:
+        for (t, _, _) in o.acc:
+            accessed[t] = lay.tensors[t]
+    # (a) budget >= footprint + ring minimum: everything that is read gets exactly one H2D, ever
+    big = policy.plan(lay.tensors, ops, steps, M, 4 * lay.pool_bytes)
+    h2d = [c for c in big.cmds if c.kind == policy.CMD_H2D]
+    assert len({c.tensor for c in h2d}) == len(h2d)
+    ro = [t for t in accessed.values() if t.flags == si.F_READONLY and not big.zc[t.tid]]
+    assert sum(c.nbytes for c in h2d) == sum(t.size for t in ro)        # KV tiles are born on the device (ALLOC)
+    assert not any(c.kind == policy.CMD_D2H for c in big.cmds)
+    # (b) no affinity bit: no pins, each step moves every accessed non-ZC byte
+    t_only = policy.plan(lay.tensors, ops, steps, M, lay.budget, bits=policy.BIT_P | policy.BIT_ZC)
+    assert t_only.pins == [] and t_only.ring_base == 0
+    validate.check(lay.tensors, ops, steps, lay.budget, t_only.blobs())
+    k = len(steps) - 1
+    step_acc = {t for o in ops[steps[k][1]: steps[k][1] + steps[k][2]] for (t, _, _) in o.acc}
+    assert t_only.totals[k][0] == sum(lay.tensors[t].size for t in step_acc if not t_only.zc[t])
+    # (c) budget below the ring minimum is an error, not a bad plan
+    with pytest.raises(policy.PlanError):
+        policy.plan(lay.tensors, ops, steps, M, 128 << 10)
+    # (d) without zero-copy the embedding table is staged like any tensor
+    nozc = policy.plan(lay.tensors, ops, steps, M, lay.budget, bits=policy.BIT_A | policy.BIT_P)
+    assert sum(nozc.zc) == 0
+    validate.check(lay.tensors, ops, steps, lay.budget, nozc.blobs())
+
+
+@dataclass
+class _T:
+    size: int
+    pool_off: int
+    flags: int = 1
+
+
+@dataclass
+class _O:
+    step: int
+    flops: int
+    hbm: int
+    acc: list
+
+
+def test_greedy_pins_match_brute_force_on_equal_sizes():
+    """<= 10 equal-size read-only tensors with different reuse counts: greedy-by-density is optimal."""
+    size = 4096
+    reuse = [5, 1, 3, 7, 2, 2, 6, 1, 4, 3]
+    tensors = [_T(size, k * size) for k in range(len(reuse))]
+    ops = []
+    for rnd in range(max(reuse)):
+        for t, r in enumerate(reuse):
+            if rnd < r:
+                ops.append(_O(0, 10, 10, [(t, 1, size)]))
+                ops += [_O(0, 10, 10, []) for _ in range(policy.W_AFF + 1)]     # gaps: no hold across uses
+    steps = [(0, 0, len(ops))]
+    for n_pin in (0, 3, 6):
+        budget = 2 * size + n_pin * size
+        pl = policy.plan(tensors, ops, steps, M, budget)
+        validate.check(tensors, ops, steps, budget, pl.blobs())
+        got = pl.totals[0][0]
+        best = min(sum(size * (1 if t in sub else reuse[t]) for t in range(len(reuse)))
+                   for sub in map(set, itertools.combinations(range(len(reuse)), n_pin)))
+        assert len(pl.pins) == n_pin and got == best
+
+
+def test_hold_window_keeps_short_reuse_in_place():
+    size = 8192
+    tensors = [_T(size, 0), _T(size, size), _T(size, 2 * size, flags=2)]
+    acc = lambda t, m=1: [(t, m, size)]
+    ops = [_O(0, 1, 1, acc(0)), _O(0, 1, 1, acc(1)), _O(0, 1, 1, acc(0)),          # reuse within the window
+           _O(0, 1, 1, []), _O(0, 1, 1, []), _O(0, 1, 1, []), _O(0, 1, 1, []), _O(0, 1, 1, []),
+           _O(0, 1, 1, acc(0)),                                                   # beyond the window: new stay
+           _O(0, 1, 1, acc(2, 2)), _O(0, 1, 1, acc(2, 1))]                        # written then read: one stay, one D2H
+    pl = policy.plan(tensors, ops, [(0, 0, len(ops))], M, 6 * size, bits=policy.BIT_P)
+    kinds = [(c.kind, c.tensor, c.first_use, c.release_after) for c in pl.cmds]
+    assert kinds == [(policy.CMD_H2D, 0, 0, 2), (policy.CMD_H2D, 1, 1, 1), (policy.CMD_H2D, 0, 8, 8),
+                     (policy.CMD_ALLOC, 2, 9, 10), (policy.CMD_D2H, 2, 10, 10)]
+    validate.check(tensors, ops, [(0, 0, len(ops))], 6 * size, pl.blobs())
