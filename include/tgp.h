@@ -1,0 +1,221 @@
+/*
+ * tgp - tensor-granular prefetch for oversubscribed transformer inference (sm_100a).
+ *
+ * C ABI of the library.  The calls follow the paper's statement of the problem:
+ * a framework allocator carves one big pool into tensors that are invisible below it
+ * (Section II-B), so the caller REGISTERS the pool and its sub-ranges (Section IV-B,
+ * stable two-level tensor identity); one pass RECORDS which tensors each op touches
+ * (Section IV-C, kernel-tensor access tracing); device capacity is CONSTRAINED to a
+ * budget (Section V-A); a roofline policy picks the transfers that matter (Section III-C,
+ * IV-C "UVM Analyzer") and an engine stages exactly those tensors ahead of use
+ * (Section IV-D "Prefetch Engine") while the model step RUNS.
+ *
+ * Conventions
+ *  - Every function returns TGP_OK (0) or a negative TGP_E_* code; nothing throws, aborts
+ *    or prints across this boundary.  tgp_strerror() names a code; tgp_last_error() adds
+ *    the detail of the last failure on that context.
+ *  - "host" pointers are CPU addresses, "dev" pointers are addresses valid on the current
+ *    CUDA device.  Streams are cudaStream_t passed as void*.
+ *  - Ownership: the caller owns the host pool, the device arena, the workspace, the logits
+ *    and token buffers and the streams, and keeps them alive while the context uses them.
+ *    The library owns the context, the plan and its CUDA events.  It allocates no device
+ *    memory except a few bytes of bookkeeping at tgp_model_bind().
+ *  - A context is used by one thread at a time.
+ *  - Export calls use the two-call form: pass buf == NULL to get the size in *bytes.
+ *  - All multi-byte fields of exported blobs are little-endian and packed.
+ */
+#ifndef TGP_H
+#define TGP_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define TGP_OK                  0
+#define TGP_E_INVAL            -1   /* bad argument or call order                                  */
+#define TGP_E_OVERLAP          -2   /* sub-range overlaps a registered one                         */
+#define TGP_E_RANGE            -3   /* sub-range or address outside its pool                       */
+#define TGP_E_UNKNOWN_TENSOR   -4   /* trace names a tensor id that was never registered           */
+#define TGP_E_BUDGET_TOO_SMALL -5   /* budget below the ring minimum, or a stay would wait on itself */
+#define TGP_E_NO_PLAN          -6   /* tgp_plan() has not succeeded yet                            */
+#define TGP_E_CUDA             -7   /* a CUDA call failed; tgp_last_error() has its text           */
+#define TGP_E_MISMATCH         -8   /* run-time access differs from the recorded trace             */
+#define TGP_E_STATE            -9   /* object not in the state this call needs                     */
+#define TGP_E_TOO_LARGE       -10   /* size beyond a documented fixed maximum                      */
+
+/* pool flags */
+#define TGP_POOL_PINNED   1u   /* page-locked host memory (cudaHostAlloc / cudaHostRegister'ed by the caller) */
+#define TGP_POOL_MANAGED  2u   /* cudaMallocManaged memory                                                    */
+#define TGP_POOL_PLAIN    4u   /* ordinary host memory: enough for planning; tgp_model_bind() page-locks it   */
+/* tensor flags */
+#define TGP_T_READONLY 1u
+#define TGP_T_MUTABLE  2u
+/* access modes */
+#define TGP_R 1u
+#define TGP_W 2u
+/* step kinds */
+#define TGP_PREFILL 0u
+#define TGP_DECODE  1u
+/* op kinds of the trace */
+#define TGP_OP_EMBED 0u
+#define TGP_OP_RMSNORM 1u
+#define TGP_OP_GEMM 2u
+#define TGP_OP_ROPE_KV 3u
+#define TGP_OP_ATTN 4u
+#define TGP_OP_SWIGLU 5u
+#define TGP_OP_ROUTER 6u
+#define TGP_OP_ARGMAX 7u
+/* tensor kinds (role of a sub-range in the model) */
+#define TGP_K_EMBED 0u
+#define TGP_K_G1 1u
+#define TGP_K_WQ 2u
+#define TGP_K_WK 3u
+#define TGP_K_WV 4u
+#define TGP_K_WO 5u
+#define TGP_K_G2 6u
+#define TGP_K_WG 7u
+#define TGP_K_WU 8u
+#define TGP_K_WD 9u
+#define TGP_K_GF 10u
+#define TGP_K_LM 11u
+#define TGP_K_ROUTER 12u
+#define TGP_K_KTILE 13u
+#define TGP_K_VTILE 14u
+/* execution variants */
+#define TGP_VAR_EXPLICIT_RING   0u  /* staged copies into the arena on a copy stream, events, no demand faults */
+#define TGP_VAR_MANAGED_HINTS   1u  /* managed pool + cudaMemPrefetchAsync on critical tensors + cudaMemAdvise on pins */
+#define TGP_VAR_MANAGED_DEMAND  2u  /* managed pool, no hints: the demand-paged baseline                        */
+/* policy bits (ablation switches of the paper's Section V-E: T is always on) */
+#define TGP_BIT_A  1u   /* look-ahead affinity: residency (pin) set              */
+#define TGP_BIT_P  2u   /* roofline selectivity; off = every op with pool traffic is link-bound */
+#define TGP_BIT_ZC 4u   /* sparse read-only accesses are served in place over the link          */
+/* plan export selectors */
+#define TGP_X_CLASSES  0u   /* u8 per op: 0 LINK, 1 HBM, 2 COMPUTE                                   */
+#define TGP_X_TENSORS  1u   /* per tensor: u8 critical, u8 zero-copy, u64 score                      */
+#define TGP_X_PINS     2u   /* (u32 tensor, u64 arena offset) ascending tensor id, then u64 ring base, u64 ring size */
+#define TGP_X_COMMANDS 3u   /* per command: u32 seq, u8 kind(0 H2D,1 ALLOC,2 D2H), u32 tensor, u64 bytes, u64 pool offset,
+                               u64 arena offset, i32 wait_op, i32 first_use, i32 release_after      */
+#define TGP_X_TOTALS   4u   /* per step: u64 h2d bytes, u64 d2h bytes, u64 zero-copy bytes, u64 commands */
+
+typedef struct tgp_ctx tgp_ctx;
+
+/* Roofline constants, integers per second: bf16 tensor peak, HBM bandwidth, host->device and
+ * device->host link bandwidth (Section III-C: compute roof, memory roof, interconnect roof). */
+typedef struct { uint64_t peak_flops, hbm_Bps, h2d_Bps, d2h_Bps; } tgp_machine;
+
+typedef struct { uint32_t tensor; uint32_t mode; uint64_t touched_bytes; } tgp_access;
+
+/* Decoder shape.  E == 0: dense SwiGLU FFN.  max_len = prompt + decode tokens; TK = tokens per KV tile. */
+typedef struct {
+    uint32_t L, d, Hq, Hkv, Dh, F, V, E, topk, B, max_len, TK;
+    float rope_base, eps;
+} tgp_model_cfg;
+
+/* One registered sub-range in its model role: rows [row0, row0+rows) of the [out, in] matrix
+ * `kind` of `layer` (expert -1 unless an expert weight); for KV tiles `block` is the tile index. */
+typedef struct { uint32_t kind; int32_t layer; int32_t expert; uint32_t block, row0, rows, tensor; } tgp_role_entry;
+
+typedef struct {
+    uint64_t h2d_bytes, d2h_bytes, zc_bytes;   /* bytes this step moved (plan figures for this step)   */
+    uint32_t n_cmds, n_launches, n_mismatch;   /* copy commands issued, kernels launched, fallbacks    */
+    float    step_ms;                          /* device time of the step, CUDA events on the compute stream */
+} tgp_step_stats;
+
+/* ---- context ------------------------------------------------------------------------------- */
+int  tgp_create(tgp_ctx **out, const tgp_machine *m);
+void tgp_destroy(tgp_ctx *ctx);
+const char *tgp_strerror(int code);
+const char *tgp_last_error(const tgp_ctx *ctx);
+
+/* ---- registry (Section II-B, IV-B): what the allocator hides -------------------------------- */
+/* Registers one pool [host_base, host_base+bytes).  host_base must be 512-byte aligned. */
+int  tgp_pool_register(tgp_ctx *ctx, void *host_base, uint64_t bytes, uint32_t flags, uint32_t *pool_id);
+/* Registers sub-range [offset, offset+bytes) of a pool.  offset must be 512-byte aligned.  site_hash stands
+ * for the creation-site call-stack hash; the library appends its own per-site allocation counter, so
+ * (site_hash, counter) is the stable identity that survives a move of the pool (Section IV-B). */
+int  tgp_tensor_register(tgp_ctx *ctx, uint32_t pool, uint64_t offset, uint64_t bytes, uint64_t site_hash,
+                         int32_t layer, uint32_t kind, uint32_t flags, uint32_t *tensor_id);
+/* Address -> (tensor, offset inside it); TGP_E_RANGE if no registered sub-range holds host_addr. */
+int  tgp_tensor_lookup(const tgp_ctx *ctx, const void *host_addr, uint32_t *tensor_id, uint64_t *inner_offset);
+/* Stable identity of a tensor: its site hash and per-site counter. */
+int  tgp_tensor_identity(const tgp_ctx *ctx, uint32_t tensor_id, uint64_t *site_hash, uint64_t *counter);
+
+/* ---- trace (Section IV-C): ordered ops, each with the tensors it touches --------------------- */
+int  tgp_trace_begin(tgp_ctx *ctx);                         /* discards any earlier trace and plan        */
+int  tgp_trace_step(tgp_ctx *ctx, uint32_t step_kind);      /* opens the next step                        */
+int  tgp_trace_op(tgp_ctx *ctx, uint64_t op_site, int32_t layer, uint32_t op_kind, uint64_t flops,
+                  uint64_t hbm_bytes, uint32_t n_acc, const tgp_access *acc);
+int  tgp_trace_end(tgp_ctx *ctx);
+/* Records the analytic trace of the bound model itself: prefill of S tokens then T decode steps.
+ * expert_counts (MoE only, else NULL): [(1+T) * L * E] tokens routed to each expert per step. */
+int  tgp_model_trace(tgp_ctx *ctx, uint32_t S, uint32_t T, const uint32_t *expert_counts);
+/* Canonical blob of the trace: per op u32 step, u64 site, i32 layer, u32 kind, u64 flops, u64 hbm bytes,
+ * u32 n_acc, then n_acc x (u32 tensor, u32 mode, u64 touched). */
+int  tgp_trace_export(const tgp_ctx *ctx, void *buf, uint64_t *bytes);
+
+/* ---- policy (Section III-C, IV-C, IV-D) ------------------------------------------------------ */
+int  tgp_set_budget(tgp_ctx *ctx, uint64_t bytes);          /* device bytes for resident pool tensors     */
+int  tgp_set_variant(tgp_ctx *ctx, uint32_t variant, uint32_t policy_bits);
+/* Classifies ops, selects critical / zero-copy / pinned tensors, sizes the ring and builds the ordered
+ * command list.  Host only; no CUDA call. */
+int  tgp_plan(tgp_ctx *ctx);
+int  tgp_plan_export(const tgp_ctx *ctx, uint32_t what, void *buf, uint64_t *bytes);
+
+/* ---- execution ------------------------------------------------------------------------------- */
+/* Device arena of at least the budget, 512-byte aligned, caller-owned. */
+int  tgp_set_arena(tgp_ctx *ctx, void *arena_dev, uint64_t bytes);
+/* Activation workspace the model needs for steps of up to max_tokens tokens (B * q_len). */
+int  tgp_model_workspace_bytes(const tgp_model_cfg *cfg, uint32_t max_tokens, uint64_t *bytes);
+/* Binds the model shape, the role of every registered tensor and the workspace.  router_bias_host: fp32
+ * [L, E] (MoE) or NULL.  May be called before tracing (tgp_model_trace needs it) with workspace NULL and
+ * again later with the workspace; page-locks a TGP_POOL_PLAIN pool when a workspace is given. */
+int  tgp_model_bind(tgp_ctx *ctx, const tgp_model_cfg *cfg, const tgp_role_entry *roles, uint32_t n_roles,
+                    const float *router_bias_host, void *workspace_dev, uint64_t ws_bytes, uint32_t max_tokens);
+/* Rewinds execution to step 0 with a cold arena (waits for work in flight first). */
+int  tgp_run_reset(tgp_ctx *ctx);
+/* Runs the next step of the plan: enqueues its copies on copy_stream and its kernels on compute_stream and
+ * returns without waiting unless stats != NULL.  tokens_host [B, q_len] int32, or NULL in a decode step to
+ * feed the previous step's argmax, which stays on the device.  logits_dev [B, V] fp32 of the last position;
+ * argmax_dev [B] int32 or NULL. */
+int  tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_host, uint32_t B, uint32_t q_len,
+              float *logits_dev, int32_t *argmax_dev, void *compute_stream, void *copy_stream,
+              tgp_step_stats *stats);
+
+/* ---- single kernels (device pointers; used by the model step, exported for parity tests and timing) ---- */
+/* x[m, :] = fp32(table[tok[m], :]);  table bf16 [V, d] (device or mapped host), tok int32 [M]. */
+int  tgp_k_embed(const void *table, const int32_t *tok_dev, float *x_dev, uint32_t M, uint32_t d, void *stream);
+/* h = bf16(x * rsqrt(mean(x^2) + eps) * g);  x fp32 [M, d] with row stride ldx elements, g bf16 [d], h bf16 [M, d]. */
+int  tgp_k_rmsnorm(const float *x_dev, uint32_t ldx, const void *g_dev, void *h_dev, uint32_t M, uint32_t d,
+                   float eps, void *stream);
+/* C[m, col0 + j] (=|+=) sum_k A[m, k] * W[j, k]: A bf16 [M, K] row-major, W bf16 [n, K] row-major (one out-row
+ * block), C fp32 with row stride ldc.  accumulate != 0 adds to C (fused residual).  K % 8 == 0. */
+int  tgp_k_gemm(const void *A_dev, const void *W_dev, float *C_dev, uint32_t M, uint32_t n, uint32_t K,
+                uint32_t ldc, uint32_t col0, int accumulate, void *stream);
+/* Fills caller-owned device tables cos/sin fp32 [max_len, Dh/2]: angle = pos * base^(-2i/Dh), evaluated in
+ * double on the host.  Synchronous. */
+int  tgp_k_rope_tables(uint32_t Dh, uint32_t max_len, float base, float *cos_dev, float *sin_dev);
+/* Rotary embedding (rotate-half pairs (i, i+Dh/2)) on q and k, bf16 rounding, and append of k, v to the KV
+ * tiles.  q32/k32/v32 fp32 [B*q_len, H*Dh]; qb bf16 out; k_tiles/v_tiles: HOST arrays of n_tiles (<= 64)
+ * device pointers, tile layout [B, Hkv, TK, Dh] bf16; token (b, p) sits at position pos0 + p. */
+int  tgp_k_rope_kv(const float *q32, const float *k32, const float *v32, void *qb, void *const *k_tiles,
+                   void *const *v_tiles, uint32_t n_tiles, const float *cos_dev, const float *sin_dev,
+                   const tgp_model_cfg *cfg, uint32_t B, uint32_t q_len, uint32_t pos0, void *stream);
+/* Causal GQA attention of q_len new queries per sequence against the tiles (kvlen = pos0 + q_len valid
+ * tokens): o = softmax(q K^T / sqrt(Dh)) V, bf16 out [B*q_len, Hq*Dh].  k_tiles/v_tiles as above (host arrays
+ * of device pointers).  Dh must be 64 or 128.  scratch_dev: fp32 workspace of
+ * tgp_k_attn_scratch_bytes() used when q_len == 1 (split over KV tiles), else may be NULL. */
+int  tgp_k_attn(const void *qb, void *const *k_tiles, void *const *v_tiles, uint32_t n_tiles, void *ob,
+                const tgp_model_cfg *cfg, uint32_t B, uint32_t q_len, uint32_t pos0, float *scratch_dev,
+                void *stream);
+int  tgp_k_attn_scratch_bytes(const tgp_model_cfg *cfg, uint64_t *bytes);
+/* a = bf16(silu(g) * u), g/u fp32 [M, F]. */
+int  tgp_k_swiglu(const float *g32, const float *u32, void *ab, uint64_t n_elems, void *stream);
+/* out[b] = argmax_j logits[b, j], lowest index on ties. */
+int  tgp_k_argmax(const float *logits, int32_t *out, uint32_t B, uint32_t V, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TGP_H */

@@ -1,0 +1,299 @@
+"""ctypes binding of libtgp.so: the same names as include/tgp.h, argument marshalling only.
+
+Every step of the path runs inside the library.  If the library is missing this module raises:
+there is no Python or CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libtgp.so")
+
+OK, E_INVAL, E_OVERLAP, E_RANGE, E_UNKNOWN_TENSOR, E_BUDGET_TOO_SMALL, E_NO_PLAN, E_CUDA, E_MISMATCH, E_STATE, E_TOO_LARGE = \
+    0, -1, -2, -3, -4, -5, -6, -7, -8, -9, -10
+POOL_PINNED, POOL_MANAGED, POOL_PLAIN = 1, 2, 4
+T_READONLY, T_MUTABLE = 1, 2
+R, W = 1, 2
+PREFILL, DECODE = 0, 1
+VAR_EXPLICIT_RING, VAR_MANAGED_HINTS, VAR_MANAGED_DEMAND = 0, 1, 2
+BIT_A, BIT_P, BIT_ZC = 1, 2, 4
+X_CLASSES, X_TENSORS, X_PINS, X_COMMANDS, X_TOTALS = range(5)
+
+
+class Machine(C.Structure):
+    _fields_ = [("peak_flops", C.c_uint64), ("hbm_Bps", C.c_uint64), ("h2d_Bps", C.c_uint64), ("d2h_Bps", C.c_uint64)]
+
+
+class Access(C.Structure):
+    _fields_ = [("tensor", C.c_uint32), ("mode", C.c_uint32), ("touched_bytes", C.c_uint64)]
+
+
+class ModelCfg(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in ("L", "d", "Hq", "Hkv", "Dh", "F", "V", "E", "topk", "B", "max_len", "TK")] + \
+               [("rope_base", C.c_float), ("eps", C.c_float)]
+
+
+class RoleEntry(C.Structure):
+    _fields_ = [("kind", C.c_uint32), ("layer", C.c_int32), ("expert", C.c_int32), ("block", C.c_uint32),
+                ("row0", C.c_uint32), ("rows", C.c_uint32), ("tensor", C.c_uint32)]
+
+
+class StepStats(C.Structure):
+    _fields_ = [("h2d_bytes", C.c_uint64), ("d2h_bytes", C.c_uint64), ("zc_bytes", C.c_uint64),
+                ("n_cmds", C.c_uint32), ("n_launches", C.c_uint32), ("n_mismatch", C.c_uint32), ("step_ms", C.c_float)]
+
+
+class TgpError(RuntimeError):
+    def __init__(self, code, where, detail=""):
+        self.code = code
+        super().__init__(f"{where}: {lib().tgp_strerror(code).decode()} ({code}) {detail}")
+
+
+_lib = None
+_P, _U32, _U64, _I32 = C.c_void_p, C.c_uint32, C.c_uint64, C.c_int32
+_SIGS = {
+    "tgp_create": [C.POINTER(_P), C.POINTER(Machine)],
+    "tgp_destroy": [_P],
+    "tgp_pool_register": [_P, _P, _U64, _U32, C.POINTER(_U32)],
+    "tgp_tensor_register": [_P, _U32, _U64, _U64, _U64, _I32, _U32, _U32, C.POINTER(_U32)],
+    "tgp_tensor_lookup": [_P, _P, C.POINTER(_U32), C.POINTER(_U64)],
+    "tgp_tensor_identity": [_P, _U32, C.POINTER(_U64), C.POINTER(_U64)],
+    "tgp_trace_begin": [_P],
+    "tgp_trace_step": [_P, _U32],
+    "tgp_trace_op": [_P, _U64, _I32, _U32, _U64, _U64, _U32, C.POINTER(Access)],
+    "tgp_trace_end": [_P],
+    "tgp_model_trace": [_P, _U32, _U32, C.POINTER(_U32)],
+    "tgp_trace_export": [_P, _P, C.POINTER(_U64)],
+    "tgp_set_budget": [_P, _U64],
+    "tgp_set_variant": [_P, _U32, _U32],
+    "tgp_plan": [_P],
+    "tgp_plan_export": [_P, _U32, _P, C.POINTER(_U64)],
+    "tgp_set_arena": [_P, _P, _U64],
+    "tgp_model_workspace_bytes": [C.POINTER(ModelCfg), _U32, C.POINTER(_U64)],
+    "tgp_model_bind": [_P, C.POINTER(ModelCfg), C.POINTER(RoleEntry), _U32, _P, _P, _U64, _U32],
+    "tgp_run_reset": [_P],
+    "tgp_step": [_P, _U32, _P, _U32, _U32, _P, _P, _P, _P, C.POINTER(StepStats)],
+    "tgp_k_embed": [_P, _P, _P, _U32, _U32, _P],
+    "tgp_k_rmsnorm": [_P, _U32, _P, _P, _U32, _U32, C.c_float, _P],
+    "tgp_k_gemm": [_P, _P, _P, _U32, _U32, _U32, _U32, _U32, C.c_int, _P],
+    "tgp_k_rope_tables": [_U32, _U32, C.c_float, _P, _P],
+    "tgp_k_rope_kv": [_P, _P, _P, _P, C.POINTER(_P), C.POINTER(_P), _U32, _P, _P, C.POINTER(ModelCfg), _U32, _U32, _U32, _P],
+    "tgp_k_attn": [_P, C.POINTER(_P), C.POINTER(_P), _U32, _P, C.POINTER(ModelCfg), _U32, _U32, _U32, _P, _P],
+    "tgp_k_attn_scratch_bytes": [C.POINTER(ModelCfg), C.POINTER(_U64)],
+    "tgp_k_swiglu": [_P, _P, _P, _U64, _P],
+    "tgp_k_argmax": [_P, _P, _U32, _U32, _P],
+}
+
+
+def lib():
+    """The loaded library; raises if it has not been built (no fallback path exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_06172_b200.build` "
+                              "(the hot path has no Python or CPU fallback)")
+        l = C.CDLL(LIB_PATH)
+        for name, args in _SIGS.items():
+            f = getattr(l, name)
+            f.argtypes = args
+            f.restype = None if name == "tgp_destroy" else C.c_int
+        l.tgp_strerror.argtypes, l.tgp_strerror.restype = [C.c_int], C.c_char_p
+        l.tgp_last_error.argtypes, l.tgp_last_error.restype = [_P], C.c_char_p
+        _lib = l
+    return _lib
+
+
+def exported_symbols():
+    return sorted(list(_SIGS) + ["tgp_strerror", "tgp_last_error"])
+
+
+def _ptr(x):
+    """Address of a numpy array / torch tensor / int / None as a void pointer value."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if isinstance(x, np.ndarray):
+        return x.ctypes.data
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    if hasattr(x, "cuda_stream"):
+        return x.cuda_stream
+    raise TypeError(type(x))
+
+
+class Ctx:
+    """One tgp_ctx.  Methods carry the C names without the prefix; each raises TgpError on a negative code."""
+
+    def __init__(self, peak_flops, hbm_Bps, h2d_Bps, d2h_Bps):
+        self._h = _P()
+        m = Machine(peak_flops, hbm_Bps, h2d_Bps, d2h_Bps)
+        rc = lib().tgp_create(C.byref(self._h), C.byref(m))
+        if rc:
+            raise TgpError(rc, "tgp_create")
+        self._keep = []
+
+    def close(self):
+        if self._h:
+            lib().tgp_destroy(self._h)
+            self._h = _P()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _ck(self, rc, where):
+        if rc:
+            raise TgpError(rc, where, lib().tgp_last_error(self._h).decode())
+        return rc
+
+    def pool_register(self, host_base, nbytes, flags):
+        out = _U32()
+        self._ck(lib().tgp_pool_register(self._h, _ptr(host_base), nbytes, flags, C.byref(out)), "tgp_pool_register")
+        self._keep.append(host_base)
+        return out.value
+
+    def tensor_register(self, pool, offset, nbytes, site_hash, layer, kind, flags):
+        out = _U32()
+        self._ck(lib().tgp_tensor_register(self._h, pool, offset, nbytes, site_hash, layer, kind, flags, C.byref(out)), "tgp_tensor_register")
+        return out.value
+
+    def tensor_lookup(self, host_addr):
+        t, o = _U32(), _U64()
+        self._ck(lib().tgp_tensor_lookup(self._h, host_addr, C.byref(t), C.byref(o)), "tgp_tensor_lookup")
+        return t.value, o.value
+
+    def tensor_identity(self, tid):
+        s, c = _U64(), _U64()
+        self._ck(lib().tgp_tensor_identity(self._h, tid, C.byref(s), C.byref(c)), "tgp_tensor_identity")
+        return s.value, c.value
+
+    def trace_begin(self):
+        self._ck(lib().tgp_trace_begin(self._h), "tgp_trace_begin")
+
+    def trace_step(self, kind):
+        self._ck(lib().tgp_trace_step(self._h, kind), "tgp_trace_step")
+
+    def trace_op(self, site, layer, kind, flops, hbm, acc):
+        arr = (Access * max(1, len(acc)))(*[Access(t, m, b) for (t, m, b) in acc])
+        self._ck(lib().tgp_trace_op(self._h, site, layer, kind, flops, hbm, len(acc), arr), "tgp_trace_op")
+
+    def trace_end(self):
+        self._ck(lib().tgp_trace_end(self._h), "tgp_trace_end")
+
+    def model_trace(self, S, T, expert_counts=None):
+        p = None
+        if expert_counts is not None:
+            ec = np.ascontiguousarray(expert_counts, dtype=np.uint32)
+            p = ec.ctypes.data_as(C.POINTER(_U32))
+        self._ck(lib().tgp_model_trace(self._h, S, T, p), "tgp_model_trace")
+
+    def trace_export(self):
+        n = _U64()
+        self._ck(lib().tgp_trace_export(self._h, None, C.byref(n)), "tgp_trace_export")
+        buf = C.create_string_buffer(max(1, n.value))
+        self._ck(lib().tgp_trace_export(self._h, buf, C.byref(n)), "tgp_trace_export")
+        return buf.raw[:n.value]
+
+    def set_budget(self, nbytes):
+        self._ck(lib().tgp_set_budget(self._h, nbytes), "tgp_set_budget")
+
+    def set_variant(self, variant, bits):
+        self._ck(lib().tgp_set_variant(self._h, variant, bits), "tgp_set_variant")
+
+    def plan(self):
+        self._ck(lib().tgp_plan(self._h), "tgp_plan")
+
+    def plan_export(self, what):
+        n = _U64()
+        self._ck(lib().tgp_plan_export(self._h, what, None, C.byref(n)), "tgp_plan_export")
+        buf = C.create_string_buffer(max(1, n.value))
+        self._ck(lib().tgp_plan_export(self._h, what, buf, C.byref(n)), "tgp_plan_export")
+        return buf.raw[:n.value]
+
+    def plan_blobs(self):
+        return {k: self.plan_export(w) for k, w in (("classes", X_CLASSES), ("tensors", X_TENSORS), ("pins", X_PINS),
+                                                    ("commands", X_COMMANDS), ("totals", X_TOTALS))}
+
+    def set_arena(self, arena, nbytes):
+        self._ck(lib().tgp_set_arena(self._h, _ptr(arena), nbytes), "tgp_set_arena")
+        self._keep.append(arena)
+
+    def model_bind(self, cfg: ModelCfg, roles, router_bias=None, workspace=None, ws_bytes=0, max_tokens=0):
+        arr = (RoleEntry * len(roles))(*[RoleEntry(*r) for r in roles])
+        rb = None if router_bias is None else np.ascontiguousarray(router_bias, dtype=np.float32)
+        self._ck(lib().tgp_model_bind(self._h, C.byref(cfg), arr, len(roles), _ptr(rb), _ptr(workspace), ws_bytes, max_tokens), "tgp_model_bind")
+        self._keep.append(workspace)
+
+    def run_reset(self):
+        self._ck(lib().tgp_run_reset(self._h), "tgp_run_reset")
+
+    def step(self, kind, tokens_host, B, q_len, logits, argmax, compute_stream, copy_stream, want_stats=False):
+        st = StepStats() if want_stats else None
+        self._ck(lib().tgp_step(self._h, kind, _ptr(tokens_host), B, q_len, _ptr(logits), _ptr(argmax), _ptr(compute_stream),
+                                _ptr(copy_stream), C.byref(st) if st is not None else None), "tgp_step")
+        return st
+
+
+def model_workspace_bytes(cfg: ModelCfg, max_tokens: int) -> int:
+    n = _U64()
+    rc = lib().tgp_model_workspace_bytes(C.byref(cfg), max_tokens, C.byref(n))
+    if rc:
+        raise TgpError(rc, "tgp_model_workspace_bytes")
+    return n.value
+
+
+def _tile_arrays(k_tiles, v_tiles):
+    n = len(k_tiles)
+    return (_P * max(1, n))(*[_ptr(t) for t in k_tiles]), (_P * max(1, n))(*[_ptr(t) for t in v_tiles]), n
+
+
+def _k(rc, where):
+    if rc:
+        raise TgpError(rc, where)
+
+
+def k_embed(table, tok, x, M, d, stream=None):
+    _k(lib().tgp_k_embed(_ptr(table), _ptr(tok), _ptr(x), M, d, _ptr(stream)), "tgp_k_embed")
+
+
+def k_rmsnorm(x, ldx, g, h, M, d, eps, stream=None):
+    _k(lib().tgp_k_rmsnorm(_ptr(x), ldx, _ptr(g), _ptr(h), M, d, eps, _ptr(stream)), "tgp_k_rmsnorm")
+
+
+def k_gemm(A, W, Cout, M, n, K, ldc, col0, accumulate, stream=None):
+    _k(lib().tgp_k_gemm(_ptr(A), _ptr(W), _ptr(Cout), M, n, K, ldc, col0, int(accumulate), _ptr(stream)), "tgp_k_gemm")
+
+
+def k_rope_tables(Dh, max_len, base, cos, sin):
+    _k(lib().tgp_k_rope_tables(Dh, max_len, base, _ptr(cos), _ptr(sin)), "tgp_k_rope_tables")
+
+
+def k_rope_kv(q32, k32, v32, qb, k_tiles, v_tiles, cos, sin, cfg, B, q_len, pos0, stream=None):
+    ka, va, n = _tile_arrays(k_tiles, v_tiles)
+    _k(lib().tgp_k_rope_kv(_ptr(q32), _ptr(k32), _ptr(v32), _ptr(qb), ka, va, n, _ptr(cos), _ptr(sin), C.byref(cfg), B, q_len, pos0, _ptr(stream)), "tgp_k_rope_kv")
+
+
+def k_attn(qb, k_tiles, v_tiles, ob, cfg, B, q_len, pos0, scratch=None, stream=None):
+    ka, va, n = _tile_arrays(k_tiles, v_tiles)
+    _k(lib().tgp_k_attn(_ptr(qb), ka, va, n, _ptr(ob), C.byref(cfg), B, q_len, pos0, _ptr(scratch), _ptr(stream)), "tgp_k_attn")
+
+
+def k_attn_scratch_bytes(cfg):
+    n = _U64()
+    _k(lib().tgp_k_attn_scratch_bytes(C.byref(cfg), C.byref(n)), "tgp_k_attn_scratch_bytes")
+    return n.value
+
+
+def k_swiglu(g, u, ab, n, stream=None):
+    _k(lib().tgp_k_swiglu(_ptr(g), _ptr(u), _ptr(ab), n, _ptr(stream)), "tgp_k_swiglu")
+
+
+def k_argmax(logits, out, B, V, stream=None):
+    _k(lib().tgp_k_argmax(_ptr(logits), _ptr(out), B, V, _ptr(stream)), "tgp_k_argmax")

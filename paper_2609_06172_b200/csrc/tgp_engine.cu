@@ -1,0 +1,376 @@
+// Step engine: executes the plan.  Copies run on the caller's copy stream (host -> arena) and on a
+// library-owned write-back stream (arena -> host); kernels run on the caller's compute stream; CUDA
+// events order the two.  No kernel ever touches a non-resident byte, so there are no demand faults.
+//
+// Ordering rules (per command c of the plan, per op i of the trace):
+//   H2D/ALLOC c : copy stream waits done[c.wait_op] (the last op that used the bytes being overwritten)
+//                 and the newest write-back, copies, then records copied[c.first_use] if c is the last
+//                 placement of that op.
+//   op i        : compute stream waits copied[i] (if the op has placements), runs, records done[i]
+//                 if some command waits on i.
+//   D2H c       : write-back stream waits done[c.wait_op], copies the tensor back, records wb.
+// A command is enqueued as soon as the op it waits on has been enqueued, so the copy stream runs as far
+// ahead of compute as ring space allows, across step boundaries too.
+#include <cuda_runtime.h>
+#include <cmath>
+#include <cstring>
+#include <vector>
+#include "tgp_internal.h"
+#include "tgp_kernels.h"
+
+extern thread_local uint64_t tgpk_launches;
+
+#define CU(ctx, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return tgp_fail(ctx, TGP_E_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } while (0)
+
+struct TgpEngine {
+    // workspace carve-up
+    int32_t *tok = nullptr, *amax = nullptr;
+    float *x = nullptr, *q32 = nullptr, *k32 = nullptr, *v32 = nullptr, *g32 = nullptr, *u32 = nullptr, *cos_t = nullptr, *sin_t = nullptr, *scratch = nullptr;
+    char *h = nullptr, *qb = nullptr, *ob = nullptr, *ab = nullptr, *hf = nullptr;
+    uint32_t max_tokens = 0;
+    // run state
+    std::vector<cudaEvent_t> done_ev, copied_ev;         // per op, created on first use
+    cudaEvent_t wb_ev = nullptr, t0 = nullptr, t1 = nullptr;
+    cudaStream_t wb_stream = nullptr;
+    bool wb_pending = false;                             // a write-back was recorded since the copy stream last waited
+    int32_t copy_waited_op = -1;
+    size_t next_cmd = 0;
+    uint32_t next_step = 0, pos = 0;
+    const int32_t *tok_src = nullptr;
+    int device = -1;
+    // managed-hints variant
+    size_t hinted_upto = 0;
+    bool advised = false;
+};
+
+static inline uint64_t up256(uint64_t x) { return (x + 255) / 256 * 256; }
+
+struct WsLayout { uint64_t tok, amax, x, h, q32, k32, v32, qb, ob, g32, u32, ab, hf, cos_t, sin_t, scratch, total; };
+
+static WsLayout ws_layout(const tgp_model_cfg &c, uint64_t Mx) {
+    WsLayout w{};
+    uint64_t o = 0;
+    auto take = [&](uint64_t bytes) { uint64_t at = o; o = up256(o + bytes); return at; };
+    const uint64_t qd = (uint64_t)c.Hq * c.Dh, kd = (uint64_t)c.Hkv * c.Dh;
+    w.tok = take(Mx * 4); w.amax = take((uint64_t)c.B * 4);
+    w.x = take(Mx * c.d * 4); w.h = take(Mx * c.d * 2);
+    w.q32 = take(Mx * qd * 4); w.k32 = take(Mx * kd * 4); w.v32 = take(Mx * kd * 4);
+    w.qb = take(Mx * qd * 2); w.ob = take(Mx * qd * 2);
+    w.g32 = take(Mx * c.F * 4); w.u32 = take(Mx * c.F * 4); w.ab = take(Mx * c.F * 2);
+    w.hf = take((uint64_t)c.B * c.d * 2);
+    w.cos_t = take((uint64_t)c.max_len * (c.Dh / 2) * 4); w.sin_t = take((uint64_t)c.max_len * (c.Dh / 2) * 4);
+    uint64_t sb = 0; tgp_k_attn_scratch_bytes(&c, &sb);
+    w.scratch = take(sb);
+    w.total = o;
+    return w;
+}
+
+int tgp_rope_tables_upload(uint32_t Dh, uint32_t max_len, float base, float *cos_dev, float *sin_dev) {
+    const uint32_t half = Dh / 2;
+    std::vector<float> c((size_t)max_len * half), s((size_t)max_len * half);
+    for (uint32_t i = 0; i < half; ++i) {
+        const double inv = std::pow((double)base, -2.0 * (double)i / (double)Dh);
+        for (uint32_t p = 0; p < max_len; ++p) { const double a = (double)p * inv; c[(size_t)p * half + i] = (float)std::cos(a); s[(size_t)p * half + i] = (float)std::sin(a); }
+    }
+    if (cudaMemcpy(cos_dev, c.data(), c.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) return TGP_E_CUDA;
+    if (cudaMemcpy(sin_dev, s.data(), s.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) return TGP_E_CUDA;
+    return TGP_OK;
+}
+
+void tgp_engine_free(tgp_ctx *ctx) {
+    if (!ctx) return;
+    for (TgpPool &p : ctx->pools)
+        if (p.locked_by_us) { cudaHostUnregister(p.host_base); p.locked_by_us = false; }
+    TgpEngine *e = ctx->eng;
+    if (!e) return;
+    cudaDeviceSynchronize();
+    for (cudaEvent_t ev : e->done_ev) if (ev) cudaEventDestroy(ev);
+    for (cudaEvent_t ev : e->copied_ev) if (ev) cudaEventDestroy(ev);
+    if (e->wb_ev) cudaEventDestroy(e->wb_ev);
+    if (e->t0) cudaEventDestroy(e->t0);
+    if (e->t1) cudaEventDestroy(e->t1);
+    if (e->wb_stream) cudaStreamDestroy(e->wb_stream);
+    delete e;
+    ctx->eng = nullptr;
+}
+
+extern "C" {
+
+int tgp_k_rope_tables(uint32_t Dh, uint32_t max_len, float base, float *cos_dev, float *sin_dev) {
+    if (!cos_dev || !sin_dev || Dh % 2 || !max_len) return TGP_E_INVAL;
+    return tgp_rope_tables_upload(Dh, max_len, base, cos_dev, sin_dev);
+}
+
+int tgp_set_arena(tgp_ctx *ctx, void *arena_dev, uint64_t bytes) {
+    if (!ctx || !arena_dev || !bytes) return TGP_E_INVAL;
+    if ((uintptr_t)arena_dev % 512) return tgp_fail(ctx, TGP_E_INVAL, "arena not 512-byte aligned");
+    ctx->arena = arena_dev; ctx->arena_bytes = bytes;
+    return TGP_OK;
+}
+
+int tgp_model_workspace_bytes(const tgp_model_cfg *cfg, uint32_t max_tokens, uint64_t *bytes) {
+    if (!cfg || !bytes || !max_tokens || !cfg->TK || !cfg->Dh) return TGP_E_INVAL;
+    *bytes = ws_layout(*cfg, max_tokens).total;
+    return TGP_OK;
+}
+
+int tgp_model_bind(tgp_ctx *ctx, const tgp_model_cfg *cfg, const tgp_role_entry *roles, uint32_t n_roles,
+                   const float *router_bias_host, void *workspace_dev, uint64_t ws_bytes, uint32_t max_tokens) {
+    if (!ctx || !cfg || !roles || !n_roles) return TGP_E_INVAL;
+    const tgp_model_cfg &c = *cfg;
+    if (!c.L || !c.d || !c.Hq || !c.Hkv || c.Hq % c.Hkv || !c.Dh || c.Dh % 2 || !c.V || !c.B || !c.TK || !c.max_len || c.d % 8 || c.F % 8)
+        return tgp_fail(ctx, TGP_E_INVAL, "model shape");
+    if ((c.max_len + c.TK - 1) / c.TK > TGP_MAX_TILES) return tgp_fail(ctx, TGP_E_TOO_LARGE, "more KV tiles per layer than a kernel can address (64)");
+    if (c.E && !router_bias_host) return tgp_fail(ctx, TGP_E_INVAL, "MoE needs the router bias");
+    std::vector<TgpRole> rs(n_roles);
+    std::vector<int32_t> rot(ctx->tensors.size(), -1);
+    for (uint32_t i = 0; i < n_roles; ++i) {
+        const tgp_role_entry &r = roles[i];
+        if (r.tensor >= ctx->tensors.size()) return tgp_fail(ctx, TGP_E_UNKNOWN_TENSOR, "role names an unregistered tensor");
+        if (r.kind > TGP_K_VTILE || !r.rows) return tgp_fail(ctx, TGP_E_INVAL, "role entry");
+        if (rot[r.tensor] >= 0) return tgp_fail(ctx, TGP_E_INVAL, "tensor bound to two roles");
+        const TgpTensor &t = ctx->tensors[r.tensor];
+        if (t.size % (2ull * r.rows)) return tgp_fail(ctx, TGP_E_INVAL, "tensor size is not rows x cols bf16");
+        rs[i] = {r.kind, r.layer, r.expert, r.block, r.row0, r.rows, r.tensor};
+        rot[r.tensor] = (int32_t)i;
+    }
+    ctx->cfg = c; ctx->roles.swap(rs); ctx->role_of_tensor.swap(rot);
+    ctx->router_bias.assign(router_bias_host ? router_bias_host : nullptr, router_bias_host ? router_bias_host + (size_t)c.L * c.E : nullptr);
+    ctx->bound = true;
+    if (!workspace_dev) return TGP_OK;
+    if (!max_tokens) return TGP_E_INVAL;
+    const WsLayout w = ws_layout(c, max_tokens);
+    if (ws_bytes < w.total) return tgp_fail(ctx, TGP_E_INVAL, "workspace smaller than tgp_model_workspace_bytes()");
+    if ((uintptr_t)workspace_dev % 256) return tgp_fail(ctx, TGP_E_INVAL, "workspace not 256-byte aligned");
+    tgp_engine_free(ctx);
+    TgpEngine *e = new TgpEngine();
+    ctx->eng = e;
+    char *b = (char *)workspace_dev;
+    e->tok = (int32_t *)(b + w.tok); e->amax = (int32_t *)(b + w.amax);
+    e->x = (float *)(b + w.x); e->h = b + w.h; e->q32 = (float *)(b + w.q32); e->k32 = (float *)(b + w.k32); e->v32 = (float *)(b + w.v32);
+    e->qb = b + w.qb; e->ob = b + w.ob; e->g32 = (float *)(b + w.g32); e->u32 = (float *)(b + w.u32); e->ab = b + w.ab; e->hf = b + w.hf;
+    e->cos_t = (float *)(b + w.cos_t); e->sin_t = (float *)(b + w.sin_t); e->scratch = (float *)(b + w.scratch);
+    e->max_tokens = max_tokens;
+    CU(ctx, cudaGetDevice(&e->device));
+    for (TgpPool &p : ctx->pools) {
+        if (p.flags == TGP_POOL_PLAIN && !p.locked_by_us) {
+            CU(ctx, cudaHostRegister(p.host_base, p.bytes, cudaHostRegisterPortable | cudaHostRegisterMapped));
+            p.locked_by_us = true;
+        }
+        if (p.flags == TGP_POOL_MANAGED) p.dev_alias = p.host_base;
+        else { void *dp = nullptr; CU(ctx, cudaHostGetDevicePointer(&dp, p.host_base, 0)); p.dev_alias = (char *)dp; }
+    }
+    if (tgp_rope_tables_upload(c.Dh, c.max_len, c.rope_base, e->cos_t, e->sin_t)) return tgp_fail(ctx, TGP_E_CUDA, "rope table upload");
+    CU(ctx, cudaEventCreateWithFlags(&e->wb_ev, cudaEventDisableTiming));
+    CU(ctx, cudaEventCreate(&e->t0));
+    CU(ctx, cudaEventCreate(&e->t1));
+    CU(ctx, cudaStreamCreateWithFlags(&e->wb_stream, cudaStreamNonBlocking));
+    return TGP_OK;
+}
+
+int tgp_run_reset(tgp_ctx *ctx) {
+    if (!ctx || !ctx->eng) return TGP_E_STATE;
+    CU(ctx, cudaDeviceSynchronize());
+    TgpEngine *e = ctx->eng;
+    e->next_cmd = 0; e->next_step = 0; e->pos = 0; e->wb_pending = false; e->copy_waited_op = -1; e->tok_src = nullptr;
+    e->hinted_upto = 0;
+    return TGP_OK;
+}
+
+}  // extern "C"
+
+static int get_event(tgp_ctx *ctx, std::vector<cudaEvent_t> &v, size_t i, cudaEvent_t *out) {
+    if (v.size() < ctx->ops.size()) v.resize(ctx->ops.size(), nullptr);
+    if (!v[i]) CU(ctx, cudaEventCreateWithFlags(&v[i], cudaEventDisableTiming));
+    *out = v[i];
+    return TGP_OK;
+}
+
+// Enqueue, in plan order, every command whose wait_op has been enqueued (wait_op <= limit).
+static int pump(tgp_ctx *ctx, int32_t limit, cudaStream_t copy, uint32_t *n_cmds) {
+    TgpEngine *e = ctx->eng;
+    const TgpPlan &pl = ctx->plan;
+    while (e->next_cmd < pl.cmds.size() && pl.cmds[e->next_cmd].wait_op <= limit) {
+        const TgpCmd &c = pl.cmds[e->next_cmd];
+        const TgpPool &pool = ctx->pools[ctx->tensors[c.tensor].pool];
+        char *dev = (char *)ctx->arena + c.arena_off;
+        char *host = pool.host_base + c.pool_off;
+        cudaEvent_t ev;
+        if (c.kind == CMD_D2H) {
+            int rc = get_event(ctx, e->done_ev, (size_t)c.wait_op, &ev);
+            if (rc) return rc;
+            CU(ctx, cudaStreamWaitEvent(e->wb_stream, ev, 0));
+            CU(ctx, cudaMemcpyAsync(host, dev, c.bytes, cudaMemcpyDeviceToHost, e->wb_stream));
+            CU(ctx, cudaEventRecord(e->wb_ev, e->wb_stream));
+            e->wb_pending = true;
+        } else {
+            if (c.wait_op > e->copy_waited_op) {
+                int rc = get_event(ctx, e->done_ev, (size_t)c.wait_op, &ev);
+                if (rc) return rc;
+                CU(ctx, cudaStreamWaitEvent(copy, ev, 0));
+                e->copy_waited_op = c.wait_op;
+            }
+            if (e->wb_pending) { CU(ctx, cudaStreamWaitEvent(copy, e->wb_ev, 0)); e->wb_pending = false; }
+            if (c.kind == CMD_H2D) CU(ctx, cudaMemcpyAsync(dev, host, c.bytes, cudaMemcpyHostToDevice, copy));
+            if (pl.op_last_place[c.first_use] == (int32_t)e->next_cmd) {
+                int rc = get_event(ctx, e->copied_ev, (size_t)c.first_use, &ev);
+                if (rc) return rc;
+                CU(ctx, cudaEventRecord(ev, copy));
+            }
+        }
+        if (n_cmds) ++*n_cmds;
+        ++e->next_cmd;
+    }
+    return TGP_OK;
+}
+
+// address of access k of op o on the device
+static inline char *where(const tgp_ctx *ctx, const TgpOp &o, uint32_t k) {
+    const tgp_access &a = ctx->acc[o.acc0 + k];
+    const TgpTensor &t = ctx->tensors[a.tensor];
+    if (ctx->variant != TGP_VAR_EXPLICIT_RING) return ctx->pools[t.pool].dev_alias + t.off;
+    const uint64_t w = ctx->plan.acc_where[o.acc0 + k];
+    return w == UINT64_MAX ? ctx->pools[t.pool].dev_alias + t.off : (char *)ctx->arena + w;
+}
+
+// managed-hints variant: prefetch the tensors of upcoming link-bound ops, advise the pin set once
+static int hint_ahead(tgp_ctx *ctx, size_t op_now, size_t step_end, cudaStream_t copy) {
+    TgpEngine *e = ctx->eng;
+    const TgpPlan &pl = ctx->plan;
+    if (!e->advised) {
+        for (auto &p : pl.pins) {
+            const TgpTensor &t = ctx->tensors[p.first];
+            CU(ctx, cudaMemAdvise(ctx->pools[t.pool].host_base + t.off, t.size, cudaMemAdviseSetPreferredLocation, e->device));
+        }
+        e->advised = true;
+    }
+    const size_t LOOKAHEAD = 8;
+    size_t upto = std::min(step_end, op_now + 1 + LOOKAHEAD);
+    for (size_t j = std::max(e->hinted_upto, op_now); j < upto; ++j) {
+        const TgpOp &o = ctx->ops[j];
+        if (pl.cls[j] != CLS_LINK) continue;
+        for (uint32_t k = 0; k < o.nacc; ++k) {
+            const tgp_access &a = ctx->acc[o.acc0 + k];
+            if (pl.zc[a.tensor]) continue;
+            const TgpTensor &t = ctx->tensors[a.tensor];
+            CU(ctx, cudaMemPrefetchAsync(ctx->pools[t.pool].host_base + t.off, t.size, e->device, copy));
+        }
+    }
+    e->hinted_upto = std::max(e->hinted_upto, upto);
+    return TGP_OK;
+}
+
+extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_host, uint32_t B, uint32_t q_len,
+                        float *logits_dev, int32_t *argmax_dev, void *compute_stream, void *copy_stream, tgp_step_stats *stats) {
+    if (!ctx || !logits_dev) return TGP_E_INVAL;
+    if (!ctx->plan.valid) return TGP_E_NO_PLAN;
+    TgpEngine *e = ctx->eng;
+    if (!e || !ctx->bound) return tgp_fail(ctx, TGP_E_STATE, "no model bound with a workspace");
+    const bool ring = ctx->variant == TGP_VAR_EXPLICIT_RING;
+    if (ring && (!ctx->arena || ctx->arena_bytes < ctx->budget)) return tgp_fail(ctx, TGP_E_STATE, "arena missing or smaller than the budget");
+    if (!ring)
+        for (const TgpPool &p : ctx->pools) if (p.flags != TGP_POOL_MANAGED) return tgp_fail(ctx, TGP_E_STATE, "managed variants need a managed pool");
+    if (e->next_step >= ctx->steps.size()) return tgp_fail(ctx, TGP_E_STATE, "the plan has no further step; call tgp_run_reset()");
+    const TgpStep &st = ctx->steps[e->next_step];
+    const tgp_model_cfg &c = ctx->cfg;
+    if (st.kind != step_kind || B != c.B || !q_len || (step_kind == TGP_DECODE && q_len != 1)) return tgp_fail(ctx, TGP_E_INVAL, "step kind, batch or q_len differ from the plan");
+    if ((uint64_t)B * q_len > e->max_tokens || e->pos + q_len > c.max_len) return tgp_fail(ctx, TGP_E_INVAL, "more tokens than the workspace or max_len allow");
+    if (!tokens_host && (step_kind != TGP_DECODE || e->next_step == 0)) return tgp_fail(ctx, TGP_E_INVAL, "tokens are required for this step");
+    cudaStream_t cs = (cudaStream_t)compute_stream, cp = (cudaStream_t)copy_stream;
+    const uint32_t M = B * q_len, pos0 = e->pos;
+    const uint64_t launches0 = tgpk_launches;
+    uint32_t n_cmds = 0;
+    if (stats) CU(ctx, cudaEventRecord(e->t0, cs));
+    const int32_t *tok = e->amax;
+    if (tokens_host) { CU(ctx, cudaMemcpyAsync(e->tok, tokens_host, (size_t)M * 4, cudaMemcpyHostToDevice, cs)); tok = e->tok; }
+    int rc;
+    if (ring && (rc = pump(ctx, (int32_t)st.op0 - 1, cp, &n_cmds))) return rc;
+    const uint32_t qd = c.Hq * c.Dh, kd = c.Hkv * c.Dh;
+    for (uint32_t i = st.op0; i < st.op0 + st.nops; ++i) {
+        const TgpOp &o = ctx->ops[i];
+        if (ring && ctx->plan.op_last_place[i] >= 0) {
+            if ((size_t)ctx->plan.op_last_place[i] >= e->next_cmd) return tgp_fail(ctx, TGP_E_STATE, "a placement was not enqueued before its op");
+            cudaEvent_t ev;
+            if ((rc = get_event(ctx, e->copied_ev, i, &ev))) return rc;
+            CU(ctx, cudaStreamWaitEvent(cs, ev, 0));
+        }
+        if (ctx->variant == TGP_VAR_MANAGED_HINTS && (rc = hint_ahead(ctx, i, st.op0 + st.nops, cp))) return rc;
+        rc = TGP_OK;
+        switch (o.kind) {
+        case TGP_OP_EMBED:
+            rc = tgpk_embed(where(ctx, o, 0), tok, e->x, M, c.d, cs);
+            break;
+        case TGP_OP_RMSNORM: {
+            const TgpRole &r = ctx->roles[ctx->role_of_tensor[ctx->acc[o.acc0].tensor]];
+            if (r.kind == TGP_K_GF) rc = tgpk_rmsnorm(e->x + (size_t)(q_len - 1) * c.d, q_len * c.d, where(ctx, o, 0), e->hf, B, c.d, c.eps, cs);
+            else rc = tgpk_rmsnorm(e->x, c.d, where(ctx, o, 0), e->h, M, c.d, c.eps, cs);
+            break;
+        }
+        case TGP_OP_GEMM: {
+            const tgp_access &a = ctx->acc[o.acc0];
+            const int32_t ri = ctx->role_of_tensor[a.tensor];
+            if (ri < 0) return tgp_fail(ctx, TGP_E_MISMATCH, "GEMM op on a tensor with no model role");
+            const TgpRole &r = ctx->roles[ri];
+            const uint32_t K = (uint32_t)(ctx->tensors[a.tensor].size / (2ull * r.rows));
+            const void *W = where(ctx, o, 0);
+            switch (r.kind) {
+            case TGP_K_WQ: rc = tgpk_gemm(e->h, W, e->q32, M, r.rows, K, qd, r.row0, 0, cs); break;
+            case TGP_K_WK: rc = tgpk_gemm(e->h, W, e->k32, M, r.rows, K, kd, r.row0, 0, cs); break;
+            case TGP_K_WV: rc = tgpk_gemm(e->h, W, e->v32, M, r.rows, K, kd, r.row0, 0, cs); break;
+            case TGP_K_WO: rc = tgpk_gemm(e->ob, W, e->x, M, r.rows, K, c.d, r.row0, 1, cs); break;
+            case TGP_K_WG: rc = tgpk_gemm(e->h, W, e->g32, M, r.rows, K, c.F, r.row0, 0, cs); break;
+            case TGP_K_WU: rc = tgpk_gemm(e->h, W, e->u32, M, r.rows, K, c.F, r.row0, 0, cs); break;
+            case TGP_K_WD: rc = tgpk_gemm(e->ab, W, e->x, M, r.rows, K, c.d, r.row0, 1, cs); break;
+            case TGP_K_LM: rc = tgpk_gemm(e->hf, W, logits_dev, B, r.rows, K, c.V, r.row0, 0, cs); break;
+            default: return tgp_fail(ctx, TGP_E_MISMATCH, "GEMM op on a tensor that is not a weight");
+            }
+            break;
+        }
+        case TGP_OP_ROPE_KV:
+        case TGP_OP_ATTN: {
+            TgpTilePtrs tp;
+            memset(&tp, 0, sizeof(tp));
+            uint32_t nt = 0;
+            for (uint32_t k = 0; k < o.nacc; ++k) {
+                const TgpRole &r = ctx->roles[ctx->role_of_tensor[ctx->acc[o.acc0 + k].tensor]];
+                if (r.block >= TGP_MAX_TILES) return tgp_fail(ctx, TGP_E_TOO_LARGE, "KV tile index");
+                (r.kind == TGP_K_KTILE ? tp.k : tp.v)[r.block] = where(ctx, o, k);
+                nt = std::max(nt, r.block + 1);
+            }
+            if (o.kind == TGP_OP_ROPE_KV) rc = tgpk_rope_kv(e->q32, e->k32, e->v32, e->qb, tp, e->cos_t, e->sin_t, &c, B, q_len, pos0, cs);
+            else rc = tgpk_attn(e->qb, tp, (c.max_len + c.TK - 1) / c.TK, e->ob, &c, B, q_len, pos0, e->scratch, cs);
+            break;
+        }
+        case TGP_OP_SWIGLU:
+            rc = tgpk_swiglu(e->g32, e->u32, e->ab, (uint64_t)M * c.F, cs);
+            break;
+        case TGP_OP_ARGMAX:
+            rc = tgpk_argmax(logits_dev, e->amax, B, c.V, cs);
+            if (!rc && argmax_dev) CU(ctx, cudaMemcpyAsync(argmax_dev, e->amax, (size_t)B * 4, cudaMemcpyDeviceToDevice, cs));
+            break;
+        default:
+            return tgp_fail(ctx, TGP_E_MISMATCH, "op kind the bound model cannot run");
+        }
+        if (rc) return tgp_fail(ctx, rc, "kernel launch failed");
+        if (ring) {
+            if (ctx->plan.op_is_wait_target[i]) {
+                cudaEvent_t ev;
+                if ((rc = get_event(ctx, e->done_ev, i, &ev))) return rc;
+                CU(ctx, cudaEventRecord(ev, cs));
+            }
+            if ((rc = pump(ctx, (int32_t)i, cp, &n_cmds))) return rc;
+        }
+    }
+    e->pos += q_len;
+    e->next_step++;
+    if (stats) {
+        CU(ctx, cudaEventRecord(e->t1, cs));
+        CU(ctx, cudaEventSynchronize(e->t1));
+        if (ring) CU(ctx, cudaStreamSynchronize(e->wb_stream));
+        const uint64_t *tot = &ctx->plan.totals[(size_t)(e->next_step - 1) * 4];
+        stats->h2d_bytes = ring ? tot[0] : 0; stats->d2h_bytes = ring ? tot[1] : 0; stats->zc_bytes = tot[2];
+        stats->n_cmds = n_cmds; stats->n_launches = (uint32_t)(tgpk_launches - launches0); stats->n_mismatch = 0;
+        CU(ctx, cudaEventElapsedTime(&stats->step_ms, e->t0, e->t1));
+    }
+    return TGP_OK;
+}

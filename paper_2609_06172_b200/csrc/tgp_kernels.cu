@@ -1,0 +1,520 @@
+// Hand-written sm_100a kernels of the forward pass and their C entry points.
+// Precision contract: bf16 weights / KV / GEMM inputs, fp32 accumulation and residual stream.
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cstdint>
+#include "tgp.h"
+#include "tgp_kernels.h"
+
+thread_local uint64_t tgpk_launches = 0;     // kernels launched by this thread (reported in the step statistics)
+#define LAUNCH_CHECK(n) do { cudaError_t e_ = cudaGetLastError(); if (e_ != cudaSuccess) return TGP_E_CUDA; tgpk_launches += (n); } while (0)
+
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ void unpack8(const uint4 &v, float *f) {
+    const __nv_bfloat162 *p = reinterpret_cast<const __nv_bfloat162 *>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { float2 t = __bfloat1622float2(p[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// ---- embedding gather ------------------------------------------------------------------------
+__global__ void embed_kernel(const bf16 *__restrict__ table, const int32_t *__restrict__ tok, float *__restrict__ x, uint32_t d) {
+    const uint32_t m = blockIdx.x;
+    const uint4 *row = reinterpret_cast<const uint4 *>(table + (size_t)tok[m] * d);
+    float4 *out = reinterpret_cast<float4 *>(x + (size_t)m * d);
+    for (uint32_t i = threadIdx.x; i < d / 8; i += blockDim.x) {
+        float f[8];
+        unpack8(row[i], f);
+        out[2 * i] = make_float4(f[0], f[1], f[2], f[3]);
+        out[2 * i + 1] = make_float4(f[4], f[5], f[6], f[7]);
+    }
+}
+
+// ---- RMSNorm -> bf16 -------------------------------------------------------------------------
+__global__ void rmsnorm_kernel(const float *__restrict__ x, uint32_t ldx, const bf16 *__restrict__ g, bf16 *__restrict__ h, uint32_t d, float eps) {
+    __shared__ float red[32];
+    const float4 *row = reinterpret_cast<const float4 *>(x + (size_t)blockIdx.x * ldx);
+    float ss = 0.f;
+    for (uint32_t i = threadIdx.x; i < d / 4; i += blockDim.x) { float4 v = row[i]; ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w; }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        float t = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
+        t = warp_sum(t);
+        if (threadIdx.x == 0) red[0] = 1.0f / sqrtf(t / (float)d + eps);
+    }
+    __syncthreads();
+    const float r = red[0];
+    __nv_bfloat162 *out = reinterpret_cast<__nv_bfloat162 *>(h + (size_t)blockIdx.x * d);
+    const __nv_bfloat162 *gg = reinterpret_cast<const __nv_bfloat162 *>(g);
+    for (uint32_t i = threadIdx.x; i < d / 4; i += blockDim.x) {
+        float4 v = row[i];
+        float2 g0 = __bfloat1622float2(gg[2 * i]), g1 = __bfloat1622float2(gg[2 * i + 1]);
+        out[2 * i] = __floats2bfloat162_rn(v.x * r * g0.x, v.y * r * g0.y);
+        out[2 * i + 1] = __floats2bfloat162_rn(v.z * r * g1.x, v.w * r * g1.y);
+    }
+}
+
+// ---- GEMV / skinny GEMM: weight streaming, one warp per R output rows, MT activation rows -------
+template <int MT, int R>
+__global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+                                                   uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t warps = (gridDim.x * blockDim.x) >> 5;
+    for (uint32_t row0 = ((blockIdx.x * blockDim.x + threadIdx.x) >> 5) * R; row0 < n; row0 += warps * R) {
+        float acc[R][MT];
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int m = 0; m < MT; ++m) acc[r][m] = 0.f;
+        for (uint32_t k = lane * 8; k < K; k += 256) {
+            uint4 wv[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                wv[r] = (row0 + r < n) ? __ldcs(reinterpret_cast<const uint4 *>(W + (size_t)(row0 + r) * K + k)) : make_uint4(0, 0, 0, 0);
+            float wf[R][8];
+#pragma unroll
+            for (int r = 0; r < R; ++r) unpack8(wv[r], wf[r]);
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                if (m < (int)Mrows) {
+                    float xf[8];
+                    unpack8(__ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)), xf);
+#pragma unroll
+                    for (int r = 0; r < R; ++r)
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) acc[r][m] = fmaf(wf[r][i], xf[i], acc[r][m]);
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                float s = warp_sum(acc[r][m]);
+                if (lane == 0 && row0 + r < n && m < (int)Mrows) {
+                    float *c = C + (size_t)m * ldc + col0 + row0 + r;
+                    *c = accumulate ? *c + s : s;
+                }
+            }
+    }
+}
+
+// ---- generic tiled GEMM on CUDA cores (any M, n; K % 8 == 0): 64x64 tile, 4x4 per thread ---------
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+                                                        uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
+    __shared__ float As[32][64 + 4];
+    __shared__ float Ws[32][64 + 4];
+    const uint32_t m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+    const uint32_t tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    float acc[4][4] = {};
+    const uint32_t lr = threadIdx.x >> 2, lk = (threadIdx.x & 3) * 8;     // 64 rows x 4 vectors of 8
+    for (uint32_t k0 = 0; k0 < K; k0 += 32) {
+        float fa[8], fw[8];
+        uint4 va = make_uint4(0, 0, 0, 0), vw = va;
+        if (m0 + lr < M && k0 + lk < K) va = *reinterpret_cast<const uint4 *>(A + (size_t)(m0 + lr) * K + k0 + lk);
+        if (n0 + lr < n && k0 + lk < K) vw = *reinterpret_cast<const uint4 *>(W + (size_t)(n0 + lr) * K + k0 + lk);
+        unpack8(va, fa); unpack8(vw, fw);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { As[lk + i][lr] = fa[i]; Ws[lk + i][lr] = fw[i]; }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < 32; ++kk) {
+            float a[4], w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { a[i] = As[kk][ty * 4 + i]; w[i] = Ws[kk][tx * 4 + i]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], w[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t m = m0 + ty * 4 + i, c = n0 + tx * 4 + j;
+            if (m < M && c < n) { float *p = C + (size_t)m * ldc + col0 + c; *p = accumulate ? *p + acc[i][j] : acc[i][j]; }
+        }
+}
+
+// ---- RoPE + bf16 rounding + KV append -----------------------------------------------------------
+struct RopeArgs {
+    const float *q32, *k32, *v32; bf16 *qb; const float *cos_t, *sin_t;
+    uint32_t Hq, Hkv, Dh, TK, q_len, pos0;
+    TgpTilePtrs tiles;
+};
+
+__global__ void rope_kv_kernel(RopeArgs a) {
+    const uint32_t m = blockIdx.x, b = m / a.q_len, pos = a.pos0 + m % a.q_len;
+    const uint32_t half = a.Dh / 2, qd = a.Hq * a.Dh, kd = a.Hkv * a.Dh;
+    const float *cs = a.cos_t + (size_t)pos * half, *sn = a.sin_t + (size_t)pos * half;
+    const uint32_t j = pos / a.TK, slot = pos % a.TK;
+    for (uint32_t idx = threadIdx.x; idx < (a.Hq + 2 * a.Hkv) * half; idx += blockDim.x) {
+        const uint32_t h = idx / half, i = idx % half;
+        if (h < a.Hq) {
+            const float *s = a.q32 + (size_t)m * qd + h * a.Dh;
+            float x0 = s[i], x1 = s[i + half], c = cs[i], sv = sn[i];
+            bf16 *o = a.qb + (size_t)m * qd + h * a.Dh;
+            o[i] = __float2bfloat16_rn(x0 * c - x1 * sv);
+            o[i + half] = __float2bfloat16_rn(x1 * c + x0 * sv);
+        } else if (h < a.Hq + a.Hkv) {
+            const uint32_t hk = h - a.Hq;
+            const float *s = a.k32 + (size_t)m * kd + hk * a.Dh;
+            float x0 = s[i], x1 = s[i + half], c = cs[i], sv = sn[i];
+            bf16 *o = reinterpret_cast<bf16 *>(a.tiles.k[j]) + ((size_t)(b * a.Hkv + hk) * a.TK + slot) * a.Dh;
+            o[i] = __float2bfloat16_rn(x0 * c - x1 * sv);
+            o[i + half] = __float2bfloat16_rn(x1 * c + x0 * sv);
+        } else {
+            const uint32_t hk = h - a.Hq - a.Hkv;
+            const float *s = a.v32 + (size_t)m * kd + hk * a.Dh;
+            bf16 *o = reinterpret_cast<bf16 *>(a.tiles.v[j]) + ((size_t)(b * a.Hkv + hk) * a.TK + slot) * a.Dh;
+            o[i] = __float2bfloat16_rn(s[i]);
+            o[i + half] = __float2bfloat16_rn(s[i + half]);
+        }
+    }
+}
+
+// ---- attention -------------------------------------------------------------------------------------
+struct AttnArgs {
+    const bf16 *qb; bf16 *ob; float *scratch;
+    uint32_t Hq, Hkv, Dh, TK, q_len, pos0, n_tiles;
+    float scale;
+    TgpTilePtrs tiles;
+};
+
+// One warp per query row, 32 keys per pass: lane = key for the scores, lane = output dims for P.V.
+template <int DH>
+__global__ void __launch_bounds__(128) attn_rows_kernel(AttnArgs a) {
+    __shared__ float qs[4][DH];
+    const uint32_t w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t p = blockIdx.x * 4 + w, hq = blockIdx.y, b = blockIdx.z;
+    const bool live = p < a.q_len;
+    const uint32_t m = b * a.q_len + (live ? p : 0), hk = hq / (a.Hq / a.Hkv);
+    const bf16 *q = a.qb + (size_t)m * a.Hq * DH + hq * DH;
+    for (int i = lane; i < DH; i += 32) qs[w][i] = __bfloat162float(q[i]);
+    __syncwarp();
+    if (!live) return;
+    const uint32_t nkeys = a.pos0 + p + 1;
+    constexpr int DPL = DH / 32;
+    float o[DPL];
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) o[i] = 0.f;
+    float mx = -INFINITY, l = 0.f;
+    for (uint32_t j0 = 0; j0 < nkeys; j0 += 32) {
+        const uint32_t j = j0 + lane;
+        float s = -INFINITY;
+        if (j < nkeys) {
+            const uint4 *kr = reinterpret_cast<const uint4 *>(reinterpret_cast<const bf16 *>(a.tiles.k[j / a.TK]) + ((size_t)(b * a.Hkv + hk) * a.TK + j % a.TK) * DH);
+            float acc = 0.f;
+#pragma unroll
+            for (int v = 0; v < DH / 8; ++v) {
+                float f[8];
+                unpack8(kr[v], f);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc = fmaf(qs[w][v * 8 + i], f[i], acc);
+            }
+            s = acc * a.scale;
+        }
+        const float mnew = fmaxf(mx, warp_max(s));
+        const float alpha = expf(mx - mnew);
+        const float pj = (j < nkeys) ? expf(s - mnew) : 0.f;
+        l = l * alpha + warp_sum(pj);
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) o[i] *= alpha;
+        const uint32_t cnt = min(32u, nkeys - j0);
+        for (uint32_t t = 0; t < cnt; ++t) {
+            const float pt = __shfl_sync(0xffffffffu, pj, t);
+            const uint32_t jj = j0 + t;
+            const bf16 *vr = reinterpret_cast<const bf16 *>(a.tiles.v[jj / a.TK]) + ((size_t)(b * a.Hkv + hk) * a.TK + jj % a.TK) * DH;
+#pragma unroll
+            for (int i = 0; i < DPL; ++i) o[i] = fmaf(pt, __bfloat162float(vr[lane + 32 * i]), o[i]);
+        }
+        mx = mnew;
+    }
+    bf16 *out = a.ob + (size_t)m * a.Hq * DH + hq * DH;
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) out[lane + 32 * i] = __float2bfloat16_rn(o[i] / l);
+}
+
+// Decode (one query per sequence): grid (tile, kv head, batch); warp g of the block serves query head
+// hk*G + g over the keys of one tile and leaves an unnormalised partial (max, sum, o[Dh]) in scratch.
+template <int DH>
+__global__ void attn_decode_partial_kernel(AttnArgs a) {
+    extern __shared__ float qsm[];
+    const uint32_t g = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t tile = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+    const uint32_t G = a.Hq / a.Hkv, hq = hk * G + g;
+    const uint32_t kvlen = a.pos0 + 1;
+    const uint32_t nk = min(a.TK, kvlen - tile * a.TK);
+    float *qs = qsm + g * DH;
+    const bf16 *q = a.qb + (size_t)b * a.Hq * DH + hq * DH;
+    for (int i = lane; i < DH; i += 32) qs[i] = __bfloat162float(q[i]);
+    __syncwarp();
+    constexpr int DPL = DH / 32;
+    float o[DPL];
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) o[i] = 0.f;
+    float mx = -INFINITY, l = 0.f;
+    const bf16 *kt = reinterpret_cast<const bf16 *>(a.tiles.k[tile]) + (size_t)(b * a.Hkv + hk) * a.TK * DH;
+    const bf16 *vt = reinterpret_cast<const bf16 *>(a.tiles.v[tile]) + (size_t)(b * a.Hkv + hk) * a.TK * DH;
+    for (uint32_t j0 = 0; j0 < nk; j0 += 32) {
+        const uint32_t j = j0 + lane;
+        float s = -INFINITY;
+        if (j < nk) {
+            const uint4 *kr = reinterpret_cast<const uint4 *>(kt + (size_t)j * DH);
+            float acc = 0.f;
+#pragma unroll
+            for (int v = 0; v < DH / 8; ++v) {
+                float f[8];
+                unpack8(kr[v], f);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc = fmaf(qs[v * 8 + i], f[i], acc);
+            }
+            s = acc * a.scale;
+        }
+        const float mnew = fmaxf(mx, warp_max(s));
+        const float alpha = expf(mx - mnew);
+        const float pj = (j < nk) ? expf(s - mnew) : 0.f;
+        l = l * alpha + warp_sum(pj);
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) o[i] *= alpha;
+        const uint32_t cnt = min(32u, nk - j0);
+        for (uint32_t t = 0; t < cnt; ++t) {
+            const float pt = __shfl_sync(0xffffffffu, pj, t);
+            const bf16 *vr = vt + (size_t)(j0 + t) * DH;
+#pragma unroll
+            for (int i = 0; i < DPL; ++i) o[i] = fmaf(pt, __bfloat162float(vr[lane + 32 * i]), o[i]);
+        }
+        mx = mnew;
+    }
+    float *part = a.scratch + ((size_t)(b * a.Hq + hq) * a.n_tiles + tile) * (DH + 2);
+    if (lane == 0) { part[0] = mx; part[1] = l; }
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) part[2 + lane + 32 * i] = o[i];
+}
+
+// Merge the per-tile partials of one (batch, query head): grid (Hq, B), DH threads.
+template <int DH>
+__global__ void attn_decode_merge_kernel(AttnArgs a) {
+    const uint32_t hq = blockIdx.x, b = blockIdx.y, i = threadIdx.x;
+    const uint32_t nt = (a.pos0 + 1 + a.TK - 1) / a.TK;
+    const float *part = a.scratch + (size_t)(b * a.Hq + hq) * a.n_tiles * (DH + 2);
+    float mx = -INFINITY;
+    for (uint32_t t = 0; t < nt; ++t) mx = fmaxf(mx, part[t * (DH + 2)]);
+    float l = 0.f, o = 0.f;
+    for (uint32_t t = 0; t < nt; ++t) {
+        const float w = expf(part[t * (DH + 2)] - mx);
+        l += w * part[t * (DH + 2) + 1];
+        o += w * part[t * (DH + 2) + 2 + i];
+    }
+    a.ob[(size_t)b * a.Hq * DH + hq * DH + i] = __float2bfloat16_rn(o / l);
+}
+
+// ---- SwiGLU -----------------------------------------------------------------------------------------
+__global__ void swiglu_kernel(const float4 *__restrict__ g, const float4 *__restrict__ u, __nv_bfloat162 *__restrict__ out, uint64_t n4) {
+    for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n4; i += (uint64_t)gridDim.x * blockDim.x) {
+        float4 a = g[i], b = u[i];
+        float r0 = a.x / (1.0f + expf(-a.x)) * b.x, r1 = a.y / (1.0f + expf(-a.y)) * b.y;
+        float r2 = a.z / (1.0f + expf(-a.z)) * b.z, r3 = a.w / (1.0f + expf(-a.w)) * b.w;
+        out[2 * i] = __floats2bfloat162_rn(r0, r1);
+        out[2 * i + 1] = __floats2bfloat162_rn(r2, r3);
+    }
+}
+
+// ---- argmax, lowest index on ties -----------------------------------------------------------------
+__global__ void __launch_bounds__(1024) argmax_kernel(const float *__restrict__ logits, int32_t *__restrict__ out, uint32_t V) {
+    __shared__ float bv[32];
+    __shared__ uint32_t bi[32];
+    const float *row = logits + (size_t)blockIdx.x * V;
+    float best = -INFINITY; uint32_t idx = 0xffffffffu;
+    for (uint32_t j = threadIdx.x; j < V; j += blockDim.x) { float v = row[j]; if (v > best || (v == best && j < idx)) { best = v; idx = j; } }
+    auto merge = [](float &v, uint32_t &i, float ov, uint32_t oi) { if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; } };
+#pragma unroll
+    for (int o = 16; o; o >>= 1) merge(best, idx, __shfl_xor_sync(0xffffffffu, best, o), __shfl_xor_sync(0xffffffffu, idx, o));
+    if ((threadIdx.x & 31) == 0) { bv[threadIdx.x >> 5] = best; bi[threadIdx.x >> 5] = idx; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        best = threadIdx.x < (blockDim.x >> 5) ? bv[threadIdx.x] : -INFINITY;
+        idx = threadIdx.x < (blockDim.x >> 5) ? bi[threadIdx.x] : 0xffffffffu;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) merge(best, idx, __shfl_xor_sync(0xffffffffu, best, o), __shfl_xor_sync(0xffffffffu, idx, o));
+        if (threadIdx.x == 0) out[blockIdx.x] = (int32_t)idx;
+    }
+}
+
+// ============================ launchers (internal) ===================================================
+int tgpk_embed(const void *table, const int32_t *tok, float *x, uint32_t M, uint32_t d, cudaStream_t st) {
+    if (!M) return TGP_OK;
+    if (d % 8) return TGP_E_INVAL;
+    embed_kernel<<<M, 128, 0, st>>>((const bf16 *)table, tok, x, d);
+    LAUNCH_CHECK(1);
+    return TGP_OK;
+}
+
+int tgpk_rmsnorm(const float *x, uint32_t ldx, const void *g, void *h, uint32_t M, uint32_t d, float eps, cudaStream_t st) {
+    if (!M) return TGP_OK;
+    if (d % 4 || ldx % 4) return TGP_E_INVAL;
+    rmsnorm_kernel<<<M, 256, 0, st>>>(x, ldx, (const bf16 *)g, (bf16 *)h, d, eps);
+    LAUNCH_CHECK(1);
+    return TGP_OK;
+}
+
+template <int MT, int R>
+static void launch_gemv(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int acc, cudaStream_t st) {
+    uint32_t warps_needed = (n + R - 1) / R;
+    uint32_t blocks = (warps_needed + 7) / 8;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    gemv_kernel<MT, R><<<blocks, 256, 0, st>>>(A, W, C, Mrows, n, K, ldc, col0, acc);
+}
+
+int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
+    if (!M || !n) return TGP_OK;
+    if (K % 8 || !K) return TGP_E_INVAL;
+    const bf16 *a = (const bf16 *)A, *w = (const bf16 *)W;
+    if (M <= 16) {
+        for (uint32_t m0 = 0; m0 < M; m0 += 8) {
+            uint32_t mr = M - m0 < 8 ? M - m0 : 8;
+            const bf16 *am = a + (size_t)m0 * K;
+            float *cm = C + (size_t)m0 * ldc;
+            if (mr == 1) launch_gemv<1, 4>(am, w, cm, mr, n, K, ldc, col0, accumulate, st);
+            else if (mr == 2) launch_gemv<2, 4>(am, w, cm, mr, n, K, ldc, col0, accumulate, st);
+            else if (mr <= 4) launch_gemv<4, 2>(am, w, cm, mr, n, K, ldc, col0, accumulate, st);
+            else launch_gemv<8, 2>(am, w, cm, mr, n, K, ldc, col0, accumulate, st);
+            if (m0) tgpk_launches += 1;
+        }
+    } else {
+        dim3 grid((n + 63) / 64, (M + 63) / 64);
+        gemm_simt_kernel<<<grid, 256, 0, st>>>(a, w, C, M, n, K, ldc, col0, accumulate);
+    }
+    LAUNCH_CHECK(1);
+    return TGP_OK;
+}
+
+int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb, const TgpTilePtrs &tiles, const float *cos_t, const float *sin_t,
+                 const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0, cudaStream_t st) {
+    if (!B || !q_len) return TGP_OK;
+    RopeArgs a{q32, k32, v32, (bf16 *)qb, cos_t, sin_t, c->Hq, c->Hkv, c->Dh, c->TK, q_len, pos0, tiles};
+    rope_kv_kernel<<<B * q_len, 256, 0, st>>>(a);
+    LAUNCH_CHECK(1);
+    return TGP_OK;
+}
+
+int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *ob, const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0,
+              float *scratch, cudaStream_t st) {
+    if (!B || !q_len) return TGP_OK;
+    if (c->Dh != 64 && c->Dh != 128) return TGP_E_INVAL;
+    AttnArgs a{(const bf16 *)qb, (bf16 *)ob, scratch, c->Hq, c->Hkv, c->Dh, c->TK, q_len, pos0, n_tiles, 1.0f / sqrtf((float)c->Dh), tiles};
+    if (q_len == 1 && scratch) {
+        const uint32_t nt = (pos0 + 1 + c->TK - 1) / c->TK, G = c->Hq / c->Hkv;
+        dim3 grid(nt, c->Hkv, B);
+        if (c->Dh == 64) {
+            attn_decode_partial_kernel<64><<<grid, 32 * G, G * 64 * sizeof(float), st>>>(a);
+            attn_decode_merge_kernel<64><<<dim3(c->Hq, B), 64, 0, st>>>(a);
+        } else {
+            attn_decode_partial_kernel<128><<<grid, 32 * G, G * 128 * sizeof(float), st>>>(a);
+            attn_decode_merge_kernel<128><<<dim3(c->Hq, B), 128, 0, st>>>(a);
+        }
+        tgpk_launches += 1;
+    } else {
+        dim3 grid((q_len + 3) / 4, c->Hq, B);
+        if (c->Dh == 64) attn_rows_kernel<64><<<grid, 128, 0, st>>>(a);
+        else attn_rows_kernel<128><<<grid, 128, 0, st>>>(a);
+    }
+    LAUNCH_CHECK(1);
+    return TGP_OK;
+}
+
+int tgpk_swiglu(const float *g, const float *u, void *ab, uint64_t n, cudaStream_t st) {
+    if (!n) return TGP_OK;
+    if (n % 4) return TGP_E_INVAL;
+    uint64_t n4 = n / 4;
+    uint32_t blocks = (uint32_t)((n4 + 255) / 256 < 148 * 16 ? (n4 + 255) / 256 : 148 * 16);
+    swiglu_kernel<<<blocks, 256, 0, st>>>((const float4 *)g, (const float4 *)u, (__nv_bfloat162 *)ab, n4);
+    LAUNCH_CHECK(1);
+    return TGP_OK;
+}
+
+int tgpk_argmax(const float *logits, int32_t *out, uint32_t B, uint32_t V, cudaStream_t st) {
+    if (!B) return TGP_OK;
+    argmax_kernel<<<B, 1024, 0, st>>>(logits, out, V);
+    LAUNCH_CHECK(1);
+    return TGP_OK;
+}
+
+// ============================ C entry points ===========================================================
+static int fill_tiles(TgpTilePtrs &t, void *const *k, void *const *v, uint32_t n) {
+    if (n > TGP_MAX_TILES) return TGP_E_TOO_LARGE;
+    if (!k || !v) return TGP_E_INVAL;
+    for (uint32_t i = 0; i < n; ++i) { t.k[i] = k[i]; t.v[i] = v[i]; }
+    return TGP_OK;
+}
+
+extern "C" {
+
+int tgp_k_embed(const void *table, const int32_t *tok_dev, float *x_dev, uint32_t M, uint32_t d, void *stream) {
+    if (!table || !tok_dev || !x_dev) return TGP_E_INVAL;
+    return tgpk_embed(table, tok_dev, x_dev, M, d, (cudaStream_t)stream);
+}
+
+int tgp_k_rmsnorm(const float *x_dev, uint32_t ldx, const void *g_dev, void *h_dev, uint32_t M, uint32_t d, float eps, void *stream) {
+    if (!x_dev || !g_dev || !h_dev) return TGP_E_INVAL;
+    return tgpk_rmsnorm(x_dev, ldx, g_dev, h_dev, M, d, eps, (cudaStream_t)stream);
+}
+
+int tgp_k_gemm(const void *A_dev, const void *W_dev, float *C_dev, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, void *stream) {
+    if (!A_dev || !W_dev || !C_dev || col0 + (uint64_t)n > ldc) return TGP_E_INVAL;
+    return tgpk_gemm(A_dev, W_dev, C_dev, M, n, K, ldc, col0, accumulate, (cudaStream_t)stream);
+}
+
+int tgp_k_rope_kv(const float *q32, const float *k32, const float *v32, void *qb, void *const *k_tiles, void *const *v_tiles, uint32_t n_tiles,
+                  const float *cos_dev, const float *sin_dev, const tgp_model_cfg *cfg, uint32_t B, uint32_t q_len, uint32_t pos0, void *stream) {
+    if (!q32 || !k32 || !v32 || !qb || !cfg || !cos_dev || !sin_dev) return TGP_E_INVAL;
+    if (pos0 + q_len > cfg->max_len || (uint64_t)n_tiles * cfg->TK < pos0 + q_len || cfg->Dh % 2) return TGP_E_INVAL;
+    TgpTilePtrs t;
+    int rc = fill_tiles(t, k_tiles, v_tiles, n_tiles);
+    if (rc) return rc;
+    return tgpk_rope_kv(q32, k32, v32, qb, t, cos_dev, sin_dev, cfg, B, q_len, pos0, (cudaStream_t)stream);
+}
+
+int tgp_k_attn(const void *qb, void *const *k_tiles, void *const *v_tiles, uint32_t n_tiles, void *ob, const tgp_model_cfg *cfg, uint32_t B, uint32_t q_len,
+               uint32_t pos0, float *scratch_dev, void *stream) {
+    if (!qb || !ob || !cfg || !cfg->Hkv || cfg->Hq % cfg->Hkv) return TGP_E_INVAL;
+    if ((uint64_t)n_tiles * cfg->TK < pos0 + q_len) return TGP_E_INVAL;
+    TgpTilePtrs t;
+    int rc = fill_tiles(t, k_tiles, v_tiles, n_tiles);
+    if (rc) return rc;
+    return tgpk_attn(qb, t, n_tiles, ob, cfg, B, q_len, pos0, scratch_dev, (cudaStream_t)stream);
+}
+
+int tgp_k_attn_scratch_bytes(const tgp_model_cfg *cfg, uint64_t *bytes) {
+    if (!cfg || !bytes || !cfg->TK) return TGP_E_INVAL;
+    uint64_t nt = (cfg->max_len + cfg->TK - 1) / cfg->TK;
+    *bytes = (uint64_t)cfg->B * cfg->Hq * nt * (cfg->Dh + 2) * sizeof(float);
+    return TGP_OK;
+}
+
+int tgp_k_swiglu(const float *g32, const float *u32, void *ab, uint64_t n_elems, void *stream) {
+    if (!g32 || !u32 || !ab) return TGP_E_INVAL;
+    return tgpk_swiglu(g32, u32, ab, n_elems, (cudaStream_t)stream);
+}
+
+int tgp_k_argmax(const float *logits, int32_t *out, uint32_t B, uint32_t V, void *stream) {
+    if (!logits || !out || !V) return TGP_E_INVAL;
+    return tgpk_argmax(logits, out, B, V, (cudaStream_t)stream);
+}
+
+}  // extern "C"

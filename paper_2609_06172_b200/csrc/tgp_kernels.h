@@ -1,0 +1,21 @@
+// Internal launch interface between the step engine and the kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+#include "tgp.h"
+
+#define TGP_MAX_TILES 64      // KV tiles per layer a kernel can address (pointer table passed by value)
+
+struct TgpTilePtrs { void *k[TGP_MAX_TILES]; void *v[TGP_MAX_TILES]; };
+
+int tgpk_embed(const void *table, const int32_t *tok, float *x, uint32_t M, uint32_t d, cudaStream_t st);
+int tgpk_rmsnorm(const float *x, uint32_t ldx, const void *g, void *h, uint32_t M, uint32_t d, float eps, cudaStream_t st);
+int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st);
+int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb, const TgpTilePtrs &tiles, const float *cos_t, const float *sin_t,
+                 const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0, cudaStream_t st);
+int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *ob, const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0,
+              float *scratch, cudaStream_t st);
+int tgpk_swiglu(const float *g, const float *u, void *ab, uint64_t n, cudaStream_t st);
+int tgpk_argmax(const float *logits, int32_t *out, uint32_t B, uint32_t V, cudaStream_t st);
+// cos/sin tables [max_len, Dh/2] fp32 (angle = pos * base^(-2i/Dh), evaluated in double) written to device memory
+int tgp_rope_tables_upload(uint32_t Dh, uint32_t max_len, float base, float *cos_dev, float *sin_dev);

@@ -1,0 +1,187 @@
+"""Kernel parity on the GPU: every kernel of the path, called through the C ABI, against the CPU oracle
+on the same seeded inputs; sizes span several tiles and ragged tails, plus the degenerate cases."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+import seeded_inputs as si
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+from oracle.forward import OracleModel, bf16_round  # noqa: E402
+from paper_2609_06172_b200 import binding as tb  # noqa: E402
+from paper_2609_06172_b200.session import model_cfg  # noqa: E402
+
+DEV = "cuda:0"
+KCFG = si.ModelConfig("k", L=1, d=128, Hq=4, Hkv=2, Dh=64, F=256, V=512, B=2, S=8, T=8, TK=4, seed=7, budget_rule="half_w")
+
+
+def bf16_dev(bits):
+    return torch.from_numpy(bits.view(np.int16)).to(DEV).view(torch.bfloat16)
+
+
+def rnd_bits(role, n):
+    return si.normal_bf16_bits(1234, role, 0, n)
+
+
+def oracle():
+    lay = si.build_layout(KCFG)
+    return OracleModel(KCFG, si.weights_as_bits(lay))
+
+
+def bf16_close(got_f32, want_f32, frac=0.01):
+    """Equal up to one bf16 ulp, and different at all in at most `frac` of the entries (rounding flips
+    where fp32 summation order differs by a last bit)."""
+    got, want = np.asarray(got_f32, np.float32), np.asarray(want_f32, np.float32)
+    tol = np.maximum(np.abs(want), 1e-30) * 2.0 ** -7
+    assert (np.abs(got - want) <= tol).all(), float(np.abs(got - want).max())
+    assert (got != want).mean() <= frac
+
+
+@pytest.mark.parametrize("M,n,K", [(1, 300, 256), (1, 4096, 2048), (2, 129, 64), (3, 1000, 512), (8, 1030, 512),
+                                   (13, 77, 128), (16, 260, 1024), (17, 64, 96), (33, 130, 96), (200, 260, 1024),
+                                   (64, 64, 32), (1, 1, 8), (70, 5, 8)])
+@pytest.mark.parametrize("accumulate", [0, 1])
+def test_gemm_matches_oracle(M, n, K, accumulate):
+    a_bits, w_bits = rnd_bits(1, M * K).reshape(M, K), rnd_bits(2, n * K).reshape(n, K)
+    A, W = bf16_dev(a_bits), bf16_dev(w_bits)
+    ldc, col0 = n + 24, 8
+    c0 = np.random.default_rng(M * n).standard_normal((M, ldc)).astype(np.float32) * 0.01
+    Cd = torch.from_numpy(c0.copy()).to(DEV)
+    tb.k_gemm(A, W, Cd, M, n, K, ldc, col0, accumulate)
+    torch.cuda.synchronize()
+    got = Cd.cpu().numpy()
+    o = oracle()
+    want = o.linear(si.bf16_bits_to_f32(a_bits), si.bf16_bits_to_f32(w_bits).astype(np.float64)).astype(np.float64)
+    exp = c0.astype(np.float64).copy()
+    exp[:, col0:col0 + n] = want + (c0[:, col0:col0 + n] if accumulate else 0)
+    scale = np.abs(want).max() + 1e-6
+    assert np.abs(got - exp).max() < 2e-5 * max(scale, 0.01) + 1e-7
+    assert np.array_equal(got[:, :col0], c0[:, :col0]) and np.array_equal(got[:, col0 + n:], c0[:, col0 + n:])
+
+
+def test_gemm_rejects_bad_arguments_and_accepts_empty():
+    A = torch.zeros(8, 16, dtype=torch.bfloat16, device=DEV)
+    Cd = torch.zeros(8, 8, dtype=torch.float32, device=DEV)
+    with pytest.raises(tb.TgpError):
+        tb.k_gemm(A, A, Cd, 8, 8, 12, 8, 0, 0)          # K % 8
+    with pytest.raises(tb.TgpError):
+        tb.k_gemm(A, A, Cd, 8, 8, 16, 8, 4, 0)          # col0 + n > ldc
+    tb.k_gemm(A, A, Cd, 0, 8, 16, 8, 0, 0)              # empty M: no launch, no error
+    torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("M,d", [(1, 128), (5, 256), (37, 2048), (3, 8192)])
+def test_rmsnorm_and_embed(M, d):
+    V = 300
+    tab_bits = rnd_bits(3, V * d).reshape(V, d)
+    tok = (np.arange(M, dtype=np.int32) * 37 + 5) % V
+    x = torch.empty(M, d, dtype=torch.float32, device=DEV)
+    tb.k_embed(bf16_dev(tab_bits), torch.from_numpy(tok).to(DEV), x, M, d)
+    torch.cuda.synchronize()
+    assert np.array_equal(x.cpu().numpy(), si.bf16_bits_to_f32(tab_bits)[tok])
+    xin = (np.random.default_rng(d).standard_normal((M, d)) * 3).astype(np.float32)
+    g_bits = si.f32_to_bf16_bits(1.0 + 0.1 * np.random.default_rng(1).standard_normal(d).astype(np.float32))
+    h = torch.empty(M, d, dtype=torch.bfloat16, device=DEV)
+    tb.k_rmsnorm(torch.from_numpy(xin).to(DEV), d, bf16_dev(g_bits), h, M, d, 1e-5)
+    torch.cuda.synchronize()
+    o = oracle()
+    want = o.rmsnorm(xin, si.bf16_bits_to_f32(g_bits).astype(np.float64))
+    bf16_close(h.float().cpu().numpy(), want)
+
+
+def make_tiles(cfg, B):
+    nt = cfg.n_tiles
+    k = [torch.zeros(B * cfg.Hkv * cfg.TK * cfg.Dh, dtype=torch.bfloat16, device=DEV) for _ in range(nt)]
+    v = [torch.zeros(B * cfg.Hkv * cfg.TK * cfg.Dh, dtype=torch.bfloat16, device=DEV) for _ in range(nt)]
+    return k, v
+
+
+def tiles_to_cache(tiles, cfg, B):
+    """[n_tiles] x [B, Hkv, TK, Dh] -> [B, Hkv, n_tiles*TK, Dh] fp32"""
+    t = torch.stack([x.view(B, cfg.Hkv, cfg.TK, cfg.Dh) for x in tiles], dim=2)
+    return t.reshape(B, cfg.Hkv, -1, cfg.Dh).float().cpu().numpy()
+
+
+@pytest.mark.parametrize("Dh,Hq,Hkv,TK,S,T", [(64, 4, 2, 4, 9, 7), (128, 8, 2, 16, 40, 5), (64, 4, 4, 8, 33, 3), (128, 8, 1, 64, 130, 2)])
+def test_rope_kv_and_attention_prefill_then_decode(Dh, Hq, Hkv, TK, S, T):
+    B = 2
+    cfg = replace(KCFG, Dh=Dh, Hq=Hq, Hkv=Hkv, TK=TK, S=S, T=T, B=B, d=Hq * Dh)
+    lay_w = {(k, 0, -1): rnd_bits(k, 8).reshape(1, 8) for k in range(13)}
+    o = OracleModel(cfg, lay_w)
+    mc = model_cfg(cfg)
+    cos = torch.empty(cfg.max_len * Dh // 2, dtype=torch.float32, device=DEV)
+    sin = torch.empty_like(cos)
+    tb.k_rope_tables(Dh, cfg.max_len, cfg.rope_base, cos, sin)
+    assert np.array_equal(cos.cpu().numpy().reshape(cfg.max_len, Dh // 2), o.cos)
+    kt, vt = make_tiles(cfg, B)
+    scratch = torch.empty(tb.k_attn_scratch_bytes(mc) // 4, dtype=torch.float32, device=DEV)
+    rng = np.random.default_rng(S)
+    pos0 = 0
+    for step in range(1 + T):
+        q = S if step == 0 else 1
+        q32 = rng.standard_normal((B * q, Hq * Dh)).astype(np.float32)
+        k32 = rng.standard_normal((B * q, Hkv * Dh)).astype(np.float32)
+        v32 = rng.standard_normal((B * q, Hkv * Dh)).astype(np.float32)
+        qb = torch.empty(B * q, Hq * Dh, dtype=torch.bfloat16, device=DEV)
+        ob = torch.empty(B * q, Hq * Dh, dtype=torch.bfloat16, device=DEV)
+        tb.k_rope_kv(torch.from_numpy(q32).to(DEV), torch.from_numpy(k32).to(DEV), torch.from_numpy(v32).to(DEV), qb, kt, vt, cos, sin, mc, B, q, pos0)
+        tb.k_attn(qb, kt, vt, ob, mc, B, q, pos0, scratch)
+        torch.cuda.synchronize()
+        # oracle: same steps
+        qo = bf16_round(o.rope(q32.reshape(B, q, Hq, Dh), pos0))
+        ko = bf16_round(o.rope(k32.reshape(B, q, Hkv, Dh), pos0))
+        vo = bf16_round(v32.reshape(B, q, Hkv, Dh))
+        o.K[0, :, :, pos0:pos0 + q] = ko.transpose(0, 2, 1, 3)
+        o.V[0, :, :, pos0:pos0 + q] = vo.transpose(0, 2, 1, 3)
+        bf16_close(qb.float().cpu().numpy().reshape(B, q, Hq, Dh), qo)
+        got_k = tiles_to_cache(kt, cfg, B)[:, :, :pos0 + q]
+        bf16_close(got_k, o.K[0, :, :, :pos0 + q])
+        assert np.array_equal(tiles_to_cache(vt, cfg, B)[:, :, :pos0 + q], o.V[0, :, :, :pos0 + q].astype(np.float32))
+        # attention on the oracle's own q and cache would differ by the rare rounding flips above; feed it the GPU's
+        o.K[0, :, :, :pos0 + q] = got_k
+        att = o.attention(0, qb.float().cpu().numpy().reshape(B, q, Hq, Dh), pos0)
+        got = ob.float().cpu().numpy().reshape(B, q, Hq, Dh)
+        assert np.abs(got - att).max() < 2.0 ** -7 * np.abs(att).max() + 1e-6
+        assert np.mean(np.abs(got - bf16_round(att))) < 1e-3 * np.abs(att).mean()
+        pos0 += q
+
+
+def test_attention_single_key_returns_v():
+    cfg = replace(KCFG, B=1, S=1, T=0)
+    mc = model_cfg(cfg)
+    kt, vt = make_tiles(cfg, 1)
+    vt[0].copy_(bf16_dev(rnd_bits(9, vt[0].numel())))
+    kt[0].copy_(bf16_dev(rnd_bits(8, kt[0].numel())))
+    qb = bf16_dev(rnd_bits(7, cfg.Hq * cfg.Dh)).view(1, -1)
+    for scratch in (None, torch.empty(tb.k_attn_scratch_bytes(mc) // 4, dtype=torch.float32, device=DEV)):
+        ob = torch.empty(1, cfg.Hq * cfg.Dh, dtype=torch.bfloat16, device=DEV)
+        tb.k_attn(qb, kt, vt, ob, mc, 1, 1, 0, scratch)
+        torch.cuda.synchronize()
+        v = vt[0].view(1, cfg.Hkv, cfg.TK, cfg.Dh)[0, :, 0]                     # first token of each kv head
+        want = v.repeat_interleave(cfg.Hq // cfg.Hkv, dim=0).reshape(1, -1)
+        assert torch.equal(ob, want)
+
+
+def test_swiglu_and_argmax():
+    n = 4 * 1000 + 4
+    rng = np.random.default_rng(4)
+    g = (rng.standard_normal(n) * 4).astype(np.float32)
+    u = rng.standard_normal(n).astype(np.float32)
+    out = torch.empty(n, dtype=torch.bfloat16, device=DEV)
+    tb.k_swiglu(torch.from_numpy(g).to(DEV), torch.from_numpy(u).to(DEV), out, n)
+    torch.cuda.synchronize()
+    gd = g.astype(np.float64)
+    bf16_close(out.float().cpu().numpy(), bf16_round((gd / (1 + np.exp(-gd)) * u).astype(np.float32)))
+    B, V = 5, 128256
+    lg = rng.standard_normal((B, V)).astype(np.float32)
+    lg[1, 77] = lg[1, 90000] = 9.0            # tie: lowest index wins
+    lg[2, :] = 0.5                            # all equal -> 0
+    lg[3, V - 1] = 11.0                       # last element
+    am = torch.empty(B, dtype=torch.int32, device=DEV)
+    tb.k_argmax(torch.from_numpy(lg).to(DEV), am, B, V)
+    torch.cuda.synchronize()
+    assert am.cpu().numpy().tolist() == np.argmax(lg, axis=1).tolist()
+    assert am.cpu().numpy()[1] == 77 and am.cpu().numpy()[2] == 0 and am.cpu().numpy()[3] == V - 1

@@ -1,0 +1,140 @@
+"""End-to-end parity on the GPU: the planned, oversubscribed forward pass through tgp_step() against the
+oracle (teacher-forced tokens), at the tolerance the benchmark spec states: max abs 3e-2, mean relative 1e-2."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+import seeded_inputs as si
+from conftest import MACHINE
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+from oracle import forward, policy, trace, validate  # noqa: E402
+from paper_2609_06172_b200 import binding as tb  # noqa: E402
+from paper_2609_06172_b200.runner import Runner, pinned_pool  # noqa: E402
+from paper_2609_06172_b200.session import Session  # noqa: E402
+
+MAX_ABS, MEAN_REL = 3e-2, 1e-2
+
+
+def setup(cfg, budget=None, bits=7, n_dec=None, cap=None):
+    lay = si.build_layout(cfg, budget=budget, cap=cap)
+    pool = pinned_pool(lay.pool_bytes)
+    si.fill_pool(lay, pool.numpy())
+    s = Session(lay, MACHINE, pool_base=pool.data_ptr(), pool_flags=tb.POOL_PINNED)
+    T = cfg.T if n_dec is None else n_dec
+    blobs = s.plan(T=T, bits=bits)
+    return lay, pool, s, blobs, T
+
+
+def check_logits(got, ref):
+    worst = 0.0
+    for a, b in zip(got, ref):
+        err = np.abs(a - b)
+        assert err.max() < MAX_ABS, err.max()
+        assert err.mean() / np.abs(b).mean() < MEAN_REL
+        worst = max(worst, err.max())
+    return worst
+
+
+def test_config_1_full_run_matches_oracle_and_schedule_is_bit_exact():
+    cfg = si.CONFIGS[1]
+    lay, pool, s, blobs, T = setup(cfg)
+    ops, steps = trace.run_trace(lay)
+    want = policy.plan(lay.tensors, ops, steps, policy.Machine(**MACHINE), lay.budget).blobs()
+    assert blobs == want
+    om = forward.OracleModel(cfg, si.weights_as_bits(lay))
+    prompt = si.prompt_tokens(cfg)
+    ref, toks = om.generate(prompt, T)
+    r = Runner(s, cfg.B * cfg.S)
+    got, _ = r.generate(prompt, T, forced=toks)
+    assert len(got) == T + 1
+    check_logits(got, ref)
+    # free-running greedy decode on the device agrees with the oracle's tokens (argmax, lowest id on ties)
+    got2, toks2 = r.generate(prompt, T)
+    agree = (toks2 == toks).mean()
+    assert agree > 0.9, agree
+    s.close()
+
+
+@pytest.mark.parametrize("bits", [0, tb.BIT_A | tb.BIT_P, 7])
+def test_oversubscribed_run_is_bitwise_equal_to_a_fully_resident_run(bits):
+    """Placement must not change a single bit: 50 % budget (ring + pins, write-backs) vs everything resident."""
+    cfg = replace(si.CONFIGS[1], B=2, S=19, T=6, TK=8)
+    prompt = si.prompt_tokens(cfg)
+    forced = (np.arange(cfg.B * cfg.T, dtype=np.int32).reshape(cfg.B, cfg.T) * 911 + 3) % cfg.V
+    outs = []
+    for budget, b in ((None, bits), (64 << 20, 7)):
+        lay, pool, s, blobs, T = setup(cfg, budget=budget, bits=b, cap=128 << 10)
+        ops, steps = trace.run_trace(lay)
+        validate.check(lay.tensors, ops, steps, lay.budget, blobs)
+        r = Runner(s, cfg.B * cfg.S)
+        got, _ = r.generate(prompt, T, forced=forced)
+        outs.append(got)
+        if budget is None:
+            # KV tiles that were streamed have been written back: host pool holds the device's K/V
+            r.sync()
+            pins = {t for t, _ in (np.frombuffer(blobs["pins"][:-16], dtype=np.dtype([("t", "<u4"), ("o", "<u8")])).tolist())}
+            streamed = [t for t in lay.tensors if t.kind >= si.K_KT and t.tid not in pins]
+            if bits == 0:
+                assert len(streamed) == len([t for t in lay.tensors if t.kind >= si.K_KT])
+            host = pool.numpy()
+            nz = sum(int(host[t.pool_off:t.pool_off + t.size].any()) for t in streamed)
+            assert nz == len(streamed)
+        s.close()
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
+
+
+def test_ragged_small_model_with_batch_and_gqa():
+    cfg = si.ModelConfig("ragged", L=3, d=128, Hq=2, Hkv=1, Dh=64, F=264, V=520, B=3, S=11, T=5, TK=4, seed=5, budget_rule="half_w_kv")
+    lay = si.build_layout(cfg, budget=None, cap=16 << 10)
+    # weights at std 0.02 and d=128 give tiny logits; scale the test's tolerance check with the reference instead
+    pool = pinned_pool(lay.pool_bytes)
+    si.fill_pool(lay, pool.numpy())
+    s = Session(lay, MACHINE, pool_base=pool.data_ptr(), pool_flags=tb.POOL_PINNED)
+    s.plan()
+    om = forward.OracleModel(cfg, si.weights_as_bits(lay))
+    prompt = si.prompt_tokens(cfg)
+    ref, toks = om.generate(prompt, cfg.T)
+    r = Runner(s, cfg.B * cfg.S)
+    got, _ = r.generate(prompt, cfg.T, forced=toks)
+    check_logits(got, ref)
+    s.close()
+
+
+def test_step_stats_and_call_order_errors():
+    cfg = si.CONFIGS[1]
+    lay, pool, s, blobs, T = setup(cfg, n_dec=2)
+    r = Runner(s, cfg.B * cfg.S)
+    prompt = si.prompt_tokens(cfg)
+    with pytest.raises(tb.TgpError):
+        r.step(tb.DECODE, None, 1)                       # plan starts with a prefill
+    st = r.step(tb.PREFILL, prompt, cfg.S, want_stats=True)
+    totals = np.frombuffer(blobs["totals"], dtype="<u8").reshape(-1, 4)
+    assert (st.h2d_bytes, st.d2h_bytes, st.zc_bytes) == tuple(int(x) for x in totals[0][:3])
+    assert st.n_launches > 0 and st.step_ms > 0
+    r.step(tb.DECODE, None, 1)
+    r.step(tb.DECODE, None, 1)
+    with pytest.raises(tb.TgpError) as ei:
+        r.step(tb.DECODE, None, 1)                       # plan exhausted
+    assert ei.value.code == tb.E_STATE
+    r.reset()
+    r.step(tb.PREFILL, prompt, cfg.S)
+    r.sync()
+    s.close()
+
+
+def test_config_2_prefill_and_first_decode_steps_match_oracle():
+    cfg = si.CONFIGS[2]
+    n_dec = 3
+    lay, pool, s, blobs, T = setup(cfg, n_dec=n_dec)
+    om = forward.OracleModel(cfg, si.weights_as_bits(lay), dtype=np.float32)
+    prompt = si.prompt_tokens(cfg)
+    ref, toks = om.generate(prompt, n_dec)
+    r = Runner(s, cfg.B * cfg.S)
+    got, _ = r.generate(prompt, n_dec, forced=toks)
+    check_logits(got, ref)
+    s.close()

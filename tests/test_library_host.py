@@ -1,0 +1,230 @@
+"""Host side of the library against the oracle: registry, trace, classification and schedule must be
+bit-exact (compared as exported blobs); error paths return codes, never crash.  No GPU needed."""
+import ctypes
+import os
+import re
+import struct
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+import seeded_inputs as si
+from conftest import MACHINE
+from oracle import policy, trace, validate
+from paper_2609_06172_b200 import binding as tb
+from paper_2609_06172_b200 import build as tbuild
+from paper_2609_06172_b200.session import Session
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    tbuild.build()
+
+
+def pack_trace(ops):
+    out = []
+    for o in ops:
+        out.append(struct.pack("<IQiIQQI", o.step, o.site, o.layer, o.kind, o.flops, o.hbm, len(o.acc)))
+        out += [struct.pack("<IIQ", *a) for a in o.acc]
+    return b"".join(out)
+
+
+def oracle_blobs(lay, bits=7, expert_counts=None, budget=None):
+    ops, steps = trace.run_trace(lay, expert_counts=expert_counts)
+    pl = policy.plan(lay.tensors, ops, steps, policy.Machine(**MACHINE), budget or lay.budget, bits)
+    return ops, steps, pl.blobs()
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(os.path.dirname(tbuild.INCLUDE), "include", "tgp.h")).read()
+    declared = set(re.findall(r"\b(tgp_[a-z_0-9]+)\s*\(", hdr))
+    lib = ctypes.CDLL(tbuild.LIB)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert declared == set(tb.exported_symbols())
+
+
+@pytest.mark.parametrize("c", [1, 2, 3, 4])
+def test_plan_bit_exact_dense_configs(c):
+    lay = si.build_layout(si.CONFIGS[c])
+    s = Session(lay, MACHINE)
+    got = s.plan()
+    ops, steps, want = oracle_blobs(lay)
+    assert s.ctx.trace_export() == pack_trace(ops)
+    for k in want:
+        assert got[k] == want[k], k
+    s.close()
+
+
+def synthetic_expert_counts(cfg, rng):
+    """Top-2 routing counts with a Zipf-like popularity (counts only; no forward pass involved)."""
+    p = np.array([r ** -1.2 for r in range(1, cfg.E + 1)])
+    p /= p.sum()
+    out = np.zeros((1 + cfg.T, cfg.L, cfg.E), dtype=np.uint32)
+    for k in range(1 + cfg.T):
+        M = cfg.B * (cfg.S if k == 0 else 1)
+        for l in range(cfg.L):
+            for _ in range(M):
+                e = rng.choice(cfg.E, size=2, replace=False, p=p)
+                out[k, l, e] += 1
+    return out
+
+
+def test_plan_bit_exact_moe_reduced_and_full_shape():
+    rng = np.random.default_rng(5)
+    small = replace(si.CONFIGS[5], L=3, B=4, S=8, T=6, TK=4)
+    lay = si.build_layout(small, budget=3 << 30)
+    ec = synthetic_expert_counts(small, rng)
+    s = Session(lay, MACHINE, router_bias=si.router_bias(small))
+    got = s.plan(expert_counts=ec)
+    ops, steps, want = oracle_blobs(lay, expert_counts=ec)
+    assert s.ctx.trace_export() == pack_trace(ops)
+    for k in want:
+        assert got[k] == want[k], k
+    validate.check(lay.tensors, ops, steps, lay.budget, got)
+    s.close()
+    # full config-5 shape and budget, every expert hit in every step (the worst case for the link)
+    cfg = si.CONFIGS[5]
+    lay = si.build_layout(cfg)
+    ec = np.zeros((1 + cfg.T, cfg.L, cfg.E), dtype=np.uint32)
+    ec[0] = cfg.B * cfg.S * 2 // cfg.E
+    ec[1:] = cfg.B * 2 // cfg.E
+    s = Session(lay, MACHINE, router_bias=si.router_bias(cfg))
+    got = s.plan(expert_counts=ec)
+    ops, steps, want = oracle_blobs(lay, expert_counts=ec)
+    for k in want:
+        assert got[k] == want[k], k
+    s.close()
+
+
+@pytest.mark.parametrize("bits", [0, tb.BIT_A, tb.BIT_P, tb.BIT_A | tb.BIT_P, tb.BIT_ZC, 7])
+def test_plan_bit_exact_under_ablation_bits(bits):
+    lay = si.build_layout(si.CONFIGS[1])
+    s = Session(lay, MACHINE)
+    try:
+        got = s.plan(bits=bits)
+    except tb.TgpError as e:
+        assert e.code == tb.E_BUDGET_TOO_SMALL
+        with pytest.raises(policy.PlanError):
+            oracle_blobs(lay, bits)
+        return
+    ops, steps, want = oracle_blobs(lay, bits)
+    for k in want:
+        assert got[k] == want[k], (bits, k)
+    validate.check(lay.tensors, ops, steps, lay.budget, got)
+    s.close()
+
+
+def test_library_plan_passes_the_validator_config_2():
+    lay = si.build_layout(si.CONFIGS[2])
+    s = Session(lay, MACHINE)
+    got = s.plan(T=8)
+    ops, steps = trace.run_trace(lay, n_decode=8)
+    validate.check(lay.tensors, ops, steps, lay.budget, got)
+    s.close()
+
+
+def test_schedule_is_independent_of_the_pool_address():
+    lay = si.build_layout(si.CONFIGS[1])
+    a = Session(lay, MACHINE, pool_base=1 << 30)
+    b = Session(lay, MACHINE, pool_base=(7 << 40) + 512 * 12345)
+    assert a.plan() == b.plan()
+    assert a.ctx.tensor_identity(17) == b.ctx.tensor_identity(17)
+    a.close(), b.close()
+
+
+def test_trace_recorded_through_the_c_calls_equals_model_trace():
+    lay = si.build_layout(si.CONFIGS[1])
+    ops, steps = trace.run_trace(lay, n_decode=2)
+    s = Session(lay, MACHINE)
+    s.ctx.trace_begin()
+    for (kind, first, count) in steps:
+        s.ctx.trace_step(kind)
+        for o in ops[first:first + count]:
+            s.ctx.trace_op(o.site, o.layer, o.kind, o.flops, o.hbm, o.acc)
+    s.ctx.trace_end()
+    s.ctx.plan()
+    manual = s.ctx.plan_blobs()
+    assert s.plan(T=2) == manual
+    s.close()
+
+
+def test_registry_lookup_identity_and_errors():
+    ctx = tb.Ctx(**MACHINE)
+    buf = np.zeros(1 << 16, dtype=np.uint8)
+    base = (buf.ctypes.data + 511) // 512 * 512
+    pool = ctx.pool_register(base, 32768, tb.POOL_PLAIN)
+    a = ctx.tensor_register(pool, 0, 1000, 0xABC, 0, 2, tb.T_READONLY)
+    b = ctx.tensor_register(pool, 4096, 2048, 0xABC, 0, 3, tb.T_READONLY)
+    c = ctx.tensor_register(pool, 1024, 512, 0xDEF, 1, 13, tb.T_MUTABLE)       # out of address order
+    assert ctx.tensor_lookup(base + 999) == (a, 999)
+    assert ctx.tensor_lookup(base + 4096 + 7) == (b, 7)
+    assert ctx.tensor_lookup(base + 1024) == (c, 0)
+    assert ctx.tensor_identity(a) == (0xABC, 0) and ctx.tensor_identity(b) == (0xABC, 1) and ctx.tensor_identity(c) == (0xDEF, 0)
+    for args, code in [((pool, 512, 1024, 1, 0, 2, tb.T_READONLY), tb.E_OVERLAP),        # into a and c
+                       ((pool, 3584, 1024, 1, 0, 2, tb.T_READONLY), tb.E_OVERLAP),       # into b
+                       ((pool, 32768 - 512, 1024, 1, 0, 2, tb.T_READONLY), tb.E_RANGE),
+                       ((pool, 100, 8, 1, 0, 2, tb.T_READONLY), tb.E_INVAL),             # unaligned
+                       ((pool + 5, 0, 8, 1, 0, 2, tb.T_READONLY), tb.E_INVAL),
+                       ((pool, 8192, 8, 1, 0, 2, 3), tb.E_INVAL)]:
+        with pytest.raises(tb.TgpError) as ei:
+            ctx.tensor_register(*args)
+        assert ei.value.code == code
+    for addr in (base + 1000, base + 3000, base - 1, base + 40000):
+        with pytest.raises(tb.TgpError) as ei:
+            ctx.tensor_lookup(addr)
+        assert ei.value.code == tb.E_RANGE
+    with pytest.raises(tb.TgpError) as ei:
+        ctx.pool_register(base + 512, 1024, tb.POOL_PLAIN)
+    assert ei.value.code == tb.E_OVERLAP
+    # trace errors
+    with pytest.raises(tb.TgpError):
+        ctx.plan()                                               # nothing traced
+    ctx.trace_begin()
+    ctx.trace_step(tb.PREFILL)
+    for acc, code in [([(99, tb.R, 8)], tb.E_UNKNOWN_TENSOR), ([(a, tb.W, 8)], tb.E_INVAL), ([(a, tb.R, 8), (a, tb.R, 8)], tb.E_INVAL)]:
+        with pytest.raises(tb.TgpError) as ei:
+            ctx.trace_op(1, 0, 2, 10, 10, acc)
+        assert ei.value.code == code
+    ctx.trace_op(1, 0, 2, 10, 10, [(a, tb.R, 1000)])
+    ctx.trace_end()
+    with pytest.raises(tb.TgpError) as ei:
+        ctx.plan()                                               # no budget
+    assert ei.value.code == tb.E_STATE
+    ctx.set_budget(1024)
+    with pytest.raises(tb.TgpError) as ei:
+        ctx.plan()
+    assert ei.value.code == tb.E_BUDGET_TOO_SMALL
+    with pytest.raises(tb.TgpError) as ei:
+        ctx.plan_export(tb.X_COMMANDS)
+    assert ei.value.code == tb.E_NO_PLAN
+    ctx.set_budget(4096)
+    ctx.plan()
+    assert len(ctx.plan_export(tb.X_COMMANDS)) == 45
+    with pytest.raises(tb.TgpError):
+        ctx.tensor_register(pool, 16384, 512, 1, 0, 2, tb.T_READONLY)     # registry frozen after tracing
+    # stepping without a device binding is a state error, not a crash
+    with pytest.raises(tb.TgpError) as ei:
+        ctx.step(tb.PREFILL, np.zeros(4, np.int32), 1, 4, 1 << 20, None, None, None)
+    assert ei.value.code == tb.E_STATE
+    ctx.close()
+
+
+def test_model_bind_rejects_bad_shapes_and_roles():
+    lay = si.build_layout(si.CONFIGS[1])
+    s = Session(lay, MACHINE)
+    bad = tb.ModelCfg(4, 256, 4, 3, 64, 1024, 4096, 0, 0, 1, 48, 16, 10000.0, 1e-5)          # Hq % Hkv != 0
+    with pytest.raises(tb.TgpError):
+        s.ctx.model_bind(bad, s.roles)
+    long_ctx = tb.ModelCfg(4, 256, 4, 4, 64, 1024, 4096, 0, 0, 1, 65 * 16, 16, 10000.0, 1e-5)   # 65 tiles > 64
+    with pytest.raises(tb.TgpError) as ei:
+        s.ctx.model_bind(long_ctx, s.roles)
+    assert ei.value.code == tb.E_TOO_LARGE
+    with pytest.raises(tb.TgpError) as ei:
+        s.ctx.model_bind(s.cfg, s.roles + [s.roles[0]])
+    assert ei.value.code == tb.E_INVAL
+    with pytest.raises(tb.TgpError) as ei:
+        s.ctx.model_trace(40, 16)                                # S + T beyond max_len
+    assert ei.value.code == tb.E_INVAL
+    s.close()
