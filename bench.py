@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the hot path: tokens/s at a fixed device budget.
+
+One "step" is one whole pass of the path over one batch: prefill of the prompt, then every decode step,
+from a cold arena, with the weight/KV pool in pinned host memory and a device budget of half the weights
+(the Llama-1B-shaped configuration, 2x oversubscribed).  `value` is tokens/s with the device feeding its own
+argmax back (no host round trip per token); `e2e` puts the host in the loop: tokens come from pinned host
+memory every step and each step's argmax (and the final logits) are read back.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--config 2]
+
+With N > 1 (torchrun) every rank runs an independent replica on its own GPU (the path does not shard:
+no collective on the data path); the line reports the whole-job rate over the slowest rank.
+`--impl reference` times the CPU oracle on the host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import struct
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+import seeded_inputs as si  # noqa: E402
+
+# roofline constants frozen for the planner (integers): sustained bf16 peak and HBM copy bandwidth measured on
+# this machine's B200, pinned host-link bandwidth at 256 MiB measured by this build (profiles/host_link.md)
+MACHINE = dict(peak_flops=1362800000000000, hbm_Bps=6541100000000, h2d_Bps=55570000000, d2h_Bps=56900000000)
+OP_NAMES = ["embed", "rmsnorm", "gemm", "rope_kv", "attn", "swiglu", "router", "argmax"]
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return dict(hbm_gbs=j["hbm_gbs"], bf16_tflops=j["bf16_tflops"], bf16_sustained=j.get("bf16_tflops_sustained"), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+        "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, index):
+        self.rows, self.proc, self.index = [], None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        sm = [float(r[0]) for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 7 and r[1].replace(".", "").isdigit()]
+        reasons = set()
+        for r in self.rows:
+            if len(r) >= 7:
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def parse_trace(blob):
+    """-> list of (step, site, layer, kind, flops, hbm, [(tensor, mode, touched)])"""
+    ops, off = [], 0
+    head = struct.Struct("<IQiIQQI")
+    while off < len(blob):
+        step, site, layer, kind, flops, hbm, n = head.unpack_from(blob, off)
+        off += head.size
+        acc = [struct.unpack_from("<IIQ", blob, off + 16 * k) for k in range(n)]
+        off += 16 * n
+        ops.append((step, site, layer, kind, flops, hbm, acc))
+    return ops
+
+
+def oracle_weights_from_pool(lay, pool_u8):
+    """bf16 bit matrices per logical weight, re-joined from the pool's blocks (input data for the oracle)."""
+    u16 = pool_u8.view(np.uint16)
+    out = {}
+    for (kind, layer, expert, rows, cols) in si.weight_matrices(lay.cfg):
+        parts = [u16[t.pool_off // 2: t.pool_off // 2 + t.rows * t.cols].reshape(t.rows, t.cols) for t in lay.blocks(kind, layer, expert)]
+        out[(kind, layer, expert)] = np.concatenate(parts, axis=0) if len(parts) > 1 else parts[0]
+    return out
+
+
+def time_oracle(lay, weights, sample_S, sample_T, reps=1):
+    """Oracle (float32 accumulate, numpy) on a bounded sample: prefill of sample_S prompt tokens + sample_T decode steps."""
+    from oracle.forward import OracleModel
+    cfg = lay.cfg
+    om = OracleModel(cfg, weights, si.router_bias(cfg) if cfg.E else None, dtype=np.float32)
+    prompt = si.prompt_tokens(cfg)[:, :sample_S]
+    best = None
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        om.generate(prompt, sample_T)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    return cfg.B * (sample_S + sample_T) / best, best
+
+
+def run_reference(args, cfg, lay):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    pool = np.empty(lay.pool_bytes, dtype=np.uint8)
+    si.fill_pool(lay, pool)
+    W = oracle_weights_from_pool(lay, pool)
+    sS, sT = min(cfg.S, 128), min(cfg.T, 4)
+    cores = len(os.sched_getaffinity(0))
+    for _ in range(args.warmup):
+        time_oracle(lay, W, 16, 1)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time_oracle(lay, W, sS, sT)
+    dt = time.perf_counter() - t0
+    val = cfg.B * (sS + sT) * args.steps / dt
+    sample = f"prefill of the first {sS} prompt tokens + {sT} decode steps per step (full widths and depth)"
+    print(json.dumps({"impl": "reference", "metric": "tokens_per_s", "value": val, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
+                      "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+                      "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": workload_name(cfg, lay), "sample": sample},
+                      "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+                      "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def workload_name(cfg, lay):
+    return (f"{cfg.name}: L={cfg.L} d={cfg.d} Hq/Hkv={cfg.Hq}/{cfg.Hkv} F={cfg.F} V={cfg.V} B={cfg.B} prompt={cfg.S} decode={cfg.T} "
+            f"pool={lay.pool_bytes} budget={lay.budget}")
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="tgp")
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--decode", type=int, default=None, help="decode steps per pass (default: the configuration's)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-uvm", action="store_true", help="skip the demand-paged managed-memory baseline")
+    args = ap.parse_args()
+    cfg = si.CONFIGS[args.config]
+    if args.decode is not None:
+        from dataclasses import replace
+        cfg = replace(cfg, T=args.decode)
+    lay = si.build_layout(cfg)
+    if args.impl == "reference":
+        return run_reference(args, cfg, lay)
+
+    import torch
+    from paper_2609_06172_b200 import binding as tb
+    from paper_2609_06172_b200.runner import Runner, pinned_pool
+    from paper_2609_06172_b200.session import Session
+    tb.lib()                                                     # fails loudly when the CUDA library is missing
+    rank, world, local = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    dev = torch.device(f"cuda:{local}")
+    torch.cuda.set_device(dev)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    pool = pinned_pool(lay.pool_bytes)
+    si.fill_pool(lay, pool.numpy())
+    s = Session(lay, MACHINE, pool_base=pool.data_ptr(), pool_flags=tb.POOL_PINNED)
+    blobs = s.plan()
+    totals = np.frombuffer(blobs["totals"], dtype="<u8").reshape(-1, 4)
+    ops = parse_trace(s.ctx.trace_export())
+    r = Runner(s, cfg.B * cfg.S, device=str(dev))
+    prompt_pinned = torch.from_numpy(si.prompt_tokens(cfg)).pin_memory()
+    tok_pinned = torch.empty((cfg.B, 1), dtype=torch.int32).pin_memory()
+    logits_host = torch.empty((cfg.B, cfg.V), dtype=torch.float32).pin_memory()
+    T = cfg.T
+
+    def one_pass(e2e=False):
+        r.reset()
+        r.step(tb.PREFILL, prompt_pinned.numpy(), cfg.S)
+        for t in range(T):
+            if e2e:
+                with torch.cuda.stream(r.compute):
+                    tok_pinned.copy_(r.argmax.view(cfg.B, 1), non_blocking=True)
+                r.compute.synchronize()
+                r.step(tb.DECODE, tok_pinned.numpy(), 1)
+            else:
+                r.step(tb.DECODE, None, 1)
+        if e2e:
+            with torch.cuda.stream(r.compute):
+                logits_host.copy_(r.logits, non_blocking=True)
+                tok_pinned.copy_(r.argmax.view(cfg.B, 1), non_blocking=True)
+            r.compute.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def timed(n, e2e):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record(r.compute)
+        for _ in range(n):
+            one_pass(e2e)
+        ev1.record(r.compute)
+        r.sync()
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if dist is not None:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(args.warmup):
+        one_pass(False)
+    r.sync()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ms = timed(args.steps, False)
+    clocks = sampler.stop() if rank == 0 else None
+    one_pass(True)
+    ms_e2e = timed(args.steps, True)
+    tokens_per_pass = cfg.B * (cfg.S + T)
+    value = world * tokens_per_pass * args.steps / (ms * 1e-3)
+    e2e_value = world * tokens_per_pass * args.steps / (ms_e2e * 1e-3)
+
+    # ---- per-phase timing, launches and the live per-kernel roofline: one extra pass with op timestamps -----------
+    r.reset()
+    s.ctx.set_op_timing(True)
+    kind_ms, kind_bytes, kind_flops, kind_n = {}, {}, {}, {}
+    launches = 0
+    step_ms = []
+    for k in range(1 + T):
+        st = r.step(tb.PREFILL if k == 0 else tb.DECODE, prompt_pinned.numpy() if k == 0 else None, cfg.S if k == 0 else 1, want_stats=True)
+        first, tms = s.ctx.op_times()
+        launches += st.n_launches
+        step_ms.append(st.step_ms)
+        phase = "prefill" if k == 0 else "decode"
+        for j, t in enumerate(tms):
+            o = ops[first + j]
+            key = (phase, OP_NAMES[o[3]])
+            kind_ms[key] = kind_ms.get(key, 0.0) + float(t)
+            kind_bytes[key] = kind_bytes.get(key, 0) + o[5]
+            kind_flops[key] = kind_flops.get(key, 0) + o[4]
+            kind_n[key] = kind_n.get(key, 0) + 1
+    s.ctx.set_op_timing(False)
+    r.sync()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    peaks = measured_peaks()
+    # dominant kernel by device time in the pass
+    dom = max(kind_ms, key=lambda k: kind_ms[k])
+    if dom[1] == "gemm" and dom[0] == "prefill":
+        ach = kind_flops[dom] / (kind_ms[dom] * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"]}
+    else:
+        ach = kind_bytes[dom] / (kind_ms[dom] * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"]}
+    roof.update({"kernel": f"{dom[1]} ({dom[0]})", "launches": kind_n[dom], "avg_us": kind_ms[dom] / kind_n[dom] * 1e3,
+                 "algorithmic_per_launch": (kind_flops[dom] if roof["bound"] == "tensor" else kind_bytes[dom]) / kind_n[dom],
+                 "peak_source": peaks["source"], "traffic": None})
+    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(prof):
+        roof["traffic"] = json.load(open(prof)).get(f"{dom[1]}_{dom[0]}_cfg{args.config}")
+    # step roofline: slowest of compute, HBM and link for the whole pass, (i) with the plan's bytes, (ii) with the lower bound
+    F = sum(o[4] for o in ops)
+    H = sum(o[5] for o in ops) + int(totals[:, 0].sum())
+    L_plan, L_d2h = int(totals[:, 0].sum() + totals[:, 2].sum()), int(totals[:, 1].sum())
+    step_of = {}
+    for o in ops:
+        for (t, mode, touched) in o[6]:
+            step_of.setdefault(o[0], {})[t] = lay.tensors[t].size if touched * 2 >= lay.tensors[t].size else touched
+    L_lb = sum(max(0, sum(d.values()) - (lay.budget if k else 0)) for k, d in step_of.items())
+    t_roof = max(F / MACHINE["peak_flops"], H / MACHINE["hbm_Bps"], L_plan / MACHINE["h2d_Bps"], L_d2h / MACHINE["d2h_Bps"])
+    t_lb = max(F / MACHINE["peak_flops"], H / MACHINE["hbm_Bps"], L_lb / MACHINE["h2d_Bps"])
+    t_meas = ms * 1e-3 / args.steps
+    step_roof = {"bound": "link", "t_roof_s_plan_bytes": t_roof, "t_roof_s_lower_bound": t_lb, "t_measured_s": t_meas,
+                 "frac_plan_bytes": t_roof / t_meas, "frac_lower_bound": t_lb / t_meas,
+                 "link_gbs_achieved": L_plan / t_meas / 1e9, "link_gbs_peak": MACHINE["h2d_Bps"] / 1e9,
+                 "h2d_bytes": int(totals[:, 0].sum()), "d2h_bytes": L_d2h, "zero_copy_bytes": int(totals[:, 2].sum()),
+                 "flops": F, "hbm_bytes": H}
+    out = {"metric": "tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+           "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+           "data": "synthetic", "config": {"workload": workload_name(cfg, lay), "l2": "inputs larger than L2: every decode step streams the 2.2 GB pool",
+                                           "step": "prefill + all decode steps from a cold arena", "tokens_per_step": tokens_per_pass,
+                                           "parallelism": "replicas" if world > 1 else "single"},
+           "prefill_tok_s": cfg.B * cfg.S / (step_ms[0] * 1e-3), "decode_tok_s": cfg.B * T / (sum(step_ms[1:]) * 1e-3) if T else None,
+           "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": int(totals[:, 0].sum()) + cfg.B * (cfg.S + T) * 4,
+                   "d2h_bytes_per_step": L_d2h + cfg.B * (T + 1) * 4 + cfg.B * cfg.V * 4},
+           "gpu_launches": launches * args.steps, "clocks": clocks, "roofline": roof, "step_roofline": step_roof,
+           "kernels": {f"{k[0]}:{k[1]}": {"ms": round(v, 3), "launches": kind_n[k], "GBps": round(kind_bytes[k] / (v * 1e-3) / 1e9, 1),
+                                           "TFLOPs": round(kind_flops[k] / (v * 1e-3) / 1e12, 2)} for k, v in sorted(kind_ms.items())}}
+    if not args.no_uvm:
+        try:
+            from paper_2609_06172_b200 import uvm_baseline
+            out["uvm_demand_paged"] = uvm_baseline.run(cfg, lay, MACHINE, dev)
+        except ImportError:
+            out["uvm_demand_paged"] = "not run: baseline module not built yet"
+        except Exception as ex:  # the baseline is reported, never fatal
+            out["uvm_demand_paged"] = f"not run: {type(ex).__name__}: {ex}"
+    if not args.no_cpu_baseline:
+        W = oracle_weights_from_pool(lay, pool.numpy())
+        sS, sT = min(cfg.S, 128), min(cfg.T, 4)
+        val, dt = time_oracle(lay, W, sS, sT)
+        out["cpu_baseline"] = {"value": val, "unit": "tokens/s", "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
+                               "sample": f"prefill of the first {sS} prompt tokens + {sT} decode steps, float32 accumulate ({dt:.1f} s)"}
+    print(json.dumps(out))
+    s.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

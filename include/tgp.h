@@ -183,6 +183,14 @@ int  tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_host, uint
               float *logits_dev, int32_t *argmax_dev, void *compute_stream, void *copy_stream,
               tgp_step_stats *stats);
 
+/* Per-op timestamps (Section IV-D "Runtime Monitor": lightweight timestamping).  While enabled, tgp_step()
+ * brackets every op with CUDA events on the compute stream (after the op's copies have been waited for, so
+ * the figure is kernel time, not stall time).  tgp_op_times() waits for the last timed step and returns one
+ * duration in ms per op of that step, ops [*first_op, *first_op + *n_ops) of the trace; ms == NULL asks
+ * for the count only. */
+int  tgp_set_op_timing(tgp_ctx *ctx, int enable);
+int  tgp_op_times(tgp_ctx *ctx, float *ms, uint32_t capacity, uint32_t *first_op, uint32_t *n_ops);
+
 /* ---- single kernels (device pointers; used by the model step, exported for parity tests and timing) ---- */
 /* x[m, :] = fp32(table[tok[m], :]);  table bf16 [V, d] (device or mapped host), tok int32 [M]. */
 int  tgp_k_embed(const void *table, const int32_t *tok_dev, float *x_dev, uint32_t M, uint32_t d, void *stream);

@@ -77,6 +77,8 @@ _SIGS = {
     "tgp_model_bind": [_P, C.POINTER(ModelCfg), C.POINTER(RoleEntry), _U32, _P, _P, _U64, _U32],
     "tgp_run_reset": [_P],
     "tgp_step": [_P, _U32, _P, _U32, _U32, _P, _P, _P, _P, C.POINTER(StepStats)],
+    "tgp_set_op_timing": [_P, C.c_int],
+    "tgp_op_times": [_P, C.POINTER(C.c_float), _U32, C.POINTER(_U32), C.POINTER(_U32)],
     "tgp_k_embed": [_P, _P, _P, _U32, _U32, _P],
     "tgp_k_rmsnorm": [_P, _U32, _P, _P, _U32, _U32, C.c_float, _P],
     "tgp_k_gemm": [_P, _P, _P, _U32, _U32, _U32, _U32, _U32, C.c_int, _P],
@@ -239,6 +241,18 @@ class Ctx:
         self._ck(lib().tgp_step(self._h, kind, _ptr(tokens_host), B, q_len, _ptr(logits), _ptr(argmax), _ptr(compute_stream),
                                 _ptr(copy_stream), C.byref(st) if st is not None else None), "tgp_step")
         return st
+
+
+    def set_op_timing(self, enable):
+        self._ck(lib().tgp_set_op_timing(self._h, int(enable)), "tgp_set_op_timing")
+
+    def op_times(self):
+        """(first op index, per-op milliseconds) of the last step that ran with op timing on."""
+        first, n = _U32(), _U32()
+        self._ck(lib().tgp_op_times(self._h, None, 0, C.byref(first), C.byref(n)), "tgp_op_times")
+        ms = (C.c_float * max(1, n.value))()
+        self._ck(lib().tgp_op_times(self._h, ms, n.value, C.byref(first), C.byref(n)), "tgp_op_times")
+        return first.value, np.frombuffer(ms, dtype=np.float32, count=n.value).copy()
 
 
 def model_workspace_bytes(cfg: ModelCfg, max_tokens: int) -> int:

@@ -38,6 +38,10 @@ struct TgpEngine {
     uint32_t next_step = 0, pos = 0;
     const int32_t *tok_src = nullptr;
     int device = -1;
+    // optional per-op timestamps (Section IV-D "Runtime Monitor": lightweight timestamping of kernels)
+    bool op_timing = false;
+    std::vector<cudaEvent_t> ta, tb_;
+    uint32_t timed_op0 = 0, timed_nops = 0;
     // managed-hints variant
     size_t hinted_upto = 0;
     bool advised = false;
@@ -86,6 +90,8 @@ void tgp_engine_free(tgp_ctx *ctx) {
     cudaDeviceSynchronize();
     for (cudaEvent_t ev : e->done_ev) if (ev) cudaEventDestroy(ev);
     for (cudaEvent_t ev : e->copied_ev) if (ev) cudaEventDestroy(ev);
+    for (cudaEvent_t ev : e->ta) if (ev) cudaEventDestroy(ev);
+    for (cudaEvent_t ev : e->tb_) if (ev) cudaEventDestroy(ev);
     if (e->wb_ev) cudaEventDestroy(e->wb_ev);
     if (e->t0) cudaEventDestroy(e->t0);
     if (e->t1) cudaEventDestroy(e->t1);
@@ -295,6 +301,12 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             CU(ctx, cudaStreamWaitEvent(cs, ev, 0));
         }
         if (ctx->variant == TGP_VAR_MANAGED_HINTS && (rc = hint_ahead(ctx, i, st.op0 + st.nops, cp))) return rc;
+        const uint32_t ti = i - st.op0;
+        if (e->op_timing) {
+            if (e->ta.size() <= ti) { e->ta.resize(ti + 1, nullptr); e->tb_.resize(ti + 1, nullptr); }
+            if (!e->ta[ti]) { CU(ctx, cudaEventCreate(&e->ta[ti])); CU(ctx, cudaEventCreate(&e->tb_[ti])); }
+            CU(ctx, cudaEventRecord(e->ta[ti], cs));
+        }
         rc = TGP_OK;
         switch (o.kind) {
         case TGP_OP_EMBED:
@@ -352,6 +364,7 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             return tgp_fail(ctx, TGP_E_MISMATCH, "op kind the bound model cannot run");
         }
         if (rc) return tgp_fail(ctx, rc, "kernel launch failed");
+        if (e->op_timing) CU(ctx, cudaEventRecord(e->tb_[ti], cs));
         if (ring) {
             if (ctx->plan.op_is_wait_target[i]) {
                 cudaEvent_t ev;
@@ -363,6 +376,7 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
     }
     e->pos += q_len;
     e->next_step++;
+    if (e->op_timing) { e->timed_op0 = st.op0; e->timed_nops = st.nops; } else e->timed_nops = 0;
     if (stats) {
         CU(ctx, cudaEventRecord(e->t1, cs));
         CU(ctx, cudaEventSynchronize(e->t1));
@@ -371,6 +385,26 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
         stats->h2d_bytes = ring ? tot[0] : 0; stats->d2h_bytes = ring ? tot[1] : 0; stats->zc_bytes = tot[2];
         stats->n_cmds = n_cmds; stats->n_launches = (uint32_t)(tgpk_launches - launches0); stats->n_mismatch = 0;
         CU(ctx, cudaEventElapsedTime(&stats->step_ms, e->t0, e->t1));
+    }
+    return TGP_OK;
+}
+
+extern "C" int tgp_set_op_timing(tgp_ctx *ctx, int enable) {
+    if (!ctx || !ctx->eng) return TGP_E_STATE;
+    ctx->eng->op_timing = enable != 0;
+    return TGP_OK;
+}
+
+extern "C" int tgp_op_times(tgp_ctx *ctx, float *ms, uint32_t capacity, uint32_t *first_op, uint32_t *n_ops) {
+    if (!ctx || !ctx->eng || !n_ops) return TGP_E_STATE;
+    TgpEngine *e = ctx->eng;
+    *n_ops = e->timed_nops;
+    if (first_op) *first_op = e->timed_op0;
+    if (!ms) return TGP_OK;
+    if (capacity < e->timed_nops) return TGP_E_INVAL;
+    for (uint32_t i = 0; i < e->timed_nops; ++i) {
+        CU(ctx, cudaEventSynchronize(e->tb_[i]));
+        CU(ctx, cudaEventElapsedTime(&ms[i], e->ta[i], e->tb_[i]));
     }
     return TGP_OK;
 }
