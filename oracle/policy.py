@@ -27,8 +27,12 @@ Steps, in order (notation: P = peak flop/s, Bh = HBM bytes/s, Bl = host-link byt
    live_i = aligned bytes of all non-ZC episodes covering op i; ring_min = 2 * max_i live_i;
    error if ring_min > budget.  pin_cap = budget - ring_min.
 5. pins (A bit): candidates score > 0, non-ZC, by density score/size descending (exact cross
-   products), tie -> lower id; greedy with skip while the aligned size fits in pin_cap.
-   Pins sit at [0, used); the ring is [used, budget).
+   products), tie -> lower id.  Groups of equal density are taken in turn: a group that fits is
+   pinned whole; one that does not has its share of pinned bytes spread evenly along the id order
+   by integer error diffusion (err += a*cap; pin iff err >= a*total; then err -= a*total), followed
+   by a greedy fill with skip.  Spreading keeps the link demand of the streamed rest uniform over a
+   step instead of leaving the copy engine idle while compute walks a pinned prefix of layers.
+   Pins sit at [0, used) in the order they were chosen; the ring is [used, budget).
 6. schedule: walk ops in order, accesses in list order.
      pinned tensor, first access: LOAD (H2D into its slot), or ALLOC if MUTABLE and the access is W.
      ring tensor, episode start: FIFO bump allocation (wrap to the ring base when the tail does
@@ -193,11 +197,33 @@ def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A |
                 return -1 if lhs > rhs else 1
             return -1 if a < b else (1 if a > b else 0)
 
-        for t in sorted(cands, key=functools.cmp_to_key(cmp)):
-            a = alignup(tensors[t].size)
-            if used + a <= pin_cap:
-                pinned_off[t] = used
-                used += a
+        order = sorted(cands, key=functools.cmp_to_key(cmp))
+        g0 = 0
+        while g0 < len(order):
+            # group of equal density (exact cross products against the group's first tensor)
+            g1 = g0 + 1
+            while g1 < len(order) and score[order[g1]] * tensors[order[g0]].size == score[order[g0]] * tensors[order[g1]].size:
+                g1 += 1
+            group = order[g0:g1]
+            g0 = g1
+            cap_left = pin_cap - used
+            total = sum(alignup(tensors[t].size) for t in group)
+            if total > cap_left:
+                # not all fit: spread the pinned bytes evenly along the id (= first-use) order by error
+                # diffusion, so that the link demand of the rest is uniform over a step
+                err = 0
+                for t in group:
+                    a = alignup(tensors[t].size)
+                    err += a * cap_left
+                    if err >= a * total:
+                        err -= a * total
+                        pinned_off[t] = used
+                        used += a
+            for t in group:                                   # everything that fits / greedy fill, with skip
+                a = alignup(tensors[t].size)
+                if t not in pinned_off and used + a <= pin_cap:
+                    pinned_off[t] = used
+                    used += a
     ring_base, ring_size = used, budget - used
     pins = sorted(pinned_off.items())
     # 6: schedule

@@ -302,9 +302,28 @@ int tgp_plan(tgp_ctx *ctx) {
             u128 l = (u128)pl.score[a] * ten[b].size, r = (u128)pl.score[b] * ten[a].size;
             return l != r ? l > r : a < b;
         });
-        for (uint32_t t : cand) {
-            uint64_t a = alignup(ten[t].size);
-            if (used + a <= pin_cap) { pin_off[t] = (int64_t)used; used += a; }
+        for (size_t g0 = 0; g0 < cand.size();) {
+            // group of equal density
+            size_t g1 = g0 + 1;
+            while (g1 < cand.size() && (u128)pl.score[cand[g1]] * ten[cand[g0]].size == (u128)pl.score[cand[g0]] * ten[cand[g1]].size) ++g1;
+            const uint64_t cap_left = pin_cap - used;
+            uint64_t total = 0;
+            for (size_t k = g0; k < g1; ++k) total += alignup(ten[cand[k]].size);
+            if (total > cap_left) {
+                // the group does not fit: spread its pinned bytes evenly along the id order (error diffusion),
+                // so the link demand of the streamed rest stays uniform over a step
+                u128 err = 0;
+                for (size_t k = g0; k < g1; ++k) {
+                    const uint64_t a = alignup(ten[cand[k]].size);
+                    err += (u128)a * cap_left;
+                    if (err >= (u128)a * total) { err -= (u128)a * total; pin_off[cand[k]] = (int64_t)used; used += a; }
+                }
+            }
+            for (size_t k = g0; k < g1; ++k) {               // whole group if it fits / greedy fill with skip
+                const uint64_t a = alignup(ten[cand[k]].size);
+                if (pin_off[cand[k]] < 0 && used + a <= pin_cap) { pin_off[cand[k]] = (int64_t)used; used += a; }
+            }
+            g0 = g1;
         }
     }
     for (size_t t = 0; t < T; ++t) if (pin_off[t] >= 0) pl.pins.push_back({(uint32_t)t, (uint64_t)pin_off[t]});

@@ -67,48 +67,59 @@ __global__ void rmsnorm_kernel(const float *__restrict__ x, uint32_t ldx, const 
     }
 }
 
-// ---- GEMV / skinny GEMM: weight streaming, one warp per R output rows, MT activation rows -------
+// ---- GEMV / skinny GEMM (M <= 8 activation rows): pure weight streaming --------------------------------
+// One block owns R output rows; its 8 warps split K, so every thread has R independent 16-byte loads in
+// flight per k-chunk and a [n, K] block of any aspect ratio fills the machine (n/R blocks).  Partial sums
+// meet in shared memory in a fixed order: results are deterministic run to run.
 template <int MT, int R>
 __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                    uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
-    const uint32_t lane = threadIdx.x & 31;
-    const uint32_t warps = (gridDim.x * blockDim.x) >> 5;
-    for (uint32_t row0 = ((blockIdx.x * blockDim.x + threadIdx.x) >> 5) * R; row0 < n; row0 += warps * R) {
-        float acc[R][MT];
+    __shared__ float part[8][R * MT];
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t row0 = blockIdx.x * R;
+    float acc[R][MT];
 #pragma unroll
-        for (int r = 0; r < R; ++r)
+    for (int r = 0; r < R; ++r)
 #pragma unroll
-            for (int m = 0; m < MT; ++m) acc[r][m] = 0.f;
-        for (uint32_t k = lane * 8; k < K; k += 256) {
-            uint4 wv[R];
+        for (int m = 0; m < MT; ++m) acc[r][m] = 0.f;
+    const bf16 *wrow[R];
 #pragma unroll
-            for (int r = 0; r < R; ++r)
-                wv[r] = (row0 + r < n) ? __ldcs(reinterpret_cast<const uint4 *>(W + (size_t)(row0 + r) * K + k)) : make_uint4(0, 0, 0, 0);
-            float wf[R][8];
+    for (int r = 0; r < R; ++r) wrow[r] = W + (size_t)min(row0 + r, n - 1) * K;     // clamp: tail rows re-read the last row, never stored
+#pragma unroll 2
+    for (uint32_t k = threadIdx.x * 8; k < K; k += 2048) {
+        uint4 wv[R];
 #pragma unroll
-            for (int r = 0; r < R; ++r) unpack8(wv[r], wf[r]);
+        for (int r = 0; r < R; ++r) wv[r] = __ldcs(reinterpret_cast<const uint4 *>(wrow[r] + k));
 #pragma unroll
-            for (int m = 0; m < MT; ++m) {
-                if (m < (int)Mrows) {
-                    float xf[8];
-                    unpack8(__ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)), xf);
+        for (int m = 0; m < MT; ++m) {
+            float xf[8];
+            unpack8(m < (int)Mrows ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)) : make_uint4(0, 0, 0, 0), xf);
 #pragma unroll
-                    for (int r = 0; r < R; ++r)
+            for (int r = 0; r < R; ++r) {
+                float wf[8];
+                unpack8(wv[r], wf);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) acc[r][m] = fmaf(wf[r][i], xf[i], acc[r][m]);
-                }
+                for (int i = 0; i < 8; ++i) acc[r][m] = fmaf(wf[i], xf[i], acc[r][m]);
             }
         }
+    }
 #pragma unroll
-        for (int r = 0; r < R; ++r)
+    for (int r = 0; r < R; ++r)
 #pragma unroll
-            for (int m = 0; m < MT; ++m) {
-                float s = warp_sum(acc[r][m]);
-                if (lane == 0 && row0 + r < n && m < (int)Mrows) {
-                    float *c = C + (size_t)m * ldc + col0 + row0 + r;
-                    *c = accumulate ? *c + s : s;
-                }
-            }
+        for (int m = 0; m < MT; ++m) {
+            const float s = warp_sum(acc[r][m]);
+            if (lane == 0) part[warp][r * MT + m] = s;
+        }
+    __syncthreads();
+    if (threadIdx.x < R * MT) {
+        const uint32_t r = threadIdx.x / MT, m = threadIdx.x % MT;
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) s += part[w][threadIdx.x];
+        if (row0 + r < n && m < Mrows) {
+            float *c = C + (size_t)m * ldc + col0 + row0 + r;
+            *c = accumulate ? *c + s : s;
+        }
     }
 }
 
@@ -375,10 +386,17 @@ int tgpk_rmsnorm(const float *x, uint32_t ldx, const void *g, void *h, uint32_t 
 
 template <int MT, int R>
 static void launch_gemv(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int acc, cudaStream_t st) {
-    uint32_t warps_needed = (n + R - 1) / R;
-    uint32_t blocks = (warps_needed + 7) / 8;
-    if (blocks > 148 * 8) blocks = 148 * 8;
-    gemv_kernel<MT, R><<<blocks, 256, 0, st>>>(A, W, C, Mrows, n, K, ldc, col0, acc);
+    gemv_kernel<MT, R><<<(n + R - 1) / R, 256, 0, st>>>(A, W, C, Mrows, n, K, ldc, col0, acc);
+}
+
+// rows per block: as many as still leave >= 4 blocks per SM
+template <int MT>
+static void launch_gemv_rows(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int acc, cudaStream_t st) {
+    if constexpr (MT <= 2) {
+        if (n >= 8 * 592) return launch_gemv<MT, 8>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
+        if (n >= 4 * 592) return launch_gemv<MT, 4>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
+    }
+    launch_gemv<MT, 2>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
 }
 
 int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
@@ -390,10 +408,10 @@ int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, ui
             uint32_t mr = M - m0 < 8 ? M - m0 : 8;
             const bf16 *am = a + (size_t)m0 * K;
             float *cm = C + (size_t)m0 * ldc;
-            if (mr == 1) launch_gemv<1, 4>(am, w, cm, mr, n, K, ldc, col0, accumulate, st);
-            else if (mr == 2) launch_gemv<2, 4>(am, w, cm, mr, n, K, ldc, col0, accumulate, st);
-            else if (mr <= 4) launch_gemv<4, 2>(am, w, cm, mr, n, K, ldc, col0, accumulate, st);
-            else launch_gemv<8, 2>(am, w, cm, mr, n, K, ldc, col0, accumulate, st);
+            if (mr == 1) launch_gemv_rows<1>(am, w, cm, mr, n, K, ldc, col0, accumulate, st);
+            else if (mr == 2) launch_gemv_rows<2>(am, w, cm, mr, n, K, ldc, col0, accumulate, st);
+            else if (mr <= 4) launch_gemv_rows<4>(am, w, cm, mr, n, K, ldc, col0, accumulate, st);
+            else launch_gemv_rows<8>(am, w, cm, mr, n, K, ldc, col0, accumulate, st);
             if (m0) tgpk_launches += 1;
         }
     } else {

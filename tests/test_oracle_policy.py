@@ -148,7 +148,7 @@ def test_validator_rejects_broken_plans():
             validate.check(lay.tensors, ops, steps, lay.budget, _tamper(good, fn))
     lay2 = si.build_layout(si.CONFIGS[2])
     ops2, steps2 = trace.run_trace(lay2, n_decode=4)
-    pl2 = policy.plan(lay2.tensors, ops2, steps2, M, lay2.budget)
+    pl2 = policy.plan(lay2.tensors, ops2, steps2, M, lay2.budget, bits=policy.BIT_P | policy.BIT_ZC)     # no pins: KV tiles stream
     assert any(c.kind == policy.CMD_D2H for c in pl2.cmds)
     validate.check(lay2.tensors, ops2, steps2, lay2.budget, pl2.blobs())
     with pytest.raises(validate.PlanInvalid):
