@@ -218,6 +218,23 @@ int  tgp_k_attn(const void *qb, void *const *k_tiles, void *const *v_tiles, uint
                 const tgp_model_cfg *cfg, uint32_t B, uint32_t q_len, uint32_t pos0, float *scratch_dev,
                 void *stream);
 int  tgp_k_attn_scratch_bytes(const tgp_model_cfg *cfg, uint64_t *bytes);
+/* (No counterpart in the paper: a convenience of this library.)
+ * Decode attention (q_len == 1) for callers that must not allocate device memory: code running where the
+ * whole device budget is already handed out to the arena and workspace, inside a serving loop that cannot
+ * afford the device-wide synchronisation an allocation or free may cause, or under a framework whose memory
+ * pool they are not allowed to touch.  Same computation and arguments as tgp_k_attn() with q_len = 1, but the
+ * per-tile partial results go to a fixed array of TGP_STATIC_SCRATCH_BYTES that is part of the library image
+ * (every GPU that loads the library holds those 4 MiB until the process exits).  The call allocates and frees
+ * nothing.  It returns TGP_E_TOO_LARGE, and launches nothing, when B * Hq * n_tiles * (Dh + 2) * 4 exceeds
+ * TGP_STATIC_SCRATCH_BYTES or the device ordinal is >= TGP_STATIC_MAX_DEVICES.
+ * The first call on each device looks up the array's device address (that device must be current); make that
+ * first call before starting any stream capture.  All calls on a device share the one array: it keeps whatever
+ * the previous call left (nothing in it needs to start at zero - every partial that is read is written first by
+ * the same call), and two calls whose kernels overlap on the GPU (different streams) race on it. */
+#define TGP_STATIC_SCRATCH_BYTES (4u << 20)
+#define TGP_STATIC_MAX_DEVICES   64
+int  tgp_k_attn_decode_static(const void *qb, void *const *k_tiles, void *const *v_tiles, uint32_t n_tiles, void *ob,
+                              const tgp_model_cfg *cfg, uint32_t B, uint32_t pos0, void *stream);
 /* a = bf16(silu(g) * u), g/u fp32 [M, F]. */
 int  tgp_k_swiglu(const float *g32, const float *u32, void *ab, uint64_t n_elems, void *stream);
 /* out[b] = argmax_j logits[b, j], lowest index on ties. */

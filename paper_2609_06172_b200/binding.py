@@ -85,6 +85,7 @@ _SIGS = {
     "tgp_k_rope_tables": [_U32, _U32, C.c_float, _P, _P],
     "tgp_k_rope_kv": [_P, _P, _P, _P, C.POINTER(_P), C.POINTER(_P), _U32, _P, _P, C.POINTER(ModelCfg), _U32, _U32, _U32, _P],
     "tgp_k_attn": [_P, C.POINTER(_P), C.POINTER(_P), _U32, _P, C.POINTER(ModelCfg), _U32, _U32, _U32, _P, _P],
+    "tgp_k_attn_decode_static": [_P, C.POINTER(_P), C.POINTER(_P), _U32, _P, C.POINTER(ModelCfg), _U32, _U32, _P],
     "tgp_k_attn_scratch_bytes": [C.POINTER(ModelCfg), C.POINTER(_U64)],
     "tgp_k_swiglu": [_P, _P, _P, _U64, _P],
     "tgp_k_argmax": [_P, _P, _U32, _U32, _P],
@@ -297,6 +298,16 @@ def k_rope_kv(q32, k32, v32, qb, k_tiles, v_tiles, cos, sin, cfg, B, q_len, pos0
 def k_attn(qb, k_tiles, v_tiles, ob, cfg, B, q_len, pos0, scratch=None, stream=None):
     ka, va, n = _tile_arrays(k_tiles, v_tiles)
     _k(lib().tgp_k_attn(_ptr(qb), ka, va, n, _ptr(ob), C.byref(cfg), B, q_len, pos0, _ptr(scratch), _ptr(stream)), "tgp_k_attn")
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def k_attn_decode_static(qb, k_tiles, v_tiles, ob, cfg, B, pos0, stream=None):
+    """Decode attention whose scratch is a fixed array inside the library: for callers that cannot allocate
+    device memory.  Raises TgpError(E_TOO_LARGE) when the partials would not fit in STATIC_SCRATCH_BYTES."""
+    ka, va, n = _tile_arrays(k_tiles, v_tiles)
+    _k(lib().tgp_k_attn_decode_static(_ptr(qb), ka, va, n, _ptr(ob), C.byref(cfg), B, pos0, _ptr(stream)), "tgp_k_attn_decode_static")
 
 
 def k_attn_scratch_bytes(cfg):

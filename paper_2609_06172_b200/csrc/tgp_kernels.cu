@@ -518,6 +518,32 @@ int tgp_k_attn(const void *qb, void *const *k_tiles, void *const *v_tiles, uint3
     return tgpk_attn(qb, t, n_tiles, ob, cfg, B, q_len, pos0, scratch_dev, (cudaStream_t)stream);
 }
 
+// ---- decode attention for callers that cannot allocate ------------------------------------------------
+// The per-tile partials live in a fixed array inside the library image instead of caller memory.  In host
+// code the array's name is only a handle; its device address is looked up once per device.
+static __device__ __align__(256) float g_static_attn_scratch[TGP_STATIC_SCRATCH_BYTES / sizeof(float)];
+static float *g_static_attn_scratch_addr[TGP_STATIC_MAX_DEVICES] = {};
+
+int tgp_k_attn_decode_static(const void *qb, void *const *k_tiles, void *const *v_tiles, uint32_t n_tiles, void *ob,
+                             const tgp_model_cfg *cfg, uint32_t B, uint32_t pos0, void *stream) {
+    if (!qb || !ob || !cfg || !cfg->Hkv || cfg->Hq % cfg->Hkv || !cfg->TK || !B) return TGP_E_INVAL;
+    if ((uint64_t)n_tiles * cfg->TK < (uint64_t)pos0 + 1) return TGP_E_INVAL;
+    const uint64_t need = (uint64_t)B * cfg->Hq * n_tiles * (cfg->Dh + 2) * sizeof(float);
+    if (need > TGP_STATIC_SCRATCH_BYTES) return TGP_E_TOO_LARGE;
+    TgpTilePtrs t;
+    int rc = fill_tiles(t, k_tiles, v_tiles, n_tiles);
+    if (rc) return rc;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return TGP_E_CUDA;
+    if (dev < 0 || dev >= TGP_STATIC_MAX_DEVICES) return TGP_E_TOO_LARGE;
+    if (!g_static_attn_scratch_addr[dev]) {                       // first call on this device, with it current
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_attn_scratch) != cudaSuccess || !p) return TGP_E_CUDA;
+        g_static_attn_scratch_addr[dev] = (float *)p;
+    }
+    return tgpk_attn(qb, t, n_tiles, ob, cfg, B, 1, pos0, g_static_attn_scratch_addr[dev], (cudaStream_t)stream);
+}
+
 int tgp_k_attn_scratch_bytes(const tgp_model_cfg *cfg, uint64_t *bytes) {
     if (!cfg || !bytes || !cfg->TK) return TGP_E_INVAL;
     uint64_t nt = (cfg->max_len + cfg->TK - 1) / cfg->TK;
