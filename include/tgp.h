@@ -201,6 +201,12 @@ int  tgp_k_rmsnorm(const float *x_dev, uint32_t ldx, const void *g_dev, void *h_
  * block), C fp32 with row stride ldc.  accumulate != 0 adds to C (fused residual).  K % 8 == 0. */
 int  tgp_k_gemm(const void *A_dev, const void *W_dev, float *C_dev, uint32_t M, uint32_t n, uint32_t K,
                 uint32_t ldc, uint32_t col0, int accumulate, void *stream);
+/* Which kernel serves M > 16: 0 (default) the tcgen05 tensor-core GEMM, 1 the CUDA-core tile kernel (an on-device
+ * cross-check).  M <= 16 always takes the weight-streaming GEMV.  Process-wide. */
+int  tgp_k_gemm_select(int impl);
+/* Error word of the tensor-core GEMM: 0, or (role << 8 | stage) of the first bounded wait that ran out
+ * (role 1 TMA producer, 2 MMA issuer, 3 epilogue).  Synchronous. */
+int  tgp_k_gemm_status(int *error_code);
 /* Fills caller-owned device tables cos/sin fp32 [max_len, Dh/2]: angle = pos * base^(-2i/Dh), evaluated in
  * double on the host.  Synchronous. */
 int  tgp_k_rope_tables(uint32_t Dh, uint32_t max_len, float base, float *cos_dev, float *sin_dev);

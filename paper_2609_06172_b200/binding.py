@@ -82,6 +82,8 @@ _SIGS = {
     "tgp_k_embed": [_P, _P, _P, _U32, _U32, _P],
     "tgp_k_rmsnorm": [_P, _U32, _P, _P, _U32, _U32, C.c_float, _P],
     "tgp_k_gemm": [_P, _P, _P, _U32, _U32, _U32, _U32, _U32, C.c_int, _P],
+    "tgp_k_gemm_select": [C.c_int],
+    "tgp_k_gemm_status": [C.POINTER(C.c_int)],
     "tgp_k_rope_tables": [_U32, _U32, C.c_float, _P, _P],
     "tgp_k_rope_kv": [_P, _P, _P, _P, C.POINTER(_P), C.POINTER(_P), _U32, _P, _P, C.POINTER(ModelCfg), _U32, _U32, _U32, _P],
     "tgp_k_attn": [_P, C.POINTER(_P), C.POINTER(_P), _U32, _P, C.POINTER(ModelCfg), _U32, _U32, _U32, _P, _P],
@@ -284,6 +286,16 @@ def k_rmsnorm(x, ldx, g, h, M, d, eps, stream=None):
 
 def k_gemm(A, W, Cout, M, n, K, ldc, col0, accumulate, stream=None):
     _k(lib().tgp_k_gemm(_ptr(A), _ptr(W), _ptr(Cout), M, n, K, ldc, col0, int(accumulate), _ptr(stream)), "tgp_k_gemm")
+
+
+def k_gemm_select(impl):
+    _k(lib().tgp_k_gemm_select(impl), "tgp_k_gemm_select")
+
+
+def k_gemm_status():
+    e = C.c_int()
+    _k(lib().tgp_k_gemm_status(C.byref(e)), "tgp_k_gemm_status")
+    return e.value
 
 
 def k_rope_tables(Dh, max_len, base, cos, sin):

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libtgp.so")
-SOURCES = ["tgp_host.cpp", "tgp_model.cpp", "tgp_kernels.cu", "tgp_engine.cu"]
+SOURCES = ["tgp_host.cpp", "tgp_model.cpp", "tgp_kernels.cu", "tgp_gemm_sm100.cu", "tgp_engine.cu"]
 
 
 def sources():
@@ -30,7 +30,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-           "-Xcompiler", "-fPIC", "-shared", "-I" + INCLUDE, "-I" + CSRC, "-o", LIB] + sources() + ["-lcuda"]
+           "-Xcompiler", "-fPIC", "-shared", "-I" + INCLUDE, "-I" + CSRC, "-o", LIB] + sources()
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     r = subprocess.run(cmd, capture_output=True, text=True)

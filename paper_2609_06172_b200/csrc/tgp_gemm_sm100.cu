@@ -1,0 +1,253 @@
+// Prefill GEMM on the 5th-generation tensor cores (sm_100a): C[M, n] (=|+=) A[M, K] * W[n, K]^T,
+// bf16 operands, fp32 accumulation in tensor memory.
+//
+// One CTA computes a 128 x BN tile.  Warp 0 (one lane) feeds a 3-stage shared-memory ring with TMA
+// (128-byte swizzle, 64 bf16 of K per stage); warp 1 (one lane) issues tcgen05.mma (M=128, N=BN, K=16,
+// four per stage) into a TMEM accumulator and releases stages with tcgen05.commit; warps 2-5 wait for the
+// last commit, read the accumulator with tcgen05.ld (each warp its own 32-lane quarter) and store fp32 rows.
+// Out-of-range rows / columns / K are zero-filled by TMA and masked in the epilogue, so any M, n and
+// any K % 8 == 0 work.  Every mbarrier wait is bounded in time: a wait that runs out records an error code
+// and the CTA drains and returns instead of hanging the GPU.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cudaTypedefs.h>
+#include <cstdint>
+#include "tgp.h"
+#include "tgp_kernels.h"
+
+namespace {
+
+constexpr int BM = 128, BK = 64, STAGES = 3;
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;      // 2 s: far beyond any legitimate wait in this kernel
+
+__device__ int g_gemm_tc_error = 0;                    // 0 ok; else (role << 8) | stage of the first wait that ran out
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint64_t now_ns() { uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+
+// Bounded wait on a phase parity.  Returns false when the time limit ran out or another role has given up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *failed) {
+    const uint32_t addr = smem_u32(bar);
+    uint64_t t0 = 0;
+    for (uint32_t spin = 0;; ++spin) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((spin & 1023u) == 1023u) {
+            if (*failed) return false;
+            const uint64_t t = now_ns();
+            if (!t0) t0 = t;
+            else if (t - t0 > WAIT_LIMIT_NS) return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows 128 bytes apart, 8-row groups
+// 1024 bytes apart (stride byte offset); descriptor version 1 (sm_100); layout type 2 = SWIZZLE_128B.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24.
+__host__ __device__ constexpr uint32_t umma_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
+    uint32_t r[32];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+                   "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),
+                   "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]),
+                   "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+template <int BN>
+struct Smem {
+    static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int BAR_OFF = STAGES * STAGE_BYTES;
+    static constexpr int TOTAL = BAR_OFF + 128 + 1024;        // barriers + slack to align the base to 1024 bytes
+};
+
+template <int BN>
+__global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                                                      float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
+    extern __shared__ uint8_t smem_raw[];
+    using S = Smem<BN>;
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + S::BAR_OFF);
+    uint64_t *empty = full + STAGES;
+    uint64_t *acc_full = empty + STAGES;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
+    volatile uint32_t *failed = tmem_slot + 1;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+    const uint32_t num_k = (K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        mbar_init(acc_full, 1);
+        *failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t armed = 0;
+            for (uint32_t kb = 0; kb < num_k; ++kb) {
+                const uint32_t s = kb % STAGES, ph = (kb / STAGES) & 1;
+                if (*failed || !mbar_wait(&empty[s], ph ^ 1, failed)) { if (!*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, (1 << 8) | (int)s); } break; }
+                mbar_expect_tx(&full[s], S::STAGE_BYTES);
+                tma_load_2d(smem + s * S::STAGE_BYTES, &tmA, (int)(kb * BK), (int)m0, &full[s]);
+                tma_load_2d(smem + s * S::STAGE_BYTES + S::A_BYTES, &tmB, (int)(kb * BK), (int)n0, &full[s]);
+                armed = kb + 1;
+            }
+            if (*failed) {
+                // let the copies this thread started land before the CTA's shared memory is given up
+                volatile uint32_t never = 0;
+                for (uint32_t kb = armed > STAGES ? armed - STAGES : 0; kb < armed; ++kb) mbar_wait(&full[kb % STAGES], (kb / STAGES) & 1, &never);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc(BN);
+            bool ok = true;
+            for (uint32_t kb = 0; kb < num_k && ok; ++kb) {
+                const uint32_t s = kb % STAGES, ph = (kb / STAGES) & 1;
+                if (*failed || !mbar_wait(&full[s], ph, failed)) { if (!*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, (2 << 8) | (int)s); } ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint64_t da = umma_desc(smem_u32(smem + s * S::STAGE_BYTES));
+                const uint64_t db = umma_desc(smem_u32(smem + s * S::STAGE_BYTES + S::A_BYTES));
+#pragma unroll
+                for (uint32_t k = 0; k < BK / 16; ++k) umma(tmem_base, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);   // +32 bytes of K per step
+                umma_commit(&empty[s]);
+            }
+            if (ok) umma_commit(acc_full);
+        }
+    } else {
+        bool ready = !*failed && mbar_wait(acc_full, 0, failed);
+        if (!ready && !*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, 3 << 8); }
+        ready = __all_sync(0xffffffffu, ready && !*failed);      // tcgen05.ld is warp-collective: decide per warp
+        if (ready) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t quarter = warp & 3;                    // TMEM lanes this warp may read
+            const uint32_t row = m0 + quarter * 32 + lane;
+            const bool vec = ((ldc | col0) & 3u) == 0 && (reinterpret_cast<uintptr_t>(C) & 15u) == 0;
+#pragma unroll 1
+            for (uint32_t c = 0; c < BN / 32; ++c) {
+                float v[32];
+                tmem_ld32(tmem_base + ((quarter * 32) << 16) + c * 32, v);
+                if (row < M) {
+                    float *dst = C + (size_t)row * ldc + col0 + n0 + c * 32;
+                    const uint32_t col = n0 + c * 32;
+                    if (vec && col + 32 <= n) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                            if (accumulate) { const float4 old = *reinterpret_cast<const float4 *>(dst + j); o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w; }
+                            *reinterpret_cast<float4 *>(dst + j) = o;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col + j < n) dst[j] = accumulate ? dst[j] + v[j] : v[j];
+                    }
+                }
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 2) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)BN) : "memory");
+    }
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 row-major [rows, K] map with a [box_rows, 64] box, 128-byte swizzle, zero fill outside.
+bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t K, uint32_t box_rows) {
+    PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {K, rows};
+    cuuint64_t strides[1] = {K * 2};
+    cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+extern thread_local uint64_t tgpk_launches;
+
+int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
+    constexpr int BN = 128;
+    if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(W)) & 15u) return TGP_E_INVAL;     // TMA needs 16-byte aligned bases
+    if (K % 8) return TGP_E_INVAL;                                                                       // and 16-byte row strides
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, A, M, K, BM) || !make_map(&mb, W, n, K, BN)) return TGP_E_CUDA;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN>::TOTAL) != cudaSuccess) return TGP_E_CUDA;
+        attr_set = true;
+    }
+    dim3 grid((M + BM - 1) / BM, (n + BN - 1) / BN);
+    gemm_tc_kernel<BN><<<grid, 192, Smem<BN>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
+    if (cudaGetLastError() != cudaSuccess) return TGP_E_CUDA;
+    tgpk_launches += 1;
+    return TGP_OK;
+}
+
+extern "C" int tgp_k_gemm_status(int *error_code) {
+    if (!error_code) return TGP_E_INVAL;
+    if (cudaMemcpyFromSymbol(error_code, g_gemm_tc_error, sizeof(int)) != cudaSuccess) return TGP_E_CUDA;
+    return TGP_OK;
+}

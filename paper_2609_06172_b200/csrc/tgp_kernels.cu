@@ -399,6 +399,8 @@ static void launch_gemv_rows(const bf16 *A, const bf16 *W, float *C, uint32_t Mr
     launch_gemv<MT, 2>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
 }
 
+static int g_gemm_impl = 0;      // 0: tensor cores for M > 16; 1: CUDA-core tiles (kept as an on-device cross-check)
+
 int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
     if (!M || !n) return TGP_OK;
     if (K % 8 || !K) return TGP_E_INVAL;
@@ -414,6 +416,8 @@ int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, ui
             else launch_gemv_rows<8>(am, w, cm, mr, n, K, ldc, col0, accumulate, st);
             if (m0) tgpk_launches += 1;
         }
+    } else if (g_gemm_impl == 0) {
+        return tgpk_gemm_tc(A, W, C, M, n, K, ldc, col0, accumulate, st);
     } else {
         dim3 grid((n + 63) / 64, (M + 63) / 64);
         gemm_simt_kernel<<<grid, 256, 0, st>>>(a, w, C, M, n, K, ldc, col0, accumulate);
@@ -491,6 +495,12 @@ int tgp_k_embed(const void *table, const int32_t *tok_dev, float *x_dev, uint32_
 int tgp_k_rmsnorm(const float *x_dev, uint32_t ldx, const void *g_dev, void *h_dev, uint32_t M, uint32_t d, float eps, void *stream) {
     if (!x_dev || !g_dev || !h_dev) return TGP_E_INVAL;
     return tgpk_rmsnorm(x_dev, ldx, g_dev, h_dev, M, d, eps, (cudaStream_t)stream);
+}
+
+int tgp_k_gemm_select(int impl) {
+    if (impl != 0 && impl != 1) return TGP_E_INVAL;
+    g_gemm_impl = impl;
+    return TGP_OK;
 }
 
 int tgp_k_gemm(const void *A_dev, const void *W_dev, float *C_dev, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, void *stream) {

@@ -11,6 +11,8 @@ struct TgpTilePtrs { void *k[TGP_MAX_TILES]; void *v[TGP_MAX_TILES]; };
 int tgpk_embed(const void *table, const int32_t *tok, float *x, uint32_t M, uint32_t d, cudaStream_t st);
 int tgpk_rmsnorm(const float *x, uint32_t ldx, const void *g, void *h, uint32_t M, uint32_t d, float eps, cudaStream_t st);
 int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st);
+// tcgen05 path (tgp_gemm_sm100.cu): any M, n; K % 8 == 0; A and W 16-byte aligned
+int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st);
 int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb, const TgpTilePtrs &tiles, const float *cos_t, const float *sin_t,
                  const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0, cudaStream_t st);
 int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *ob, const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0,

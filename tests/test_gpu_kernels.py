@@ -42,7 +42,8 @@ def bf16_close(got_f32, want_f32, frac=0.01):
 
 @pytest.mark.parametrize("M,n,K", [(1, 300, 256), (1, 4096, 2048), (2, 129, 64), (3, 1000, 512), (8, 1030, 512),
                                    (13, 77, 128), (16, 260, 1024), (17, 64, 96), (33, 130, 96), (200, 260, 1024),
-                                   (64, 64, 32), (1, 1, 8), (70, 5, 8)])
+                                   (64, 64, 32), (1, 1, 8), (70, 5, 8), (129, 257, 72), (300, 520, 1096), (512, 2048, 2048),
+                                   (1000, 136, 8192)])
 @pytest.mark.parametrize("accumulate", [0, 1])
 def test_gemm_matches_oracle(M, n, K, accumulate):
     a_bits, w_bits = rnd_bits(1, M * K).reshape(M, K), rnd_bits(2, n * K).reshape(n, K)
@@ -60,6 +61,24 @@ def test_gemm_matches_oracle(M, n, K, accumulate):
     scale = np.abs(want).max() + 1e-6
     assert np.abs(got - exp).max() < 2e-5 * max(scale, 0.01) + 1e-7
     assert np.array_equal(got[:, :col0], c0[:, :col0]) and np.array_equal(got[:, col0 + n:], c0[:, col0 + n:])
+
+
+def test_tensor_core_gemm_agrees_with_cuda_core_gemm_and_reports_no_timeout():
+    """Same inputs through both M > 16 kernels: the tcgen05 path and the CUDA-core tiles (an on-device cross-check
+    besides the oracle), then the tensor-core kernel's bounded-wait error word must still be zero."""
+    M, n, K = 640, 1408, 2048
+    A, W = bf16_dev(rnd_bits(5, M * K).reshape(M, K)), bf16_dev(rnd_bits(6, n * K).reshape(n, K))
+    outs = []
+    for impl in (0, 1):
+        tb.k_gemm_select(impl)
+        Cd = torch.zeros(M, n, dtype=torch.float32, device=DEV)
+        tb.k_gemm(A, W, Cd, M, n, K, n, 0, 0)
+        torch.cuda.synchronize()
+        outs.append(Cd.cpu().numpy())
+    tb.k_gemm_select(0)
+    assert np.abs(outs[0] - outs[1]).max() < 2e-5 * np.abs(outs[1]).max()
+    assert np.abs(outs[0]).max() > 0
+    assert tb.k_gemm_status() == 0
 
 
 def test_gemm_rejects_bad_arguments_and_accepts_empty():
