@@ -68,58 +68,58 @@ __global__ void rmsnorm_kernel(const float *__restrict__ x, uint32_t ldx, const 
 }
 
 // ---- GEMV / skinny GEMM (M <= 8 activation rows): pure weight streaming --------------------------------
-// One block owns R output rows; its 8 warps split K, so every thread has R independent 16-byte loads in
-// flight per k-chunk and a [n, K] block of any aspect ratio fills the machine (n/R blocks).  Partial sums
-// meet in shared memory in a fixed order: results are deterministic run to run.
-template <int MT, int R>
+// Persistent warps: the grid fills every SM once; each warp walks row groups of R output rows with a
+// grid stride and keeps R x U independent 16-byte loads in flight per lane (U chunks of 256 K-elements).
+// No block barrier and no shared memory, so no SM idles while another warp reduces; the summation order
+// is fixed (lane-strided partials, butterfly), hence results are deterministic run to run.
+template <int MT, int R, int U>
 __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                    uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
-    __shared__ float part[8][R * MT];
-    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t row0 = blockIdx.x * R;
-    float acc[R][MT];
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarp = (gridDim.x * blockDim.x) >> 5;
+    for (uint32_t row0 = gwarp * R; row0 < n; row0 += nwarp * R) {
+        float acc[R][MT];
 #pragma unroll
-    for (int r = 0; r < R; ++r)
+        for (int r = 0; r < R; ++r)
 #pragma unroll
-        for (int m = 0; m < MT; ++m) acc[r][m] = 0.f;
-    const bf16 *wrow[R];
+            for (int m = 0; m < MT; ++m) acc[r][m] = 0.f;
+        const bf16 *wrow[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) wrow[r] = W + (size_t)min(row0 + r, n - 1) * K;     // clamp: tail rows re-read the last row, never stored
-#pragma unroll 2
-    for (uint32_t k = threadIdx.x * 8; k < K; k += 2048) {
-        uint4 wv[R];
+        for (int r = 0; r < R; ++r) wrow[r] = W + (size_t)min(row0 + r, n - 1) * K;   // tail rows re-read the last row, never stored
+        for (uint32_t k0 = lane * 8; k0 < K; k0 += 256 * U) {
+            uint4 wv[U][R];
 #pragma unroll
-        for (int r = 0; r < R; ++r) wv[r] = __ldcs(reinterpret_cast<const uint4 *>(wrow[r] + k));
+            for (int u = 0; u < U; ++u)
 #pragma unroll
-        for (int m = 0; m < MT; ++m) {
-            float xf[8];
-            unpack8(m < (int)Mrows ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)) : make_uint4(0, 0, 0, 0), xf);
+                for (int r = 0; r < R; ++r)
+                    wv[u][r] = (k0 + 256 * u < K) ? __ldcs(reinterpret_cast<const uint4 *>(wrow[r] + k0 + 256 * u)) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                float wf[8];
-                unpack8(wv[r], wf);
+            for (int u = 0; u < U; ++u) {
+                const uint32_t k = k0 + 256 * u;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) acc[r][m] = fmaf(wf[i], xf[i], acc[r][m]);
+                for (int m = 0; m < MT; ++m) {
+                    float xf[8];
+                    unpack8((k < K && m < (int)Mrows) ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)) : make_uint4(0, 0, 0, 0), xf);
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        float wf[8];
+                        unpack8(wv[u][r], wf);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) acc[r][m] = fmaf(wf[i], xf[i], acc[r][m]);
+                    }
+                }
             }
         }
-    }
 #pragma unroll
-    for (int r = 0; r < R; ++r)
+        for (int r = 0; r < R; ++r)
 #pragma unroll
-        for (int m = 0; m < MT; ++m) {
-            const float s = warp_sum(acc[r][m]);
-            if (lane == 0) part[warp][r * MT + m] = s;
-        }
-    __syncthreads();
-    if (threadIdx.x < R * MT) {
-        const uint32_t r = threadIdx.x / MT, m = threadIdx.x % MT;
-        float s = 0.f;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) s += part[w][threadIdx.x];
-        if (row0 + r < n && m < Mrows) {
-            float *c = C + (size_t)m * ldc + col0 + row0 + r;
-            *c = accumulate ? *c + s : s;
-        }
+            for (int m = 0; m < MT; ++m) {
+                const float s = warp_sum(acc[r][m]);
+                if (lane == 0 && row0 + r < n && m < (int)Mrows) {
+                    float *c = C + (size_t)m * ldc + col0 + row0 + r;
+                    *c = accumulate ? *c + s : s;
+                }
+            }
     }
 }
 
@@ -384,19 +384,30 @@ int tgpk_rmsnorm(const float *x, uint32_t ldx, const void *g, void *h, uint32_t 
     return TGP_OK;
 }
 
-template <int MT, int R>
+template <int MT, int R, int U>
 static void launch_gemv(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int acc, cudaStream_t st) {
-    gemv_kernel<MT, R><<<(n + R - 1) / R, 256, 0, st>>>(A, W, C, Mrows, n, K, ldc, col0, acc);
+    static int blocks_per_sm = 0, sms = 0;
+    if (!blocks_per_sm) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, gemv_kernel<MT, R, U>, 256, 0) != cudaSuccess || blocks_per_sm < 1) blocks_per_sm = 1;
+        if (sms < 1) sms = 148;
+    }
+    uint32_t need = (n + R * 8 - 1) / (R * 8), full = (uint32_t)(sms * blocks_per_sm);
+    gemv_kernel<MT, R, U><<<need < full ? need : full, 256, 0, st>>>(A, W, C, Mrows, n, K, ldc, col0, acc);
 }
 
-// rows per block: as many as still leave >= 4 blocks per SM
+// rows per warp: fewer when the block has few rows, so that every SM still gets warps
 template <int MT>
 static void launch_gemv_rows(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int acc, cudaStream_t st) {
     if constexpr (MT <= 2) {
-        if (n >= 8 * 592) return launch_gemv<MT, 8>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
-        if (n >= 4 * 592) return launch_gemv<MT, 4>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
+        if (n >= 2 * 148 * 16) return launch_gemv<MT, 2, 4>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
+        return launch_gemv<MT, 1, 8>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
+    } else {
+        if (n >= 2 * 148 * 16) return launch_gemv<MT, 2, 2>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
+        return launch_gemv<MT, 1, 4>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
     }
-    launch_gemv<MT, 2>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
 }
 
 static int g_gemm_impl = 0;      // 0: tensor cores for M > 16; 1: CUDA-core tiles (kept as an on-device cross-check)
