@@ -207,6 +207,18 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
     return sec, bytes_per, flops_per, len(shapes), table
 
 
+def whole_job_rate(units_per_rank, ms_local, dist=None, device=None):
+    """Replicas: every rank processed `units_per_rank` units in `ms_local`; the job's rate is all units over the
+    slowest rank's time.  The only collective is this MAX reduction of the timing (none on the data path)."""
+    world, ms = 1, float(ms_local)
+    if dist is not None and dist.is_initialized():
+        import torch
+        t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, world = float(t.item()), dist.get_world_size()
+    return world * units_per_rank / (ms * 1e-3), ms, world
+
+
 def run_reference(args, cfg, lay):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -327,12 +339,7 @@ def main():
         ev1.record(r.compute)
         r.sync()
         barrier()
-        ms = ev0.elapsed_time(ev1)
-        if dist is not None:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return whole_job_rate(1, ev0.elapsed_time(ev1), dist, dev)[1]
 
     for _ in range(args.warmup):
         one_pass(False)
@@ -432,11 +439,17 @@ def main():
     if not args.no_uvm:
         try:
             from paper_2609_06172_b200 import uvm_baseline
-            out["uvm_demand_paged"] = uvm_baseline.run(cfg, lay, MACHINE, dev)
-        except ImportError:
-            out["uvm_demand_paged"] = "not run: baseline module not built yet"
+            del r
+            s.close()
+            torch.cuda.empty_cache()
+            uvm = uvm_baseline.run(cfg, lay, MACHINE, dev, si.fill_pool)
+            dec = cfg.B * T / (sum(step_ms[1:]) * 1e-3) if T else None
+            for v in uvm.values():
+                if dec and v.get("decode_tok_s"):
+                    v["explicit_ring_speedup_decode"] = dec / v["decode_tok_s"]
+            out["uvm"] = uvm
         except Exception as ex:  # the baseline is reported, never fatal
-            out["uvm_demand_paged"] = f"not run: {type(ex).__name__}: {ex}"
+            out["uvm"] = f"not run: {type(ex).__name__}: {ex}"
     if not args.no_cpu_baseline:
         W = oracle_weights_from_pool(lay, pool.numpy())
         sS, sT = min(cfg.S, 128), min(cfg.T, 4)
@@ -444,7 +457,6 @@ def main():
         out["cpu_baseline"] = {"value": val, "unit": "tokens/s", "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
                                "sample": f"prefill of the first {sS} prompt tokens + {sT} decode steps, float32 accumulate ({dt:.1f} s)"}
     print(json.dumps(out))
-    s.close()
     if dist is not None:
         dist.destroy_process_group()
 

@@ -183,6 +183,14 @@ int  tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_host, uint
               float *logits_dev, int32_t *argmax_dev, void *compute_stream, void *copy_stream,
               tgp_step_stats *stats);
 
+/* Managed-memory helpers for the two managed variants (Section II-A: cudaMallocManaged pools that migrate on
+ * demand).  tgp_managed_alloc() returns cudaMallocManaged memory the caller fills and registers with
+ * TGP_POOL_MANAGED and later frees with tgp_managed_free(); tgp_managed_evict() moves a managed range back to
+ * host memory and waits (a cold start for a managed run). */
+int  tgp_managed_alloc(void **out, uint64_t bytes);
+int  tgp_managed_free(void *ptr);
+int  tgp_managed_evict(void *ptr, uint64_t bytes);
+
 /* Per-op timestamps (Section IV-D "Runtime Monitor": lightweight timestamping).  While enabled, tgp_step()
  * brackets every op with CUDA events on the compute stream (after the op's copies have been waited for, so
  * the figure is kernel time, not stall time).  tgp_op_times() waits for the last timed step and returns one

@@ -77,6 +77,9 @@ _SIGS = {
     "tgp_model_bind": [_P, C.POINTER(ModelCfg), C.POINTER(RoleEntry), _U32, _P, _P, _U64, _U32],
     "tgp_run_reset": [_P],
     "tgp_step": [_P, _U32, _P, _U32, _U32, _P, _P, _P, _P, C.POINTER(StepStats)],
+    "tgp_managed_alloc": [C.POINTER(_P), _U64],
+    "tgp_managed_free": [_P],
+    "tgp_managed_evict": [_P, _U64],
     "tgp_set_op_timing": [_P, C.c_int],
     "tgp_op_times": [_P, C.POINTER(C.c_float), _U32, C.POINTER(_U32), C.POINTER(_U32)],
     "tgp_k_embed": [_P, _P, _P, _U32, _U32, _P],
@@ -256,6 +259,20 @@ class Ctx:
         ms = (C.c_float * max(1, n.value))()
         self._ck(lib().tgp_op_times(self._h, ms, n.value, C.byref(first), C.byref(n)), "tgp_op_times")
         return first.value, np.frombuffer(ms, dtype=np.float32, count=n.value).copy()
+
+
+def managed_alloc(nbytes: int) -> int:
+    p = _P()
+    _k(lib().tgp_managed_alloc(C.byref(p), nbytes), "tgp_managed_alloc")
+    return p.value
+
+
+def managed_free(ptr: int):
+    _k(lib().tgp_managed_free(ptr), "tgp_managed_free")
+
+
+def managed_evict(ptr: int, nbytes: int):
+    _k(lib().tgp_managed_evict(ptr, nbytes), "tgp_managed_evict")
 
 
 def model_workspace_bytes(cfg: ModelCfg, max_tokens: int) -> int:

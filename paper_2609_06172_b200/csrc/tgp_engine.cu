@@ -408,3 +408,24 @@ extern "C" int tgp_op_times(tgp_ctx *ctx, float *ms, uint32_t capacity, uint32_t
     }
     return TGP_OK;
 }
+
+// ---- managed-memory helpers for the managed variants (the pool itself stays caller-owned) ----------------
+extern "C" int tgp_managed_alloc(void **out, uint64_t bytes) {
+    if (!out || !bytes) return TGP_E_INVAL;
+    void *p = nullptr;
+    if (cudaMallocManaged(&p, bytes, cudaMemAttachGlobal) != cudaSuccess) { cudaGetLastError(); return TGP_E_CUDA; }
+    *out = p;
+    return TGP_OK;
+}
+
+extern "C" int tgp_managed_free(void *ptr) {
+    if (!ptr) return TGP_OK;
+    return cudaFree(ptr) == cudaSuccess ? TGP_OK : TGP_E_CUDA;
+}
+
+// Moves a managed range back to host memory (cold start for a managed run) and waits for it.
+extern "C" int tgp_managed_evict(void *ptr, uint64_t bytes) {
+    if (!ptr || !bytes) return TGP_E_INVAL;
+    if (cudaMemPrefetchAsync(ptr, bytes, cudaCpuDeviceId, 0) != cudaSuccess) { cudaGetLastError(); return TGP_E_CUDA; }
+    return cudaDeviceSynchronize() == cudaSuccess ? TGP_OK : TGP_E_CUDA;
+}

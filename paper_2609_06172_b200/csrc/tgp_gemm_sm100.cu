@@ -17,7 +17,7 @@
 
 namespace {
 
-constexpr int BM = 128, BK = 64, STAGES = 3;
+constexpr int BM = 128, BK = 64, STAGES = 3, GROUP_M = 16;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;      // 2 s: far beyond any legitimate wait in this kernel
 
 __device__ int g_gemm_tc_error = 0;                    // 0 ok; else (role << 8) | stage of the first wait that ran out
@@ -110,7 +110,14 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
     volatile uint32_t *failed = tmem_slot + 1;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+    // Tile order: groups of GROUP_M row tiles are swept across all column tiles before the next group starts, so the
+    // CTAs in flight together share a few A panels and a few W panels that fit in L2 (instead of re-streaming A from
+    // HBM once per column tile when M is large).
+    const uint32_t tiles_m = (M + BM - 1) / BM, tiles_n = (n + BN - 1) / BN;
+    const uint32_t group = blockIdx.x / (GROUP_M * tiles_n), first_m = group * GROUP_M;
+    const uint32_t rows_in_group = min((uint32_t)GROUP_M, tiles_m - first_m);
+    const uint32_t in_group = blockIdx.x - group * GROUP_M * tiles_n;
+    const uint32_t m0 = (first_m + in_group % rows_in_group) * BM, n0 = (in_group / rows_in_group) * BN;
     const uint32_t num_k = (K + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
@@ -239,7 +246,7 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
         if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN>::TOTAL) != cudaSuccess) return TGP_E_CUDA;
         attr_set = true;
     }
-    dim3 grid((M + BM - 1) / BM, (n + BN - 1) / BN);
+    dim3 grid(((M + BM - 1) / BM) * ((n + BN - 1) / BN));
     gemm_tc_kernel<BN><<<grid, 192, Smem<BN>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
     if (cudaGetLastError() != cudaSuccess) return TGP_E_CUDA;
     tgpk_launches += 1;

@@ -19,7 +19,7 @@ def pinned_pool(nbytes: int) -> torch.Tensor:
 class Runner:
     """Owns arena, workspace, logits and streams for one Session and drives tgp_step()."""
 
-    def __init__(self, session: Session, max_tokens: int, device="cuda:0"):
+    def __init__(self, session: Session, max_tokens: int, device="cuda:0", arena=True):
         self.s = session
         cfg = session.layout.cfg
         self.cfg = cfg
@@ -28,13 +28,16 @@ class Runner:
         self.ws_bytes = tb.model_workspace_bytes(session.cfg, max_tokens)
         self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=self.dev)
         self.arena_bytes = session.layout.budget
-        self.arena = torch.empty((self.arena_bytes + 511) // 512 * 512, dtype=torch.uint8, device=self.dev)
-        assert self.arena.data_ptr() % 512 == 0 and self.workspace.data_ptr() % 256 == 0
+        self.arena = torch.empty((self.arena_bytes + 511) // 512 * 512, dtype=torch.uint8, device=self.dev) if arena else None
+        assert (self.arena is None or self.arena.data_ptr() % 512 == 0) and self.workspace.data_ptr() % 256 == 0
         self.logits = torch.empty((cfg.B, cfg.V), dtype=torch.float32, device=self.dev)
         self.argmax = torch.empty((cfg.B,), dtype=torch.int32, device=self.dev)
         self.compute = torch.cuda.Stream(device=self.dev)
         self.copy = torch.cuda.Stream(device=self.dev)
-        session.attach_device(self.arena, self.arena_bytes, self.workspace, self.ws_bytes, max_tokens)
+        if arena:
+            session.attach_device(self.arena, self.arena_bytes, self.workspace, self.ws_bytes, max_tokens)
+        else:                                   # managed variants read the pool in place: no arena
+            session.ctx.model_bind(session.cfg, session.roles, session.router_bias, self.workspace, self.ws_bytes, max_tokens)
 
     def reset(self):
         self.s.ctx.run_reset()

@@ -1,0 +1,85 @@
+"""Managed-memory runs of the same kernels: the demand-paged baseline (no hints) and the hinted variant
+(cudaMemPrefetchAsync for link-bound ops, cudaMemAdvise for the pin set), with the device capacity cut to
+the budget by a ballast allocation, as the paper does with a helper process (Section V-A)."""
+from __future__ import annotations
+
+import ctypes
+
+import numpy as np
+import torch
+
+from . import binding as tb
+from .runner import Runner
+from .session import Session
+
+
+class ManagedPool:
+    def __init__(self, nbytes):
+        self.nbytes = nbytes
+        self.ptr = tb.managed_alloc(nbytes)
+
+    def numpy(self):
+        return np.ctypeslib.as_array((ctypes.c_uint8 * self.nbytes).from_address(self.ptr))
+
+    def free(self):
+        if self.ptr:
+            tb.managed_free(self.ptr)
+            self.ptr = 0
+
+
+def run(cfg, lay, machine, dev, fill, variants=(tb.VAR_MANAGED_DEMAND, tb.VAR_MANAGED_HINTS), decode_cap=16, slack=768 << 20, ballast=True):
+    """Returns {variant name: {...}}.  `fill(layout, uint8 array)` writes the pool contents.  Capacity: after the
+    workspace is allocated, everything but budget + slack of the free device memory is held by a ballast tensor.
+    Decode is capped at `decode_cap` steps (demand paging under 2x oversubscription is slow); rates are per step."""
+    torch.cuda.set_device(dev)
+    out = {}
+    pool = ManagedPool(lay.pool_bytes)
+    try:
+        fill(lay, pool.numpy())
+        T = min(cfg.T, decode_cap)
+        prompt = np.ascontiguousarray(_prompt(cfg))
+        for var in variants:
+            name = "managed_demand" if var == tb.VAR_MANAGED_DEMAND else "managed_hints"
+            s = Session(lay, machine, pool_base=pool.ptr, pool_flags=tb.POOL_MANAGED)
+            s.plan(T=T, variant=var)
+            r = Runner(s, cfg.B * cfg.S, device=str(dev), arena=False)
+            hold = None
+            info = {"decode_steps": T}
+            if ballast:
+                torch.cuda.synchronize()
+                free, total = torch.cuda.mem_get_info(dev)
+                nb = free - lay.budget - slack
+                if nb > 0:
+                    try:
+                        hold = torch.empty(nb, dtype=torch.uint8, device=dev)
+                        info["ballast_bytes"] = int(nb)
+                    except RuntimeError as ex:
+                        info["ballast"] = f"not allocated: {ex}"
+                free2, _ = torch.cuda.mem_get_info(dev)
+                info["free_device_bytes_during_run"] = int(free2)
+            times = []
+            for rep in range(2):                          # first pass warms code paths; second is reported
+                tb.managed_evict(pool.ptr, lay.pool_bytes)
+                r.reset()
+                st = [r.step(tb.PREFILL, prompt, cfg.S, want_stats=True).step_ms]
+                for _ in range(T):
+                    st.append(r.step(tb.DECODE, None, 1, want_stats=True).step_ms)
+                times = st
+            r.sync()
+            info.update({"prefill_ms": times[0], "decode_ms_per_step": float(np.mean(times[1:])) if T else None,
+                         "decode_tok_s": cfg.B * T / (sum(times[1:]) * 1e-3) if T else None,
+                         "prefill_tok_s": cfg.B * cfg.S / (times[0] * 1e-3)})
+            out[name] = info
+            del hold
+            s.close()
+            del r
+            torch.cuda.empty_cache()
+    finally:
+        torch.cuda.synchronize()
+        pool.free()
+    return out
+
+
+def _prompt(cfg):
+    import seeded_inputs as si
+    return si.prompt_tokens(cfg)

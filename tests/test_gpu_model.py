@@ -155,3 +155,42 @@ def test_config_2_prefill_and_first_decode_steps_match_oracle():
     check_logits(got, ref, max(MAX_ABS, 2 * fl_max), max(MEAN_REL, 2 * fl_rel))
     assert all(np.argmax(a[0]) == np.argmax(b[0]) or abs(np.sort(b[0])[-1] - np.sort(b[0])[-2]) < 2 * fl_max for a, b in zip(got, ref))
     s.close()
+
+
+def test_managed_variants_give_the_same_bits_as_the_explicit_ring():
+    """Same kernels reading a cudaMallocManaged pool in place (demand paging, and prefetch/advise hints):
+    only the placement mechanism differs, so logits must be bitwise equal to the explicit engine's."""
+    from paper_2609_06172_b200 import uvm_baseline
+    cfg = replace(si.CONFIGS[1], T=4)
+    prompt = si.prompt_tokens(cfg)
+    forced = (np.arange(cfg.B * cfg.T, dtype=np.int32).reshape(cfg.B, cfg.T) * 577 + 11) % cfg.V
+    lay, pool, s, blobs, T = setup(cfg)
+    ref, _ = Runner(s, cfg.B * cfg.S).generate(prompt, T, forced=forced)
+    s.close()
+    mp = uvm_baseline.ManagedPool(lay.pool_bytes)
+    try:
+        si.fill_pool(lay, mp.numpy())
+        for var in (tb.VAR_MANAGED_DEMAND, tb.VAR_MANAGED_HINTS):
+            sm = Session(lay, MACHINE, pool_base=mp.ptr, pool_flags=tb.POOL_MANAGED)
+            sm.plan(T=T, variant=var)
+            r = Runner(sm, cfg.B * cfg.S, arena=False)
+            tb.managed_evict(mp.ptr, lay.pool_bytes)
+            got, _ = r.generate(prompt, T, forced=forced)
+            for a, b in zip(got, ref):
+                assert np.array_equal(a, b)
+            # KV tiles were written in place: start from zeros again for the next variant
+            sm.close()
+            si.fill_pool(lay, mp.numpy())
+        # a pinned pool cannot run a managed variant: state error, not a fault
+        lay2, pool2, s2, _, _ = setup(cfg)
+        s2.ctx.set_variant(tb.VAR_MANAGED_DEMAND, 7)
+        s2.ctx.model_trace(cfg.S, T)
+        s2.ctx.plan()
+        r2 = Runner(s2, cfg.B * cfg.S)
+        with pytest.raises(tb.TgpError) as ei:
+            r2.step(tb.PREFILL, prompt, cfg.S)
+        assert ei.value.code == tb.E_STATE
+        s2.close()
+    finally:
+        torch.cuda.synchronize()
+        mp.free()
