@@ -219,6 +219,13 @@ def whole_job_rate(units_per_rank, ms_local, dist=None, device=None):
     return world * units_per_rank / (ms * 1e-3), ms, world
 
 
+def oracle_sample(cfg, lay):
+    """Bounded sample for timing the oracle: about 5e11 flops of prefill (at most 128 prompt tokens per sequence)
+    plus up to 4 decode steps, at full widths and depth."""
+    params = lay.weight_bytes // 2
+    return int(max(4, min(128, cfg.S, 5e11 / (2 * params * cfg.B)))), min(cfg.T, 4)
+
+
 def run_reference(args, cfg, lay):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -226,7 +233,7 @@ def run_reference(args, cfg, lay):
     pool = np.empty(lay.pool_bytes, dtype=np.uint8)
     si.fill_pool(lay, pool)
     W = oracle_weights_from_pool(lay, pool)
-    sS, sT = min(cfg.S, 128), min(cfg.T, 4)
+    sS, sT = oracle_sample(cfg, lay)
     cores = len(os.sched_getaffinity(0))
     for _ in range(args.warmup):
         time_oracle(lay, W, 16, 1)
@@ -296,7 +303,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     pool = pinned_pool(lay.pool_bytes)
-    si.fill_pool(lay, pool.numpy())
+    si.fill_pool_torch(lay, pool, device=dev)
     s = Session(lay, MACHINE, pool_base=pool.data_ptr(), pool_flags=tb.POOL_PINNED)
     blobs = s.plan()
     totals = np.frombuffer(blobs["totals"], dtype="<u8").reshape(-1, 4)
@@ -427,7 +434,7 @@ def main():
                  "flops": F, "hbm_bytes": H}
     out = {"metric": "tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-           "data": "synthetic", "config": {"workload": workload_name(cfg, lay), "l2": "inputs larger than L2: every decode step streams the 2.2 GB pool",
+           "data": "synthetic", "config": {"workload": workload_name(cfg, lay), "l2": f"inputs larger than L2: every decode step streams the {lay.pool_bytes / 1e9:.1f} GB pool",
                                            "step": "prefill + all decode steps from a cold arena", "tokens_per_step": tokens_per_pass,
                                            "parallelism": "replicas" if world > 1 else "single"},
            "prefill_tok_s": cfg.B * cfg.S / (step_ms[0] * 1e-3), "decode_tok_s": cfg.B * T / (sum(step_ms[1:]) * 1e-3) if T else None,
@@ -442,7 +449,8 @@ def main():
             del r
             s.close()
             torch.cuda.empty_cache()
-            uvm = uvm_baseline.run(cfg, lay, MACHINE, dev, si.fill_pool)
+            uvm = uvm_baseline.run(cfg, lay, MACHINE, dev, lambda l, arr: arr.__setitem__(slice(None), pool.numpy()),
+                                   decode_cap=16 if lay.pool_bytes < (4 << 30) else 4)
             dec = cfg.B * T / (sum(step_ms[1:]) * 1e-3) if T else None
             for v in uvm.values():
                 if dec and v.get("decode_tok_s"):
@@ -452,7 +460,7 @@ def main():
             out["uvm"] = f"not run: {type(ex).__name__}: {ex}"
     if not args.no_cpu_baseline:
         W = oracle_weights_from_pool(lay, pool.numpy())
-        sS, sT = min(cfg.S, 128), min(cfg.T, 4)
+        sS, sT = oracle_sample(cfg, lay)
         val, dt = time_oracle(lay, W, sS, sT)
         out["cpu_baseline"] = {"value": val, "unit": "tokens/s", "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
                                "sample": f"prefill of the first {sS} prompt tokens + {sT} decode steps, float32 accumulate ({dt:.1f} s)"}

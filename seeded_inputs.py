@@ -289,6 +289,49 @@ def fill_pool(lay: PoolLayout, pool_u8: np.ndarray) -> None:
         fill_tensor(lay.cfg, t, u16[t.pool_off // 2: t.pool_off // 2 + t.rows * t.cols])
 
 
+def _torch_normal_bits(seed: int, role: int, start: int, count: int, device):
+    """Same stream as normal_bf16_bits(), evaluated with torch integer ops (int64 wraps like uint64; logical
+    right shifts are emulated by masking).  Returns an int16 tensor of bf16 bit patterns on `device`."""
+    import torch
+
+    def sgn(v):                       # two's-complement view of a uint64 constant
+        v &= MASK64
+        return v - (1 << 64) if v >= (1 << 63) else v
+
+    def lsr(z, k):
+        return (z >> k) & ((1 << (64 - k)) - 1)
+
+    idx = torch.arange(start, start + count, dtype=torch.int64, device=device)
+    z = (idx ^ sgn(seed ^ (role << 40))) + sgn(0x9E3779B97F4A7C15)
+    z = (z ^ lsr(z, 30)) * sgn(0xBF58476D1CE4E5B9)
+    z = (z ^ lsr(z, 27)) * sgn(0x94D049BB133111EB)
+    h = z ^ lsr(z, 31)
+    s = (h & 0xFFFF) + (lsr(h, 16) & 0xFFFF) + (lsr(h, 32) & 0xFFFF) + lsr(h, 48) - 131070
+    w = (s.to(torch.float32) * float(_C_SCALE)).to(torch.bfloat16)
+    return w.view(torch.int16)
+
+
+def fill_pool_torch(lay: PoolLayout, pool_u8, device="cuda:0", chunk: int = 1 << 26) -> None:
+    """fill_pool() for large pools: generates on `device` and copies into the (pinned) torch uint8 pool tensor.
+    Bit-identical to the numpy path (tested)."""
+    import torch
+    i16 = pool_u8.view(torch.int16)
+    for t in lay.tensors:
+        n = t.rows * t.cols
+        dst = i16[t.pool_off // 2: t.pool_off // 2 + n]
+        if t.kind in (K_G1, K_G2, K_GF):
+            dst.fill_(0x3F80)
+        elif t.kind in (K_KT, K_VT):
+            dst.zero_()
+        else:
+            role = weight_role(t.kind, t.layer, t.expert)
+            for o in range(0, n, chunk):
+                c = min(chunk, n - o)
+                dst[o:o + c].copy_(_torch_normal_bits(lay.cfg.seed, role, t.row0 * t.cols + o, c, device))
+    if str(device).startswith("cuda"):
+        torch.cuda.synchronize()
+
+
 def weights_as_bits(lay: PoolLayout) -> Dict[tuple, np.ndarray]:
     """Whole logical matrices (blocks re-joined) as bf16 bit arrays ``[rows, cols]``, keyed (kind, layer, expert)."""
     out = {}

@@ -76,3 +76,14 @@ def test_router_bias_is_zipf_permutation():
     for l in range(cfg.L):
         assert np.allclose(np.sort(p[l])[::-1], ref, atol=1e-6)
     assert len({tuple(np.argsort(-b[l])) for l in range(cfg.L)}) > 1
+
+
+def test_torch_generator_matches_numpy_generator_bit_for_bit():
+    import torch
+    cfg = si.CONFIGS[1]
+    lay = si.build_layout(cfg)
+    a = np.zeros(lay.pool_bytes, dtype=np.uint8)
+    si.fill_pool(lay, a)
+    b = torch.zeros(lay.pool_bytes, dtype=torch.uint8)
+    si.fill_pool_torch(lay, b, device="cuda:0" if torch.cuda.is_available() else "cpu", chunk=100000)
+    assert np.array_equal(a, b.numpy())
