@@ -93,7 +93,7 @@ extern "C" {
 #define TGP_BIT_ZC 4u   /* sparse read-only accesses are served in place over the link          */
 /* plan export selectors */
 #define TGP_X_CLASSES  0u   /* u8 per op: 0 LINK, 1 HBM, 2 COMPUTE                                   */
-#define TGP_X_TENSORS  1u   /* per tensor: u8 critical, u8 zero-copy, u64 score                      */
+#define TGP_X_TENSORS  1u   /* per tensor: u8 critical, u8 zero-copy, u64 score (link bytes residency saves) */
 #define TGP_X_PINS     2u   /* (u32 tensor, u64 arena offset) ascending tensor id, then u64 ring base, u64 ring size */
 #define TGP_X_COMMANDS 3u   /* per command: u32 seq, u8 kind(0 H2D,1 ALLOC,2 D2H), u32 tensor, u64 bytes, u64 pool offset,
                                u64 arena offset, i32 wait_op, i32 first_use, i32 release_after      */
@@ -182,6 +182,13 @@ int  tgp_run_reset(tgp_ctx *ctx);
 int  tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_host, uint32_t B, uint32_t q_len,
               float *logits_dev, int32_t *argmax_dev, void *compute_stream, void *copy_stream,
               tgp_step_stats *stats);
+
+/* MoE profile (Section IV-C: one profiling pass recovers which tensors the kernels really touch): the tokens
+ * routed to each expert, per step and layer, in the run since the last tgp_run_reset(): uint32 [steps, L, E].
+ * Two-call form: out == NULL returns the element count in *n.  Feed it to tgp_model_trace() to trace exactly the
+ * experts in use.  At run time an expert the router picks but the trace does not list is fetched synchronously
+ * into a spill buffer and counted in tgp_step_stats.n_mismatch. */
+int  tgp_expert_counts(tgp_ctx *ctx, uint32_t *out, uint64_t *n);
 
 /* Managed-memory helpers for the two managed variants (Section II-A: cudaMallocManaged pools that migrate on
  * demand).  tgp_managed_alloc() returns cudaMallocManaged memory the caller fills and registers with

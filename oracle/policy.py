@@ -20,7 +20,8 @@ Steps, in order (notation: P = peak flop/s, Bh = HBM bytes/s, Bl = host-link byt
      LINK    iff mig_i*P > flops_i*Bl and mig_i*Bh > hbm_i*Bl   (the link time exceeds both others)
      COMPUTE iff not LINK and flops_i*Bh >= hbm_i*P
      HBM     otherwise.                With the P bit off every op with mig_i > 0 is LINK.
-2. crit[t] iff a LINK op accesses t;  score[t] = sum of touched bytes over LINK-op accesses.
+2. crit[t] iff a LINK op accesses t;  score[t] = link bytes residency would save: over LINK-op accesses,
+   the touched bytes, plus the tensor's size for each write (a written stay ends in a whole-tensor D2H).
 3. zero-copy (ZC bit): a READONLY tensor whose every access touches < size/ZC_DEN bytes is read
    in place over the link and never staged.
 4. residency episodes: consecutive accesses of t (same step, gap <= W_AFF ops) share one stay.
@@ -137,9 +138,9 @@ def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A |
         c = classify(op.flops, op.hbm, mig, machine, bool(bits & BIT_P))
         cls.append(c)
         if c == CLS_LINK:
-            for (t, _, touched) in op.acc:
+            for (t, mode, touched) in op.acc:
                 crit[t] = 1
-                score[t] += touched
+                score[t] += touched + (tensors[t].size if mode & MODE_W else 0)
     # 3: zero-copy
     accessed = [0] * T
     sparse = [1] * T

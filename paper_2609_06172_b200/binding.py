@@ -77,6 +77,7 @@ _SIGS = {
     "tgp_model_bind": [_P, C.POINTER(ModelCfg), C.POINTER(RoleEntry), _U32, _P, _P, _U64, _U32],
     "tgp_run_reset": [_P],
     "tgp_step": [_P, _U32, _P, _U32, _U32, _P, _P, _P, _P, C.POINTER(StepStats)],
+    "tgp_expert_counts": [_P, C.POINTER(_U32), C.POINTER(_U64)],
     "tgp_managed_alloc": [C.POINTER(_P), _U64],
     "tgp_managed_free": [_P],
     "tgp_managed_evict": [_P, _U64],
@@ -248,6 +249,14 @@ class Ctx:
                                 _ptr(copy_stream), C.byref(st) if st is not None else None), "tgp_step")
         return st
 
+
+    def expert_counts(self, L, E):
+        """uint32 [steps run, L, E]: tokens routed to each expert since the last run_reset()."""
+        n = _U64()
+        self._ck(lib().tgp_expert_counts(self._h, None, C.byref(n)), "tgp_expert_counts")
+        a = np.zeros(max(1, n.value), dtype=np.uint32)
+        self._ck(lib().tgp_expert_counts(self._h, a.ctypes.data_as(C.POINTER(_U32)), C.byref(n)), "tgp_expert_counts")
+        return a[:n.value].reshape(-1, L, E)
 
     def set_op_timing(self, enable):
         self._ck(lib().tgp_set_op_timing(self._h, int(enable)), "tgp_set_op_timing")

@@ -12,6 +12,7 @@
 // A command is enqueued as soon as the op it waits on has been enqueued, so the copy stream runs as far
 // ahead of compute as ring space allows, across step boundaries too.
 #include <cuda_runtime.h>
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <vector>
@@ -27,6 +28,13 @@ struct TgpEngine {
     int32_t *tok = nullptr, *amax = nullptr;
     float *x = nullptr, *q32 = nullptr, *k32 = nullptr, *v32 = nullptr, *g32 = nullptr, *u32 = nullptr, *cos_t = nullptr, *sin_t = nullptr, *scratch = nullptr;
     char *h = nullptr, *qb = nullptr, *ob = nullptr, *ab = nullptr, *hf = nullptr;
+    // MoE
+    int32_t *topk_idx = nullptr, *erow = nullptr, *ecount = nullptr;
+    float *topk_gate = nullptr, *egate = nullptr, *y32 = nullptr, *bias_dev = nullptr;
+    char *hg = nullptr, *spill = nullptr;
+    int32_t *ecount_host = nullptr;                      // pinned mirror of the per-expert counts
+    std::vector<uint32_t> cnt;                           // counts of the layer being executed
+    int32_t cur_expert = -1;
     uint32_t max_tokens = 0;
     // run state
     std::vector<cudaEvent_t> done_ev, copied_ev;         // per op, created on first use
@@ -49,7 +57,7 @@ struct TgpEngine {
 
 static inline uint64_t up256(uint64_t x) { return (x + 255) / 256 * 256; }
 
-struct WsLayout { uint64_t tok, amax, x, h, q32, k32, v32, qb, ob, g32, u32, ab, hf, cos_t, sin_t, scratch, total; };
+struct WsLayout { uint64_t tok, amax, x, h, q32, k32, v32, qb, ob, g32, u32, ab, hf, cos_t, sin_t, scratch, topk_idx, topk_gate, erow, egate, ecount, hg, y32, bias, spill, total; };
 
 static WsLayout ws_layout(const tgp_model_cfg &c, uint64_t Mx) {
     WsLayout w{};
@@ -65,6 +73,12 @@ static WsLayout ws_layout(const tgp_model_cfg &c, uint64_t Mx) {
     w.cos_t = take((uint64_t)c.max_len * (c.Dh / 2) * 4); w.sin_t = take((uint64_t)c.max_len * (c.Dh / 2) * 4);
     uint64_t sb = 0; tgp_k_attn_scratch_bytes(&c, &sb);
     w.scratch = take(sb);
+    if (c.E) {
+        w.topk_idx = take(Mx * 2 * 4); w.topk_gate = take(Mx * 2 * 4);
+        w.erow = take((uint64_t)c.E * Mx * 4); w.egate = take((uint64_t)c.E * Mx * 4); w.ecount = take((uint64_t)c.E * 4);
+        w.hg = take(Mx * c.d * 2); w.y32 = take(Mx * c.d * 4); w.bias = take((uint64_t)c.L * c.E * 4);
+        w.spill = take(std::max<uint64_t>((uint64_t)c.F * c.d * 2, 512));        // one whole expert matrix: the largest block a fallback fetches
+    }
     w.total = o;
     return w;
 }
@@ -96,6 +110,7 @@ void tgp_engine_free(tgp_ctx *ctx) {
     if (e->t0) cudaEventDestroy(e->t0);
     if (e->t1) cudaEventDestroy(e->t1);
     if (e->wb_stream) cudaStreamDestroy(e->wb_stream);
+    if (e->ecount_host) cudaFreeHost(e->ecount_host);
     delete e;
     ctx->eng = nullptr;
 }
@@ -143,6 +158,10 @@ int tgp_model_bind(tgp_ctx *ctx, const tgp_model_cfg *cfg, const tgp_role_entry 
     ctx->cfg = c; ctx->roles.swap(rs); ctx->role_of_tensor.swap(rot);
     ctx->router_bias.assign(router_bias_host ? router_bias_host : nullptr, router_bias_host ? router_bias_host + (size_t)c.L * c.E : nullptr);
     ctx->bound = true;
+    ctx->role_index.clear();
+    for (uint32_t i = 0; i < n_roles; ++i) ctx->role_index[std::make_tuple(ctx->roles[i].kind, ctx->roles[i].layer, ctx->roles[i].expert)].push_back(i);
+    for (auto &kv : ctx->role_index)
+        std::sort(kv.second.begin(), kv.second.end(), [&](uint32_t a, uint32_t b) { return ctx->roles[a].block < ctx->roles[b].block; });
     if (!workspace_dev) return TGP_OK;
     if (!max_tokens) return TGP_E_INVAL;
     const WsLayout w = ws_layout(c, max_tokens);
@@ -157,6 +176,14 @@ int tgp_model_bind(tgp_ctx *ctx, const tgp_model_cfg *cfg, const tgp_role_entry 
     e->qb = b + w.qb; e->ob = b + w.ob; e->g32 = (float *)(b + w.g32); e->u32 = (float *)(b + w.u32); e->ab = b + w.ab; e->hf = b + w.hf;
     e->cos_t = (float *)(b + w.cos_t); e->sin_t = (float *)(b + w.sin_t); e->scratch = (float *)(b + w.scratch);
     e->max_tokens = max_tokens;
+    if (c.E) {
+        e->topk_idx = (int32_t *)(b + w.topk_idx); e->topk_gate = (float *)(b + w.topk_gate); e->erow = (int32_t *)(b + w.erow);
+        e->egate = (float *)(b + w.egate); e->ecount = (int32_t *)(b + w.ecount); e->hg = b + w.hg; e->y32 = (float *)(b + w.y32);
+        e->bias_dev = (float *)(b + w.bias); e->spill = b + w.spill;
+        CU(ctx, cudaMemcpy(e->bias_dev, ctx->router_bias.data(), (size_t)c.L * c.E * 4, cudaMemcpyHostToDevice));
+        CU(ctx, cudaHostAlloc((void **)&e->ecount_host, (size_t)c.E * 4, cudaHostAllocDefault));
+        e->cnt.assign(c.E, 0);
+    }
     CU(ctx, cudaGetDevice(&e->device));
     for (TgpPool &p : ctx->pools) {
         if (p.flags == TGP_POOL_PLAIN && !p.locked_by_us) {
@@ -180,6 +207,7 @@ int tgp_run_reset(tgp_ctx *ctx) {
     TgpEngine *e = ctx->eng;
     e->next_cmd = 0; e->next_step = 0; e->pos = 0; e->wb_pending = false; e->copy_waited_op = -1; e->tok_src = nullptr;
     e->hinted_upto = 0;
+    ctx->run_counts.clear();
     return TGP_OK;
 }
 
@@ -266,6 +294,54 @@ static int hint_ahead(tgp_ctx *ctx, size_t op_now, size_t step_end, cudaStream_t
     return TGP_OK;
 }
 
+// One weight block of expert r.expert applied to the rows routed to it.  Gate/up read the gathered rows of h,
+// down writes y32 and, with its last block, the gate-scaled rows are added into the residual stream.
+static int run_expert_block(tgp_ctx *ctx, const TgpRole &r, const void *W, uint32_t K, cudaStream_t cs) {
+    TgpEngine *e = ctx->eng;
+    const tgp_model_cfg &c = ctx->cfg;
+    const uint32_t me = e->cnt[r.expert];
+    if (!me) return TGP_OK;                                // traced but not routed to in this run: nothing to compute
+    const int32_t *rows = e->erow + (size_t)r.expert * e->max_tokens;
+    const float *gates = e->egate + (size_t)r.expert * e->max_tokens;
+    int rc = TGP_OK;
+    switch (r.kind) {
+    case TGP_K_WG:
+        if (r.row0 == 0 && (rc = tgpk_gather_rows(e->h, rows, e->hg, me, c.d, cs))) return rc;
+        return tgpk_gemm(e->hg, W, e->g32, me, r.rows, K, c.F, r.row0, 0, cs);
+    case TGP_K_WU:
+        return tgpk_gemm(e->hg, W, e->u32, me, r.rows, K, c.F, r.row0, 0, cs);
+    case TGP_K_WD:
+        if ((rc = tgpk_gemm(e->ab, W, e->y32, me, r.rows, K, c.d, r.row0, 0, cs))) return rc;
+        if (r.row0 + r.rows == c.d) rc = tgpk_scatter_add(e->x, e->y32, rows, gates, me, c.d, cs);
+        return rc;
+    default:
+        return TGP_E_MISMATCH;
+    }
+}
+
+// An expert the router chose but the trace does not list (Section IV-C: identity mismatch -> no prefetch for it):
+// its blocks are fetched one at a time into the spill buffer on the compute stream and used at once.
+static int run_expert_fallback(tgp_ctx *ctx, int32_t layer, int32_t expert, cudaStream_t cs) {
+    TgpEngine *e = ctx->eng;
+    const tgp_model_cfg &c = ctx->cfg;
+    const uint32_t kinds[3] = {TGP_K_WG, TGP_K_WU, TGP_K_WD};
+    for (uint32_t kind : kinds) {
+        auto it = ctx->role_index.find(std::make_tuple(kind, layer, expert));
+        if (it == ctx->role_index.end()) return TGP_E_MISMATCH;
+        if (kind == TGP_K_WD) { int rc = tgpk_swiglu(e->g32, e->u32, e->ab, (uint64_t)e->cnt[expert] * c.F, cs); if (rc) return rc; }
+        for (uint32_t ri : it->second) {
+            const TgpRole &r = ctx->roles[ri];
+            const TgpTensor &t = ctx->tensors[r.tensor];
+            if (t.size > std::max<uint64_t>((uint64_t)c.F * c.d * 2, 512)) return TGP_E_TOO_LARGE;
+            const char *src = ctx->pools[t.pool].host_base + t.off;
+            if (cudaMemcpyAsync(e->spill, src, t.size, ctx->pools[t.pool].flags == TGP_POOL_MANAGED ? cudaMemcpyDefault : cudaMemcpyHostToDevice, cs) != cudaSuccess) return TGP_E_CUDA;
+            int rc = run_expert_block(ctx, r, e->spill, (uint32_t)(t.size / (2ull * r.rows)), cs);
+            if (rc) return rc;
+        }
+    }
+    return TGP_OK;
+}
+
 extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_host, uint32_t B, uint32_t q_len,
                         float *logits_dev, int32_t *argmax_dev, void *compute_stream, void *copy_stream, tgp_step_stats *stats) {
     if (!ctx || !logits_dev) return TGP_E_INVAL;
@@ -285,7 +361,8 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
     cudaStream_t cs = (cudaStream_t)compute_stream, cp = (cudaStream_t)copy_stream;
     const uint32_t M = B * q_len, pos0 = e->pos;
     const uint64_t launches0 = tgpk_launches;
-    uint32_t n_cmds = 0;
+    uint32_t n_cmds = 0, n_mismatch = 0;
+    e->cur_expert = -1;
     if (stats) CU(ctx, cudaEventRecord(e->t0, cs));
     const int32_t *tok = e->amax;
     if (tokens_host) { CU(ctx, cudaMemcpyAsync(e->tok, tokens_host, (size_t)M * 4, cudaMemcpyHostToDevice, cs)); tok = e->tok; }
@@ -325,6 +402,12 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             const TgpRole &r = ctx->roles[ri];
             const uint32_t K = (uint32_t)(ctx->tensors[a.tensor].size / (2ull * r.rows));
             const void *W = where(ctx, o, 0);
+            if (r.expert >= 0) {                          // expert weight block: rows of the tokens routed to that expert
+                if ((uint32_t)r.expert >= c.E || !c.E) return tgp_fail(ctx, TGP_E_MISMATCH, "expert weight in a dense model");
+                e->cur_expert = r.expert;
+                rc = run_expert_block(ctx, r, W, K, cs);
+                break;
+            }
             switch (r.kind) {
             case TGP_K_WQ: rc = tgpk_gemm(e->h, W, e->q32, M, r.rows, K, qd, r.row0, 0, cs); break;
             case TGP_K_WK: rc = tgpk_gemm(e->h, W, e->k32, M, r.rows, K, kd, r.row0, 0, cs); break;
@@ -335,6 +418,33 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             case TGP_K_WD: rc = tgpk_gemm(e->ab, W, e->x, M, r.rows, K, c.d, r.row0, 1, cs); break;
             case TGP_K_LM: rc = tgpk_gemm(e->hf, W, logits_dev, B, r.rows, K, c.V, r.row0, 0, cs); break;
             default: return tgp_fail(ctx, TGP_E_MISMATCH, "GEMM op on a tensor that is not a weight");
+            }
+            break;
+        }
+        case TGP_OP_ROUTER: {
+            if (!c.E) return tgp_fail(ctx, TGP_E_MISMATCH, "router op in a dense model");
+            rc = tgpk_router(e->h, where(ctx, o, 0), e->bias_dev + (size_t)o.layer * c.E, e->topk_idx, e->topk_gate, e->erow, e->egate, e->ecount,
+                             M, c.d, c.E, c.topk, cs);
+            if (rc) break;
+            // the host needs the counts to size the expert launches (and to detect experts the trace does not list)
+            CU(ctx, cudaMemcpyAsync(e->ecount_host, e->ecount, (size_t)c.E * 4, cudaMemcpyDeviceToHost, cs));
+            CU(ctx, cudaStreamSynchronize(cs));
+            std::vector<uint8_t> traced(c.E, 0);
+            for (uint32_t j = i + 1; j < st.op0 + st.nops && ctx->ops[j].layer == o.layer; ++j) {
+                const TgpOp &f = ctx->ops[j];
+                if (f.kind != TGP_OP_GEMM) { if (f.kind == TGP_OP_SWIGLU) continue; break; }
+                const int32_t fr = ctx->role_of_tensor[ctx->acc[f.acc0].tensor];
+                if (fr >= 0 && ctx->roles[fr].expert >= 0) traced[ctx->roles[fr].expert] = 1;
+            }
+            const size_t slot = ((size_t)e->next_step * c.L + o.layer) * c.E;
+            if (ctx->run_counts.size() < slot + c.E) ctx->run_counts.resize(slot + c.E, 0);
+            for (uint32_t x = 0; x < c.E; ++x) {
+                e->cnt[x] = (uint32_t)e->ecount_host[x];
+                ctx->run_counts[slot + x] = e->cnt[x];
+                if (e->cnt[x] && !traced[x]) {            // run-time access the trace does not have: fetch synchronously, count it
+                    if ((rc = run_expert_fallback(ctx, o.layer, (int32_t)x, cs))) return tgp_fail(ctx, rc, "expert fallback failed");
+                    ++n_mismatch;
+                }
             }
             break;
         }
@@ -354,7 +464,8 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             break;
         }
         case TGP_OP_SWIGLU:
-            rc = tgpk_swiglu(e->g32, e->u32, e->ab, (uint64_t)M * c.F, cs);
+            if (c.E) { if (e->cur_expert >= 0 && e->cnt[e->cur_expert]) rc = tgpk_swiglu(e->g32, e->u32, e->ab, (uint64_t)e->cnt[e->cur_expert] * c.F, cs); }
+            else rc = tgpk_swiglu(e->g32, e->u32, e->ab, (uint64_t)M * c.F, cs);
             break;
         case TGP_OP_ARGMAX:
             rc = tgpk_argmax(logits_dev, e->amax, B, c.V, cs);
@@ -383,7 +494,7 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
         if (ring) CU(ctx, cudaStreamSynchronize(e->wb_stream));
         const uint64_t *tot = &ctx->plan.totals[(size_t)(e->next_step - 1) * 4];
         stats->h2d_bytes = ring ? tot[0] : 0; stats->d2h_bytes = ring ? tot[1] : 0; stats->zc_bytes = tot[2];
-        stats->n_cmds = n_cmds; stats->n_launches = (uint32_t)(tgpk_launches - launches0); stats->n_mismatch = 0;
+        stats->n_cmds = n_cmds; stats->n_launches = (uint32_t)(tgpk_launches - launches0); stats->n_mismatch = n_mismatch;
         CU(ctx, cudaEventElapsedTime(&stats->step_ms, e->t0, e->t1));
     }
     return TGP_OK;
@@ -428,4 +539,13 @@ extern "C" int tgp_managed_evict(void *ptr, uint64_t bytes) {
     if (!ptr || !bytes) return TGP_E_INVAL;
     if (cudaMemPrefetchAsync(ptr, bytes, cudaCpuDeviceId, 0) != cudaSuccess) { cudaGetLastError(); return TGP_E_CUDA; }
     return cudaDeviceSynchronize() == cudaSuccess ? TGP_OK : TGP_E_CUDA;
+}
+
+// Tokens routed to each expert in the run since the last tgp_run_reset(): [steps run, L, E] (MoE only).  This is
+// the profile a first pass records so that the next trace lists exactly the experts that are used.
+extern "C" int tgp_expert_counts(tgp_ctx *ctx, uint32_t *out, uint64_t *n) {
+    if (!ctx || !n) return TGP_E_INVAL;
+    if (out) { if (*n < ctx->run_counts.size()) return TGP_E_INVAL; memcpy(out, ctx->run_counts.data(), ctx->run_counts.size() * 4); }
+    *n = ctx->run_counts.size();
+    return TGP_OK;
 }

@@ -250,7 +250,8 @@ int tgp_plan(tgp_ctx *ctx) {
         if (pl.cls[i] == CLS_LINK)
             for (uint32_t k = 0; k < o.nacc; ++k) {
                 const tgp_access &a = ctx->acc[o.acc0 + k];
-                pl.crit[a.tensor] = 1; pl.score[a.tensor] += a.touched_bytes;
+                // link bytes residency would save: what the op touches, plus the whole-tensor write-back a write causes
+                pl.crit[a.tensor] = 1; pl.score[a.tensor] += a.touched_bytes + ((a.mode & TGP_W) ? ten[a.tensor].size : 0);
             }
     }
     // zero-copy: read-only, accessed, and every access sparse

@@ -4,6 +4,7 @@
 #include <string>
 #include <vector>
 #include <map>
+#include <tuple>
 #include "tgp.h"
 
 struct TgpPool { char *host_base; uint64_t bytes; uint32_t flags; char *dev_alias; bool locked_by_us; };
@@ -67,6 +68,8 @@ struct tgp_ctx {
     std::vector<TgpRole> roles;
     std::vector<int32_t> role_of_tensor;                 // tensor id -> index in roles, or -1
     std::vector<float> router_bias;
+    std::map<std::tuple<uint32_t, int32_t, int32_t>, std::vector<uint32_t>> role_index;   // (kind, layer, expert) -> roles by block
+    std::vector<uint32_t> run_counts;                    // MoE: tokens routed per (step, layer, expert) in the current run
     TgpEngine *eng = nullptr;
     void *arena = nullptr; uint64_t arena_bytes = 0;
     std::string err;

@@ -367,7 +367,132 @@ __global__ void __launch_bounds__(1024) argmax_kernel(const float *__restrict__ 
     }
 }
 
+// ---- MoE: router, top-2, gates (one warp per token) ------------------------------------------------------
+// logits[e] = sum_k h[m,k] * Wr[e,k] + bias[e] in fp32; the two largest (ties: lower expert id); gates = softmax
+// over those two logits.
+template <int E>
+__global__ void __launch_bounds__(256) router_kernel(const bf16 *__restrict__ h, const bf16 *__restrict__ Wr, const float *__restrict__ bias,
+                                                     int32_t *__restrict__ idx, float *__restrict__ gate, uint32_t M, uint32_t d, uint32_t topk) {
+    const uint32_t m = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (m >= M) return;
+    float acc[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) acc[e] = 0.f;
+    for (uint32_t k = lane * 8; k < d; k += 256) {
+        float xf[8];
+        unpack8(*reinterpret_cast<const uint4 *>(h + (size_t)m * d + k), xf);
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            float wf[8];
+            unpack8(__ldg(reinterpret_cast<const uint4 *>(Wr + (size_t)e * d + k)), wf);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[e] = fmaf(xf[i], wf[i], acc[e]);
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < E; ++e) acc[e] = warp_sum(acc[e]) + bias[e];
+    if (lane == 0) {
+        int i0 = 0;                                    // strict > while visiting ascending ids keeps the lower id on ties
+#pragma unroll
+        for (int e = 1; e < E; ++e) if (acc[e] > acc[i0]) i0 = e;
+        if (E == 1 || topk == 1) {
+            idx[2 * m] = i0; idx[2 * m + 1] = -1;
+            gate[2 * m] = 1.0f; gate[2 * m + 1] = 0.0f;
+        } else {
+            int i1 = i0 == 0 ? 1 : 0;
+#pragma unroll
+            for (int e = 0; e < E; ++e) if (e != i0 && acc[e] > acc[i1]) i1 = e;
+            const float e1 = expf(acc[i1] - acc[i0]);
+            idx[2 * m] = i0; idx[2 * m + 1] = i1;
+            gate[2 * m] = 1.0f / (1.0f + e1); gate[2 * m + 1] = e1 / (1.0f + e1);
+        }
+    }
+}
+
+// Tokens of expert e in ascending token order: rows[e*M + pos] = m, gates[e*M + pos] = that token's gate for e.
+// One block per expert walks the tokens in chunks; positions come from a block-wide exclusive scan, so the
+// grouping is deterministic.  topk = number of routed slots per token (1 or 2).
+__global__ void __launch_bounds__(1024) route_fill_kernel(const int32_t *__restrict__ idx, const float *__restrict__ gate, int32_t *__restrict__ rows,
+                                                          float *__restrict__ gates, int32_t *__restrict__ counts, uint32_t M, uint32_t topk) {
+    __shared__ uint32_t warp_tot[32];
+    __shared__ uint32_t base;
+    const uint32_t e = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) base = 0;
+    __syncthreads();
+    for (uint32_t m0 = 0; m0 < M; m0 += blockDim.x) {
+        const uint32_t m = m0 + threadIdx.x;
+        int slot = -1;
+        if (m < M) {
+            if (idx[2 * m] == (int)e) slot = 0;
+            else if (topk > 1 && idx[2 * m + 1] == (int)e) slot = 1;
+        }
+        const uint32_t bal = __ballot_sync(0xffffffffu, slot >= 0);
+        const uint32_t before = __popc(bal & ((1u << lane) - 1));
+        if (lane == 0) warp_tot[warp] = __popc(bal);
+        __syncthreads();
+        uint32_t woff = 0;
+        for (uint32_t w = 0; w < warp; ++w) woff += warp_tot[w];
+        const uint32_t b0 = base;
+        if (slot >= 0) { rows[(size_t)e * M + b0 + woff + before] = (int32_t)m; gates[(size_t)e * M + b0 + woff + before] = gate[2 * m + slot]; }
+        __syncthreads();
+        if (threadIdx.x == 0) { uint32_t t = 0; for (uint32_t w = 0; w < (blockDim.x >> 5); ++w) t += warp_tot[w]; base = b0 + t; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) counts[e] = (int32_t)base;
+}
+
+__global__ void gather_rows_kernel(const bf16 *__restrict__ src, const int32_t *__restrict__ rows, bf16 *__restrict__ dst, uint32_t d) {
+    const uint4 *s = reinterpret_cast<const uint4 *>(src + (size_t)rows[blockIdx.x] * d);
+    uint4 *o = reinterpret_cast<uint4 *>(dst + (size_t)blockIdx.x * d);
+    for (uint32_t i = threadIdx.x; i < d / 8; i += blockDim.x) o[i] = s[i];
+}
+
+// x[rows[i], :] += gates[i] * y[i, :]   (each token appears at most once per expert: no write conflicts)
+__global__ void scatter_add_kernel(float *__restrict__ x, const float *__restrict__ y, const int32_t *__restrict__ rows, const float *__restrict__ gates, uint32_t d) {
+    const float g = gates[blockIdx.x];
+    float4 *o = reinterpret_cast<float4 *>(x + (size_t)rows[blockIdx.x] * d);
+    const float4 *s = reinterpret_cast<const float4 *>(y + (size_t)blockIdx.x * d);
+    for (uint32_t i = threadIdx.x; i < d / 4; i += blockDim.x) {
+        float4 a = o[i];
+        const float4 b = s[i];
+        a.x += g * b.x; a.y += g * b.y; a.z += g * b.z; a.w += g * b.w;
+        o[i] = a;
+    }
+}
+
 // ============================ launchers (internal) ===================================================
+int tgpk_router(const void *h, const void *Wr, const float *bias, int32_t *idx, float *gate, int32_t *rows, float *gates, int32_t *counts,
+                uint32_t M, uint32_t d, uint32_t E, uint32_t topk, cudaStream_t st) {
+    if (!M) return TGP_OK;
+    if (d % 8 || topk < 1 || topk > 2) return TGP_E_INVAL;
+    const uint32_t blocks = (M + 7) / 8;
+    switch (E) {
+    case 1: router_kernel<1><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
+    case 2: router_kernel<2><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
+    case 4: router_kernel<4><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
+    case 8: router_kernel<8><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
+    case 16: router_kernel<16><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
+    default: return TGP_E_INVAL;
+    }
+    route_fill_kernel<<<E, 1024, 0, st>>>(idx, gate, rows, gates, counts, M, topk);
+    LAUNCH_CHECK(2);
+    return TGP_OK;
+}
+
+int tgpk_gather_rows(const void *src, const int32_t *rows, void *dst, uint32_t m, uint32_t d, cudaStream_t st) {
+    if (!m) return TGP_OK;
+    gather_rows_kernel<<<m, 128, 0, st>>>((const bf16 *)src, rows, (bf16 *)dst, d);
+    LAUNCH_CHECK(1);
+    return TGP_OK;
+}
+
+int tgpk_scatter_add(float *x, const float *y, const int32_t *rows, const float *gates, uint32_t m, uint32_t d, cudaStream_t st) {
+    if (!m) return TGP_OK;
+    scatter_add_kernel<<<m, 256, 0, st>>>(x, y, rows, gates, d);
+    LAUNCH_CHECK(1);
+    return TGP_OK;
+}
+
 int tgpk_embed(const void *table, const int32_t *tok, float *x, uint32_t M, uint32_t d, cudaStream_t st) {
     if (!M) return TGP_OK;
     if (d % 8) return TGP_E_INVAL;

@@ -46,6 +46,7 @@ def run(cfg, lay, machine, dev, fill, variants=(tb.VAR_MANAGED_DEMAND, tb.VAR_MA
             hold = None
             info = {"decode_steps": T}
             if ballast:
+                tb.managed_evict(pool.ptr, lay.pool_bytes)      # resident managed pages would count as used memory
                 torch.cuda.synchronize()
                 free, total = torch.cuda.mem_get_info(dev)
                 nb = free - lay.budget - slack

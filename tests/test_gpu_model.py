@@ -194,3 +194,98 @@ def test_managed_variants_give_the_same_bits_as_the_explicit_ring():
     finally:
         torch.cuda.synchronize()
         mp.free()
+
+
+MOE = si.ModelConfig("moe_small", L=2, d=256, Hq=4, Hkv=2, Dh=64, F=512, V=512, B=3, S=9, T=4, TK=4, E=4, topk=2, seed=77,
+                     budget_rule="half_w")
+
+
+def _run_steps(r, cfg, prompt, forced, T):
+    """prefill + T teacher-forced decode steps with statistics; returns (logits per step, mismatches per step)."""
+    r.reset()
+    out, mism = [], []
+    st = r.step(tb.PREFILL, np.ascontiguousarray(prompt, dtype=np.int32), cfg.S, want_stats=True)
+    for t in range(T + 1):
+        out.append(r.logits.cpu().numpy().copy())
+        mism.append(st.n_mismatch)
+        if t < T:
+            st = r.step(tb.DECODE, np.ascontiguousarray(forced[:, t:t + 1], dtype=np.int32), 1, want_stats=True)
+    r.sync()
+    return out, mism
+
+
+def test_moe_profile_pass_planned_run_and_mismatch_fallback():
+    """Mixture-of-experts path: (1) a profile pass with every expert traced records the routed-token counts, which
+    must equal the oracle's routing; (2) the run planned from that profile matches the oracle's logits with no
+    fallback; (3) with an expert missing from the trace the engine fetches it synchronously, counts the mismatch,
+    and still produces the same logits."""
+    cfg = MOE
+    lay = si.build_layout(cfg, cap=64 << 10)
+    bias = si.router_bias(cfg)
+    pool = pinned_pool(lay.pool_bytes)
+    si.fill_pool(lay, pool.numpy())
+    om = forward.OracleModel(cfg, si.weights_as_bits(lay), bias)
+    prompt = si.prompt_tokens(cfg)
+    ref, toks = om.generate(prompt, cfg.T)
+    want_counts = np.array([[c.tolist() for c in step] for step in om.expert_counts], dtype=np.uint32)     # [steps, L, E]
+    assert want_counts.shape == (1 + cfg.T, cfg.L, cfg.E) and (want_counts.sum(axis=2) == cfg.topk * np.array([cfg.B * cfg.S] + [cfg.B] * cfg.T)[:, None]).all()
+    s = Session(lay, MACHINE, pool_base=pool.data_ptr(), pool_flags=tb.POOL_PINNED, router_bias=bias)
+    # (1) profile pass: all experts traced
+    s.plan(expert_counts=np.ones_like(want_counts))
+    r = Runner(s, cfg.B * cfg.S)
+    got, mism = _run_steps(r, cfg, prompt, toks, cfg.T)
+    assert sum(mism) == 0
+    counts = s.ctx.expert_counts(cfg.L, cfg.E)
+    assert np.array_equal(counts, want_counts)
+    check_logits(got, ref)
+    # (2) plan from the profile: only the experts in use are staged
+    blobs_all = s.ctx.plan_blobs()
+    blobs = s.plan(expert_counts=counts)
+    ops, steps = trace.run_trace(lay, expert_counts=want_counts)
+    want = policy.plan(lay.tensors, ops, steps, policy.Machine(**MACHINE), lay.budget).blobs()
+    assert blobs == want
+    validate.check(lay.tensors, ops, steps, lay.budget, blobs)
+    got2, mism2 = _run_steps(r, cfg, prompt, toks, cfg.T)
+    assert sum(mism2) == 0
+    check_logits(got2, ref)
+    if (want_counts == 0).any():
+        assert len(blobs["commands"]) < len(blobs_all["commands"])
+    # (3) drop one expert that is in use from the trace of the first decode step, layer 1
+    e_used = int(np.argmax(want_counts[1, 1]))
+    wrong = counts.copy()
+    wrong[1, 1, e_used] = 0
+    s.plan(expert_counts=wrong)
+    got3, mism3 = _run_steps(r, cfg, prompt, toks, cfg.T)
+    assert mism3[1] == 1 and sum(mism3) == 1
+    check_logits(got3, ref)
+    s.close()
+
+
+def test_router_topk_ties_and_single_expert_equals_dense():
+    """E = 1, top-1 routes every token to the one expert with gate 1: same logits as the dense model with those weights."""
+    dense = replace(MOE, E=0, topk=0, L=1)
+    moe1 = replace(MOE, E=1, topk=1, L=1)
+    lay_d, lay_m = si.build_layout(dense, cap=64 << 10), si.build_layout(moe1, cap=64 << 10)
+    pd, pm = pinned_pool(lay_d.pool_bytes), pinned_pool(lay_m.pool_bytes)
+    si.fill_pool(lay_d, pd.numpy())
+    si.fill_pool(lay_m, pm.numpy())
+    # give the single expert the dense FFN's weights (block by block) and share all other weights
+    for t in lay_m.tensors:
+        key = (t.kind, t.layer, -1 if t.expert == 0 else t.expert)
+        if t.kind == si.K_ROUTER or t.kind >= si.K_KT:
+            continue
+        src = lay_d.blocks(*key)[t.block]
+        assert src.size == t.size
+        pm.numpy()[t.pool_off:t.pool_off + t.size] = pd.numpy()[src.pool_off:src.pool_off + src.size]
+    prompt = si.prompt_tokens(dense)
+    forced = (np.arange(dense.B * dense.T, dtype=np.int32).reshape(dense.B, dense.T) * 131 + 5) % dense.V
+    sd = Session(lay_d, MACHINE, pool_base=pd.data_ptr(), pool_flags=tb.POOL_PINNED)
+    sd.plan()
+    a, _ = Runner(sd, dense.B * dense.S).generate(prompt, dense.T, forced=forced)
+    sm = Session(lay_m, MACHINE, pool_base=pm.data_ptr(), pool_flags=tb.POOL_PINNED, router_bias=np.zeros((1, 1), np.float32))
+    counts = np.array([[[dense.B * dense.S]]] + [[[dense.B]]] * dense.T, dtype=np.uint32)
+    sm.plan(expert_counts=counts)
+    b, _ = Runner(sm, dense.B * dense.S).generate(prompt, dense.T, forced=forced)
+    for x, y in zip(a, b):
+        assert np.abs(x - y).max() < 1e-5
+    sd.close(), sm.close()
