@@ -424,7 +424,7 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
         case TGP_OP_ROUTER: {
             if (!c.E) return tgp_fail(ctx, TGP_E_MISMATCH, "router op in a dense model");
             rc = tgpk_router(e->h, where(ctx, o, 0), e->bias_dev + (size_t)o.layer * c.E, e->topk_idx, e->topk_gate, e->erow, e->egate, e->ecount,
-                             M, c.d, c.E, c.topk, cs);
+                             M, e->max_tokens, c.d, c.E, c.topk, cs);
             if (rc) break;
             // the host needs the counts to size the expert launches (and to detect experts the trace does not list)
             CU(ctx, cudaMemcpyAsync(e->ecount_host, e->ecount, (size_t)c.E * 4, cudaMemcpyDeviceToHost, cs));

@@ -409,11 +409,11 @@ __global__ void __launch_bounds__(256) router_kernel(const bf16 *__restrict__ h,
     }
 }
 
-// Tokens of expert e in ascending token order: rows[e*M + pos] = m, gates[e*M + pos] = that token's gate for e.
+// Tokens of expert e in ascending token order: rows[e*stride + pos] = m, gates[e*stride + pos] = that token's gate for e.
 // One block per expert walks the tokens in chunks; positions come from a block-wide exclusive scan, so the
 // grouping is deterministic.  topk = number of routed slots per token (1 or 2).
 __global__ void __launch_bounds__(1024) route_fill_kernel(const int32_t *__restrict__ idx, const float *__restrict__ gate, int32_t *__restrict__ rows,
-                                                          float *__restrict__ gates, int32_t *__restrict__ counts, uint32_t M, uint32_t topk) {
+                                                          float *__restrict__ gates, int32_t *__restrict__ counts, uint32_t M, uint32_t stride, uint32_t topk) {
     __shared__ uint32_t warp_tot[32];
     __shared__ uint32_t base;
     const uint32_t e = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -433,7 +433,7 @@ __global__ void __launch_bounds__(1024) route_fill_kernel(const int32_t *__restr
         uint32_t woff = 0;
         for (uint32_t w = 0; w < warp; ++w) woff += warp_tot[w];
         const uint32_t b0 = base;
-        if (slot >= 0) { rows[(size_t)e * M + b0 + woff + before] = (int32_t)m; gates[(size_t)e * M + b0 + woff + before] = gate[2 * m + slot]; }
+        if (slot >= 0) { rows[(size_t)e * stride + b0 + woff + before] = (int32_t)m; gates[(size_t)e * stride + b0 + woff + before] = gate[2 * m + slot]; }
         __syncthreads();
         if (threadIdx.x == 0) { uint32_t t = 0; for (uint32_t w = 0; w < (blockDim.x >> 5); ++w) t += warp_tot[w]; base = b0 + t; }
         __syncthreads();
@@ -462,7 +462,7 @@ __global__ void scatter_add_kernel(float *__restrict__ x, const float *__restric
 
 // ============================ launchers (internal) ===================================================
 int tgpk_router(const void *h, const void *Wr, const float *bias, int32_t *idx, float *gate, int32_t *rows, float *gates, int32_t *counts,
-                uint32_t M, uint32_t d, uint32_t E, uint32_t topk, cudaStream_t st) {
+                uint32_t M, uint32_t stride, uint32_t d, uint32_t E, uint32_t topk, cudaStream_t st) {
     if (!M) return TGP_OK;
     if (d % 8 || topk < 1 || topk > 2) return TGP_E_INVAL;
     const uint32_t blocks = (M + 7) / 8;
@@ -474,7 +474,7 @@ int tgpk_router(const void *h, const void *Wr, const float *bias, int32_t *idx, 
     case 16: router_kernel<16><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
     default: return TGP_E_INVAL;
     }
-    route_fill_kernel<<<E, 1024, 0, st>>>(idx, gate, rows, gates, counts, M, topk);
+    route_fill_kernel<<<E, 1024, 0, st>>>(idx, gate, rows, gates, counts, M, stride, topk);
     LAUNCH_CHECK(2);
     return TGP_OK;
 }

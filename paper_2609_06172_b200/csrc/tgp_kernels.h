@@ -18,9 +18,9 @@ int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb,
 int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *ob, const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0,
               float *scratch, cudaStream_t st);
 int tgpk_swiglu(const float *g, const float *u, void *ab, uint64_t n, cudaStream_t st);
-// MoE: router logits + top-k (1 or 2) + gates, then per-expert token lists rows[e*M + i], gates[e*M + i], counts[e]
+// MoE: router logits + top-k (1 or 2) + gates, then per-expert token lists rows[e*stride + i], gates[e*stride + i], counts[e]
 int tgpk_router(const void *h, const void *Wr, const float *bias, int32_t *idx, float *gate, int32_t *rows, float *gates, int32_t *counts,
-                uint32_t M, uint32_t d, uint32_t E, uint32_t topk, cudaStream_t st);
+                uint32_t M, uint32_t stride, uint32_t d, uint32_t E, uint32_t topk, cudaStream_t st);
 int tgpk_gather_rows(const void *src, const int32_t *rows, void *dst, uint32_t m, uint32_t d, cudaStream_t st);
 int tgpk_scatter_add(float *x, const float *y, const int32_t *rows, const float *gates, uint32_t m, uint32_t d, cudaStream_t st);
 int tgpk_argmax(const float *logits, int32_t *out, uint32_t B, uint32_t V, cudaStream_t st);
