@@ -219,6 +219,9 @@ int  tgp_k_gemm(const void *A_dev, const void *W_dev, float *C_dev, uint32_t M, 
 /* Which kernel serves M > 16: 0 (default) the tcgen05 tensor-core GEMM, 1 the CUDA-core tile kernel (an on-device
  * cross-check).  M <= 16 always takes the weight-streaming GEMV.  Process-wide. */
 int  tgp_k_gemm_select(int impl);
+/* Which kernel serves attention with q_len >= 16: 0 (default) the tensor-core flash-style kernel, 1 the
+ * warp-per-query-row CUDA-core kernel (an on-device cross-check).  Process-wide. */
+int  tgp_k_attn_select(int impl);
 /* Error word of the tensor-core GEMM: 0, or (role << 8 | stage) of the first bounded wait that ran out
  * (role 1 TMA producer, 2 MMA issuer, 3 epilogue).  Synchronous. */
 int  tgp_k_gemm_status(int *error_code);

@@ -87,6 +87,7 @@ _SIGS = {
     "tgp_k_rmsnorm": [_P, _U32, _P, _P, _U32, _U32, C.c_float, _P],
     "tgp_k_gemm": [_P, _P, _P, _U32, _U32, _U32, _U32, _U32, C.c_int, _P],
     "tgp_k_gemm_select": [C.c_int],
+    "tgp_k_attn_select": [C.c_int],
     "tgp_k_gemm_status": [C.POINTER(C.c_int)],
     "tgp_k_rope_tables": [_U32, _U32, C.c_float, _P, _P],
     "tgp_k_rope_kv": [_P, _P, _P, _P, C.POINTER(_P), C.POINTER(_P), _U32, _P, _P, C.POINTER(ModelCfg), _U32, _U32, _U32, _P],
@@ -316,6 +317,10 @@ def k_gemm(A, W, Cout, M, n, K, ldc, col0, accumulate, stream=None):
 
 def k_gemm_select(impl):
     _k(lib().tgp_k_gemm_select(impl), "tgp_k_gemm_select")
+
+
+def k_attn_select(impl):
+    _k(lib().tgp_k_attn_select(impl), "tgp_k_attn_select")
 
 
 def k_gemm_status():

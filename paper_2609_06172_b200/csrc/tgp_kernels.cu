@@ -571,6 +571,8 @@ int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb,
     return TGP_OK;
 }
 
+static int g_attn_impl = 0;      // 0: tensor cores for q_len >= 16; 1: warp-per-row CUDA-core kernel (an on-device cross-check)
+
 int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *ob, const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0,
               float *scratch, cudaStream_t st) {
     if (!B || !q_len) return TGP_OK;
@@ -587,6 +589,8 @@ int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *
             attn_decode_merge_kernel<128><<<dim3(c->Hq, B), 128, 0, st>>>(a);
         }
         tgpk_launches += 1;
+    } else if (q_len >= 16 && g_attn_impl == 0) {
+        return tgpk_attn_prefill_tc(qb, tiles, ob, c, B, q_len, pos0, st);
     } else {
         dim3 grid((q_len + 3) / 4, c->Hq, B);
         if (c->Dh == 64) attn_rows_kernel<64><<<grid, 128, 0, st>>>(a);
@@ -631,6 +635,12 @@ int tgp_k_embed(const void *table, const int32_t *tok_dev, float *x_dev, uint32_
 int tgp_k_rmsnorm(const float *x_dev, uint32_t ldx, const void *g_dev, void *h_dev, uint32_t M, uint32_t d, float eps, void *stream) {
     if (!x_dev || !g_dev || !h_dev) return TGP_E_INVAL;
     return tgpk_rmsnorm(x_dev, ldx, g_dev, h_dev, M, d, eps, (cudaStream_t)stream);
+}
+
+int tgp_k_attn_select(int impl) {
+    if (impl != 0 && impl != 1) return TGP_E_INVAL;
+    g_attn_impl = impl;
+    return TGP_OK;
 }
 
 int tgp_k_gemm_select(int impl) {
