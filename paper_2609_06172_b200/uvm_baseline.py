@@ -28,8 +28,10 @@ class ManagedPool:
 
 
 def run(cfg, lay, machine, dev, fill, variants=(tb.VAR_MANAGED_DEMAND, tb.VAR_MANAGED_HINTS), decode_cap=16, slack=768 << 20, ballast=True):
-    """Returns {variant name: {...}}.  `fill(layout, uint8 array)` writes the pool contents.  Capacity: after the
-    workspace is allocated, everything but budget + slack of the free device memory is held by a ballast tensor.
+    """Returns {variant name: {...}}.  `fill(layout, uint8 array)` writes the pool contents.  Capacity: the workspace
+    and then a ballast tensor are allocated ONCE, before the GPU has touched the managed pool, so that budget + slack
+    bytes of device memory are all the managed pages can ever occupy; both variants then run under that same cap
+    (the driver caches chunks it evicted, so a cap computed after a managed run would be too generous).
     Decode is capped at `decode_cap` steps (demand paging under 2x oversubscription is slow); rates are per step."""
     torch.cuda.set_device(dev)
     out = {}
@@ -38,26 +40,25 @@ def run(cfg, lay, machine, dev, fill, variants=(tb.VAR_MANAGED_DEMAND, tb.VAR_MA
         fill(lay, pool.numpy())
         T = min(cfg.T, decode_cap)
         prompt = np.ascontiguousarray(_prompt(cfg))
+        s = Session(lay, machine, pool_base=pool.ptr, pool_flags=tb.POOL_MANAGED)
+        s.plan(T=T, variant=variants[0])
+        r = Runner(s, cfg.B * cfg.S, device=str(dev), arena=False)
+        hold, cap = None, {}
+        if ballast:
+            torch.cuda.synchronize()
+            free, total = torch.cuda.mem_get_info(dev)
+            nb = free - lay.budget - slack
+            if nb > 0:
+                try:
+                    hold = torch.empty(nb, dtype=torch.uint8, device=dev)
+                    cap["ballast_bytes"] = int(nb)
+                except RuntimeError as ex:
+                    cap["ballast"] = f"not allocated: {ex}"
+            cap["device_bytes_left_for_managed_pages"] = int(torch.cuda.mem_get_info(dev)[0])
         for var in variants:
             name = "managed_demand" if var == tb.VAR_MANAGED_DEMAND else "managed_hints"
-            s = Session(lay, machine, pool_base=pool.ptr, pool_flags=tb.POOL_MANAGED)
             s.plan(T=T, variant=var)
-            r = Runner(s, cfg.B * cfg.S, device=str(dev), arena=False)
-            hold = None
-            info = {"decode_steps": T}
-            if ballast:
-                tb.managed_evict(pool.ptr, lay.pool_bytes)      # resident managed pages would count as used memory
-                torch.cuda.synchronize()
-                free, total = torch.cuda.mem_get_info(dev)
-                nb = free - lay.budget - slack
-                if nb > 0:
-                    try:
-                        hold = torch.empty(nb, dtype=torch.uint8, device=dev)
-                        info["ballast_bytes"] = int(nb)
-                    except RuntimeError as ex:
-                        info["ballast"] = f"not allocated: {ex}"
-                free2, _ = torch.cuda.mem_get_info(dev)
-                info["free_device_bytes_during_run"] = int(free2)
+            info = {"decode_steps": T, **cap}
             times = []
             for rep in range(2):                          # first pass warms code paths; second is reported
                 tb.managed_evict(pool.ptr, lay.pool_bytes)
@@ -71,10 +72,10 @@ def run(cfg, lay, machine, dev, fill, variants=(tb.VAR_MANAGED_DEMAND, tb.VAR_MA
                          "decode_tok_s": cfg.B * T / (sum(times[1:]) * 1e-3) if T else None,
                          "prefill_tok_s": cfg.B * cfg.S / (times[0] * 1e-3)})
             out[name] = info
-            del hold
-            s.close()
-            del r
-            torch.cuda.empty_cache()
+        del hold
+        s.close()
+        del r
+        torch.cuda.empty_cache()
     finally:
         torch.cuda.synchronize()
         pool.free()
