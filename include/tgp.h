@@ -219,6 +219,9 @@ int  tgp_k_gemm(const void *A_dev, const void *W_dev, float *C_dev, uint32_t M, 
 /* Which kernel serves M > 16: 0 (default) the tcgen05 tensor-core GEMM, 1 the CUDA-core tile kernel (an on-device
  * cross-check).  M <= 16 always takes the weight-streaming GEMV.  Process-wide. */
 int  tgp_k_gemm_select(int impl);
+/* Tensor-core GEMM variant: 0 (default) picks by problem size, 1 forces the 128x128 one-tile-per-CTA kernel,
+ * 2 forces the persistent 128x256 kernel with double-buffered accumulators.  Process-wide; for tests and timing. */
+int  tgp_k_gemm_tc_variant(int variant);
 /* Which kernel serves attention with q_len >= 16: 0 (default) the tensor-core flash-style kernel, 1 the
  * warp-per-query-row CUDA-core kernel (an on-device cross-check).  Process-wide. */
 int  tgp_k_attn_select(int impl);

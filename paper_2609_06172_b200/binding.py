@@ -88,6 +88,7 @@ _SIGS = {
     "tgp_k_gemm": [_P, _P, _P, _U32, _U32, _U32, _U32, _U32, C.c_int, _P],
     "tgp_k_gemm_select": [C.c_int],
     "tgp_k_attn_select": [C.c_int],
+    "tgp_k_gemm_tc_variant": [C.c_int],
     "tgp_k_gemm_status": [C.POINTER(C.c_int)],
     "tgp_k_rope_tables": [_U32, _U32, C.c_float, _P, _P],
     "tgp_k_rope_kv": [_P, _P, _P, _P, C.POINTER(_P), C.POINTER(_P), _U32, _P, _P, C.POINTER(ModelCfg), _U32, _U32, _U32, _P],
@@ -321,6 +322,10 @@ def k_gemm_select(impl):
 
 def k_attn_select(impl):
     _k(lib().tgp_k_attn_select(impl), "tgp_k_attn_select")
+
+
+def k_gemm_tc_variant(v):
+    _k(lib().tgp_k_gemm_tc_variant(v), "tgp_k_gemm_tc_variant")
 
 
 def k_gemm_status():

@@ -208,6 +208,143 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
     }
 }
 
+// ---- persistent variant for large problems ------------------------------------------------------------------
+// One CTA per SM walks 128 x 256 tiles (grouped order as above).  Four TMA stages of 48 KB; the TMEM holds two
+// 256-column accumulators, so the MMA warp starts the next tile while the four epilogue warps drain the previous
+// one (acc_full / acc_empty barriers per buffer).  Same bounded waits and error word as the kernel above.
+constexpr int P_BN = 256, P_STAGES = 4;
+
+__global__ void __launch_bounds__(192, 1) gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                                                                    float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
+    extern __shared__ uint8_t smem_raw[];
+    constexpr int A_BYTES = BM * BK * 2, B_BYTES = P_BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + P_STAGES * STAGE_BYTES);
+    uint64_t *empty = full + P_STAGES;
+    uint64_t *acc_full = empty + P_STAGES;           // [2]
+    uint64_t *acc_empty = acc_full + 2;              // [2]
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+    volatile uint32_t *failed = tmem_slot + 1;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t num_k = (K + BK - 1) / BK;
+    const uint32_t tiles_m = (M + BM - 1) / BM, tiles_n = (n + P_BN - 1) / P_BN, tiles = tiles_m * tiles_n;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < P_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+        *failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    auto tile_origin = [&](uint32_t tile, uint32_t &m0, uint32_t &n0) {
+        const uint32_t group = tile / (GROUP_M * tiles_n), first_m = group * GROUP_M;
+        const uint32_t rows_in_group = min((uint32_t)GROUP_M, tiles_m - first_m);
+        const uint32_t in_group = tile - group * GROUP_M * tiles_n;
+        m0 = (first_m + in_group % rows_in_group) * BM;
+        n0 = (in_group / rows_in_group) * P_BN;
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0, armed = 0;
+            bool ok = true;
+            for (uint32_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
+                uint32_t m0, n0;
+                tile_origin(tile, m0, n0);
+                for (uint32_t kb = 0; kb < num_k; ++kb, ++it) {
+                    const uint32_t s = it % P_STAGES, ph = (it / P_STAGES) & 1;
+                    if (*failed || !mbar_wait(&empty[s], ph ^ 1, failed)) { if (!*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, (1 << 8) | (int)s); } ok = false; break; }
+                    mbar_expect_tx(&full[s], STAGE_BYTES);
+                    tma_load_2d(smem + s * STAGE_BYTES, &tmA, (int)(kb * BK), (int)m0, &full[s]);
+                    tma_load_2d(smem + s * STAGE_BYTES + A_BYTES, &tmB, (int)(kb * BK), (int)n0, &full[s]);
+                    armed = it + 1;
+                }
+            }
+            if (*failed) {
+                volatile uint32_t never = 0;
+                for (uint32_t k = armed > P_STAGES ? armed - P_STAGES : 0; k < armed; ++k) mbar_wait(&full[k % P_STAGES], (k / P_STAGES) & 1, &never);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc(P_BN);
+            uint32_t it = 0, lt = 0;
+            bool ok = true;
+            for (uint32_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++lt) {
+                const uint32_t buf = lt & 1, use = lt >> 1;
+                if (*failed || !mbar_wait(&acc_empty[buf], (use & 1) ^ 1, failed)) { if (!*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, (2 << 8) | 0x80 | (int)buf); } break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tacc = tmem_base + buf * P_BN;
+                for (uint32_t kb = 0; kb < num_k; ++kb, ++it) {
+                    const uint32_t s = it % P_STAGES, ph = (it / P_STAGES) & 1;
+                    if (*failed || !mbar_wait(&full[s], ph, failed)) { if (!*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, (2 << 8) | (int)s); } ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint64_t da = umma_desc(smem_u32(smem + s * STAGE_BYTES));
+                    const uint64_t db = umma_desc(smem_u32(smem + s * STAGE_BYTES + A_BYTES));
+#pragma unroll
+                    for (uint32_t k = 0; k < BK / 16; ++k) umma(tacc, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+                    umma_commit(&empty[s]);
+                }
+                if (ok) umma_commit(&acc_full[buf]);
+            }
+        }
+    } else {
+        const uint32_t quarter = warp & 3;
+        const bool vec = ((ldc | col0) & 3u) == 0 && (reinterpret_cast<uintptr_t>(C) & 15u) == 0;
+        uint32_t lt = 0;
+        for (uint32_t tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++lt) {
+            const uint32_t buf = lt & 1, use = lt >> 1;
+            bool ready = !*failed && mbar_wait(&acc_full[buf], use & 1, failed);
+            if (!ready && !*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, 3 << 8); }
+            ready = __all_sync(0xffffffffu, ready && !*failed);
+            if (!ready) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            uint32_t m0, n0;
+            tile_origin(tile, m0, n0);
+            const uint32_t row = m0 + quarter * 32 + lane;
+#pragma unroll 1
+            for (uint32_t c = 0; c < P_BN / 32; ++c) {
+                float v[32];
+                tmem_ld32(tmem_base + ((quarter * 32) << 16) + buf * P_BN + c * 32, v);
+                const uint32_t col = n0 + c * 32;
+                if (row < M && col < n) {
+                    float *dst = C + (size_t)row * ldc + col0 + col;
+                    if (vec && col + 32 <= n) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                            if (accumulate) { const float4 old = *reinterpret_cast<const float4 *>(dst + j); o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w; }
+                            *reinterpret_cast<float4 *>(dst + j) = o;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col + j < n) dst[j] = accumulate ? dst[j] + v[j] : v[j];
+                    }
+                }
+            }
+            // this warp has read its quarter of the buffer: hand it back to the MMA warp
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(&acc_empty[buf])) : "memory");
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 2) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
 PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
     static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
     if (!fn) {
@@ -235,21 +372,43 @@ bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t K, uin
 
 extern thread_local uint64_t tgpk_launches;
 
+static int g_tc_variant = 0;     // 0 auto, 1 force the 128x128 per-tile kernel, 2 force the persistent 128x256 kernel
+
 int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
     constexpr int BN = 128;
     if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(W)) & 15u) return TGP_E_INVAL;     // TMA needs 16-byte aligned bases
     if (K % 8) return TGP_E_INVAL;                                                                       // and 16-byte row strides
+    static int sms = 0;
+    if (!sms) { int dev = 0; cudaGetDevice(&dev); if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148; }
+    const uint32_t tiles_p = ((M + BM - 1) / BM) * ((n + P_BN - 1) / P_BN);
+    const bool persistent = g_tc_variant == 2 || (g_tc_variant == 0 && tiles_p >= 2u * (uint32_t)sms);
     CUtensorMap ma, mb;
-    if (!make_map(&ma, A, M, K, BM) || !make_map(&mb, W, n, K, BN)) return TGP_E_CUDA;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN>::TOTAL) != cudaSuccess) return TGP_E_CUDA;
-        attr_set = true;
+    if (!make_map(&ma, A, M, K, BM) || !make_map(&mb, W, n, K, persistent ? P_BN : BN)) return TGP_E_CUDA;
+    if (persistent) {
+        constexpr int SMEM = P_STAGES * (BM * BK * 2 + P_BN * BK * 2) + 128 + 1024;
+        static bool attr_p = false;
+        if (!attr_p) {
+            if (cudaFuncSetAttribute(gemm_tc_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess) return TGP_E_CUDA;
+            attr_p = true;
+        }
+        gemm_tc_persistent_kernel<<<tiles_p < (uint32_t)sms ? tiles_p : (uint32_t)sms, 192, SMEM, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
+    } else {
+        static bool attr_set = false;
+        if (!attr_set) {
+            if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN>::TOTAL) != cudaSuccess) return TGP_E_CUDA;
+            attr_set = true;
+        }
+        dim3 grid(((M + BM - 1) / BM) * ((n + BN - 1) / BN));
+        gemm_tc_kernel<BN><<<grid, 192, Smem<BN>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
     }
-    dim3 grid(((M + BM - 1) / BM) * ((n + BN - 1) / BN));
-    gemm_tc_kernel<BN><<<grid, 192, Smem<BN>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
     if (cudaGetLastError() != cudaSuccess) return TGP_E_CUDA;
     tgpk_launches += 1;
+    return TGP_OK;
+}
+
+extern "C" int tgp_k_gemm_tc_variant(int v) {
+    if (v < 0 || v > 2) return TGP_E_INVAL;
+    g_tc_variant = v;
     return TGP_OK;
 }
 
