@@ -261,20 +261,27 @@ __global__ void __launch_bounds__(128) attn_rows_kernel(AttnArgs a) {
     for (int i = 0; i < DPL; ++i) out[lane + 32 * i] = __float2bfloat16_rn(o[i] / l);
 }
 
-// Decode (one query per sequence): grid (tile, kv head, batch); warp g of the block serves query head
-// hk*G + g over the keys of one tile and leaves an unnormalised partial (max, sum, o[Dh]) in scratch.
+// Decode (one query per sequence): grid (tile, kv head, batch).  The block has G x SPLIT warps: SPLIT warps share
+// one query head of the group and take the tile's keys in strided 32-key passes (lane = key for the scores, lane =
+// output dims for P.V, fully unrolled so a pass's V loads are in flight together); their partial (max, sum, o[Dh])
+// meet in shared memory and one unnormalised partial per (query head, tile) goes to scratch.
 template <int DH>
-__global__ void attn_decode_partial_kernel(AttnArgs a) {
-    extern __shared__ float qsm[];
-    const uint32_t g = threadIdx.x >> 5, lane = threadIdx.x & 31;
+__global__ void attn_decode_partial_kernel(AttnArgs a, uint32_t SPLIT) {
+    extern __shared__ float dsm[];
+    const uint32_t G = a.Hq / a.Hkv;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t g = warp / SPLIT, sp = warp % SPLIT;
     const uint32_t tile = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
-    const uint32_t G = a.Hq / a.Hkv, hq = hk * G + g;
+    const uint32_t hq = hk * G + g;
     const uint32_t kvlen = a.pos0 + 1;
     const uint32_t nk = min(a.TK, kvlen - tile * a.TK);
-    float *qs = qsm + g * DH;
-    const bf16 *q = a.qb + (size_t)b * a.Hq * DH + hq * DH;
-    for (int i = lane; i < DH; i += 32) qs[i] = __bfloat162float(q[i]);
-    __syncwarp();
+    float *qs = dsm + g * DH;                               // [G][DH] query rows as fp32
+    float *parts = dsm + G * DH;                            // [G][SPLIT][DH + 2]
+    if (sp == 0) {
+        const bf16 *q = a.qb + (size_t)b * a.Hq * DH + hq * DH;
+        for (int i = lane; i < DH; i += 32) qs[i] = __bfloat162float(q[i]);
+    }
+    __syncthreads();
     constexpr int DPL = DH / 32;
     float o[DPL];
 #pragma unroll
@@ -282,7 +289,7 @@ __global__ void attn_decode_partial_kernel(AttnArgs a) {
     float mx = -INFINITY, l = 0.f;
     const bf16 *kt = reinterpret_cast<const bf16 *>(a.tiles.k[tile]) + (size_t)(b * a.Hkv + hk) * a.TK * DH;
     const bf16 *vt = reinterpret_cast<const bf16 *>(a.tiles.v[tile]) + (size_t)(b * a.Hkv + hk) * a.TK * DH;
-    for (uint32_t j0 = 0; j0 < nk; j0 += 32) {
+    for (uint32_t j0 = sp * 32; j0 < nk; j0 += SPLIT * 32) {
         const uint32_t j = j0 + lane;
         float s = -INFINITY;
         if (j < nk) {
@@ -304,18 +311,38 @@ __global__ void attn_decode_partial_kernel(AttnArgs a) {
 #pragma unroll
         for (int i = 0; i < DPL; ++i) o[i] *= alpha;
         const uint32_t cnt = min(32u, nk - j0);
-        for (uint32_t t = 0; t < cnt; ++t) {
+#pragma unroll
+        for (uint32_t t = 0; t < 32; ++t) {                 // rows past the end re-read the last valid row with weight 0
             const float pt = __shfl_sync(0xffffffffu, pj, t);
-            const bf16 *vr = vt + (size_t)(j0 + t) * DH;
+            const bf16 *vr = vt + (size_t)(j0 + min(t, cnt - 1)) * DH;
 #pragma unroll
             for (int i = 0; i < DPL; ++i) o[i] = fmaf(pt, __bfloat162float(vr[lane + 32 * i]), o[i]);
         }
         mx = mnew;
     }
-    float *part = a.scratch + ((size_t)(b * a.Hq + hq) * a.n_tiles + tile) * (DH + 2);
-    if (lane == 0) { part[0] = mx; part[1] = l; }
+    float *mine = parts + (size_t)(g * SPLIT + sp) * (DH + 2);
+    if (lane == 0) { mine[0] = mx; mine[1] = l; }
 #pragma unroll
-    for (int i = 0; i < DPL; ++i) part[2 + lane + 32 * i] = o[i];
+    for (int i = 0; i < DPL; ++i) mine[2 + lane + 32 * i] = o[i];
+    __syncthreads();
+    if (sp == 0) {                                          // fixed-order merge of the SPLIT partials of this head
+        const float *p0 = parts + (size_t)g * SPLIT * (DH + 2);
+        float m = -INFINITY;
+        for (uint32_t k = 0; k < SPLIT; ++k) m = fmaxf(m, p0[k * (DH + 2)]);
+        float lsum = 0.f, acc[DPL];
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
+        for (uint32_t k = 0; k < SPLIT; ++k) {
+            const float w = expf(p0[k * (DH + 2)] - m);     // a warp that saw no key has max -inf and weight 0
+            lsum += w * p0[k * (DH + 2) + 1];
+#pragma unroll
+            for (int i = 0; i < DPL; ++i) acc[i] += w * p0[k * (DH + 2) + 2 + lane + 32 * i];
+        }
+        float *part = a.scratch + ((size_t)(b * a.Hq + hq) * a.n_tiles + tile) * (DH + 2);
+        if (lane == 0) { part[0] = m; part[1] = lsum; }
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) part[2 + lane + 32 * i] = acc[i];
+    }
 }
 
 // Merge the per-tile partials of one (batch, query head): grid (Hq, B), DH threads.
@@ -580,12 +607,17 @@ int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *
     AttnArgs a{(const bf16 *)qb, (bf16 *)ob, scratch, c->Hq, c->Hkv, c->Dh, c->TK, q_len, pos0, n_tiles, 1.0f / sqrtf((float)c->Dh), tiles};
     if (q_len == 1 && scratch) {
         const uint32_t nt = (pos0 + 1 + c->TK - 1) / c->TK, G = c->Hq / c->Hkv;
+        if (G > 32) return TGP_E_TOO_LARGE;
+        uint32_t split = (c->TK + 31) / 32;
+        if (split > 32 / G) split = 32 / G;
+        if (split < 1) split = 1;
         dim3 grid(nt, c->Hkv, B);
+        const size_t sm = (size_t)(G * c->Dh + G * split * (c->Dh + 2)) * sizeof(float);
         if (c->Dh == 64) {
-            attn_decode_partial_kernel<64><<<grid, 32 * G, G * 64 * sizeof(float), st>>>(a);
+            attn_decode_partial_kernel<64><<<grid, 32 * G * split, sm, st>>>(a, split);
             attn_decode_merge_kernel<64><<<dim3(c->Hq, B), 64, 0, st>>>(a);
         } else {
-            attn_decode_partial_kernel<128><<<grid, 32 * G, G * 128 * sizeof(float), st>>>(a);
+            attn_decode_partial_kernel<128><<<grid, 32 * G * split, sm, st>>>(a, split);
             attn_decode_merge_kernel<128><<<dim3(c->Hq, B), 128, 0, st>>>(a);
         }
         tgpk_launches += 1;
