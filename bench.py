@@ -126,8 +126,12 @@ def gemm_shapes_of_step(lay, M):
     cfg = lay.cfg
     out = []
     for l in range(cfg.L):
-        for kind, res in ((si.K_WQ, 0), (si.K_WK, 0), (si.K_WV, 0), (si.K_WO, 1), (si.K_WG, 0), (si.K_WU, 0), (si.K_WD, 1)):
+        for kind, res in ((si.K_WQ, 0), (si.K_WK, 0), (si.K_WV, 0), (si.K_WO, 1)):
             out += [(t.rows, t.cols, res, M) for t in lay.blocks(kind, l)]
+        for e in (range(cfg.E) if cfg.E else (-1,)):          # MoE: tokens spread evenly over the experts (top-k picks each)
+            me = M if not cfg.E else max(1, M * cfg.topk // cfg.E)
+            for kind, res in ((si.K_WG, 0), (si.K_WU, 0), (si.K_WD, 0 if cfg.E else 1)):
+                out += [(t.rows, t.cols, res, me) for t in lay.blocks(kind, l, e)]
     out += [(t.rows, t.cols, 0, cfg.B) for t in lay.blocks(si.K_LM)]
     return out
 
@@ -269,12 +273,24 @@ def main():
     ap.add_argument("--kernel-loop", choices=["decode", "prefill"], default=None,
                     help="only run the back-to-back weight-product loop of one step (small, for ncu captures)")
     ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--layers", type=int, default=None, help="run the shape at reduced depth; a byte budget is scaled in proportion")
+    ap.add_argument("--bits", type=int, default=7, help="policy bits: 1 affinity/pins, 2 roofline selectivity, 4 zero-copy")
+    ap.add_argument("--budget-frac", type=float, default=None, help="device budget as a fraction of the pool (oversubscription sweep)")
     args = ap.parse_args()
     cfg = si.CONFIGS[args.config]
     if args.decode is not None:
         from dataclasses import replace
         cfg = replace(cfg, T=args.decode)
-    lay = si.build_layout(cfg)
+    budget = None
+    if args.layers is not None and args.layers != cfg.L:
+        from dataclasses import replace
+        full = si.build_layout(cfg)
+        cfg2 = replace(cfg, L=args.layers, name=f"{cfg.name}_L{args.layers}")
+        budget = int(full.budget * si.build_layout(cfg2, budget=1 << 40).pool_bytes / full.pool_bytes) // 512 * 512
+        cfg = cfg2
+    lay = si.build_layout(cfg, budget=budget)
+    if args.budget_frac is not None:
+        lay = si.build_layout(cfg, budget=int(lay.pool_bytes * args.budget_frac) // 512 * 512)
     if args.impl == "reference":
         return run_reference(args, cfg, lay)
 
@@ -304,11 +320,23 @@ def main():
 
     pool = pinned_pool(lay.pool_bytes)
     si.fill_pool_torch(lay, pool, device=dev)
-    s = Session(lay, MACHINE, pool_base=pool.data_ptr(), pool_flags=tb.POOL_PINNED)
-    blobs = s.plan()
+    bias = si.router_bias(cfg) if cfg.E else None
+    s = Session(lay, MACHINE, pool_base=pool.data_ptr(), pool_flags=tb.POOL_PINNED, router_bias=bias)
+    profile_s = None
+    if cfg.E:
+        # MoE: one profile pass with every expert traced records which experts each step really uses
+        s.plan(expert_counts=np.ones((1 + cfg.T, cfg.L, cfg.E), dtype=np.uint32), bits=args.bits)
+        r = Runner(s, cfg.B * cfg.S, device=str(dev))
+        t0 = time.perf_counter()
+        r.generate(si.prompt_tokens(cfg), cfg.T, keep_logits=False)
+        profile_s = time.perf_counter() - t0
+        counts = s.ctx.expert_counts(cfg.L, cfg.E)
+        blobs = s.plan(expert_counts=counts, bits=args.bits)
+    else:
+        blobs = s.plan(bits=args.bits)
+        r = Runner(s, cfg.B * cfg.S, device=str(dev))
     totals = np.frombuffer(blobs["totals"], dtype="<u8").reshape(-1, 4)
     ops = parse_trace(s.ctx.trace_export())
-    r = Runner(s, cfg.B * cfg.S, device=str(dev))
     prompt_pinned = torch.from_numpy(si.prompt_tokens(cfg)).pin_memory()
     tok_pinned = torch.empty((cfg.B, 1), dtype=torch.int32).pin_memory()
     logits_host = torch.empty((cfg.B, cfg.V), dtype=torch.float32).pin_memory()
@@ -366,12 +394,13 @@ def main():
     r.reset()
     s.ctx.set_op_timing(True)
     kind_ms, kind_bytes, kind_flops, kind_n = {}, {}, {}, {}
-    launches = 0
+    launches = mismatches = 0
     step_ms = []
     for k in range(1 + T):
         st = r.step(tb.PREFILL if k == 0 else tb.DECODE, prompt_pinned.numpy() if k == 0 else None, cfg.S if k == 0 else 1, want_stats=True)
         first, tms = s.ctx.op_times()
         launches += st.n_launches
+        mismatches += st.n_mismatch
         step_ms.append(st.step_ms)
         phase = "prefill" if k == 0 else "decode"
         for j, t in enumerate(tms):
@@ -440,6 +469,7 @@ def main():
            "prefill_tok_s": cfg.B * cfg.S / (step_ms[0] * 1e-3), "decode_tok_s": cfg.B * T / (sum(step_ms[1:]) * 1e-3) if T else None,
            "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": int(totals[:, 0].sum()) + cfg.B * (cfg.S + T) * 4,
                    "d2h_bytes_per_step": L_d2h + cfg.B * (T + 1) * 4 + cfg.B * cfg.V * 4},
+           "policy_bits": args.bits, "trace_mismatches": mismatches, "moe_profile_pass_s": profile_s,
            "gpu_launches": launches * args.steps, "clocks": clocks, "roofline": roof, "step_roofline": step_roof,
            "kernels": {f"{k[0]}:{k[1]}": {"ms": round(v, 3), "launches": kind_n[k], "GBps": round(kind_bytes[k] / (v * 1e-3) / 1e9, 1),
                                            "TFLOPs": round(kind_flops[k] / (v * 1e-3) / 1e12, 2)} for k, v in sorted(kind_ms.items())}}
