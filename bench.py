@@ -452,12 +452,28 @@ def main():
     for o in ops:
         for (t, mode, touched) in o[6]:
             step_of.setdefault(o[0], {})[t] = lay.tensors[t].size if touched * 2 >= lay.tensors[t].size else touched
-    L_lb = sum(max(0, sum(d.values()) - (lay.budget if k else 0)) for k, d in step_of.items())
-    t_roof = max(F / MACHINE["peak_flops"], H / MACHINE["hbm_Bps"], L_plan / MACHINE["h2d_Bps"], L_d2h / MACHINE["d2h_Bps"])
-    t_lb = max(F / MACHINE["peak_flops"], H / MACHINE["hbm_Bps"], L_lb / MACHINE["h2d_Bps"])
+    # per step the slowest of compute, HBM and link; the pass roofline is the sum over its steps (a pass mixes a
+    # possibly compute-bound prefill with link-bound decode steps)
+    nsteps = len(totals)
+    Fs, Hs = [0] * nsteps, [0] * nsteps
+    for o in ops:
+        Fs[o[0]] += o[4]
+        Hs[o[0]] += o[5]
+    lb = {k: max(0, sum(d.values()) - (lay.budget if k else 0)) for k, d in step_of.items()}
+    t_roof = t_lb = 0.0
+    bound_of = []
+    for k in range(nsteps):
+        cands = {"tensor": Fs[k] / MACHINE["peak_flops"], "hbm": (Hs[k] + int(totals[k][0])) / MACHINE["hbm_Bps"],
+                 "link": (int(totals[k][0]) + int(totals[k][2])) / MACHINE["h2d_Bps"], "link_d2h": int(totals[k][1]) / MACHINE["d2h_Bps"]}
+        bound_of.append(max(cands, key=cands.get))
+        t_roof += max(cands.values())
+        t_lb += max(cands["tensor"], cands["hbm"], lb.get(k, 0) / MACHINE["h2d_Bps"])
     t_meas = ms * 1e-3 / args.steps
-    step_roof = {"bound": "link", "t_roof_s_plan_bytes": t_roof, "t_roof_s_lower_bound": t_lb, "t_measured_s": t_meas,
+    step_roof = {"bound": {"prefill": bound_of[0], "decode": max(set(bound_of[1:]), key=bound_of[1:].count) if nsteps > 1 else None},
+                 "t_roof_s_plan_bytes": t_roof, "t_roof_s_lower_bound": t_lb, "t_measured_s": t_meas,
                  "frac_plan_bytes": t_roof / t_meas, "frac_lower_bound": t_lb / t_meas,
+                 "prefill": {"t_roof_s": max(Fs[0] / MACHINE["peak_flops"], (int(totals[0][0]) + int(totals[0][2])) / MACHINE["h2d_Bps"]),
+                             "t_measured_s": step_ms[0] * 1e-3},
                  "link_gbs_achieved": L_plan / t_meas / 1e9, "link_gbs_peak": MACHINE["h2d_Bps"] / 1e9,
                  "h2d_bytes": int(totals[:, 0].sum()), "d2h_bytes": L_d2h, "zero_copy_bytes": int(totals[:, 2].sum()),
                  "flops": F, "hbm_bytes": H}

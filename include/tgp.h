@@ -198,6 +198,21 @@ int  tgp_managed_alloc(void **out, uint64_t bytes);
 int  tgp_managed_free(void *ptr);
 int  tgp_managed_evict(void *ptr, uint64_t bytes);
 
+/* Activation tap, for parity checks at every rounding point.  While a tap buffer is set, tgp_step() copies each
+ * bf16-rounded activation it produces into it (on the compute stream, 256-byte aligned, in op order): normed
+ * hidden states, rotated q, the KV tiles an append touched, attention output, the SwiGLU output (dense FFN),
+ * the final normed state.  tgp_tap_index() returns 5 uint64 per record: op index, tag, sub-index (tile), offset,
+ * bytes (two-call form: out == NULL gives the word count).  tgp_set_tap() also rewinds the buffer; NULL disables. */
+#define TGP_TAP_H 0u
+#define TGP_TAP_HF 1u
+#define TGP_TAP_Q 2u
+#define TGP_TAP_KTILE 3u
+#define TGP_TAP_VTILE 4u
+#define TGP_TAP_O 5u
+#define TGP_TAP_A 6u
+int  tgp_set_tap(tgp_ctx *ctx, void *tap_dev, uint64_t bytes);
+int  tgp_tap_index(tgp_ctx *ctx, uint64_t *out, uint64_t *n_words);
+
 /* Per-op timestamps (Section IV-D "Runtime Monitor": lightweight timestamping).  While enabled, tgp_step()
  * brackets every op with CUDA events on the compute stream (after the op's copies have been waited for, so
  * the figure is kernel time, not stall time).  tgp_op_times() waits for the last timed step and returns one

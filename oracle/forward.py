@@ -56,13 +56,23 @@ class OracleModel:
         self.K = np.zeros((cfg.L, cfg.B, cfg.Hkv, cfg.max_len, cfg.Dh), dtype=dtype)
         self.V = np.zeros_like(self.K)
         self.expert_counts = []          # per step: [L][E] token counts (MoE only)
+        # optional hook(name, layer, pre, rounded) -> array to continue with, called at every bf16 rounding point with
+        # the fp32 value before rounding and the oracle's rounding of it (used by the lockstep parity test)
+        self.hook = None
 
     # ---- pieces -------------------------------------------------------------------------
-    def rmsnorm(self, x, g):
+    def _round(self, name, layer, pre):
+        pre = to_f32(pre)
+        out = bf16_round(pre)
+        if self.hook is not None:
+            out = np.asarray(self.hook(name, layer, pre, out), dtype=np.float32)
+        return out
+
+    def rmsnorm(self, x, g, name="h", layer=-1):
         """bf16( x / sqrt(mean(x^2) + eps) * g ) per row."""
         xd = x.astype(self.dt)
         ms = np.mean(xd * xd, axis=-1, keepdims=True)
-        return bf16_round(to_f32(xd / np.sqrt(ms + self.cfg.eps) * g)).astype(self.dt)
+        return self._round(name, layer, xd / np.sqrt(ms + self.cfg.eps) * g).astype(self.dt)
 
     def linear(self, a, W):
         """fp32( a @ W^T ), W stored [out, in]."""
@@ -102,7 +112,7 @@ class OracleModel:
     def ffn_dense(self, l, h2, e=-1):
         g = self.linear(h2, self.w[(self.WG, l, e)]).astype(self.dt)
         u = self.linear(h2, self.w[(self.WU, l, e)]).astype(self.dt)
-        a = bf16_round(to_f32(g / (1.0 + np.exp(-g)) * u))
+        a = self._round("a", l, g / (1.0 + np.exp(-g)) * u) if e < 0 else bf16_round(to_f32(g / (1.0 + np.exp(-g)) * u))
         return self.linear(a, self.w[(self.WD, l, e)])
 
     def ffn_moe(self, l, h2, x):
@@ -134,18 +144,18 @@ class OracleModel:
         x = to_f32(self.w[(self.EMBED, -1, -1)][tokens])                      # [B, q, d]
         counts_step = []
         for l in range(cfg.L):
-            h = self.rmsnorm(x, self.w[(self.G1, l, -1)][0])
+            h = self.rmsnorm(x, self.w[(self.G1, l, -1)][0], "h", l)
             qv = self.linear(h, self.w[(self.WQ, l, -1)]).reshape(B, q, cfg.Hq, cfg.Dh)
             kv = self.linear(h, self.w[(self.WK, l, -1)]).reshape(B, q, cfg.Hkv, cfg.Dh)
             vv = self.linear(h, self.w[(self.WV, l, -1)]).reshape(B, q, cfg.Hkv, cfg.Dh)
-            qb = bf16_round(self.rope(qv, pos0))
-            kb = bf16_round(self.rope(kv, pos0))
-            vb = bf16_round(vv)
+            qb = self._round("q", l, self.rope(qv, pos0))
+            kb = self._round("k", l, self.rope(kv, pos0))
+            vb = self._round("v", l, vv)
             self.K[l, :, :, pos0:pos0 + q] = kb.transpose(0, 2, 1, 3)
             self.V[l, :, :, pos0:pos0 + q] = vb.transpose(0, 2, 1, 3)
-            o = bf16_round(self.attention(l, qb, pos0)).reshape(B, q, cfg.Hq * cfg.Dh)
+            o = self._round("o", l, self.attention(l, qb, pos0)).reshape(B, q, cfg.Hq * cfg.Dh)
             x = to_f32(x.astype(self.dt) + self.linear(o, self.w[(self.WO, l, -1)]).astype(self.dt))
-            h2 = self.rmsnorm(x, self.w[(self.G2, l, -1)][0])
+            h2 = self.rmsnorm(x, self.w[(self.G2, l, -1)][0], "h2", l)
             if cfg.E == 0:
                 x = to_f32(x.astype(self.dt) + self.ffn_dense(l, h2).astype(self.dt))
             else:
@@ -154,7 +164,7 @@ class OracleModel:
                 counts_step.append(c)
         self.expert_counts.append(counts_step)
         xs = x if all_positions else x[:, -1:, :]
-        hf = self.rmsnorm(xs, self.w[(self.GF, -1, -1)][0])
+        hf = self.rmsnorm(xs, self.w[(self.GF, -1, -1)][0], "hf", -1)
         logits = self.linear(hf, self.w[(self.LM, -1, -1)])
         return logits if all_positions else logits[:, 0, :]
 

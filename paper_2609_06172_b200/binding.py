@@ -22,6 +22,7 @@ PREFILL, DECODE = 0, 1
 VAR_EXPLICIT_RING, VAR_MANAGED_HINTS, VAR_MANAGED_DEMAND = 0, 1, 2
 BIT_A, BIT_P, BIT_ZC = 1, 2, 4
 X_CLASSES, X_TENSORS, X_PINS, X_COMMANDS, X_TOTALS = range(5)
+TAP_H, TAP_HF, TAP_Q, TAP_KTILE, TAP_VTILE, TAP_O, TAP_A = range(7)
 
 
 class Machine(C.Structure):
@@ -81,6 +82,8 @@ _SIGS = {
     "tgp_managed_alloc": [C.POINTER(_P), _U64],
     "tgp_managed_free": [_P],
     "tgp_managed_evict": [_P, _U64],
+    "tgp_set_tap": [_P, _P, _U64],
+    "tgp_tap_index": [_P, C.POINTER(_U64), C.POINTER(_U64)],
     "tgp_set_op_timing": [_P, C.c_int],
     "tgp_op_times": [_P, C.POINTER(C.c_float), _U32, C.POINTER(_U32), C.POINTER(_U32)],
     "tgp_k_embed": [_P, _P, _P, _U32, _U32, _P],
@@ -259,6 +262,18 @@ class Ctx:
         a = np.zeros(max(1, n.value), dtype=np.uint32)
         self._ck(lib().tgp_expert_counts(self._h, a.ctypes.data_as(C.POINTER(_U32)), C.byref(n)), "tgp_expert_counts")
         return a[:n.value].reshape(-1, L, E)
+
+    def set_tap(self, tap, nbytes):
+        self._ck(lib().tgp_set_tap(self._h, _ptr(tap), nbytes), "tgp_set_tap")
+        self._keep.append(tap)
+
+    def tap_index(self):
+        """uint64 [records, 5]: op index, tag, sub-index, offset, bytes."""
+        n = _U64()
+        self._ck(lib().tgp_tap_index(self._h, None, C.byref(n)), "tgp_tap_index")
+        a = np.zeros(max(1, n.value), dtype=np.uint64)
+        self._ck(lib().tgp_tap_index(self._h, a.ctypes.data_as(C.POINTER(_U64)), C.byref(n)), "tgp_tap_index")
+        return a[:n.value].reshape(-1, 5)
 
     def set_op_timing(self, enable):
         self._ck(lib().tgp_set_op_timing(self._h, int(enable)), "tgp_set_op_timing")

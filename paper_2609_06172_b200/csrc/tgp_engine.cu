@@ -50,6 +50,9 @@ struct TgpEngine {
     bool op_timing = false;
     std::vector<cudaEvent_t> ta, tb_;
     uint32_t timed_op0 = 0, timed_nops = 0;
+    // activation tap (parity testing): device buffer the rounded activations are copied to, and what went where
+    char *tap = nullptr; uint64_t tap_bytes = 0, tap_used = 0;
+    std::vector<uint64_t> tap_index;                     // 5 words per record: op, tag, sub-index, offset, bytes
     // managed-hints variant
     size_t hinted_upto = 0;
     bool advised = false;
@@ -475,6 +478,33 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             return tgp_fail(ctx, TGP_E_MISMATCH, "op kind the bound model cannot run");
         }
         if (rc) return tgp_fail(ctx, rc, "kernel launch failed");
+        if (e->tap) {
+            auto tap_copy = [&](uint64_t tag, uint64_t sub, const void *src, uint64_t bytes) -> int {
+                const uint64_t at = (e->tap_used + 255) / 256 * 256;
+                if (at + bytes > e->tap_bytes) return tgp_fail(ctx, TGP_E_TOO_LARGE, "activation tap buffer is full");
+                CU(ctx, cudaMemcpyAsync(e->tap + at, src, bytes, cudaMemcpyDeviceToDevice, cs));
+                const uint64_t rec[5] = {i, tag, sub, at, bytes};
+                e->tap_index.insert(e->tap_index.end(), rec, rec + 5);
+                e->tap_used = at + bytes;
+                return TGP_OK;
+            };
+            int trc = TGP_OK;
+            if (o.kind == TGP_OP_RMSNORM) {
+                const bool fin = ctx->roles[ctx->role_of_tensor[ctx->acc[o.acc0].tensor]].kind == TGP_K_GF;
+                trc = fin ? tap_copy(TGP_TAP_HF, 0, e->hf, (uint64_t)B * c.d * 2) : tap_copy(TGP_TAP_H, 0, e->h, (uint64_t)M * c.d * 2);
+            } else if (o.kind == TGP_OP_ROPE_KV) {
+                trc = tap_copy(TGP_TAP_Q, 0, e->qb, (uint64_t)M * qd * 2);
+                for (uint32_t k = 0; k < o.nacc && !trc; ++k) {
+                    const TgpRole &r = ctx->roles[ctx->role_of_tensor[ctx->acc[o.acc0 + k].tensor]];
+                    trc = tap_copy(r.kind == TGP_K_KTILE ? TGP_TAP_KTILE : TGP_TAP_VTILE, r.block, where(ctx, o, k), ctx->tensors[ctx->acc[o.acc0 + k].tensor].size);
+                }
+            } else if (o.kind == TGP_OP_ATTN) {
+                trc = tap_copy(TGP_TAP_O, 0, e->ob, (uint64_t)M * qd * 2);
+            } else if (o.kind == TGP_OP_SWIGLU && !c.E) {
+                trc = tap_copy(TGP_TAP_A, 0, e->ab, (uint64_t)M * c.F * 2);
+            }
+            if (trc) return trc;
+        }
         if (e->op_timing) CU(ctx, cudaEventRecord(e->tb_[ti], cs));
         if (ring) {
             if (ctx->plan.op_is_wait_target[i]) {
@@ -547,5 +577,20 @@ extern "C" int tgp_expert_counts(tgp_ctx *ctx, uint32_t *out, uint64_t *n) {
     if (!ctx || !n) return TGP_E_INVAL;
     if (out) { if (*n < ctx->run_counts.size()) return TGP_E_INVAL; memcpy(out, ctx->run_counts.data(), ctx->run_counts.size() * 4); }
     *n = ctx->run_counts.size();
+    return TGP_OK;
+}
+
+extern "C" int tgp_set_tap(tgp_ctx *ctx, void *tap_dev, uint64_t bytes) {
+    if (!ctx || !ctx->eng) return TGP_E_STATE;
+    ctx->eng->tap = (char *)tap_dev; ctx->eng->tap_bytes = tap_dev ? bytes : 0; ctx->eng->tap_used = 0;
+    ctx->eng->tap_index.clear();
+    return TGP_OK;
+}
+
+extern "C" int tgp_tap_index(tgp_ctx *ctx, uint64_t *out, uint64_t *n_words) {
+    if (!ctx || !ctx->eng || !n_words) return TGP_E_STATE;
+    const std::vector<uint64_t> &v = ctx->eng->tap_index;
+    if (out) { if (*n_words < v.size()) return TGP_E_INVAL; memcpy(out, v.data(), v.size() * 8); }
+    *n_words = v.size();
     return TGP_OK;
 }
