@@ -331,9 +331,11 @@ def _lockstep(cfg, lay, pool, W, n_dec, dtype):
     per_layer = cfg.B * cfg.S * (2 * d + 2 * qd + F) * 2 + 2 * cfg.n_tiles * cfg.B * cfg.Hkv * cfg.TK * cfg.Dh * 2 + 16 * 256
     tap = torch.empty(per_layer * cfg.L + (1 << 20), dtype=torch.uint8, device="cuda:0")
     om = forward.OracleModel(cfg, W, dtype=dtype)
-    # slack per rounding point, relative to |pre| + mean|pre|: fp32 summation order / libm vs device exp; the attention
-    # output also carries the tensor-core kernel's bf16 rounding of the softmax weights (not mirrored by the oracle)
-    rtol = {"h": 2e-5, "h2": 2e-5, "hf": 2e-5, "q": 5e-5, "k": 5e-5, "v": 5e-5, "a": 5e-5, "o": 4e-3}
+    # slack per rounding point, relative to |pre| + mean|pre|: fp32 summation order and libm vs device exp.  The normed
+    # states sit behind the residual stream, which sums tensor-core products of K up to 8192 per layer (their fp32
+    # accumulation is not round-to-nearest: ~5e-5 typical, 3e-4 covers the tail of 1e6 elements); the attention output
+    # also carries the tensor-core kernel's bf16 rounding of the softmax weights (not mirrored by the oracle)
+    rtol = {"h": 3e-4, "h2": 3e-4, "hf": 3e-4, "q": 1e-4, "k": 1e-4, "v": 1e-4, "a": 1e-4, "o": 4e-3}
     flips = {k: [0, 0] for k in rtol}
     prompt = si.prompt_tokens(cfg)
     worst = 0.0
@@ -375,7 +377,9 @@ def _lockstep(cfg, lay, pool, W, n_dec, dtype):
                     new[:, p - pos0] = g[p // cfg.TK][:, :, p % cfg.TK, :]
                 g = new
             g = g.reshape(pre.shape)
-            bound = 0.5 * _bf16_ulp(pre) * (1 + 1e-6) + rtol[name] * (np.abs(pre) + np.abs(pre).mean())
+            # (the attention output averages rows of V, so its P-rounding error scales with |V| ~ max|o|, not with |o|)
+            scale = np.abs(pre).max() if name == "o" else np.abs(pre).mean()
+            bound = 0.5 * _bf16_ulp(pre) * (1 + 1e-6) + rtol[name] * (np.abs(pre) + scale)
             bad = np.abs(g.astype(np.float64) - pre.astype(np.float64)) > bound
             assert not bad.any(), (name, layer, int(bad.sum()), float(np.abs(g - pre)[bad].max()))
             flips[name][0] += int((g != out).sum())
