@@ -441,9 +441,12 @@ def main():
                 "kernel": f"{dom[1]} ({dom[0]})", "launches": kind_n[dom], "avg_us": kind_ms[dom] / kind_n[dom] * 1e3,
                 "algorithmic_per_launch": kind_bytes[dom] / kind_n[dom], "timing": "in-step CUDA events per op"}
     roof.update({"peak_source": peaks["source"], "traffic": None})
-    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    prof = os.path.join(ROOT, "profiles", "traffic.txt")          # DRAM bytes per launch from the committed ncu summaries
     if os.path.exists(prof):
-        roof["traffic"] = json.load(open(prof)).get(f"{dom[1]}_{dom[0]}_cfg{args.config}")
+        for line in open(prof):
+            f = line.split()
+            if f and f[0] == f"{dom[1]}_{dom[0]}_cfg{args.config}":
+                roof["traffic"] = float(f[1])
     # step roofline: slowest of compute, HBM and link for the whole pass, (i) with the plan's bytes, (ii) with the lower bound
     F = sum(o[4] for o in ops)
     H = sum(o[5] for o in ops) + int(totals[:, 0].sum())
