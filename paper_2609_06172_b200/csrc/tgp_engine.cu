@@ -14,7 +14,9 @@
 #include <cuda_runtime.h>
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
+#include <map>
 #include <vector>
 #include "tgp_internal.h"
 #include "tgp_kernels.h"
@@ -54,8 +56,8 @@ struct TgpEngine {
     char *tap = nullptr; uint64_t tap_bytes = 0, tap_used = 0;
     std::vector<uint64_t> tap_index;                     // 5 words per record: op, tag, sub-index, offset, bytes
     // managed-hints variant
-    size_t hinted_upto = 0;
-    bool advised = false;
+    bool advised = false, evict_explicit = true;
+    std::map<int32_t, std::vector<uint32_t>> evict_at;   // op -> read-only ring tensors whose planned stay ends there
 };
 
 static inline uint64_t up256(uint64_t x) { return (x + 255) / 256 * 256; }
@@ -209,7 +211,7 @@ int tgp_run_reset(tgp_ctx *ctx) {
     CU(ctx, cudaDeviceSynchronize());
     TgpEngine *e = ctx->eng;
     e->next_cmd = 0; e->next_step = 0; e->pos = 0; e->wb_pending = false; e->copy_waited_op = -1; e->tok_src = nullptr;
-    e->hinted_upto = 0;
+    e->evict_at.clear();
     ctx->run_counts.clear();
     return TGP_OK;
 }
@@ -270,30 +272,89 @@ static inline char *where(const tgp_ctx *ctx, const TgpOp &o, uint32_t k) {
     return w == UINT64_MAX ? ctx->pools[t.pool].dev_alias + t.off : (char *)ctx->arena + w;
 }
 
-// managed-hints variant: prefetch the tensors of upcoming link-bound ops, advise the pin set once
-static int hint_ahead(tgp_ctx *ctx, size_t op_now, size_t step_end, cudaStream_t copy) {
+// ---- managed-hints variant (the paper's mechanism, Section IV-D: cudaMemPrefetchAsync at tensor granularity and
+// cudaMemAdvise for resident tensors) driven by the same plan as the ring --------------------------------------------
+// advice, once per run: pins prefer the device; in-place (zero-copy) tensors stay on the host, mapped into the GPU.
+// (Read-mostly duplication of the weights was measured slower here than plain migration with explicit eviction.)
+static int advise_once(tgp_ctx *ctx) {
+    TgpEngine *e = ctx->eng;
+    if (e->advised) return TGP_OK;
+    const TgpPlan &pl = ctx->plan;
+    for (size_t t = 0; t < ctx->tensors.size(); ++t) {
+        const TgpTensor &tt = ctx->tensors[t];
+        char *p = ctx->pools[tt.pool].host_base + tt.off;
+        if (pl.zc[t]) {
+            CU(ctx, cudaMemAdvise(p, tt.size, cudaMemAdviseSetPreferredLocation, cudaCpuDeviceId));
+            CU(ctx, cudaMemAdvise(p, tt.size, cudaMemAdviseSetAccessedBy, e->device));
+        }
+    }
+    for (auto &pin : pl.pins) {
+        const TgpTensor &tt = ctx->tensors[pin.first];
+        CU(ctx, cudaMemAdvise(ctx->pools[tt.pool].host_base + tt.off, tt.size, cudaMemAdviseSetPreferredLocation, e->device));
+    }
+    e->advised = true;
+    return TGP_OK;
+}
+
+// Same walk as pump(): a planned H2D becomes a prefetch to the device on the copy stream (after the op that frees its
+// room), a planned write-back becomes a prefetch home; the stay's tensor is queued for eviction at its release op.
+static int pump_managed(tgp_ctx *ctx, int32_t limit, cudaStream_t copy, uint32_t *n_cmds) {
     TgpEngine *e = ctx->eng;
     const TgpPlan &pl = ctx->plan;
-    if (!e->advised) {
-        for (auto &p : pl.pins) {
-            const TgpTensor &t = ctx->tensors[p.first];
-            CU(ctx, cudaMemAdvise(ctx->pools[t.pool].host_base + t.off, t.size, cudaMemAdviseSetPreferredLocation, e->device));
+    while (e->next_cmd < pl.cmds.size() && pl.cmds[e->next_cmd].wait_op <= limit) {
+        const TgpCmd &c = pl.cmds[e->next_cmd];
+        const TgpTensor &tt = ctx->tensors[c.tensor];
+        char *p = ctx->pools[tt.pool].host_base + tt.off;
+        cudaEvent_t ev;
+        if (c.kind == CMD_D2H) {
+            int rc = get_event(ctx, e->done_ev, (size_t)c.wait_op, &ev);
+            if (rc) return rc;
+            CU(ctx, cudaStreamWaitEvent(e->wb_stream, ev, 0));
+            CU(ctx, cudaMemPrefetchAsync(p, c.bytes, cudaCpuDeviceId, e->wb_stream));
+            CU(ctx, cudaEventRecord(e->wb_ev, e->wb_stream));
+            e->wb_pending = true;
+        } else {
+            if (c.wait_op > e->copy_waited_op) {
+                int rc = get_event(ctx, e->done_ev, (size_t)c.wait_op, &ev);
+                if (rc) return rc;
+                CU(ctx, cudaStreamWaitEvent(copy, ev, 0));
+                e->copy_waited_op = c.wait_op;
+            }
+            if (e->wb_pending) { CU(ctx, cudaStreamWaitEvent(copy, e->wb_ev, 0)); e->wb_pending = false; }
+            if (c.kind == CMD_H2D) CU(ctx, cudaMemPrefetchAsync(p, c.bytes, e->device, copy));
+            if (pl.op_last_place[c.first_use] == (int32_t)e->next_cmd) {
+                int rc = get_event(ctx, e->copied_ev, (size_t)c.first_use, &ev);
+                if (rc) return rc;
+                CU(ctx, cudaEventRecord(ev, copy));
+            }
+            if (c.arena_off >= pl.ring_base && tt.flags == TGP_T_READONLY && e->evict_explicit) e->evict_at[c.release_after].push_back(c.tensor);
         }
-        e->advised = true;
+        if (n_cmds) ++*n_cmds;
+        ++e->next_cmd;
     }
-    const size_t LOOKAHEAD = 8;
-    size_t upto = std::min(step_end, op_now + 1 + LOOKAHEAD);
-    for (size_t j = std::max(e->hinted_upto, op_now); j < upto; ++j) {
-        const TgpOp &o = ctx->ops[j];
-        if (pl.cls[j] != CLS_LINK) continue;
-        for (uint32_t k = 0; k < o.nacc; ++k) {
-            const tgp_access &a = ctx->acc[o.acc0 + k];
-            if (pl.zc[a.tensor]) continue;
-            const TgpTensor &t = ctx->tensors[a.tensor];
-            CU(ctx, cudaMemPrefetchAsync(ctx->pools[t.pool].host_base + t.off, t.size, e->device, copy));
+    return TGP_OK;
+}
+
+// after op i: record its completion if anything waits on it, and send home the read-only tensors released there
+static int after_op_managed(tgp_ctx *ctx, uint32_t i, cudaStream_t cs) {
+    TgpEngine *e = ctx->eng;
+    auto it = e->evict_at.find((int32_t)i);
+    const bool evict = it != e->evict_at.end();
+    if (!ctx->plan.op_is_wait_target[i] && !evict) return TGP_OK;
+    cudaEvent_t ev;
+    int rc = get_event(ctx, e->done_ev, i, &ev);
+    if (rc) return rc;
+    CU(ctx, cudaEventRecord(ev, cs));
+    if (evict) {
+        CU(ctx, cudaStreamWaitEvent(e->wb_stream, ev, 0));
+        for (uint32_t t : it->second) {
+            const TgpTensor &tt = ctx->tensors[t];
+            CU(ctx, cudaMemPrefetchAsync(ctx->pools[tt.pool].host_base + tt.off, tt.size, cudaCpuDeviceId, e->wb_stream));
         }
+        CU(ctx, cudaEventRecord(e->wb_ev, e->wb_stream));
+        e->wb_pending = true;
+        e->evict_at.erase(it);
     }
-    e->hinted_upto = std::max(e->hinted_upto, upto);
     return TGP_OK;
 }
 
@@ -370,17 +431,19 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
     const int32_t *tok = e->amax;
     if (tokens_host) { CU(ctx, cudaMemcpyAsync(e->tok, tokens_host, (size_t)M * 4, cudaMemcpyHostToDevice, cs)); tok = e->tok; }
     int rc;
+    const bool hints = ctx->variant == TGP_VAR_MANAGED_HINTS;
+    if (hints && (rc = advise_once(ctx))) return rc;
     if (ring && (rc = pump(ctx, (int32_t)st.op0 - 1, cp, &n_cmds))) return rc;
+    if (hints && (rc = pump_managed(ctx, (int32_t)st.op0 - 1, cp, &n_cmds))) return rc;
     const uint32_t qd = c.Hq * c.Dh, kd = c.Hkv * c.Dh;
     for (uint32_t i = st.op0; i < st.op0 + st.nops; ++i) {
         const TgpOp &o = ctx->ops[i];
-        if (ring && ctx->plan.op_last_place[i] >= 0) {
+        if ((ring || hints) && ctx->plan.op_last_place[i] >= 0) {
             if ((size_t)ctx->plan.op_last_place[i] >= e->next_cmd) return tgp_fail(ctx, TGP_E_STATE, "a placement was not enqueued before its op");
             cudaEvent_t ev;
             if ((rc = get_event(ctx, e->copied_ev, i, &ev))) return rc;
             CU(ctx, cudaStreamWaitEvent(cs, ev, 0));
         }
-        if (ctx->variant == TGP_VAR_MANAGED_HINTS && (rc = hint_ahead(ctx, i, st.op0 + st.nops, cp))) return rc;
         const uint32_t ti = i - st.op0;
         if (e->op_timing) {
             if (e->ta.size() <= ti) { e->ta.resize(ti + 1, nullptr); e->tb_.resize(ti + 1, nullptr); }
@@ -513,6 +576,9 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
                 CU(ctx, cudaEventRecord(ev, cs));
             }
             if ((rc = pump(ctx, (int32_t)i, cp, &n_cmds))) return rc;
+        } else if (hints) {
+            if ((rc = after_op_managed(ctx, i, cs))) return rc;
+            if ((rc = pump_managed(ctx, (int32_t)i, cp, &n_cmds))) return rc;
         }
     }
     e->pos += q_len;

@@ -27,7 +27,7 @@ class ManagedPool:
             self.ptr = 0
 
 
-def run(cfg, lay, machine, dev, fill, variants=(tb.VAR_MANAGED_DEMAND, tb.VAR_MANAGED_HINTS), decode_cap=16, slack=768 << 20, ballast=True):
+def run(cfg, lay, machine, dev, fill, variants=(tb.VAR_MANAGED_DEMAND, tb.VAR_MANAGED_HINTS), decode_cap=16, slack=64 << 20, ballast=True):
     """Returns {variant name: {...}}.  `fill(layout, uint8 array)` writes the pool contents.  Capacity: the workspace
     and then a ballast tensor are allocated ONCE, before the GPU has touched the managed pool, so that budget + slack
     bytes of device memory are all the managed pages can ever occupy; both variants then run under that same cap
