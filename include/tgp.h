@@ -158,6 +158,12 @@ int  tgp_trace_export(const tgp_ctx *ctx, void *buf, uint64_t *bytes);
 /* ---- policy (Section III-C, IV-C, IV-D) ------------------------------------------------------ */
 int  tgp_set_budget(tgp_ctx *ctx, uint64_t bytes);          /* device bytes for resident pool tensors     */
 int  tgp_set_variant(tgp_ctx *ctx, uint32_t variant, uint32_t policy_bits);
+/* Runtime monitor (Section IV-D): measured kernel times, one per op of the finished trace, in integer nanoseconds
+ * (0 = not measured: that op keeps its analytic class).  With a time t the link test becomes mig / Bl > t, i.e. an
+ * op is link-bound iff moving its pool bytes takes longer than the kernel ran; the next tgp_plan() uses it.
+ * n_ops == 0 clears the log; a new trace clears it too.  Integers make the re-plan reproducible: the same log fed
+ * to another planner gives the same schedule. */
+int  tgp_set_measured_times(tgp_ctx *ctx, const uint64_t *op_ns, uint64_t n_ops);
 /* Classifies ops, selects critical / zero-copy / pinned tensors, sizes the ring and builds the ordered
  * command list.  Host only; no CUDA call. */
 int  tgp_plan(tgp_ctx *ctx);

@@ -92,9 +92,16 @@ def alignup(x: int) -> int:
     return (x + ALIGN - 1) // ALIGN * ALIGN
 
 
-def classify(flops: int, hbm: int, mig: int, m: Machine, bit_p: bool = True) -> int:
+def classify(flops: int, hbm: int, mig: int, m: Machine, bit_p: bool = True, measured_ns: int = 0) -> int:
+    """measured_ns > 0: the runtime monitor's kernel time replaces both analytic roofs in the link test
+    (Section IV-D "Runtime Monitor": classes are re-evaluated from measured kernel time): LINK iff moving the op's
+    pool bytes over the link takes longer than the kernel itself ran, mig / Bl > t  <=>  mig * 1e9 > t_ns * Bl."""
     if mig > 0 and not bit_p:
         return CLS_LINK
+    if measured_ns > 0:
+        if mig * 1_000_000_000 > measured_ns * m.h2d_Bps:
+            return CLS_LINK
+        return CLS_COMPUTE if flops * m.hbm_Bps >= hbm * m.peak_flops else CLS_HBM
     if mig * m.peak_flops > flops * m.h2d_Bps and mig * m.hbm_Bps > hbm * m.h2d_Bps:
         return CLS_LINK
     if flops * m.hbm_Bps >= hbm * m.peak_flops:
@@ -125,17 +132,17 @@ class Plan:
         }
 
 
-def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A | BIT_P | BIT_ZC) -> Plan:
+def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A | BIT_P | BIT_ZC, measured_ns=None) -> Plan:
     """tensors: list of objects with .size .pool_off .flags; ops: list with .step .flops .hbm .acc;
-    steps: [(kind, first op, count)]."""
+    steps: [(kind, first op, count)]; measured_ns: optional per-op kernel times in integer nanoseconds (0 = none)."""
     T, N = len(tensors), len(ops)
     # 1-2: classes, criticality, score
     cls = []
     crit = [0] * T
     score = [0] * T
-    for op in ops:
+    for i, op in enumerate(ops):
         mig = sum(a[2] for a in op.acc)
-        c = classify(op.flops, op.hbm, mig, machine, bool(bits & BIT_P))
+        c = classify(op.flops, op.hbm, mig, machine, bool(bits & BIT_P), int(measured_ns[i]) if measured_ns is not None else 0)
         cls.append(c)
         if c == CLS_LINK:
             for (t, mode, touched) in op.acc:

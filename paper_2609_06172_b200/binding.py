@@ -71,6 +71,7 @@ _SIGS = {
     "tgp_trace_export": [_P, _P, C.POINTER(_U64)],
     "tgp_set_budget": [_P, _U64],
     "tgp_set_variant": [_P, _U32, _U32],
+    "tgp_set_measured_times": [_P, C.POINTER(_U64), _U64],
     "tgp_plan": [_P],
     "tgp_plan_export": [_P, _U32, _P, C.POINTER(_U64)],
     "tgp_set_arena": [_P, _P, _U64],
@@ -220,6 +221,14 @@ class Ctx:
 
     def set_variant(self, variant, bits):
         self._ck(lib().tgp_set_variant(self._h, variant, bits), "tgp_set_variant")
+
+    def set_measured_times(self, op_ns):
+        """Per-op kernel times in integer ns (0 = keep the analytic class); None or empty clears the log."""
+        if op_ns is None or len(op_ns) == 0:
+            self._ck(lib().tgp_set_measured_times(self._h, None, 0), "tgp_set_measured_times")
+            return
+        a = np.ascontiguousarray(op_ns, dtype=np.uint64)
+        self._ck(lib().tgp_set_measured_times(self._h, a.ctypes.data_as(C.POINTER(_U64)), len(a)), "tgp_set_measured_times")
 
     def plan(self):
         self._ck(lib().tgp_plan(self._h), "tgp_plan")

@@ -160,6 +160,7 @@ int tgp_tensor_identity(const tgp_ctx *ctx, uint32_t id, uint64_t *site_hash, ui
 int tgp_trace_begin(tgp_ctx *ctx) {
     if (!ctx) return TGP_E_INVAL;
     ctx->ops.clear(); ctx->acc.clear(); ctx->steps.clear();
+    ctx->measured_ns.clear();
     ctx->plan = TgpPlan();
     ctx->tracing = true; ctx->traced = false;
     return TGP_OK;
@@ -219,14 +220,29 @@ int tgp_set_budget(tgp_ctx *ctx, uint64_t bytes) {
     return TGP_OK;
 }
 
+int tgp_set_measured_times(tgp_ctx *ctx, const uint64_t *op_ns, uint64_t n_ops) {
+    if (!ctx) return TGP_E_INVAL;
+    if (!n_ops) { ctx->measured_ns.clear(); ctx->plan.valid = false; return TGP_OK; }
+    if (!op_ns) return TGP_E_INVAL;
+    if (!ctx->traced || n_ops != ctx->ops.size()) return tgp_fail(ctx, TGP_E_STATE, "one time per op of the finished trace is required");
+    ctx->measured_ns.assign(op_ns, op_ns + n_ops);
+    ctx->plan.valid = false;
+    return TGP_OK;
+}
+
 int tgp_set_variant(tgp_ctx *ctx, uint32_t variant, uint32_t bits) {
     if (!ctx || variant > TGP_VAR_MANAGED_DEMAND || (bits & ~7u)) return TGP_E_INVAL;
     ctx->variant = variant; ctx->bits = bits; ctx->plan.valid = false;
     return TGP_OK;
 }
 
-static uint8_t classify(const tgp_machine &m, uint64_t flops, uint64_t hbm, uint64_t mig, bool selective) {
+static uint8_t classify(const tgp_machine &m, uint64_t flops, uint64_t hbm, uint64_t mig, bool selective, uint64_t measured_ns) {
     if (mig > 0 && !selective) return CLS_LINK;
+    if (measured_ns > 0) {
+        // runtime monitor: the measured kernel time replaces both analytic roofs in the link test, mig/Bl > t
+        if ((u128)mig * 1000000000ull > (u128)measured_ns * m.h2d_Bps) return CLS_LINK;
+        return (u128)flops * m.hbm_Bps >= (u128)hbm * m.peak_flops ? CLS_COMPUTE : CLS_HBM;
+    }
     // link time strictly above both other roofs: mig/Bl > flops/P and mig/Bl > hbm/Bh
     if ((u128)mig * m.peak_flops > (u128)flops * m.h2d_Bps && (u128)mig * m.hbm_Bps > (u128)hbm * m.h2d_Bps) return CLS_LINK;
     if ((u128)flops * m.hbm_Bps >= (u128)hbm * m.peak_flops) return CLS_COMPUTE;
@@ -246,7 +262,7 @@ int tgp_plan(tgp_ctx *ctx) {
         const TgpOp &o = ctx->ops[i];
         uint64_t mig = 0;
         for (uint32_t k = 0; k < o.nacc; ++k) mig += ctx->acc[o.acc0 + k].touched_bytes;
-        pl.cls[i] = classify(ctx->mach, o.flops, o.hbm, mig, ctx->bits & TGP_BIT_P);
+        pl.cls[i] = classify(ctx->mach, o.flops, o.hbm, mig, ctx->bits & TGP_BIT_P, ctx->measured_ns.size() == N ? ctx->measured_ns[i] : 0);
         if (pl.cls[i] == CLS_LINK)
             for (uint32_t k = 0; k < o.nacc; ++k) {
                 const tgp_access &a = ctx->acc[o.acc0 + k];

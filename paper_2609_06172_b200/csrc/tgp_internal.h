@@ -61,6 +61,7 @@ struct tgp_ctx {
     // policy inputs
     uint64_t budget = 0;
     uint32_t variant = TGP_VAR_EXPLICIT_RING, bits = TGP_BIT_A | TGP_BIT_P | TGP_BIT_ZC;
+    std::vector<uint64_t> measured_ns;                   // runtime monitor: kernel time per op in ns (0 = not measured), or empty
     TgpPlan plan;
     // model
     bool bound = false;

@@ -417,3 +417,39 @@ def test_lockstep_parity_config_2_full_size_prefill_and_decode():
     worst, flips = _lockstep(cfg, lay, pool, W, 2, np.float32)
     assert worst < 5e-3
     assert all(v < 0.02 for k, v in flips.items() if k != "o") and flips["o"] < 0.5
+
+
+def test_runtime_monitor_replan_from_measured_kernel_times():
+    """Second half of the paper's runtime monitor: kernel timestamps of a real run re-classify the ops, the schedule is
+    rebuilt, and (the log being integers) the oracle's planner rebuilds the identical schedule from the same log.
+    Placement changes, results do not: logits are bitwise equal before and after the re-plan."""
+    cfg = si.CONFIGS[1]
+    lay, pool, s, blobs, T = setup(cfg)
+    r = Runner(s, cfg.B * cfg.S)
+    prompt = si.prompt_tokens(cfg)
+    forced = (np.arange(cfg.B * T, dtype=np.int32).reshape(cfg.B, T) * 313 + 7) % cfg.V
+    before, _ = r.generate(prompt, T, forced=forced)
+    ops, steps = trace.run_trace(lay)
+    ns = np.zeros(len(ops), dtype=np.uint64)
+    r.reset()
+    s.ctx.set_op_timing(True)
+    for k in range(1 + T):
+        tok = prompt if k == 0 else np.ascontiguousarray(forced[:, k - 1:k], dtype=np.int32)
+        r.step(tb.PREFILL if k == 0 else tb.DECODE, tok, tok.shape[1], want_stats=True)
+        first, ms = s.ctx.op_times()
+        ns[first:first + len(ms)] = np.maximum(1, np.round(ms.astype(np.float64) * 1e6)).astype(np.uint64)
+    s.ctx.set_op_timing(False)
+    r.sync()
+    assert (ns > 0).all()
+    s.ctx.set_measured_times(ns)
+    s.ctx.plan()
+    got = s.ctx.plan_blobs()
+    want = policy.plan(lay.tensors, ops, steps, policy.Machine(**MACHINE), lay.budget, measured_ns=ns.tolist()).blobs()
+    assert got == want
+    validate.check(lay.tensors, ops, steps, lay.budget, got)
+    # microsecond kernels on a 55 GB/s link: small tensors' ops stop being link-bound
+    assert got["classes"] != blobs["classes"]
+    after, _ = r.generate(prompt, T, forced=forced)
+    for a, b in zip(before, after):
+        assert np.array_equal(a, b)
+    s.close()

@@ -228,3 +228,47 @@ def test_model_bind_rejects_bad_shapes_and_roles():
         s.ctx.model_trace(40, 16)                                # S + T beyond max_len
     assert ei.value.code == tb.E_INVAL
     s.close()
+
+
+def test_replan_from_a_timing_log_is_bit_exact_and_changes_classes():
+    """Runtime monitor: the same integer log of kernel times fed to both planners gives the same schedule; an op whose
+    kernel ran longer than its bytes take on the link stops being link-bound, and its tensors lose their pin score."""
+    lay = si.build_layout(si.CONFIGS[1])
+    ops, steps = trace.run_trace(lay)
+    rng = np.random.default_rng(11)
+    # synthetic log: most ops fast (1 us), a third not measured (0), norm ops slow (20 us >> 512 B over the link)
+    ns = np.where(rng.random(len(ops)) < 0.33, 0, 1000).astype(np.uint64)
+    for i, o in enumerate(ops):
+        if o.kind == trace.OP_RMSNORM:
+            ns[i] = 20000
+    s = Session(lay, MACHINE)
+    base = s.plan()
+    s.ctx.set_measured_times(ns)
+    s.ctx.plan()
+    got = s.ctx.plan_blobs()
+    want = policy.plan(lay.tensors, ops, steps, policy.Machine(**MACHINE), lay.budget, measured_ns=ns.tolist()).blobs()
+    assert got == want
+    validate.check(lay.tensors, ops, steps, lay.budget, got)
+    assert got["classes"] != base["classes"]
+    norm_ops = [i for i, o in enumerate(ops) if o.kind == trace.OP_RMSNORM]
+    assert all(base["classes"][i] == policy.CLS_LINK for i in norm_ops) and all(got["classes"][i] != policy.CLS_LINK for i in norm_ops)
+    gain = lay.blocks(si.K_G1, 0)[0].tid
+    crit = lambda blobs, t: blobs["tensors"][t * 10]
+    assert crit(base, gain) == 1 and crit(got, gain) == 0
+    # clearing the log restores the analytic plan; a log of the wrong length is refused
+    s.ctx.set_measured_times(None)
+    s.ctx.plan()
+    assert s.ctx.plan_blobs() == base
+    with pytest.raises(tb.TgpError) as ei:
+        s.ctx.set_measured_times(ns[:-1])
+    assert ei.value.code == tb.E_STATE
+    s.close()
+
+
+def test_measured_time_link_test_by_hand():
+    toy = policy.Machine(1000, 100, 10, 10)            # link 10 B/s
+    # 100 bytes over the link take 10 s: a 9 s kernel is link-bound, a 10 s or 11 s kernel is not
+    assert policy.classify(5000, 300, 100, toy, measured_ns=9_000_000_000) == policy.CLS_LINK
+    assert policy.classify(5000, 300, 100, toy, measured_ns=10_000_000_000) == policy.CLS_COMPUTE
+    assert policy.classify(100, 600, 100, toy, measured_ns=11_000_000_000) == policy.CLS_HBM
+    assert policy.classify(5000, 300, 100, toy, measured_ns=0) == policy.CLS_LINK          # no measurement: analytic
