@@ -240,6 +240,13 @@ int  tgp_k_gemm(const void *A_dev, const void *W_dev, float *C_dev, uint32_t M, 
 /* Which kernel serves M > 16: 0 (default) the tcgen05 tensor-core GEMM, 1 the CUDA-core tile kernel (an on-device
  * cross-check).  M <= 16 always takes the weight-streaming GEMV.  Process-wide. */
 int  tgp_k_gemm_select(int impl);
+/* Which kernel serves 3 <= M <= 32 (K % 32 == 0): 0 (default) the weight-streaming tensor-core kernel, 1 the
+ * CUDA-core GEMV (M <= 16) / GEMM paths (an on-device cross-check).  Process-wide. */
+int  tgp_k_skinny_select(int impl);
+/* Weight-streaming launches (M <= 32) use programmatic dependent launch so that a launch may begin reading its
+ * weights while the previous kernel of the stream drains; 0 switches that off (each launch then starts after the
+ * previous one has completed).  Results are identical either way.  Process-wide; default on. */
+int  tgp_k_gemv_overlap(int enable);
 /* Tensor-core GEMM variant: 0 (default) picks by problem size, 1 forces the 128x128 one-tile-per-CTA kernel,
  * 2 forces the persistent 128x256 kernel with double-buffered accumulators.  Process-wide; for tests and timing. */
 int  tgp_k_gemm_tc_variant(int variant);

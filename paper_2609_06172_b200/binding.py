@@ -92,6 +92,8 @@ _SIGS = {
     "tgp_k_gemm": [_P, _P, _P, _U32, _U32, _U32, _U32, _U32, C.c_int, _P],
     "tgp_k_gemm_select": [C.c_int],
     "tgp_k_attn_select": [C.c_int],
+    "tgp_k_gemv_overlap": [C.c_int],
+    "tgp_k_skinny_select": [C.c_int],
     "tgp_k_gemm_tc_variant": [C.c_int],
     "tgp_k_gemm_status": [C.POINTER(C.c_int)],
     "tgp_k_rope_tables": [_U32, _U32, C.c_float, _P, _P],
@@ -342,6 +344,14 @@ def k_gemm(A, W, Cout, M, n, K, ldc, col0, accumulate, stream=None):
 
 def k_gemm_select(impl):
     _k(lib().tgp_k_gemm_select(impl), "tgp_k_gemm_select")
+
+
+def k_skinny_select(impl):
+    _k(lib().tgp_k_skinny_select(impl), "tgp_k_skinny_select")
+
+
+def k_gemv_overlap(enable):
+    _k(lib().tgp_k_gemv_overlap(int(enable)), "tgp_k_gemv_overlap")
 
 
 def k_attn_select(impl):

@@ -77,6 +77,11 @@ __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, c
                                                    uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarp = (gridDim.x * blockDim.x) >> 5;
+    // Programmatic dependent launch: the weights are not produced by the previous kernel in the stream, so this grid
+    // may start streaming them while that kernel drains.  Everything it does produce (the activations A, the output C)
+    // is touched only after griddepcontrol.wait, which returns once the previous grid has completed and flushed.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    bool synced = false;
     for (uint32_t row0 = gwarp * R; row0 < n; row0 += nwarp * R) {
         float acc[R][MT];
 #pragma unroll
@@ -93,6 +98,7 @@ __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, c
 #pragma unroll
                 for (int r = 0; r < R; ++r)
                     wv[u][r] = (k0 + 256 * u < K) ? __ldcs(reinterpret_cast<const uint4 *>(wrow[r] + k0 + 256 * u)) : make_uint4(0, 0, 0, 0);
+            if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const uint32_t k = k0 + 256 * u;
@@ -110,6 +116,7 @@ __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, c
                 }
             }
         }
+        if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }      // K == 0 never happens; belt and braces
 #pragma unroll
         for (int r = 0; r < R; ++r)
 #pragma unroll
@@ -118,6 +125,66 @@ __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, c
                 if (lane == 0 && row0 + r < n && m < (int)Mrows) {
                     float *c = C + (size_t)m * ldc + col0 + row0 + r;
                     *c = accumulate ? *c + s : s;
+                }
+            }
+    }
+}
+
+// ---- skinny GEMM for 3 <= M <= 32 activation rows: weight streaming through mma.sync ---------------------------
+// out^T[16 rows of W, 8 activation rows] += W[16 x 16] * x^T[16 x 8] per instruction.  Each lane loads 16 contiguous
+// bytes (8 values of K) of W rows g and g+8 and of activation row g straight from global memory; the 8 values feed two
+// instructions.  Which physical k lands in which logical k-slot of the instruction does not matter for a dot product
+// as long as both operands use the same assignment, and they do (same lane, same byte offsets), so no shuffle or
+// shared-memory staging is needed and every weight byte is loaded exactly once.  Persistent warps, 16 rows each,
+// NB groups of 8 activation rows re-use the weight registers.  Same dependent-launch protocol as gemv_kernel.
+__device__ __forceinline__ void mma_bf16_16816(float *d, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int NB, int U>
+__global__ void __launch_bounds__(256) gemv_mma_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+                                                       uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
+    const uint32_t lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
+    const uint32_t gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarp = (gridDim.x * blockDim.x) >> 5;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    bool synced = false;
+    for (uint32_t row0 = gwarp * 16; row0 < n; row0 += nwarp * 16) {
+        const bf16 *wlo = W + (size_t)min(row0 + g, n - 1) * K + c * 8;        // tail rows re-read the last row, never stored
+        const bf16 *whi = W + (size_t)min(row0 + g + 8, n - 1) * K + c * 8;
+        float acc[NB][4];
+#pragma unroll
+        for (int b = 0; b < NB; ++b) { acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f; }
+        for (uint32_t k0 = 0; k0 < K; k0 += 32 * U) {
+            uint4 lo[U], hi[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const bool in = k0 + 32 * u < K;
+                lo[u] = in ? __ldcs(reinterpret_cast<const uint4 *>(wlo + k0 + 32 * u)) : make_uint4(0, 0, 0, 0);
+                hi[u] = in ? __ldcs(reinterpret_cast<const uint4 *>(whi + k0 + 32 * u)) : make_uint4(0, 0, 0, 0);
+            }
+            if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t k = k0 + 32 * u;
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    const uint32_t m = b * 8 + g;
+                    const uint4 xv = (k < K && m < Mrows) ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k + c * 8)) : make_uint4(0, 0, 0, 0);
+                    mma_bf16_16816(acc[b], lo[u].x, hi[u].x, lo[u].y, hi[u].y, xv.x, xv.y);
+                    mma_bf16_16816(acc[b], lo[u].z, hi[u].z, lo[u].w, hi[u].w, xv.z, xv.w);
+                }
+            }
+        }
+        if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
+#pragma unroll
+        for (int b = 0; b < NB; ++b)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t m = b * 8 + 2 * c + (i & 1), row = row0 + g + 8 * (i >> 1);
+                if (m < Mrows && row < n) {
+                    float *p = C + (size_t)m * ldc + col0 + row;
+                    *p = accumulate ? *p + acc[b][i] : acc[b][i];
                 }
             }
     }
@@ -536,6 +603,8 @@ int tgpk_rmsnorm(const float *x, uint32_t ldx, const void *g, void *h, uint32_t 
     return TGP_OK;
 }
 
+static int g_gemv_pdl = 1;       // consecutive weight-streaming launches may overlap (programmatic dependent launch)
+
 template <int MT, int R, int U>
 static void launch_gemv(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int acc, cudaStream_t st) {
     static int blocks_per_sm = 0, sms = 0;
@@ -547,7 +616,103 @@ static void launch_gemv(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, 
         if (sms < 1) sms = 148;
     }
     uint32_t need = (n + R * 8 - 1) / (R * 8), full = (uint32_t)(sms * blocks_per_sm);
-    gemv_kernel<MT, R, U><<<need < full ? need : full, 256, 0, st>>>(A, W, C, Mrows, n, K, ldc, col0, acc);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(need < full ? need : full);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = g_gemv_pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, gemv_kernel<MT, R, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
+}
+
+// Same product for blocks with few rows: one CTA owns 16 rows of W and its 8 warps split K (interleaved chunks of
+// 32*U), so n/16 CTAs of 8 warps fill the machine where n/16 warps would not.  The eight partial tiles meet in shared
+// memory and are summed in warp order: deterministic.
+template <int NB, int U>
+__global__ void __launch_bounds__(256) gemv_mma_splitk_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+                                                              uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
+    __shared__ float part[8][NB * 4][32];
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, c = lane & 3;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    bool synced = false;
+    for (uint32_t row0 = blockIdx.x * 16; row0 < n; row0 += gridDim.x * 16) {
+        const bf16 *wlo = W + (size_t)min(row0 + g, n - 1) * K + c * 8;
+        const bf16 *whi = W + (size_t)min(row0 + g + 8, n - 1) * K + c * 8;
+        float acc[NB][4];
+#pragma unroll
+        for (int b = 0; b < NB; ++b) { acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f; }
+        for (uint32_t k0 = warp * 32 * U; k0 < K; k0 += 8 * 32 * U) {
+            uint4 lo[U], hi[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const bool in = k0 + 32 * u < K;
+                lo[u] = in ? __ldcs(reinterpret_cast<const uint4 *>(wlo + k0 + 32 * u)) : make_uint4(0, 0, 0, 0);
+                hi[u] = in ? __ldcs(reinterpret_cast<const uint4 *>(whi + k0 + 32 * u)) : make_uint4(0, 0, 0, 0);
+            }
+            if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t k = k0 + 32 * u;
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    const uint32_t m = b * 8 + g;
+                    const uint4 xv = (k < K && m < Mrows) ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k + c * 8)) : make_uint4(0, 0, 0, 0);
+                    mma_bf16_16816(acc[b], lo[u].x, hi[u].x, lo[u].y, hi[u].y, xv.x, xv.y);
+                    mma_bf16_16816(acc[b], lo[u].z, hi[u].z, lo[u].w, hi[u].w, xv.z, xv.w);
+                }
+            }
+        }
+        if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
+#pragma unroll
+        for (int b = 0; b < NB; ++b)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) part[warp][b * 4 + i][lane] = acc[b][i];
+        __syncthreads();
+        for (uint32_t v = threadIdx.x; v < NB * 4 * 32; v += 256) {
+            const uint32_t slot = v >> 5, ln = v & 31, b = slot >> 2, i = slot & 3;
+            float sum = 0.f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) sum += part[w][slot][ln];
+            const uint32_t m = b * 8 + 2 * (ln & 3) + (i & 1), row = row0 + (ln >> 2) + 8 * (i >> 1);
+            if (m < Mrows && row < n) {
+                float *p = C + (size_t)m * ldc + col0 + row;
+                *p = accumulate ? *p + sum : sum;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+template <int NB, int U>
+static void launch_gemv_mma(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int acc, cudaStream_t st) {
+    static int blocks_per_sm = 0, sms = 0;
+    if (!blocks_per_sm) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, gemv_mma_kernel<NB, U>, 256, 0) != cudaSuccess || blocks_per_sm < 1) blocks_per_sm = 1;
+        if (sms < 1) sms = 148;
+    }
+    static int blocks_per_sm_split = 0;
+    if (!blocks_per_sm_split && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm_split, gemv_mma_splitk_kernel<NB, U>, 256, 0) != cudaSuccess || blocks_per_sm_split < 1))
+        blocks_per_sm_split = 1;
+    const bool split = n < 16u * 8u * (uint32_t)sms;                 // too few 16-row groups to give every SM eight warps
+    uint32_t need = split ? (n + 15) / 16 : (n + 16 * 8 - 1) / (16 * 8);
+    uint32_t full = (uint32_t)(sms * (split ? blocks_per_sm_split : blocks_per_sm));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(need < full ? need : full);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = g_gemv_pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (split) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
+    else cudaLaunchKernelEx(&cfg, gemv_mma_kernel<NB, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
 }
 
 // rows per warp: fewer when the block has few rows, so that every SM still gets warps
@@ -562,13 +727,18 @@ static void launch_gemv_rows(const bf16 *A, const bf16 *W, float *C, uint32_t Mr
     }
 }
 
+static int g_skinny_impl = 0;    // 0: tensor-core skinny kernel for 3 <= M <= 32; 1: CUDA-core GEMV (an on-device cross-check)
 static int g_gemm_impl = 0;      // 0: tensor cores for M > 16; 1: CUDA-core tiles (kept as an on-device cross-check)
 
 int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
     if (!M || !n) return TGP_OK;
     if (K % 8 || !K) return TGP_E_INVAL;
     const bf16 *a = (const bf16 *)A, *w = (const bf16 *)W;
-    if (M <= 16) {
+    if (M >= 3 && M <= 32 && K % 32 == 0 && g_skinny_impl == 0) {
+        if (M <= 8) launch_gemv_mma<1, 4>(a, w, C, M, n, K, ldc, col0, accumulate, st);
+        else if (M <= 16) launch_gemv_mma<2, 4>(a, w, C, M, n, K, ldc, col0, accumulate, st);
+        else launch_gemv_mma<4, 2>(a, w, C, M, n, K, ldc, col0, accumulate, st);
+    } else if (M <= 16) {
         for (uint32_t m0 = 0; m0 < M; m0 += 8) {
             uint32_t mr = M - m0 < 8 ? M - m0 : 8;
             const bf16 *am = a + (size_t)m0 * K;
@@ -667,6 +837,17 @@ int tgp_k_embed(const void *table, const int32_t *tok_dev, float *x_dev, uint32_
 int tgp_k_rmsnorm(const float *x_dev, uint32_t ldx, const void *g_dev, void *h_dev, uint32_t M, uint32_t d, float eps, void *stream) {
     if (!x_dev || !g_dev || !h_dev) return TGP_E_INVAL;
     return tgpk_rmsnorm(x_dev, ldx, g_dev, h_dev, M, d, eps, (cudaStream_t)stream);
+}
+
+int tgp_k_skinny_select(int impl) {
+    if (impl != 0 && impl != 1) return TGP_E_INVAL;
+    g_skinny_impl = impl;
+    return TGP_OK;
+}
+
+int tgp_k_gemv_overlap(int enable) {
+    g_gemv_pdl = enable ? 1 : 0;
+    return TGP_OK;
 }
 
 int tgp_k_attn_select(int impl) {

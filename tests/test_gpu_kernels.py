@@ -252,3 +252,52 @@ def test_swiglu_and_argmax():
     torch.cuda.synchronize()
     assert am.cpu().numpy().tolist() == np.argmax(lg, axis=1).tolist()
     assert am.cpu().numpy()[1] == 77 and am.cpu().numpy()[2] == 0 and am.cpu().numpy()[3] == V - 1
+
+
+def test_overlapping_gemv_launches_keep_their_dependencies():
+    """Back-to-back weight-streaming launches accumulate into the same output (each depends on the one before through C).
+    With dependent-launch overlap a launch starts loading weights early but must not touch C before its predecessor has
+    finished: the chain must give bit-identical results with overlap on and off, and equal the oracle's sum."""
+    M, n, K, reps = 2, 4100, 2048, 12
+    a_bits = rnd_bits(21, M * K).reshape(M, K)
+    A = bf16_dev(a_bits)
+    Ws = [rnd_bits(30 + i, n * K).reshape(n, K) for i in range(3)]
+    Wd = [bf16_dev(w) for w in Ws]
+    outs = []
+    for overlap in (1, 0):
+        tb.k_gemv_overlap(overlap)
+        Cd = torch.zeros(M, n, dtype=torch.float32, device=DEV)
+        for i in range(reps):
+            tb.k_gemm(A, Wd[i % 3], Cd, M, n, K, n, 0, 1)
+        torch.cuda.synchronize()
+        outs.append(Cd.cpu().numpy())
+    tb.k_gemv_overlap(1)
+    assert np.array_equal(outs[0], outs[1])
+    o = oracle()
+    a = si.bf16_bits_to_f32(a_bits)
+    want = sum(o.linear(a, si.bf16_bits_to_f32(Ws[i % 3]).astype(np.float64)).astype(np.float64) for i in range(reps))
+    assert np.abs(outs[0] - want).max() < 1e-4 * np.abs(want).max()
+
+
+@pytest.mark.parametrize("M,n,K", [(3, 100, 64), (8, 4096, 4096), (8, 1030, 512), (13, 77, 128), (16, 260, 1024), (17, 64, 96), (24, 2049, 2048),
+                                   (32, 4100, 8192), (5, 16, 32)])
+@pytest.mark.parametrize("accumulate", [0, 1])
+def test_skinny_tensor_core_gemv_matches_oracle_and_cuda_core_path(M, n, K, accumulate):
+    a_bits, w_bits = rnd_bits(41, M * K).reshape(M, K), rnd_bits(42, n * K).reshape(n, K)
+    A, W = bf16_dev(a_bits), bf16_dev(w_bits)
+    c0 = np.random.default_rng(M + n).standard_normal((M, n + 8)).astype(np.float32) * 0.01
+    outs = []
+    for impl in (0, 1):
+        tb.k_skinny_select(impl)
+        Cd = torch.from_numpy(c0.copy()).to(DEV)
+        tb.k_gemm(A, W, Cd, M, n, K, n + 8, 4, accumulate)
+        torch.cuda.synchronize()
+        outs.append(Cd.cpu().numpy())
+    tb.k_skinny_select(0)
+    want = c0.astype(np.float64).copy()
+    prod = oracle().linear(si.bf16_bits_to_f32(a_bits), si.bf16_bits_to_f32(w_bits).astype(np.float64)).astype(np.float64)
+    want[:, 4:4 + n] = prod + (c0[:, 4:4 + n] if accumulate else 0)
+    scale = max(np.abs(prod).max(), 0.01)
+    assert np.abs(outs[0] - want).max() < 2e-5 * scale + 1e-7
+    assert np.abs(outs[0] - outs[1]).max() < 2e-5 * scale + 1e-7
+    assert np.array_equal(outs[0][:, :4], c0[:, :4]) and np.array_equal(outs[0][:, 4 + n:], c0[:, 4 + n:])
