@@ -275,6 +275,7 @@ def main():
     ap.add_argument("--kernel-loop", choices=["decode", "prefill"], default=None,
                     help="only run the back-to-back weight-product loop of one step (small, for ncu captures)")
     ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--graph", action="store_true", help="replay the whole planned run as one CUDA graph (dense models; for host-bound tiny steps)")
     ap.add_argument("--layers", type=int, default=None, help="run the shape at reduced depth; a byte budget is scaled in proportion")
     ap.add_argument("--bits", type=int, default=7, help="policy bits: 1 affinity/pins, 2 roofline selectivity, 4 zero-copy")
     ap.add_argument("--budget-frac", type=float, default=None, help="device budget as a fraction of the pool (oversubscription sweep)")
@@ -344,7 +345,12 @@ def main():
     logits_host = torch.empty((cfg.B, cfg.V), dtype=torch.float32).pin_memory()
     T = cfg.T
 
+    use_graph = args.graph and not cfg.E
+
     def one_pass(e2e=False):
+        if use_graph and not e2e:
+            r.replay()
+            return
         r.reset()
         r.step(tb.PREFILL, prompt_pinned.numpy(), cfg.S)
         for t in range(T):
@@ -378,6 +384,13 @@ def main():
         barrier()
         return whole_job_rate(1, ev0.elapsed_time(ev1), dist, dev)[1]
 
+    if use_graph:
+        r.reset()
+        r.step(tb.PREFILL, prompt_pinned.numpy(), cfg.S)             # one plain pass first: kernel attributes are set up outside capture
+        for t in range(T):
+            r.step(tb.DECODE, None, 1)
+        r.sync()
+        r.capture_run(prompt_pinned, T)
     for _ in range(args.warmup):
         one_pass(False)
     r.sync()
@@ -386,6 +399,9 @@ def main():
         sampler.start()
     ms = timed(args.steps, False)
     clocks = sampler.stop() if rank == 0 else None
+    if use_graph:
+        r.sync()
+        r.reset()
     one_pass(True)
     ms_e2e = timed(args.steps, True)
     tokens_per_pass = cfg.B * (cfg.S + T)
@@ -482,15 +498,28 @@ def main():
                  "link_gbs_achieved": L_plan / t_meas / 1e9, "link_gbs_peak": MACHINE["h2d_Bps"] / 1e9,
                  "h2d_bytes": int(totals[:, 0].sum()), "d2h_bytes": L_d2h, "zero_copy_bytes": int(totals[:, 2].sum()),
                  "flops": F, "hbm_bytes": H}
+    # the paper's motivation experiment (Section III-B) on this workload, analytically: a prefetcher that sees only
+    # allocator segments (20 MiB, the large-block size of PyTorch's caching allocator) and prefetches every segment
+    # an op's tensors overlap moves this many useless bytes per useful byte
+    SEG = 20 << 20
+    useful = useless = 0
+    for o in ops:
+        segs = set()
+        for (t, mode, touched) in o[6]:
+            tt = lay.tensors[t]
+            segs.update(range(tt.pool_off // SEG, (tt.pool_off + tt.size - 1) // SEG + 1))
+            useful += touched
+        useless += len(segs) * SEG
+    object_level = {"segment_bytes": SEG, "useless_over_useful": (useless - useful) / max(1, useful), "kind": "analytic, from the trace"}
     out = {"metric": "tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
            "data": "synthetic", "config": {"workload": workload_name(cfg, lay), "l2": f"inputs larger than L2: every decode step streams the {lay.pool_bytes / 1e9:.1f} GB pool",
-                                           "step": "prefill + all decode steps from a cold arena", "tokens_per_step": tokens_per_pass,
+                                           "step": "prefill + all decode steps from a cold arena" + (", replayed as one CUDA graph" if use_graph else ""), "tokens_per_step": tokens_per_pass,
                                            "parallelism": "replicas" if world > 1 else "single"},
            "prefill_tok_s": cfg.B * cfg.S / (step_ms[0] * 1e-3), "decode_tok_s": cfg.B * T / (sum(step_ms[1:]) * 1e-3) if T else None,
            "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": int(totals[:, 0].sum()) + cfg.B * (cfg.S + T) * 4,
                    "d2h_bytes_per_step": L_d2h + cfg.B * (T + 1) * 4 + cfg.B * cfg.V * 4},
-           "policy_bits": args.bits, "trace_mismatches": mismatches, "moe_profile_pass_s": profile_s,
+           "object_level_prefetch": object_level, "policy_bits": args.bits, "trace_mismatches": mismatches, "moe_profile_pass_s": profile_s,
            "gpu_launches": launches * args.steps, "clocks": clocks, "roofline": roof, "step_roofline": step_roof,
            "kernels": {f"{k[0]}:{k[1]}": {"ms": round(v, 3), "launches": kind_n[k], "GBps": round(kind_bytes[k] / (v * 1e-3) / 1e9, 1),
                                            "TFLOPs": round(kind_flops[k] / (v * 1e-3) / 1e12, 2)} for k, v in sorted(kind_ms.items())}}

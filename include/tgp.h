@@ -227,6 +227,18 @@ int  tgp_tap_index(tgp_ctx *ctx, uint64_t *out, uint64_t *n_words);
 int  tgp_set_op_timing(tgp_ctx *ctx, int enable);
 int  tgp_op_times(tgp_ctx *ctx, float *ms, uint32_t capacity, uint32_t *first_op, uint32_t *n_ops);
 
+/* Whole-run CUDA graph (dense models, explicit engine).  Between tgp_run_capture_begin() and tgp_run_capture_end()
+ * the caller issues the run's tgp_step() calls as usual (same two streams, stats == NULL, decode steps with
+ * tokens_host == NULL so the device's own argmax is fed back); nothing executes, the copies, kernels and their
+ * cross-stream ordering are recorded instead.  tgp_run_graph_launch() then replays the whole run - cold arena to
+ * last logits - with a single launch; logits_dev / argmax_dev given to the captured steps receive each step's result.
+ * The prompt buffer given to the captured prefill step is read again at every replay and must stay valid.
+ * Call tgp_run_reset() before capturing, run the plan once un-captured first (one-time kernel attribute set-up is not
+ * capturable), and call tgp_run_reset() again before going back to plain tgp_step() calls. */
+int  tgp_run_capture_begin(tgp_ctx *ctx, void *compute_stream, void *copy_stream);
+int  tgp_run_capture_end(tgp_ctx *ctx);
+int  tgp_run_graph_launch(tgp_ctx *ctx, void *stream);
+
 /* ---- single kernels (device pointers; used by the model step, exported for parity tests and timing) ---- */
 /* x[m, :] = fp32(table[tok[m], :]);  table bf16 [V, d] (device or mapped host), tok int32 [M]. */
 int  tgp_k_embed(const void *table, const int32_t *tok_dev, float *x_dev, uint32_t M, uint32_t d, void *stream);

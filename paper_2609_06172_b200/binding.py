@@ -83,6 +83,9 @@ _SIGS = {
     "tgp_managed_alloc": [C.POINTER(_P), _U64],
     "tgp_managed_free": [_P],
     "tgp_managed_evict": [_P, _U64],
+    "tgp_run_capture_begin": [_P, _P, _P],
+    "tgp_run_capture_end": [_P],
+    "tgp_run_graph_launch": [_P, _P],
     "tgp_set_tap": [_P, _P, _U64],
     "tgp_tap_index": [_P, C.POINTER(_U64), C.POINTER(_U64)],
     "tgp_set_op_timing": [_P, C.c_int],
@@ -273,6 +276,15 @@ class Ctx:
         a = np.zeros(max(1, n.value), dtype=np.uint32)
         self._ck(lib().tgp_expert_counts(self._h, a.ctypes.data_as(C.POINTER(_U32)), C.byref(n)), "tgp_expert_counts")
         return a[:n.value].reshape(-1, L, E)
+
+    def run_capture_begin(self, compute_stream, copy_stream):
+        self._ck(lib().tgp_run_capture_begin(self._h, _ptr(compute_stream), _ptr(copy_stream)), "tgp_run_capture_begin")
+
+    def run_capture_end(self):
+        self._ck(lib().tgp_run_capture_end(self._h), "tgp_run_capture_end")
+
+    def run_graph_launch(self, stream):
+        self._ck(lib().tgp_run_graph_launch(self._h, _ptr(stream)), "tgp_run_graph_launch")
 
     def set_tap(self, tap, nbytes):
         self._ck(lib().tgp_set_tap(self._h, _ptr(tap), nbytes), "tgp_set_tap")

@@ -52,6 +52,12 @@ struct TgpEngine {
     bool op_timing = false;
     std::vector<cudaEvent_t> ta, tb_;
     uint32_t timed_op0 = 0, timed_nops = 0;
+    // whole-run CUDA graph (dense models): capture state and the instantiated graph
+    bool capturing = false;
+    cudaStream_t cap_cs = nullptr, cap_cp = nullptr;
+    cudaEvent_t fork_ev = nullptr, join_cp = nullptr, join_wb = nullptr;
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t graph_exec = nullptr;
     // activation tap (parity testing): device buffer the rounded activations are copied to, and what went where
     char *tap = nullptr; uint64_t tap_bytes = 0, tap_used = 0;
     std::vector<uint64_t> tap_index;                     // 5 words per record: op, tag, sub-index, offset, bytes
@@ -114,6 +120,9 @@ void tgp_engine_free(tgp_ctx *ctx) {
     if (e->wb_ev) cudaEventDestroy(e->wb_ev);
     if (e->t0) cudaEventDestroy(e->t0);
     if (e->t1) cudaEventDestroy(e->t1);
+    if (e->graph_exec) cudaGraphExecDestroy(e->graph_exec);
+    if (e->graph) cudaGraphDestroy(e->graph);
+    for (cudaEvent_t ev : {e->fork_ev, e->join_cp, e->join_wb}) if (ev) cudaEventDestroy(ev);
     if (e->wb_stream) cudaStreamDestroy(e->wb_stream);
     if (e->ecount_host) cudaFreeHost(e->ecount_host);
     delete e;
@@ -212,6 +221,7 @@ int tgp_run_reset(tgp_ctx *ctx) {
     TgpEngine *e = ctx->eng;
     e->next_cmd = 0; e->next_step = 0; e->pos = 0; e->wb_pending = false; e->copy_waited_op = -1; e->tok_src = nullptr;
     e->evict_at.clear();
+    e->advised = false;                                  // the plan may have changed since the last run
     ctx->run_counts.clear();
     return TGP_OK;
 }
@@ -286,6 +296,8 @@ static int advise_once(tgp_ctx *ctx) {
         if (pl.zc[t]) {
             CU(ctx, cudaMemAdvise(p, tt.size, cudaMemAdviseSetPreferredLocation, cudaCpuDeviceId));
             CU(ctx, cudaMemAdvise(p, tt.size, cudaMemAdviseSetAccessedBy, e->device));
+        } else {
+            CU(ctx, cudaMemAdvise(p, tt.size, cudaMemAdviseUnsetPreferredLocation, e->device));   // advice of an earlier plan
         }
     }
     for (auto &pin : pl.pins) {
@@ -422,6 +434,8 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
     if (st.kind != step_kind || B != c.B || !q_len || (step_kind == TGP_DECODE && q_len != 1)) return tgp_fail(ctx, TGP_E_INVAL, "step kind, batch or q_len differ from the plan");
     if ((uint64_t)B * q_len > e->max_tokens || e->pos + q_len > c.max_len) return tgp_fail(ctx, TGP_E_INVAL, "more tokens than the workspace or max_len allow");
     if (!tokens_host && (step_kind != TGP_DECODE || e->next_step == 0)) return tgp_fail(ctx, TGP_E_INVAL, "tokens are required for this step");
+    if (e->capturing && (stats || e->op_timing || e->tap || compute_stream != (void *)e->cap_cs || copy_stream != (void *)e->cap_cp))
+        return tgp_fail(ctx, TGP_E_STATE, "while a run is being captured: no statistics, timing or tap, and the streams given to tgp_run_capture_begin()");
     cudaStream_t cs = (cudaStream_t)compute_stream, cp = (cudaStream_t)copy_stream;
     const uint32_t M = B * q_len, pos0 = e->pos;
     const uint64_t launches0 = tgpk_launches;
@@ -658,5 +672,72 @@ extern "C" int tgp_tap_index(tgp_ctx *ctx, uint64_t *out, uint64_t *n_words) {
     const std::vector<uint64_t> &v = ctx->eng->tap_index;
     if (out) { if (*n_words < v.size()) return TGP_E_INVAL; memcpy(out, v.data(), v.size() * 8); }
     *n_words = v.size();
+    return TGP_OK;
+}
+
+// ---- whole-run CUDA graph ----------------------------------------------------------------------------------------
+// A planned run of a dense model is a fixed DAG of copies and kernels over three streams (tokens come from the prompt
+// and then from the device-side argmax), so it can be captured once and replayed: the host then issues one graph
+// launch per pass instead of a few hundred API calls per step, which is what bounds steps of ~0.1 ms.
+extern "C" int tgp_run_capture_begin(tgp_ctx *ctx, void *compute_stream, void *copy_stream) {
+    if (!ctx || !ctx->eng) return TGP_E_STATE;
+    TgpEngine *e = ctx->eng;
+    if (!ctx->plan.valid) return TGP_E_NO_PLAN;
+    if (ctx->variant != TGP_VAR_EXPLICIT_RING) return tgp_fail(ctx, TGP_E_STATE, "only the explicit engine can be captured");
+    if (ctx->cfg.E) return tgp_fail(ctx, TGP_E_STATE, "an MoE step reads routing counts on the host and cannot be captured");
+    if (e->capturing || e->next_step != 0 || e->next_cmd != 0) return tgp_fail(ctx, TGP_E_STATE, "call tgp_run_reset() first");
+    if (e->op_timing || e->tap) return tgp_fail(ctx, TGP_E_STATE, "switch timing and tap off before capturing");
+    if (!compute_stream || !copy_stream || compute_stream == copy_stream) return tgp_fail(ctx, TGP_E_INVAL, "two distinct non-default streams are required");
+    if (e->graph_exec) { cudaGraphExecDestroy(e->graph_exec); e->graph_exec = nullptr; }
+    if (e->graph) { cudaGraphDestroy(e->graph); e->graph = nullptr; }
+    for (cudaEvent_t *ev : {&e->fork_ev, &e->join_cp, &e->join_wb})
+        if (!*ev) CU(ctx, cudaEventCreateWithFlags(ev, cudaEventDisableTiming));
+    // every event the run will use exists before capture starts (creation is not a stream operation)
+    for (size_t i = 0; i < ctx->ops.size(); ++i) {
+        cudaEvent_t ev;
+        int rc;
+        if (ctx->plan.op_is_wait_target[i] && (rc = get_event(ctx, e->done_ev, i, &ev))) return rc;
+        if (ctx->plan.op_last_place[i] >= 0 && (rc = get_event(ctx, e->copied_ev, i, &ev))) return rc;
+    }
+    e->cap_cs = (cudaStream_t)compute_stream; e->cap_cp = (cudaStream_t)copy_stream;
+    CU(ctx, cudaStreamBeginCapture(e->cap_cs, cudaStreamCaptureModeRelaxed));
+    // fork: the copy and write-back streams join the capture
+    cudaError_t er = cudaEventRecord(e->fork_ev, e->cap_cs);
+    if (er == cudaSuccess) er = cudaStreamWaitEvent(e->cap_cp, e->fork_ev, 0);
+    if (er == cudaSuccess) er = cudaStreamWaitEvent(e->wb_stream, e->fork_ev, 0);
+    if (er != cudaSuccess) {
+        cudaGraph_t g = nullptr;
+        cudaStreamEndCapture(e->cap_cs, &g);
+        if (g) cudaGraphDestroy(g);
+        return tgp_fail(ctx, TGP_E_CUDA, std::string("capture fork: ") + cudaGetErrorString(er));
+    }
+    e->capturing = true;
+    return TGP_OK;
+}
+
+extern "C" int tgp_run_capture_end(tgp_ctx *ctx) {
+    if (!ctx || !ctx->eng || !ctx->eng->capturing) return TGP_E_STATE;
+    TgpEngine *e = ctx->eng;
+    e->capturing = false;
+    // join: the capturing stream waits for everything the other two streams were given
+    cudaError_t er = cudaEventRecord(e->join_cp, e->cap_cp);
+    if (er == cudaSuccess) er = cudaEventRecord(e->join_wb, e->wb_stream);
+    if (er == cudaSuccess) er = cudaStreamWaitEvent(e->cap_cs, e->join_cp, 0);
+    if (er == cudaSuccess) er = cudaStreamWaitEvent(e->cap_cs, e->join_wb, 0);
+    cudaGraph_t g = nullptr;
+    cudaError_t ee = cudaStreamEndCapture(e->cap_cs, &g);
+    if (er != cudaSuccess || ee != cudaSuccess || !g) {
+        if (g) cudaGraphDestroy(g);
+        cudaGetLastError();
+        return tgp_fail(ctx, TGP_E_CUDA, std::string("capture end: ") + cudaGetErrorString(er != cudaSuccess ? er : ee));
+    }
+    e->graph = g;
+    CU(ctx, cudaGraphInstantiate(&e->graph_exec, e->graph, 0));
+    return TGP_OK;
+}
+
+extern "C" int tgp_run_graph_launch(tgp_ctx *ctx, void *stream) {
+    if (!ctx || !ctx->eng || !ctx->eng->graph_exec) return TGP_E_STATE;
+    CU(ctx, cudaGraphLaunch(ctx->eng->graph_exec, (cudaStream_t)stream));
     return TGP_OK;
 }

@@ -74,3 +74,20 @@ class Runner:
                 self.step(tb.DECODE, None, 1)
         self.sync()
         return out, (np.stack(toks, axis=1) if toks else np.zeros((self.cfg.B, 0), np.int32))
+
+    def capture_run(self, prompt_pinned, n_decode: int):
+        """Captures prefill + n_decode free-running decode steps into one CUDA graph (dense models).  prompt_pinned:
+        int32 host tensor/array [B, S] that stays alive and unchanged while the graph is replayed."""
+        self._prompt_keep = prompt_pinned
+        arr = prompt_pinned.numpy() if hasattr(prompt_pinned, "numpy") else prompt_pinned
+        self.reset()
+        self.s.ctx.run_capture_begin(self.compute, self.copy)
+        try:
+            self.step(tb.PREFILL, arr, arr.shape[1])
+            for _ in range(n_decode):
+                self.step(tb.DECODE, None, 1)
+        finally:
+            self.s.ctx.run_capture_end()
+
+    def replay(self):
+        self.s.ctx.run_graph_launch(self.compute)

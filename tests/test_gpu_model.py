@@ -453,3 +453,30 @@ def test_runtime_monitor_replan_from_measured_kernel_times():
     for a, b in zip(before, after):
         assert np.array_equal(a, b)
     s.close()
+
+
+def test_whole_run_cuda_graph_replays_bit_identically():
+    """The planned run (copies, kernels, cross-stream ordering, device-side argmax feedback) captured as one CUDA graph:
+    two replays give exactly the logits and tokens of the plain stepped run, and call-order mistakes are state errors."""
+    cfg = replace(si.CONFIGS[1], B=2, S=21, T=9, TK=8)
+    lay, pool, s, blobs, T = setup(cfg, cap=128 << 10)
+    r = Runner(s, cfg.B * cfg.S)
+    prompt = torch.from_numpy(si.prompt_tokens(cfg)).pin_memory()
+    plain, toks = r.generate(prompt.numpy(), T)                      # free-running greedy decode, stepped
+    with pytest.raises(tb.TgpError) as ei:
+        s.ctx.run_graph_launch(r.compute)                            # nothing captured yet
+    assert ei.value.code == tb.E_STATE
+    r.capture_run(prompt, T)
+    with pytest.raises(tb.TgpError):
+        s.ctx.run_capture_end()                                      # not capturing any more
+    for _ in range(2):
+        r.logits.zero_()
+        r.argmax.zero_()
+        r.replay()
+        r.sync()
+        assert np.array_equal(r.logits.cpu().numpy(), plain[-1])
+        assert np.array_equal(r.argmax.cpu().numpy(), np.argmax(plain[-1], axis=-1).astype(np.int32))
+    # back to plain stepping after a reset
+    again, toks2 = r.generate(prompt.numpy(), T)
+    assert np.array_equal(again[-1], plain[-1]) and np.array_equal(toks, toks2)
+    s.close()
