@@ -480,3 +480,41 @@ def test_whole_run_cuda_graph_replays_bit_identically():
     again, toks2 = r.generate(prompt.numpy(), T)
     assert np.array_equal(again[-1], plain[-1]) and np.array_equal(toks, toks2)
     s.close()
+
+
+def test_edge_shapes_single_token_prompt_no_decode_and_maximum_tile_count():
+    """Degenerate sizes: a prompt of one token with no decode step, and a context that needs all 64 KV tiles a kernel
+    can address (TK = 1), both against the oracle; requests beyond the workspace or max_len are refused."""
+    one = si.ModelConfig("one", L=2, d=128, Hq=2, Hkv=2, Dh=64, F=256, V=300, B=1, S=1, T=0, TK=4, seed=9, budget_rule="half_w_kv")
+    lay = si.build_layout(one, cap=16 << 10)
+    pool = pinned_pool(lay.pool_bytes)
+    si.fill_pool(lay, pool.numpy())
+    s = Session(lay, MACHINE, pool_base=pool.data_ptr(), pool_flags=tb.POOL_PINNED)
+    s.plan()
+    ref, _ = forward.OracleModel(one, si.weights_as_bits(lay)).generate(si.prompt_tokens(one), 0)
+    r = Runner(s, 1)
+    got, toks = r.generate(si.prompt_tokens(one), 0)
+    assert len(got) == 1 and toks.shape == (1, 0)
+    check_logits(got, ref)
+    with pytest.raises(tb.TgpError) as ei:
+        r.step(tb.DECODE, None, 1)                                   # the plan has no decode step
+    assert ei.value.code == tb.E_STATE
+    s.close()
+    many = si.ModelConfig("tiles", L=1, d=128, Hq=4, Hkv=2, Dh=64, F=256, V=300, B=2, S=40, T=24, TK=1, seed=10, budget_rule="half_w_kv")
+    assert many.n_tiles == 64
+    lay = si.build_layout(many, cap=16 << 10)
+    pool = pinned_pool(lay.pool_bytes)
+    si.fill_pool(lay, pool.numpy())
+    s = Session(lay, MACHINE, pool_base=pool.data_ptr(), pool_flags=tb.POOL_PINNED)
+    s.plan()
+    om = forward.OracleModel(many, si.weights_as_bits(lay))
+    prompt = si.prompt_tokens(many)
+    ref, toks = om.generate(prompt, many.T)
+    r = Runner(s, many.B * many.S)
+    got, _ = r.generate(prompt, many.T, forced=toks)
+    check_logits(got, ref)
+    r.reset()
+    with pytest.raises(tb.TgpError) as ei:
+        r.step(tb.PREFILL, np.zeros((many.B, many.S + 1), np.int32), many.S + 1)      # more tokens than the workspace holds
+    assert ei.value.code == tb.E_INVAL
+    s.close()
