@@ -277,6 +277,7 @@ def main():
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--graph", action="store_true", help="replay the whole planned run as one CUDA graph (dense models; for host-bound tiny steps)")
     ap.add_argument("--layers", type=int, default=None, help="run the shape at reduced depth; a byte budget is scaled in proportion")
+    ap.add_argument("--cap-mib", type=float, default=None, help="sub-range cap in MiB (default: the input recipe's rule)")
     ap.add_argument("--bits", type=int, default=7, help="policy bits: 1 affinity/pins, 2 roofline selectivity, 4 zero-copy")
     ap.add_argument("--budget-frac", type=float, default=None, help="device budget as a fraction of the pool (oversubscription sweep)")
     args = ap.parse_args()
@@ -291,9 +292,10 @@ def main():
         cfg2 = replace(cfg, L=args.layers, name=f"{cfg.name}_L{args.layers}")
         budget = int(full.budget * si.build_layout(cfg2, budget=1 << 40).pool_bytes / full.pool_bytes) // 512 * 512
         cfg = cfg2
-    lay = si.build_layout(cfg, budget=budget)
+    cap = int(args.cap_mib * (1 << 20)) if args.cap_mib else None
+    lay = si.build_layout(cfg, budget=budget, cap=cap)
     if args.budget_frac is not None:
-        lay = si.build_layout(cfg, budget=int(lay.pool_bytes * args.budget_frac) // 512 * 512)
+        lay = si.build_layout(cfg, budget=int(lay.pool_bytes * args.budget_frac) // 512 * 512, cap=cap)
     if args.impl == "reference":
         return run_reference(args, cfg, lay)
 

@@ -22,6 +22,8 @@ PREFILL, DECODE = 0, 1
 VAR_EXPLICIT_RING, VAR_MANAGED_HINTS, VAR_MANAGED_DEMAND = 0, 1, 2
 BIT_A, BIT_P, BIT_ZC = 1, 2, 4
 X_CLASSES, X_TENSORS, X_PINS, X_COMMANDS, X_TOTALS = range(5)
+# tensor kinds (TGP_K_*)
+(K_EMBED, K_G1, K_WQ, K_WK, K_WV, K_WO, K_G2, K_WG, K_WU, K_WD, K_GF, K_LM, K_ROUTER, K_KTILE, K_VTILE) = range(15)
 TAP_H, TAP_HF, TAP_Q, TAP_KTILE, TAP_VTILE, TAP_O, TAP_A = range(7)
 
 

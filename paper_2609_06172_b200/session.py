@@ -29,7 +29,8 @@ class Session:
         for t in layout.tensors:
             tid = self.ctx.tensor_register(self.pool, t.pool_off, t.size, t.site_hash, t.layer, t.kind, t.flags)
             assert tid == t.tid
-            rows = t.rows if t.kind < 13 else layout.cfg.B * layout.cfg.Hkv * layout.cfg.TK
+            is_tile = t.kind in (tb.K_KTILE, tb.K_VTILE)                 # a KV tile is [B * Hkv * TK rows, Dh]
+            rows = layout.cfg.B * layout.cfg.Hkv * layout.cfg.TK if is_tile else t.rows
             self.roles.append((t.kind, t.layer, t.expert, t.block, t.row0, rows, tid))
         self.cfg = model_cfg(layout.cfg)
         self.router_bias = router_bias

@@ -199,9 +199,10 @@ def _align(x: int, a: int = POOL_ALIGN) -> int:
 
 
 def sub_range_cap(budget: int) -> int:
-    """Largest power of two <= budget/32, clamped to [128 KiB, 256 MiB]."""
+    """Largest power of two <= budget/32, clamped to [128 KiB, 32 MiB].  (32 MiB copies already run at the link's
+    full rate; larger blocks only enlarge the staging ring, which is sized as two of them, at the expense of pins.)"""
     c = 1 << max(0, (budget // 32).bit_length() - 1)
-    return max(128 << 10, min(256 << 20, c))
+    return max(128 << 10, min(32 << 20, c))
 
 
 def block_rows(rows: int, cols: int, cap: int) -> int:

@@ -31,7 +31,7 @@ def test_layout_sizes(c):
 def test_sub_range_cap_rule():
     assert si.sub_range_cap(6_392_064) == 128 << 10
     assert si.sub_range_cap(1_104_218_112) == 32 << 20
-    assert si.sub_range_cap(64 << 30) == 256 << 20
+    assert si.sub_range_cap(64 << 30) == 32 << 20
 
 
 def test_generator_statistics_and_determinism():
