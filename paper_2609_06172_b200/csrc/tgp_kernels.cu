@@ -628,13 +628,13 @@ static void launch_gemv(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, 
     cudaLaunchKernelEx(&cfg, gemv_kernel<MT, R, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
 }
 
-// Same product for blocks with few rows: one CTA owns 16 rows of W and its 8 warps split K (interleaved chunks of
-// 32*U), so n/16 CTAs of 8 warps fill the machine where n/16 warps would not.  The eight partial tiles meet in shared
-// memory and are summed in warp order: deterministic.
-template <int NB, int U>
-__global__ void __launch_bounds__(256) gemv_mma_splitk_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+// Same product for blocks with few rows: one CTA owns 16 rows of W and its NW (8 or 16) warps split K (interleaved
+// chunks of 32*U), so n/16 CTAs of NW warps fill the machine where n/16 warps would not.  The partial tiles meet in
+// shared memory and are summed in warp order: deterministic.
+template <int NB, int U, int NW>
+__global__ void __launch_bounds__(NW * 32) gemv_mma_splitk_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                               uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
-    __shared__ float part[8][NB * 4][32];
+    __shared__ float part[NW][NB * 4][32];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, c = lane & 3;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     bool synced = false;
@@ -644,7 +644,7 @@ __global__ void __launch_bounds__(256) gemv_mma_splitk_kernel(const bf16 *__rest
         float acc[NB][4];
 #pragma unroll
         for (int b = 0; b < NB; ++b) { acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f; }
-        for (uint32_t k0 = warp * 32 * U; k0 < K; k0 += 8 * 32 * U) {
+        for (uint32_t k0 = warp * 32 * U; k0 < K; k0 += NW * 32 * U) {
             uint4 lo[U], hi[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
@@ -671,11 +671,11 @@ __global__ void __launch_bounds__(256) gemv_mma_splitk_kernel(const bf16 *__rest
 #pragma unroll
             for (int i = 0; i < 4; ++i) part[warp][b * 4 + i][lane] = acc[b][i];
         __syncthreads();
-        for (uint32_t v = threadIdx.x; v < NB * 4 * 32; v += 256) {
+        for (uint32_t v = threadIdx.x; v < NB * 4 * 32; v += NW * 32) {
             const uint32_t slot = v >> 5, ln = v & 31, b = slot >> 2, i = slot & 3;
             float sum = 0.f;
 #pragma unroll
-            for (int w = 0; w < 8; ++w) sum += part[w][slot][ln];
+            for (int w = 0; w < NW; ++w) sum += part[w][slot][ln];
             const uint32_t m = b * 8 + 2 * (ln & 3) + (i & 1), row = row0 + (ln >> 2) + 8 * (i >> 1);
             if (m < Mrows && row < n) {
                 float *p = C + (size_t)m * ldc + col0 + row;
@@ -697,21 +697,23 @@ static void launch_gemv_mma(const bf16 *A, const bf16 *W, float *C, uint32_t Mro
         if (sms < 1) sms = 148;
     }
     static int blocks_per_sm_split = 0;
-    if (!blocks_per_sm_split && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm_split, gemv_mma_splitk_kernel<NB, U>, 256, 0) != cudaSuccess || blocks_per_sm_split < 1))
+    if (!blocks_per_sm_split && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm_split, gemv_mma_splitk_kernel<NB, U, 8>, 256, 0) != cudaSuccess || blocks_per_sm_split < 1))
         blocks_per_sm_split = 1;
     const bool split = n < 16u * 8u * (uint32_t)sms;                 // too few 16-row groups to give every SM eight warps
+    const bool wide = split && (n + 15) / 16 < (uint32_t)sms;        // fewer 16-row groups than SMs: 16 warps per CTA
     uint32_t need = split ? (n + 15) / 16 : (n + 16 * 8 - 1) / (16 * 8);
     uint32_t full = (uint32_t)(sms * (split ? blocks_per_sm_split : blocks_per_sm));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(need < full ? need : full);
-    cfg.blockDim = dim3(256);
+    cfg.blockDim = dim3(wide ? 512 : 256);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = g_gemv_pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (split) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
+    if (wide) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16>, A, W, C, Mrows, n, K, ldc, col0, acc);
+    else if (split) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 8>, A, W, C, Mrows, n, K, ldc, col0, acc);
     else cudaLaunchKernelEx(&cfg, gemv_mma_kernel<NB, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
 }
 
