@@ -262,9 +262,12 @@ int  tgp_k_gemv_overlap(int enable);
 /* Tensor-core GEMM variant: 0 (default) picks by problem size, 1 forces the 128x128 one-tile-per-CTA kernel,
  * 2 forces the persistent 128x256 kernel with double-buffered accumulators.  Process-wide; for tests and timing. */
 int  tgp_k_gemm_tc_variant(int variant);
-/* Which kernel serves attention with q_len >= 16: 0 (default) the tensor-core flash-style kernel, 1 the
- * warp-per-query-row CUDA-core kernel (an on-device cross-check).  Process-wide. */
+/* Which kernel serves attention with q_len >= 16: 0 (default) the tcgen05 kernel (S and O_j in TMEM), 2 the
+ * mma.sync flash-style kernel, 1 the warp-per-query-row CUDA-core kernel (on-device cross-checks).  Process-wide. */
 int  tgp_k_attn_select(int impl);
+/* Error word of the tcgen05 attention kernel: 0, or the phase (1 waiting for S, 2 waiting for O_j) of the first
+ * bounded wait that ran out.  Synchronous. */
+int  tgp_k_attn_status(int *error_code);
 /* Error word of the tensor-core GEMM: 0, or (role << 8 | stage) of the first bounded wait that ran out
  * (role 1 TMA producer, 2 MMA issuer, 3 epilogue).  Synchronous. */
 int  tgp_k_gemm_status(int *error_code);

@@ -101,6 +101,7 @@ _SIGS = {
     "tgp_k_skinny_select": [C.c_int],
     "tgp_k_gemm_tc_variant": [C.c_int],
     "tgp_k_gemm_status": [C.POINTER(C.c_int)],
+    "tgp_k_attn_status": [C.POINTER(C.c_int)],
     "tgp_k_rope_tables": [_U32, _U32, C.c_float, _P, _P],
     "tgp_k_rope_kv": [_P, _P, _P, _P, C.POINTER(_P), C.POINTER(_P), _U32, _P, _P, C.POINTER(ModelCfg), _U32, _U32, _U32, _P],
     "tgp_k_attn": [_P, C.POINTER(_P), C.POINTER(_P), _U32, _P, C.POINTER(ModelCfg), _U32, _U32, _U32, _P, _P],
@@ -374,6 +375,12 @@ def k_attn_select(impl):
 
 def k_gemm_tc_variant(v):
     _k(lib().tgp_k_gemm_tc_variant(v), "tgp_k_gemm_tc_variant")
+
+
+def k_attn_status():
+    e = C.c_int()
+    _k(lib().tgp_k_attn_status(C.byref(e)), "tgp_k_attn_status")
+    return e.value
 
 
 def k_gemm_status():

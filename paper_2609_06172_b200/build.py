@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libtgp.so")
-SOURCES = ["tgp_host.cpp", "tgp_model.cpp", "tgp_kernels.cu", "tgp_gemm_sm100.cu", "tgp_attn_prefill.cu", "tgp_engine.cu"]
+SOURCES = ["tgp_host.cpp", "tgp_model.cpp", "tgp_kernels.cu", "tgp_gemm_sm100.cu", "tgp_attn_prefill.cu", "tgp_attn_sm100.cu", "tgp_engine.cu"]
 
 
 def sources():

@@ -770,7 +770,7 @@ int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb,
     return TGP_OK;
 }
 
-static int g_attn_impl = 0;      // 0: tensor cores for q_len >= 16; 1: warp-per-row CUDA-core kernel (an on-device cross-check)
+static int g_attn_impl = 0;      // q_len >= 16: 0 tcgen05 kernel, 2 mma.sync flash kernel, 1 warp-per-row CUDA-core kernel (cross-checks)
 
 int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *ob, const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0,
               float *scratch, cudaStream_t st) {
@@ -794,6 +794,8 @@ int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *
         }
         tgpk_launches += 1;
     } else if (q_len >= 16 && g_attn_impl == 0) {
+        return tgpk_attn_prefill_tc5(qb, tiles, ob, c, B, q_len, pos0, st);
+    } else if (q_len >= 16 && g_attn_impl == 2) {
         return tgpk_attn_prefill_tc(qb, tiles, ob, c, B, q_len, pos0, st);
     } else {
         dim3 grid((q_len + 3) / 4, c->Hq, B);
@@ -853,7 +855,7 @@ int tgp_k_gemv_overlap(int enable) {
 }
 
 int tgp_k_attn_select(int impl) {
-    if (impl != 0 && impl != 1) return TGP_E_INVAL;
+    if (impl < 0 || impl > 2) return TGP_E_INVAL;
     g_attn_impl = impl;
     return TGP_OK;
 }

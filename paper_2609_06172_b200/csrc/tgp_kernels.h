@@ -17,7 +17,9 @@ int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb,
                  const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0, cudaStream_t st);
 int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *ob, const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0,
               float *scratch, cudaStream_t st);
-// tensor-core causal attention for q_len > 1 (tgp_attn_prefill.cu); Dh 64 or 128
+// tcgen05 causal attention for q_len > 1 (tgp_attn_sm100.cu); Dh 64 or 128
+int tgpk_attn_prefill_tc5(const void *qb, const TgpTilePtrs &tiles, void *ob, const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0, cudaStream_t st);
+// mma.sync flash-style causal attention for q_len > 1 (tgp_attn_prefill.cu); Dh 64 or 128
 int tgpk_attn_prefill_tc(const void *qb, const TgpTilePtrs &tiles, void *ob, const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0, cudaStream_t st);
 int tgpk_swiglu(const float *g, const float *u, void *ab, uint64_t n, cudaStream_t st);
 // MoE: router logits + top-k (1 or 2) + gates, then per-expert token lists rows[e*stride + i], gates[e*stride + i], counts[e]
