@@ -2,8 +2,10 @@
 //
 // One CTA of 128 threads owns 128 consecutive queries of one (sequence, query head); thread t is query row t and
 // TMEM lane t.  For every block of 64 keys:
-//   1. all threads stage K (cp.async, 16-byte chunks) and V transposed (so that keys are the contiguous dimension)
-//      into shared memory, both in the K-major 128-byte-swizzle layout tcgen05 descriptors address;
+//   1. all threads stage K and V (cp.async, 16-byte chunks) into shared memory as 64-wide head-dimension blocks of
+//      [64 keys x 128 B] with the 128-byte swizzle; K is then a K-major operand (head dimension contiguous) and V,
+//      in the very same layout, an MN-major operand (its contiguous dimension is the output dimension of P V);
+//      the next block's K is requested as soon as S has been computed, the next V as soon as O_j has;
 //   2. one thread issues S = Q K^T (M=128, N=64) into TMEM and commits to an mbarrier;
 //   3. every thread reads its row of S from TMEM, applies scale and causal mask, updates its running max / sum and
 //      writes P = exp2(S - max) as bf16 into a K-major shared tile;
@@ -40,6 +42,12 @@ __device__ __forceinline__ void cp_async16z(uint32_t dst, const void *src, bool 
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
 }
 
+// MN-major operand in the same swizzled storage: 64 contiguous elements (128 B) of the MN dimension per row, rows are
+// K; the next 64 MN elements start `lbo` bytes further (leading byte offset), the next 8 K rows 1024 bytes further.
+__device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr, uint32_t lbo) {
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+
 // byte offset of 16-byte chunk c (0..7) of row r inside a [rows x 128 B] K-major tile with 128-byte swizzle
 __device__ __forceinline__ uint32_t sw128(uint32_t r, uint32_t c) { return r * 128u + ((c ^ (r & 7u)) << 4); }
 
@@ -47,9 +55,9 @@ template <int DH>
 __global__ void __launch_bounds__(128, 2) attn_prefill_tc_kernel(TArgs a) {
     extern __shared__ uint8_t smem_raw[];
     constexpr int KB = DH / 64;                          // 64-wide blocks of the head dimension
-    constexpr int Q_BYTES = KB * BQ * 128, K_BYTES = KB * BKV * 128, V_BYTES = DH * 128, P_BYTES = BQ * 128;
+    constexpr int Q_BYTES = KB * BQ * 128, K_BYTES = KB * BKV * 128, V_BYTES = KB * BKV * 128, P_BYTES = BQ * 128;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *Qs = smem, *Ks = Qs + Q_BYTES, *Vt = Ks + K_BYTES, *Ps = Vt + V_BYTES;
+    uint8_t *Qs = smem, *Ks = Qs + Q_BYTES, *Vs = Ks + K_BYTES, *Ps = Vs + V_BYTES;
     uint64_t *bar_s = reinterpret_cast<uint64_t *>(Ps + P_BYTES);
     uint64_t *bar_o = bar_s + 1;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bar_o + 1);
@@ -91,29 +99,22 @@ __global__ void __launch_bounds__(128, 2) attn_prefill_tc_kernel(TArgs a) {
 #pragma unroll
     for (int i = 0; i < DH; ++i) o[i] = 0.f;
     float mrow = -INFINITY, lrow = 0.f;
-    constexpr uint32_t idesc_s = umma_idesc(BKV), idesc_o = umma_idesc(DH);
+    constexpr uint32_t idesc_s = umma_idesc(BKV), idesc_o = umma_idesc(DH) | (1u << 16);     // bit 16: B operand is MN-major
 
-    for (uint32_t jb = 0; jb < nblk; ++jb) {
-        // ---- 1. stage K block and transposed V block ----
+    auto stage = [&](uint8_t *dst, void *const *tiles, uint32_t jb) {      // one [64 keys x DH] block, 64-wide dh blocks
         for (uint32_t i = tid; i < BKV * (DH / 8); i += 128) {
             const uint32_t r = i / (DH / 8), c = i % (DH / 8), j = jb * BKV + r;
             const bool ok = j < kvlen;
             const uint32_t jj = ok ? j : 0;
-            const bf16 *src = reinterpret_cast<const bf16 *>(a.tiles.k[jj / a.TK]) + ((size_t)(b * a.Hkv + hk) * a.TK + jj % a.TK) * DH + c * 8;
-            cp_async16z(smem_u32(Ks + (c / 8) * (BKV * 128) + sw128(r, c % 8)), src, ok);
+            const bf16 *src = reinterpret_cast<const bf16 *>(tiles[jj / a.TK]) + ((size_t)(b * a.Hkv + hk) * a.TK + jj % a.TK) * DH + c * 8;
+            cp_async16z(smem_u32(dst + (c / 8) * (BKV * 128) + sw128(r, c % 8)), src, ok);
         }
-        for (uint32_t i = tid; i < BKV * (DH / 8); i += 128) {
-            const uint32_t key = i % BKV, c = i / BKV, j = jb * BKV + key;      // lanes walk keys: conflict-free transposed stores
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (j < kvlen)
-                v = *reinterpret_cast<const uint4 *>(reinterpret_cast<const bf16 *>(a.tiles.v[j / a.TK]) + ((size_t)(b * a.Hkv + hk) * a.TK + j % a.TK) * DH + c * 8);
-            const uint16_t *e = reinterpret_cast<const uint16_t *>(&v);
-#pragma unroll
-            for (uint32_t t = 0; t < 8; ++t) {
-                const uint32_t d = c * 8 + t;
-                *reinterpret_cast<uint16_t *>(Vt + sw128(d, key >> 3) + (key & 7u) * 2) = e[t];
-            }
-        }
+    };
+    stage(Ks, a.tiles.k, 0);
+    stage(Vs, a.tiles.v, 0);
+
+    for (uint32_t jb = 0; jb < nblk; ++jb) {
+        // ---- 1. this block's K and V (requested one phase ahead) have landed ----
         asm volatile("cp.async.wait_all;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");        // generic-proxy writes -> visible to the tensor core
         __syncthreads();
@@ -132,6 +133,7 @@ __global__ void __launch_bounds__(128, 2) attn_prefill_tc_kernel(TArgs a) {
         bool ok = mbar_wait(bar_s, jb & 1, failed);
         if (!ok && !*failed) { *failed = 1; atomicCAS(&g_attn_tc_error, 0, 1); }
         ok = __all_sync(0xffffffffu, ok);
+        if (ok && jb + 1 < nblk) stage(Ks, a.tiles.k, jb + 1);            // the tensor core is done with K_j
         float alpha = 1.f;
         if (ok) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -176,15 +178,16 @@ __global__ void __launch_bounds__(128, 2) attn_prefill_tc_kernel(TArgs a) {
         // ---- 4. O_j = P V_j ----
         if (tid == 0) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint64_t dp = umma_desc(smem_u32(Ps)), dv = umma_desc(smem_u32(Vt));
+            const uint64_t dp = umma_desc(smem_u32(Ps)), dv = umma_desc_mn(smem_u32(Vs), BKV * 128);
 #pragma unroll
-            for (uint32_t k = 0; k < 4; ++k) umma(tmem_O, dp + 2 * k, dv + 2 * k, idesc_o, k != 0);
+            for (uint32_t k = 0; k < 4; ++k) umma(tmem_O, dp + 2 * k, dv + 128 * k, idesc_o, k != 0);   // 16 keys = 2048 B of V rows per step
             umma_commit(bar_o);
         }
         // ---- 5. fold O_j into the register accumulator ----
         ok = mbar_wait(bar_o, jb & 1, failed);
         if (!ok && !*failed) { *failed = 1; atomicCAS(&g_attn_tc_error, 0, 2); }
         ok = __all_sync(0xffffffffu, ok);
+        if (ok && jb + 1 < nblk) stage(Vs, a.tiles.v, jb + 1);            // the tensor core is done with V_j
         if (ok) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
@@ -222,7 +225,7 @@ __global__ void __launch_bounds__(128, 2) attn_prefill_tc_kernel(TArgs a) {
     }
 }
 
-template <int DH> constexpr int smem_bytes() { return (DH / 64) * (BQ + BKV) * 128 + DH * 128 + BQ * 128 + 64 + 1024; }
+template <int DH> constexpr int smem_bytes() { return (DH / 64) * (BQ + 2 * BKV) * 128 + BQ * 128 + 64 + 1024; }
 
 }  // namespace
 
