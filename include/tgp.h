@@ -262,8 +262,9 @@ int  tgp_k_gemv_overlap(int enable);
 /* Tensor-core GEMM variant: 0 (default) picks by problem size, 1 forces the 128x128 one-tile-per-CTA kernel,
  * 2 forces the persistent 128x256 kernel with double-buffered accumulators.  Process-wide; for tests and timing. */
 int  tgp_k_gemm_tc_variant(int variant);
-/* Which kernel serves attention with q_len >= 16: 0 (default) the tcgen05 kernel (S and O_j in TMEM), 2 the
- * mma.sync flash-style kernel, 1 the warp-per-query-row CUDA-core kernel (on-device cross-checks).  Process-wide. */
+/* Which kernel serves attention with q_len >= 16: 0 (default) by problem size - the tcgen05 kernel (S and O_j in
+ * TMEM) when the grid has at least two CTAs of 128 queries per SM, else the mma.sync flash-style kernel; 3 / 2 force
+ * one or the other; 1 the warp-per-query-row CUDA-core kernel (an on-device cross-check).  Process-wide. */
 int  tgp_k_attn_select(int impl);
 /* Error word of the tcgen05 attention kernel: 0, or the phase (1 waiting for S, 2 waiting for O_j) of the first
  * bounded wait that ran out.  Synchronous. */

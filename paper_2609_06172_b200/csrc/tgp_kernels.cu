@@ -770,7 +770,7 @@ int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb,
     return TGP_OK;
 }
 
-static int g_attn_impl = 0;      // q_len >= 16: 0 tcgen05 kernel, 2 mma.sync flash kernel, 1 warp-per-row CUDA-core kernel (cross-checks)
+static int g_attn_impl = 0;      // q_len >= 16: 0 by problem size, 3 tcgen05 kernel, 2 mma.sync flash kernel, 1 warp-per-row CUDA-core kernel
 
 int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *ob, const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0,
               float *scratch, cudaStream_t st) {
@@ -793,9 +793,13 @@ int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *
             attn_decode_merge_kernel<128><<<dim3(c->Hq, B), 128, 0, st>>>(a);
         }
         tgpk_launches += 1;
-    } else if (q_len >= 16 && g_attn_impl == 0) {
-        return tgpk_attn_prefill_tc5(qb, tiles, ob, c, B, q_len, pos0, st);
-    } else if (q_len >= 16 && g_attn_impl == 2) {
+    } else if (q_len >= 16 && (g_attn_impl == 0 || g_attn_impl == 2 || g_attn_impl == 3)) {
+        // the tcgen05 kernel (128 queries per CTA, a serial chain per key block) needs at least two CTAs per SM of
+        // parallel work to beat the mma.sync kernel (64 queries per CTA)
+        static int sms = 0;
+        if (!sms) { int dev = 0; cudaGetDevice(&dev); if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148; }
+        const uint64_t ctas = (uint64_t)((q_len + 127) / 128) * c->Hq * B;
+        if (g_attn_impl == 3 || (g_attn_impl == 0 && ctas >= 2ull * sms)) return tgpk_attn_prefill_tc5(qb, tiles, ob, c, B, q_len, pos0, st);
         return tgpk_attn_prefill_tc(qb, tiles, ob, c, B, q_len, pos0, st);
     } else {
         dim3 grid((q_len + 3) / 4, c->Hq, B);
@@ -855,7 +859,7 @@ int tgp_k_gemv_overlap(int enable) {
 }
 
 int tgp_k_attn_select(int impl) {
-    if (impl < 0 || impl > 2) return TGP_E_INVAL;
+    if (impl < 0 || impl > 3) return TGP_E_INVAL;
     g_attn_impl = impl;
     return TGP_OK;
 }

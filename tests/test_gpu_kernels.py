@@ -146,9 +146,11 @@ def tiles_to_cache(tiles, cfg, B):
     return t.reshape(B, cfg.Hkv, -1, cfg.Dh).float().cpu().numpy()
 
 
+@pytest.mark.parametrize("attn_impl", [3, 2])
 @pytest.mark.parametrize("Dh,Hq,Hkv,TK,S,T", [(64, 4, 2, 4, 9, 7), (128, 8, 2, 16, 40, 5), (64, 4, 4, 8, 33, 3), (128, 8, 1, 64, 130, 2)])
-def test_rope_kv_and_attention_prefill_then_decode(Dh, Hq, Hkv, TK, S, T):
+def test_rope_kv_and_attention_prefill_then_decode(Dh, Hq, Hkv, TK, S, T, attn_impl):
     B = 2
+    tb.k_attn_select(attn_impl)
     cfg = replace(KCFG, Dh=Dh, Hq=Hq, Hkv=Hkv, TK=TK, S=S, T=T, B=B, d=Hq * Dh)
     lay_w = {(k, 0, -1): rnd_bits(k, 8).reshape(1, 8) for k in range(13)}
     o = OracleModel(cfg, lay_w)
@@ -188,6 +190,7 @@ def test_rope_kv_and_attention_prefill_then_decode(Dh, Hq, Hkv, TK, S, T):
         assert np.abs(got - att).max() < 2.0 ** -7 * np.abs(att).max() + 1e-6
         assert np.mean(np.abs(got - bf16_round(att))) < 3e-3 * np.abs(att).mean()     # incl. the kernel's bf16 rounding of softmax weights
         pos0 += q
+    tb.k_attn_select(0)
 
 
 @pytest.mark.parametrize("Dh,Hq,Hkv,TK,S,B", [(64, 32, 8, 128, 512, 1), (128, 8, 2, 256, 300, 2), (64, 4, 4, 16, 100, 3)])
@@ -203,7 +206,7 @@ def test_tensor_core_prefill_attention_agrees_with_cuda_core_kernel(Dh, Hq, Hkv,
         v.copy_(bf16_dev(rnd_bits(400 + j, v.numel())) * 30)
     qb = (bf16_dev(rnd_bits(9, B * S * Hq * Dh)) * 30).view(B * S, Hq * Dh)
     outs = []
-    for impl in (0, 2, 1):
+    for impl in (3, 2, 1):
         tb.k_attn_select(impl)
         ob = torch.zeros(B * S, Hq * Dh, dtype=torch.bfloat16, device=DEV)
         tb.k_attn(qb, kt, vt, ob, mc, B, S, 0, None)
