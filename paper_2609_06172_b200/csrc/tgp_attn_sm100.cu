@@ -6,7 +6,8 @@
 //      [64 keys x 128 B] with the 128-byte swizzle; K is then a K-major operand (head dimension contiguous) and V,
 //      in the very same layout, an MN-major operand (its contiguous dimension is the output dimension of P V);
 //      the next block's K is requested as soon as S has been computed, the next V as soon as O_j has;
-//   2. one thread issues S = Q K^T (M=128, N=64) into TMEM and commits to an mbarrier;
+//   2. one thread issues S = Q K^T (M=128, N=64) into TMEM and commits to an mbarrier (for block j+1 this happens
+//      right behind step 4 of block j, so that its latency hides behind step 5);
 //   3. every thread reads its row of S from TMEM, applies scale and causal mask, updates its running max / sum and
 //      writes P = exp2(S - max) as bf16 into a K-major shared tile;
 //   4. one thread issues O_j = P V_j (M=128, N=Dh) into a second TMEM accumulator;
@@ -113,22 +114,24 @@ __global__ void __launch_bounds__(128, 2) attn_prefill_tc_kernel(TArgs a) {
     stage(Ks, a.tiles.k, 0);
     stage(Vs, a.tiles.v, 0);
 
-    for (uint32_t jb = 0; jb < nblk; ++jb) {
-        // ---- 1. this block's K and V (requested one phase ahead) have landed ----
-        asm volatile("cp.async.wait_all;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");        // generic-proxy writes -> visible to the tensor core
-        __syncthreads();
-        // ---- 2. S = Q K^T ----
-        if (tid == 0) {
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    auto issue_s = [&]() {                                   // S = Q K^T for the K block now in shared memory
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-            for (uint32_t kb = 0; kb < KB; ++kb) {
-                const uint64_t dq = umma_desc(smem_u32(Qs + kb * (BQ * 128))), dk = umma_desc(smem_u32(Ks + kb * (BKV * 128)));
+        for (uint32_t kb = 0; kb < KB; ++kb) {
+            const uint64_t dq = umma_desc(smem_u32(Qs + kb * (BQ * 128))), dk = umma_desc(smem_u32(Ks + kb * (BKV * 128)));
 #pragma unroll
-                for (uint32_t k = 0; k < 4; ++k) umma(tmem_S, dq + 2 * k, dk + 2 * k, idesc_s, (kb | k) != 0);
-            }
-            umma_commit(bar_s);
+            for (uint32_t k = 0; k < 4; ++k) umma(tmem_S, dq + 2 * k, dk + 2 * k, idesc_s, (kb | k) != 0);
         }
+        umma_commit(bar_s);
+    };
+    // ---- prologue: Q, K_0, V_0 have landed; S_0 is issued ----
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");            // generic-proxy writes -> visible to the tensor core
+    __syncthreads();
+    if (tid == 0) issue_s();
+
+    for (uint32_t jb = 0; jb < nblk; ++jb) {
+        // (S_jb was issued one step ahead: behind P V of the previous block, or in the prologue)
         // ---- 3. softmax on this thread's row ----
         bool ok = mbar_wait(bar_s, jb & 1, failed);
         if (!ok && !*failed) { *failed = 1; atomicCAS(&g_attn_tc_error, 0, 1); }
@@ -171,17 +174,19 @@ __global__ void __launch_bounds__(128, 2) attn_prefill_tc_kernel(TArgs a) {
             }
             lrow = lrow * alpha + lsum;
         }
+        asm volatile("cp.async.wait_all;" ::: "memory");                     // V_jb and the prefetched K_jb+1 have landed
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncthreads();
+        __syncthreads();                                                     // every thread has read S_jb and written its row of P
         if (*failed) break;
-        // ---- 4. O_j = P V_j ----
+        // ---- 4. O_j = P V_j, and right behind it S of the next block (its accumulator is free again) ----
         if (tid == 0) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t dp = umma_desc(smem_u32(Ps)), dv = umma_desc_mn(smem_u32(Vs), BKV * 128);
 #pragma unroll
             for (uint32_t k = 0; k < 4; ++k) umma(tmem_O, dp + 2 * k, dv + 128 * k, idesc_o, k != 0);   // 16 keys = 2048 B of V rows per step
             umma_commit(bar_o);
+            if (jb + 1 < nblk) issue_s();
         }
         // ---- 5. fold O_j into the register accumulator ----
         ok = mbar_wait(bar_o, jb & 1, failed);
