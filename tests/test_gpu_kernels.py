@@ -222,6 +222,45 @@ def test_tensor_core_prefill_attention_agrees_with_cuda_core_kernel(Dh, Hq, Hkv,
         assert np.abs(a - ref).mean() < 4e-3 * np.abs(ref).mean()
 
 
+@pytest.mark.parametrize("Dh", [64, 128])
+def test_tensor_core_prefill_attention_with_growing_scores(Dh):
+    """Scores that grow along the sequence by far more than 2^8 per key block: the tcgen05 kernel has to move its
+    exponent reference and rescale its TMEM accumulator at almost every block.  Checked against the oracle."""
+    B, Hq, Hkv, TK, S = 2, 4, 2, 64, 400
+    cfg = replace(KCFG, Dh=Dh, Hq=Hq, Hkv=Hkv, TK=TK, S=S, T=0, B=B, d=Hq * Dh)
+    mc = model_cfg(cfg)
+    o = OracleModel(cfg, {(k, 0, -1): rnd_bits(k, 8).reshape(1, 8) for k in range(13)})
+    rng = np.random.default_rng(Dh)
+    u = rng.standard_normal(Dh).astype(np.float32)
+    u /= np.linalg.norm(u)
+    ramp = (np.arange(S, dtype=np.float32) / 4.0)[None, None, :, None]                  # + ~16 in log2 units per 64 keys
+    k32 = bf16_round(rng.standard_normal((B, Hkv, S, Dh)).astype(np.float32) + ramp * u)
+    v32 = bf16_round(rng.standard_normal((B, Hkv, S, Dh)).astype(np.float32))
+    q32 = bf16_round(rng.standard_normal((B, S, Hq, Dh)).astype(np.float32) + np.sqrt(Dh).astype(np.float32) * u)
+    sgn = np.where(np.arange(Hq) % 2 == 0, 1.0, -1.0).astype(np.float32)[None, None, :, None]
+    q32 = q32 * sgn                                                                     # odd heads: scores fall instead
+    kt, vt = make_tiles(cfg, B)
+    for t in range(cfg.n_tiles):
+        lo, hi = t * TK, min(S, (t + 1) * TK)
+        kt[t].view(B, Hkv, TK, Dh)[:, :, :hi - lo].copy_(torch.from_numpy(k32[:, :, lo:hi]).to(DEV))
+        vt[t].view(B, Hkv, TK, Dh)[:, :, :hi - lo].copy_(torch.from_numpy(v32[:, :, lo:hi]).to(DEV))
+    o.K[0, :, :, :S] = k32
+    o.V[0, :, :, :S] = v32
+    att = o.attention(0, q32, 0)
+    qb = torch.from_numpy(q32.reshape(B * S, Hq * Dh)).to(DEV).bfloat16()
+    for impl in (3, 2):
+        tb.k_attn_select(impl)
+        ob = torch.zeros(B * S, Hq * Dh, dtype=torch.bfloat16, device=DEV)
+        tb.k_attn(qb, kt, vt, ob, mc, B, S, 0, None)
+        torch.cuda.synchronize()
+        got = ob.float().cpu().numpy().reshape(B, S, Hq, Dh)
+        assert np.isfinite(got).all()
+        assert np.abs(got - att).max() < 2.0 ** -6 * np.abs(att).max() + 1e-6
+        assert np.mean(np.abs(got - bf16_round(att))) < 4e-3 * np.abs(att).mean()
+    tb.k_attn_select(0)
+    assert tb.k_attn_status() == 0
+
+
 def test_attention_single_key_returns_v():
     cfg = replace(KCFG, B=1, S=1, T=0)
     mc = model_cfg(cfg)
