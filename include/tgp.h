@@ -262,12 +262,15 @@ int  tgp_k_gemv_overlap(int enable);
 /* Tensor-core GEMM variant: 0 (default) picks by problem size, 1 forces the 128x128 one-tile-per-CTA kernel,
  * 2 forces the persistent 128x256 kernel with double-buffered accumulators.  Process-wide; for tests and timing. */
 int  tgp_k_gemm_tc_variant(int variant);
-/* Which kernel serves attention with q_len >= 16: 0 (default) by problem size - the tcgen05 kernel (S and O_j in
- * TMEM) when the grid has at least two CTAs of 128 queries per SM, else the mma.sync flash-style kernel; 3 / 2 force
- * one or the other; 1 the warp-per-query-row CUDA-core kernel (an on-device cross-check).  Process-wide. */
+/* Which kernel serves attention with q_len >= 16: 0 (default) by problem size - the tcgen05 kernel (S and O in TMEM,
+ * K/V fed by TMA) when the grid has at least two CTAs of 128 queries per SM, else the mma.sync flash-style kernel;
+ * 3 / 2 force one or the other; 1 the warp-per-query-row CUDA-core kernel (an on-device cross-check).  The tcgen05
+ * kernel needs KV tiles of a multiple of 64 keys whose base addresses differ by whole rows of Dh elements (and
+ * 16-byte aligned q); any other geometry is served by the mma.sync kernel even when 3 is forced.  Process-wide. */
 int  tgp_k_attn_select(int impl);
-/* Error word of the tcgen05 attention kernel: 0, or the phase (1 waiting for S, 2 waiting for O_j) of the first
- * bounded wait that ran out.  Synchronous. */
+/* Error word of the tcgen05 attention kernel: 0, or which bounded wait ran out first (1 for S, 2 for P V, 3 for a K/V
+ * load, 4 for the hand-over between the softmax warps and the MMA warp), or 5 if shared memory was not 1024-byte
+ * aligned.  A CTA that gives up stores nothing.  Synchronous. */
 int  tgp_k_attn_status(int *error_code);
 /* Error word of the tensor-core GEMM: 0, or (role << 8 | stage) of the first bounded wait that ran out
  * (role 1 TMA producer, 2 MMA issuer, 3 epilogue).  Synchronous. */
