@@ -263,7 +263,7 @@ int  tgp_k_gemv_overlap(int enable);
  * 2 forces the persistent 128x256 kernel with double-buffered accumulators.  Process-wide; for tests and timing. */
 int  tgp_k_gemm_tc_variant(int variant);
 /* Which kernel serves attention with q_len >= 16: 0 (default) by problem size - the tcgen05 kernel (S and O in TMEM,
- * K/V fed by TMA) when the grid has at least two CTAs of 128 queries per SM, else the mma.sync flash-style kernel;
+ * K/V fed by TMA) for q_len >= 128, else the mma.sync flash-style kernel;
  * 3 / 2 force one or the other; 1 the warp-per-query-row CUDA-core kernel (an on-device cross-check).  The tcgen05
  * kernel needs KV tiles of a multiple of 64 keys whose base addresses differ by whole rows of Dh elements (and
  * 16-byte aligned q); any other geometry is served by the mma.sync kernel even when 3 is forced.  Process-wide. */

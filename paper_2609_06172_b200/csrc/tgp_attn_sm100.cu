@@ -34,7 +34,7 @@ namespace {
 
 using namespace tgp_sm100;
 typedef __nv_bfloat16 bf16;
-constexpr int BQ = 128, BKV = 64, THREADS = 160;
+constexpr int BQ = 128, BKV = 64, THREADS = 192;
 
 __device__ int g_attn_tc_error = 0;   // 0 ok; 1 S, 2 P V, 3 K/V load, 4 softmax hand-over: the wait that ran out; 5 shared memory misaligned
 
@@ -51,24 +51,22 @@ __device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr, uint32_t lb
     return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
 
-// byte offset of 16-byte chunk c (0..7) of row r inside a [rows x 128 B] K-major tile with 128-byte swizzle
-__device__ __forceinline__ uint32_t sw128(uint32_t r, uint32_t c) { return r * 128u + ((c ^ (r & 7u)) << 4); }
-
 __device__ __forceinline__ float ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
 
 template <int DH>
 __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV, const TArgs a) {
     extern __shared__ __align__(1024) uint8_t smem[];
     constexpr int KB = DH / 64;                          // 64-wide blocks of the head dimension
-    constexpr uint32_t Q_BYTES = KB * BQ * 128, KV_BYTES = KB * BKV * 128, P_BYTES = BQ * 128;
-    uint8_t *Qs = smem, *Ks = Qs + Q_BYTES, *Vs = Ks + 2 * KV_BYTES, *Ps = Vs + 2 * KV_BYTES;      // K and V: two stages each
-    uint64_t *bar_k = reinterpret_cast<uint64_t *>(Ps + P_BYTES);      // [2] K stage landed (stage 0's first use also carries Q)
+    constexpr uint32_t Q_BYTES = KB * BQ * 128, KV_BYTES = KB * BKV * 128;
+    uint8_t *Qs = smem, *Ks = Qs + Q_BYTES, *Vs = Ks + 2 * KV_BYTES;                            // K and V: two stages each
+    uint64_t *bar_k = reinterpret_cast<uint64_t *>(Vs + 2 * KV_BYTES);      // [2] K stage landed (stage 0's first use also carries Q)
     uint64_t *bar_v = bar_k + 2;                                       // [2] V stage landed
     uint64_t *bar_s = bar_v + 2;                                       // S complete in TMEM (tensor core)
     uint64_t *bar_sfree = bar_s + 1;                                   // all 128 rows of S are in registers
-    uint64_t *bar_p = bar_sfree + 1;                                   // all 128 rows of P written, O rescaled where needed
-    uint64_t *bar_o = bar_p + 1;                                       // P V complete (tensor core): P, O and the V stage are free
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bar_o + 1);
+    uint64_t *bar_p = bar_sfree + 1;                                   // [2] all 128 rows of P_j (buffer j & 1) written, O rescaled where needed
+    uint64_t *bar_o = bar_p + 2;                                       // [2] P V_j complete (tensor core): P buffer j & 1 and the V stage are free
+    uint64_t *bar_kfree = bar_o + 2;                                   // [2] S_j complete: K stage j & 1 is free
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bar_kfree + 2);
     volatile uint32_t *failed = tmem_slot + 1;
 
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -83,7 +81,7 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
 
     if (tid == 0) {
         mbar_init(bar_k, 1); mbar_init(bar_k + 1, 1); mbar_init(bar_v, 1); mbar_init(bar_v + 1, 1);
-        mbar_init(bar_s, 1); mbar_init(bar_sfree, 128); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
+        mbar_init(bar_s, 1); mbar_init(bar_sfree, 128); mbar_init(bar_p, 128); mbar_init(bar_p + 1, 128); mbar_init(bar_o, 1); mbar_init(bar_o + 1, 1); mbar_init(bar_kfree, 1); mbar_init(bar_kfree + 1, 1);
         failed[0] = 0;
         failed[1] = 0;                                       // a flag nothing ever sets, for waits that must not be cut short
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -96,22 +94,58 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 64;
+    const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 64, tmem_P = tmem_base + 192;     // P: two buffers of 32 columns (bf16 pairs)
     auto give_up = [&](int code) { if (!*failed) { *failed = 1; atomicCAS(&g_attn_tc_error, 0, code); } };
 
-    if (warp == 4) {
-        // ======================= feeder: every TMA load and every MMA =======================
-        constexpr uint32_t idesc_s = umma_idesc(BKV), idesc_o = umma_idesc(DH) | (1u << 16);     // bit 16: B operand is MN-major
-        const uint32_t head_row = (b * a.Hkv + hk) * a.TK;
-        uint32_t k_issued[2] = {0, 0}, k_waited[2] = {0, 0}, v_issued[2] = {0, 0}, v_waited[2] = {0, 0};
-        auto load_kv = [&](uint8_t *dst, const int32_t *first_row, uint32_t jb, uint64_t *bar, uint32_t more_bytes) {
-            const uint32_t j0 = jb * BKV;
-            const int y = first_row[j0 / a.TK] + (int)(head_row + j0 % a.TK);
-            mbar_expect_tx(bar, KV_BYTES + more_bytes);
+    if (warp == 5) {
+        // ======================= producer: every TMA load (lane 0) =======================
+        uint32_t nk = 0, nv = 0;                             // K / V blocks requested so far (block i uses stage i & 1)
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmQ) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmKV) : "memory");
+            const uint32_t head_row = (b * a.Hkv + hk) * a.TK;
+            uint32_t k_tile = 0, k_off = 0, v_tile = 0, v_off = 0;           // tile and key offset inside it of the next block
+            auto load_kv = [&](uint8_t *dst, int y, uint64_t *bar, uint32_t more_bytes) {
+                mbar_expect_tx(bar, KV_BYTES + more_bytes);
 #pragma unroll
-            for (uint32_t kb = 0; kb < KB; ++kb) tma_load_2d(dst + kb * (BKV * 128), &tmKV, kb * 64, y, bar);
-        };
-        auto issue_s = [&](uint32_t jb) {                    // S = Q K_jb^T
+                for (uint32_t kb = 0; kb < KB; ++kb) tma_load_2d(dst + kb * (BKV * 128), &tmKV, kb * 64, y, bar);
+            };
+            auto next_k = [&](uint32_t more_bytes) {
+                load_kv(Ks + (nk & 1) * KV_BYTES, a.krow[k_tile] + (int)(head_row + k_off), bar_k + (nk & 1), more_bytes);
+                nk += 1;
+                if ((k_off += BKV) == a.TK) { k_off = 0; k_tile += 1; }
+            };
+            auto next_v = [&]() {
+                load_kv(Vs + (nv & 1) * KV_BYTES, a.vrow[v_tile] + (int)(head_row + v_off), bar_v + (nv & 1), 0);
+                nv += 1;
+                if ((v_off += BKV) == a.TK) { v_off = 0; v_tile += 1; }
+            };
+            next_k(Q_BYTES);
+#pragma unroll
+            for (uint32_t kb = 0; kb < KB; ++kb) tma_load_2d(Qs + kb * (BQ * 128), &tmQ, hq * DH + kb * 64, b * a.q_len + q0, bar_k);
+            if (1 < nblk) next_k(0);
+            next_v();
+            for (uint32_t jb = 0; jb + 1 < nblk; ++jb) {
+                const uint32_t st = jb & 1;
+                if (jb + 2 < nblk) {                                         // K_jb+2 goes where K_jb is, once S_jb is complete
+                    if (!mbar_wait(bar_kfree + st, (jb >> 1) & 1, failed)) { give_up(1); break; }
+                    next_k(0);
+                }
+                if (jb >= 1 && !mbar_wait(bar_o + (st ^ 1), ((jb - 1) >> 1) & 1, failed)) { give_up(2); break; }   // V_jb+1 goes where V_jb-1 is
+                next_v();
+            }
+            // every load requested must have landed before the CTA may exit (bounded; `never` is never set)
+            volatile uint32_t *never = failed + 1;
+            for (uint32_t st = 0; st < 2; ++st) {
+                const uint32_t ck = (nk + 1 - st) >> 1, cv = (nv + 1 - st) >> 1;     // loads requested into this stage
+                if (ck) mbar_wait(bar_k + st, (ck - 1) & 1, never);
+                if (cv) mbar_wait(bar_v + st, (cv - 1) & 1, never);
+            }
+        }
+    } else if (warp == 4) {
+        // ======================= MMA warp: lane 0 issues every MMA =======================
+        constexpr uint32_t idesc_s = umma_idesc(BKV), idesc_o = umma_idesc(DH) | (1u << 16);     // bit 16: B operand is MN-major
+        auto issue_s = [&](uint32_t jb) {                    // S = Q K_jb^T; its completion also frees the K stage
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint8_t *Kj = Ks + (jb & 1) * KV_BYTES;
 #pragma unroll
@@ -121,45 +155,24 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
                 for (uint32_t k = 0; k < 4; ++k) umma(tmem_S, dq + 2 * k, dk + 2 * k, idesc_s, (kb | k) != 0);
             }
             umma_commit(bar_s);
+            umma_commit(bar_kfree + (jb & 1));
         };
         auto wait = [&](uint64_t *bar, uint32_t parity, int code) {
             bool ok = mbar_wait(bar, parity, failed);
             if (!ok) give_up(code);
             return __all_sync(0xffffffffu, ok);
         };
-        if (lane == 0) {
-            load_kv(Ks, a.krow, 0, bar_k, Q_BYTES);
-#pragma unroll
-            for (uint32_t kb = 0; kb < KB; ++kb) tma_load_2d(Qs + kb * (BQ * 128), &tmQ, hq * DH + kb * 64, b * a.q_len + q0, bar_k);
-            if (1 < nblk) load_kv(Ks + KV_BYTES, a.krow, 1, bar_k + 1, 0);
-            load_kv(Vs, a.vrow, 0, bar_v, 0);
-        }
-        k_issued[0] = 1; k_issued[1] = 1 < nblk ? 1 : 0; v_issued[0] = 1;
         bool ok = wait(bar_k, 0, 3);
-        if (ok) {
-            k_waited[0] = 1;
-            if (lane == 0) issue_s(0);
-        }
+        if (ok && lane == 0) issue_s(0);
         for (uint32_t jb = 0; ok && jb < nblk; ++jb) {
             const uint32_t st = jb & 1;
             if (jb + 1 < nblk) {
-                if (!(ok = wait(bar_sfree, st, 4))) break;                   // S_jb is in registers, so K stage st is free too
-                if (jb + 2 < nblk) {
-                    if (lane == 0) load_kv(Ks + st * KV_BYTES, a.krow, jb + 2, bar_k + st, 0);
-                    k_issued[st] += 1;
-                }
+                if (!(ok = wait(bar_sfree, st, 4))) break;                   // S_jb is in registers
                 if (!(ok = wait(bar_k + (st ^ 1), ((jb + 1) >> 1) & 1, 3))) break;
-                k_waited[st ^ 1] += 1;
                 if (lane == 0) issue_s(jb + 1);
             }
-            if (jb >= 1 && !(ok = wait(bar_o, (jb - 1) & 1, 2))) break;       // P V of the previous block: its V stage is free
-            if (jb + 1 < nblk) {
-                if (lane == 0) load_kv(Vs + (st ^ 1) * KV_BYTES, a.vrow, jb + 1, bar_v + (st ^ 1), 0);
-                v_issued[st ^ 1] += 1;
-            }
-            if (!(ok = wait(bar_p, st, 4))) break;
+            if (!(ok = wait(bar_p + st, (jb >> 1) & 1, 4))) break;
             if (!(ok = wait(bar_v + st, (jb >> 1) & 1, 3))) break;
-            v_waited[st] += 1;
             if (jb * BKV + BKV > kvlen) {                                    // rows past the sequence: whatever the tile holds there
                 const uint32_t valid = kvlen - jb * BKV;
                 for (uint32_t i = lane; i < (BKV - valid) * KB * 8; i += 32) {
@@ -171,17 +184,12 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
             }
             if (lane == 0) {                                                 // O += P V_jb
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint64_t dp = umma_desc(smem_u32(Ps)), dv = umma_desc_mn(smem_u32(Vs + st * KV_BYTES), BKV * 128);
+                const uint64_t dv = umma_desc_mn(smem_u32(Vs + st * KV_BYTES), BKV * 128);
 #pragma unroll
-                for (uint32_t k = 0; k < 4; ++k) umma(tmem_O, dp + 2 * k, dv + 128 * k, idesc_o, (jb | k) != 0);   // 16 keys = 2048 B of V rows per step
-                umma_commit(bar_o);
+                for (uint32_t k = 0; k < 4; ++k)                             // 16 keys per step: 8 columns of P, 2048 B of V rows
+                    umma_ts(tmem_O, tmem_P + st * 32 + 8 * k, dv + 128 * k, idesc_o, (jb | k) != 0);
+                umma_commit(bar_o + st);
             }
-        }
-        // loads still in flight after a failed wait must land before the CTA may exit (bounded; `never` is never set)
-        volatile uint32_t *never = failed + 1;
-        for (uint32_t st = 0; st < 2; ++st) {
-            if (k_issued[st] != k_waited[st]) mbar_wait(bar_k + st, (k_issued[st] - 1) & 1, never);
-            if (v_issued[st] != v_waited[st]) mbar_wait(bar_v + st, (v_issued[st] - 1) & 1, never);
         }
     } else {
         // ======================= softmax warps: thread = query row = TMEM lane =======================
@@ -211,10 +219,11 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
 #pragma unroll
             for (uint32_t i = 4; i < BKV; ++i) mx[i & 3] = fmaxf(mx[i & 3], s[i]);
             const float mblk = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * a.scale_log2;     // scale > 0: max commutes with it
-            if (jb > 0 && !(ok = wait(bar_o, (jb - 1) & 1, 2))) break;       // P V of the previous block: P and O are free
+            if (jb >= 2 && !(ok = wait(bar_o + (jb & 1), ((jb - 2) >> 1) & 1, 2))) break;      // P V_{j-2}: this P buffer is free
             if (jb == 0) {
                 m_ref = mblk;                                                // block 0 holds key 0 <= qpos: finite
             } else if (__any_sync(0xffffffffu, mblk > m_ref + 8.f)) {
+                if (!(ok = wait(bar_o + ((jb - 1) & 1), ((jb - 1) >> 1) & 1, 2))) break;           // P V_{j-1}: nothing is accumulating into O
                 const float m_new = fmaxf(m_ref, mblk), alpha = ex2(m_ref - m_new);
                 m_ref = m_new;
                 lrow *= alpha;
@@ -222,37 +231,35 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
 #pragma unroll
                 for (uint32_t h = 0; h < DH / 32; ++h) {
                     float v[32];
+                    uint32_t w[32];
                     tmem_ld32(tmem_O + lane_addr + h * 32, v);
 #pragma unroll
-                    for (uint32_t i = 0; i < 32; ++i) v[i] *= alpha;
-                    tmem_st32(tmem_O + lane_addr + h * 32, v);
+                    for (uint32_t i = 0; i < 32; ++i) w[i] = __float_as_uint(v[i] * alpha);
+                    tmem_st32(tmem_O + lane_addr + h * 32, w);
                 }
                 tmem_wait_st();
             }
-            // P = exp2(S * scale - m) as bf16: this thread's row of the K-major tile (a masked score is -inf: p = 0)
+            // P = exp2(S * scale - m) as bf16 pairs into this row's 32 columns of the P buffer (a masked score is -inf: p = 0)
             const float nm = -m_ref;
             float l0 = 0.f, l1 = 0.f;
+            uint32_t w[BKV / 2];
 #pragma unroll
-            for (uint32_t c = 0; c < BKV / 8; ++c) {
-                uint32_t w[4];
-#pragma unroll
-                for (uint32_t i = 0; i < 4; ++i) {
-                    const float p0 = ex2(fmaf(s[c * 8 + 2 * i], a.scale_log2, nm));
-                    const float p1 = ex2(fmaf(s[c * 8 + 2 * i + 1], a.scale_log2, nm));
-                    l0 += p0;
-                    l1 += p1;
-                    __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                    w[i] = *reinterpret_cast<uint32_t *>(&pk);
-                }
-                *reinterpret_cast<uint4 *>(Ps + sw128(tid, c)) = make_uint4(w[0], w[1], w[2], w[3]);
+            for (uint32_t i = 0; i < BKV / 2; ++i) {
+                const float p0 = ex2(fmaf(s[2 * i], a.scale_log2, nm));
+                const float p1 = ex2(fmaf(s[2 * i + 1], a.scale_log2, nm));
+                l0 += p0;
+                l1 += p1;
+                __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);           // .x = p0 in the lower half
+                w[i] = *reinterpret_cast<uint32_t *>(&pk);
             }
             lrow += l0 + l1;
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes of P -> visible to the tensor core
+            tmem_st32(tmem_P + (jb & 1) * 32 + lane_addr, w);
+            tmem_wait_st();
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            mbar_arrive(bar_p);
+            mbar_arrive(bar_p + (jb & 1));
         }
         // ---- the last P V; normalise and store this thread's row ----
-        if (ok) ok = wait(bar_o, (nblk - 1) & 1, 2);
+        if (ok) ok = wait(bar_o + ((nblk - 1) & 1), ((nblk - 1) >> 1) & 1, 2);
         if (ok) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const float inv = 1.0f / lrow;
@@ -284,7 +291,7 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
     }
 }
 
-template <int DH> constexpr int smem_bytes() { return (DH / 64) * (BQ + 4 * BKV) * 128 + BQ * 128 + 128; }
+template <int DH> constexpr int smem_bytes() { return (DH / 64) * (BQ + 4 * BKV) * 128 + 128; }
 
 }  // namespace
 

@@ -794,12 +794,9 @@ int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *
         }
         tgpk_launches += 1;
     } else if (q_len >= 16 && (g_attn_impl == 0 || g_attn_impl == 2 || g_attn_impl == 3)) {
-        // the tcgen05 kernel (128 queries per CTA, a serial chain per key block) needs at least two CTAs per SM of
-        // parallel work to beat the mma.sync kernel (64 queries per CTA)
-        static int sms = 0;
-        if (!sms) { int dev = 0; cudaGetDevice(&dev); if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148; }
-        const uint64_t ctas = (uint64_t)((q_len + 127) / 128) * c->Hq * B;
-        if (g_attn_impl == 3 || (g_attn_impl == 0 && ctas >= 2ull * sms)) return tgpk_attn_prefill_tc5(qb, tiles, ob, c, B, q_len, pos0, st);
+        // the tcgen05 kernel works on 128 queries per CTA (it hands geometries it cannot map with TMA to the mma.sync
+        // kernel itself); below that the mma.sync kernel's 64-query CTAs waste less
+        if (g_attn_impl == 3 || (g_attn_impl == 0 && q_len >= 128)) return tgpk_attn_prefill_tc5(qb, tiles, ob, c, B, q_len, pos0, st);
         return tgpk_attn_prefill_tc(qb, tiles, ob, c, B, q_len, pos0, st);
     } else {
         dim3 grid((q_len + 3) / 4, c->Hq, B);
