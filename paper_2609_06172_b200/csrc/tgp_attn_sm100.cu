@@ -34,7 +34,7 @@ namespace {
 
 using namespace tgp_sm100;
 typedef __nv_bfloat16 bf16;
-constexpr int BQ = 128, BKV = 64, THREADS = 192;
+constexpr int BQ = 128, BKV = 64, THREADS = 224;
 
 __device__ int g_attn_tc_error = 0;   // 0 ok; 1 S, 2 P V, 3 K/V load, 4 softmax hand-over: the wait that ran out; 5 shared memory misaligned
 
@@ -143,36 +143,42 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
             }
         }
     } else if (warp == 4) {
-        // ======================= MMA warp: lane 0 issues every MMA =======================
-        constexpr uint32_t idesc_s = umma_idesc(BKV), idesc_o = umma_idesc(DH) | (1u << 16);     // bit 16: B operand is MN-major
-        auto issue_s = [&](uint32_t jb) {                    // S = Q K_jb^T; its completion also frees the K stage
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint8_t *Kj = Ks + (jb & 1) * KV_BYTES;
-#pragma unroll
-            for (uint32_t kb = 0; kb < KB; ++kb) {
-                const uint64_t dq = umma_desc(smem_u32(Qs + kb * (BQ * 128))), dk = umma_desc(smem_u32(Kj + kb * (BKV * 128)));
-#pragma unroll
-                for (uint32_t k = 0; k < 4; ++k) umma(tmem_S, dq + 2 * k, dk + 2 * k, idesc_s, (kb | k) != 0);
-            }
-            umma_commit(bar_s);
-            umma_commit(bar_kfree + (jb & 1));
-        };
+        // ======================= S warp: lane 0 issues S_j = Q K_j^T =======================
+        constexpr uint32_t idesc_s = umma_idesc(BKV);
         auto wait = [&](uint64_t *bar, uint32_t parity, int code) {
             bool ok = mbar_wait(bar, parity, failed);
             if (!ok) give_up(code);
             return __all_sync(0xffffffffu, ok);
         };
-        bool ok = wait(bar_k, 0, 3);
-        if (ok && lane == 0) issue_s(0);
-        for (uint32_t jb = 0; ok && jb < nblk; ++jb) {
-            const uint32_t st = jb & 1;
-            if (jb + 1 < nblk) {
-                if (!(ok = wait(bar_sfree, st, 4))) break;                   // S_jb is in registers
-                if (!(ok = wait(bar_k + (st ^ 1), ((jb + 1) >> 1) & 1, 3))) break;
-                if (lane == 0) issue_s(jb + 1);
+        for (uint32_t jb = 0; jb < nblk; ++jb) {
+            if (jb >= 1 && !wait(bar_sfree, (jb - 1) & 1, 4)) break;         // S_jb-1 is in registers
+            if (!wait(bar_k + (jb & 1), (jb >> 1) & 1, 3)) break;            // K_jb (and Q with K_0) has landed
+            if (lane == 0) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint8_t *Kj = Ks + (jb & 1) * KV_BYTES;
+#pragma unroll
+                for (uint32_t kb = 0; kb < KB; ++kb) {
+                    const uint64_t dq = umma_desc(smem_u32(Qs + kb * (BQ * 128))), dk = umma_desc(smem_u32(Kj + kb * (BKV * 128)));
+#pragma unroll
+                    for (uint32_t k = 0; k < 4; ++k) umma(tmem_S, dq + 2 * k, dk + 2 * k, idesc_s, (kb | k) != 0);
+                }
+                umma_commit(bar_s);
+                umma_commit(bar_kfree + (jb & 1));                           // its completion also frees the K stage
             }
-            if (!(ok = wait(bar_p + st, (jb >> 1) & 1, 4))) break;
-            if (!(ok = wait(bar_v + st, (jb >> 1) & 1, 3))) break;
+            __syncwarp();
+        }
+    } else if (warp == 6) {
+        // ======================= P V warp: lane 0 issues O += P_j V_j =======================
+        constexpr uint32_t idesc_o = umma_idesc(DH) | (1u << 16);           // bit 16: B operand is MN-major
+        auto wait = [&](uint64_t *bar, uint32_t parity, int code) {
+            bool ok = mbar_wait(bar, parity, failed);
+            if (!ok) give_up(code);
+            return __all_sync(0xffffffffu, ok);
+        };
+        for (uint32_t jb = 0; jb < nblk; ++jb) {
+            const uint32_t st = jb & 1;
+            if (!wait(bar_p + st, (jb >> 1) & 1, 4)) break;
+            if (!wait(bar_v + st, (jb >> 1) & 1, 3)) break;
             if (jb * BKV + BKV > kvlen) {                                    // rows past the sequence: whatever the tile holds there
                 const uint32_t valid = kvlen - jb * BKV;
                 for (uint32_t i = lane; i < (BKV - valid) * KB * 8; i += 32) {
@@ -182,7 +188,7 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
             }
-            if (lane == 0) {                                                 // O += P V_jb
+            if (lane == 0) {
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint64_t dv = umma_desc_mn(smem_u32(Vs + st * KV_BYTES), BKV * 128);
 #pragma unroll
@@ -190,6 +196,7 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
                     umma_ts(tmem_O, tmem_P + st * 32 + 8 * k, dv + 128 * k, idesc_o, (jb | k) != 0);
                 umma_commit(bar_o + st);
             }
+            __syncwarp();
         }
     } else {
         // ======================= softmax warps: thread = query row = TMEM lane =======================
