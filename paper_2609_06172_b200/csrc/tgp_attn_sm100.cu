@@ -51,10 +51,13 @@ __device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr, uint32_t lb
     return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
 
+// byte offset of 16-byte chunk c (0..7) of row r inside a [rows x 128 B] tile with the 128-byte swizzle
+__device__ __forceinline__ uint32_t sw128(uint32_t r, uint32_t c) { return r * 128u + ((c ^ (r & 7u)) << 4); }
+
 __device__ __forceinline__ float ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
 
 template <int DH>
-__global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV, const TArgs a) {
+__global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUtensorMap tmO, const TArgs a) {
     extern __shared__ __align__(1024) uint8_t smem[];
     constexpr int KB = DH / 64;                          // 64-wide blocks of the head dimension
     constexpr uint32_t Q_BYTES = KB * BQ * 128, KV_BYTES = KB * BKV * 128;
@@ -74,7 +77,7 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
         if (tid == 0) atomicCAS(&g_attn_tc_error, 0, 5);
         return;
     }
-    const uint32_t qblk = blockIdx.x, hq = blockIdx.y, b = blockIdx.z, hk = hq / (a.Hq / a.Hkv);
+    const uint32_t qblk = gridDim.x - 1 - blockIdx.x, hq = blockIdx.y, b = blockIdx.z, hk = hq / (a.Hq / a.Hkv);      // longest (latest) query blocks are launched first
     const uint32_t q0 = qblk * BQ, kvlen = a.pos0 + a.q_len;
     const uint32_t last_q = min(a.q_len, q0 + BQ) - 1;
     const uint32_t nblk = (a.pos0 + last_q + 1 + BKV - 1) / BKV;
@@ -270,22 +273,35 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
         if (ok) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const float inv = 1.0f / lrow;
+            const bool full_tile = q0 + BQ <= a.q_len;                       // a TMA store would spill padding rows into the next sequence
             bf16 *dst = a.ob + ((size_t)(b * a.q_len + q0 + tid) * a.Hq + hq) * DH;
 #pragma unroll
             for (uint32_t h = 0; h < DH / 32; ++h) {
                 float v[32];
                 tmem_ld32(tmem_O + lane_addr + h * 32, v);
-                if (row_ok) {
 #pragma unroll
-                    for (uint32_t c = 0; c < 4; ++c) {
-                        uint32_t w[4];
+                for (uint32_t c = 0; c < 4; ++c) {
+                    uint32_t w[4];
 #pragma unroll
-                        for (uint32_t i = 0; i < 4; ++i) {
-                            __nv_bfloat162 pk = __floats2bfloat162_rn(v[c * 8 + 2 * i] * inv, v[c * 8 + 2 * i + 1] * inv);
-                            w[i] = *reinterpret_cast<uint32_t *>(&pk);
-                        }
-                        *reinterpret_cast<uint4 *>(dst + h * 32 + c * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                    for (uint32_t i = 0; i < 4; ++i) {
+                        __nv_bfloat162 pk = __floats2bfloat162_rn(v[c * 8 + 2 * i] * inv, v[c * 8 + 2 * i + 1] * inv);
+                        w[i] = *reinterpret_cast<uint32_t *>(&pk);
                     }
+                    // the Q tile is no longer read (every S is complete): it stages the output tile in the same layout
+                    if (full_tile) *reinterpret_cast<uint4 *>(Qs + (h / 2) * (BQ * 128) + sw128(tid, (h % 2) * 4 + c)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    else if (row_ok) *reinterpret_cast<uint4 *>(dst + h * 32 + c * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+            if (full_tile) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(bar_sfree);                                      // one more phase of this barrier: the four softmax warps meet
+                if (wait(bar_sfree, nblk & 1, 4) && tid == 0) {
+#pragma unroll
+                    for (uint32_t kb = 0; kb < KB; ++kb)
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                                     ::"l"(&tmO), "r"((int)(hq * DH + kb * 64)), "r"((int)(b * a.q_len + q0)), "r"(smem_u32(Qs + kb * (BQ * 128))) : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");     // shared memory must outlive the read
                 }
             }
         }
@@ -317,7 +333,7 @@ int tgpk_attn_prefill_tc5(const void *qb, const TgpTilePtrs &tiles, void *ob, co
             lo = lo < p ? lo : p;
             hi = hi > p ? hi : p;
         }
-    bool fits = c->TK % BKV == 0 && lo % 16 == 0 && (uintptr_t)qb % 16 == 0 && ((hi - lo) / row_bytes + tile_rows) < (1ull << 31);
+    bool fits = c->TK % BKV == 0 && lo % 16 == 0 && (uintptr_t)qb % 16 == 0 && (uintptr_t)ob % 16 == 0 && ((hi - lo) / row_bytes + tile_rows) < (1ull << 31);
     for (uint32_t t = 0; fits && t < n_tiles; ++t)
         fits = ((uintptr_t)tiles.k[t] - lo) % row_bytes == 0 && ((uintptr_t)tiles.v[t] - lo) % row_bytes == 0;
     if (!fits) return tgpk_attn_prefill_tc(qb, tiles, ob, c, B, q_len, pos0, st);
@@ -326,9 +342,10 @@ int tgpk_attn_prefill_tc5(const void *qb, const TgpTilePtrs &tiles, void *ob, co
         a.krow[t] = (int32_t)(((uintptr_t)tiles.k[t] - lo) / row_bytes);
         a.vrow[t] = (int32_t)(((uintptr_t)tiles.v[t] - lo) / row_bytes);
     }
-    CUtensorMap mq, mkv;
+    CUtensorMap mq, mkv, mo;
     if (!tensor_map_bf16_2d(&mq, qb, (uint64_t)B * q_len, (uint64_t)c->Hq * c->Dh, (uint64_t)c->Hq * c->Dh * 2, BQ) ||
-        !tensor_map_bf16_2d(&mkv, (const void *)lo, (hi - lo) / row_bytes + tile_rows, c->Dh, row_bytes, BKV))
+        !tensor_map_bf16_2d(&mkv, (const void *)lo, (hi - lo) / row_bytes + tile_rows, c->Dh, row_bytes, BKV) ||
+        !tensor_map_bf16_2d(&mo, ob, (uint64_t)B * q_len, (uint64_t)c->Hq * c->Dh, (uint64_t)c->Hq * c->Dh * 2, BQ))
         return TGP_E_CUDA;
     dim3 grid((q_len + BQ - 1) / BQ, c->Hq, B);
     static bool attr64 = false, attr128 = false;
@@ -338,14 +355,14 @@ int tgpk_attn_prefill_tc5(const void *qb, const TgpTilePtrs &tiles, void *ob, co
             cudaFuncSetAttribute(attn_prefill_tc_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
             attr64 = true;
         }
-        attn_prefill_tc_kernel<64><<<grid, THREADS, smem_bytes<64>(), st>>>(mq, mkv, a);
+        attn_prefill_tc_kernel<64><<<grid, THREADS, smem_bytes<64>(), st>>>(mq, mkv, mo, a);
     } else {
         if (!attr128) {
             if (cudaFuncSetAttribute(attn_prefill_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128>()) != cudaSuccess) return TGP_E_CUDA;
             cudaFuncSetAttribute(attn_prefill_tc_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
             attr128 = true;
         }
-        attn_prefill_tc_kernel<128><<<grid, THREADS, smem_bytes<128>(), st>>>(mq, mkv, a);
+        attn_prefill_tc_kernel<128><<<grid, THREADS, smem_bytes<128>(), st>>>(mq, mkv, mo, a);
     }
     if (cudaGetLastError() != cudaSuccess) return TGP_E_CUDA;
     tgpk_launches += 1;
