@@ -55,6 +55,12 @@ __device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr, uint32_t lb
 __device__ __forceinline__ uint32_t sw128(uint32_t r, uint32_t c) { return r * 128u + ((c ^ (r & 7u)) << 4); }
 
 __device__ __forceinline__ float ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+// two fp32 values per instruction (sm_100 packed arithmetic) and the three-input maximum
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r; }
+__device__ __forceinline__ void unpack2(uint64_t r, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(r)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t x, uint64_t y, uint64_t z) { uint64_t d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(x), "l"(y), "l"(z)); return d; }
+__device__ __forceinline__ uint64_t add2(uint64_t x, uint64_t y) { uint64_t d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(x), "l"(y)); return d; }
+__device__ __forceinline__ float max3(float x, float y, float z) { float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(x), "f"(y), "f"(z)); return d; }
 
 template <int DH>
 __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUtensorMap tmO, const TArgs a) {
@@ -225,44 +231,53 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
                 for (uint32_t i = 0; i < BKV; ++i)
                     if (jb * BKV + i > qpos) s[i] = -INFINITY;
             }
-            float mx[4] = {s[0], s[1], s[2], s[3]};
+            auto row_max = [&]() {                                           // of the scaled scores (scale > 0: max commutes with it)
+                float m0 = max3(s[0], s[1], s[2]), m1 = max3(s[3], s[4], s[5]);
 #pragma unroll
-            for (uint32_t i = 4; i < BKV; ++i) mx[i & 3] = fmaxf(mx[i & 3], s[i]);
-            const float mblk = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * a.scale_log2;     // scale > 0: max commutes with it
-            if (jb >= 2 && !(ok = wait(bar_o + (jb & 1), ((jb - 2) >> 1) & 1, 2))) break;      // P V_{j-2}: this P buffer is free
-            if (jb == 0) {
-                m_ref = mblk;                                                // block 0 holds key 0 <= qpos: finite
-            } else if (__any_sync(0xffffffffu, mblk > m_ref + 8.f)) {
+                for (uint32_t i = 6; i + 3 < BKV; i += 4) { m0 = max3(m0, s[i], s[i + 1]); m1 = max3(m1, s[i + 2], s[i + 3]); }
+                return max3(m0, m1, fmaxf(s[BKV - 2], s[BKV - 1])) * a.scale_log2;
+            };
+            uint32_t w[BKV / 2];
+            auto exps = [&](float m) {                                       // w = exp2(S * scale - m) as bf16 pairs; returns their fp32 sum
+                const uint64_t sc2 = pack2(a.scale_log2, a.scale_log2), nm2 = pack2(-m, -m);
+                uint64_t acc0 = pack2(0.f, 0.f), acc1 = acc0;
+#pragma unroll
+                for (uint32_t i = 0; i < BKV / 2; ++i) {
+                    float x0, x1;
+                    unpack2(fma2(pack2(s[2 * i], s[2 * i + 1]), sc2, nm2), x0, x1);
+                    const float p0 = ex2(x0), p1 = ex2(x1);                  // a masked score is -inf: p = 0
+                    if (i & 1) acc1 = add2(acc1, pack2(p0, p1)); else acc0 = add2(acc0, pack2(p0, p1));
+                    __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);       // .x = p0 in the lower half
+                    w[i] = *reinterpret_cast<uint32_t *>(&pk);
+                }
+                float l0, l1;
+                unpack2(add2(acc0, acc1), l0, l1);
+                return l0 + l1;
+            };
+            // The exponent reference m is the row max of block 0 (which holds key 0 <= qpos: finite).  Later blocks use it
+            // as it is and never look for their own max: only when a block's sum says that a score of one of the warp's
+            // rows lies more than about 2^40 above m (or overflowed) does the warp take the slow path.
+            if (jb == 0) m_ref = row_max();
+            float lblk = exps(m_ref);
+            if (jb > 0 && __any_sync(0xffffffffu, !(lblk <= 0x1p40f))) {
                 if (!(ok = wait(bar_o + ((jb - 1) & 1), ((jb - 1) >> 1) & 1, 2))) break;           // P V_{j-1}: nothing is accumulating into O
-                const float m_new = fmaxf(m_ref, mblk), alpha = ex2(m_ref - m_new);
+                const float m_new = fmaxf(m_ref, row_max()), alpha = ex2(m_ref - m_new);
                 m_ref = m_new;
                 lrow *= alpha;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
                 for (uint32_t h = 0; h < DH / 32; ++h) {
                     float v[32];
-                    uint32_t w[32];
+                    uint32_t u[32];
                     tmem_ld32(tmem_O + lane_addr + h * 32, v);
 #pragma unroll
-                    for (uint32_t i = 0; i < 32; ++i) w[i] = __float_as_uint(v[i] * alpha);
-                    tmem_st32(tmem_O + lane_addr + h * 32, w);
+                    for (uint32_t i = 0; i < 32; ++i) u[i] = __float_as_uint(v[i] * alpha);
+                    tmem_st32(tmem_O + lane_addr + h * 32, u);
                 }
-                tmem_wait_st();
+                lblk = exps(m_ref);
             }
-            // P = exp2(S * scale - m) as bf16 pairs into this row's 32 columns of the P buffer (a masked score is -inf: p = 0)
-            const float nm = -m_ref;
-            float l0 = 0.f, l1 = 0.f;
-            uint32_t w[BKV / 2];
-#pragma unroll
-            for (uint32_t i = 0; i < BKV / 2; ++i) {
-                const float p0 = ex2(fmaf(s[2 * i], a.scale_log2, nm));
-                const float p1 = ex2(fmaf(s[2 * i + 1], a.scale_log2, nm));
-                l0 += p0;
-                l1 += p1;
-                __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);           // .x = p0 in the lower half
-                w[i] = *reinterpret_cast<uint32_t *>(&pk);
-            }
-            lrow += l0 + l1;
+            lrow += lblk;
+            if (jb >= 2 && !(ok = wait(bar_o + (jb & 1), ((jb - 2) >> 1) & 1, 2))) break;      // P V_{j-2}: this P buffer is free
             tmem_st32(tmem_P + (jb & 1) * 32 + lane_addr, w);
             tmem_wait_st();
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
