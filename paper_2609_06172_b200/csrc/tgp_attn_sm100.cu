@@ -1,28 +1,37 @@
 // Causal GQA attention for prefill on the 5th-generation tensor cores (sm_100a).
 //
-// One CTA owns 128 consecutive queries of one (sequence, query head).  Warps 0-3 are the softmax warps: thread t is
-// query row t and TMEM lane t.  Warp 4 feeds the tensor core: its lane 0 issues every TMA load and every MMA.
-// Shared memory holds Q, two stages each of K and V blocks of 64 keys, and P, all as 64-wide blocks of
-// [rows x 128 B] with the 128-byte swizzle (what a TMA box of 64 elements writes); K is then a K-major operand (head
-// dimension contiguous) and V, in the very same layout, an MN-major operand (its contiguous dimension is the output
-// dimension of P V).  One tensor map covers the address span of all KV tiles of the layer (tile bases differ by whole
-// rows, a key block never crosses a tile), a second one the query activations.
-// TMEM holds S (64 columns) and the output accumulator O (Dh columns), accumulated over all key blocks.
-// Per key block j, with no CTA-wide barrier anywhere in the loop:
-//   feeder:  wait "S_j is in registers" -> load K_{j+2} into the stage S_j used, wait K_{j+1}, issue S_{j+1};
-//            wait P V_{j-1} -> load V_{j+1};   wait "P_j written", V_j -> issue O += P_j V_j.
-//   softmax: wait S_j, read the row, signal; row max of the scaled, masked scores.  The exponent reference m only
-//            moves when some row of the warp exceeds it by more than 8 (log2 units): then the warp multiplies its 32
-//            rows of O in TMEM and its sums by 2^(m_old - m_new); otherwise P may reach 2^8, which fp32 sums and bf16
-//            P hold without loss, and the CUDA cores never touch O.  Wait P V_{j-1} (P and O are free), write
-//            P = exp2(S - m) as bf16, signal.
-// At the end every thread reads its row of O once, divides by its sum and stores bf16.
-// Two CTAs fit on an SM (112 KB of shared memory, 256 TMEM columns each).  KV tiles must hold a multiple of 64 keys;
-// other geometries go to the mma.sync kernel.  Rows of the last V block past the sequence are zeroed in shared memory
+// One CTA of eight warps owns 128 consecutive queries of one (sequence, query head); the longest query blocks are
+// launched first.  Roles:
+//   warps 0-3  softmax: thread t is query row t and TMEM lane t;
+//   warp 4     lane 0 issues S_j = Q K_j^T;          warp 6  lane 0 issues O += P_j V_j;
+//   warp 5     lane 0 issues every TMA load;         warp 7  idle (completes the second warpgroup for setmaxnreg).
+// Shared memory holds Q and two stages each of K and V blocks of 64 keys as 64-wide blocks of [rows x 128 B] with the
+// 128-byte swizzle (what a TMA box of 64 elements writes); K is then a K-major operand (head dimension contiguous) and
+// V, in the very same layout, an MN-major operand (its contiguous dimension is the output dimension of P V).  One tensor
+// map covers the address span of all KV tiles of the layer (tile bases differ by whole rows, a key block never crosses
+// a tile), one the query activations, one the output.
+// TMEM (256 columns): S (64, fp32), the output accumulator O (Dh, fp32, accumulated over all key blocks by the tensor
+// core) and two buffers of P (32 each: bf16 pairs, read by the second product as its A operand straight from TMEM).
+// Nothing in the key loop is a CTA-wide barrier; the roles hand over through mbarriers:
+//   K_j landed, S_{j-1} in registers  -> S warp issues S_j; its completion releases S to the softmax warps and the K
+//                                        stage to the TMA warp, which refills it with K_{j+2};
+//   P_j written, V_j landed           -> P V warp issues O += P_j V_j; its completion releases the P buffer and the V
+//                                        stage (refilled with V_{j+2}).
+// An MMA accumulating into the same TMEM tile costs 75-90 cycles whatever its N <= 128, so S (8 MMAs) and P V (4) are
+// issued by different warps and overlap with each other and with the other CTA of the SM.
+// Softmax: the exponent reference m of a row is its max over block 0.  Later blocks use it as it is - P = exp2(S - m)
+// may then exceed 1, which fp32 sums and bf16 P hold without loss of precision - and never compute a row max; only
+// when a block's sum of exponentials exceeds 2^40 (or overflowed) does the warp wait for the P V in flight, move m to
+// the new max and multiply its 32 rows of O in TMEM and its sums by 2^(m_old - m_new).  Scale-and-subtract and the sums
+// use packed fp32 pairs.  At the end every thread reads its row of O once, divides by its sum, and the tile leaves
+// through the (now free) Q buffer by TMA store (partial tiles: plain stores).
+// Two CTAs fit on an SM (96 KB of shared memory, 256 TMEM columns, 128 registers per thread each, of which setmaxnreg
+// moves the single-thread warps' share to the softmax warps).  KV tiles must hold a multiple of 64 keys; other
+// geometries go to the mma.sync kernel.  Rows of the last V block past the sequence are zeroed in shared memory
 // (0 * stale NaN would poison O); stale K rows only produce masked scores.
 // P is rounded to bf16 for the second product (the one rounding of this path the CPU oracle does not mirror).
-// Every mbarrier wait is bounded; a wait that runs out sets an error word, every role leaves its loop, the feeder waits
-// (bounded) for the loads it still has in flight, TMEM is freed and nothing is stored.
+// Every mbarrier wait is bounded; a wait that runs out sets an error word, every role leaves its loop, the TMA warp
+// waits (bounded) for the loads it still has in flight, TMEM is freed and nothing is stored.
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <cstdint>
@@ -34,7 +43,7 @@ namespace {
 
 using namespace tgp_sm100;
 typedef __nv_bfloat16 bf16;
-constexpr int BQ = 128, BKV = 64, THREADS = 224;
+constexpr int BQ = 128, BKV = 64, THREADS = 256;   // warps 0-3 softmax, 4 S, 5 TMA, 6 P V, 7 idle (fills the second warpgroup)
 
 __device__ int g_attn_tc_error = 0;   // 0 ok; 1 S, 2 P V, 3 K/V load, 4 softmax hand-over: the wait that ran out; 5 shared memory misaligned
 
@@ -105,7 +114,14 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 64, tmem_P = tmem_base + 192;     // P: two buffers of 32 columns (bf16 pairs)
     auto give_up = [&](int code) { if (!*failed) { *failed = 1; atomicCAS(&g_attn_tc_error, 0, code); } };
+    // registers move from the second warpgroup (three single-thread roles) to the softmax warpgroup: 128 * 48 + 128 * 208
+    // is the 128 per thread the CTA was launched with
 
+
+    // Registers move from the second warpgroup (three single-thread roles and an idle warp) to the softmax warpgroup:
+    // 128 * 64 + 128 * 192 is the 128 per thread the CTA is launched with.
+    if (warp >= 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;" ::: "memory");
     if (warp == 5) {
         // ======================= producer: every TMA load (lane 0) =======================
         uint32_t nk = 0, nv = 0;                             // K / V blocks requested so far (block i uses stage i & 1)
@@ -207,7 +223,9 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
             }
             __syncwarp();
         }
+    }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 192;" ::: "memory");
         // ======================= softmax warps: thread = query row = TMEM lane =======================
         const bool row_ok = q0 + tid < a.q_len;
         const uint32_t qpos = a.pos0 + min(q0 + tid, a.q_len - 1);          // padding rows take the last query's mask
