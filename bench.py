@@ -16,6 +16,7 @@ no collective on the data path); the line reports the whole-job rate over the sl
 from __future__ import annotations
 
 import argparse
+from dataclasses import replace
 import json
 import os
 import struct
@@ -213,6 +214,47 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
     return sec, bytes_per, flops_per, len(shapes), table
 
 
+def attention_loop(cfg, reps, device):
+    """Times the causal prefill attention of one layer at the workload's shape (B sequences of S queries, KV in the
+    engine's tile layout), once per kernel: the tcgen05 kernel, the mma.sync kernel, and the automatic choice.
+    Flops are the causal ones, 4 * B * Hq * Dh * S (S + 1) / 2.  Q, K, V: seeded normal values."""
+    import torch
+    from paper_2609_06172_b200 import binding as tb
+    from paper_2609_06172_b200.session import model_cfg
+    mc = model_cfg(cfg)
+    B, S = cfg.B, cfg.S
+    g = torch.Generator(device=device)
+    g.manual_seed(cfg.seed)
+    n = B * cfg.Hkv * cfg.TK * cfg.Dh
+    n_tiles = (S + cfg.TK - 1) // cfg.TK
+    kt = [torch.randn(n, device=device, generator=g).bfloat16() for _ in range(n_tiles)]
+    vt = [torch.randn(n, device=device, generator=g).bfloat16() for _ in range(n_tiles)]
+    qb = torch.randn(B * S, cfg.Hq * cfg.Dh, device=device, generator=g).bfloat16()
+    ob = torch.zeros(B * S, cfg.Hq * cfg.Dh, dtype=torch.bfloat16, device=device)
+    flops = 4 * B * cfg.Hq * cfg.Dh * S * (S + 1) / 2
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)         # larger than L2: written between timed launches
+    out = {}
+    for name, impl in (("tcgen05", 3), ("mma_sync", 2), ("auto", 0)):
+        tb.k_attn_select(impl)
+        for _ in range(3):
+            tb.k_attn(qb, kt, vt, ob, mc, B, S, 0, None)
+        torch.cuda.synchronize()
+        ms = 0.0
+        for _ in range(reps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            tb.k_attn(qb, kt, vt, ob, mc, B, S, 0, None)
+            e1.record()
+            torch.cuda.synchronize()
+            ms += e0.elapsed_time(e1)
+        t = ms * 1e-3 / reps
+        out[name] = {"us": round(t * 1e6, 1), "TFLOPs": round(flops / t / 1e12, 1)}
+    tb.k_attn_select(0)
+    out["status"] = tb.k_attn_status()
+    return out, flops
+
+
 def whole_job_rate(units_per_rank, ms_local, dist=None, device=None):
     """Replicas: every rank processed `units_per_rank` units in `ms_local`; the job's rate is all units over the
     slowest rank's time.  The only collective is this MAX reduction of the timing (none on the data path)."""
@@ -272,9 +314,10 @@ def main():
     ap.add_argument("--decode", type=int, default=None, help="decode steps per pass (default: the configuration's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-uvm", action="store_true", help="skip the demand-paged managed-memory baseline")
-    ap.add_argument("--kernel-loop", choices=["decode", "prefill"], default=None,
+    ap.add_argument("--kernel-loop", choices=["decode", "prefill", "attention"], default=None,
                     help="only run the back-to-back weight-product loop of one step (small, for ncu captures)")
     ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--seq", type=int, default=None, help="with --kernel-loop attention: prompt length instead of the configuration's")
     ap.add_argument("--graph", action="store_true", help="replay the whole planned run as one CUDA graph (dense models; for host-bound tiny steps)")
     ap.add_argument("--layers", type=int, default=None, help="run the shape at reduced depth; a byte budget is scaled in proportion")
     ap.add_argument("--cap-mib", type=float, default=None, help="sub-range cap in MiB (default: the input recipe's rule)")
@@ -283,11 +326,9 @@ def main():
     args = ap.parse_args()
     cfg = si.CONFIGS[args.config]
     if args.decode is not None:
-        from dataclasses import replace
         cfg = replace(cfg, T=args.decode)
     budget = None
     if args.layers is not None and args.layers != cfg.L:
-        from dataclasses import replace
         full = si.build_layout(cfg)
         cfg2 = replace(cfg, L=args.layers, name=f"{cfg.name}_L{args.layers}")
         budget = int(full.budget * si.build_layout(cfg2, budget=1 << 40).pool_bytes / full.pool_bytes) // 512 * 512
@@ -303,6 +344,13 @@ def main():
         import torch
         from paper_2609_06172_b200 import binding as tb
         tb.lib()
+        if args.kernel_loop == "attention":
+            if args.seq:
+                cfg = replace(cfg, S=args.seq)
+            table, flops = attention_loop(cfg, args.reps, torch.device("cuda:0"))
+            print(json.dumps({"kernel_loop": "attention", "config": cfg.name, "B": cfg.B, "S": cfg.S, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "Dh": cfg.Dh,
+                              "TK": cfg.TK, "causal_flops": flops, "L2_flushed_between_launches": True, "kernels": table}))
+            return
         M = cfg.B * (cfg.S if args.kernel_loop == "prefill" else 1)
         sec, b, f, nl, table = kernel_loop(lay, M, args.reps, torch.device("cuda:0"))
         print(json.dumps({"kernel_loop": args.kernel_loop, "M": M, "avg_us": sec * 1e6, "GBps": b / sec / 1e9, "TFLOPs": f / sec / 1e12,
