@@ -580,12 +580,22 @@ def main():
             s.close()
             torch.cuda.empty_cache()
             uvm = uvm_baseline.run(cfg, lay, MACHINE, dev, lambda l, arr: arr.__setitem__(slice(None), pool.numpy()),
-                                   decode_cap=16 if lay.pool_bytes < (4 << 30) else 4)
+                                   variants=(tb.VAR_MANAGED_DEMAND, tb.VAR_MANAGED_HINTS, tb.VAR_MANAGED_OBJECT),
+                                   decode_cap=16 if lay.pool_bytes < (4 << 30) else 4, object_bytes=SEG)
             dec = cfg.B * T / (sum(step_ms[1:]) * 1e-3) if T else None
             for v in uvm.values():
                 if dec and v.get("decode_tok_s"):
                     v["explicit_ring_speedup_decode"] = dec / v["decode_tok_s"]
             out["uvm"] = uvm
+            mo = uvm.get("managed_object")
+            if mo and mo.get("asked_bytes_per_decode_step"):
+                # the same experiment run for real: the managed pool with the segment-granular prefetcher one op ahead
+                touched = sum(a[2] for o in ops if o[0] >= 1 for a in o[6]) / max(1, T)
+                object_level["measured"] = {"decode_tok_s": mo["decode_tok_s"], "asked_bytes_per_decode_step": mo["asked_bytes_per_decode_step"],
+                                            "touched_bytes_per_decode_step": touched,
+                                            "asked_over_touched": mo["asked_bytes_per_decode_step"] / max(1.0, touched),
+                                            "tensor_level_hints_speedup": uvm["managed_hints"]["decode_tok_s"] / mo["decode_tok_s"],
+                                            "explicit_ring_speedup": mo.get("explicit_ring_speedup_decode")}
         except Exception as ex:  # the baseline is reported, never fatal
             out["uvm"] = f"not run: {type(ex).__name__}: {ex}"
     if not args.no_cpu_baseline:

@@ -87,6 +87,7 @@ extern "C" {
 #define TGP_VAR_EXPLICIT_RING   0u  /* staged copies into the arena on a copy stream, events, no demand faults */
 #define TGP_VAR_MANAGED_HINTS   1u  /* managed pool + cudaMemPrefetchAsync on critical tensors + cudaMemAdvise on pins */
 #define TGP_VAR_MANAGED_DEMAND  2u  /* managed pool, no hints: the demand-paged baseline                        */
+#define TGP_VAR_MANAGED_OBJECT  3u  /* managed pool; ahead of each op, a prefetch of every whole allocator segment its tensors overlap */
 /* policy bits (ablation switches of the paper's Section V-E: T is always on) */
 #define TGP_BIT_A  1u   /* look-ahead affinity: residency (pin) set              */
 #define TGP_BIT_P  2u   /* roofline selectivity; off = every op with pool traffic is link-bound */
@@ -158,6 +159,12 @@ int  tgp_trace_export(const tgp_ctx *ctx, void *buf, uint64_t *bytes);
 /* ---- policy (Section III-C, IV-C, IV-D) ------------------------------------------------------ */
 int  tgp_set_budget(tgp_ctx *ctx, uint64_t bytes);          /* device bytes for resident pool tensors     */
 int  tgp_set_variant(tgp_ctx *ctx, uint32_t variant, uint32_t policy_bits);
+/* Segment size of TGP_VAR_MANAGED_OBJECT: the prefetcher of the paper's motivation (Section III-B) sees the
+ * allocator's objects, not the tensors inside them, so it asks for every `bytes`-sized, `bytes`-aligned piece of the
+ * pool that a tensor of the coming op overlaps, whole (default 20 MiB, the large-block size of PyTorch's caching
+ * allocator; at least 64 KiB).  tgp_step_stats.h2d_bytes then counts the bytes it asked for, whether they were
+ * already resident or not; nothing is advised and nothing is evicted explicitly. */
+int  tgp_set_object_bytes(tgp_ctx *ctx, uint64_t bytes);
 /* Runtime monitor (Section IV-D): measured kernel times, one per op of the finished trace, in integer nanoseconds
  * (0 = not measured: that op keeps its analytic class).  With a time t the link test becomes mig / Bl > t, i.e. an
  * op is link-bound iff moving its pool bytes takes longer than the kernel ran; the next tgp_plan() uses it.

@@ -19,7 +19,7 @@ POOL_PINNED, POOL_MANAGED, POOL_PLAIN = 1, 2, 4
 T_READONLY, T_MUTABLE = 1, 2
 R, W = 1, 2
 PREFILL, DECODE = 0, 1
-VAR_EXPLICIT_RING, VAR_MANAGED_HINTS, VAR_MANAGED_DEMAND = 0, 1, 2
+VAR_EXPLICIT_RING, VAR_MANAGED_HINTS, VAR_MANAGED_DEMAND, VAR_MANAGED_OBJECT = 0, 1, 2, 3
 BIT_A, BIT_P, BIT_ZC = 1, 2, 4
 X_CLASSES, X_TENSORS, X_PINS, X_COMMANDS, X_TOTALS = range(5)
 # tensor kinds (TGP_K_*)
@@ -73,6 +73,7 @@ _SIGS = {
     "tgp_trace_export": [_P, _P, C.POINTER(_U64)],
     "tgp_set_budget": [_P, _U64],
     "tgp_set_variant": [_P, _U32, _U32],
+    "tgp_set_object_bytes": [_P, _U64],
     "tgp_set_measured_times": [_P, C.POINTER(_U64), _U64],
     "tgp_plan": [_P],
     "tgp_plan_export": [_P, _U32, _P, C.POINTER(_U64)],
@@ -229,6 +230,10 @@ class Ctx:
 
     def set_variant(self, variant, bits):
         self._ck(lib().tgp_set_variant(self._h, variant, bits), "tgp_set_variant")
+
+    def set_object_bytes(self, nbytes):
+        """Segment size of VAR_MANAGED_OBJECT, the object-level prefetcher."""
+        self._ck(lib().tgp_set_object_bytes(self._h, nbytes), "tgp_set_object_bytes")
 
     def set_measured_times(self, op_ns):
         """Per-op kernel times in integer ns (0 = keep the analytic class); None or empty clears the log."""

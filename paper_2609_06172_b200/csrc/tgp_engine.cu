@@ -63,6 +63,8 @@ struct TgpEngine {
     std::vector<uint64_t> tap_index;                     // 5 words per record: op, tag, sub-index, offset, bytes
     // managed-hints variant
     bool advised = false, evict_explicit = true;
+    uint64_t recent_objects[8] = {~0ull, ~0ull, ~0ull, ~0ull, ~0ull, ~0ull, ~0ull, ~0ull};      // object-level variant: last segments requested
+    uint32_t recent_pos = 0;
     std::map<int32_t, std::vector<uint32_t>> evict_at;   // op -> read-only ring tensors whose planned stay ends there
 };
 
@@ -222,6 +224,7 @@ int tgp_run_reset(tgp_ctx *ctx) {
     e->next_cmd = 0; e->next_step = 0; e->pos = 0; e->wb_pending = false; e->copy_waited_op = -1; e->tok_src = nullptr;
     e->evict_at.clear();
     e->advised = false;                                  // the plan may have changed since the last run
+    for (uint64_t &r : e->recent_objects) r = ~0ull;
     ctx->run_counts.clear();
     return TGP_OK;
 }
@@ -347,6 +350,30 @@ static int pump_managed(tgp_ctx *ctx, int32_t limit, cudaStream_t copy, uint32_t
     return TGP_OK;
 }
 
+// Object-level prefetch (the strawman of Section III-B): before op i runs, every whole segment of the pool that one of
+// its tensors overlaps is requested on the copy stream.  No events: a kernel that gets there first faults the pages
+// in itself, as under any managed-memory prefetcher.  A segment requested among the last eight is not requested again.
+static int prefetch_objects(tgp_ctx *ctx, uint32_t i, cudaStream_t copy, uint64_t *bytes) {
+    TgpEngine *e = ctx->eng;
+    const TgpOp &o = ctx->ops[i];
+    const uint64_t seg = ctx->object_bytes;
+    for (uint32_t k = 0; k < o.nacc; ++k) {
+        const TgpTensor &tt = ctx->tensors[ctx->acc[o.acc0 + k].tensor];
+        const TgpPool &p = ctx->pools[tt.pool];
+        for (uint64_t sgm = tt.off / seg; sgm <= (tt.off + tt.size - 1) / seg; ++sgm) {
+            const uint64_t key = ((uint64_t)tt.pool << 48) | sgm;
+            bool recent = false;
+            for (uint64_t r : e->recent_objects) recent |= r == key;
+            if (recent) continue;
+            const uint64_t lo = sgm * seg, len = std::min(seg, p.bytes - lo);
+            CU(ctx, cudaMemPrefetchAsync(p.host_base + lo, len, e->device, copy));
+            e->recent_objects[e->recent_pos++ % 8] = key;
+            *bytes += len;
+        }
+    }
+    return TGP_OK;
+}
+
 // after op i: record its completion if anything waits on it, and send home the read-only tensors released there
 static int after_op_managed(tgp_ctx *ctx, uint32_t i, cudaStream_t cs) {
     TgpEngine *e = ctx->eng;
@@ -445,8 +472,10 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
     const int32_t *tok = e->amax;
     if (tokens_host) { CU(ctx, cudaMemcpyAsync(e->tok, tokens_host, (size_t)M * 4, cudaMemcpyHostToDevice, cs)); tok = e->tok; }
     int rc;
-    const bool hints = ctx->variant == TGP_VAR_MANAGED_HINTS;
+    const bool hints = ctx->variant == TGP_VAR_MANAGED_HINTS, objects = ctx->variant == TGP_VAR_MANAGED_OBJECT;
+    uint64_t object_bytes_asked = 0;
     if (hints && (rc = advise_once(ctx))) return rc;
+    if (objects && (rc = prefetch_objects(ctx, st.op0, cp, &object_bytes_asked))) return rc;
     if (ring && (rc = pump(ctx, (int32_t)st.op0 - 1, cp, &n_cmds))) return rc;
     if (hints && (rc = pump_managed(ctx, (int32_t)st.op0 - 1, cp, &n_cmds))) return rc;
     const uint32_t qd = c.Hq * c.Dh, kd = c.Hkv * c.Dh;
@@ -593,6 +622,8 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
         } else if (hints) {
             if ((rc = after_op_managed(ctx, i, cs))) return rc;
             if ((rc = pump_managed(ctx, (int32_t)i, cp, &n_cmds))) return rc;
+        } else if (objects && i + 1 < st.op0 + st.nops) {
+            if ((rc = prefetch_objects(ctx, i + 1, cp, &object_bytes_asked))) return rc;
         }
     }
     e->pos += q_len;
@@ -603,7 +634,7 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
         CU(ctx, cudaEventSynchronize(e->t1));
         if (ring) CU(ctx, cudaStreamSynchronize(e->wb_stream));
         const uint64_t *tot = &ctx->plan.totals[(size_t)(e->next_step - 1) * 4];
-        stats->h2d_bytes = ring ? tot[0] : 0; stats->d2h_bytes = ring ? tot[1] : 0; stats->zc_bytes = tot[2];
+        stats->h2d_bytes = ring ? tot[0] : objects ? object_bytes_asked : 0; stats->d2h_bytes = ring ? tot[1] : 0; stats->zc_bytes = objects ? 0 : tot[2];
         stats->n_cmds = n_cmds; stats->n_launches = (uint32_t)(tgpk_launches - launches0); stats->n_mismatch = n_mismatch;
         CU(ctx, cudaEventElapsedTime(&stats->step_ms, e->t0, e->t1));
     }

@@ -231,8 +231,14 @@ int tgp_set_measured_times(tgp_ctx *ctx, const uint64_t *op_ns, uint64_t n_ops) 
 }
 
 int tgp_set_variant(tgp_ctx *ctx, uint32_t variant, uint32_t bits) {
-    if (!ctx || variant > TGP_VAR_MANAGED_DEMAND || (bits & ~7u)) return TGP_E_INVAL;
+    if (!ctx || variant > TGP_VAR_MANAGED_OBJECT || (bits & ~7u)) return TGP_E_INVAL;
     ctx->variant = variant; ctx->bits = bits; ctx->plan.valid = false;
+    return TGP_OK;
+}
+
+int tgp_set_object_bytes(tgp_ctx *ctx, uint64_t bytes) {
+    if (!ctx || bytes < (64u << 10)) return TGP_E_INVAL;
+    ctx->object_bytes = bytes;
     return TGP_OK;
 }
 

@@ -59,7 +59,7 @@ struct tgp_ctx {
     std::vector<tgp_access> acc;
     std::vector<TgpStep> steps;
     // policy inputs
-    uint64_t budget = 0;
+    uint64_t budget = 0, object_bytes = 20ull << 20;
     uint32_t variant = TGP_VAR_EXPLICIT_RING, bits = TGP_BIT_A | TGP_BIT_P | TGP_BIT_ZC;
     std::vector<uint64_t> measured_ns;                   // runtime monitor: kernel time per op in ns (0 = not measured), or empty
     TgpPlan plan;

@@ -27,7 +27,8 @@ class ManagedPool:
             self.ptr = 0
 
 
-def run(cfg, lay, machine, dev, fill, variants=(tb.VAR_MANAGED_DEMAND, tb.VAR_MANAGED_HINTS), decode_cap=16, slack=64 << 20, ballast=True):
+def run(cfg, lay, machine, dev, fill, variants=(tb.VAR_MANAGED_DEMAND, tb.VAR_MANAGED_HINTS), decode_cap=16, slack=64 << 20, ballast=True,
+        object_bytes=20 << 20):
     """Returns {variant name: {...}}.  `fill(layout, uint8 array)` writes the pool contents.  Capacity: the workspace
     and then a ballast tensor are allocated ONCE, before the GPU has touched the managed pool, so that budget + slack
     bytes of device memory are all the managed pages can ever occupy; both variants then run under that same cap
@@ -56,21 +57,27 @@ def run(cfg, lay, machine, dev, fill, variants=(tb.VAR_MANAGED_DEMAND, tb.VAR_MA
                     cap["ballast"] = f"not allocated: {ex}"
             cap["device_bytes_left_for_managed_pages"] = int(torch.cuda.mem_get_info(dev)[0])
         for var in variants:
-            name = "managed_demand" if var == tb.VAR_MANAGED_DEMAND else "managed_hints"
+            name = {tb.VAR_MANAGED_DEMAND: "managed_demand", tb.VAR_MANAGED_HINTS: "managed_hints", tb.VAR_MANAGED_OBJECT: "managed_object"}[var]
             s.plan(T=T, variant=var)
+            if var == tb.VAR_MANAGED_OBJECT:
+                s.ctx.set_object_bytes(object_bytes)
             info = {"decode_steps": T, **cap}
             times = []
             for rep in range(2):                          # first pass warms code paths; second is reported
                 tb.managed_evict(pool.ptr, lay.pool_bytes)
                 r.reset()
-                st = [r.step(tb.PREFILL, prompt, cfg.S, want_stats=True).step_ms]
+                st = [r.step(tb.PREFILL, prompt, cfg.S, want_stats=True)]
                 for _ in range(T):
-                    st.append(r.step(tb.DECODE, None, 1, want_stats=True).step_ms)
-                times = st
+                    st.append(r.step(tb.DECODE, None, 1, want_stats=True))
+                times = [x.step_ms for x in st]
+                asked = [int(x.h2d_bytes) for x in st]
             r.sync()
             info.update({"prefill_ms": times[0], "decode_ms_per_step": float(np.mean(times[1:])) if T else None,
                          "decode_tok_s": cfg.B * T / (sum(times[1:]) * 1e-3) if T else None,
                          "prefill_tok_s": cfg.B * cfg.S / (times[0] * 1e-3)})
+            if var == tb.VAR_MANAGED_OBJECT:                  # bytes the object-level prefetcher asked for (resident or not)
+                info.update({"object_bytes": int(object_bytes), "asked_bytes_prefill": asked[0],
+                             "asked_bytes_per_decode_step": float(np.mean(asked[1:])) if T else None})
             out[name] = info
         del hold
         s.close()

@@ -178,8 +178,9 @@ def test_config_2_prefill_and_first_decode_steps_match_oracle():
 
 
 def test_managed_variants_give_the_same_bits_as_the_explicit_ring():
-    """Same kernels reading a cudaMallocManaged pool in place (demand paging, and prefetch/advise hints):
-    only the placement mechanism differs, so logits must be bitwise equal to the explicit engine's."""
+    """Same kernels reading a cudaMallocManaged pool in place (demand paging, prefetch/advise hints, and the
+    object-level prefetcher that asks for whole segments): only the placement mechanism differs, so logits must be
+    bitwise equal to the explicit engine's."""
     from paper_2609_06172_b200 import uvm_baseline
     cfg = replace(si.CONFIGS[1], T=4)
     prompt = si.prompt_tokens(cfg)
@@ -190,14 +191,28 @@ def test_managed_variants_give_the_same_bits_as_the_explicit_ring():
     mp = uvm_baseline.ManagedPool(lay.pool_bytes)
     try:
         si.fill_pool(lay, mp.numpy())
-        for var in (tb.VAR_MANAGED_DEMAND, tb.VAR_MANAGED_HINTS):
+        for var in (tb.VAR_MANAGED_DEMAND, tb.VAR_MANAGED_HINTS, tb.VAR_MANAGED_OBJECT):
             sm = Session(lay, MACHINE, pool_base=mp.ptr, pool_flags=tb.POOL_MANAGED)
             sm.plan(T=T, variant=var)
+            if var == tb.VAR_MANAGED_OBJECT:
+                with pytest.raises(tb.TgpError):
+                    sm.ctx.set_object_bytes(4096)                             # below the 64 KiB minimum
+                sm.ctx.set_object_bytes(1 << 20)
             r = Runner(sm, cfg.B * cfg.S, arena=False)
             tb.managed_evict(mp.ptr, lay.pool_bytes)
             got, _ = r.generate(prompt, T, forced=forced)
             for a, b in zip(got, ref):
                 assert np.array_equal(a, b)
+            if var == tb.VAR_MANAGED_OBJECT:
+                # the prefetcher asks for whole 1 MiB segments: at least every touched byte, at most the pool per op
+                r.reset()
+                st = r.step(tb.PREFILL, np.ascontiguousarray(prompt, dtype=np.int32), cfg.S, want_stats=True)
+                from bench import parse_trace
+                acc = [a for o in parse_trace(sm.ctx.trace_export()) if o[0] == 0 for a in o[6]]
+                whole = sum(t.size for t in lay.tensors if t.kind not in (si.K_EMBED, si.K_KT, si.K_VT))      # read whole by a prefill
+                assert st.zc_bytes == 0 and st.d2h_bytes == 0
+                assert 0.9 * whole <= st.h2d_bytes <= sum(lay.tensors[a[0]].size + (2 << 20) for a in acc)
+                r.sync()
             # KV tiles were written in place: start from zeros again for the next variant
             sm.close()
             si.fill_pool(lay, mp.numpy())
