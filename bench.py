@@ -317,6 +317,7 @@ def main():
     ap.add_argument("--kernel-loop", choices=["decode", "prefill", "attention"], default=None,
                     help="only run the back-to-back weight-product loop of one step (small, for ncu captures)")
     ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--unseen-prompts", action="store_true", help="MoE: time prompts of another seed than the profile pass saw")
     ap.add_argument("--seq", type=int, default=None, help="with --kernel-loop attention: prompt length instead of the configuration's")
     ap.add_argument("--graph", action="store_true", help="replay the whole planned run as one CUDA graph (dense models; for host-bound tiny steps)")
     ap.add_argument("--layers", type=int, default=None, help="run the shape at reduced depth; a byte budget is scaled in proportion")
@@ -390,7 +391,10 @@ def main():
         r = Runner(s, cfg.B * cfg.S, device=str(dev))
     totals = np.frombuffer(blobs["totals"], dtype="<u8").reshape(-1, 4)
     ops = parse_trace(s.ctx.trace_export())
-    prompt_pinned = torch.from_numpy(si.prompt_tokens(cfg)).pin_memory()
+    # --unseen-prompts (MoE): the timed passes run prompts the profile pass never saw, so the plan's expert sets are a
+    # prediction; an expert the router picks outside its step's set is fetched synchronously and counted
+    run_cfg = replace(cfg, seed=cfg.seed ^ 0x5EED) if args.unseen_prompts else cfg
+    prompt_pinned = torch.from_numpy(si.prompt_tokens(run_cfg)).pin_memory()
     tok_pinned = torch.empty((cfg.B, 1), dtype=torch.int32).pin_memory()
     logits_host = torch.empty((cfg.B, cfg.V), dtype=torch.float32).pin_memory()
     T = cfg.T
@@ -480,6 +484,13 @@ def main():
             kind_n[key] = kind_n.get(key, 0) + 1
     s.ctx.set_op_timing(False)
     r.sync()
+    moe_prediction = None
+    if cfg.E:
+        ran = s.ctx.expert_counts(cfg.L, cfg.E)
+        n = min(len(ran), len(counts))
+        planned, used = np.asarray(counts[:n]) > 0, np.asarray(ran[:n]) > 0
+        moe_prediction = {"expert_slots_planned": int(planned.sum()), "planned_but_unused": int((planned & ~used).sum()),
+                          "used_but_unplanned": int((~planned & used).sum()), "slots": int(planned.size)}
 
     if rank != 0:
         if dist is not None:
@@ -569,7 +580,7 @@ def main():
            "prefill_tok_s": cfg.B * cfg.S / (step_ms[0] * 1e-3), "decode_tok_s": cfg.B * T / (sum(step_ms[1:]) * 1e-3) if T else None,
            "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": int(totals[:, 0].sum()) + cfg.B * (cfg.S + T) * 4,
                    "d2h_bytes_per_step": L_d2h + cfg.B * (T + 1) * 4 + cfg.B * cfg.V * 4},
-           "object_level_prefetch": object_level, "policy_bits": args.bits, "trace_mismatches": mismatches, "moe_profile_pass_s": profile_s,
+           "object_level_prefetch": object_level, "policy_bits": args.bits, "trace_mismatches": mismatches, "moe_profile_pass_s": profile_s, "unseen_prompts": bool(args.unseen_prompts), "moe_prediction": moe_prediction,
            "gpu_launches": launches * args.steps, "clocks": clocks, "roofline": roof, "step_roofline": step_roof,
            "kernels": {f"{k[0]}:{k[1]}": {"ms": round(v, 3), "launches": kind_n[k], "GBps": round(kind_bytes[k] / (v * 1e-3) / 1e9, 1),
                                            "TFLOPs": round(kind_flops[k] / (v * 1e-3) / 1e12, 2)} for k, v in sorted(kind_ms.items())}}

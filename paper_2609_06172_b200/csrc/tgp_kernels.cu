@@ -91,6 +91,12 @@ __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, c
         const bf16 *wrow[R];
 #pragma unroll
         for (int r = 0; r < R; ++r) wrow[r] = W + (size_t)min(row0 + r, n - 1) * K;   // tail rows re-read the last row, never stored
+        // the value this product is added to: lane r * MT + m fetches it as early as the protocol allows, so that its
+        // latency hides behind the weight stream instead of following it
+        float cprev = 0.f;
+        const bool mine = accumulate && lane < R * MT && row0 + lane / MT < n && lane % MT < Mrows;
+        const float *cptr = C + (size_t)(lane % MT) * ldc + col0 + row0 + lane / MT;
+        if (synced && mine) cprev = *cptr;
         for (uint32_t k0 = lane * 8; k0 < K; k0 += 256 * U) {
             uint4 wv[U][R];
 #pragma unroll
@@ -98,7 +104,7 @@ __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, c
 #pragma unroll
                 for (int r = 0; r < R; ++r)
                     wv[u][r] = (k0 + 256 * u < K) ? __ldcs(reinterpret_cast<const uint4 *>(wrow[r] + k0 + 256 * u)) : make_uint4(0, 0, 0, 0);
-            if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
+            if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; if (mine) cprev = *cptr; }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const uint32_t k = k0 + 256 * u;
@@ -116,17 +122,83 @@ __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, c
                 }
             }
         }
-        if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }      // K == 0 never happens; belt and braces
+        if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; if (mine) cprev = *cptr; }      // K == 0 never happens; belt and braces
 #pragma unroll
         for (int r = 0; r < R; ++r)
 #pragma unroll
             for (int m = 0; m < MT; ++m) {
                 const float s = warp_sum(acc[r][m]);
-                if (lane == 0 && row0 + r < n && m < (int)Mrows) {
-                    float *c = C + (size_t)m * ldc + col0 + row0 + r;
-                    *c = accumulate ? *c + s : s;
+                if ((int)lane == r * MT + m && row0 + r < n && m < (int)Mrows)
+                    C[(size_t)m * ldc + col0 + row0 + r] = accumulate ? cprev + s : s;
+            }
+    }
+}
+
+// Same product for blocks with few rows (n below two waves of warps): one CTA of 8 warps owns RB rows and its warps
+// split K in interleaved chunks of 256 elements, so n / RB CTAs spread over the SMs almost evenly where n warps of whole
+// rows leave a quarter of them with half the work.  The 8 partial sums of a row meet in shared memory and are added in
+// warp order: deterministic.  Same dependent-launch protocol.
+template <int MT, int RB, int U>
+__global__ void __launch_bounds__(256) gemv_splitk_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+                                                          uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
+    __shared__ float part[8][RB * MT];
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    bool synced = false;
+    for (uint32_t row0 = blockIdx.x * RB; row0 < n; row0 += gridDim.x * RB) {
+        float acc[RB][MT];
+#pragma unroll
+        for (int r = 0; r < RB; ++r)
+#pragma unroll
+            for (int m = 0; m < MT; ++m) acc[r][m] = 0.f;
+        const bf16 *wrow[RB];
+#pragma unroll
+        for (int r = 0; r < RB; ++r) wrow[r] = W + (size_t)min(row0 + r, n - 1) * K;
+        float cprev = 0.f;
+        const bool mine = threadIdx.x < RB * MT && row0 + threadIdx.x / MT < n && threadIdx.x % MT < Mrows;
+        const float *cptr = C + (size_t)(threadIdx.x % MT) * ldc + col0 + row0 + threadIdx.x / MT;
+        if (synced && mine && accumulate) cprev = *cptr;
+        for (uint32_t k0 = warp * 256 + lane * 8; k0 < K; k0 += 2048 * U) {
+            uint4 wv[U][RB];
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int r = 0; r < RB; ++r)
+                    wv[u][r] = (k0 + 2048 * u < K) ? __ldcs(reinterpret_cast<const uint4 *>(wrow[r] + k0 + 2048 * u)) : make_uint4(0, 0, 0, 0);
+            if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; if (mine && accumulate) cprev = *cptr; }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t k = k0 + 2048 * u;
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    float xf[8];
+                    unpack8((k < K && m < (int)Mrows) ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)) : make_uint4(0, 0, 0, 0), xf);
+#pragma unroll
+                    for (int r = 0; r < RB; ++r) {
+                        float wf[8];
+                        unpack8(wv[u][r], wf);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) acc[r][m] = fmaf(wf[i], xf[i], acc[r][m]);
+                    }
                 }
             }
+        }
+        if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; if (mine && accumulate) cprev = *cptr; }     // a warp whose K slice is empty
+#pragma unroll
+        for (int r = 0; r < RB; ++r)
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                const float sacc = warp_sum(acc[r][m]);
+                if (lane == 0) part[warp][r * MT + m] = sacc;
+            }
+        __syncthreads();
+        if (mine) {
+            float t = 0.f;
+#pragma unroll
+            for (int w = 0; w < 8; ++w) t += part[w][threadIdx.x];
+            C[(size_t)(threadIdx.x % MT) * ldc + col0 + row0 + threadIdx.x / MT] = accumulate ? cprev + t : t;
+        }
+        __syncthreads();
     }
 }
 
@@ -718,10 +790,39 @@ static void launch_gemv_mma(const bf16 *A, const bf16 *W, float *C, uint32_t Mro
 }
 
 // rows per warp: fewer when the block has few rows, so that every SM still gets warps
+template <int MT, int RB, int U>
+static void launch_gemv_splitk(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int acc, cudaStream_t st) {
+    static int blocks_per_sm = 0, sms = 0;
+    if (!blocks_per_sm) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, gemv_splitk_kernel<MT, RB, U>, 256, 0) != cudaSuccess || blocks_per_sm < 1) blocks_per_sm = 1;
+        if (sms < 1) sms = 148;
+    }
+    uint32_t need = (n + RB - 1) / RB, full = (uint32_t)(sms * blocks_per_sm);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(need < full ? need : full);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = g_gemv_pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, gemv_splitk_kernel<MT, RB, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
+}
+
+static int g_gemv_splitk = 1;    // small-n blocks at M <= 2: CTA per RB rows with K split over its warps (0: one warp per row)
+
 template <int MT>
 static void launch_gemv_rows(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int acc, cudaStream_t st) {
     if constexpr (MT <= 2) {
         if (n >= 2 * 148 * 16) return launch_gemv<MT, 2, 4>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
+        if (g_gemv_splitk && K >= 8192) {                    // at least four 256-element chunks per warp and row
+            if (n <= 1024) return launch_gemv_splitk<MT, 1, 4>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
+            return launch_gemv_splitk<MT, 2, 4>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
+        }
         return launch_gemv<MT, 1, 8>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
     } else {
         if (n >= 2 * 148 * 16) return launch_gemv<MT, 2, 2>(A, W, C, Mrows, n, K, ldc, col0, acc, st);

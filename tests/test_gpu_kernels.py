@@ -43,7 +43,10 @@ def bf16_close(got_f32, want_f32, frac=0.01):
 @pytest.mark.parametrize("M,n,K", [(1, 300, 256), (1, 4096, 2048), (2, 129, 64), (3, 1000, 512), (8, 1030, 512),
                                    (13, 77, 128), (16, 260, 1024), (17, 64, 96), (33, 130, 96), (200, 260, 1024),
                                    (64, 64, 32), (1, 1, 8), (70, 5, 8), (129, 257, 72), (300, 520, 1096), (512, 2048, 2048),
-                                   (1000, 136, 8192)])
+                                   (1000, 136, 8192),
+                                   # few rows, long K at M <= 2: the split-K GEMV (two rows per CTA; one row per CTA up to 1024 rows),
+                                   # odd row counts, K not a multiple of the 256-element chunk, more CTAs than resident slots
+                                   (1, 2048, 8192), (2, 2051, 8200), (1, 513, 8192), (2, 1, 16384), (1, 4735, 8192)])
 @pytest.mark.parametrize("accumulate", [0, 1])
 def test_gemm_matches_oracle(M, n, K, accumulate):
     a_bits, w_bits = rnd_bits(1, M * K).reshape(M, K), rnd_bits(2, n * K).reshape(n, K)
@@ -257,6 +260,41 @@ def test_tensor_core_prefill_attention_with_growing_scores(Dh):
         assert np.isfinite(got).all()
         assert np.abs(got - att).max() < 2.0 ** -6 * np.abs(att).max() + 1e-6
         assert np.mean(np.abs(got - bf16_round(att))) < 4e-3 * np.abs(att).mean()
+    tb.k_attn_select(0)
+    assert tb.k_attn_status() == 0
+
+
+@pytest.mark.parametrize("Dh,TK", [(128, 64), (64, 128)])
+def test_tensor_core_prefill_attention_of_a_later_chunk(Dh, TK):
+    """A prompt processed in two chunks: the second chunk's queries start at position 192 and see the first chunk's keys
+    unmasked plus their own causally.  Both tensor-core kernels against the oracle."""
+    B, Hq, Hkv, P0, Q2 = 2, 4, 2, 192, 200
+    S = P0 + Q2
+    cfg = replace(KCFG, Dh=Dh, Hq=Hq, Hkv=Hkv, TK=TK, S=S, T=0, B=B, d=Hq * Dh)
+    mc = model_cfg(cfg)
+    o = OracleModel(cfg, {(k, 0, -1): rnd_bits(k, 8).reshape(1, 8) for k in range(13)})
+    rng = np.random.default_rng(7 * Dh + TK)
+    k32 = bf16_round(rng.standard_normal((B, Hkv, S, Dh)).astype(np.float32))
+    v32 = bf16_round(rng.standard_normal((B, Hkv, S, Dh)).astype(np.float32))
+    q32 = bf16_round(rng.standard_normal((B, Q2, Hq, Dh)).astype(np.float32))
+    kt, vt = make_tiles(cfg, B)
+    for t in range(cfg.n_tiles):
+        lo, hi = t * TK, min(S, (t + 1) * TK)
+        if lo < hi:
+            kt[t].view(B, Hkv, TK, Dh)[:, :, :hi - lo].copy_(torch.from_numpy(k32[:, :, lo:hi]).to(DEV))
+            vt[t].view(B, Hkv, TK, Dh)[:, :, :hi - lo].copy_(torch.from_numpy(v32[:, :, lo:hi]).to(DEV))
+    o.K[0, :, :, :S] = k32
+    o.V[0, :, :, :S] = v32
+    att = o.attention(0, q32, P0)
+    qb = torch.from_numpy(q32.reshape(B * Q2, Hq * Dh)).to(DEV).bfloat16()
+    for impl in (3, 2):
+        tb.k_attn_select(impl)
+        ob = torch.zeros(B * Q2, Hq * Dh, dtype=torch.bfloat16, device=DEV)
+        tb.k_attn(qb, kt, vt, ob, mc, B, Q2, P0, None)
+        torch.cuda.synchronize()
+        got = ob.float().cpu().numpy().reshape(B, Q2, Hq, Dh)
+        assert np.abs(got - att).max() < 2.0 ** -7 * np.abs(att).max() + 1e-6
+        assert np.mean(np.abs(got - bf16_round(att))) < 3e-3 * np.abs(att).mean()
     tb.k_attn_select(0)
     assert tb.k_attn_status() == 0
 
