@@ -675,6 +675,7 @@ int tgpk_rmsnorm(const float *x, uint32_t ldx, const void *g, void *h, uint32_t 
     return TGP_OK;
 }
 
+static int g_gemv_rows8 = 1;     // skinny products of few rows and long K: 8-row CTAs (0: always 16)
 static int g_gemv_pdl = 1;       // consecutive weight-streaming launches may overlap (programmatic dependent launch)
 
 template <int MT, int R, int U>
@@ -700,33 +701,34 @@ static void launch_gemv(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, 
     cudaLaunchKernelEx(&cfg, gemv_kernel<MT, R, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
 }
 
-// Same product for blocks with few rows: one CTA owns 16 rows of W and its NW (8 or 16) warps split K (interleaved
-// chunks of 32*U), so n/16 CTAs of NW warps fill the machine where n/16 warps would not.  The partial tiles meet in
-// shared memory and are summed in warp order: deterministic.
-template <int NB, int U, int NW>
+// Same product for blocks with few rows: one CTA owns ROWS (16, or 8 with the upper half of the MMA tile left empty)
+// rows of W and its NW (8 or 16) warps split K (interleaved chunks of 32*U), so n/ROWS CTAs of NW warps fill the machine
+// where n/16 warps would not.  The partial tiles meet in shared memory and are summed in warp order: deterministic.
+template <int NB, int U, int NW, int ROWS>
 __global__ void __launch_bounds__(NW * 32) gemv_mma_splitk_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                               uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
+    constexpr int UL = ROWS == 8 ? 2 * U : U;             // half a tile per load step: twice the steps in flight
     __shared__ float part[NW][NB * 4][32];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, c = lane & 3;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     bool synced = false;
-    for (uint32_t row0 = blockIdx.x * 16; row0 < n; row0 += gridDim.x * 16) {
+    for (uint32_t row0 = blockIdx.x * ROWS; row0 < n; row0 += gridDim.x * ROWS) {
         const bf16 *wlo = W + (size_t)min(row0 + g, n - 1) * K + c * 8;
         const bf16 *whi = W + (size_t)min(row0 + g + 8, n - 1) * K + c * 8;
         float acc[NB][4];
 #pragma unroll
         for (int b = 0; b < NB; ++b) { acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f; }
-        for (uint32_t k0 = warp * 32 * U; k0 < K; k0 += NW * 32 * U) {
-            uint4 lo[U], hi[U];
+        for (uint32_t k0 = warp * 32 * UL; k0 < K; k0 += NW * 32 * UL) {
+            uint4 lo[UL], hi[UL];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
+            for (int u = 0; u < UL; ++u) {
                 const bool in = k0 + 32 * u < K;
                 lo[u] = in ? __ldcs(reinterpret_cast<const uint4 *>(wlo + k0 + 32 * u)) : make_uint4(0, 0, 0, 0);
-                hi[u] = in ? __ldcs(reinterpret_cast<const uint4 *>(whi + k0 + 32 * u)) : make_uint4(0, 0, 0, 0);
+                hi[u] = (in && ROWS == 16) ? __ldcs(reinterpret_cast<const uint4 *>(whi + k0 + 32 * u)) : make_uint4(0, 0, 0, 0);   // ROWS == 8: the upper half of the tile stays empty
             }
             if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
+            for (int u = 0; u < UL; ++u) {
                 const uint32_t k = k0 + 32 * u;
 #pragma unroll
                 for (int b = 0; b < NB; ++b) {
@@ -749,7 +751,7 @@ __global__ void __launch_bounds__(NW * 32) gemv_mma_splitk_kernel(const bf16 *__
 #pragma unroll
             for (int w = 0; w < NW; ++w) sum += part[w][slot][ln];
             const uint32_t m = b * 8 + 2 * (ln & 3) + (i & 1), row = row0 + (ln >> 2) + 8 * (i >> 1);
-            if (m < Mrows && row < n) {
+            if (m < Mrows && row < n && (ROWS == 16 || (i >> 1) == 0)) {
                 float *p = C + (size_t)m * ldc + col0 + row;
                 *p = accumulate ? *p + sum : sum;
             }
@@ -769,11 +771,14 @@ static void launch_gemv_mma(const bf16 *A, const bf16 *W, float *C, uint32_t Mro
         if (sms < 1) sms = 148;
     }
     static int blocks_per_sm_split = 0;
-    if (!blocks_per_sm_split && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm_split, gemv_mma_splitk_kernel<NB, U, 8>, 256, 0) != cudaSuccess || blocks_per_sm_split < 1))
+    if (!blocks_per_sm_split && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm_split, gemv_mma_splitk_kernel<NB, U, 8, 16>, 256, 0) != cudaSuccess || blocks_per_sm_split < 1))
         blocks_per_sm_split = 1;
     const bool split = n < 16u * 8u * (uint32_t)sms;                 // too few 16-row groups to give every SM eight warps
-    const bool wide = split && (n + 15) / 16 < (uint32_t)sms;        // fewer 16-row groups than SMs: 16 warps per CTA
-    uint32_t need = split ? (n + 15) / 16 : (n + 16 * 8 - 1) / (16 * 8);
+    const bool wide = split && (n + 15) / 16 < 2u * (uint32_t)sms;   // fewer than two 16-row groups per SM: 16 warps per CTA
+    // 16-row groups for at most half the SMs and a K long enough to keep all 16 warps loading: 8 rows per CTA, twice the
+    // CTAs (each CTA reads its slice of the activations whatever its rows, so fewer rows per CTA cost L2 traffic)
+    const bool half = wide && g_gemv_rows8 && 2 * ((n + 15) / 16) <= (uint32_t)sms && K >= 16u * 32u * 2u * U;
+    uint32_t need = split ? (half ? (n + 7) / 8 : (n + 15) / 16) : (n + 16 * 8 - 1) / (16 * 8);
     uint32_t full = (uint32_t)(sms * (split ? blocks_per_sm_split : blocks_per_sm));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(need < full ? need : full);
@@ -784,12 +789,13 @@ static void launch_gemv_mma(const bf16 *A, const bf16 *W, float *C, uint32_t Mro
     attr[0].val.programmaticStreamSerializationAllowed = g_gemv_pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (wide) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16>, A, W, C, Mrows, n, K, ldc, col0, acc);
-    else if (split) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 8>, A, W, C, Mrows, n, K, ldc, col0, acc);
+    if (wide && half) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 8>, A, W, C, Mrows, n, K, ldc, col0, acc);
+    else if (wide) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 16>, A, W, C, Mrows, n, K, ldc, col0, acc);
+    else if (half) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 8, 8>, A, W, C, Mrows, n, K, ldc, col0, acc);
+    else if (split) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 8, 16>, A, W, C, Mrows, n, K, ldc, col0, acc);
     else cudaLaunchKernelEx(&cfg, gemv_mma_kernel<NB, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
 }
 
-// rows per warp: fewer when the block has few rows, so that every SM still gets warps
 template <int MT, int RB, int U>
 static void launch_gemv_splitk(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int acc, cudaStream_t st) {
     static int blocks_per_sm = 0, sms = 0;
@@ -815,6 +821,7 @@ static void launch_gemv_splitk(const bf16 *A, const bf16 *W, float *C, uint32_t 
 
 static int g_gemv_splitk = 1;    // small-n blocks at M <= 2: CTA per RB rows with K split over its warps (0: one warp per row)
 
+// rows per warp: fewer when the block has few rows, so that every SM still gets warps
 template <int MT>
 static void launch_gemv_rows(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int acc, cudaStream_t st) {
     if constexpr (MT <= 2) {
@@ -838,9 +845,13 @@ int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, ui
     if (K % 8 || !K) return TGP_E_INVAL;
     const bf16 *a = (const bf16 *)A, *w = (const bf16 *)W;
     if (M >= 3 && M <= 32 && K % 32 == 0 && g_skinny_impl == 0) {
-        if (M <= 8) launch_gemv_mma<1, 4>(a, w, C, M, n, K, ldc, col0, accumulate, st);
-        else if (M <= 16) launch_gemv_mma<2, 4>(a, w, C, M, n, K, ldc, col0, accumulate, st);
-        else launch_gemv_mma<4, 2>(a, w, C, M, n, K, ldc, col0, accumulate, st);
+        // fewer 16-row groups than SMs: few CTAs, so each warp keeps twice the loads in flight
+        static int sms = 0;
+        if (!sms) { int dev = 0; cudaGetDevice(&dev); if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148; }
+        const bool few = (n + 15) / 16 < (uint32_t)sms;
+        if (M <= 8) { if (few) launch_gemv_mma<1, 8>(a, w, C, M, n, K, ldc, col0, accumulate, st); else launch_gemv_mma<1, 4>(a, w, C, M, n, K, ldc, col0, accumulate, st); }
+        else if (M <= 16) { if (few) launch_gemv_mma<2, 8>(a, w, C, M, n, K, ldc, col0, accumulate, st); else launch_gemv_mma<2, 4>(a, w, C, M, n, K, ldc, col0, accumulate, st); }
+        else { if (few) launch_gemv_mma<4, 4>(a, w, C, M, n, K, ldc, col0, accumulate, st); else launch_gemv_mma<4, 2>(a, w, C, M, n, K, ldc, col0, accumulate, st); }
     } else if (M <= 16) {
         for (uint32_t m0 = 0; m0 < M; m0 += 8) {
             uint32_t mr = M - m0 < 8 ? M - m0 : 8;

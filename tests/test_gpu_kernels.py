@@ -363,7 +363,10 @@ def test_overlapping_gemv_launches_keep_their_dependencies():
 
 
 @pytest.mark.parametrize("M,n,K", [(3, 100, 64), (8, 4096, 4096), (8, 1030, 512), (13, 77, 128), (16, 260, 1024), (17, 64, 96), (24, 2049, 2048),
-                                   (32, 4100, 8192), (5, 16, 32)])
+                                   (32, 4100, 8192), (5, 16, 32),
+                                   # few rows and long K: K split over a thread-block cluster of 8, 4, 2 CTAs (ragged rows, K that leaves
+                                   # the last ranks without a chunk)
+                                   (8, 1152, 14336), (5, 650, 14368), (16, 1024, 4096), (9, 24, 2080), (8, 16, 16384)])
 @pytest.mark.parametrize("accumulate", [0, 1])
 def test_skinny_tensor_core_gemv_matches_oracle_and_cuda_core_path(M, n, K, accumulate):
     a_bits, w_bits = rnd_bits(41, M * K).reshape(M, K), rnd_bits(42, n * K).reshape(n, K)
