@@ -114,116 +114,112 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 64, tmem_P = tmem_base + 192;     // P: two buffers of 32 columns (bf16 pairs)
     auto give_up = [&](int code) { if (!*failed) { *failed = 1; atomicCAS(&g_attn_tc_error, 0, code); } };
-    // registers move from the second warpgroup (three single-thread roles) to the softmax warpgroup: 128 * 48 + 128 * 208
-    // is the 128 per thread the CTA was launched with
-
-
     // Registers move from the second warpgroup (three single-thread roles and an idle warp) to the softmax warpgroup:
     // 128 * 64 + 128 * 192 is the 128 per thread the CTA is launched with.
     if (warp >= 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;" ::: "memory");
-    if (warp == 5) {
-        // ======================= producer: every TMA load (lane 0) =======================
-        uint32_t nk = 0, nv = 0;                             // K / V blocks requested so far (block i uses stage i & 1)
-        if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmQ) : "memory");
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmKV) : "memory");
-            const uint32_t head_row = (b * a.Hkv + hk) * a.TK;
-            uint32_t k_tile = 0, k_off = 0, v_tile = 0, v_off = 0;           // tile and key offset inside it of the next block
-            auto load_kv = [&](uint8_t *dst, int y, uint64_t *bar, uint32_t more_bytes) {
-                mbar_expect_tx(bar, KV_BYTES + more_bytes);
-#pragma unroll
-                for (uint32_t kb = 0; kb < KB; ++kb) tma_load_2d(dst + kb * (BKV * 128), &tmKV, kb * 64, y, bar);
-            };
-            auto next_k = [&](uint32_t more_bytes) {
-                load_kv(Ks + (nk & 1) * KV_BYTES, a.krow[k_tile] + (int)(head_row + k_off), bar_k + (nk & 1), more_bytes);
-                nk += 1;
-                if ((k_off += BKV) == a.TK) { k_off = 0; k_tile += 1; }
-            };
-            auto next_v = [&]() {
-                load_kv(Vs + (nv & 1) * KV_BYTES, a.vrow[v_tile] + (int)(head_row + v_off), bar_v + (nv & 1), 0);
-                nv += 1;
-                if ((v_off += BKV) == a.TK) { v_off = 0; v_tile += 1; }
-            };
-            next_k(Q_BYTES);
-#pragma unroll
-            for (uint32_t kb = 0; kb < KB; ++kb) tma_load_2d(Qs + kb * (BQ * 128), &tmQ, hq * DH + kb * 64, b * a.q_len + q0, bar_k);
-            if (1 < nblk) next_k(0);
-            next_v();
-            for (uint32_t jb = 0; jb + 1 < nblk; ++jb) {
-                const uint32_t st = jb & 1;
-                if (jb + 2 < nblk) {                                         // K_jb+2 goes where K_jb is, once S_jb is complete
-                    if (!mbar_wait(bar_kfree + st, (jb >> 1) & 1, failed)) { give_up(1); break; }
-                    next_k(0);
-                }
-                if (jb >= 1 && !mbar_wait(bar_o + (st ^ 1), ((jb - 1) >> 1) & 1, failed)) { give_up(2); break; }   // V_jb+1 goes where V_jb-1 is
-                next_v();
-            }
-            // every load requested must have landed before the CTA may exit (bounded; `never` is never set)
-            volatile uint32_t *never = failed + 1;
-            for (uint32_t st = 0; st < 2; ++st) {
-                const uint32_t ck = (nk + 1 - st) >> 1, cv = (nv + 1 - st) >> 1;     // loads requested into this stage
-                if (ck) mbar_wait(bar_k + st, (ck - 1) & 1, never);
-                if (cv) mbar_wait(bar_v + st, (cv - 1) & 1, never);
-            }
-        }
-    } else if (warp == 4) {
-        // ======================= S warp: lane 0 issues S_j = Q K_j^T =======================
-        constexpr uint32_t idesc_s = umma_idesc(BKV);
-        auto wait = [&](uint64_t *bar, uint32_t parity, int code) {
-            bool ok = mbar_wait(bar, parity, failed);
-            if (!ok) give_up(code);
-            return __all_sync(0xffffffffu, ok);
-        };
-        for (uint32_t jb = 0; jb < nblk; ++jb) {
-            if (jb >= 1 && !wait(bar_sfree, (jb - 1) & 1, 4)) break;         // S_jb-1 is in registers
-            if (!wait(bar_k + (jb & 1), (jb >> 1) & 1, 3)) break;            // K_jb (and Q with K_0) has landed
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 64;" ::: "memory");
+        if (warp == 5) {
+            // ======================= producer: every TMA load (lane 0) =======================
+            uint32_t nk = 0, nv = 0;                             // K / V blocks requested so far (block i uses stage i & 1)
             if (lane == 0) {
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint8_t *Kj = Ks + (jb & 1) * KV_BYTES;
-#pragma unroll
-                for (uint32_t kb = 0; kb < KB; ++kb) {
-                    const uint64_t dq = umma_desc(smem_u32(Qs + kb * (BQ * 128))), dk = umma_desc(smem_u32(Kj + kb * (BKV * 128)));
-#pragma unroll
-                    for (uint32_t k = 0; k < 4; ++k) umma(tmem_S, dq + 2 * k, dk + 2 * k, idesc_s, (kb | k) != 0);
+                asm volatile("prefetch.tensormap [%0];" ::"l"(&tmQ) : "memory");
+                asm volatile("prefetch.tensormap [%0];" ::"l"(&tmKV) : "memory");
+                const uint32_t head_row = (b * a.Hkv + hk) * a.TK;
+                uint32_t k_tile = 0, k_off = 0, v_tile = 0, v_off = 0;           // tile and key offset inside it of the next block
+                auto load_kv = [&](uint8_t *dst, int y, uint64_t *bar, uint32_t more_bytes) {
+                    mbar_expect_tx(bar, KV_BYTES + more_bytes);
+    #pragma unroll
+                    for (uint32_t kb = 0; kb < KB; ++kb) tma_load_2d(dst + kb * (BKV * 128), &tmKV, kb * 64, y, bar);
+                };
+                auto next_k = [&](uint32_t more_bytes) {
+                    load_kv(Ks + (nk & 1) * KV_BYTES, a.krow[k_tile] + (int)(head_row + k_off), bar_k + (nk & 1), more_bytes);
+                    nk += 1;
+                    if ((k_off += BKV) == a.TK) { k_off = 0; k_tile += 1; }
+                };
+                auto next_v = [&]() {
+                    load_kv(Vs + (nv & 1) * KV_BYTES, a.vrow[v_tile] + (int)(head_row + v_off), bar_v + (nv & 1), 0);
+                    nv += 1;
+                    if ((v_off += BKV) == a.TK) { v_off = 0; v_tile += 1; }
+                };
+                next_k(Q_BYTES);
+    #pragma unroll
+                for (uint32_t kb = 0; kb < KB; ++kb) tma_load_2d(Qs + kb * (BQ * 128), &tmQ, hq * DH + kb * 64, b * a.q_len + q0, bar_k);
+                if (1 < nblk) next_k(0);
+                next_v();
+                for (uint32_t jb = 0; jb + 1 < nblk; ++jb) {
+                    const uint32_t st = jb & 1;
+                    if (jb + 2 < nblk) {                                         // K_jb+2 goes where K_jb is, once S_jb is complete
+                        if (!mbar_wait(bar_kfree + st, (jb >> 1) & 1, failed)) { give_up(1); break; }
+                        next_k(0);
+                    }
+                    if (jb >= 1 && !mbar_wait(bar_o + (st ^ 1), ((jb - 1) >> 1) & 1, failed)) { give_up(2); break; }   // V_jb+1 goes where V_jb-1 is
+                    next_v();
                 }
-                umma_commit(bar_s);
-                umma_commit(bar_kfree + (jb & 1));                           // its completion also frees the K stage
+                // every load requested must have landed before the CTA may exit (bounded; `never` is never set)
+                volatile uint32_t *never = failed + 1;
+                for (uint32_t st = 0; st < 2; ++st) {
+                    const uint32_t ck = (nk + 1 - st) >> 1, cv = (nv + 1 - st) >> 1;     // loads requested into this stage
+                    if (ck) mbar_wait(bar_k + st, (ck - 1) & 1, never);
+                    if (cv) mbar_wait(bar_v + st, (cv - 1) & 1, never);
+                }
             }
-            __syncwarp();
-        }
-    } else if (warp == 6) {
-        // ======================= P V warp: lane 0 issues O += P_j V_j =======================
-        constexpr uint32_t idesc_o = umma_idesc(DH) | (1u << 16);           // bit 16: B operand is MN-major
-        auto wait = [&](uint64_t *bar, uint32_t parity, int code) {
-            bool ok = mbar_wait(bar, parity, failed);
-            if (!ok) give_up(code);
-            return __all_sync(0xffffffffu, ok);
-        };
-        for (uint32_t jb = 0; jb < nblk; ++jb) {
-            const uint32_t st = jb & 1;
-            if (!wait(bar_p + st, (jb >> 1) & 1, 4)) break;
-            if (!wait(bar_v + st, (jb >> 1) & 1, 3)) break;
-            if (jb * BKV + BKV > kvlen) {                                    // rows past the sequence: whatever the tile holds there
-                const uint32_t valid = kvlen - jb * BKV;
-                for (uint32_t i = lane; i < (BKV - valid) * KB * 8; i += 32) {
-                    const uint32_t r = valid + i / (KB * 8), kb = (i / 8) % KB, c = i % 8;
-                    *reinterpret_cast<uint4 *>(Vs + st * KV_BYTES + kb * (BKV * 128) + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+        } else if (warp == 4) {
+            // ======================= S warp: lane 0 issues S_j = Q K_j^T =======================
+            constexpr uint32_t idesc_s = umma_idesc(BKV);
+            auto wait = [&](uint64_t *bar, uint32_t parity, int code) {
+                bool ok = mbar_wait(bar, parity, failed);
+                if (!ok) give_up(code);
+                return __all_sync(0xffffffffu, ok);
+            };
+            for (uint32_t jb = 0; jb < nblk; ++jb) {
+                if (jb >= 1 && !wait(bar_sfree, (jb - 1) & 1, 4)) break;         // S_jb-1 is in registers
+                if (!wait(bar_k + (jb & 1), (jb >> 1) & 1, 3)) break;            // K_jb (and Q with K_0) has landed
+                if (lane == 0) {
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint8_t *Kj = Ks + (jb & 1) * KV_BYTES;
+    #pragma unroll
+                    for (uint32_t kb = 0; kb < KB; ++kb) {
+                        const uint64_t dq = umma_desc(smem_u32(Qs + kb * (BQ * 128))), dk = umma_desc(smem_u32(Kj + kb * (BKV * 128)));
+    #pragma unroll
+                        for (uint32_t k = 0; k < 4; ++k) umma(tmem_S, dq + 2 * k, dk + 2 * k, idesc_s, (kb | k) != 0);
+                    }
+                    umma_commit(bar_s);
+                    umma_commit(bar_kfree + (jb & 1));                           // its completion also frees the K stage
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
             }
-            if (lane == 0) {
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint64_t dv = umma_desc_mn(smem_u32(Vs + st * KV_BYTES), BKV * 128);
-#pragma unroll
-                for (uint32_t k = 0; k < 4; ++k)                             // 16 keys per step: 8 columns of P, 2048 B of V rows
-                    umma_ts(tmem_O, tmem_P + st * 32 + 8 * k, dv + 128 * k, idesc_o, (jb | k) != 0);
-                umma_commit(bar_o + st);
+        } else if (warp == 6) {
+            // ======================= P V warp: lane 0 issues O += P_j V_j =======================
+            constexpr uint32_t idesc_o = umma_idesc(DH) | (1u << 16);           // bit 16: B operand is MN-major
+            auto wait = [&](uint64_t *bar, uint32_t parity, int code) {
+                bool ok = mbar_wait(bar, parity, failed);
+                if (!ok) give_up(code);
+                return __all_sync(0xffffffffu, ok);
+            };
+            for (uint32_t jb = 0; jb < nblk; ++jb) {
+                const uint32_t st = jb & 1;
+                if (!wait(bar_p + st, (jb >> 1) & 1, 4)) break;
+                if (!wait(bar_v + st, (jb >> 1) & 1, 3)) break;
+                if (jb * BKV + BKV > kvlen) {                                    // rows past the sequence: whatever the tile holds there
+                    const uint32_t valid = kvlen - jb * BKV;
+                    for (uint32_t i = lane; i < (BKV - valid) * KB * 8; i += 32) {
+                        const uint32_t r = valid + i / (KB * 8), kb = (i / 8) % KB, c = i % 8;
+                        *reinterpret_cast<uint4 *>(Vs + st * KV_BYTES + kb * (BKV * 128) + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                }
+                if (lane == 0) {
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint64_t dv = umma_desc_mn(smem_u32(Vs + st * KV_BYTES), BKV * 128);
+    #pragma unroll
+                    for (uint32_t k = 0; k < 4; ++k)                             // 16 keys per step: 8 columns of P, 2048 B of V rows
+                        umma_ts(tmem_O, tmem_P + st * 32 + 8 * k, dv + 128 * k, idesc_o, (jb | k) != 0);
+                    umma_commit(bar_o + st);
+                }
+                __syncwarp();
             }
-            __syncwarp();
         }
-    }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 192;" ::: "memory");
         // ======================= softmax warps: thread = query row = TMEM lane =======================
