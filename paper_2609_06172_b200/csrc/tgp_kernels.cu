@@ -485,6 +485,132 @@ __global__ void attn_decode_partial_kernel(AttnArgs a, uint32_t SPLIT) {
 }
 
 // Merge the per-tile partials of one (batch, query head): grid (Hq, B), DH threads.
+// Decode attention over one KV tile for all G query heads of a KV head at once (G = Hq / Hkv in {1, 2, 4, 8}): the tile's
+// K and V rows are read once, not once per query head.  One CTA per (tile, KV head, sequence); warp w walks the keys
+// w*32, (w + SPLIT)*32, ... of the tile in chunks of 32: lane = key for the scores (the lane reads its whole K row with
+// 16-byte loads, all in flight at once, and dots it with the G queries held in shared memory), then lane = DH/32
+// consecutive output dimensions for P V (each V row is one coalesced warp load; the G weights of a key come by
+// shuffle).  Per-warp online softmax; the SPLIT partials of a head are merged in warp order; output as in the
+// per-head kernel: (max, sum, unnormalised o[DH]) per (sequence, head, tile) for attn_decode_merge_kernel.
+template <int DH, int G>
+__global__ void __launch_bounds__(256) attn_decode_group_kernel(AttnArgs a, uint32_t SPLIT) {
+    extern __shared__ float dsm[];
+    constexpr int DPL = DH / 32;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t tile = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+    const uint32_t kvlen = a.pos0 + 1;
+    const uint32_t nk = min(a.TK, kvlen - tile * a.TK);
+    float *qs = dsm;                                        // [G][DH] query rows as fp32
+    float *parts = dsm + G * DH;                            // [G][SPLIT][DH + 2]
+    {
+        const bf16 *q = a.qb + ((size_t)b * a.Hq + hk * G) * DH;          // the G heads of this group are contiguous
+        for (uint32_t i = threadIdx.x; i < G * DH; i += blockDim.x) qs[i] = __bfloat162float(q[i]);
+    }
+    __syncthreads();
+    float o[G][DPL], mx[G], l[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        mx[g] = -INFINITY; l[g] = 0.f;
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) o[g][i] = 0.f;
+    }
+    const bf16 *kt = reinterpret_cast<const bf16 *>(a.tiles.k[tile]) + (size_t)(b * a.Hkv + hk) * a.TK * DH;
+    const bf16 *vt = reinterpret_cast<const bf16 *>(a.tiles.v[tile]) + (size_t)(b * a.Hkv + hk) * a.TK * DH;
+    for (uint32_t j0 = warp * 32; j0 < nk; j0 += SPLIT * 32) {
+        const uint32_t j = j0 + lane, cnt = min(32u, nk - j0);
+        const bool valid = j < nk;
+        // ---- scores: this lane's key against the G queries ----
+        float acc[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) acc[g] = 0.f;
+        {
+            const uint4 *kr = reinterpret_cast<const uint4 *>(kt + (size_t)min(j, nk - 1) * DH);
+            uint4 kv[4], nx[4];                                      // 64 bytes of the row at a time, the next 64 already requested
+#pragma unroll
+            for (int v = 0; v < 4; ++v) kv[v] = kr[v];
+#pragma unroll 1
+            for (int v0 = 0; v0 < DH / 8; v0 += 4) {
+                if (v0 + 4 < DH / 8) {
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) nx[v] = kr[v0 + 4 + v];
+                }
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    float f[8];
+                    unpack8(kv[v], f);
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        const float4 q0 = *reinterpret_cast<const float4 *>(qs + g * DH + (v0 + v) * 8), q1 = *reinterpret_cast<const float4 *>(qs + g * DH + (v0 + v) * 8 + 4);
+                        acc[g] = fmaf(q0.x, f[0], acc[g]); acc[g] = fmaf(q0.y, f[1], acc[g]); acc[g] = fmaf(q0.z, f[2], acc[g]); acc[g] = fmaf(q0.w, f[3], acc[g]);
+                        acc[g] = fmaf(q1.x, f[4], acc[g]); acc[g] = fmaf(q1.y, f[5], acc[g]); acc[g] = fmaf(q1.z, f[6], acc[g]); acc[g] = fmaf(q1.w, f[7], acc[g]);
+                    }
+                }
+#pragma unroll
+                for (int v = 0; v < 4; ++v) kv[v] = nx[v];
+            }
+        }
+        float p[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const float sc = valid ? acc[g] * a.scale : -INFINITY;
+            const float mnew = fmaxf(mx[g], warp_max(sc));
+            const float alpha = expf(mx[g] - mnew);
+            p[g] = valid ? expf(sc - mnew) : 0.f;
+            l[g] = l[g] * alpha + warp_sum(p[g]);
+#pragma unroll
+            for (int i = 0; i < DPL; ++i) o[g][i] *= alpha;
+            mx[g] = mnew;
+        }
+        // ---- P V: this lane's DPL output dimensions; rows past the end re-read the last valid row with weight 0 ----
+#pragma unroll 16
+        for (uint32_t t = 0; t < 32; ++t) {
+            const bf16 *vr = vt + (size_t)(j0 + min(t, cnt - 1)) * DH + lane * DPL;
+            float f[DPL];
+            if (DPL == 4) {
+                const uint2 raw = *reinterpret_cast<const uint2 *>(vr);
+                const __nv_bfloat162 a0 = *reinterpret_cast<const __nv_bfloat162 *>(&raw.x), a1 = *reinterpret_cast<const __nv_bfloat162 *>(&raw.y);
+                f[0] = __low2float(a0); f[1] = __high2float(a0); f[2 % DPL] = __low2float(a1); f[3 % DPL] = __high2float(a1);
+            } else {
+                const uint32_t raw = *reinterpret_cast<const uint32_t *>(vr);
+                const __nv_bfloat162 a0 = *reinterpret_cast<const __nv_bfloat162 *>(&raw);
+                f[0] = __low2float(a0); f[1 % DPL] = __high2float(a0);
+            }
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const float pt = __shfl_sync(0xffffffffu, p[g], t);
+#pragma unroll
+                for (int i = 0; i < DPL; ++i) o[g][i] = fmaf(pt, f[i], o[g][i]);
+            }
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        float *mine = parts + (size_t)(g * SPLIT + warp) * (DH + 2);
+        if (lane == 0) { mine[0] = mx[g]; mine[1] = l[g]; }
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) mine[2 + lane * DPL + i] = o[g][i];
+    }
+    __syncthreads();
+    for (uint32_t g = warp; g < G; g += SPLIT) {            // fixed-order merge of the SPLIT partials of head g
+        const float *p0 = parts + (size_t)g * SPLIT * (DH + 2);
+        float m = -INFINITY;
+        for (uint32_t k = 0; k < SPLIT; ++k) m = fmaxf(m, p0[k * (DH + 2)]);
+        float lsum = 0.f, accm[DPL];
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) accm[i] = 0.f;
+        for (uint32_t k = 0; k < SPLIT; ++k) {
+            const float w = expf(p0[k * (DH + 2)] - m);     // a warp that saw no key has max -inf and weight 0
+            lsum += w * p0[k * (DH + 2) + 1];
+#pragma unroll
+            for (int i = 0; i < DPL; ++i) accm[i] += w * p0[k * (DH + 2) + 2 + lane * DPL + i];
+        }
+        float *part = a.scratch + ((size_t)(b * a.Hq + hk * G + g) * a.n_tiles + tile) * (DH + 2);
+        if (lane == 0) { part[0] = m; part[1] = lsum; }
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) part[2 + lane * DPL + i] = accm[i];
+    }
+}
+
 template <int DH>
 __global__ void attn_decode_merge_kernel(AttnArgs a) {
     const uint32_t hq = blockIdx.x, b = blockIdx.y, i = threadIdx.x;
@@ -882,6 +1008,7 @@ int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb,
     return TGP_OK;
 }
 
+static int g_attn_decode_grouped = 1;   // decode: one pass over a KV tile serves all query heads of the group (0: one pass per head)
 static int g_attn_impl = 0;      // q_len >= 16: 0 by problem size, 3 tcgen05 kernel, 2 mma.sync flash kernel, 1 warp-per-row CUDA-core kernel
 
 int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *ob, const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0,
@@ -896,14 +1023,25 @@ int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *
         if (split > 32 / G) split = 32 / G;
         if (split < 1) split = 1;
         dim3 grid(nt, c->Hkv, B);
+        const bool grouped = g_attn_decode_grouped && (G == 1 || G == 2 || G == 4 || G == 8) && c->Hq % c->Hkv == 0;
+        if (grouped) {                                      // K and V read once for the whole group of query heads
+            split = (c->TK + 31) / 32;
+            if (split > 8) split = 8;
+        }
         const size_t sm = (size_t)(G * c->Dh + G * split * (c->Dh + 2)) * sizeof(float);
+#define TGP_DECODE_GROUP(DH_) do { \
+            if (G == 1) attn_decode_group_kernel<DH_, 1><<<grid, 32 * split, sm, st>>>(a, split); \
+            else if (G == 2) attn_decode_group_kernel<DH_, 2><<<grid, 32 * split, sm, st>>>(a, split); \
+            else if (G == 4) attn_decode_group_kernel<DH_, 4><<<grid, 32 * split, sm, st>>>(a, split); \
+            else attn_decode_group_kernel<DH_, 8><<<grid, 32 * split, sm, st>>>(a, split); } while (0)
         if (c->Dh == 64) {
-            attn_decode_partial_kernel<64><<<grid, 32 * G * split, sm, st>>>(a, split);
+            if (grouped) TGP_DECODE_GROUP(64); else attn_decode_partial_kernel<64><<<grid, 32 * G * split, sm, st>>>(a, split);
             attn_decode_merge_kernel<64><<<dim3(c->Hq, B), 64, 0, st>>>(a);
         } else {
-            attn_decode_partial_kernel<128><<<grid, 32 * G * split, sm, st>>>(a, split);
+            if (grouped) TGP_DECODE_GROUP(128); else attn_decode_partial_kernel<128><<<grid, 32 * G * split, sm, st>>>(a, split);
             attn_decode_merge_kernel<128><<<dim3(c->Hq, B), 128, 0, st>>>(a);
         }
+#undef TGP_DECODE_GROUP
         tgpk_launches += 1;
     } else if (q_len >= 16 && (g_attn_impl == 0 || g_attn_impl == 2 || g_attn_impl == 3)) {
         // the tcgen05 kernel works on 128 queries per CTA (it hands geometries it cannot map with TMA to the mma.sync
