@@ -150,7 +150,8 @@ def tiles_to_cache(tiles, cfg, B):
 
 
 @pytest.mark.parametrize("attn_impl", [3, 2])
-@pytest.mark.parametrize("Dh,Hq,Hkv,TK,S,T", [(64, 4, 2, 4, 9, 7), (128, 8, 2, 16, 40, 5), (64, 4, 4, 8, 33, 3), (128, 8, 1, 64, 130, 2)])
+@pytest.mark.parametrize("Dh,Hq,Hkv,TK,S,T", [(64, 4, 2, 4, 9, 7), (128, 8, 2, 16, 40, 5), (64, 4, 4, 8, 33, 3), (128, 8, 1, 64, 130, 2),
+                                             (64, 6, 2, 32, 70, 3)])      # three query heads per KV head: the per-head decode kernel
 def test_rope_kv_and_attention_prefill_then_decode(Dh, Hq, Hkv, TK, S, T, attn_impl):
     B = 2
     tb.k_attn_select(attn_impl)
