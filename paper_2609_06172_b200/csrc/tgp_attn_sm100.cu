@@ -97,12 +97,39 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
     const uint32_t last_q = min(a.q_len, q0 + BQ) - 1;
     const uint32_t nblk = (a.pos0 + last_q + 1 + BKV - 1) / BKV;
 
-    if (tid == 0) {
+    // The TMA thread (warp 5, lane 0) initialises the barriers and requests Q and the first K and V blocks at once, before
+    // the TMEM allocation and the CTA-wide barrier below.  Its state: blocks requested so far (block i uses stage i & 1)
+    // and, for the next K and V block, the KV tile and the key offset inside it.
+    uint32_t nk = 0, nv = 0, k_tile = 0, k_off = 0, v_tile = 0, v_off = 0;
+    const uint32_t head_row = (b * a.Hkv + hk) * a.TK;
+    auto load_kv = [&](uint8_t *dst, int y, uint64_t *bar, uint32_t more_bytes) {
+        mbar_expect_tx(bar, KV_BYTES + more_bytes);
+#pragma unroll
+        for (uint32_t kb = 0; kb < KB; ++kb) tma_load_2d(dst + kb * (BKV * 128), &tmKV, kb * 64, y, bar);
+    };
+    auto next_k = [&](uint32_t more_bytes) {
+        load_kv(Ks + (nk & 1) * KV_BYTES, a.krow[k_tile] + (int)(head_row + k_off), bar_k + (nk & 1), more_bytes);
+        nk += 1;
+        if ((k_off += BKV) == a.TK) { k_off = 0; k_tile += 1; }
+    };
+    auto next_v = [&]() {
+        load_kv(Vs + (nv & 1) * KV_BYTES, a.vrow[v_tile] + (int)(head_row + v_off), bar_v + (nv & 1), 0);
+        nv += 1;
+        if ((v_off += BKV) == a.TK) { v_off = 0; v_tile += 1; }
+    };
+    if (warp == 5 && lane == 0) {
         mbar_init(bar_k, 1); mbar_init(bar_k + 1, 1); mbar_init(bar_v, 1); mbar_init(bar_v + 1, 1);
         mbar_init(bar_s, 1); mbar_init(bar_sfree, 128); mbar_init(bar_p, 128); mbar_init(bar_p + 1, 128); mbar_init(bar_o, 1); mbar_init(bar_o + 1, 1); mbar_init(bar_kfree, 1); mbar_init(bar_kfree + 1, 1);
         failed[0] = 0;
         failed[1] = 0;                                       // a flag nothing ever sets, for waits that must not be cut short
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmQ) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmKV) : "memory");
+        next_k(Q_BYTES);                                     // K_0 and, on the same barrier, Q
+#pragma unroll
+        for (uint32_t kb = 0; kb < KB; ++kb) tma_load_2d(Qs + kb * (BQ * 128), &tmQ, hq * DH + kb * 64, b * a.q_len + q0, bar_k);
+        if (1 < nblk) next_k(0);
+        next_v();
     }
     if (warp == 4) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(256u) : "memory");
@@ -119,33 +146,8 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
     if (warp >= 4) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 64;" ::: "memory");
         if (warp == 5) {
-            // ======================= producer: every TMA load (lane 0) =======================
-            uint32_t nk = 0, nv = 0;                             // K / V blocks requested so far (block i uses stage i & 1)
+            // ======================= TMA warp: lane 0 requests the remaining K and V blocks =======================
             if (lane == 0) {
-                asm volatile("prefetch.tensormap [%0];" ::"l"(&tmQ) : "memory");
-                asm volatile("prefetch.tensormap [%0];" ::"l"(&tmKV) : "memory");
-                const uint32_t head_row = (b * a.Hkv + hk) * a.TK;
-                uint32_t k_tile = 0, k_off = 0, v_tile = 0, v_off = 0;           // tile and key offset inside it of the next block
-                auto load_kv = [&](uint8_t *dst, int y, uint64_t *bar, uint32_t more_bytes) {
-                    mbar_expect_tx(bar, KV_BYTES + more_bytes);
-    #pragma unroll
-                    for (uint32_t kb = 0; kb < KB; ++kb) tma_load_2d(dst + kb * (BKV * 128), &tmKV, kb * 64, y, bar);
-                };
-                auto next_k = [&](uint32_t more_bytes) {
-                    load_kv(Ks + (nk & 1) * KV_BYTES, a.krow[k_tile] + (int)(head_row + k_off), bar_k + (nk & 1), more_bytes);
-                    nk += 1;
-                    if ((k_off += BKV) == a.TK) { k_off = 0; k_tile += 1; }
-                };
-                auto next_v = [&]() {
-                    load_kv(Vs + (nv & 1) * KV_BYTES, a.vrow[v_tile] + (int)(head_row + v_off), bar_v + (nv & 1), 0);
-                    nv += 1;
-                    if ((v_off += BKV) == a.TK) { v_off = 0; v_tile += 1; }
-                };
-                next_k(Q_BYTES);
-    #pragma unroll
-                for (uint32_t kb = 0; kb < KB; ++kb) tma_load_2d(Qs + kb * (BQ * 128), &tmQ, hq * DH + kb * 64, b * a.q_len + q0, bar_k);
-                if (1 < nblk) next_k(0);
-                next_v();
                 for (uint32_t jb = 0; jb + 1 < nblk; ++jb) {
                     const uint32_t st = jb & 1;
                     if (jb + 2 < nblk) {                                         // K_jb+2 goes where K_jb is, once S_jb is complete
@@ -177,10 +179,10 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
                 if (lane == 0) {
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint8_t *Kj = Ks + (jb & 1) * KV_BYTES;
-    #pragma unroll
+#pragma unroll
                     for (uint32_t kb = 0; kb < KB; ++kb) {
                         const uint64_t dq = umma_desc(smem_u32(Qs + kb * (BQ * 128))), dk = umma_desc(smem_u32(Kj + kb * (BKV * 128)));
-    #pragma unroll
+#pragma unroll
                         for (uint32_t k = 0; k < 4; ++k) umma(tmem_S, dq + 2 * k, dk + 2 * k, idesc_s, (kb | k) != 0);
                     }
                     umma_commit(bar_s);
@@ -212,7 +214,7 @@ __global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __gri
                 if (lane == 0) {
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t dv = umma_desc_mn(smem_u32(Vs + st * KV_BYTES), BKV * 128);
-    #pragma unroll
+#pragma unroll
                     for (uint32_t k = 0; k < 4; ++k)                             // 16 keys per step: 8 columns of P, 2048 B of V rows
                         umma_ts(tmem_O, tmem_P + st * 32 + 8 * k, dv + 128 * k, idesc_o, (jb | k) != 0);
                     umma_commit(bar_o + st);
