@@ -336,6 +336,7 @@ def main():
     ap.add_argument("--kernel-loop", choices=["decode", "prefill", "attention"], default=None,
                     help="only run the back-to-back weight-product loop of one step (small, for ncu captures)")
     ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--alias-layers", type=int, default=None, help="host pool with this many physical layers: layers l and l + N share host pages (for pools larger than the host can page-lock)")
     ap.add_argument("--unseen-prompts", action="store_true", help="MoE: time prompts of another seed than the profile pass saw")
     ap.add_argument("--seq", type=int, default=None, help="with --kernel-loop attention: prompt length instead of the configuration's")
     ap.add_argument("--graph", action="store_true", help="replay the whole planned run as one CUDA graph (dense models; for host-bound tiny steps)")
@@ -391,7 +392,16 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    pool = pinned_pool(lay.pool_bytes)
+    aliased = None
+    if args.alias_layers:
+        # more weights than this host can page-lock: layers l and l + alias_layers share physical host pages (same
+        # virtual layout, same bytes over the link, same arithmetic; logits are those of a model with repeated layers)
+        from paper_2609_06172_b200.runner import AliasedPool
+        aliased = AliasedPool(lay, args.alias_layers)
+        pool = torch.from_numpy(aliased.numpy())
+        aliased.page_lock()
+    else:
+        pool = pinned_pool(lay.pool_bytes)
     si.fill_pool_torch(lay, pool, device=dev)
     bias = si.router_bias(cfg) if cfg.E else None
     s = Session(lay, MACHINE, pool_base=pool.data_ptr(), pool_flags=tb.POOL_PINNED, router_bias=bias)
@@ -599,7 +609,7 @@ def main():
            "prefill_tok_s": cfg.B * cfg.S / (step_ms[0] * 1e-3), "decode_tok_s": cfg.B * T / (sum(step_ms[1:]) * 1e-3) if T else None,
            "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": int(totals[:, 0].sum()) + cfg.B * (cfg.S + T) * 4,
                    "d2h_bytes_per_step": L_d2h + cfg.B * (T + 1) * 4 + cfg.B * cfg.V * 4},
-           "object_level_prefetch": object_level, "policy_bits": args.bits, "trace_mismatches": mismatches, "moe_profile_pass_s": profile_s, "unseen_prompts": bool(args.unseen_prompts), "moe_prediction": moe_prediction,
+           "object_level_prefetch": object_level, "policy_bits": args.bits, "trace_mismatches": mismatches, "moe_profile_pass_s": profile_s, "unseen_prompts": bool(args.unseen_prompts), "host_pool": ({"aliased_physical_layers": args.alias_layers, "physical_bytes": aliased.phys_bytes, "virtual_bytes": lay.pool_bytes} if aliased else "pinned, one physical page per byte"), "moe_prediction": moe_prediction,
            "gpu_launches": launches * args.steps, "clocks": clocks, "roofline": roof, "step_roofline": step_roof,
            "kernels": {f"{k[0]}:{k[1]}": {"ms": round(v, 3), "launches": kind_n[k], "GBps": round(kind_bytes[k] / (v * 1e-3) / 1e9, 1),
                                            "TFLOPs": round(kind_flops[k] / (v * 1e-3) / 1e12, 2)} for k, v in sorted(kind_ms.items())}}

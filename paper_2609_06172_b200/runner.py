@@ -16,6 +16,92 @@ def pinned_pool(nbytes: int) -> torch.Tensor:
     return t
 
 
+class AliasedPool:
+    """Host pool for shapes whose weights exceed what this host can page-lock: the weight regions of layers l and
+    l + phys_layers, l + 2 * phys_layers, ... are the same physical pages (one memfd mapped several times into one
+    contiguous virtual range), so the pool keeps its full virtual layout - every tensor at its own address, nothing the
+    library could tell apart - while physical memory holds only phys_layers layers.  Bytes moved over the link and
+    arithmetic per step are unchanged; the weights of aliased layers are equal, so logits are those of another model:
+    for throughput runs only.  Embedding, head and KV tiles are never aliased.  The memory is not page-locked yet:
+    page_lock() registers it mapping by mapping (one cudaHostRegister over several mappings is refused by the OS layer),
+    after which the pool is registered with POOL_PINNED."""
+
+    def __init__(self, layout, phys_layers):
+        import ctypes as C
+        import mmap
+        import os
+        import seeded_inputs as si
+        cfg = layout.cfg
+        kv = (si.K_KT, si.K_VT)
+        start = [min(t.pool_off for t in layout.tensors if t.layer == l and t.kind not in kv) for l in range(cfg.L)]
+        end = max(t.pool_off + t.size for t in layout.tensors if t.layer == cfg.L - 1 and t.kind not in kv)
+        lb = (end - start[0]) // cfg.L
+        page = mmap.PAGESIZE
+        if any(start[l] != start[0] + l * lb for l in range(cfg.L)) or end != start[0] + cfg.L * lb or lb % page or start[0] % page:
+            raise ValueError("layer regions are not contiguous, equal and page-aligned")
+        if not 1 <= phys_layers <= cfg.L:
+            raise ValueError("phys_layers out of range")
+        self.nbytes = layout.pool_bytes
+        self.layer_bytes, self.first_layer_off, self.phys_layers = lb, start[0], phys_layers
+        vlen = (self.nbytes + page - 1) // page * page
+        tail_v = start[0] + cfg.L * lb                                  # first virtual byte after the layers
+        self.phys_bytes = start[0] + phys_layers * lb + (vlen - tail_v)
+        libc = C.CDLL(None, use_errno=True)
+        libc.mmap.restype, libc.mmap.argtypes = C.c_void_p, [C.c_void_p, C.c_size_t, C.c_int, C.c_int, C.c_int, C.c_long]
+        libc.munmap.restype, libc.munmap.argtypes = C.c_int, [C.c_void_p, C.c_size_t]
+        self._libc, self._vlen = libc, vlen
+        self._fd = os.memfd_create("tgp_pool")
+        os.ftruncate(self._fd, self.phys_bytes)
+        failed = C.c_void_p(-1).value                                   # MAP_FAILED; protection 0 below is PROT_NONE: address space only
+        base = libc.mmap(None, vlen, 0, mmap.MAP_PRIVATE | mmap.MAP_ANONYMOUS | getattr(mmap, "MAP_NORESERVE", 0x4000), -1, 0)
+        if base in (None, failed):
+            raise OSError(C.get_errno(), "mmap (reserve) failed")
+        self._base = base
+
+        self.pieces = []                                                # (virtual offset, length) of every mapping
+
+        def place(voff, length, foff):
+            got = libc.mmap(C.c_void_p(base + voff), length, mmap.PROT_READ | mmap.PROT_WRITE, mmap.MAP_SHARED | 0x10, self._fd, foff)   # 0x10 = MAP_FIXED
+            if got != base + voff:
+                raise OSError(C.get_errno(), "mmap (place) failed")
+            self.pieces.append((voff, length))
+
+        place(0, start[0], 0)                                           # embedding
+        for l0 in range(0, cfg.L, phys_layers):                         # each group of layers onto the same file range
+            n = min(phys_layers, cfg.L - l0)
+            place(start[0] + l0 * lb, n * lb, start[0])
+        place(tail_v, vlen - tail_v, start[0] + phys_layers * lb)        # final norm, head, KV tiles
+        self._buf = (C.c_uint8 * self.nbytes).from_address(base)
+
+    def data_ptr(self):
+        return self._base
+
+    def page_lock(self):
+        """cudaHostRegister, one call per mapping.  Raises on the first refusal (what was registered stays registered
+        until close())."""
+        rt = torch.cuda.cudart()
+        self._locked = getattr(self, "_locked", [])
+        for voff, length in self.pieces:
+            rc = int(rt.cudaHostRegister(self._base + voff, length, 0))
+            if rc != 0:
+                raise RuntimeError(f"cudaHostRegister refused {length} bytes at pool offset {voff}: cudaError {rc}")
+            self._locked.append(voff)
+
+    def numpy(self):
+        return np.ctypeslib.as_array(self._buf)
+
+    def close(self):
+        import os
+        if self._base:
+            for voff in getattr(self, "_locked", []):
+                torch.cuda.cudart().cudaHostUnregister(self._base + voff)
+            self._locked = []
+            self._buf = None
+            self._libc.munmap(self._base, self._vlen)
+            os.close(self._fd)
+            self._base = 0
+
+
 class Runner:
     """Owns arena, workspace, logits and streams for one Session and drives tgp_step()."""
 

@@ -272,3 +272,29 @@ def test_measured_time_link_test_by_hand():
     assert policy.classify(5000, 300, 100, toy, measured_ns=10_000_000_000) == policy.CLS_COMPUTE
     assert policy.classify(100, 600, 100, toy, measured_ns=11_000_000_000) == policy.CLS_HBM
     assert policy.classify(5000, 300, 100, toy, measured_ns=0) == policy.CLS_LINK          # no measurement: analytic
+
+
+def test_aliased_host_pool_shares_pages_between_layer_groups_only():
+    """The fallback for pools larger than the host can page-lock: layers l and l + phys share physical pages, everything
+    else (embedding, head, KV tiles) stays private, and the virtual layout is the ordinary one."""
+    from paper_2609_06172_b200.runner import AliasedPool
+    cfg = replace(si.CONFIGS[1], L=6, d=1024, F=4096, Hq=16, Hkv=16)   # layer regions are multiples of the page size here
+    lay = si.build_layout(cfg)
+    try:
+        p = AliasedPool(lay, 2)
+    except ValueError as ex:
+        pytest.skip(f"layout not page-aligned on this machine: {ex}")
+    a = p.numpy()
+    assert a.size == lay.pool_bytes and p.phys_bytes - lay.pool_bytes + 4 * p.layer_bytes in range(0, 4096)      # fresh pages read as zero
+    w = [t for t in lay.tensors if t.kind == si.K_WQ]
+    by_layer = {t.layer: t for t in w}
+    a[by_layer[1].pool_off] = 7                                     # layer 1 ...
+    assert a[by_layer[3].pool_off] == 7 and a[by_layer[5].pool_off] == 7        # ... is layers 3 and 5
+    assert a[by_layer[0].pool_off] == 0 and a[by_layer[2].pool_off] == 0
+    kv = [t for t in lay.tensors if t.kind == si.K_KT]
+    a[kv[0].pool_off] = 9
+    assert sum(int(a[t.pool_off] == 9) for t in kv) == 1            # KV tiles are private
+    emb = next(t for t in lay.tensors if t.kind == si.K_EMBED)
+    a[emb.pool_off + 5] = 3
+    assert int((a[:emb.size] == 3).sum()) == 1 and all(int(a[t.pool_off + 5]) != 3 for t in w)
+    p.close()
