@@ -352,6 +352,37 @@ def test_mixtral_widths_at_one_layer_match_oracle_batch_of_eight():
     s.close()
 
 
+def test_layer_aliased_host_pool_runs_like_a_pool_with_repeated_layers():
+    """The host pool for shapes too large to page-lock (layers l and l + 2 on the same physical pages, page-locked mapping
+    by mapping) against an ordinary pinned pool that holds the same bytes: same plan, bitwise equal logits."""
+    from paper_2609_06172_b200.runner import AliasedPool
+    cfg = replace(si.CONFIGS[1], L=4, d=1024, F=4096, Hq=16, Hkv=16, T=3, budget_rule="half_w")
+    lay = si.build_layout(cfg)
+    ap = AliasedPool(lay, 2)
+    ap.page_lock()
+    try:
+        si.fill_pool(lay, ap.numpy())                        # layers 2, 3 are written last: layers 0, 1 now hold their values too
+        pool = pinned_pool(lay.pool_bytes)
+        pool.numpy()[:] = ap.numpy()
+        prompt = si.prompt_tokens(cfg)
+        forced = (np.arange(cfg.B * cfg.T, dtype=np.int32).reshape(cfg.B, cfg.T) * 131 + 7) % cfg.V
+        outs = []
+        for base in (pool.data_ptr(), ap.data_ptr()):
+            s = Session(lay, MACHINE, pool_base=base, pool_flags=tb.POOL_PINNED)
+            blobs = s.plan(T=cfg.T)
+            got, _ = Runner(s, cfg.B * cfg.S).generate(prompt, cfg.T, forced=forced)
+            outs.append((blobs, got))
+            s.close()
+        assert outs[0][0] == outs[1][0]
+        for a, b in zip(outs[0][1], outs[1][1]):
+            assert np.array_equal(a, b) and np.isfinite(a).all()
+        w = {t.layer: t for t in lay.tensors if t.kind == si.K_WQ}
+        assert np.array_equal(ap.numpy()[w[0].pool_off: w[0].pool_off + 64], ap.numpy()[w[2].pool_off: w[2].pool_off + 64])
+    finally:
+        torch.cuda.synchronize()
+        ap.close()
+
+
 def test_router_topk_ties_and_single_expert_equals_dense():
     """E = 1, top-1 routes every token to the one expert with gate 1: same logits as the dense model with those weights."""
     dense = replace(MOE, E=0, topk=0, L=1)
