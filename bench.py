@@ -147,12 +147,19 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
     from paper_2609_06172_b200 import binding as tb
     cfg = lay.cfg
     shapes = gemm_shapes_of_step(lay, M)
+    # random operands with the weights' distribution: constant data would toggle few wires, draw little power and let
+    # a seconds-long tensor-core loop run at clocks the real step (random weights, power-capped) never sees
+    gen = torch.Generator(device=device)
+    gen.manual_seed(lay.cfg.seed)
     wbuf = torch.empty(cold_bytes, dtype=torch.uint8, device=device)
-    wbuf.view(torch.int16).fill_(0x3C00)                                  # bf16 0.0078: finite values
+    w16 = wbuf.view(torch.bfloat16)
+    for o in range(0, w16.numel(), 1 << 26):
+        c = min(1 << 26, w16.numel() - o)
+        w16[o:o + c] = (torch.randn(c, device=device, generator=gen) * 0.02).bfloat16()
     kmax = max(k for (_, k, _, _) in shapes)
     nmax = max(n for (n, _, _, _) in shapes)
     mmax = max(m for (_, _, _, m) in shapes)
-    A = torch.full((mmax, kmax), 0.01, dtype=torch.bfloat16, device=device)
+    A = torch.randn((mmax, kmax), device=device, generator=gen).bfloat16()
     Cbuf = torch.zeros((mmax, nmax), dtype=torch.float32, device=device)
     stream = torch.cuda.Stream(device=device)
     off = 0

@@ -267,7 +267,8 @@ int  tgp_k_skinny_select(int impl);
  * previous one has completed).  Results are identical either way.  Process-wide; default on. */
 int  tgp_k_gemv_overlap(int enable);
 /* Tensor-core GEMM variant: 0 (default) picks by problem size, 1 forces the 128x128 one-tile-per-CTA kernel,
- * 2 forces the persistent 128x256 kernel with double-buffered accumulators.  Process-wide; for tests and timing. */
+ * 2 the persistent 128x256 kernel with double-buffered accumulators, 3 the paired kernel (256x256 tiles on the two SMs
+ * of a CTA pair, each loading half of the weight tile).  Process-wide; for tests and timing. */
 int  tgp_k_gemm_tc_variant(int variant);
 /* Which kernel serves attention with q_len >= 16: 0 (default) by problem size - the tcgen05 kernel (S and O in TMEM,
  * K/V fed by TMA) for q_len >= 128, else the mma.sync flash-style kernel;

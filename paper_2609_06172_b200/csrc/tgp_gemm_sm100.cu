@@ -277,6 +277,150 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_persistent_kernel(const __grid
     }
 }
 
+// ---- paired variant: one 256 x 256 tile per CTA pair (cta_group::2) -------------------------------------------------
+// What limits the kernel above is not the tensor pipe but what an SM can pull from L2: 48 KB per 64-wide K block is
+// 54 B per clock, and the MMA thread waits for data a third of the time.  Here the two CTAs of a cluster sit on the two
+// SMs of a TPC and share one MMA of M = 256: each loads its own 128 rows of A and HALF of the 256 rows of W (B), 32 KB
+// per K block for the same arithmetic per SM, six stages deep.  Only the even CTA (the leader) issues MMAs; the TMA loads
+// of both CTAs count on the leader's `full` barrier; an MMA commit arrives on the `empty` / `acc_full` barriers of both
+// CTAs; both CTAs drain their own 128 rows of the accumulator from their own TMEM and arrive (the odd one remotely) on
+// the leader's `acc_empty`.  No multicast load anywhere.  Same bounded waits and error word; a cluster barrier before
+// TMEM is freed keeps either CTA from leaving while its partner still works on its memory.
+constexpr int Q_STAGES = 6;
+
+__global__ void __launch_bounds__(192, 1) gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                                                              float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
+    extern __shared__ uint8_t smem_raw[];
+    constexpr int A_BYTES = BM * BK * 2, B_BYTES = (P_BN / 2) * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + Q_STAGES * STAGE_BYTES);      // used in the leader only
+    uint64_t *empty = full + Q_STAGES;
+    uint64_t *acc_full = empty + Q_STAGES;           // [2]
+    uint64_t *acc_empty = acc_full + 2;              // [2], used in the leader only: 4 warps of each CTA
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+    volatile uint32_t *failed = tmem_slot + 1;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank(), pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
+    const uint32_t num_k = (K + BK - 1) / BK;
+    const uint32_t tiles_m = (M + 2 * BM - 1) / (2 * BM), tiles_n = (n + P_BN - 1) / P_BN, tiles = tiles_m * tiles_n;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < Q_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 8); }
+        *failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 2) {                                  // the same warp in both CTAs of the pair
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    cluster_sync_all();                               // barriers of both CTAs initialised, TMEM allocated
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    auto tile_origin = [&](uint32_t tile, uint32_t &m0, uint32_t &n0) {       // of the pair's 256 x 256 tile
+        const uint32_t group = tile / (GROUP_M * tiles_n), first_m = group * GROUP_M;
+        const uint32_t rows_in_group = min((uint32_t)GROUP_M, tiles_m - first_m);
+        const uint32_t in_group = tile - group * GROUP_M * tiles_n;
+        m0 = (first_m + in_group % rows_in_group) * (2 * BM);
+        n0 = (in_group / rows_in_group) * P_BN;
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {                              // TMA thread of this CTA: its rows of A, its half of B
+            uint32_t it = 0, armed = 0;
+            for (uint32_t tile = pair; tile < tiles; tile += pairs) {
+                uint32_t m0, n0;
+                tile_origin(tile, m0, n0);
+                bool ok = true;
+                for (uint32_t kb = 0; kb < num_k; ++kb, ++it) {
+                    const uint32_t s = it % Q_STAGES, ph = (it / Q_STAGES) & 1;
+                    if (*failed || !mbar_wait(&empty[s], ph ^ 1, failed)) { if (!*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, (1 << 8) | (int)s); } ok = false; break; }
+                    if (rank == 0) mbar_expect_tx(&full[s], 2 * STAGE_BYTES);
+                    tma_load_2d_pair(smem + s * STAGE_BYTES, &tmA, (int)(kb * BK), (int)(m0 + rank * BM), &full[s]);
+                    tma_load_2d_pair(smem + s * STAGE_BYTES + A_BYTES, &tmB, (int)(kb * BK), (int)(n0 + rank * (P_BN / 2)), &full[s]);
+                    armed = it + 1;
+                }
+                if (!ok) break;
+            }
+            if (*failed && rank == 0) {               // loads of both CTAs still in flight land on these barriers (bounded wait)
+                volatile uint32_t never = 0;
+                for (uint32_t q = armed > Q_STAGES ? armed - Q_STAGES : 0; q < armed; ++q) mbar_wait(&full[q % Q_STAGES], (q / Q_STAGES) & 1, &never);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {                 // MMA thread of the pair
+            constexpr uint32_t idesc = umma_idesc_pair(P_BN);
+            uint32_t it = 0, lt = 0;
+            bool ok = true;
+            for (uint32_t tile = pair; tile < tiles && ok; tile += pairs, ++lt) {
+                const uint32_t buf = lt & 1, use = lt >> 1;
+                if (*failed || !mbar_wait(&acc_empty[buf], (use & 1) ^ 1, failed)) { if (!*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, (2 << 8) | 0x80 | (int)buf); } break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tacc = tmem_base + buf * P_BN;
+                for (uint32_t kb = 0; kb < num_k; ++kb, ++it) {
+                    const uint32_t s = it % Q_STAGES, ph = (it / Q_STAGES) & 1;
+                    if (*failed || !mbar_wait(&full[s], ph, failed)) { if (!*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, (2 << 8) | (int)s); } ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint64_t da = umma_desc(smem_u32(smem + s * STAGE_BYTES));
+                    const uint64_t db = umma_desc(smem_u32(smem + s * STAGE_BYTES + A_BYTES));
+#pragma unroll
+                    for (uint32_t k = 0; k < BK / 16; ++k) umma_pair(tacc, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+                    umma_commit_pair(&empty[s]);
+                }
+                if (ok) umma_commit_pair(&acc_full[buf]);
+            }
+        }
+    } else {
+        const uint32_t quarter = warp & 3;
+        const bool vec = ((ldc | col0) & 3u) == 0 && (reinterpret_cast<uintptr_t>(C) & 15u) == 0;
+        uint32_t lt = 0;
+        for (uint32_t tile = pair; tile < tiles; tile += pairs, ++lt) {
+            const uint32_t buf = lt & 1, use = lt >> 1;
+            bool ready = !*failed && mbar_wait(&acc_full[buf], use & 1, failed);
+            if (!ready && !*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, 3 << 8); }
+            ready = __all_sync(0xffffffffu, ready && !*failed);
+            if (!ready) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            uint32_t m0, n0;
+            tile_origin(tile, m0, n0);
+            const uint32_t row = m0 + rank * BM + quarter * 32 + lane;
+#pragma unroll 1
+            for (uint32_t c = 0; c < P_BN / 32; ++c) {
+                float v[32];
+                tmem_ld32(tmem_base + ((quarter * 32) << 16) + buf * P_BN + c * 32, v);
+                const uint32_t col = n0 + c * 32;
+                if (row < M && col < n) {
+                    float *dst = C + (size_t)row * ldc + col0 + col;
+                    if (vec && col + 32 <= n) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                            if (accumulate) { const float4 old = *reinterpret_cast<const float4 *>(dst + j); o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w; }
+                            *reinterpret_cast<float4 *>(dst + j) = o;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col + j < n) dst[j] = accumulate ? dst[j] + v[j] : v[j];
+                    }
+                }
+            }
+            // this warp has read its quarter of this CTA's half of the buffer: tell the pair's MMA thread
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(&acc_empty[buf], 0);
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    cluster_sync_all();                               // neither CTA frees TMEM or leaves while its partner may still touch it
+    if (warp == 2) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
 // 2-D bf16 row-major [rows, K] map with a [box_rows, 64] box, 128-byte swizzle, zero fill outside.
 bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t K, uint32_t box_rows) {
     static_assert(BK == 64, "the shared tensor-map helper encodes 64-element boxes");
@@ -287,7 +431,7 @@ bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t K, uin
 
 extern thread_local uint64_t tgpk_launches;
 
-static int g_tc_variant = 0;     // 0 auto, 1 force the 128x128 per-tile kernel, 2 force the persistent 128x256 kernel
+static int g_tc_variant = 0;     // 0 auto, 1 force the 128x128 per-tile kernel, 2 the persistent 128x256 kernel, 3 the paired 256x256 kernel
 
 int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
     constexpr int BN = 128;
@@ -296,10 +440,31 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
     static int sms = 0;
     if (!sms) { int dev = 0; cudaGetDevice(&dev); if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148; }
     const uint32_t tiles_p = ((M + BM - 1) / BM) * ((n + P_BN - 1) / P_BN);
-    const bool persistent = g_tc_variant == 2 || (g_tc_variant == 0 && tiles_p >= 2u * (uint32_t)sms);
+    const uint32_t tiles_q = ((M + 2 * BM - 1) / (2 * BM)) * ((n + P_BN - 1) / P_BN);
+    const bool paired = g_tc_variant == 3 || (g_tc_variant == 0 && tiles_q >= (uint32_t)sms);          // two tiles per pair of SMs or more
+    const bool persistent = !paired && (g_tc_variant == 2 || (g_tc_variant == 0 && tiles_p >= 2u * (uint32_t)sms));
     CUtensorMap ma, mb;
-    if (!make_map(&ma, A, M, K, BM) || !make_map(&mb, W, n, K, persistent ? P_BN : BN)) return TGP_E_CUDA;
-    if (persistent) {
+    if (!make_map(&ma, A, M, K, BM) || !make_map(&mb, W, n, K, paired ? P_BN / 2 : persistent ? P_BN : BN)) return TGP_E_CUDA;
+    if (paired) {
+        constexpr int SMEM = Q_STAGES * (BM * BK * 2 + (P_BN / 2) * BK * 2) + 160 + 1024;
+        static bool attr_q = false;
+        if (!attr_q) {
+            if (cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess) return TGP_E_CUDA;
+            attr_q = true;
+        }
+        const uint32_t pairs_max = (uint32_t)sms / 2, npairs = tiles_q < pairs_max ? tiles_q : pairs_max;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * npairs);
+        cfg.blockDim = dim3(192);
+        cfg.dynamicSmemBytes = SMEM;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, gemm_tc_pair_kernel, ma, mb, C, M, n, K, ldc, col0, accumulate) != cudaSuccess) return TGP_E_CUDA;
+    } else if (persistent) {
         constexpr int SMEM = P_STAGES * (BM * BK * 2 + P_BN * BK * 2) + 128 + 1024;
         static bool attr_p = false;
         if (!attr_p) {
@@ -322,7 +487,7 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
 }
 
 extern "C" int tgp_k_gemm_tc_variant(int v) {
-    if (v < 0 || v > 2) return TGP_E_INVAL;
+    if (v < 0 || v > 3) return TGP_E_INVAL;
     g_tc_variant = v;
     return TGP_OK;
 }

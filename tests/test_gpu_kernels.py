@@ -86,13 +86,14 @@ def test_tensor_core_gemm_agrees_with_cuda_core_gemm_and_reports_no_timeout():
 
 @pytest.mark.parametrize("M,n,K,acc", [(300, 520, 1096, 0), (129, 257, 72, 1), (1024, 1536, 512, 0), (640, 2300, 2048, 1), (4096, 4096, 256, 0)])
 def test_persistent_tensor_core_gemm_matches_per_tile_kernel_and_oracle(M, n, K, acc):
-    """The persistent 128x256 kernel (forced, even on small problems: ragged tiles, fewer tiles than SMs, several
-    tiles per CTA) against the per-tile kernel and the oracle."""
+    """The paired 256x256 kernel and the persistent 128x256 kernel (forced, even on small problems: ragged tiles, a pair
+    whose second CTA has no valid row, fewer tiles than SMs, several tiles per CTA) against the per-tile kernel and the
+    oracle."""
     a_bits, w_bits = rnd_bits(11, M * K).reshape(M, K), rnd_bits(12, n * K).reshape(n, K)
     A, W = bf16_dev(a_bits), bf16_dev(w_bits)
     c0 = np.random.default_rng(7).standard_normal((M, n)).astype(np.float32) * 0.01
     outs = []
-    for variant in (2, 1):
+    for variant in (3, 2, 1):
         tb.k_gemm_tc_variant(variant)
         Cd = torch.from_numpy(c0.copy()).to(DEV)
         tb.k_gemm(A, W, Cd, M, n, K, n, 0, acc)
@@ -102,8 +103,9 @@ def test_persistent_tensor_core_gemm_matches_per_tile_kernel_and_oracle(M, n, K,
     assert tb.k_gemm_status() == 0
     want = oracle().linear(si.bf16_bits_to_f32(a_bits), si.bf16_bits_to_f32(w_bits).astype(np.float64)).astype(np.float64) + (c0 if acc else 0)
     scale = np.abs(want).max()
-    assert np.abs(outs[0] - want).max() < 2e-5 * scale + 1e-7
-    assert np.abs(outs[0] - outs[1]).max() < 2e-5 * scale + 1e-7
+    for o in outs:
+        assert np.abs(o - want).max() < 2e-5 * scale + 1e-7
+    assert np.abs(outs[0] - outs[2]).max() < 2e-5 * scale + 1e-7 and np.abs(outs[1] - outs[2]).max() < 2e-5 * scale + 1e-7
 
 
 def test_gemm_rejects_bad_arguments_and_accepts_empty():
