@@ -542,7 +542,13 @@ def main():
         sec, bpl, fpl, nl, table = kernel_loop(lay, Mk, args.reps, dev)
         if dom[0] == "prefill" and fpl / MACHINE["peak_flops"] > bpl / MACHINE["hbm_Bps"]:
             ach = fpl / sec / 1e12
-            roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"]}
+            # the loop below replays the step's launches for seconds under the power cap: the matching denominator is the
+            # sustained cuBLAS figure (the burst figure is for a kernel timed alone for a millisecond)
+            loop_s = sec * nl * args.reps * 4
+            pk = peaks["bf16_sustained"] if (loop_s > 1.0 and peaks.get("bf16_sustained")) else peaks["bf16_tflops"]
+            roof = {"bound": "tensor", "achieved": ach, "peak": pk, "unit": "TFLOP/s", "frac": ach / pk,
+                    "peak_kind": "sustained cuBLAS bf16 (timed loop of %.1f s)" % loop_s if pk != peaks["bf16_tflops"] else "burst cuBLAS bf16",
+                    "frac_of_burst_peak": ach / peaks["bf16_tflops"]}
         else:
             ach = bpl / sec / 1e9
             roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"]}
