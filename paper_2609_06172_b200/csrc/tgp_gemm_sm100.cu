@@ -1,5 +1,7 @@
 // Prefill GEMM on the 5th-generation tensor cores (sm_100a): C[M, n] (=|+=) A[M, K] * W[n, K]^T,
-// bf16 operands, fp32 accumulation in tensor memory.
+// bf16 operands, fp32 accumulation in tensor memory.  Three kernels, chosen by problem size in tgpk_gemm_tc(): one
+// tile per CTA (below), a persistent kernel with 128 x 256 tiles and double-buffered accumulators, and - for the large
+// products of a prefill - a kernel in which the two CTAs of a cluster share 256 x 256 tiles through the two-SM MMA.
 //
 // One CTA computes a 128 x BN tile.  Warp 0 (one lane) feeds a 3-stage shared-memory ring with TMA
 // (128-byte swizzle, 64 bf16 of K per stage); warp 1 (one lane) issues tcgen05.mma (M=128, N=BN, K=16,
