@@ -188,32 +188,34 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
         run_all(stream)
     stream.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    g, passes = graph_of()
-    with torch.cuda.stream(stream):
-        g.replay()
-        stream.synchronize()
-        e0.record(stream)
-        for _ in range(reps):
+    def bounded(g, budget_s):
+        """One untimed-for-the-result replay measures a replay's length; then as many of the `reps` replays as fit in
+        budget_s seconds are timed (a deep model's step has thousands of launches: 20 replays would run for minutes)."""
+        with torch.cuda.stream(stream):
+            e0.record(stream)
             g.replay()
-        e1.record(stream)
-    stream.synchronize()
-    reps_eff = reps * passes
-    sec = e0.elapsed_time(e1) * 1e-3 / (reps_eff * len(shapes))
+            e1.record(stream)
+            stream.synchronize()
+            n = max(1, min(reps, int(budget_s / max(1e-6, e0.elapsed_time(e1) * 1e-3))))
+            e0.record(stream)
+            for _ in range(n):
+                g.replay()
+            e1.record(stream)
+        stream.synchronize()
+        return n, e0.elapsed_time(e1) * 1e-3
+
+    g, passes = graph_of()
+    n_rep, total_s = bounded(g, 4.0)
+    kernel_loop.last = {"reps": n_rep, "passes": passes, "seconds": total_s}
+    sec = total_s / (n_rep * passes * len(shapes))
     bytes_per = sum(2 * m * K + 2 * K * n + 4 * m * n * (2 if res else 1) for (n, K, res, m) in shapes) / len(shapes)
     flops_per = sum(2 * m * K * n for (n, K, res, m) in shapes) / len(shapes)
     table = {}
     for sh in sorted(set(shapes)):
         cnt = shapes.count(sh)
         g, passes = graph_of(only=sh)
-        with torch.cuda.stream(stream):
-            g.replay()
-            stream.synchronize()
-            e0.record(stream)
-            for _ in range(reps):
-                g.replay()
-            e1.record(stream)
-        stream.synchronize()
-        t = e0.elapsed_time(e1) * 1e-3 / (reps * passes * cnt)
+        n_sh, t_sh = bounded(g, 1.0)
+        t = t_sh / (n_sh * passes * cnt)
         n, K, res, m = sh
         b = 2 * m * K + 2 * K * n + 4 * m * n * (2 if res else 1)
         table[f"n={n} K={K} M={m} res={res}"] = {"launches_per_step": cnt, "us": round(t * 1e6, 2), "GBps": round(b / t / 1e9, 1),
@@ -544,7 +546,7 @@ def main():
             ach = fpl / sec / 1e12
             # the loop below replays the step's launches for seconds under the power cap: the matching denominator is the
             # sustained cuBLAS figure (the burst figure is for a kernel timed alone for a millisecond)
-            loop_s = sec * nl * args.reps * 4
+            loop_s = kernel_loop.last["seconds"]
             pk = peaks["bf16_sustained"] if (loop_s > 1.0 and peaks.get("bf16_sustained")) else peaks["bf16_tflops"]
             roof = {"bound": "tensor", "achieved": ach, "peak": pk, "unit": "TFLOP/s", "frac": ach / pk,
                     "peak_kind": "sustained cuBLAS bf16 (timed loop of %.1f s)" % loop_s if pk != peaks["bf16_tflops"] else "burst cuBLAS bf16",
@@ -554,7 +556,7 @@ def main():
             roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"]}
         roof.update({"kernel": f"weight-block product ({dom[0]}, M={Mk}): " + ("gemv_kernel" if Mk <= 16 else "gemm_tc_kernel"),
                      "launches": kind_n[dom], "avg_us": sec * 1e6, "algorithmic_per_launch": fpl if roof["bound"] == "tensor" else bpl,
-                     "timing": f"CUDA-graph replay of the {nl} launches of one step, {args.reps} x 4 passes back to back, cold inputs cycling through 1 GiB, CUDA events on the launch stream",
+                     "timing": f"CUDA-graph replay of the {nl} launches of one step, {kernel_loop.last['reps']} x {kernel_loop.last['passes']} passes back to back ({kernel_loop.last['seconds']:.1f} s), random operands, cold inputs cycling through 1 GiB, CUDA events on the launch stream",
                      "in_step_avg_us": kind_ms[dom] / kind_n[dom] * 1e3, "shapes": table})
     else:
         ach = kind_bytes[dom] / (kind_ms[dom] * 1e-3) / 1e9
