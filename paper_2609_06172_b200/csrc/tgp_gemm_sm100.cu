@@ -451,8 +451,10 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
     if (!sms) { int dev = 0; cudaGetDevice(&dev); if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148; }
     const uint32_t tiles_p = ((M + BM - 1) / BM) * ((n + P_BN - 1) / P_BN);
     const uint32_t tiles_q = ((M + 2 * BM - 1) / (2 * BM)) * ((n + P_BN - 1) / P_BN);
-    const bool paired = g_tc_variant == 3 || (g_tc_variant == 0 && tiles_q >= (uint32_t)sms);          // two tiles per pair of SMs or more
-    const bool persistent = !paired && (g_tc_variant == 2 || (g_tc_variant == 0 && tiles_p >= 2u * (uint32_t)sms));
+    // measured on 8192 x {640 .. 4096} x {4096, 14336}, {1024 .. 4096} x 4096 x 4096 and {512, 1024} x 8192 x 2048: the paired
+    // kernel is ahead as soon as every pair of SMs has a 256 x 256 tile, the persistent one from about 64 tiles of 128 x 256
+    const bool paired = g_tc_variant == 3 || (g_tc_variant == 0 && 2 * tiles_q >= (uint32_t)sms);
+    const bool persistent = !paired && (g_tc_variant == 2 || (g_tc_variant == 0 && tiles_p >= 64u));
     CUtensorMap ma, mb;
     if (!make_map(&ma, A, M, K, BM) || !make_map(&mb, W, n, K, paired ? P_BN / 2 : persistent ? P_BN : BN)) return TGP_E_CUDA;
     if (paired) {
