@@ -584,6 +584,24 @@ def test_whole_run_cuda_graph_replays_bit_identically():
     s.close()
 
 
+def test_whole_run_cuda_graph_with_cluster_launched_and_tma_kernels():
+    """Graph capture of a run whose prefill is large enough for the cluster-launched paired GEMM and the TMA-fed tcgen05
+    attention (tensor maps are kernel arguments baked into the graph): the replay equals the stepped run bit for bit."""
+    cfg = replace(si.CONFIGS[1], L=2, d=1024, F=4096, Hq=16, Hkv=4, V=8192, B=4, S=512, T=2, TK=128, budget_rule="half_w")
+    lay, pool, s, blobs, T = setup(cfg)
+    r = Runner(s, cfg.B * cfg.S)
+    prompt = torch.from_numpy(si.prompt_tokens(cfg)).pin_memory()
+    plain, toks = r.generate(prompt.numpy(), T)
+    r.capture_run(prompt, T)
+    for _ in range(2):
+        r.logits.zero_()
+        r.replay()
+        r.sync()
+        assert np.array_equal(r.logits.cpu().numpy(), plain[-1])
+    assert tb.k_gemm_status() == 0 and tb.k_attn_status() == 0
+    s.close()
+
+
 def test_edge_shapes_single_token_prompt_no_decode_and_maximum_tile_count():
     """Degenerate sizes: a prompt of one token with no decode step, and a context that needs all 64 KV tiles a kernel
     can address (TK = 1), both against the oracle; requests beyond the workspace or max_len are refused."""
