@@ -25,6 +25,8 @@ extern thread_local uint64_t tgpk_launches;
 
 #define CU(ctx, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return tgp_fail(ctx, TGP_E_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } while (0)
 
+static int g_small_copy_streams = 1;     // plans of small copies use three copy streams (0: always one)
+
 struct TgpEngine {
     // workspace carve-up
     int32_t *tok = nullptr, *amax = nullptr;
@@ -44,6 +46,16 @@ struct TgpEngine {
     cudaStream_t wb_stream = nullptr;
     bool wb_pending = false;                             // a write-back was recorded since the copy stream last waited
     int32_t copy_waited_op = -1;
+    // A plan made of small copies only (a pinned copy of 128 KiB moves at a third of the link rate: latency) spreads
+    // its H2D commands round-robin over the caller's copy stream and two library-owned ones, so that their latencies
+    // overlap; the streams meet at every op's last placement.  Large copies, and a run being captured into a graph,
+    // keep the one FIFO stream.
+    static constexpr int NCOPY = 3;
+    cudaStream_t xcopy[NCOPY - 1] = {nullptr, nullptr};
+    cudaEvent_t xmark[NCOPY] = {nullptr, nullptr, nullptr};
+    uint32_t n_copy = 1, rr = 0;
+    int32_t waited[NCOPY] = {-1, -1, -1};
+    bool wb_pend[NCOPY] = {false, false, false};
     size_t next_cmd = 0;
     uint32_t next_step = 0, pos = 0;
     const int32_t *tok_src = nullptr;
@@ -125,6 +137,8 @@ void tgp_engine_free(tgp_ctx *ctx) {
     if (e->graph_exec) cudaGraphExecDestroy(e->graph_exec);
     if (e->graph) cudaGraphDestroy(e->graph);
     for (cudaEvent_t ev : {e->fork_ev, e->join_cp, e->join_wb}) if (ev) cudaEventDestroy(ev);
+    for (cudaEvent_t ev : e->xmark) if (ev) cudaEventDestroy(ev);
+    for (cudaStream_t xs : e->xcopy) if (xs) cudaStreamDestroy(xs);
     if (e->wb_stream) cudaStreamDestroy(e->wb_stream);
     if (e->ecount_host) cudaFreeHost(e->ecount_host);
     delete e;
@@ -214,6 +228,8 @@ int tgp_model_bind(tgp_ctx *ctx, const tgp_model_cfg *cfg, const tgp_role_entry 
     CU(ctx, cudaEventCreate(&e->t0));
     CU(ctx, cudaEventCreate(&e->t1));
     CU(ctx, cudaStreamCreateWithFlags(&e->wb_stream, cudaStreamNonBlocking));
+    for (cudaStream_t &xs : e->xcopy) CU(ctx, cudaStreamCreateWithFlags(&xs, cudaStreamNonBlocking));
+    for (cudaEvent_t &ev : e->xmark) CU(ctx, cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
     return TGP_OK;
 }
 
@@ -222,6 +238,13 @@ int tgp_run_reset(tgp_ctx *ctx) {
     CU(ctx, cudaDeviceSynchronize());
     TgpEngine *e = ctx->eng;
     e->next_cmd = 0; e->next_step = 0; e->pos = 0; e->wb_pending = false; e->copy_waited_op = -1; e->tok_src = nullptr;
+    e->rr = 0;
+    for (int i = 0; i < TgpEngine::NCOPY; ++i) { e->waited[i] = -1; e->wb_pend[i] = false; }
+    {   // small-copy plans use all copy streams (decided per run: the plan may have changed)
+        uint64_t biggest = 0;
+        for (const TgpCmd &c : ctx->plan.cmds) if (c.kind == CMD_H2D && c.bytes > biggest) biggest = c.bytes;
+        e->n_copy = (ctx->plan.valid && biggest && biggest <= (512u << 10) && g_small_copy_streams) ? TgpEngine::NCOPY : 1;
+    }
     e->evict_at.clear();
     e->advised = false;                                  // the plan may have changed since the last run
     for (uint64_t &r : e->recent_objects) r = ~0ull;
@@ -255,6 +278,33 @@ static int pump(tgp_ctx *ctx, int32_t limit, cudaStream_t copy, uint32_t *n_cmds
             CU(ctx, cudaMemcpyAsync(host, dev, c.bytes, cudaMemcpyDeviceToHost, e->wb_stream));
             CU(ctx, cudaEventRecord(e->wb_ev, e->wb_stream));
             e->wb_pending = true;
+            for (bool &b : e->wb_pend) b = true;
+        } else if (e->n_copy > 1) {
+            // small copies: this command goes to the next of the copy streams; each stream keeps its own record of what
+            // it has already waited for
+            const uint32_t si = e->rr++ % e->n_copy;
+            cudaStream_t mine = si ? e->xcopy[si - 1] : copy;
+            if (c.wait_op > e->waited[si]) {
+                int rc = get_event(ctx, e->done_ev, (size_t)c.wait_op, &ev);
+                if (rc) return rc;
+                CU(ctx, cudaStreamWaitEvent(mine, ev, 0));
+                e->waited[si] = c.wait_op;
+            }
+            if (e->wb_pend[si]) { CU(ctx, cudaStreamWaitEvent(mine, e->wb_ev, 0)); e->wb_pend[si] = false; }
+            if (c.kind == CMD_H2D) CU(ctx, cudaMemcpyAsync(dev, host, c.bytes, cudaMemcpyHostToDevice, mine));
+            if (pl.op_last_place[c.first_use] == (int32_t)e->next_cmd) {
+                // commands are in first-use order, so everything the other streams hold is wanted by this op or an
+                // earlier one: this stream waits for what they hold now, and its event covers all of it
+                for (uint32_t sj = 0; sj < e->n_copy; ++sj) {
+                    if (sj == si) continue;
+                    cudaStream_t other = sj ? e->xcopy[sj - 1] : copy;
+                    CU(ctx, cudaEventRecord(e->xmark[sj], other));
+                    CU(ctx, cudaStreamWaitEvent(mine, e->xmark[sj], 0));
+                }
+                int rc = get_event(ctx, e->copied_ev, (size_t)c.first_use, &ev);
+                if (rc) return rc;
+                CU(ctx, cudaEventRecord(ev, mine));
+            }
         } else {
             if (c.wait_op > e->copy_waited_op) {
                 int rc = get_event(ctx, e->done_ev, (size_t)c.wait_op, &ev);
@@ -731,6 +781,7 @@ extern "C" int tgp_run_capture_begin(tgp_ctx *ctx, void *compute_stream, void *c
         if (ctx->plan.op_last_place[i] >= 0 && (rc = get_event(ctx, e->copied_ev, i, &ev))) return rc;
     }
     e->cap_cs = (cudaStream_t)compute_stream; e->cap_cp = (cudaStream_t)copy_stream;
+    e->n_copy = 1;                                       // in a graph the joins of several copy branches cost more than they hide (measured)
     CU(ctx, cudaStreamBeginCapture(e->cap_cs, cudaStreamCaptureModeRelaxed));
     // fork: the copy and write-back streams join the capture
     cudaError_t er = cudaEventRecord(e->fork_ev, e->cap_cs);
