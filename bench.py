@@ -529,6 +529,16 @@ def main():
         planned, used = np.asarray(counts[:n]) > 0, np.asarray(ran[:n]) > 0
         moe_prediction = {"expert_slots_planned": int(planned.sum()), "planned_but_unused": int((planned & ~used).sum()),
                           "used_but_unplanned": int((~planned & used).sum()), "slots": int(planned.size)}
+        # realised popularity: share of routed (token, slot) pairs by the expert's rank in its layer's bias, beside the
+        # Zipf law the bias encodes for the first choice (top-2 routing flattens it: the second choice is someone else)
+        order = np.argsort(-np.asarray(bias), axis=1)                                   # [L, E]: experts by falling bias
+        by_rank = np.zeros(cfg.E)
+        tot = np.asarray(ran[:n], dtype=np.float64).sum(axis=0)                          # [L, E]
+        for l in range(cfg.L):
+            by_rank += tot[l][order[l]]
+        zipf = np.array([r ** (-cfg.zipf_s) for r in range(1, cfg.E + 1)])
+        moe_prediction["routed_share_by_bias_rank"] = [round(float(x), 4) for x in by_rank / max(1.0, by_rank.sum())]
+        moe_prediction["zipf_first_choice"] = [round(float(x), 4) for x in zipf / zipf.sum()]
 
     if rank != 0:
         if dist is not None:
