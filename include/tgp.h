@@ -191,7 +191,8 @@ int  tgp_run_reset(tgp_ctx *ctx);
 /* Runs the next step of the plan: enqueues its copies on copy_stream and its kernels on compute_stream and
  * returns without waiting unless stats != NULL.  tokens_host [B, q_len] int32, or NULL in a decode step to
  * feed the previous step's argmax, which stays on the device.  logits_dev [B, V] fp32 of the last position;
- * argmax_dev [B] int32 or NULL. */
+ * argmax_dev [B] int32 or NULL.  With stats the step is waited for, and TGP_E_CUDA is returned if a tensor-core kernel
+ * of this process has recorded a bounded wait that ran out (tgp_k_gemm_status / tgp_k_attn_status). */
 int  tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_host, uint32_t B, uint32_t q_len,
               float *logits_dev, int32_t *argmax_dev, void *compute_stream, void *copy_stream,
               tgp_step_stats *stats);

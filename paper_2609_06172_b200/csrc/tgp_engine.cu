@@ -687,6 +687,10 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
         stats->h2d_bytes = ring ? tot[0] : objects ? object_bytes_asked : 0; stats->d2h_bytes = ring ? tot[1] : 0; stats->zc_bytes = objects ? 0 : tot[2];
         stats->n_cmds = n_cmds; stats->n_launches = (uint32_t)(tgpk_launches - launches0); stats->n_mismatch = n_mismatch;
         CU(ctx, cudaEventElapsedTime(&stats->step_ms, e->t0, e->t1));
+        // the step has been waited for: a tensor-core kernel whose bounded wait ran out has left its mark
+        int gemm_err = 0, attn_err = 0;
+        if (tgp_k_gemm_status(&gemm_err) == TGP_OK && tgp_k_attn_status(&attn_err) == TGP_OK && (gemm_err || attn_err))
+            return tgp_fail(ctx, TGP_E_CUDA, "a tensor-core kernel gave up on a bounded wait (GEMM code " + std::to_string(gemm_err) + ", attention code " + std::to_string(attn_err) + "): results of this step are incomplete");
     }
     return TGP_OK;
 }
