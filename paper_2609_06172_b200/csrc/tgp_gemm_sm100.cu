@@ -3,7 +3,7 @@
 // tile per CTA (below), a persistent kernel with 128 x 256 tiles and double-buffered accumulators, and - for the large
 // products of a prefill - a kernel in which the two CTAs of a cluster share 256 x 256 tiles through the two-SM MMA.
 //
-// One CTA computes a 128 x BN tile.  Warp 0 (one lane) feeds a 3-stage shared-memory ring with TMA
+// One CTA computes a 128 x BN tile.  Warp 0 (one lane) feeds a shared-memory ring of ST stages with TMA
 // (128-byte swizzle, 64 bf16 of K per stage); warp 1 (one lane) issues tcgen05.mma (M=128, N=BN, K=16,
 // four per stage) into a TMEM accumulator and releases stages with tcgen05.commit; warps 2-5 wait for the
 // last commit, read the accumulator with tcgen05.ld (each warp its own 32-lane quarter) and store fp32 rows.
@@ -21,22 +21,23 @@
 namespace {
 
 using namespace tgp_sm100;
-constexpr int BK = 64, STAGES = 3, GROUP_M = 16;
+constexpr int BK = 64, GROUP_M = 16;
 
 __device__ int g_gemm_tc_error = 0;                    // 0 ok; else (role << 8) | stage of the first wait that ran out
 
-template <int BN>
+template <int BN, int ST>
 struct Smem {
     static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int BAR_OFF = STAGES * STAGE_BYTES;
-    static constexpr int TOTAL = BAR_OFF + 128 + 1024;        // barriers + slack to align the base to 1024 bytes
+    static constexpr int BAR_OFF = ST * STAGE_BYTES;
+    static constexpr int TOTAL = BAR_OFF + 256 + 1024;        // barriers (2 * ST + 1, TMEM slot, flag) + slack to align the base to 1024 bytes
 };
 
-template <int BN>
+template <int BN, int ST>
 __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                                                       float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     extern __shared__ uint8_t smem_raw[];
-    using S = Smem<BN>;
+    using S = Smem<BN, ST>;
+    constexpr int STAGES = ST;                      // depth of this instantiation's TMA ring
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + S::BAR_OFF);
     uint64_t *empty = full + STAGES;
@@ -441,6 +442,18 @@ bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t K, uin
 
 extern thread_local uint64_t tgpk_launches;
 
+template <int BN, int ST>
+static bool launch_tile(const CUtensorMap &ma, const CUtensorMap &mb, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(gemm_tc_kernel<BN, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN, ST>::TOTAL) != cudaSuccess) return false;
+        attr_set = true;
+    }
+    dim3 grid(((M + BM - 1) / BM) * ((n + BN - 1) / BN));
+    gemm_tc_kernel<BN, ST><<<grid, 192, Smem<BN, ST>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
+    return true;
+}
+
 static int g_tc_variant = 0;     // 0 auto, 1 force the 128x128 per-tile kernel, 2 the persistent 128x256 kernel, 3 the paired 256x256 kernel
 
 int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
@@ -455,8 +468,15 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
     // kernel is ahead as soon as every pair of SMs has a 256 x 256 tile, the persistent one from about 64 tiles of 128 x 256
     const bool paired = g_tc_variant == 3 || (g_tc_variant == 0 && 2 * tiles_q >= (uint32_t)sms);
     const bool persistent = !paired && (g_tc_variant == 2 || (g_tc_variant == 0 && tiles_p >= 64u));
+    // small problems, one tile per CTA: an MMA into one accumulator costs the same 75 cycles for N = 32 as for N = 128, so
+    // a CTA's time is set by its K loop, and narrower tiles simply put more CTAs to work: the widest tile that still
+    // gives every SM one
+    const uint32_t tm = (M + BM - 1) / BM;
+    uint32_t bn = BN;
+    // ... as long as the A panel is not re-read by more than 32 column tiles (L2 bandwidth then takes over)
+    if (g_tc_variant == 0) while (bn > 32 && tm * ((n + bn - 1) / bn) < (uint32_t)sms && (n + bn / 2 - 1) / (bn / 2) <= 32) bn /= 2;
     CUtensorMap ma, mb;
-    if (!make_map(&ma, A, M, K, BM) || !make_map(&mb, W, n, K, paired ? P_BN / 2 : persistent ? P_BN : BN)) return TGP_E_CUDA;
+    if (!make_map(&ma, A, M, K, BM) || !make_map(&mb, W, n, K, paired ? P_BN / 2 : persistent ? P_BN : bn)) return TGP_E_CUDA;
     if (paired) {
         constexpr int SMEM = Q_STAGES * Q_HALVES * (BM * BK * 2 + (P_BN / 2) * BK * 2) + 160 + 1024;
         static bool attr_q = false;
@@ -484,14 +504,15 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
             attr_p = true;
         }
         gemm_tc_persistent_kernel<<<tiles_p < (uint32_t)sms ? tiles_p : (uint32_t)sms, 192, SMEM, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
+    } else if (bn == 128) {
+        // fewer tiles than SMs: one CTA per SM, so the ring may take all of shared memory (a 3-stage ring leaves a lone
+        // CTA waiting on L2 latency); otherwise two CTAs per SM with three stages each
+        const bool lone = tm * ((n + 127) / 128) <= (uint32_t)sms;
+        if (!(lone ? launch_tile<128, 6>(ma, mb, C, M, n, K, ldc, col0, accumulate, st) : launch_tile<128, 3>(ma, mb, C, M, n, K, ldc, col0, accumulate, st))) return TGP_E_CUDA;
+    } else if (bn == 64) {
+        if (!launch_tile<64, 8>(ma, mb, C, M, n, K, ldc, col0, accumulate, st)) return TGP_E_CUDA;
     } else {
-        static bool attr_set = false;
-        if (!attr_set) {
-            if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN>::TOTAL) != cudaSuccess) return TGP_E_CUDA;
-            attr_set = true;
-        }
-        dim3 grid(((M + BM - 1) / BM) * ((n + BN - 1) / BN));
-        gemm_tc_kernel<BN><<<grid, 192, Smem<BN>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
+        if (!launch_tile<32, 8>(ma, mb, C, M, n, K, ldc, col0, accumulate, st)) return TGP_E_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return TGP_E_CUDA;
     tgpk_launches += 1;
