@@ -638,7 +638,7 @@ def main():
            "gpu_launches": launches * args.steps, "clocks": clocks, "roofline": roof, "step_roofline": step_roof,
            "kernels": {f"{k[0]}:{k[1]}": {"ms": round(v, 3), "launches": kind_n[k], "GBps": round(kind_bytes[k] / (v * 1e-3) / 1e9, 1),
                                            "TFLOPs": round(kind_flops[k] / (v * 1e-3) / 1e12, 2)} for k, v in sorted(kind_ms.items())}}
-    if not args.no_uvm:
+    if not args.no_uvm and world == 1:                 # the baselines are single-GPU measurements: reported at N = 1 only
         try:
             from paper_2609_06172_b200 import uvm_baseline
             del r
@@ -663,7 +663,7 @@ def main():
                                             "explicit_ring_speedup": mo.get("explicit_ring_speedup_decode")}
         except Exception as ex:  # the baseline is reported, never fatal
             out["uvm"] = f"not run: {type(ex).__name__}: {ex}"
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:
         om = make_oracle(lay, oracle_weights_from_pool(lay, pool.numpy()))
         sS, sT = oracle_sample(cfg, lay)
         time_oracle(lay, om, min(16, sS), 1)
