@@ -25,18 +25,19 @@ constexpr int BK = 64, GROUP_M = 16;
 
 __device__ int g_gemm_tc_error = 0;                    // 0 ok; else (role << 8) | stage of the first wait that ran out
 
-template <int BN, int ST>
+template <int BN, int ST, int KH>
 struct Smem {
-    static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, HALF_BYTES = A_BYTES + B_BYTES, STAGE_BYTES = KH * HALF_BYTES;
     static constexpr int BAR_OFF = ST * STAGE_BYTES;
     static constexpr int TOTAL = BAR_OFF + 256 + 1024;        // barriers (2 * ST + 1, TMEM slot, flag) + slack to align the base to 1024 bytes
 };
 
-template <int BN, int ST>
+// (ST stages of KH 64-wide K blocks each: with KH = 2 the producer and the MMA thread meet half as often)
+template <int BN, int ST, int KH>
 __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                                                       float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     extern __shared__ uint8_t smem_raw[];
-    using S = Smem<BN, ST>;
+    using S = Smem<BN, ST, KH>;
     constexpr int STAGES = ST;                      // depth of this instantiation's TMA ring
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + S::BAR_OFF);
@@ -53,7 +54,7 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
     const uint32_t rows_in_group = min((uint32_t)GROUP_M, tiles_m - first_m);
     const uint32_t in_group = blockIdx.x - group * GROUP_M * tiles_n;
     const uint32_t m0 = (first_m + in_group % rows_in_group) * BM, n0 = (in_group / rows_in_group) * BN;
-    const uint32_t num_k = (K + BK - 1) / BK;
+    const uint32_t num_k = (K + KH * BK - 1) / (KH * BK);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -77,8 +78,11 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
                 const uint32_t s = kb % STAGES, ph = (kb / STAGES) & 1;
                 if (*failed || !mbar_wait(&empty[s], ph ^ 1, failed)) { if (!*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, (1 << 8) | (int)s); } break; }
                 mbar_expect_tx(&full[s], S::STAGE_BYTES);
-                tma_load_2d(smem + s * S::STAGE_BYTES, &tmA, (int)(kb * BK), (int)m0, &full[s]);
-                tma_load_2d(smem + s * S::STAGE_BYTES + S::A_BYTES, &tmB, (int)(kb * BK), (int)n0, &full[s]);
+#pragma unroll
+                for (int h = 0; h < KH; ++h) {
+                    tma_load_2d(smem + s * S::STAGE_BYTES + h * S::HALF_BYTES, &tmA, (int)((kb * KH + h) * BK), (int)m0, &full[s]);
+                    tma_load_2d(smem + s * S::STAGE_BYTES + h * S::HALF_BYTES + S::A_BYTES, &tmB, (int)((kb * KH + h) * BK), (int)n0, &full[s]);
+                }
                 armed = kb + 1;
             }
             if (*failed) {
@@ -95,10 +99,13 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
                 const uint32_t s = kb % STAGES, ph = (kb / STAGES) & 1;
                 if (*failed || !mbar_wait(&full[s], ph, failed)) { if (!*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, (2 << 8) | (int)s); } ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint64_t da = umma_desc(smem_u32(smem + s * S::STAGE_BYTES));
-                const uint64_t db = umma_desc(smem_u32(smem + s * S::STAGE_BYTES + S::A_BYTES));
 #pragma unroll
-                for (uint32_t k = 0; k < BK / 16; ++k) umma(tmem_base, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);   // +32 bytes of K per step
+                for (uint32_t h = 0; h < KH; ++h) {
+                    const uint64_t da = umma_desc(smem_u32(smem + s * S::STAGE_BYTES + h * S::HALF_BYTES));
+                    const uint64_t db = umma_desc(smem_u32(smem + s * S::STAGE_BYTES + h * S::HALF_BYTES + S::A_BYTES));
+#pragma unroll
+                    for (uint32_t k = 0; k < BK / 16; ++k) umma(tmem_base, da + 2 * k, db + 2 * k, idesc, (kb | h | k) != 0);   // +32 bytes of K per step
+                }
                 umma_commit(&empty[s]);
             }
             if (ok) umma_commit(acc_full);
@@ -442,15 +449,15 @@ bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t K, uin
 
 extern thread_local uint64_t tgpk_launches;
 
-template <int BN, int ST>
+template <int BN, int ST, int KH>
 static bool launch_tile(const CUtensorMap &ma, const CUtensorMap &mb, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(gemm_tc_kernel<BN, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN, ST>::TOTAL) != cudaSuccess) return false;
+        if (cudaFuncSetAttribute(gemm_tc_kernel<BN, ST, KH>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN, ST, KH>::TOTAL) != cudaSuccess) return false;
         attr_set = true;
     }
     dim3 grid(((M + BM - 1) / BM) * ((n + BN - 1) / BN));
-    gemm_tc_kernel<BN, ST><<<grid, 192, Smem<BN, ST>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
+    gemm_tc_kernel<BN, ST, KH><<<grid, 192, Smem<BN, ST, KH>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
     return true;
 }
 
@@ -508,11 +515,11 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
         // fewer tiles than SMs: one CTA per SM, so the ring may take all of shared memory (a 3-stage ring leaves a lone
         // CTA waiting on L2 latency); otherwise two CTAs per SM with three stages each
         const bool lone = tm * ((n + 127) / 128) <= (uint32_t)sms;
-        if (!(lone ? launch_tile<128, 6>(ma, mb, C, M, n, K, ldc, col0, accumulate, st) : launch_tile<128, 3>(ma, mb, C, M, n, K, ldc, col0, accumulate, st))) return TGP_E_CUDA;
+        if (!(lone ? launch_tile<128, 2, 3>(ma, mb, C, M, n, K, ldc, col0, accumulate, st) : launch_tile<128, 3, 1>(ma, mb, C, M, n, K, ldc, col0, accumulate, st))) return TGP_E_CUDA;
     } else if (bn == 64) {
-        if (!launch_tile<64, 8>(ma, mb, C, M, n, K, ldc, col0, accumulate, st)) return TGP_E_CUDA;
+        if (!launch_tile<64, 3, 3>(ma, mb, C, M, n, K, ldc, col0, accumulate, st)) return TGP_E_CUDA;
     } else {
-        if (!launch_tile<32, 8>(ma, mb, C, M, n, K, ldc, col0, accumulate, st)) return TGP_E_CUDA;
+        if (!launch_tile<32, 3, 3>(ma, mb, C, M, n, K, ldc, col0, accumulate, st)) return TGP_E_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return TGP_E_CUDA;
     tgpk_launches += 1;
