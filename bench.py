@@ -129,8 +129,15 @@ def gemm_shapes_of_step(lay, M):
     cfg = lay.cfg
     out = []
     for l in range(cfg.L):
-        for kind, res in ((si.K_WQ, 0), (si.K_WK, 0), (si.K_WV, 0), (si.K_WO, 1)):
-            out += [(t.rows, t.cols, res, M) for t in lay.blocks(kind, l)]
+        qkv = [lay.blocks(kind, l) for kind in (si.K_WQ, si.K_WK, si.K_WV)]
+        if (M <= 2 and all(len(b) == 1 for b in qkv) and len({b[0].cols for b in qkv}) == 1 and qkv[0][0].cols < 8192
+                and sum(b[0].rows for b in qkv) < 2 * 148 * 16):
+            # the step runs these three as one launch (tgp_k_gemm_group's rule): n is the tuple of their row counts
+            out.append((tuple(b[0].rows for b in qkv), qkv[0][0].cols, 0, M))
+        else:
+            for b in qkv:
+                out += [(t.rows, t.cols, 0, M) for t in b]
+        out += [(t.rows, t.cols, 1, M) for t in lay.blocks(si.K_WO, l)]
         for e in (range(cfg.E) if cfg.E else (-1,)):          # MoE: tokens spread evenly over the experts (top-k picks each)
             me = M if not cfg.E else max(1, M * cfg.topk // cfg.E)
             for kind, res in ((si.K_WG, 0), (si.K_WU, 0), (si.K_WD, 0 if cfg.E else 1)):
@@ -156,8 +163,9 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
     for o in range(0, w16.numel(), 1 << 26):
         c = min(1 << 26, w16.numel() - o)
         w16[o:o + c] = (torch.randn(c, device=device, generator=gen) * 0.02).bfloat16()
+    rows_of = lambda n: sum(n) if isinstance(n, tuple) else n
     kmax = max(k for (_, k, _, _) in shapes)
-    nmax = max(n for (n, _, _, _) in shapes)
+    nmax = max(rows_of(n) for (n, _, _, _) in shapes)
     mmax = max(m for (_, _, _, m) in shapes)
     A = torch.randn((mmax, kmax), device=device, generator=gen).bfloat16()
     Cbuf = torch.zeros((mmax, nmax), dtype=torch.float32, device=device)
@@ -169,10 +177,15 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
         for (n, K, res, m) in shapes:
             if only is not None and (n, K, res, m) != only:
                 continue
-            nb = (n * K * 2 + 511) // 512 * 512
+            nb = (rows_of(n) * K * 2 + 511) // 512 * 512
             if off + nb > cold_bytes:
                 off = 0
-            tb.k_gemm(A, wbuf.data_ptr() + off, Cbuf, m, n, K, nmax, 0, res, st)
+            if isinstance(n, tuple):
+                starts = [sum(n[:i]) for i in range(len(n))]
+                tb.k_gemm_group(A, [wbuf.data_ptr() + off + r0 * K * 2 for r0 in starts], [Cbuf.data_ptr() + r0 * 4 for r0 in starts],
+                                m, list(n), K, [nmax] * len(n), st)
+            else:
+                tb.k_gemm(A, wbuf.data_ptr() + off, Cbuf, m, n, K, nmax, 0, res, st)
             off += nb
 
     def graph_of(only=None, passes=4):
@@ -208,18 +221,20 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
     n_rep, total_s = bounded(g, 4.0)
     kernel_loop.last = {"reps": n_rep, "passes": passes, "seconds": total_s}
     sec = total_s / (n_rep * passes * len(shapes))
-    bytes_per = sum(2 * m * K + 2 * K * n + 4 * m * n * (2 if res else 1) for (n, K, res, m) in shapes) / len(shapes)
-    flops_per = sum(2 * m * K * n for (n, K, res, m) in shapes) / len(shapes)
+    bytes_per = sum(2 * m * K + 2 * K * rows_of(n) + 4 * m * rows_of(n) * (2 if res else 1) for (n, K, res, m) in shapes) / len(shapes)
+    flops_per = sum(2 * m * K * rows_of(n) for (n, K, res, m) in shapes) / len(shapes)
     table = {}
-    for sh in sorted(set(shapes)):
+    for sh in sorted(set(shapes), key=lambda q: (rows_of(q[0]),) + tuple(q[1:])):
         cnt = shapes.count(sh)
         g, passes = graph_of(only=sh)
         n_sh, t_sh = bounded(g, 1.0)
         t = t_sh / (n_sh * passes * cnt)
         n, K, res, m = sh
-        b = 2 * m * K + 2 * K * n + 4 * m * n * (2 if res else 1)
-        table[f"n={n} K={K} M={m} res={res}"] = {"launches_per_step": cnt, "us": round(t * 1e6, 2), "GBps": round(b / t / 1e9, 1),
-                                                   "TFLOPs": round(2 * m * K * n / t / 1e12, 2)}
+        nr = rows_of(n)
+        b = 2 * m * K + 2 * K * nr + 4 * m * nr * (2 if res else 1)
+        name = "+".join(str(x) for x in n) if isinstance(n, tuple) else str(n)
+        table[f"n={name} K={K} M={m} res={res}"] = {"launches_per_step": cnt, "us": round(t * 1e6, 2), "GBps": round(b / t / 1e9, 1),
+                                                      "TFLOPs": round(2 * m * K * nr / t / 1e12, 2)}
     return sec, bytes_per, flops_per, len(shapes), table
 
 

@@ -257,6 +257,17 @@ int  tgp_k_rmsnorm(const float *x_dev, uint32_t ldx, const void *g_dev, void *h_
  * block), C fp32 with row stride ldc.  accumulate != 0 adds to C (fused residual).  K % 8 == 0. */
 int  tgp_k_gemm(const void *A_dev, const void *W_dev, float *C_dev, uint32_t M, uint32_t n, uint32_t K,
                 uint32_t ldc, uint32_t col0, int accumulate, void *stream);
+/* Several products over the same activations in one call (the q, k and v projections of a decode step, Section II-B's
+ * kernel sequence): C_dev[s][m, j] = sum_k A[m, k] * W_dev[s][j, k] for s < count <= TGP_GEMM_GROUP_MAX, W_dev[s] bf16
+ * [n[s], K], C_dev[s] fp32 with row stride ldc[s] >= n[s].  The pointer and size arrays are host arrays of device
+ * pointers, read before the call returns.  For M <= 2 with fewer than 4736 rows in total and K < 8192 one launch serves
+ * all parts; otherwise the parts are launched one after the other.  The results are bit-identical to tgp_k_gemm() per
+ * part either way.  tgp_k_gemm_group_select(0) forces one launch per part (process-wide; default 1), also inside
+ * tgp_step(), which groups the q, k and v projections of a layer this way when no tap or op timing is set. */
+#define TGP_GEMM_GROUP_MAX 4u
+int  tgp_k_gemm_group(const void *A_dev, uint32_t count, const void *const *W_dev, float *const *C_dev, const uint32_t *n,
+                      const uint32_t *ldc, uint32_t M, uint32_t K, void *stream);
+int  tgp_k_gemm_group_select(int enable);
 /* Which kernel serves M > 16: 0 (default) the tcgen05 tensor-core GEMM, 1 the CUDA-core tile kernel (an on-device
  * cross-check).  M <= 16 always takes the weight-streaming GEMV.  Process-wide. */
 int  tgp_k_gemm_select(int impl);

@@ -96,6 +96,8 @@ _SIGS = {
     "tgp_k_embed": [_P, _P, _P, _U32, _U32, _P],
     "tgp_k_rmsnorm": [_P, _U32, _P, _P, _U32, _U32, C.c_float, _P],
     "tgp_k_gemm": [_P, _P, _P, _U32, _U32, _U32, _U32, _U32, C.c_int, _P],
+    "tgp_k_gemm_group": [_P, _U32, _P, _P, C.POINTER(_U32), C.POINTER(_U32), _U32, _U32, _P],
+    "tgp_k_gemm_group_select": [C.c_int],
     "tgp_k_gemm_select": [C.c_int],
     "tgp_k_attn_select": [C.c_int],
     "tgp_k_gemv_overlap": [C.c_int],
@@ -360,6 +362,17 @@ def k_rmsnorm(x, ldx, g, h, M, d, eps, stream=None):
 
 def k_gemm(A, W, Cout, M, n, K, ldc, col0, accumulate, stream=None):
     _k(lib().tgp_k_gemm(_ptr(A), _ptr(W), _ptr(Cout), M, n, K, ldc, col0, int(accumulate), _ptr(stream)), "tgp_k_gemm")
+
+
+def k_gemm_group(A, Ws, Couts, M, ns, K, ldcs, stream=None):
+    """Products of the same activations A [M, K] with several weight blocks Ws[s] [ns[s], K] into Couts[s] (row stride ldcs[s])."""
+    c = len(Ws)
+    _k(lib().tgp_k_gemm_group(_ptr(A), c, (_P * c)(*[_ptr(w) for w in Ws]), (_P * c)(*[_ptr(o) for o in Couts]),
+                              (_U32 * c)(*ns), (_U32 * c)(*ldcs), M, K, _ptr(stream)), "tgp_k_gemm_group")
+
+
+def k_gemm_group_select(enable):
+    _k(lib().tgp_k_gemm_group_select(int(enable)), "tgp_k_gemm_group_select")
 
 
 def k_gemm_select(impl):

@@ -531,12 +531,32 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
     const uint32_t qd = c.Hq * c.Dh, kd = c.Hkv * c.Dh;
     for (uint32_t i = st.op0; i < st.op0 + st.nops; ++i) {
         const TgpOp &o = ctx->ops[i];
-        if ((ring || hints) && ctx->plan.op_last_place[i] >= 0) {
-            if ((size_t)ctx->plan.op_last_place[i] >= e->next_cmd) return tgp_fail(ctx, TGP_E_STATE, "a placement was not enqueued before its op");
-            cudaEvent_t ev;
-            if ((rc = get_event(ctx, e->copied_ev, i, &ev))) return rc;
-            CU(ctx, cudaStreamWaitEvent(cs, ev, 0));
+        // The q, k and v projections of a layer read the same activations: when each is one whole tensor, their copies
+        // have all been enqueued already and one launch can serve the three, ops [i, i + 3) run as one launch.
+        uint32_t span = 1, gn[3] = {0, 0, 0}, gK = 0;
+        if (ring && o.kind == TGP_OP_GEMM && M <= 2 && !e->op_timing && !e->tap && i + 2 < st.op0 + st.nops) {
+            bool ok = true;
+            for (uint32_t j = 0; j < 3 && ok; ++j) {
+                const TgpOp &f = ctx->ops[i + j];
+                ok = f.kind == TGP_OP_GEMM && f.layer == o.layer && f.nacc >= 1;
+                const int32_t ri = ok ? ctx->role_of_tensor[ctx->acc[f.acc0].tensor] : -1;
+                if (!(ok = ok && ri >= 0)) break;
+                const TgpRole &r = ctx->roles[ri];
+                const uint32_t Kj = r.rows ? (uint32_t)(ctx->tensors[ctx->acc[f.acc0].tensor].size / (2ull * r.rows)) : 0;
+                ok = r.kind == (j == 0 ? TGP_K_WQ : j == 1 ? TGP_K_WK : TGP_K_WV) && r.expert < 0 && r.row0 == 0 && r.rows == (j == 0 ? qd : kd) &&
+                     (j == 0 || Kj == gK) && (ctx->plan.op_last_place[i + j] < 0 || (size_t)ctx->plan.op_last_place[i + j] < e->next_cmd);
+                gn[j] = r.rows;
+                gK = Kj;
+            }
+            if (ok && tgpk_gemm_group_fused(3, gn, M, gK)) span = 3;
         }
+        for (uint32_t j = i; j < i + span; ++j)
+            if ((ring || hints) && ctx->plan.op_last_place[j] >= 0) {
+                if ((size_t)ctx->plan.op_last_place[j] >= e->next_cmd) return tgp_fail(ctx, TGP_E_STATE, "a placement was not enqueued before its op");
+                cudaEvent_t ev;
+                if ((rc = get_event(ctx, e->copied_ev, j, &ev))) return rc;
+                CU(ctx, cudaStreamWaitEvent(cs, ev, 0));
+            }
         const uint32_t ti = i - st.op0;
         if (e->op_timing) {
             if (e->ta.size() <= ti) { e->ta.resize(ti + 1, nullptr); e->tb_.resize(ti + 1, nullptr); }
@@ -561,6 +581,13 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             const TgpRole &r = ctx->roles[ri];
             const uint32_t K = (uint32_t)(ctx->tensors[a.tensor].size / (2ull * r.rows));
             const void *W = where(ctx, o, 0);
+            if (span == 3) {
+                const void *gW[3] = {W, where(ctx, ctx->ops[i + 1], 0), where(ctx, ctx->ops[i + 2], 0)};
+                float *gC[3] = {e->q32, e->k32, e->v32};
+                const uint32_t gld[3] = {qd, kd, kd};
+                rc = tgpk_gemm_group(e->h, 3, gW, gC, gn, gld, M, K, cs);
+                break;
+            }
             if (r.expert >= 0) {                          // expert weight block: rows of the tokens routed to that expert
                 if ((uint32_t)r.expert >= c.E || !c.E) return tgp_fail(ctx, TGP_E_MISMATCH, "expert weight in a dense model");
                 e->cur_expert = r.expert;
@@ -663,12 +690,15 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
         }
         if (e->op_timing) CU(ctx, cudaEventRecord(e->tb_[ti], cs));
         if (ring) {
-            if (ctx->plan.op_is_wait_target[i]) {
-                cudaEvent_t ev;
-                if ((rc = get_event(ctx, e->done_ev, i, &ev))) return rc;
-                CU(ctx, cudaEventRecord(ev, cs));
+            for (uint32_t j = i; j < i + span; ++j) {
+                if (ctx->plan.op_is_wait_target[j]) {
+                    cudaEvent_t ev;
+                    if ((rc = get_event(ctx, e->done_ev, j, &ev))) return rc;
+                    CU(ctx, cudaEventRecord(ev, cs));
+                }
+                if ((rc = pump(ctx, (int32_t)j, cp, &n_cmds))) return rc;
             }
-            if ((rc = pump(ctx, (int32_t)i, cp, &n_cmds))) return rc;
+            i += span - 1;
         } else if (hints) {
             if ((rc = after_op_managed(ctx, i, cs))) return rc;
             if ((rc = pump_managed(ctx, (int32_t)i, cp, &n_cmds))) return rc;

@@ -91,12 +91,6 @@ __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, c
         const bf16 *wrow[R];
 #pragma unroll
         for (int r = 0; r < R; ++r) wrow[r] = W + (size_t)min(row0 + r, n - 1) * K;   // tail rows re-read the last row, never stored
-        // the value this product is added to: lane r * MT + m fetches it as early as the protocol allows, so that its
-        // latency hides behind the weight stream instead of following it
-        float cprev = 0.f;
-        const bool mine = accumulate && lane < R * MT && row0 + lane / MT < n && lane % MT < Mrows;
-        const float *cptr = C + (size_t)(lane % MT) * ldc + col0 + row0 + lane / MT;
-        if (synced && mine) cprev = *cptr;
         for (uint32_t k0 = lane * 8; k0 < K; k0 += 256 * U) {
             uint4 wv[U][R];
 #pragma unroll
@@ -104,7 +98,7 @@ __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, c
 #pragma unroll
                 for (int r = 0; r < R; ++r)
                     wv[u][r] = (k0 + 256 * u < K) ? __ldcs(reinterpret_cast<const uint4 *>(wrow[r] + k0 + 256 * u)) : make_uint4(0, 0, 0, 0);
-            if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; if (mine) cprev = *cptr; }
+            if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const uint32_t k = k0 + 256 * u;
@@ -122,15 +116,73 @@ __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, c
                 }
             }
         }
-        if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; if (mine) cprev = *cptr; }      // K == 0 never happens; belt and braces
+        if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }      // K == 0 never happens; belt and braces
+        // a product added to the residual stream goes out as a reduction (one add per element, by one thread: the same
+        // rounded sum as load, add, store, and deterministic) that nothing waits for: the launch ends a memory round trip sooner
 #pragma unroll
         for (int r = 0; r < R; ++r)
 #pragma unroll
             for (int m = 0; m < MT; ++m) {
                 const float s = warp_sum(acc[r][m]);
-                if ((int)lane == r * MT + m && row0 + r < n && m < (int)Mrows)
-                    C[(size_t)m * ldc + col0 + row0 + r] = accumulate ? cprev + s : s;
+                if ((int)lane == r * MT + m && row0 + r < n && m < (int)Mrows) {
+                    if (accumulate) atomicAdd(&C[(size_t)m * ldc + col0 + row0 + r], s);
+                    else C[(size_t)m * ldc + col0 + row0 + r] = s;
+                }
             }
+    }
+}
+
+// Several products that read the same activations (the q, k and v projections of a layer) in one launch: the output
+// rows of the parts are walked as one list, one warp per row, with exactly the arithmetic of gemv_kernel<MT, 1, U>, so
+// the result is bit-identical to separate launches; what is saved is two launch floors of about a microsecond each.
+struct GemvParts { const bf16 *W[TGP_GEMM_GROUP_MAX]; float *C[TGP_GEMM_GROUP_MAX]; uint32_t n[TGP_GEMM_GROUP_MAX], ldc[TGP_GEMM_GROUP_MAX], count; };
+
+template <int MT, int U>
+__global__ void __launch_bounds__(256) gemv_group_kernel(const bf16 *__restrict__ A, const GemvParts p, uint32_t Mrows, uint32_t n_total, uint32_t K) {
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarp = (gridDim.x * blockDim.x) >> 5;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    bool synced = false;
+    for (uint32_t row = gwarp; row < n_total; row += nwarp) {
+        const bf16 *W = p.W[0];
+        float *C = p.C[0];
+        uint32_t ldc = p.ldc[0], r = row, start = p.n[0];
+#pragma unroll
+        for (int s = 1; s < TGP_GEMM_GROUP_MAX; ++s)
+            if (s < (int)p.count) {
+                if (row >= start) { W = p.W[s]; C = p.C[s]; ldc = p.ldc[s]; r = row - start; }
+                start += p.n[s];
+            }
+        const bf16 *wrow = W + (size_t)r * K;
+        float acc[MT];
+#pragma unroll
+        for (int m = 0; m < MT; ++m) acc[m] = 0.f;
+        for (uint32_t k0 = lane * 8; k0 < K; k0 += 256 * U) {
+            uint4 wv[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                wv[u] = (k0 + 256 * u < K) ? __ldcs(reinterpret_cast<const uint4 *>(wrow + k0 + 256 * u)) : make_uint4(0, 0, 0, 0);
+            if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t k = k0 + 256 * u;
+                float wf[8];
+                unpack8(wv[u], wf);
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    float xf[8];
+                    unpack8((k < K && m < (int)Mrows) ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)) : make_uint4(0, 0, 0, 0), xf);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) acc[m] = fmaf(wf[i], xf[i], acc[m]);
+                }
+            }
+        }
+        if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            const float s = warp_sum(acc[m]);
+            if ((int)lane == m && m < (int)Mrows) C[(size_t)m * ldc + r] = s;
+        }
     }
 }
 
@@ -154,10 +206,7 @@ __global__ void __launch_bounds__(256) gemv_splitk_kernel(const bf16 *__restrict
         const bf16 *wrow[RB];
 #pragma unroll
         for (int r = 0; r < RB; ++r) wrow[r] = W + (size_t)min(row0 + r, n - 1) * K;
-        float cprev = 0.f;
         const bool mine = threadIdx.x < RB * MT && row0 + threadIdx.x / MT < n && threadIdx.x % MT < Mrows;
-        const float *cptr = C + (size_t)(threadIdx.x % MT) * ldc + col0 + row0 + threadIdx.x / MT;
-        if (synced && mine && accumulate) cprev = *cptr;
         for (uint32_t k0 = warp * 256 + lane * 8; k0 < K; k0 += 2048 * U) {
             uint4 wv[U][RB];
 #pragma unroll
@@ -165,7 +214,7 @@ __global__ void __launch_bounds__(256) gemv_splitk_kernel(const bf16 *__restrict
 #pragma unroll
                 for (int r = 0; r < RB; ++r)
                     wv[u][r] = (k0 + 2048 * u < K) ? __ldcs(reinterpret_cast<const uint4 *>(wrow[r] + k0 + 2048 * u)) : make_uint4(0, 0, 0, 0);
-            if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; if (mine && accumulate) cprev = *cptr; }
+            if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const uint32_t k = k0 + 2048 * u;
@@ -183,7 +232,7 @@ __global__ void __launch_bounds__(256) gemv_splitk_kernel(const bf16 *__restrict
                 }
             }
         }
-        if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; if (mine && accumulate) cprev = *cptr; }     // a warp whose K slice is empty
+        if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }     // a warp whose K slice is empty
 #pragma unroll
         for (int r = 0; r < RB; ++r)
 #pragma unroll
@@ -196,7 +245,9 @@ __global__ void __launch_bounds__(256) gemv_splitk_kernel(const bf16 *__restrict
             float t = 0.f;
 #pragma unroll
             for (int w = 0; w < 8; ++w) t += part[w][threadIdx.x];
-            C[(size_t)(threadIdx.x % MT) * ldc + col0 + row0 + threadIdx.x / MT] = accumulate ? cprev + t : t;
+            float *cptr = C + (size_t)(threadIdx.x % MT) * ldc + col0 + row0 + threadIdx.x / MT;
+            if (accumulate) atomicAdd(cptr, t);                 // one add per element by one thread, not waited for
+            else *cptr = t;
         }
         __syncthreads();
     }
@@ -256,7 +307,8 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const bf16 *__restrict__ 
                 const uint32_t m = b * 8 + 2 * c + (i & 1), row = row0 + g + 8 * (i >> 1);
                 if (m < Mrows && row < n) {
                     float *p = C + (size_t)m * ldc + col0 + row;
-                    *p = accumulate ? *p + acc[b][i] : acc[b][i];
+                    if (accumulate) atomicAdd(p, acc[b][i]);      // one add per element by one thread, not waited for
+                    else *p = acc[b][i];
                 }
             }
     }
@@ -879,7 +931,8 @@ __global__ void __launch_bounds__(NW * 32) gemv_mma_splitk_kernel(const bf16 *__
             const uint32_t m = b * 8 + 2 * (ln & 3) + (i & 1), row = row0 + (ln >> 2) + 8 * (i >> 1);
             if (m < Mrows && row < n && (ROWS == 16 || (i >> 1) == 0)) {
                 float *p = C + (size_t)m * ldc + col0 + row;
-                *p = accumulate ? *p + sum : sum;
+                if (accumulate) atomicAdd(p, sum);               // one add per element by one thread, not waited for
+                else *p = sum;
             }
         }
         __syncthreads();
@@ -961,6 +1014,59 @@ static void launch_gemv_rows(const bf16 *A, const bf16 *W, float *C, uint32_t Mr
         if (n >= 2 * 148 * 16) return launch_gemv<MT, 2, 2>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
         return launch_gemv<MT, 1, 4>(A, W, C, Mrows, n, K, ldc, col0, acc, st);
     }
+}
+
+static int g_gemm_group = 1;     // products over the same activations: one launch where the parts allow it (0: always one launch each)
+
+template <int MT>
+static void launch_gemv_group(const bf16 *A, const GemvParts &p, uint32_t Mrows, uint32_t n_total, uint32_t K, cudaStream_t st) {
+    static int blocks_per_sm = 0, sms = 0;
+    if (!blocks_per_sm) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, gemv_group_kernel<MT, 8>, 256, 0) != cudaSuccess || blocks_per_sm < 1) blocks_per_sm = 1;
+        if (sms < 1) sms = 148;
+    }
+    uint32_t need = (n_total + 7) / 8, full = (uint32_t)(sms * blocks_per_sm);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(need < full ? need : full);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = g_gemv_pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, gemv_group_kernel<MT, 8>, A, p, Mrows, n_total, K);
+}
+
+// One launch serves the whole group exactly when every part alone would take gemv_kernel<MT, 1, 8> (M <= 2, fewer rows
+// in total than two waves of warps, K below the split-K threshold): same arithmetic, so the same bits.
+bool tgpk_gemm_group_fused(uint32_t count, const uint32_t *n, uint32_t M, uint32_t K) {
+    if (!g_gemm_group || count < 2 || count > TGP_GEMM_GROUP_MAX || !M || M > 2 || !K || K % 8) return false;
+    uint64_t total = 0;
+    for (uint32_t s = 0; s < count; ++s) { if (!n[s]) return false; total += n[s]; }
+    return total < 2 * 148 * 16 && !(g_gemv_splitk && K >= 8192);
+}
+
+int tgpk_gemm_group(const void *A, uint32_t count, const void *const *W, float *const *C, const uint32_t *n, const uint32_t *ldc, uint32_t M, uint32_t K, cudaStream_t st) {
+    if (!tgpk_gemm_group_fused(count, n, M, K)) {
+        for (uint32_t s = 0; s < count; ++s) {
+            const int rc = tgpk_gemm(A, W[s], C[s], M, n[s], K, ldc[s], 0, 0, st);
+            if (rc) return rc;
+        }
+        return TGP_OK;
+    }
+    GemvParts p;
+    memset(&p, 0, sizeof(p));
+    uint32_t total = 0;
+    for (uint32_t s = 0; s < count; ++s) { p.W[s] = (const bf16 *)W[s]; p.C[s] = C[s]; p.n[s] = n[s]; p.ldc[s] = ldc[s]; total += n[s]; }
+    p.count = count;
+    if (M == 1) launch_gemv_group<1>((const bf16 *)A, p, M, total, K, st);
+    else launch_gemv_group<2>((const bf16 *)A, p, M, total, K, st);
+    LAUNCH_CHECK(1);
+    return TGP_OK;
 }
 
 static int g_skinny_impl = 0;    // 0: tensor-core skinny kernel for 3 <= M <= 32; 1: CUDA-core GEMV (an on-device cross-check)
@@ -1097,6 +1203,18 @@ int tgp_k_rmsnorm(const float *x_dev, uint32_t ldx, const void *g_dev, void *h_d
 int tgp_k_skinny_select(int impl) {
     if (impl != 0 && impl != 1) return TGP_E_INVAL;
     g_skinny_impl = impl;
+    return TGP_OK;
+}
+
+int tgp_k_gemm_group(const void *A_dev, uint32_t count, const void *const *W_dev, float *const *C_dev, const uint32_t *n, const uint32_t *ldc,
+                     uint32_t M, uint32_t K, void *stream) {
+    if (!A_dev || !W_dev || !C_dev || !n || !ldc || !count || count > TGP_GEMM_GROUP_MAX) return TGP_E_INVAL;
+    for (uint32_t s = 0; s < count; ++s) if (!W_dev[s] || !C_dev[s] || n[s] > ldc[s]) return TGP_E_INVAL;
+    return tgpk_gemm_group(A_dev, count, W_dev, C_dev, n, ldc, M, K, (cudaStream_t)stream);
+}
+
+int tgp_k_gemm_group_select(int enable) {
+    g_gemm_group = enable ? 1 : 0;
     return TGP_OK;
 }
 

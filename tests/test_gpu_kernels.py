@@ -365,6 +365,45 @@ def test_overlapping_gemv_launches_keep_their_dependencies():
     assert np.abs(outs[0] - want).max() < 1e-4 * np.abs(want).max()
 
 
+@pytest.mark.parametrize("M,ns,K", [(1, (2048, 512, 512), 2048),      # the q, k, v projections of the 1B shape: one launch
+                                    (2, (300, 7, 129, 1), 264),         # four ragged parts, K not a multiple of the chunk
+                                    (1, (4096, 1024), 4096),            # too many rows for one launch: one launch per part
+                                    (2, (640, 640, 64), 8192),          # long K: the parts take the split-K kernel
+                                    (8, (1024, 256, 256), 512)])        # M > 2: one launch per part
+def test_grouped_products_equal_single_products_and_oracle(M, ns, K):
+    """Products that share their activations: the grouped call must give the bits of one tgp_k_gemm() call per part,
+    whether it runs as one launch or falls back to one launch per part, with the switch on and off, and leave the
+    columns beyond each part untouched; the values are checked against the oracle's linear()."""
+    a_bits = rnd_bits(51, M * K).reshape(M, K)
+    A = bf16_dev(a_bits)
+    w_bits = [rnd_bits(60 + s, n * K).reshape(n, K) for s, n in enumerate(ns)]
+    Wd = [bf16_dev(w) for w in w_bits]
+    ldcs = [n + 8 * (s + 1) for s, n in enumerate(ns)]
+    single = [torch.full((M, ld), -7.0, dtype=torch.float32, device=DEV) for ld in ldcs]
+    for s, n in enumerate(ns):
+        tb.k_gemm(A, Wd[s], single[s], M, n, K, ldcs[s], 0, 0)
+    outs = []
+    for enable in (1, 0):
+        tb.k_gemm_group_select(enable)
+        grouped = [torch.full((M, ld), -7.0, dtype=torch.float32, device=DEV) for ld in ldcs]
+        tb.k_gemm_group(A, Wd, grouped, M, list(ns), K, ldcs)
+        torch.cuda.synchronize()
+        outs.append([g.cpu().numpy() for g in grouped])
+    tb.k_gemm_group_select(1)
+    o = oracle()
+    a = si.bf16_bits_to_f32(a_bits)
+    for s, n in enumerate(ns):
+        ref = single[s].cpu().numpy()
+        assert np.array_equal(outs[0][s], ref) and np.array_equal(outs[1][s], ref)
+        assert (ref[:, n:] == -7.0).all()
+        want = o.linear(a, si.bf16_bits_to_f32(w_bits[s]).astype(np.float64)).astype(np.float64)
+        assert np.abs(ref[:, :n] - want).max() < 2e-5 * max(np.abs(want).max(), 0.01) + 1e-7
+    with pytest.raises(tb.TgpError):
+        tb.k_gemm_group(A, Wd[:1] * 5, [single[0]] * 5, M, [ns[0]] * 5, K, [ldcs[0]] * 5)      # more parts than the call takes
+    with pytest.raises(tb.TgpError):
+        tb.k_gemm_group(A, Wd[:2], single[:2], M, [ns[0], ns[1]], K, [ns[0] - 1, ldcs[1]])       # row stride below the part's width
+
+
 @pytest.mark.parametrize("M,n,K", [(3, 100, 64), (8, 4096, 4096), (8, 1030, 512), (13, 77, 128), (16, 260, 1024), (17, 64, 96), (24, 2049, 2048),
                                    (32, 4100, 8192), (5, 16, 32),
                                    # few rows and long K: K split over a thread-block cluster of 8, 4, 2 CTAs (ragged rows, K that leaves

@@ -138,6 +138,34 @@ def test_step_stats_and_call_order_errors():
     s.close()
 
 
+@pytest.mark.parametrize("B", [1, 2])
+def test_decode_step_groups_qkv_into_one_launch_with_the_same_bits(B):
+    """A decode step of at most two sequences runs a layer's q, k and v projections as one launch: two launches fewer per
+    layer, not a bit of difference in the logits, under a budget that keeps the ring turning; with the switch off every projection
+    is its own launch."""
+    cfg = replace(si.CONFIGS[1], B=B, S=19, T=5, TK=8)
+    prompt = si.prompt_tokens(cfg)
+    forced = (np.arange(cfg.B * cfg.T, dtype=np.int32).reshape(cfg.B, cfg.T) * 577 + 11) % cfg.V
+    lay, pool, s, blobs, T = setup(cfg, cap=128 << 10)
+    r = Runner(s, cfg.B * cfg.S)
+    runs = {}
+    for enable in (1, 0):
+        tb.k_gemm_group_select(enable)
+        logits, launches = [], []
+        r.reset()
+        r.step(tb.PREFILL, prompt, cfg.S)
+        for t in range(T):
+            st = r.step(tb.DECODE, np.ascontiguousarray(forced[:, t:t + 1]), 1, want_stats=True)
+            launches.append(st.n_launches)
+            logits.append(r.logits.cpu().numpy().copy())
+        runs[enable] = (logits, launches)
+    tb.k_gemm_group_select(1)
+    s.close()
+    for a, b in zip(runs[1][0], runs[0][0]):
+        assert np.array_equal(a, b)
+    assert [u - f for f, u in zip(runs[1][1], runs[0][1])] == [2 * cfg.L] * T
+
+
 _CFG2 = {}
 
 
