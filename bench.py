@@ -580,9 +580,9 @@ def main():
             ach = bpl / sec / 1e9
             roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"]}
         roof.update({"kernel": f"weight-block product ({dom[0]}, M={Mk}): " + ("gemv_kernel" if Mk <= 16 else "gemm_tc_kernel"),
-                     "launches": kind_n[dom], "avg_us": sec * 1e6, "algorithmic_per_launch": fpl if roof["bound"] == "tensor" else bpl,
+                     "launches": nl * (T if dom[0] == "decode" else 1), "avg_us": sec * 1e6, "algorithmic_per_launch": fpl if roof["bound"] == "tensor" else bpl,
                      "timing": f"CUDA-graph replay of the {nl} launches of one step, {kernel_loop.last['reps']} x {kernel_loop.last['passes']} passes back to back ({kernel_loop.last['seconds']:.1f} s), random operands, cold inputs cycling through 1 GiB, CUDA events on the launch stream",
-                     "in_step_avg_us": kind_ms[dom] / kind_n[dom] * 1e3, "shapes": table})
+                     "in_step_avg_us": kind_ms[dom] / (nl * (T if dom[0] == "decode" else 1)) * 1e3, "shapes": table})
     else:
         ach = kind_bytes[dom] / (kind_ms[dom] * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
@@ -651,7 +651,7 @@ def main():
                    "d2h_bytes_per_step": L_d2h + cfg.B * (T + 1) * 4 + cfg.B * cfg.V * 4},
            "object_level_prefetch": object_level, "policy_bits": args.bits, "trace_mismatches": mismatches, "moe_profile_pass_s": profile_s, "unseen_prompts": bool(args.unseen_prompts), "host_pool": ({"aliased_physical_layers": args.alias_layers, "physical_bytes": aliased.phys_bytes, "virtual_bytes": lay.pool_bytes} if aliased else "pinned, one physical page per byte"), "moe_prediction": moe_prediction,
            "gpu_launches": launches * args.steps, "clocks": clocks, "roofline": roof, "step_roofline": step_roof,
-           "kernels": {f"{k[0]}:{k[1]}": {"ms": round(v, 3), "launches": kind_n[k], "GBps": round(kind_bytes[k] / (v * 1e-3) / 1e9, 1),
+           "kernels": {f"{k[0]}:{k[1]}": {"ms": round(v, 3), "ops": kind_n[k], "GBps": round(kind_bytes[k] / (v * 1e-3) / 1e9, 1),
                                            "TFLOPs": round(kind_flops[k] / (v * 1e-3) / 1e12, 2)} for k, v in sorted(kind_ms.items())}}
     if not args.no_uvm and world == 1:                 # the baselines are single-GPU measurements: reported at N = 1 only
         try:

@@ -263,7 +263,8 @@ int  tgp_k_gemm(const void *A_dev, const void *W_dev, float *C_dev, uint32_t M, 
  * pointers, read before the call returns.  For M <= 2 with fewer than 4736 rows in total and K < 8192 one launch serves
  * all parts; otherwise the parts are launched one after the other.  The results are bit-identical to tgp_k_gemm() per
  * part either way.  tgp_k_gemm_group_select(0) forces one launch per part (process-wide; default 1), also inside
- * tgp_step(), which groups the q, k and v projections of a layer this way when no tap or op timing is set. */
+ * tgp_step(), which groups the q, k and v projections of a layer this way when no tap is set (with op timing the launch's
+ * time is reported for the q projection and an empty bracket for the other two). */
 #define TGP_GEMM_GROUP_MAX 4u
 int  tgp_k_gemm_group(const void *A_dev, uint32_t count, const void *const *W_dev, float *const *C_dev, const uint32_t *n,
                       const uint32_t *ldc, uint32_t M, uint32_t K, void *stream);

@@ -534,7 +534,7 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
         // The q, k and v projections of a layer read the same activations: when each is one whole tensor, their copies
         // have all been enqueued already and one launch can serve the three, ops [i, i + 3) run as one launch.
         uint32_t span = 1, gn[3] = {0, 0, 0}, gK = 0;
-        if (ring && o.kind == TGP_OP_GEMM && M <= 2 && !e->op_timing && !e->tap && i + 2 < st.op0 + st.nops) {
+        if (ring && o.kind == TGP_OP_GEMM && M <= 2 && !e->tap && i + 2 < st.op0 + st.nops) {
             bool ok = true;
             for (uint32_t j = 0; j < 3 && ok; ++j) {
                 const TgpOp &f = ctx->ops[i + j];
@@ -559,8 +559,9 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             }
         const uint32_t ti = i - st.op0;
         if (e->op_timing) {
-            if (e->ta.size() <= ti) { e->ta.resize(ti + 1, nullptr); e->tb_.resize(ti + 1, nullptr); }
-            if (!e->ta[ti]) { CU(ctx, cudaEventCreate(&e->ta[ti])); CU(ctx, cudaEventCreate(&e->tb_[ti])); }
+            if (e->ta.size() < ti + span) { e->ta.resize(ti + span, nullptr); e->tb_.resize(ti + span, nullptr); }
+            for (uint32_t j = ti; j < ti + span; ++j)
+                if (!e->ta[j]) { CU(ctx, cudaEventCreate(&e->ta[j])); CU(ctx, cudaEventCreate(&e->tb_[j])); }
             CU(ctx, cudaEventRecord(e->ta[ti], cs));
         }
         rc = TGP_OK;
@@ -688,7 +689,10 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             }
             if (trc) return trc;
         }
-        if (e->op_timing) CU(ctx, cudaEventRecord(e->tb_[ti], cs));
+        if (e->op_timing) {                              // ops that shared a launch: its time goes to the first, the others get an empty bracket
+            CU(ctx, cudaEventRecord(e->tb_[ti], cs));
+            for (uint32_t j = ti + 1; j < ti + span; ++j) { CU(ctx, cudaEventRecord(e->ta[j], cs)); CU(ctx, cudaEventRecord(e->tb_[j], cs)); }
+        }
         if (ring) {
             for (uint32_t j = i; j < i + span; ++j) {
                 if (ctx->plan.op_is_wait_target[j]) {
