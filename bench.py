@@ -125,25 +125,51 @@ def time_oracle(lay, om, sample_S, sample_T):
 
 
 def gemm_shapes_of_step(lay, M):
-    """(n, K, residual) of every weight-block product of one step, in trace order (lm_head at M = B)."""
+    """(n, K, residual, M) of every weight-block launch of one step, in trace order (lm_head at M = B).  Consecutive dense
+    blocks that read the same activations and carry the same non-zero tgp_k_gemm_group_key() share a launch, as in
+    tgp_step() once their copies are enqueued; n is then the tuple of their row counts."""
+    from paper_2609_06172_b200 import binding as tb
     cfg = lay.cfg
     out = []
+
+    def emit(blocks, res, m):
+        """blocks: weight blocks in op order, all multiplied with the same activations."""
+        run = []
+        def flush():
+            if len(run) == 1:
+                out.append((run[0].rows, run[0].cols, res, m))
+            elif run:
+                out.append((tuple(t.rows for t in run), run[0].cols, res, m))
+            run.clear()
+        for t in blocks:
+            key = tb.k_gemm_group_key(m, t.rows, t.cols) if m <= 32 else 0
+            if run and (not key or key != run_key[0] or t.cols != run[0].cols or len(run) == GROUP_MAX):
+                flush()
+            if not key:
+                out.append((t.rows, t.cols, res, m))
+                continue
+            if not run:
+                run_key[0] = key
+            run.append(t)
+        flush()
+
+    run_key = [0]
     for l in range(cfg.L):
-        qkv = [lay.blocks(kind, l) for kind in (si.K_WQ, si.K_WK, si.K_WV)]
-        if (M <= 2 and all(len(b) == 1 for b in qkv) and len({b[0].cols for b in qkv}) == 1 and qkv[0][0].cols < 8192
-                and sum(b[0].rows for b in qkv) < 2 * 148 * 16):
-            # the step runs these three as one launch (tgp_k_gemm_group's rule): n is the tuple of their row counts
-            out.append((tuple(b[0].rows for b in qkv), qkv[0][0].cols, 0, M))
+        emit([t for kind in (si.K_WQ, si.K_WK, si.K_WV) for t in lay.blocks(kind, l)], 0, M)
+        emit(lay.blocks(si.K_WO, l), 1, M)
+        if cfg.E:                                             # MoE: tokens spread evenly over the experts (top-k picks each)
+            me = max(1, M * cfg.topk // cfg.E)
+            for e in range(cfg.E):
+                emit([t for kind in (si.K_WG, si.K_WU) for t in lay.blocks(kind, l, e)], 0, me)
+                emit(lay.blocks(si.K_WD, l, e), 0, me)
         else:
-            for b in qkv:
-                out += [(t.rows, t.cols, 0, M) for t in b]
-        out += [(t.rows, t.cols, 1, M) for t in lay.blocks(si.K_WO, l)]
-        for e in (range(cfg.E) if cfg.E else (-1,)):          # MoE: tokens spread evenly over the experts (top-k picks each)
-            me = M if not cfg.E else max(1, M * cfg.topk // cfg.E)
-            for kind, res in ((si.K_WG, 0), (si.K_WU, 0), (si.K_WD, 0 if cfg.E else 1)):
-                out += [(t.rows, t.cols, res, me) for t in lay.blocks(kind, l, e)]
-    out += [(t.rows, t.cols, 0, cfg.B) for t in lay.blocks(si.K_LM)]
+            emit([t for kind in (si.K_WG, si.K_WU) for t in lay.blocks(kind, l)], 0, M)
+            emit(lay.blocks(si.K_WD, l), 1, M)
+    emit(lay.blocks(si.K_LM), 0, cfg.B)
     return out
+
+
+GROUP_MAX = 8     # TGP_GEMM_GROUP_MAX
 
 
 def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
@@ -183,7 +209,7 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
             if isinstance(n, tuple):
                 starts = [sum(n[:i]) for i in range(len(n))]
                 tb.k_gemm_group(A, [wbuf.data_ptr() + off + r0 * K * 2 for r0 in starts], [Cbuf.data_ptr() + r0 * 4 for r0 in starts],
-                                m, list(n), K, [nmax] * len(n), st)
+                                m, list(n), K, [nmax] * len(n), res, st)
             else:
                 tb.k_gemm(A, wbuf.data_ptr() + off, Cbuf, m, n, K, nmax, 0, res, st)
             off += nb

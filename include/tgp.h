@@ -257,17 +257,22 @@ int  tgp_k_rmsnorm(const float *x_dev, uint32_t ldx, const void *g_dev, void *h_
  * block), C fp32 with row stride ldc.  accumulate != 0 adds to C (fused residual).  K % 8 == 0. */
 int  tgp_k_gemm(const void *A_dev, const void *W_dev, float *C_dev, uint32_t M, uint32_t n, uint32_t K,
                 uint32_t ldc, uint32_t col0, int accumulate, void *stream);
-/* Several products over the same activations in one call (the q, k and v projections of a decode step, Section II-B's
- * kernel sequence): C_dev[s][m, j] = sum_k A[m, k] * W_dev[s][j, k] for s < count <= TGP_GEMM_GROUP_MAX, W_dev[s] bf16
- * [n[s], K], C_dev[s] fp32 with row stride ldc[s] >= n[s].  The pointer and size arrays are host arrays of device
- * pointers, read before the call returns.  For M <= 2 with fewer than 4736 rows in total and K < 8192 one launch serves
- * all parts; otherwise the parts are launched one after the other.  The results are bit-identical to tgp_k_gemm() per
- * part either way.  tgp_k_gemm_group_select(0) forces one launch per part (process-wide; default 1), also inside
- * tgp_step(), which groups the q, k and v projections of a layer this way when no tap is set (with op timing the launch's
- * time is reported for the q projection and an empty bracket for the other two). */
-#define TGP_GEMM_GROUP_MAX 4u
+/* Several products over the same activations in one call (Section II-B's kernel sequence: the q, k and v projections of a
+ * layer, or the pieces a large matrix was registered as): C_dev[s][m, j] (=|+=) sum_k A[m, k] * W_dev[s][j, k] for
+ * s < count <= TGP_GEMM_GROUP_MAX, W_dev[s] bf16 [n[s], K], C_dev[s] fp32 with row stride ldc[s] >= n[s]; accumulate != 0
+ * adds to C (fused residual).  The pointer and size arrays are host arrays (of device pointers), read before the call
+ * returns.  Blocks whose tgp_k_gemm_group_key() is the same non-zero value are served by one launch - a block of few
+ * rows alone leaves most SMs without work - anything else by one launch per part; the results are bit-identical to
+ * tgp_k_gemm() per part either way, because the key names the kernel the block takes on its own (M <= 2: fewer than
+ * 4736 rows and K < 8192; 3 <= M <= 32 with K % 32 == 0: the blocks of fewer than 128 rows per SM).
+ * tgp_k_gemm_group_select(0) makes every key 0 (process-wide; default 1), also inside tgp_step(), which groups
+ * consecutive weight-block products of a decode step that read the same activations this way when their copies have
+ * all been enqueued and no tap is set (with op timing the launch's time is reported for the first product of the group
+ * and an empty bracket for the others). */
+#define TGP_GEMM_GROUP_MAX 8u
 int  tgp_k_gemm_group(const void *A_dev, uint32_t count, const void *const *W_dev, float *const *C_dev, const uint32_t *n,
-                      const uint32_t *ldc, uint32_t M, uint32_t K, void *stream);
+                      const uint32_t *ldc, uint32_t M, uint32_t K, int accumulate, void *stream);
+int  tgp_k_gemm_group_key(uint32_t M, uint32_t n, uint32_t K, uint32_t *key);
 int  tgp_k_gemm_group_select(int enable);
 /* Which kernel serves M > 16: 0 (default) the tcgen05 tensor-core GEMM, 1 the CUDA-core tile kernel (an on-device
  * cross-check).  M <= 16 always takes the weight-streaming GEMV.  Process-wide. */

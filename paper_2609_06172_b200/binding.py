@@ -96,7 +96,8 @@ _SIGS = {
     "tgp_k_embed": [_P, _P, _P, _U32, _U32, _P],
     "tgp_k_rmsnorm": [_P, _U32, _P, _P, _U32, _U32, C.c_float, _P],
     "tgp_k_gemm": [_P, _P, _P, _U32, _U32, _U32, _U32, _U32, C.c_int, _P],
-    "tgp_k_gemm_group": [_P, _U32, _P, _P, C.POINTER(_U32), C.POINTER(_U32), _U32, _U32, _P],
+    "tgp_k_gemm_group": [_P, _U32, _P, _P, C.POINTER(_U32), C.POINTER(_U32), _U32, _U32, C.c_int, _P],
+    "tgp_k_gemm_group_key": [_U32, _U32, _U32, C.POINTER(_U32)],
     "tgp_k_gemm_group_select": [C.c_int],
     "tgp_k_gemm_select": [C.c_int],
     "tgp_k_attn_select": [C.c_int],
@@ -364,11 +365,18 @@ def k_gemm(A, W, Cout, M, n, K, ldc, col0, accumulate, stream=None):
     _k(lib().tgp_k_gemm(_ptr(A), _ptr(W), _ptr(Cout), M, n, K, ldc, col0, int(accumulate), _ptr(stream)), "tgp_k_gemm")
 
 
-def k_gemm_group(A, Ws, Couts, M, ns, K, ldcs, stream=None):
+def k_gemm_group(A, Ws, Couts, M, ns, K, ldcs, accumulate=False, stream=None):
     """Products of the same activations A [M, K] with several weight blocks Ws[s] [ns[s], K] into Couts[s] (row stride ldcs[s])."""
     c = len(Ws)
     _k(lib().tgp_k_gemm_group(_ptr(A), c, (_P * c)(*[_ptr(w) for w in Ws]), (_P * c)(*[_ptr(o) for o in Couts]),
-                              (_U32 * c)(*ns), (_U32 * c)(*ldcs), M, K, _ptr(stream)), "tgp_k_gemm_group")
+                              (_U32 * c)(*ns), (_U32 * c)(*ldcs), M, K, int(accumulate), _ptr(stream)), "tgp_k_gemm_group")
+
+
+def k_gemm_group_key(M, n, K):
+    """Blocks with the same non-zero key may share a launch (0: launched alone)."""
+    key = _U32(0)
+    _k(lib().tgp_k_gemm_group_key(M, n, K, C.byref(key)), "tgp_k_gemm_group_key")
+    return key.value
 
 
 def k_gemm_group_select(enable):

@@ -495,6 +495,35 @@ static int run_expert_fallback(tgp_ctx *ctx, int32_t layer, int32_t expert, cuda
     return TGP_OK;
 }
 
+// What a dense weight block is multiplied with and where its product goes: activations, output (row stride ldc, the
+// block writes columns [row0, row0 + rows)), whether it is added to the residual stream, and the activation rows.
+struct GemmTarget { const void *A; float *C; uint32_t ldc, Mrows; int acc; };
+
+static bool gemm_target(const TgpEngine *e, const tgp_model_cfg &c, const TgpRole &r, uint32_t M, uint32_t B, float *logits_dev, GemmTarget *t) {
+    const uint32_t qd = c.Hq * c.Dh, kd = c.Hkv * c.Dh;
+    if (r.expert >= 0) {                                  // expert block: the gathered rows of the tokens routed to it (see run_expert_block)
+        if ((uint32_t)r.expert >= c.E) return false;
+        const uint32_t me = e->cnt[r.expert];
+        switch (r.kind) {
+        case TGP_K_WG: *t = {e->hg, e->g32, c.F, me, 0}; return true;
+        case TGP_K_WU: *t = {e->hg, e->u32, c.F, me, 0}; return true;
+        case TGP_K_WD: *t = {e->ab, e->y32, c.d, me, 0}; return true;
+        default: return false;
+        }
+    }
+    switch (r.kind) {
+    case TGP_K_WQ: *t = {e->h, e->q32, qd, M, 0}; return true;
+    case TGP_K_WK: *t = {e->h, e->k32, kd, M, 0}; return true;
+    case TGP_K_WV: *t = {e->h, e->v32, kd, M, 0}; return true;
+    case TGP_K_WO: *t = {e->ob, e->x, c.d, M, 1}; return true;
+    case TGP_K_WG: *t = {e->h, e->g32, c.F, M, 0}; return true;
+    case TGP_K_WU: *t = {e->h, e->u32, c.F, M, 0}; return true;
+    case TGP_K_WD: *t = {e->ab, e->x, c.d, M, 1}; return true;
+    case TGP_K_LM: *t = {e->hf, logits_dev, c.V, B, 0}; return true;
+    default: return false;
+    }
+}
+
 extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_host, uint32_t B, uint32_t q_len,
                         float *logits_dev, int32_t *argmax_dev, void *compute_stream, void *copy_stream, tgp_step_stats *stats) {
     if (!ctx || !logits_dev) return TGP_E_INVAL;
@@ -531,24 +560,39 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
     const uint32_t qd = c.Hq * c.Dh, kd = c.Hkv * c.Dh;
     for (uint32_t i = st.op0; i < st.op0 + st.nops; ++i) {
         const TgpOp &o = ctx->ops[i];
-        // The q, k and v projections of a layer read the same activations: when each is one whole tensor, their copies
-        // have all been enqueued already and one launch can serve the three, ops [i, i + 3) run as one launch.
-        uint32_t span = 1, gn[3] = {0, 0, 0}, gK = 0;
-        if (ring && o.kind == TGP_OP_GEMM && M <= 2 && !e->tap && i + 2 < st.op0 + st.nops) {
-            bool ok = true;
-            for (uint32_t j = 0; j < 3 && ok; ++j) {
+        // Consecutive weight-block products of a decode step that read the same activations (the q, k and v projections, gate
+        // and up, the pieces one large matrix is registered as) run as one launch when the kernels say they may share one
+        // and their copies have all been enqueued already: a block of few rows alone leaves most SMs without work.
+        uint32_t span = 1, gK = 0, gn[TGP_GEMM_GROUP_MAX], gld[TGP_GEMM_GROUP_MAX];
+        float *gC[TGP_GEMM_GROUP_MAX];
+        GemmTarget g0 = {};
+        int32_t g_expert = -1;
+        bool g_gather = false, g_scatter = false;
+        if (ring && o.kind == TGP_OP_GEMM && !e->tap) {
+            uint32_t cnt = 0, key0 = 0;
+            for (uint32_t j = 0; j < TGP_GEMM_GROUP_MAX && i + j < st.op0 + st.nops; ++j) {
                 const TgpOp &f = ctx->ops[i + j];
-                ok = f.kind == TGP_OP_GEMM && f.layer == o.layer && f.nacc >= 1;
-                const int32_t ri = ok ? ctx->role_of_tensor[ctx->acc[f.acc0].tensor] : -1;
-                if (!(ok = ok && ri >= 0)) break;
+                if (f.kind != TGP_OP_GEMM || f.layer != o.layer || !f.nacc) break;
+                const int32_t ri = ctx->role_of_tensor[ctx->acc[f.acc0].tensor];
+                if (ri < 0) break;
                 const TgpRole &r = ctx->roles[ri];
-                const uint32_t Kj = r.rows ? (uint32_t)(ctx->tensors[ctx->acc[f.acc0].tensor].size / (2ull * r.rows)) : 0;
-                ok = r.kind == (j == 0 ? TGP_K_WQ : j == 1 ? TGP_K_WK : TGP_K_WV) && r.expert < 0 && r.row0 == 0 && r.rows == (j == 0 ? qd : kd) &&
-                     (j == 0 || Kj == gK) && (ctx->plan.op_last_place[i + j] < 0 || (size_t)ctx->plan.op_last_place[i + j] < e->next_cmd);
-                gn[j] = r.rows;
-                gK = Kj;
+                GemmTarget t;
+                if (!r.rows || !gemm_target(e, c, r, M, B, logits_dev, &t) || !t.Mrows || t.Mrows > 32) break;
+                const uint32_t Kj = (uint32_t)(ctx->tensors[ctx->acc[f.acc0].tensor].size / (2ull * r.rows));
+                const uint32_t key = tgpk_gemm_group_key(t.Mrows, r.rows, Kj);
+                if (!key) break;
+                if (j == 0) { g0 = t; gK = Kj; key0 = key; g_expert = r.expert; }
+                else if (t.A != g0.A || t.acc != g0.acc || t.Mrows != g0.Mrows || Kj != gK || key != key0 || r.expert != g_expert) break;
+                if (ctx->plan.op_last_place[i + j] >= 0 && (size_t)ctx->plan.op_last_place[i + j] >= e->next_cmd) break;   // its copy is not enqueued yet
+                gC[j] = t.C + r.row0; gn[j] = r.rows; gld[j] = t.ldc;
+                cnt = j + 1;
             }
-            if (ok && tgpk_gemm_group_fused(3, gn, M, gK)) span = 3;
+            if (cnt >= 2) span = cnt;
+            for (uint32_t j = 0; j < span && span > 1 && g_expert >= 0; ++j) {       // what run_expert_block does around an expert's products
+                const TgpRole &r = ctx->roles[ctx->role_of_tensor[ctx->acc[ctx->ops[i + j].acc0].tensor]];
+                g_gather |= r.kind == TGP_K_WG && r.row0 == 0;
+                g_scatter |= r.kind == TGP_K_WD && r.row0 + r.rows == c.d;
+            }
         }
         for (uint32_t j = i; j < i + span; ++j)
             if ((ring || hints) && ctx->plan.op_last_place[j] >= 0) {
@@ -582,11 +626,18 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             const TgpRole &r = ctx->roles[ri];
             const uint32_t K = (uint32_t)(ctx->tensors[a.tensor].size / (2ull * r.rows));
             const void *W = where(ctx, o, 0);
-            if (span == 3) {
-                const void *gW[3] = {W, where(ctx, ctx->ops[i + 1], 0), where(ctx, ctx->ops[i + 2], 0)};
-                float *gC[3] = {e->q32, e->k32, e->v32};
-                const uint32_t gld[3] = {qd, kd, kd};
-                rc = tgpk_gemm_group(e->h, 3, gW, gC, gn, gld, M, K, cs);
+            if (span > 1) {
+                const void *gW[TGP_GEMM_GROUP_MAX];
+                for (uint32_t j = 0; j < span; ++j) gW[j] = where(ctx, ctx->ops[i + j], 0);
+                if (g_expert >= 0) {
+                    e->cur_expert = g_expert;
+                    const int32_t *rows = e->erow + (size_t)g_expert * e->max_tokens;
+                    if (g_gather && (rc = tgpk_gather_rows(e->h, rows, e->hg, g0.Mrows, c.d, cs))) break;
+                    if ((rc = tgpk_gemm_group(g0.A, span, gW, gC, gn, gld, g0.Mrows, gK, 0, cs))) break;
+                    if (g_scatter) rc = tgpk_scatter_add(e->x, e->y32, rows, e->egate + (size_t)g_expert * e->max_tokens, g0.Mrows, c.d, cs);
+                    break;
+                }
+                rc = tgpk_gemm_group(g0.A, span, gW, gC, gn, gld, g0.Mrows, gK, g0.acc, cs);
                 break;
             }
             if (r.expert >= 0) {                          // expert weight block: rows of the tokens routed to that expert
@@ -595,17 +646,9 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
                 rc = run_expert_block(ctx, r, W, K, cs);
                 break;
             }
-            switch (r.kind) {
-            case TGP_K_WQ: rc = tgpk_gemm(e->h, W, e->q32, M, r.rows, K, qd, r.row0, 0, cs); break;
-            case TGP_K_WK: rc = tgpk_gemm(e->h, W, e->k32, M, r.rows, K, kd, r.row0, 0, cs); break;
-            case TGP_K_WV: rc = tgpk_gemm(e->h, W, e->v32, M, r.rows, K, kd, r.row0, 0, cs); break;
-            case TGP_K_WO: rc = tgpk_gemm(e->ob, W, e->x, M, r.rows, K, c.d, r.row0, 1, cs); break;
-            case TGP_K_WG: rc = tgpk_gemm(e->h, W, e->g32, M, r.rows, K, c.F, r.row0, 0, cs); break;
-            case TGP_K_WU: rc = tgpk_gemm(e->h, W, e->u32, M, r.rows, K, c.F, r.row0, 0, cs); break;
-            case TGP_K_WD: rc = tgpk_gemm(e->ab, W, e->x, M, r.rows, K, c.d, r.row0, 1, cs); break;
-            case TGP_K_LM: rc = tgpk_gemm(e->hf, W, logits_dev, B, r.rows, K, c.V, r.row0, 0, cs); break;
-            default: return tgp_fail(ctx, TGP_E_MISMATCH, "GEMM op on a tensor that is not a weight");
-            }
+            GemmTarget t;
+            if (!gemm_target(e, c, r, M, B, logits_dev, &t)) return tgp_fail(ctx, TGP_E_MISMATCH, "GEMM op on a tensor that is not a weight");
+            rc = tgpk_gemm(t.A, W, t.C, t.Mrows, r.rows, K, t.ldc, r.row0, t.acc, cs);
             break;
         }
         case TGP_OP_ROUTER: {

@@ -135,10 +135,11 @@ __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, c
 // Several products that read the same activations (the q, k and v projections of a layer) in one launch: the output
 // rows of the parts are walked as one list, one warp per row, with exactly the arithmetic of gemv_kernel<MT, 1, U>, so
 // the result is bit-identical to separate launches; what is saved is two launch floors of about a microsecond each.
-struct GemvParts { const bf16 *W[TGP_GEMM_GROUP_MAX]; float *C[TGP_GEMM_GROUP_MAX]; uint32_t n[TGP_GEMM_GROUP_MAX], ldc[TGP_GEMM_GROUP_MAX], count; };
+// (groups[s]: CTAs' worth of rows in part s, for the kernels that walk row groups instead of rows)
+struct GemvParts { const bf16 *W[TGP_GEMM_GROUP_MAX]; float *C[TGP_GEMM_GROUP_MAX]; uint32_t n[TGP_GEMM_GROUP_MAX], ldc[TGP_GEMM_GROUP_MAX], groups[TGP_GEMM_GROUP_MAX], count; };
 
 template <int MT, int U>
-__global__ void __launch_bounds__(256) gemv_group_kernel(const bf16 *__restrict__ A, const GemvParts p, uint32_t Mrows, uint32_t n_total, uint32_t K) {
+__global__ void __launch_bounds__(256) gemv_group_kernel(const bf16 *__restrict__ A, const GemvParts p, uint32_t Mrows, uint32_t n_total, uint32_t K, int accumulate) {
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarp = (gridDim.x * blockDim.x) >> 5;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -148,7 +149,7 @@ __global__ void __launch_bounds__(256) gemv_group_kernel(const bf16 *__restrict_
         float *C = p.C[0];
         uint32_t ldc = p.ldc[0], r = row, start = p.n[0];
 #pragma unroll
-        for (int s = 1; s < TGP_GEMM_GROUP_MAX; ++s)
+        for (int s = 1; s < (int)TGP_GEMM_GROUP_MAX; ++s)
             if (s < (int)p.count) {
                 if (row >= start) { W = p.W[s]; C = p.C[s]; ldc = p.ldc[s]; r = row - start; }
                 start += p.n[s];
@@ -181,7 +182,10 @@ __global__ void __launch_bounds__(256) gemv_group_kernel(const bf16 *__restrict_
 #pragma unroll
         for (int m = 0; m < MT; ++m) {
             const float s = warp_sum(acc[m]);
-            if ((int)lane == m && m < (int)Mrows) C[(size_t)m * ldc + r] = s;
+            if ((int)lane == m && m < (int)Mrows) {
+                if (accumulate) atomicAdd(&C[(size_t)m * ldc + r], s);
+                else C[(size_t)m * ldc + r] = s;
+            }
         }
     }
 }
@@ -853,6 +857,10 @@ int tgpk_rmsnorm(const float *x, uint32_t ldx, const void *g, void *h, uint32_t 
     return TGP_OK;
 }
 
+static int g_skinny_impl = 0;    // 0: tensor-core skinny kernel for 3 <= M <= 32; 1: CUDA-core GEMV (an on-device cross-check)
+static int g_gemm_impl = 0;      // 0: tensor cores for M > 16; 1: CUDA-core tiles (kept as an on-device cross-check)
+static int g_gemv_splitk = 1;    // small-n blocks at M <= 2: CTA per RB rows with K split over its warps (0: one warp per row)
+static int g_gemm_group = 1;     // products over the same activations: one launch where the parts allow it (0: always one launch each)
 static int g_gemv_rows8 = 1;     // skinny products of few rows and long K: 8-row CTAs (0: always 16)
 static int g_gemv_pdl = 1;       // consecutive weight-streaming launches may overlap (programmatic dependent launch)
 
@@ -939,40 +947,189 @@ __global__ void __launch_bounds__(NW * 32) gemv_mma_splitk_kernel(const bf16 *__
     }
 }
 
-template <int NB, int U>
-static void launch_gemv_mma(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int acc, cudaStream_t st) {
-    static int blocks_per_sm = 0, sms = 0;
-    if (!blocks_per_sm) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, gemv_mma_kernel<NB, U>, 256, 0) != cudaSuccess || blocks_per_sm < 1) blocks_per_sm = 1;
-        if (sms < 1) sms = 148;
+// The same kernel over several weight blocks that read the same activations (the pieces of one matrix; the q, k and v
+// projections): their row groups are walked as one list and a CTA takes RG consecutive groups, whose MMAs share each
+// activation fragment - every CTA reads its K slices of all activation rows from L2, so at 8 or 16 rows per CTA that
+// traffic equals or exceeds the weights' and bounds the kernel; RG row groups divide it by RG.  A group's arithmetic
+// (which warp adds which k, in which order) is that of gemv_mma_splitk_kernel<NB, U, NW, ROWS> whatever RG and the list:
+// same bits as one launch per block.
+template <int NB, int U, int NW, int ROWS, int RG>
+__global__ void __launch_bounds__(NW * 32) gemv_mma_group_kernel(const bf16 *__restrict__ A, const GemvParts p, uint32_t Mrows, uint32_t groups_total,
+                                                              uint32_t K, int accumulate) {
+    constexpr int UL = ROWS == 8 ? 2 * U : U;             // half a tile per load step: twice the steps in flight
+    constexpr int G = RG, SUB = UL / G;                  // SUB load steps of G groups in flight at a time: as many loads as UL of one
+    static_assert(UL % G == 0, "row groups per CTA must divide the load steps");
+    __shared__ float part[NW][G * NB * 4][32];
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, c = lane & 3;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    bool synced = false;
+    for (uint32_t grp0 = blockIdx.x * G; grp0 < groups_total; grp0 += gridDim.x * G) {
+        // which block a group belongs to: looked up here for the weights and again after the K loop for the output, so
+        // that the output's pointer and stride do not occupy registers while the loads are in flight
+        const bf16 *wlo[G], *whi[G];
+#pragma unroll
+        for (int r = 0; r < G; ++r) {
+            const uint32_t grp = min(grp0 + r, groups_total - 1);          // a group past the end re-reads the last one, never stored
+            const bf16 *W = p.W[0];
+            uint32_t n = p.n[0], local = grp;
+            {
+                uint32_t start = p.groups[0];
+#pragma unroll
+                for (int s = 1; s < (int)TGP_GEMM_GROUP_MAX; ++s)
+                    if (s < (int)p.count) {
+                        if (grp >= start) { W = p.W[s]; n = p.n[s]; local = grp - start; }
+                        start += p.groups[s];
+                    }
+            }
+            wlo[r] = W + (size_t)min(local * ROWS + g, n - 1) * K + c * 8;
+            whi[r] = W + (size_t)min(local * ROWS + g + 8, n - 1) * K + c * 8;
+        }
+        float acc[G][NB][4];
+#pragma unroll
+        for (int r = 0; r < G; ++r)
+#pragma unroll
+            for (int b = 0; b < NB; ++b) { acc[r][b][0] = acc[r][b][1] = acc[r][b][2] = acc[r][b][3] = 0.f; }
+        for (uint32_t k0 = warp * 32 * UL; k0 < K; k0 += NW * 32 * UL) {
+#pragma unroll
+            for (int sub = 0; sub < G; ++sub) {
+                uint4 lo[G][SUB], hi[G][SUB];
+#pragma unroll
+                for (int u = 0; u < SUB; ++u) {
+                    const uint32_t k = k0 + 32 * (sub * SUB + u);
+#pragma unroll
+                    for (int r = 0; r < G; ++r) {
+                        lo[r][u] = k < K ? __ldcs(reinterpret_cast<const uint4 *>(wlo[r] + k)) : make_uint4(0, 0, 0, 0);
+                        hi[r][u] = (k < K && ROWS == 16) ? __ldcs(reinterpret_cast<const uint4 *>(whi[r] + k)) : make_uint4(0, 0, 0, 0);   // ROWS == 8: the upper half of the tile stays empty
+                    }
+                }
+                if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
+#pragma unroll
+                for (int u = 0; u < SUB; ++u) {
+                    const uint32_t k = k0 + 32 * (sub * SUB + u);
+#pragma unroll
+                    for (int b = 0; b < NB; ++b) {
+                        const uint32_t m = b * 8 + g;
+                        const uint4 xv = (k < K && m < Mrows) ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k + c * 8)) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                        for (int r = 0; r < G; ++r) {
+                            mma_bf16_16816(acc[r][b], lo[r][u].x, hi[r][u].x, lo[r][u].y, hi[r][u].y, xv.x, xv.y);
+                            mma_bf16_16816(acc[r][b], lo[r][u].z, hi[r][u].z, lo[r][u].w, hi[r][u].w, xv.z, xv.w);
+                        }
+                    }
+                }
+            }
+        }
+        if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
+#pragma unroll
+        for (int r = 0; r < G; ++r)
+#pragma unroll
+            for (int b = 0; b < NB; ++b)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) part[warp][(r * NB + b) * 4 + i][lane] = acc[r][b][i];
+        __syncthreads();
+        for (uint32_t v = threadIdx.x; v < G * NB * 4 * 32; v += NW * 32) {
+            const uint32_t slot = v >> 5, ln = v & 31, r = slot / (NB * 4), b = (slot >> 2) % NB, i = slot & 3;
+            const uint32_t grp = grp0 + r;
+            if (grp >= groups_total) continue;
+            float sum = 0.f;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) sum += part[w][slot][ln];
+            float *C = p.C[0];
+            uint32_t ldc = p.ldc[0], n = p.n[0], row0 = grp * ROWS;
+            {
+                uint32_t start = p.groups[0];
+#pragma unroll
+                for (int s = 1; s < (int)TGP_GEMM_GROUP_MAX; ++s)
+                    if (s < (int)p.count) {
+                        if (grp >= start) { C = p.C[s]; ldc = p.ldc[s]; n = p.n[s]; row0 = (grp - start) * ROWS; }
+                        start += p.groups[s];
+                    }
+            }
+            const uint32_t m = b * 8 + 2 * (ln & 3) + (i & 1), row = row0 + (ln >> 2) + 8 * (i >> 1);
+            if (m < Mrows && row < n && (ROWS == 16 || (i >> 1) == 0)) {
+                float *out = C + (size_t)m * ldc + row;
+                if (accumulate) atomicAdd(out, sum);             // one add per element by one thread, not waited for
+                else *out = sum;
+            }
+        }
+        __syncthreads();
     }
-    static int blocks_per_sm_split = 0;
-    if (!blocks_per_sm_split && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm_split, gemv_mma_splitk_kernel<NB, U, 8, 16>, 256, 0) != cudaSuccess || blocks_per_sm_split < 1))
-        blocks_per_sm_split = 1;
-    const bool split = n < 16u * 8u * (uint32_t)sms;                 // too few 16-row groups to give every SM eight warps
-    const bool wide = split && (n + 15) / 16 < 2u * (uint32_t)sms;   // fewer than two 16-row groups per SM: 16 warps per CTA
+}
+
+// Which skinny kernel serves a block of n rows at M activation rows: NB groups of 8 activation rows, U load steps in
+// flight, and for blocks too small to give every SM eight 16-row warps the split-K kernel with NW warps per CTA over
+// ROWS rows.  The choice depends on the block alone, so a block computes the same bits alone or as part of a group.
+struct SkinnyPick { int nb, u, nw, rows; bool split; };
+
+static int device_sms() {
+    static int sms = 0;
+    if (!sms) { int dev = 0; cudaGetDevice(&dev); if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148; }
+    return sms;
+}
+
+static SkinnyPick pick_skinny(uint32_t M, uint32_t n, uint32_t K) {
+    const uint32_t sms = (uint32_t)device_sms(), groups16 = (n + 15) / 16;
+    const bool few = groups16 < sms;                      // fewer 16-row groups than SMs: few CTAs, so each warp keeps twice the loads in flight
+    SkinnyPick k;
+    k.nb = M <= 8 ? 1 : M <= 16 ? 2 : 4;
+    k.u = M <= 16 ? (few ? 8 : 4) : (few ? 4 : 2);
+    k.split = n < 16u * 8u * sms;                         // too few 16-row groups to give every SM eight warps
+    const bool wide = k.split && groups16 < 2u * sms;     // fewer than two 16-row groups per SM: 16 warps per CTA
     // 16-row groups for at most half the SMs and a K long enough to keep all 16 warps loading: 8 rows per CTA, twice the
     // CTAs (each CTA reads its slice of the activations whatever its rows, so fewer rows per CTA cost L2 traffic)
-    const bool half = wide && g_gemv_rows8 && 2 * ((n + 15) / 16) <= (uint32_t)sms && K >= 16u * 32u * 2u * U;
-    uint32_t need = split ? (half ? (n + 7) / 8 : (n + 15) / 16) : (n + 16 * 8 - 1) / (16 * 8);
-    uint32_t full = (uint32_t)(sms * (split ? blocks_per_sm_split : blocks_per_sm));
+    const bool half = wide && g_gemv_rows8 && 2 * groups16 <= sms && K >= 16u * 32u * 2u * (uint32_t)k.u;
+    k.nw = wide ? 16 : 8;
+    k.rows = half ? 8 : 16;
+    return k;
+}
+
+template <int NB, int U>
+static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint32_t Mrows, uint32_t K, int acc, cudaStream_t st) {
+    static int blocks_per_sm = 0, blocks_per_sm_split = 0;
+    if (!blocks_per_sm && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, gemv_mma_kernel<NB, U>, 256, 0) != cudaSuccess || blocks_per_sm < 1)) blocks_per_sm = 1;
+    if (!blocks_per_sm_split && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm_split, gemv_mma_splitk_kernel<NB, U, 8, 16>, 256, 0) != cudaSuccess || blocks_per_sm_split < 1))
+        blocks_per_sm_split = 1;
+    const uint32_t sms = (uint32_t)device_sms();
+    uint32_t need = 0;
+    if (k.split) for (uint32_t s = 0; s < p.count; ++s) { p.groups[s] = (p.n[s] + k.rows - 1) / k.rows; need += p.groups[s]; }
+    else need = (p.n[0] + 16 * 8 - 1) / (16 * 8);           // whole blocks of many rows are launched alone
+    // several blocks in one launch: two row groups per CTA share each activation fragment when that still leaves a CTA per SM
+    // (four groups of activation rows would need twice the shared memory a CTA may declare)
+    const bool pairs = k.split && p.count > 1 && NB <= 2 && need >= 2 * sms;
+    if (pairs) need = (need + 1) / 2;
+    const uint32_t full = sms * (uint32_t)(k.split ? blocks_per_sm_split : blocks_per_sm);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(need < full ? need : full);
-    cfg.blockDim = dim3(wide ? 512 : 256);
+    cfg.blockDim = dim3(k.split ? k.nw * 32 : 256);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = g_gemv_pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (wide && half) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 8>, A, W, C, Mrows, n, K, ldc, col0, acc);
-    else if (wide) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 16>, A, W, C, Mrows, n, K, ldc, col0, acc);
-    else if (half) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 8, 8>, A, W, C, Mrows, n, K, ldc, col0, acc);
-    else if (split) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 8, 16>, A, W, C, Mrows, n, K, ldc, col0, acc);
-    else cudaLaunchKernelEx(&cfg, gemv_mma_kernel<NB, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
+    uint32_t total = 0;
+    for (uint32_t s = 0; k.split && s < p.count; ++s) total += p.groups[s];
+    if (!k.split) cudaLaunchKernelEx(&cfg, gemv_mma_kernel<NB, U>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
+    else if (p.count > 1) {                               // only few-row blocks are ever grouped: 16 warps, doubled load steps
+        if constexpr (NB <= 2 && U == 8) {
+            if (pairs && k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 8, 2>, A, p, Mrows, total, K, acc);
+            else if (pairs) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 16, 2>, A, p, Mrows, total, K, acc);
+            else if (k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 8, 1>, A, p, Mrows, total, K, acc);
+            else cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc);
+        } else if constexpr (NB == 4 && U == 4) {
+            if (k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 8, 1>, A, p, Mrows, total, K, acc);
+            else cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc);
+        }
+    }
+    else if (k.nw == 16 && k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 8>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
+    else if (k.nw == 16) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 16>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
+    else cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 8, 16>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
+}
+
+static void launch_skinny_pick(const bf16 *A, const GemvParts &p, const SkinnyPick &k, uint32_t Mrows, uint32_t K, int acc, cudaStream_t st) {
+    if (k.nb == 1) { if (k.u == 8) launch_skinny<1, 8>(A, p, k, Mrows, K, acc, st); else launch_skinny<1, 4>(A, p, k, Mrows, K, acc, st); }
+    else if (k.nb == 2) { if (k.u == 8) launch_skinny<2, 8>(A, p, k, Mrows, K, acc, st); else launch_skinny<2, 4>(A, p, k, Mrows, K, acc, st); }
+    else { if (k.u == 4) launch_skinny<4, 4>(A, p, k, Mrows, K, acc, st); else launch_skinny<4, 2>(A, p, k, Mrows, K, acc, st); }
 }
 
 template <int MT, int RB, int U>
@@ -998,8 +1155,6 @@ static void launch_gemv_splitk(const bf16 *A, const bf16 *W, float *C, uint32_t 
     cudaLaunchKernelEx(&cfg, gemv_splitk_kernel<MT, RB, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
 }
 
-static int g_gemv_splitk = 1;    // small-n blocks at M <= 2: CTA per RB rows with K split over its warps (0: one warp per row)
-
 // rows per warp: fewer when the block has few rows, so that every SM still gets warps
 template <int MT>
 static void launch_gemv_rows(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int acc, cudaStream_t st) {
@@ -1016,10 +1171,8 @@ static void launch_gemv_rows(const bf16 *A, const bf16 *W, float *C, uint32_t Mr
     }
 }
 
-static int g_gemm_group = 1;     // products over the same activations: one launch where the parts allow it (0: always one launch each)
-
 template <int MT>
-static void launch_gemv_group(const bf16 *A, const GemvParts &p, uint32_t Mrows, uint32_t n_total, uint32_t K, cudaStream_t st) {
+static void launch_gemv_group(const bf16 *A, const GemvParts &p, uint32_t Mrows, uint32_t n_total, uint32_t K, int acc, cudaStream_t st) {
     static int blocks_per_sm = 0, sms = 0;
     if (!blocks_per_sm) {
         int dev = 0;
@@ -1038,22 +1191,33 @@ static void launch_gemv_group(const bf16 *A, const GemvParts &p, uint32_t Mrows,
     attr[0].val.programmaticStreamSerializationAllowed = g_gemv_pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, gemv_group_kernel<MT, 8>, A, p, Mrows, n_total, K);
+    cudaLaunchKernelEx(&cfg, gemv_group_kernel<MT, 8>, A, p, Mrows, n_total, K, acc);
 }
 
-// One launch serves the whole group exactly when every part alone would take gemv_kernel<MT, 1, 8> (M <= 2, fewer rows
-// in total than two waves of warps, K below the split-K threshold): same arithmetic, so the same bits.
-bool tgpk_gemm_group_fused(uint32_t count, const uint32_t *n, uint32_t M, uint32_t K) {
-    if (!g_gemm_group || count < 2 || count > TGP_GEMM_GROUP_MAX || !M || M > 2 || !K || K % 8) return false;
-    uint64_t total = 0;
-    for (uint32_t s = 0; s < count; ++s) { if (!n[s]) return false; total += n[s]; }
-    return total < 2 * 148 * 16 && !(g_gemv_splitk && K >= 8192);
+// Which products may share a launch: those with the same non-zero key.  A key names the kernel a block takes on its own
+// (M <= 2: gemv_kernel<MT, 1, 8>; 3 <= M <= 32: one instance of the split-K skinny kernel); blocks of so many rows that
+// they fill the machine alone, and the shapes served by other kernels, have key 0 and are launched alone.
+uint32_t tgpk_gemm_group_key(uint32_t M, uint32_t n, uint32_t K) {
+    if (!g_gemm_group || !M || !n || !K || K % 8) return 0;
+    if (M >= 3 && M <= 32 && K % 32 == 0 && g_skinny_impl == 0) {
+        const SkinnyPick k = pick_skinny(M, n, K);
+        // grouping pays where a block alone has fewer 16-row groups than the GPU has SMs (those take the 16-warp kernels)
+        const bool few = (n + 15) / 16 < (uint32_t)device_sms();
+        return (k.split && few && k.nw == 16) ? (0x1000000u | (uint32_t)k.nb | (uint32_t)k.u << 4 | (uint32_t)k.nw << 8 | (uint32_t)k.rows << 16) : 0;
+    }
+    if (M <= 2) return (n < 2 * 148 * 16 && !(g_gemv_splitk && K >= 8192)) ? M : 0;
+    return 0;
 }
 
-int tgpk_gemm_group(const void *A, uint32_t count, const void *const *W, float *const *C, const uint32_t *n, const uint32_t *ldc, uint32_t M, uint32_t K, cudaStream_t st) {
-    if (!tgpk_gemm_group_fused(count, n, M, K)) {
+int tgpk_gemm_group(const void *A, uint32_t count, const void *const *W, float *const *C, const uint32_t *n, const uint32_t *ldc, uint32_t M, uint32_t K,
+                    int accumulate, cudaStream_t st) {
+    if (!count || !M) return TGP_OK;
+    const uint32_t key = tgpk_gemm_group_key(M, n[0], K);
+    bool same = key != 0 && count >= 2 && count <= TGP_GEMM_GROUP_MAX;
+    for (uint32_t s = 1; s < count && same; ++s) same = tgpk_gemm_group_key(M, n[s], K) == key;
+    if (!same) {
         for (uint32_t s = 0; s < count; ++s) {
-            const int rc = tgpk_gemm(A, W[s], C[s], M, n[s], K, ldc[s], 0, 0, st);
+            const int rc = tgpk_gemm(A, W[s], C[s], M, n[s], K, ldc[s], 0, accumulate, st);
             if (rc) return rc;
         }
         return TGP_OK;
@@ -1063,27 +1227,23 @@ int tgpk_gemm_group(const void *A, uint32_t count, const void *const *W, float *
     uint32_t total = 0;
     for (uint32_t s = 0; s < count; ++s) { p.W[s] = (const bf16 *)W[s]; p.C[s] = C[s]; p.n[s] = n[s]; p.ldc[s] = ldc[s]; total += n[s]; }
     p.count = count;
-    if (M == 1) launch_gemv_group<1>((const bf16 *)A, p, M, total, K, st);
-    else launch_gemv_group<2>((const bf16 *)A, p, M, total, K, st);
+    if (M == 1) launch_gemv_group<1>((const bf16 *)A, p, M, total, K, accumulate, st);
+    else if (M == 2) launch_gemv_group<2>((const bf16 *)A, p, M, total, K, accumulate, st);
+    else launch_skinny_pick((const bf16 *)A, p, pick_skinny(M, n[0], K), M, K, accumulate, st);
     LAUNCH_CHECK(1);
     return TGP_OK;
 }
 
-static int g_skinny_impl = 0;    // 0: tensor-core skinny kernel for 3 <= M <= 32; 1: CUDA-core GEMV (an on-device cross-check)
-static int g_gemm_impl = 0;      // 0: tensor cores for M > 16; 1: CUDA-core tiles (kept as an on-device cross-check)
 
 int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
     if (!M || !n) return TGP_OK;
     if (K % 8 || !K) return TGP_E_INVAL;
     const bf16 *a = (const bf16 *)A, *w = (const bf16 *)W;
     if (M >= 3 && M <= 32 && K % 32 == 0 && g_skinny_impl == 0) {
-        // fewer 16-row groups than SMs: few CTAs, so each warp keeps twice the loads in flight
-        static int sms = 0;
-        if (!sms) { int dev = 0; cudaGetDevice(&dev); if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148; }
-        const bool few = (n + 15) / 16 < (uint32_t)sms;
-        if (M <= 8) { if (few) launch_gemv_mma<1, 8>(a, w, C, M, n, K, ldc, col0, accumulate, st); else launch_gemv_mma<1, 4>(a, w, C, M, n, K, ldc, col0, accumulate, st); }
-        else if (M <= 16) { if (few) launch_gemv_mma<2, 8>(a, w, C, M, n, K, ldc, col0, accumulate, st); else launch_gemv_mma<2, 4>(a, w, C, M, n, K, ldc, col0, accumulate, st); }
-        else { if (few) launch_gemv_mma<4, 4>(a, w, C, M, n, K, ldc, col0, accumulate, st); else launch_gemv_mma<4, 2>(a, w, C, M, n, K, ldc, col0, accumulate, st); }
+        GemvParts p;
+        memset(&p, 0, sizeof(p));
+        p.W[0] = w; p.C[0] = C + col0; p.n[0] = n; p.ldc[0] = ldc; p.count = 1;
+        launch_skinny_pick(a, p, pick_skinny(M, n, K), M, K, accumulate, st);
     } else if (M <= 16) {
         for (uint32_t m0 = 0; m0 < M; m0 += 8) {
             uint32_t mr = M - m0 < 8 ? M - m0 : 8;
@@ -1207,10 +1367,16 @@ int tgp_k_skinny_select(int impl) {
 }
 
 int tgp_k_gemm_group(const void *A_dev, uint32_t count, const void *const *W_dev, float *const *C_dev, const uint32_t *n, const uint32_t *ldc,
-                     uint32_t M, uint32_t K, void *stream) {
-    if (!A_dev || !W_dev || !C_dev || !n || !ldc || !count || count > TGP_GEMM_GROUP_MAX) return TGP_E_INVAL;
+                     uint32_t M, uint32_t K, int accumulate, void *stream) {
+    if (!A_dev || !W_dev || !C_dev || !n || !ldc || !count || count > TGP_GEMM_GROUP_MAX || !K || K % 8) return TGP_E_INVAL;
     for (uint32_t s = 0; s < count; ++s) if (!W_dev[s] || !C_dev[s] || n[s] > ldc[s]) return TGP_E_INVAL;
-    return tgpk_gemm_group(A_dev, count, W_dev, C_dev, n, ldc, M, K, (cudaStream_t)stream);
+    return tgpk_gemm_group(A_dev, count, W_dev, C_dev, n, ldc, M, K, accumulate, (cudaStream_t)stream);
+}
+
+int tgp_k_gemm_group_key(uint32_t M, uint32_t n, uint32_t K, uint32_t *key) {
+    if (!key) return TGP_E_INVAL;
+    *key = tgpk_gemm_group_key(M, n, K);
+    return TGP_OK;
 }
 
 int tgp_k_gemm_group_select(int enable) {

@@ -11,10 +11,12 @@ struct TgpTilePtrs { void *k[TGP_MAX_TILES]; void *v[TGP_MAX_TILES]; };
 int tgpk_embed(const void *table, const int32_t *tok, float *x, uint32_t M, uint32_t d, cudaStream_t st);
 int tgpk_rmsnorm(const float *x, uint32_t ldx, const void *g, void *h, uint32_t M, uint32_t d, float eps, cudaStream_t st);
 int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st);
-// count (2..TGP_GEMM_GROUP_MAX) products over the same activations A [M, K]: C[s][m, j] = sum_k A[m, k] * W[s][j, k]; one launch when
-// tgpk_gemm_group_fused() says so, else one launch per part; the bits are the same either way
-bool tgpk_gemm_group_fused(uint32_t count, const uint32_t *n, uint32_t M, uint32_t K);
-int tgpk_gemm_group(const void *A, uint32_t count, const void *const *W, float *const *C, const uint32_t *n, const uint32_t *ldc, uint32_t M, uint32_t K, cudaStream_t st);
+// products over the same activations A [M, K]: C[s][m, j] (=|+=) sum_k A[m, k] * W[s][j, k].  Blocks with the same non-zero
+// tgpk_gemm_group_key() are served by one launch (up to TGP_GEMM_GROUP_MAX of them), anything else by one launch per part;
+// the bits are the same either way
+uint32_t tgpk_gemm_group_key(uint32_t M, uint32_t n, uint32_t K);
+int tgpk_gemm_group(const void *A, uint32_t count, const void *const *W, float *const *C, const uint32_t *n, const uint32_t *ldc, uint32_t M, uint32_t K,
+                    int accumulate, cudaStream_t st);
 // tcgen05 path (tgp_gemm_sm100.cu): any M, n; K % 8 == 0; A and W 16-byte aligned
 int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st);
 int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb, const TgpTilePtrs &tiles, const float *cos_t, const float *sin_t,

@@ -365,43 +365,57 @@ def test_overlapping_gemv_launches_keep_their_dependencies():
     assert np.abs(outs[0] - want).max() < 1e-4 * np.abs(want).max()
 
 
-@pytest.mark.parametrize("M,ns,K", [(1, (2048, 512, 512), 2048),      # the q, k, v projections of the 1B shape: one launch
-                                    (2, (300, 7, 129, 1), 264),         # four ragged parts, K not a multiple of the chunk
-                                    (1, (4096, 1024), 4096),            # too many rows for one launch: one launch per part
-                                    (2, (640, 640, 64), 8192),          # long K: the parts take the split-K kernel
-                                    (8, (1024, 256, 256), 512)])        # M > 2: one launch per part
-def test_grouped_products_equal_single_products_and_oracle(M, ns, K):
+@pytest.mark.parametrize("M,ns,K,grouped", [
+    (1, (2048, 512, 512), 2048, True),            # the q, k, v projections of the 1B shape: one launch
+    (2, (300, 7, 129, 1), 264, True),             # four ragged parts, K not a multiple of the chunk
+    (1, (4096, 8192), 4096, False),               # a block of many rows is launched alone
+    (2, (640, 640, 64), 8192, False),             # long K at M <= 2: the parts take the split-K kernel, alone
+    (8, (1152, 1152, 1152, 640), 14336, True),    # the pieces of an 8B down projection: 8-row CTAs, 16 warps
+    (16, (512,) * 8, 28672, True),                # eight pieces of a 70B down projection
+    (8, (1024, 1024), 4096, True),                # k and v of the 8B shape
+    (8, (4096, 1024), 4096, False),               # q and k pick different kernels: one launch each
+    (32, (500, 260, 33), 160, True),              # ragged row counts, four groups of activation rows
+    (5, (24000, 64), 64, False),                  # a block that fills the machine alone
+    (40, (256, 256), 512, False)])                # more activation rows than the skinny kernels take
+@pytest.mark.parametrize("accumulate", [0, 1])
+def test_grouped_products_equal_single_products_and_oracle(M, ns, K, grouped, accumulate):
     """Products that share their activations: the grouped call must give the bits of one tgp_k_gemm() call per part,
     whether it runs as one launch or falls back to one launch per part, with the switch on and off, and leave the
     columns beyond each part untouched; the values are checked against the oracle's linear()."""
+    keys = {tb.k_gemm_group_key(M, n, K) for n in ns}
+    assert (len(keys) == 1 and 0 not in keys) == grouped
     a_bits = rnd_bits(51, M * K).reshape(M, K)
     A = bf16_dev(a_bits)
     w_bits = [rnd_bits(60 + s, n * K).reshape(n, K) for s, n in enumerate(ns)]
     Wd = [bf16_dev(w) for w in w_bits]
     ldcs = [n + 8 * (s + 1) for s, n in enumerate(ns)]
-    single = [torch.full((M, ld), -7.0, dtype=torch.float32, device=DEV) for ld in ldcs]
+    c0 = [np.random.default_rng(100 + s).standard_normal((M, ld)).astype(np.float32) * 0.01 for s, ld in enumerate(ldcs)]
+    fresh = lambda: [torch.from_numpy(c.copy()).to(DEV) for c in c0]
+    single = fresh()
     for s, n in enumerate(ns):
-        tb.k_gemm(A, Wd[s], single[s], M, n, K, ldcs[s], 0, 0)
+        tb.k_gemm(A, Wd[s], single[s], M, n, K, ldcs[s], 0, accumulate)
     outs = []
     for enable in (1, 0):
         tb.k_gemm_group_select(enable)
-        grouped = [torch.full((M, ld), -7.0, dtype=torch.float32, device=DEV) for ld in ldcs]
-        tb.k_gemm_group(A, Wd, grouped, M, list(ns), K, ldcs)
+        out = fresh()
+        tb.k_gemm_group(A, Wd, out, M, list(ns), K, ldcs, accumulate)
         torch.cuda.synchronize()
-        outs.append([g.cpu().numpy() for g in grouped])
+        outs.append([g.cpu().numpy() for g in out])
+        assert enable or tb.k_gemm_group_key(M, ns[0], K) == 0
     tb.k_gemm_group_select(1)
     o = oracle()
     a = si.bf16_bits_to_f32(a_bits)
     for s, n in enumerate(ns):
         ref = single[s].cpu().numpy()
         assert np.array_equal(outs[0][s], ref) and np.array_equal(outs[1][s], ref)
-        assert (ref[:, n:] == -7.0).all()
-        want = o.linear(a, si.bf16_bits_to_f32(w_bits[s]).astype(np.float64)).astype(np.float64)
+        assert np.array_equal(ref[:, n:], c0[s][:, n:])
+        want = o.linear(a, si.bf16_bits_to_f32(w_bits[s]).astype(np.float64)).astype(np.float64) + (c0[s][:, :n] if accumulate else 0)
         assert np.abs(ref[:, :n] - want).max() < 2e-5 * max(np.abs(want).max(), 0.01) + 1e-7
-    with pytest.raises(tb.TgpError):
-        tb.k_gemm_group(A, Wd[:1] * 5, [single[0]] * 5, M, [ns[0]] * 5, K, [ldcs[0]] * 5)      # more parts than the call takes
-    with pytest.raises(tb.TgpError):
-        tb.k_gemm_group(A, Wd[:2], single[:2], M, [ns[0], ns[1]], K, [ns[0] - 1, ldcs[1]])       # row stride below the part's width
+    if M == 1 and accumulate == 0:
+        with pytest.raises(tb.TgpError):
+            tb.k_gemm_group(A, Wd[:1] * 9, [single[0]] * 9, M, [ns[0]] * 9, K, [ldcs[0]] * 9)      # more parts than the call takes
+        with pytest.raises(tb.TgpError):
+            tb.k_gemm_group(A, Wd[:2], single[:2], M, [ns[0], ns[1]], K, [ns[0] - 1, ldcs[1]])       # row stride below the part's width
 
 
 @pytest.mark.parametrize("M,n,K", [(3, 100, 64), (8, 4096, 4096), (8, 1030, 512), (13, 77, 128), (16, 260, 1024), (17, 64, 96), (24, 2049, 2048),
