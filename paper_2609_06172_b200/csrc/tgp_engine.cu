@@ -587,6 +587,11 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
                 gC[j] = t.C + r.row0; gn[j] = r.rows; gld[j] = t.ldc;
                 cnt = j + 1;
             }
+            // A grouped launch keeps the ring slots of its first blocks until its last block has arrived and the launch has
+            // run.  Against copies of megabytes that wait is a percent of the copy time; against copies of a few
+            // microseconds it is as long as the copies themselves, so small blocks whose slot a later copy waits for stay alone.
+            for (uint32_t j = 0; j + 1 < cnt; ++j)
+                if (ctx->plan.op_is_wait_target[i + j] && ctx->tensors[ctx->acc[ctx->ops[i + j].acc0].tensor].size < (2u << 20)) cnt = 0;
             if (cnt >= 2) span = cnt;
             for (uint32_t j = 0; j < span && span > 1 && g_expert >= 0; ++j) {       // what run_expert_block does around an expert's products
                 const TgpRole &r = ctx->roles[ctx->role_of_tensor[ctx->acc[ctx->ops[i + j].acc0].tensor]];
