@@ -264,14 +264,17 @@ int  tgp_k_gemm(const void *A_dev, const void *W_dev, float *C_dev, uint32_t M, 
  * returns.  Blocks whose tgp_k_gemm_group_key() is the same non-zero value are served by one launch - a block of few
  * rows alone leaves most SMs without work - anything else by one launch per part; the results are bit-identical to
  * tgp_k_gemm() per part either way, because the key names the kernel the block takes on its own (M <= 2: fewer than
- * 4736 rows and K < 8192; 3 <= M <= 32 with K % 32 == 0: the blocks of fewer than 128 rows per SM).
+ * 4736 rows and K < 8192; 3 <= M <= 32 with K % 32 == 0: blocks of fewer 16-row groups than the GPU has SMs, which pick
+ * the same split-K kernel instance).
  * tgp_k_gemm_group_select(0) makes every key 0 (process-wide; default 1), also inside tgp_step(), which groups
  * consecutive weight-block products of a decode step that read the same activations this way when their copies have
- * all been enqueued and no tap is set (with op timing the launch's time is reported for the first product of the group
- * and an empty bracket for the others). */
+ * all been enqueued and no tap is set, except blocks under 2 MiB whose arena slot a later copy waits for (with op timing
+ * the launch's time is reported for the first product of the group and an empty bracket for the others). */
 #define TGP_GEMM_GROUP_MAX 8u
 int  tgp_k_gemm_group(const void *A_dev, uint32_t count, const void *const *W_dev, float *const *C_dev, const uint32_t *n,
                       const uint32_t *ldc, uint32_t M, uint32_t K, int accumulate, void *stream);
+/* *key = 0 if a block [n, K] at M activation rows is always launched alone, else a value such that blocks of equal
+ * key may share a launch.  Needs a current device (the rule depends on its SM count). */
 int  tgp_k_gemm_group_key(uint32_t M, uint32_t n, uint32_t K, uint32_t *key);
 int  tgp_k_gemm_group_select(int enable);
 /* Which kernel serves M > 16: 0 (default) the tcgen05 tensor-core GEMM, 1 the CUDA-core tile kernel (an on-device
