@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <cstdint>
+#include <type_traits>
 #include "tgp.h"
 #include "tgp_kernels.h"
 
@@ -549,7 +550,7 @@ __global__ void attn_decode_partial_kernel(AttnArgs a, uint32_t SPLIT) {
 // shuffle).  Per-warp online softmax; the SPLIT partials of a head are merged in warp order; output as in the
 // per-head kernel: (max, sum, unnormalised o[DH]) per (sequence, head, tile) for attn_decode_merge_kernel.
 template <int DH, int G>
-__global__ void __launch_bounds__(256) attn_decode_group_kernel(AttnArgs a, uint32_t SPLIT) {
+__global__ void __launch_bounds__(256, 2) attn_decode_group_kernel(AttnArgs a, uint32_t SPLIT) {
     extern __shared__ float dsm[];
     constexpr int DPL = DH / 32;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -575,6 +576,14 @@ __global__ void __launch_bounds__(256) attn_decode_group_kernel(AttnArgs a, uint
     for (uint32_t j0 = warp * 32; j0 < nk; j0 += SPLIT * 32) {
         const uint32_t j = j0 + lane, cnt = min(32u, nk - j0);
         const bool valid = j < nk;
+        // the first 16 value rows are requested before the scores are computed: they depend on nothing computed here, and
+        // the chunk is one serial chain per warp (key rows, scores, softmax, value rows), so every load moved off it counts
+        typedef typename std::conditional<DPL == 4, uint2, uint32_t>::type vraw_t;
+        constexpr uint32_t PRE = (G * DPL >= 32) ? 4 : 16;          // eight heads of 128 dimensions leave few registers for it
+        vraw_t vpre[PRE];
+#pragma unroll
+        for (uint32_t t = 0; t < PRE; ++t)
+            vpre[t] = *reinterpret_cast<const vraw_t *>(vt + (size_t)(j0 + min(t, cnt - 1)) * DH + lane * DPL);
         // ---- scores: this lane's key against the G queries ----
         float acc[G];
 #pragma unroll
@@ -618,16 +627,23 @@ __global__ void __launch_bounds__(256) attn_decode_group_kernel(AttnArgs a, uint
             mx[g] = mnew;
         }
         // ---- P V: this lane's DPL output dimensions; rows past the end re-read the last valid row with weight 0 ----
-#pragma unroll 16
+        vraw_t vlate[16];
+#pragma unroll
+        for (uint32_t t = 0; t < 16; ++t)
+            vlate[t] = *reinterpret_cast<const vraw_t *>(vt + (size_t)(j0 + min(t + PRE, cnt - 1)) * DH + lane * DPL);
+#pragma unroll
         for (uint32_t t = 0; t < 32; ++t) {
-            const bf16 *vr = vt + (size_t)(j0 + min(t, cnt - 1)) * DH + lane * DPL;
+            if (t == PRE + 16) {                                     // (only when fewer than 16 rows were requested early)
+#pragma unroll
+                for (uint32_t u = 0; u < 16 - PRE; ++u)
+                    vlate[u] = *reinterpret_cast<const vraw_t *>(vt + (size_t)(j0 + min(u + PRE + 16, cnt - 1)) * DH + lane * DPL);
+            }
+            const vraw_t raw = t < PRE ? vpre[t % PRE] : vlate[(t - PRE) % 16];
             float f[DPL];
-            if (DPL == 4) {
-                const uint2 raw = *reinterpret_cast<const uint2 *>(vr);
+            if constexpr (DPL == 4) {
                 const __nv_bfloat162 a0 = *reinterpret_cast<const __nv_bfloat162 *>(&raw.x), a1 = *reinterpret_cast<const __nv_bfloat162 *>(&raw.y);
-                f[0] = __low2float(a0); f[1] = __high2float(a0); f[2 % DPL] = __low2float(a1); f[3 % DPL] = __high2float(a1);
+                f[0] = __low2float(a0); f[1] = __high2float(a0); f[2] = __low2float(a1); f[3] = __high2float(a1);
             } else {
-                const uint32_t raw = *reinterpret_cast<const uint32_t *>(vr);
                 const __nv_bfloat162 a0 = *reinterpret_cast<const __nv_bfloat162 *>(&raw);
                 f[0] = __low2float(a0); f[1 % DPL] = __high2float(a0);
             }
