@@ -633,10 +633,12 @@ __global__ void __launch_bounds__(256, 2) attn_decode_group_kernel(AttnArgs a, u
             vlate[t] = *reinterpret_cast<const vraw_t *>(vt + (size_t)(j0 + min(t + PRE, cnt - 1)) * DH + lane * DPL);
 #pragma unroll
         for (uint32_t t = 0; t < 32; ++t) {
-            if (t == PRE + 16) {                                     // (only when fewer than 16 rows were requested early)
+            if constexpr (PRE < 16) {                                // fewer than 16 rows were requested early: a third batch
+                if (t == PRE + 16) {
 #pragma unroll
-                for (uint32_t u = 0; u < 16 - PRE; ++u)
-                    vlate[u] = *reinterpret_cast<const vraw_t *>(vt + (size_t)(j0 + min(u + PRE + 16, cnt - 1)) * DH + lane * DPL);
+                    for (uint32_t u = 0; u + PRE < 16; ++u)
+                        vlate[u] = *reinterpret_cast<const vraw_t *>(vt + (size_t)(j0 + min(u + PRE + 16, cnt - 1)) * DH + lane * DPL);
+                }
             }
             const vraw_t raw = t < PRE ? vpre[t % PRE] : vlate[(t - PRE) % 16];
             float f[DPL];
