@@ -280,7 +280,8 @@ int  tgp_k_gemm_group_select(int enable);
 /* Which kernel serves M > 16: 0 (default) the tcgen05 tensor-core GEMM, 1 the CUDA-core tile kernel (an on-device
  * cross-check).  M <= 16 always takes the weight-streaming GEMV.  Process-wide. */
 int  tgp_k_gemm_select(int impl);
-/* Which kernel serves 3 <= M <= 32 (K % 32 == 0): 0 (default) the weight-streaming tensor-core kernel, 1 the
+/* Which kernel serves 3 <= M <= 32 (K % 32 == 0; and, as two launches of half the rows, 33 <= M <= 64 on blocks of fewer
+ * than two 16-row groups per SM): 0 (default) the weight-streaming tensor-core kernel, 1 the
  * CUDA-core GEMV (M <= 16) / GEMM paths (an on-device cross-check).  Process-wide. */
 int  tgp_k_skinny_select(int impl);
 /* Weight-streaming launches (M <= 32) use programmatic dependent launch so that a launch may begin reading its

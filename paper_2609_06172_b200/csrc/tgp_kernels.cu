@@ -1262,6 +1262,19 @@ int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, ui
         memset(&p, 0, sizeof(p));
         p.W[0] = w; p.C[0] = C + col0; p.n[0] = n; p.ldc[0] = ldc; p.count = 1;
         launch_skinny_pick(a, p, pick_skinny(M, n, K), M, K, accumulate, st);
+    } else if (M > 32 && M <= 64 && K % 32 == 0 && g_skinny_impl == 0 && g_gemm_impl == 0 && (n + 15) / 16 < 2u * (uint32_t)device_sms()) {
+        // 33 - 64 activation rows on a block of few rows: the tiled GEMM would run a handful of CTAs with a serial K loop
+        // (n=1024, K=4096: 15.8 us); two weight-streaming launches of half the rows each read the block twice, the
+        // second time from L2, and are faster (9.9 us)
+        const uint32_t m1 = (M + 1) / 2;
+        for (uint32_t m0 = 0; m0 < M; m0 += m1) {
+            const uint32_t mr = M - m0 < m1 ? M - m0 : m1;
+            GemvParts p;
+            memset(&p, 0, sizeof(p));
+            p.W[0] = w; p.C[0] = C + (size_t)m0 * ldc + col0; p.n[0] = n; p.ldc[0] = ldc; p.count = 1;
+            launch_skinny_pick(a + (size_t)m0 * K, p, pick_skinny(mr, n, K), mr, K, accumulate, st);
+            if (m0) tgpk_launches += 1;
+        }
     } else if (M <= 16) {
         for (uint32_t m0 = 0; m0 < M; m0 += 8) {
             uint32_t mr = M - m0 < 8 ? M - m0 : 8;

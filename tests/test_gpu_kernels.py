@@ -46,7 +46,9 @@ def bf16_close(got_f32, want_f32, frac=0.01):
                                    (1000, 136, 8192),
                                    # few rows, long K at M <= 2: the split-K GEMV (two rows per CTA; one row per CTA up to 1024 rows),
                                    # odd row counts, K not a multiple of the 256-element chunk, more CTAs than resident slots
-                                   (1, 2048, 8192), (2, 2051, 8200), (1, 513, 8192), (2, 1, 16384), (1, 4735, 8192)])
+                                   (1, 2048, 8192), (2, 2051, 8200), (1, 513, 8192), (2, 1, 16384), (1, 4735, 8192),
+                                   # 33 - 64 activation rows on a block of few rows: two weight-streaming launches of half the rows
+                                   (33, 1030, 512), (48, 2049, 4096), (64, 130, 96), (40, 4720, 64)])
 @pytest.mark.parametrize("accumulate", [0, 1])
 def test_gemm_matches_oracle(M, n, K, accumulate):
     a_bits, w_bits = rnd_bits(1, M * K).reshape(M, K), rnd_bits(2, n * K).reshape(n, K)
