@@ -281,7 +281,7 @@ int  tgp_k_gemm_group_select(int enable);
  * cross-check).  M <= 16 always takes the weight-streaming GEMV.  Process-wide. */
 int  tgp_k_gemm_select(int impl);
 /* Which kernel serves 3 <= M <= 32 (K % 32 == 0; and, as two launches of half the rows, 33 <= M <= 64 on blocks of fewer
- * than two 16-row groups per SM): 0 (default) the weight-streaming tensor-core kernel, 1 the
+ * than 4096 rows): 0 (default) the weight-streaming tensor-core kernel, 1 the
  * CUDA-core GEMV (M <= 16) / GEMM paths (an on-device cross-check).  Process-wide. */
 int  tgp_k_skinny_select(int impl);
 /* Weight-streaming launches (M <= 32) use programmatic dependent launch so that a launch may begin reading its
@@ -290,7 +290,9 @@ int  tgp_k_skinny_select(int impl);
 int  tgp_k_gemv_overlap(int enable);
 /* Tensor-core GEMM variant: 0 (default) picks by problem size, 1 forces the 128x128 one-tile-per-CTA kernel,
  * 2 the persistent 128x256 kernel with double-buffered accumulators, 3 the paired kernel (256x256 tiles on the two SMs
- * of a CTA pair, each loading half of the weight tile).  Process-wide; for tests and timing. */
+ * of a CTA pair, each loading half of the weight tile), 4 the one-tile-per-CTA kernel with the operands swapped (the
+ * weights are the 128-row operand, the tile is stored transposed; for M <= 128, else as 0; picked by size for M <= 64 on
+ * blocks of many rows).  Process-wide; for tests and timing. */
 int  tgp_k_gemm_tc_variant(int variant);
 /* Which kernel serves attention with q_len >= 16: 0 (default) by problem size - the tcgen05 kernel (S and O in TMEM,
  * K/V fed by TMA) for q_len >= 128, else the mma.sync flash-style kernel;

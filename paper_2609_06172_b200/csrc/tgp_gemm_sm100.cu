@@ -33,7 +33,11 @@ struct Smem {
 };
 
 // (ST stages of KH 64-wide K blocks each: with KH = 2 the producer and the MMA thread meet half as often)
-template <int BN, int ST, int KH>
+// SWAP: the operands trade places - the tile's 128 rows are weight rows (M counts them), its BN columns activation rows
+// (n counts them) - and the tile is stored transposed, C[activation row][col0 + weight row].  For products of up to 128
+// activation rows a CTA then streams 128 weight rows through its TMA ring instead of BN, which is what such a product
+// is bound by.
+template <int BN, int ST, int KH, bool SWAP>
 __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                                                       float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     extern __shared__ uint8_t smem_raw[];
@@ -123,7 +127,17 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
             for (uint32_t c = 0; c < BN / 32; ++c) {
                 float v[32];
                 tmem_ld32(tmem_base + ((quarter * 32) << 16) + c * 32, v);
-                if (row < M) {
+                if (SWAP) {
+                    // a warp's 32 lanes hold 32 consecutive weight rows: for each activation row they write 128 contiguous bytes
+                    if (row < M) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + c * 32 + j < n) {
+                                float *d = C + (size_t)(n0 + c * 32 + j) * ldc + col0 + row;
+                                *d = accumulate ? *d + v[j] : v[j];
+                            }
+                    }
+                } else if (row < M) {
                     float *dst = C + (size_t)row * ldc + col0 + n0 + c * 32;
                     const uint32_t col = n0 + c * 32;
                     if (vec && col + 32 <= n) {
@@ -449,19 +463,20 @@ bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t K, uin
 
 extern thread_local uint64_t tgpk_launches;
 
-template <int BN, int ST, int KH>
+template <int BN, int ST, int KH, bool SWAP = false>
 static bool launch_tile(const CUtensorMap &ma, const CUtensorMap &mb, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(gemm_tc_kernel<BN, ST, KH>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN, ST, KH>::TOTAL) != cudaSuccess) return false;
+        if (cudaFuncSetAttribute(gemm_tc_kernel<BN, ST, KH, SWAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN, ST, KH>::TOTAL) != cudaSuccess) return false;
         attr_set = true;
     }
     dim3 grid(((M + BM - 1) / BM) * ((n + BN - 1) / BN));
-    gemm_tc_kernel<BN, ST, KH><<<grid, 192, Smem<BN, ST, KH>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
+    gemm_tc_kernel<BN, ST, KH, SWAP><<<grid, 192, Smem<BN, ST, KH>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
     return true;
 }
 
-static int g_tc_variant = 0;     // 0 auto, 1 force the 128x128 per-tile kernel, 2 the persistent 128x256 kernel, 3 the paired 256x256 kernel
+static int g_tc_variant = 0;     // 0 auto, 1 force the 128x128 per-tile kernel, 2 the persistent 128x256 kernel, 3 the paired 256x256 kernel,
+                                 // 4 the per-tile kernel with the weights as the 128-row operand (M <= 128 only; else as 0)
 
 int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
     constexpr int BN = 128;
@@ -469,6 +484,23 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
     if (K % 8) return TGP_E_INVAL;                                                                       // and 16-byte row strides
     static int sms = 0;
     if (!sms) { int dev = 0; cudaGetDevice(&dev); if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148; }
+    // Up to 64 activation rows on a block with 128-row tiles for a good part of the SMs: the weights become the 128-row
+    // operand (see gemm_tc_kernel), the activations the narrow one.  A CTA takes in about 100 GB/s through its TMA ring
+    // whatever the tile, so the form pays from 64 weight tiles on (n=8192, K=8192, M=64: 34 us against 47 us), for more
+    // than 32 rows from 32 tiles on (n=4096, K=14336, M=64: 48 us against 70 us); with fewer tiles the weight-streaming
+    // kernels and the narrow tiles below have more CTAs at work
+    const uint32_t w_tiles = (n + BM - 1) / BM;
+    if (M <= 128 && (g_tc_variant == 4 || (g_tc_variant == 0 && M <= 64 && (w_tiles >= 64 || (M > 32 && w_tiles >= 32))))) {
+        CUtensorMap mw, mx;
+        const uint32_t bx = M <= 32 ? 32 : M <= 64 ? 64 : 128;
+        if (!make_map(&mw, W, n, K, BM) || !make_map(&mx, A, M, K, bx)) return TGP_E_CUDA;
+        const bool ok = bx == 32 ? launch_tile<32, 3, 3, true>(mw, mx, C, n, M, K, ldc, col0, accumulate, st)
+                      : bx == 64 ? launch_tile<64, 3, 3, true>(mw, mx, C, n, M, K, ldc, col0, accumulate, st)
+                                 : launch_tile<128, 2, 3, true>(mw, mx, C, n, M, K, ldc, col0, accumulate, st);
+        if (!ok || cudaGetLastError() != cudaSuccess) return TGP_E_CUDA;
+        tgpk_launches += 1;
+        return TGP_OK;
+    }
     const uint32_t tiles_p = ((M + BM - 1) / BM) * ((n + P_BN - 1) / P_BN);
     const uint32_t tiles_q = ((M + 2 * BM - 1) / (2 * BM)) * ((n + P_BN - 1) / P_BN);
     // measured on 8192 x {640 .. 4096} x {4096, 14336}, {1024 .. 4096} x 4096 x 4096 and {512, 1024} x 8192 x 2048: the paired
@@ -527,7 +559,7 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
 }
 
 extern "C" int tgp_k_gemm_tc_variant(int v) {
-    if (v < 0 || v > 3) return TGP_E_INVAL;
+    if (v < 0 || v > 4) return TGP_E_INVAL;
     g_tc_variant = v;
     return TGP_OK;
 }

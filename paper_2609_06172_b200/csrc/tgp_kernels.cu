@@ -1257,15 +1257,19 @@ int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, ui
     if (!M || !n) return TGP_OK;
     if (K % 8 || !K) return TGP_E_INVAL;
     const bf16 *a = (const bf16 *)A, *w = (const bf16 *)W;
-    if (M >= 3 && M <= 32 && K % 32 == 0 && g_skinny_impl == 0) {
+    // 17 - 32 activation rows on a block of 64 or more 128-row tiles: the tiled GEMM with the weights as its 128-row operand
+    // is ahead of the weight-streaming kernel (n=8192, K=8192, M=32: 33 us against 41 us)
+    const bool tiles_win = M > 16 && (n + 127) / 128 >= 64 && g_gemm_impl == 0;
+    if (M >= 3 && M <= 32 && K % 32 == 0 && g_skinny_impl == 0 && !tiles_win) {
         GemvParts p;
         memset(&p, 0, sizeof(p));
         p.W[0] = w; p.C[0] = C + col0; p.n[0] = n; p.ldc[0] = ldc; p.count = 1;
         launch_skinny_pick(a, p, pick_skinny(M, n, K), M, K, accumulate, st);
-    } else if (M > 32 && M <= 64 && K % 32 == 0 && g_skinny_impl == 0 && g_gemm_impl == 0 && (n + 15) / 16 < 2u * (uint32_t)device_sms()) {
+    } else if (M > 32 && M <= 64 && K % 32 == 0 && g_skinny_impl == 0 && g_gemm_impl == 0 && n < 4096) {
         // 33 - 64 activation rows on a block of few rows: the tiled GEMM would run a handful of CTAs with a serial K loop
         // (n=1024, K=4096: 15.8 us); two weight-streaming launches of half the rows each read the block twice, the
-        // second time from L2, and are faster (9.9 us)
+        // second time from L2, and are faster (9.9 us); from 32 tiles of 128 rows on the tiled GEMM takes the weights as its
+        // 128-row operand instead
         const uint32_t m1 = (M + 1) / 2;
         for (uint32_t m0 = 0; m0 < M; m0 += m1) {
             const uint32_t mr = M - m0 < m1 ? M - m0 : m1;

@@ -48,7 +48,9 @@ def bf16_close(got_f32, want_f32, frac=0.01):
                                    # odd row counts, K not a multiple of the 256-element chunk, more CTAs than resident slots
                                    (1, 2048, 8192), (2, 2051, 8200), (1, 513, 8192), (2, 1, 16384), (1, 4735, 8192),
                                    # 33 - 64 activation rows on a block of few rows: two weight-streaming launches of half the rows
-                                   (33, 1030, 512), (48, 2049, 4096), (64, 130, 96), (40, 4720, 64)])
+                                   (33, 1030, 512), (48, 2049, 4096), (64, 130, 96), (40, 4090, 64),
+                                   # ... and on blocks of many rows the tiled GEMM with the weights as its 128-row operand
+                                   (40, 4720, 64), (64, 4096, 1032), (20, 8200, 128)])
 @pytest.mark.parametrize("accumulate", [0, 1])
 def test_gemm_matches_oracle(M, n, K, accumulate):
     a_bits, w_bits = rnd_bits(1, M * K).reshape(M, K), rnd_bits(2, n * K).reshape(n, K)
@@ -108,6 +110,31 @@ def test_persistent_tensor_core_gemm_matches_per_tile_kernel_and_oracle(M, n, K,
     for o in outs:
         assert np.abs(o - want).max() < 2e-5 * scale + 1e-7
     assert np.abs(outs[0] - outs[2]).max() < 2e-5 * scale + 1e-7 and np.abs(outs[1] - outs[2]).max() < 2e-5 * scale + 1e-7
+
+
+@pytest.mark.parametrize("M,n,K,acc", [(17, 300, 264, 0), (32, 4100, 1024, 1), (33, 1030, 512, 1), (64, 130, 96, 0), (65, 2049, 1024, 1),
+                                       (128, 4096, 512, 0), (100, 129, 72, 1), (48, 8200, 256, 0)])
+def test_tensor_core_gemm_with_the_weights_as_the_128_row_operand(M, n, K, acc):
+    """Up to 128 activation rows: the per-tile kernel with its operands swapped (tile rows are weight rows, the tile is
+    stored transposed), forced, against the oracle; ragged weight tiles, ragged token counts, a column offset."""
+    a_bits, w_bits = rnd_bits(13, M * K).reshape(M, K), rnd_bits(14, n * K).reshape(n, K)
+    A, W = bf16_dev(a_bits), bf16_dev(w_bits)
+    ldc, col0 = n + 12, 4
+    c0 = np.random.default_rng(9).standard_normal((M, ldc)).astype(np.float32) * 0.01
+    tb.k_gemm_tc_variant(4)
+    tb.k_skinny_select(1)            # 17 - 32 rows reach the tiled GEMM only with the weight-streaming kernel switched off
+    Cd = torch.from_numpy(c0.copy()).to(DEV)
+    tb.k_gemm(A, W, Cd, M, n, K, ldc, col0, acc)
+    torch.cuda.synchronize()
+    tb.k_gemm_tc_variant(0)
+    tb.k_skinny_select(0)
+    assert tb.k_gemm_status() == 0
+    got = Cd.cpu().numpy()
+    want = oracle().linear(si.bf16_bits_to_f32(a_bits), si.bf16_bits_to_f32(w_bits).astype(np.float64)).astype(np.float64)
+    exp = c0.astype(np.float64).copy()
+    exp[:, col0:col0 + n] = want + (c0[:, col0:col0 + n] if acc else 0)
+    assert np.abs(got - exp).max() < 2e-5 * max(np.abs(want).max(), 0.01) + 1e-7
+    assert np.array_equal(got[:, :col0], c0[:, :col0]) and np.array_equal(got[:, col0 + n:], c0[:, col0 + n:])
 
 
 def test_gemm_rejects_bad_arguments_and_accepts_empty():
