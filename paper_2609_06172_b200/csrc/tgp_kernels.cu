@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cstdint>
 #include <type_traits>
+#include <algorithm>
 #include "tgp.h"
 #include "tgp_kernels.h"
 
@@ -879,6 +880,7 @@ static int g_skinny_impl = 0;    // 0: tensor-core skinny kernel for 3 <= M <= 3
 static int g_gemm_impl = 0;      // 0: tensor cores for M > 16; 1: CUDA-core tiles (kept as an on-device cross-check)
 static int g_gemv_splitk = 1;    // small-n blocks at M <= 2: CTA per RB rows with K split over its warps (0: one warp per row)
 static int g_gemm_group = 1;     // products over the same activations: one launch where the parts allow it (0: always one launch each)
+static int g_gemv_balance = 1;   // grouped skinny launches: rows per group chosen so that every persistent CTA gets the same number of groups
 static int g_gemv_rows8 = 1;     // skinny products of few rows and long K: 8-row CTAs (0: always 16)
 static int g_gemv_pdl = 1;       // consecutive weight-streaming launches may overlap (programmatic dependent launch)
 
@@ -973,7 +975,7 @@ __global__ void __launch_bounds__(NW * 32) gemv_mma_splitk_kernel(const bf16 *__
 // same bits as one launch per block.
 template <int NB, int U, int NW, int ROWS, int RG>
 __global__ void __launch_bounds__(NW * 32) gemv_mma_group_kernel(const bf16 *__restrict__ A, const GemvParts p, uint32_t Mrows, uint32_t groups_total,
-                                                              uint32_t K, int accumulate) {
+                                                              uint32_t K, int accumulate, uint32_t rpc) {
     constexpr int UL = ROWS == 8 ? 2 * U : U;             // half a tile per load step: twice the steps in flight
     constexpr int G = RG, SUB = UL / G;                  // SUB load steps of G groups in flight at a time: as many loads as UL of one
     static_assert(UL % G == 0, "row groups per CTA must divide the load steps");
@@ -999,8 +1001,12 @@ __global__ void __launch_bounds__(NW * 32) gemv_mma_group_kernel(const bf16 *__r
                         start += p.groups[s];
                     }
             }
-            wlo[r] = W + (size_t)min(local * ROWS + g, n - 1) * K + c * 8;
-            whi[r] = W + (size_t)min(local * ROWS + g + 8, n - 1) * K + c * 8;
+            // rpc <= ROWS rows per group, chosen by the launcher so that the persistent CTAs all get the same number of
+            // groups; the tile's rows beyond rpc re-read the group's last row and are not stored (a row's sum does not
+            // depend on its place in the tile)
+            const uint32_t rlast = min(local * rpc + rpc, n) - 1;
+            wlo[r] = W + (size_t)min(local * rpc + g, rlast) * K + c * 8;
+            whi[r] = W + (size_t)min(local * rpc + g + 8, rlast) * K + c * 8;
         }
         float acc[G][NB][4];
 #pragma unroll
@@ -1053,18 +1059,18 @@ __global__ void __launch_bounds__(NW * 32) gemv_mma_group_kernel(const bf16 *__r
 #pragma unroll
             for (int w = 0; w < NW; ++w) sum += part[w][slot][ln];
             float *C = p.C[0];
-            uint32_t ldc = p.ldc[0], n = p.n[0], row0 = grp * ROWS;
+            uint32_t ldc = p.ldc[0], n = p.n[0], row0 = grp * rpc;
             {
                 uint32_t start = p.groups[0];
 #pragma unroll
                 for (int s = 1; s < (int)TGP_GEMM_GROUP_MAX; ++s)
                     if (s < (int)p.count) {
-                        if (grp >= start) { C = p.C[s]; ldc = p.ldc[s]; n = p.n[s]; row0 = (grp - start) * ROWS; }
+                        if (grp >= start) { C = p.C[s]; ldc = p.ldc[s]; n = p.n[s]; row0 = (grp - start) * rpc; }
                         start += p.groups[s];
                     }
             }
             const uint32_t m = b * 8 + 2 * (ln & 3) + (i & 1), row = row0 + (ln >> 2) + 8 * (i >> 1);
-            if (m < Mrows && row < n && (ROWS == 16 || (i >> 1) == 0)) {
+            if (m < Mrows && row < min(row0 + rpc, n) && (ROWS == 16 || (i >> 1) == 0)) {
                 float *out = C + (size_t)m * ldc + row;
                 if (accumulate) atomicAdd(out, sum);             // one add per element by one thread, not waited for
                 else *out = sum;
@@ -1108,14 +1114,32 @@ static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint3
     if (!blocks_per_sm_split && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm_split, gemv_mma_splitk_kernel<NB, U, 8, 16>, 256, 0) != cudaSuccess || blocks_per_sm_split < 1))
         blocks_per_sm_split = 1;
     const uint32_t sms = (uint32_t)device_sms();
-    uint32_t need = 0;
-    if (k.split) for (uint32_t s = 0; s < p.count; ++s) { p.groups[s] = (p.n[s] + k.rows - 1) / k.rows; need += p.groups[s]; }
+    uint32_t need = 0, rows_total = 0, rpc = (uint32_t)k.rows;
+    if (k.split) for (uint32_t s = 0; s < p.count; ++s) { p.groups[s] = (p.n[s] + k.rows - 1) / k.rows; need += p.groups[s]; rows_total += p.n[s]; }
     else need = (p.n[0] + 16 * 8 - 1) / (16 * 8);           // whole blocks of many rows are launched alone
     // several blocks in one launch: two row groups per CTA share each activation fragment when that still leaves a CTA per SM
     // (four groups of activation rows would need twice the shared memory a CTA may declare)
     const bool pairs = k.split && p.count > 1 && NB <= 2 && need >= 2 * sms;
     if (pairs) need = (need + 1) / 2;
-    const uint32_t full = sms * (uint32_t)(k.split ? blocks_per_sm_split : blocks_per_sm);
+    // (the grouped kernels are 16 warps of more than 64 registers each: one CTA per SM)
+    const uint32_t full = (k.split && p.count > 1) ? sms : sms * (uint32_t)(k.split ? blocks_per_sm_split : blocks_per_sm);
+    if (k.split && p.count > 1 && need > full && g_gemv_balance) {
+        // The grid is one persistent CTA per resident slot, each walking its share of the row groups: 256 pairs of groups
+        // on 148 CTAs give 108 of them two and 40 one.  Slightly smaller groups (14 rows instead of 16) make the count a
+        // multiple of the grid, so that no CTA waits for the others' second round; not below half a tile plus one row.
+        const uint32_t per_cta = pairs ? 2 : 1, rounds = (need + full - 1) / full, target = rounds * full;
+        uint32_t r = (rows_total + per_cta * target - 1) / (per_cta * target);
+        r = std::min<uint32_t>((uint32_t)k.rows, std::max<uint32_t>(r, (uint32_t)k.rows / 2 + 1));
+        for (;; ++r) {                                    // per-block rounding may push the count past the target: one more row then
+            uint32_t groups = 0;
+            for (uint32_t s = 0; s < p.count; ++s) groups += (p.n[s] + r - 1) / r;
+            if (r >= (uint32_t)k.rows || (groups + per_cta - 1) / per_cta <= target) break;
+        }
+        rpc = r;
+        uint32_t groups = 0;
+        for (uint32_t s = 0; s < p.count; ++s) { p.groups[s] = (p.n[s] + rpc - 1) / rpc; groups += p.groups[s]; }
+        need = (groups + per_cta - 1) / per_cta;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(need < full ? need : full);
     cfg.blockDim = dim3(k.split ? k.nw * 32 : 256);
@@ -1130,13 +1154,13 @@ static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint3
     if (!k.split) cudaLaunchKernelEx(&cfg, gemv_mma_kernel<NB, U>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
     else if (p.count > 1) {                               // only few-row blocks are ever grouped: 16 warps, doubled load steps
         if constexpr (NB <= 2 && U == 8) {
-            if (pairs && k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 8, 2>, A, p, Mrows, total, K, acc);
-            else if (pairs) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 16, 2>, A, p, Mrows, total, K, acc);
-            else if (k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 8, 1>, A, p, Mrows, total, K, acc);
-            else cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc);
+            if (pairs && k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 8, 2>, A, p, Mrows, total, K, acc, rpc);
+            else if (pairs) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 16, 2>, A, p, Mrows, total, K, acc, rpc);
+            else if (k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 8, 1>, A, p, Mrows, total, K, acc, rpc);
+            else cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc, rpc);
         } else if constexpr (NB == 4 && U == 4) {
-            if (k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 8, 1>, A, p, Mrows, total, K, acc);
-            else cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc);
+            if (k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 8, 1>, A, p, Mrows, total, K, acc, rpc);
+            else cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc, rpc);
         }
     }
     else if (k.nw == 16 && k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 8>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
