@@ -910,7 +910,9 @@ static void launch_gemv(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, 
 // Same product for blocks with few rows: one CTA owns ROWS (16, or 8 with the upper half of the MMA tile left empty)
 // rows of W and its NW (8 or 16) warps split K (interleaved chunks of 32*U), so n/ROWS CTAs of NW warps fill the machine
 // where n/16 warps would not.  The partial tiles meet in shared memory and are summed in warp order: deterministic.
-template <int NB, int U, int NW, int ROWS>
+// RPC <= ROWS: rows a CTA owns (the tile's remaining rows re-read its last row and are not stored; a row's sum does not
+// depend on its place in the tile).  14 of 16 turns the 256 CTAs of a 4096-row block into 293, two for every SM.
+template <int NB, int U, int NW, int ROWS, int RPC = ROWS>
 __global__ void __launch_bounds__(NW * 32) gemv_mma_splitk_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                               uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     constexpr int UL = ROWS == 8 ? 2 * U : U;             // half a tile per load step: twice the steps in flight
@@ -918,9 +920,10 @@ __global__ void __launch_bounds__(NW * 32) gemv_mma_splitk_kernel(const bf16 *__
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, c = lane & 3;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     bool synced = false;
-    for (uint32_t row0 = blockIdx.x * ROWS; row0 < n; row0 += gridDim.x * ROWS) {
-        const bf16 *wlo = W + (size_t)min(row0 + g, n - 1) * K + c * 8;
-        const bf16 *whi = W + (size_t)min(row0 + g + 8, n - 1) * K + c * 8;
+    for (uint32_t row0 = blockIdx.x * RPC; row0 < n; row0 += gridDim.x * RPC) {
+        const uint32_t rlast = min(row0 + RPC, n) - 1;
+        const bf16 *wlo = W + (size_t)min(row0 + g, rlast) * K + c * 8;
+        const bf16 *whi = W + (size_t)min(row0 + g + 8, rlast) * K + c * 8;
         float acc[NB][4];
 #pragma unroll
         for (int b = 0; b < NB; ++b) { acc[b][0] = acc[b][1] = acc[b][2] = acc[b][3] = 0.f; }
@@ -957,7 +960,7 @@ __global__ void __launch_bounds__(NW * 32) gemv_mma_splitk_kernel(const bf16 *__
 #pragma unroll
             for (int w = 0; w < NW; ++w) sum += part[w][slot][ln];
             const uint32_t m = b * 8 + 2 * (ln & 3) + (i & 1), row = row0 + (ln >> 2) + 8 * (i >> 1);
-            if (m < Mrows && row < n && (ROWS == 16 || (i >> 1) == 0)) {
+            if (m < Mrows && row < n && (RPC == ROWS || row < row0 + RPC) && (ROWS == 16 || (i >> 1) == 0)) {
                 float *p = C + (size_t)m * ldc + col0 + row;
                 if (accumulate) atomicAdd(p, sum);               // one add per element by one thread, not waited for
                 else *p = sum;
@@ -1164,7 +1167,18 @@ static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint3
         }
     }
     else if (k.nw == 16 && k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 8>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
-    else if (k.nw == 16) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 16>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
+    else if (k.nw == 16) {
+        if constexpr (NB == 1 && U == 4) {
+            // 33.5 MB blocks at M <= 8, two CTAs per SM: 14 rows per CTA when that gives every SM two
+            const uint32_t c14 = (p.n[0] + 13) / 14;
+            if (g_gemv_balance && need > sms && c14 <= 2 * sms && c14 > need) {
+                cfg.gridDim = dim3(c14);
+                cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 16, 14>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
+                return;
+            }
+        }
+        cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 16>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
+    }
     else cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 8, 16>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
 }
 
