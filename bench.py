@@ -84,19 +84,6 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def parse_trace(blob):
-    """-> list of (step, site, layer, kind, flops, hbm, [(tensor, mode, touched)])"""
-    ops, off = [], 0
-    head = struct.Struct("<IQiIQQI")
-    while off < len(blob):
-        step, site, layer, kind, flops, hbm, n = head.unpack_from(blob, off)
-        off += head.size
-        acc = [struct.unpack_from("<IIQ", blob, off + 16 * k) for k in range(n)]
-        off += 16 * n
-        ops.append((step, site, layer, kind, flops, hbm, acc))
-    return ops
-
-
 def oracle_weights_from_pool(lay, pool_u8):
     """bf16 bit matrices per logical weight, re-joined from the pool's blocks (input data for the oracle)."""
     u16 = pool_u8.view(np.uint16)
@@ -172,10 +159,12 @@ def gemm_shapes_of_step(lay, M):
 GROUP_MAX = 8     # TGP_GEMM_GROUP_MAX
 
 
-def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
+def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30, min_seconds=1.5):
     """Times the weight-block products of one step back to back on one stream, every launch reading a different
     (cold) region of a buffer larger than L2, exactly as tgp_step launches them (same entry point, shapes, M).
-    Returns (avg seconds per launch, algorithmic bytes per launch, flops per launch, launches per rep, per-shape table)."""
+    The whole-step loop is replayed for at least min_seconds (and at least `reps` replays when min_seconds is 0: the small
+    form for ncu captures).  Returns (avg seconds per launch, algorithmic bytes per launch, flops per launch, launches
+    per rep, per-shape table with the name of the kernel the library launched for each shape)."""
     import torch
     from paper_2609_06172_b200 import binding as tb
     cfg = lay.cfg
@@ -198,6 +187,8 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
     stream = torch.cuda.Stream(device=device)
     off = 0
 
+    kernel_of = {}
+
     def run_all(st, only=None):
         nonlocal off
         for (n, K, res, m) in shapes:
@@ -212,6 +203,7 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
                                 m, list(n), K, [nmax] * len(n), res, st)
             else:
                 tb.k_gemm(A, wbuf.data_ptr() + off, Cbuf, m, n, K, nmax, 0, res, st)
+            kernel_of[(n, K, res, m)] = tb.k_gemm_last_kernel()
             off += nb
 
     def graph_of(only=None, passes=4):
@@ -227,15 +219,16 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
         run_all(stream)
     stream.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    def bounded(g, budget_s):
-        """One untimed-for-the-result replay measures a replay's length; then as many of the `reps` replays as fit in
-        budget_s seconds are timed (a deep model's step has thousands of launches: 20 replays would run for minutes)."""
+    def bounded(g, want_s):
+        """One untimed-for-the-result replay measures a replay's length; then as many replays as fill want_s seconds are
+        timed (want_s == 0: `reps` replays, but no more than fit in 4 s - a deep model's step has thousands of launches)."""
         with torch.cuda.stream(stream):
             e0.record(stream)
             g.replay()
             e1.record(stream)
             stream.synchronize()
-            n = max(1, min(reps, int(budget_s / max(1e-6, e0.elapsed_time(e1) * 1e-3))))
+            one = max(1e-6, e0.elapsed_time(e1) * 1e-3)
+            n = max(1, min(200000, int(np.ceil(want_s / one)))) if want_s > 0 else max(1, min(reps, int(4.0 / one)))
             e0.record(stream)
             for _ in range(n):
                 g.replay()
@@ -244,7 +237,7 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
         return n, e0.elapsed_time(e1) * 1e-3
 
     g, passes = graph_of()
-    n_rep, total_s = bounded(g, 4.0)
+    n_rep, total_s = bounded(g, min_seconds)
     kernel_loop.last = {"reps": n_rep, "passes": passes, "seconds": total_s}
     sec = total_s / (n_rep * passes * len(shapes))
     bytes_per = sum(2 * m * K + 2 * K * rows_of(n) + 4 * m * rows_of(n) * (2 if res else 1) for (n, K, res, m) in shapes) / len(shapes)
@@ -253,14 +246,14 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30):
     for sh in sorted(set(shapes), key=lambda q: (rows_of(q[0]),) + tuple(q[1:])):
         cnt = shapes.count(sh)
         g, passes = graph_of(only=sh)
-        n_sh, t_sh = bounded(g, 1.0)
+        n_sh, t_sh = bounded(g, min(0.3, min_seconds))
         t = t_sh / (n_sh * passes * cnt)
         n, K, res, m = sh
         nr = rows_of(n)
         b = 2 * m * K + 2 * K * nr + 4 * m * nr * (2 if res else 1)
         name = "+".join(str(x) for x in n) if isinstance(n, tuple) else str(n)
-        table[f"n={name} K={K} M={m} res={res}"] = {"launches_per_step": cnt, "us": round(t * 1e6, 2), "GBps": round(b / t / 1e9, 1),
-                                                      "TFLOPs": round(2 * m * K * nr / t / 1e12, 2)}
+        table[f"n={name} K={K} M={m} res={res}"] = {"kernel": kernel_of.get(sh, "?"), "launches_per_step": cnt, "us": round(t * 1e6, 2),
+                                                      "GBps": round(b / t / 1e9, 1), "TFLOPs": round(2 * m * K * nr / t / 1e12, 2)}
     return sec, bytes_per, flops_per, len(shapes), table
 
 
@@ -343,13 +336,28 @@ def oracle_sample(cfg, lay):
     return int(max(4, min(128, cfg.S, 5e11 / (2 * params * cfg.B)))), min(cfg.T, 4)
 
 
-def run_reference(args, cfg, lay):
+def run_reference(args, cfg, lay, full_T=None):
+    """The CPU oracle, as it stands, through the bench contract: every step is a bounded sample of the workload named in
+    `config` (full widths and depth, a prefix of the prompt and of the decode steps), on the host cores of rank 0."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     pool = np.empty(lay.pool_bytes, dtype=np.uint8)
-    si.fill_pool(lay, pool)
+    filled = False
+    if lay.pool_bytes > (1 << 30):
+        # seeded inputs of a multi-gigabyte pool: the same generator evaluated on a GPU when one is there (bit-identical
+        # to the numpy generator, tested); the oracle's arithmetic below runs on the host cores either way
+        try:
+            import torch
+            if torch.cuda.is_available():
+                si.fill_pool_torch(lay, torch.from_numpy(pool), device="cuda:0")
+                filled = True
+        except Exception:
+            filled = False
+    if not filled:
+        si.fill_pool(lay, pool)
     om = make_oracle(lay, oracle_weights_from_pool(lay, pool))
+    del pool
     sS, sT = oracle_sample(cfg, lay)
     cores = len(os.sched_getaffinity(0))
     for _ in range(args.warmup):
@@ -363,14 +371,94 @@ def run_reference(args, cfg, lay):
     print(json.dumps({"impl": "reference", "metric": "tokens_per_s", "value": val, "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps,
                       "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
                       "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                      "config": {"workload": workload_name(cfg, lay), "sample": sample},
+                      "config": config_dict(cfg, lay, full_T, int(os.environ.get("WORLD_SIZE", "1"))), "sample": sample,
                       "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
                       "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
-def workload_name(cfg, lay):
-    return (f"{cfg.name}: L={cfg.L} d={cfg.d} Hq/Hkv={cfg.Hq}/{cfg.Hkv} F={cfg.F} V={cfg.V} B={cfg.B} prompt={cfg.S} decode={cfg.T} "
+# decode steps per timed pass where the configuration's own count would make a pass run for tens of seconds (per-step
+# rates do not depend on the count; the workload string names what ran): headline pass, one-pass summary
+DECODE_PER_PASS = {3: 32, 4: 4, 5: 8}
+DECODE_PER_SUMMARY = {3: 16, 4: 2, 5: 4}
+ALIAS_LAYERS = {4: 40}          # the 70B shape's 152 GB pool cannot be page-locked on a 206 GB host: 40 physical layers, each mapped twice
+HEADLINE_CONFIG = 3
+
+
+def workload_name(cfg, lay, full_T=None):
+    dec = f"{cfg.T}" if full_T in (None, cfg.T) else f"{cfg.T} of {full_T}"
+    return (f"{cfg.name}: L={cfg.L} d={cfg.d} Hq/Hkv={cfg.Hq}/{cfg.Hkv} F={cfg.F} V={cfg.V} B={cfg.B} prompt={cfg.S} decode={dec} "
             f"pool={lay.pool_bytes} budget={lay.budget}")
+
+
+def config_dict(cfg, lay, full_T, world=1, graph=False):
+    return {"workload": workload_name(cfg, lay, full_T), "l2": f"inputs larger than L2: every decode step streams the {lay.pool_bytes / 1e9:.1f} GB pool",
+            "step": "prefill + %d decode steps from a cold arena" % cfg.T + (", replayed as one CUDA graph" if graph else ""),
+            "tokens_per_step": cfg.B * (cfg.S + cfg.T), "parallelism": "replicas" if world > 1 else "single"}
+
+
+def lower_bound_bytes(ops, lay):
+    """Per step: bytes that must cross the link whatever the schedule = accessed pool bytes - budget (all of them for
+    the cold first step); a tensor counts once per step, at its largest access of the step (whole if any access
+    touches half of it or more)."""
+    step_of = {}
+    for o in ops:
+        d = step_of.setdefault(o[0], {})
+        for (t, mode, touched) in o[6]:
+            b = lay.tensors[t].size if touched * 2 >= lay.tensors[t].size else touched
+            d[t] = max(d.get(t, 0), b)
+    return {k: max(0, sum(d.values()) - (lay.budget if k else 0)) for k, d in step_of.items()}
+
+
+def step_roofline(ops, totals, lay, t_meas, step_ms):
+    """Slowest of compute, HBM and link per step, summed over the steps of a pass: (i) with the plan's link bytes,
+    (ii) with the lower bound on them."""
+    nsteps = len(totals)
+    Fs, Hs = [0] * nsteps, [0] * nsteps
+    for o in ops:
+        Fs[o[0]] += o[4]
+        Hs[o[0]] += o[5]
+    lb = lower_bound_bytes(ops, lay)
+    t_roof = t_lb = 0.0
+    bound_of = []
+    for k in range(nsteps):
+        cands = {"tensor": Fs[k] / MACHINE["peak_flops"], "hbm": (Hs[k] + int(totals[k][0])) / MACHINE["hbm_Bps"],
+                 "link": (int(totals[k][0]) + int(totals[k][2])) / MACHINE["h2d_Bps"], "link_d2h": int(totals[k][1]) / MACHINE["d2h_Bps"]}
+        bound_of.append(max(cands, key=cands.get))
+        t_roof += max(cands.values())
+        t_lb += max(cands["tensor"], cands["hbm"], lb.get(k, 0) / MACHINE["h2d_Bps"])
+    L_plan = int(totals[:, 0].sum() + totals[:, 2].sum())
+    return {"bound": {"prefill": bound_of[0], "decode": max(set(bound_of[1:]), key=bound_of[1:].count) if nsteps > 1 else None},
+            "t_roof_s_plan_bytes": t_roof, "t_roof_s_lower_bound": t_lb, "t_measured_s": t_meas,
+            "frac_plan_bytes": t_roof / t_meas, "frac_lower_bound": t_lb / t_meas,
+            "prefill": {"t_roof_s": max(Fs[0] / MACHINE["peak_flops"], (int(totals[0][0]) + int(totals[0][2])) / MACHINE["h2d_Bps"]),
+                        "t_measured_s": step_ms[0] * 1e-3 if step_ms else None},
+            "link_gbs_achieved": L_plan / t_meas / 1e9, "link_gbs_peak": MACHINE["h2d_Bps"] / 1e9,
+            "h2d_bytes": int(totals[:, 0].sum()), "d2h_bytes": int(totals[:, 1].sum()), "zero_copy_bytes": int(totals[:, 2].sum()),
+            "flops": sum(Fs), "hbm_bytes": sum(Hs) + int(totals[:, 0].sum())}
+
+
+def other_config_summaries(args, budget_s):
+    """One-pass summaries of the other configurations, each in a process of its own (its host pool is released when it
+    exits) under a time limit; what does not fit the remaining budget is reported as skipped, never silently dropped."""
+    out = {}
+    t_end = time.monotonic() + budget_s
+    for c in (1, 2, 5, 4):
+        if c == args.config:
+            continue
+        left = t_end - time.monotonic()
+        if left < 60:
+            out[str(c)] = {"skipped": "time budget of this run spent"}
+            continue
+        cmd = [sys.executable, os.path.abspath(__file__), "--config", str(c), "--summary"]
+        t0 = time.monotonic()
+        try:
+            r = subprocess.run(cmd, capture_output=True, text=True, timeout=min(left, 600))
+            line = [l for l in r.stdout.splitlines() if l.startswith("{")]
+            out[str(c)] = json.loads(line[-1]) if r.returncode == 0 and line else {"failed": f"rc {r.returncode}", "stderr_tail": r.stderr[-400:]}
+        except subprocess.TimeoutExpired:
+            out[str(c)] = {"failed": "time limit"}
+        out[str(c)]["wall_s"] = round(time.monotonic() - t0, 1)
+    return out
 
 
 def main():
@@ -379,8 +467,10 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="tgp")
-    ap.add_argument("--config", type=int, default=2)
-    ap.add_argument("--decode", type=int, default=None, help="decode steps per pass (default: the configuration's)")
+    ap.add_argument("--config", type=int, default=HEADLINE_CONFIG)
+    ap.add_argument("--decode", type=int, default=None, help="decode steps per pass (default: the configuration's, bounded for configs 3-5)")
+    ap.add_argument("--summary", action="store_true", help="one warm-up pass and one timed pass, compact output (what the headline run collects for the other configurations)")
+    ap.add_argument("--no-configs", action="store_true", help="skip the one-pass summaries of the other configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-uvm", action="store_true", help="skip the demand-paged managed-memory baseline")
     ap.add_argument("--kernel-loop", choices=["decode", "prefill", "attention"], default=None,
@@ -396,8 +486,16 @@ def main():
     ap.add_argument("--budget-frac", type=float, default=None, help="device budget as a fraction of the pool (oversubscription sweep)")
     args = ap.parse_args()
     cfg = si.CONFIGS[args.config]
+    full_T = cfg.T
     if args.decode is not None:
         cfg = replace(cfg, T=args.decode)
+    elif args.config in DECODE_PER_PASS and not args.kernel_loop:
+        cfg = replace(cfg, T=min(cfg.T, (DECODE_PER_SUMMARY if args.summary else DECODE_PER_PASS)[args.config]))
+    if args.alias_layers is None and args.config in ALIAS_LAYERS and args.layers is None and args.impl != "reference" and not args.kernel_loop:
+        args.alias_layers = ALIAS_LAYERS[args.config]
+    if args.summary:
+        args.steps, args.warmup, args.no_configs, args.no_cpu_baseline = 1, 1, True, True
+        args.no_uvm = args.no_uvm or args.config != 2
     budget = None
     if args.layers is not None and args.layers != cfg.L:
         full = si.build_layout(cfg)
@@ -409,7 +507,7 @@ def main():
     if args.budget_frac is not None:
         lay = si.build_layout(cfg, budget=int(lay.pool_bytes * args.budget_frac) // 512 * 512, cap=cap)
     if args.impl == "reference":
-        return run_reference(args, cfg, lay)
+        return run_reference(args, cfg, lay, full_T)
 
     if args.kernel_loop:
         import torch
@@ -423,11 +521,12 @@ def main():
                               "TK": cfg.TK, "causal_flops": flops, "L2_flushed_between_launches": True, "kernels": table}))
             return
         M = cfg.B * (cfg.S if args.kernel_loop == "prefill" else 1)
-        sec, b, f, nl, table = kernel_loop(lay, M, args.reps, torch.device("cuda:0"))
+        sec, b, f, nl, table = kernel_loop(lay, M, args.reps, torch.device("cuda:0"), min_seconds=0.0)
         print(json.dumps({"kernel_loop": args.kernel_loop, "M": M, "avg_us": sec * 1e6, "GBps": b / sec / 1e9, "TFLOPs": f / sec / 1e12,
-                          "launches_per_step": nl, "shapes": table}))
+                          "launches_per_step": nl, "timed": kernel_loop.last, "shapes": table}))
         return
 
+    t_start = time.monotonic()
     import torch
     from paper_2609_06172_b200 import binding as tb
     from paper_2609_06172_b200.runner import Runner, pinned_pool
@@ -469,7 +568,7 @@ def main():
         blobs = s.plan(bits=args.bits)
         r = Runner(s, cfg.B * cfg.S, device=str(dev))
     totals = np.frombuffer(blobs["totals"], dtype="<u8").reshape(-1, 4)
-    ops = parse_trace(s.ctx.trace_export())
+    ops = s.ctx.trace_ops()
     # --unseen-prompts (MoE): the timed passes run prompts the profile pass never saw, so the plan's expert sets are a
     # prediction; an expert the router picks outside its step's set is fetched synchronously and counted
     run_cfg = replace(cfg, seed=cfg.seed ^ 0x5EED) if args.unseen_prompts else cfg
@@ -512,6 +611,7 @@ def main():
         ev0.record(r.compute)
         for _ in range(n):
             one_pass(e2e)
+        r.sync()                                                 # every stream of the device, the library's write-back stream included
         ev1.record(r.compute)
         r.sync()
         barrier()
@@ -535,11 +635,13 @@ def main():
     if use_graph:
         r.sync()
         r.reset()
-    one_pass(True)
-    ms_e2e = timed(args.steps, True)
+    ms_e2e = None
+    if not args.summary:
+        one_pass(True)
+        ms_e2e = timed(args.steps, True)
     tokens_per_pass = cfg.B * (cfg.S + T)
     value = world * tokens_per_pass * args.steps / (ms * 1e-3)
-    e2e_value = world * tokens_per_pass * args.steps / (ms_e2e * 1e-3)
+    e2e_value = world * tokens_per_pass * args.steps / (ms_e2e * 1e-3) if ms_e2e else None
 
     # ---- per-phase timing, launches and the live per-kernel roofline: one extra pass with op timestamps -----------
     r.reset()
@@ -577,13 +679,30 @@ def main():
         tot = np.asarray(ran[:n], dtype=np.float64).sum(axis=0)                          # [L, E]
         for l in range(cfg.L):
             by_rank += tot[l][order[l]]
-        zipf = np.array([r ** (-cfg.zipf_s) for r in range(1, cfg.E + 1)])
+        zipf = np.array([r_ ** (-cfg.zipf_s) for r_ in range(1, cfg.E + 1)])
         moe_prediction["routed_share_by_bias_rank"] = [round(float(x), 4) for x in by_rank / max(1.0, by_rank.sum())]
         moe_prediction["zipf_first_choice"] = [round(float(x), 4) for x in zipf / zipf.sum()]
 
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
+        return
+    t_meas = ms * 1e-3 / args.steps
+    step_roof = step_roofline(ops, totals, lay, t_meas, step_ms)
+    host_pool = ({"aliased_physical_layers": args.alias_layers, "physical_bytes": aliased.phys_bytes, "virtual_bytes": lay.pool_bytes,
+                  "note": "layers l and l + %d share host pages: link bytes, schedule and arithmetic are the full model's; throughput only" % args.alias_layers}
+                 if aliased else "pinned, one physical page per byte")
+    prefill_tok_s = cfg.B * cfg.S / (step_ms[0] * 1e-3)
+    decode_tok_s = cfg.B * T / (sum(step_ms[1:]) * 1e-3) if T else None
+    if args.summary:
+        out = {"config": args.config, "workload": workload_name(cfg, lay, full_T), "passes_timed": args.steps, "tokens_per_s": value,
+               "prefill_tok_s": prefill_tok_s, "decode_tok_s": decode_tok_s, "ms_per_pass": ms / args.steps,
+               "step_roofline": {k: step_roof[k] for k in ("bound", "frac_plan_bytes", "frac_lower_bound", "link_gbs_achieved", "link_gbs_peak", "t_measured_s")},
+               "host_pool": host_pool, "gpu_launches": launches, "clocks": clocks, "trace_mismatches": mismatches, "graph": bool(use_graph),
+               "kernels_ms": {f"{k[0]}:{k[1]}": round(v, 3) for k, v in sorted(kind_ms.items())}}
+        if not args.no_uvm:
+            out["uvm"] = uvm_runs(args, cfg, lay, dev, pool, r, s, step_ms, T, only_demand=True)
+        print(json.dumps(out))
         return
     peaks = measured_peaks()
     # dominant kernel by device time in the pass; its launch duration is measured in a dedicated region: the same
@@ -605,9 +724,15 @@ def main():
         else:
             ach = bpl / sec / 1e9
             roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"]}
-        roof.update({"kernel": f"weight-block product ({dom[0]}, M={Mk}): " + ("gemv_kernel" if Mk <= 16 else "gemm_tc_kernel"),
+        # the kernels that ran, as the library reports them per launch (its choice depends on M, n, K), heaviest first
+        by_kernel = {}
+        for v in table.values():
+            by_kernel[v["kernel"]] = by_kernel.get(v["kernel"], 0.0) + v["us"] * v["launches_per_step"]
+        names = sorted(by_kernel, key=by_kernel.get, reverse=True)
+        roof.update({"kernel": f"weight-block product ({dom[0]}, M={Mk}): " + " + ".join(names),
+                     "kernel_time_share": {k: round(by_kernel[k] / sum(by_kernel.values()), 3) for k in names},
                      "launches": nl * (T if dom[0] == "decode" else 1), "avg_us": sec * 1e6, "algorithmic_per_launch": fpl if roof["bound"] == "tensor" else bpl,
-                     "timing": f"CUDA-graph replay of the {nl} launches of one step, {kernel_loop.last['reps']} x {kernel_loop.last['passes']} passes back to back ({kernel_loop.last['seconds']:.1f} s), random operands, cold inputs cycling through 1 GiB, CUDA events on the launch stream",
+                     "timing": f"CUDA-graph replay of the {nl} launches of one step, {kernel_loop.last['reps']} x {kernel_loop.last['passes']} passes back to back ({kernel_loop.last['seconds']:.2f} s), random operands, cold inputs cycling through 1 GiB, CUDA events on the launch stream",
                      "in_step_avg_us": kind_ms[dom] / (nl * (T if dom[0] == "decode" else 1)) * 1e3, "shapes": table})
     else:
         ach = kind_bytes[dom] / (kind_ms[dom] * 1e-3) / 1e9
@@ -618,42 +743,10 @@ def main():
     prof = os.path.join(ROOT, "profiles", "traffic.txt")          # DRAM bytes per launch from the committed ncu summaries
     if os.path.exists(prof):
         for line in open(prof):
-            f = line.split()
+            f = line.split(None, 2)
             if f and f[0] == f"{dom[1]}_{dom[0]}_cfg{args.config}":
                 roof["traffic"] = float(f[1])
-    # step roofline: slowest of compute, HBM and link for the whole pass, (i) with the plan's bytes, (ii) with the lower bound
-    F = sum(o[4] for o in ops)
-    H = sum(o[5] for o in ops) + int(totals[:, 0].sum())
-    L_plan, L_d2h = int(totals[:, 0].sum() + totals[:, 2].sum()), int(totals[:, 1].sum())
-    step_of = {}
-    for o in ops:
-        for (t, mode, touched) in o[6]:
-            step_of.setdefault(o[0], {})[t] = lay.tensors[t].size if touched * 2 >= lay.tensors[t].size else touched
-    # per step the slowest of compute, HBM and link; the pass roofline is the sum over its steps (a pass mixes a
-    # possibly compute-bound prefill with link-bound decode steps)
-    nsteps = len(totals)
-    Fs, Hs = [0] * nsteps, [0] * nsteps
-    for o in ops:
-        Fs[o[0]] += o[4]
-        Hs[o[0]] += o[5]
-    lb = {k: max(0, sum(d.values()) - (lay.budget if k else 0)) for k, d in step_of.items()}
-    t_roof = t_lb = 0.0
-    bound_of = []
-    for k in range(nsteps):
-        cands = {"tensor": Fs[k] / MACHINE["peak_flops"], "hbm": (Hs[k] + int(totals[k][0])) / MACHINE["hbm_Bps"],
-                 "link": (int(totals[k][0]) + int(totals[k][2])) / MACHINE["h2d_Bps"], "link_d2h": int(totals[k][1]) / MACHINE["d2h_Bps"]}
-        bound_of.append(max(cands, key=cands.get))
-        t_roof += max(cands.values())
-        t_lb += max(cands["tensor"], cands["hbm"], lb.get(k, 0) / MACHINE["h2d_Bps"])
-    t_meas = ms * 1e-3 / args.steps
-    step_roof = {"bound": {"prefill": bound_of[0], "decode": max(set(bound_of[1:]), key=bound_of[1:].count) if nsteps > 1 else None},
-                 "t_roof_s_plan_bytes": t_roof, "t_roof_s_lower_bound": t_lb, "t_measured_s": t_meas,
-                 "frac_plan_bytes": t_roof / t_meas, "frac_lower_bound": t_lb / t_meas,
-                 "prefill": {"t_roof_s": max(Fs[0] / MACHINE["peak_flops"], (int(totals[0][0]) + int(totals[0][2])) / MACHINE["h2d_Bps"]),
-                             "t_measured_s": step_ms[0] * 1e-3},
-                 "link_gbs_achieved": L_plan / t_meas / 1e9, "link_gbs_peak": MACHINE["h2d_Bps"] / 1e9,
-                 "h2d_bytes": int(totals[:, 0].sum()), "d2h_bytes": L_d2h, "zero_copy_bytes": int(totals[:, 2].sum()),
-                 "flops": F, "hbm_bytes": H}
+                roof["traffic_source"] = "profiles/traffic.txt: " + (f[2].strip().strip('"') if len(f) > 2 else "ncu capture")
     # the paper's motivation experiment (Section III-B) on this workload, analytically: a prefetcher that sees only
     # allocator segments (20 MiB, the large-block size of PyTorch's caching allocator) and prefetches every segment
     # an op's tensors overlap moves this many useless bytes per useful byte
@@ -667,53 +760,81 @@ def main():
             useful += touched
         useless += len(segs) * SEG
     object_level = {"segment_bytes": SEG, "useless_over_useful": (useless - useful) / max(1, useful), "kind": "analytic, from the trace"}
+    L_d2h = int(totals[:, 1].sum())
     out = {"metric": "tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-           "data": "synthetic", "config": {"workload": workload_name(cfg, lay), "l2": f"inputs larger than L2: every decode step streams the {lay.pool_bytes / 1e9:.1f} GB pool",
-                                           "step": "prefill + all decode steps from a cold arena" + (", replayed as one CUDA graph" if use_graph else ""), "tokens_per_step": tokens_per_pass,
-                                           "parallelism": "replicas" if world > 1 else "single"},
-           "prefill_tok_s": cfg.B * cfg.S / (step_ms[0] * 1e-3), "decode_tok_s": cfg.B * T / (sum(step_ms[1:]) * 1e-3) if T else None,
+           "data": "synthetic", "config": config_dict(cfg, lay, full_T, world, use_graph),
+           "prefill_tok_s": prefill_tok_s, "decode_tok_s": decode_tok_s,
            "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": int(totals[:, 0].sum()) + cfg.B * (cfg.S + T) * 4,
                    "d2h_bytes_per_step": L_d2h + cfg.B * (T + 1) * 4 + cfg.B * cfg.V * 4},
-           "object_level_prefetch": object_level, "policy_bits": args.bits, "trace_mismatches": mismatches, "moe_profile_pass_s": profile_s, "unseen_prompts": bool(args.unseen_prompts), "host_pool": ({"aliased_physical_layers": args.alias_layers, "physical_bytes": aliased.phys_bytes, "virtual_bytes": lay.pool_bytes} if aliased else "pinned, one physical page per byte"), "moe_prediction": moe_prediction,
+           "object_level_prefetch": object_level, "policy_bits": args.bits, "trace_mismatches": mismatches, "moe_profile_pass_s": profile_s, "unseen_prompts": bool(args.unseen_prompts),
+           "host_pool": host_pool, "moe_prediction": moe_prediction,
            "gpu_launches": launches * args.steps, "clocks": clocks, "roofline": roof, "step_roofline": step_roof,
            "kernels": {f"{k[0]}:{k[1]}": {"ms": round(v, 3), "ops": kind_n[k], "GBps": round(kind_bytes[k] / (v * 1e-3) / 1e9, 1),
                                            "TFLOPs": round(kind_flops[k] / (v * 1e-3) / 1e12, 2)} for k, v in sorted(kind_ms.items())}}
+    pool_np = pool.numpy()
     if not args.no_uvm and world == 1:                 # the baselines are single-GPU measurements: reported at N = 1 only
-        try:
-            from paper_2609_06172_b200 import uvm_baseline
-            del r
-            s.close()
-            torch.cuda.empty_cache()
-            uvm = uvm_baseline.run(cfg, lay, MACHINE, dev, lambda l, arr: arr.__setitem__(slice(None), pool.numpy()),
-                                   variants=(tb.VAR_MANAGED_DEMAND, tb.VAR_MANAGED_HINTS, tb.VAR_MANAGED_OBJECT),
-                                   decode_cap=16 if lay.pool_bytes < (4 << 30) else 4, object_bytes=SEG)
-            dec = cfg.B * T / (sum(step_ms[1:]) * 1e-3) if T else None
-            for v in uvm.values():
-                if dec and v.get("decode_tok_s"):
-                    v["explicit_ring_speedup_decode"] = dec / v["decode_tok_s"]
-            out["uvm"] = uvm
-            mo = uvm.get("managed_object")
-            if mo and mo.get("asked_bytes_per_decode_step"):
-                # the same experiment run for real: the managed pool with the segment-granular prefetcher one op ahead
-                touched = sum(a[2] for o in ops if o[0] >= 1 for a in o[6]) / max(1, T)
-                object_level["measured"] = {"decode_tok_s": mo["decode_tok_s"], "asked_bytes_per_decode_step": mo["asked_bytes_per_decode_step"],
-                                            "touched_bytes_per_decode_step": touched,
-                                            "asked_over_touched": mo["asked_bytes_per_decode_step"] / max(1.0, touched),
-                                            "tensor_level_hints_speedup": uvm["managed_hints"]["decode_tok_s"] / mo["decode_tok_s"],
-                                            "explicit_ring_speedup": mo.get("explicit_ring_speedup_decode")}
-        except Exception as ex:  # the baseline is reported, never fatal
-            out["uvm"] = f"not run: {type(ex).__name__}: {ex}"
+        uvm = uvm_runs(args, cfg, lay, dev, pool, r, s, step_ms, T, only_demand=False)
+        out["uvm"] = uvm
+        mo = uvm.get("managed_object") if isinstance(uvm, dict) else None
+        if mo and mo.get("asked_bytes_per_decode_step"):
+            # the same experiment run for real: the managed pool with the segment-granular prefetcher one op ahead
+            touched = sum(a[2] for o in ops if o[0] >= 1 for a in o[6]) / max(1, T)
+            object_level["measured"] = {"decode_tok_s": mo["decode_tok_s"], "asked_bytes_per_decode_step": mo["asked_bytes_per_decode_step"],
+                                        "touched_bytes_per_decode_step": touched,
+                                        "asked_over_touched": mo["asked_bytes_per_decode_step"] / max(1.0, touched),
+                                        "tensor_level_hints_speedup": uvm["managed_hints"]["decode_tok_s"] / mo["decode_tok_s"],
+                                        "explicit_ring_speedup": mo.get("explicit_ring_speedup_decode")}
+    else:
+        del r
+        s.close()
+        torch.cuda.empty_cache()
     if not args.no_cpu_baseline and world == 1:
-        om = make_oracle(lay, oracle_weights_from_pool(lay, pool.numpy()))
+        om = make_oracle(lay, oracle_weights_from_pool(lay, pool_np))
         sS, sT = oracle_sample(cfg, lay)
         time_oracle(lay, om, min(16, sS), 1)
         val, dt = time_oracle(lay, om, sS, sT)
+        del om
         out["cpu_baseline"] = {"value": val, "unit": "tokens/s", "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
                                "sample": f"prefill of the first {sS} prompt tokens + {sT} decode steps, float32 accumulate ({dt:.1f} s)"}
+    if not args.no_configs and world == 1:
+        # the other configurations, one pass each in a process of its own; this process gives its host pool and device memory back first
+        del pool_np, pool
+        if aliased:
+            aliased.close()
+        import gc
+        gc.collect()
+        torch.cuda.empty_cache()
+        try:
+            torch._C._host_emptyCache()
+        except Exception:
+            pass
+        out["configs"] = other_config_summaries(args, max(120.0, 1500.0 - (time.monotonic() - t_start)))
     print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def uvm_runs(args, cfg, lay, dev, pool, r, s, step_ms, T, only_demand):
+    """The managed-memory runs of the same kernels under a ballast cap; reported, never fatal.  Frees the explicit
+    engine's runner and session first (the ballast is sized from the free device memory)."""
+    import torch
+    from paper_2609_06172_b200 import binding as tb
+    try:
+        from paper_2609_06172_b200 import uvm_baseline
+        s.close()
+        r.arena = r.workspace = None
+        torch.cuda.empty_cache()
+        variants = (tb.VAR_MANAGED_DEMAND,) if only_demand else (tb.VAR_MANAGED_DEMAND, tb.VAR_MANAGED_HINTS, tb.VAR_MANAGED_OBJECT)
+        uvm = uvm_baseline.run(cfg, lay, MACHINE, dev, lambda l, arr: arr.__setitem__(slice(None), pool.numpy()), variants=variants,
+                               decode_cap=16 if lay.pool_bytes < (4 << 30) else 4, object_bytes=20 << 20)
+        dec = cfg.B * T / (sum(step_ms[1:]) * 1e-3) if T else None
+        for v in uvm.values():
+            if dec and v.get("decode_tok_s"):
+                v["explicit_ring_speedup_decode"] = dec / v["decode_tok_s"]
+        return uvm
+    except Exception as ex:
+        return f"not run: {type(ex).__name__}: {ex}"
 
 
 if __name__ == "__main__":

@@ -5,10 +5,10 @@
  * a framework allocator carves one big pool into tensors that are invisible below it
  * (Section II-B), so the caller REGISTERS the pool and its sub-ranges (Section IV-B,
  * stable two-level tensor identity); one pass RECORDS which tensors each op touches
- * (Section IV-C, kernel-tensor access tracing); device capacity is CONSTRAINED to a
+ * (Section IV-D, kernel-tensor access tracing); device capacity is CONSTRAINED to a
  * budget (Section V-A); a roofline policy picks the transfers that matter (Section III-C,
- * IV-C "UVM Analyzer") and an engine stages exactly those tensors ahead of use
- * (Section IV-D "Prefetch Engine") while the model step RUNS.
+ * IV-D "UVM Analyzer") and an engine stages exactly those tensors ahead of use
+ * (Section IV-E "Prefetch Engine") while the model step RUNS.
  *
  * Conventions
  *  - Every function returns TGP_OK (0) or a negative TGP_E_* code; nothing throws, aborts
@@ -143,7 +143,7 @@ int  tgp_tensor_lookup(const tgp_ctx *ctx, const void *host_addr, uint32_t *tens
 /* Stable identity of a tensor: its site hash and per-site counter. */
 int  tgp_tensor_identity(const tgp_ctx *ctx, uint32_t tensor_id, uint64_t *site_hash, uint64_t *counter);
 
-/* ---- trace (Section IV-C): ordered ops, each with the tensors it touches --------------------- */
+/* ---- trace (Section IV-D): ordered ops, each with the tensors it touches --------------------- */
 int  tgp_trace_begin(tgp_ctx *ctx);                         /* discards any earlier trace and plan        */
 int  tgp_trace_step(tgp_ctx *ctx, uint32_t step_kind);      /* opens the next step                        */
 int  tgp_trace_op(tgp_ctx *ctx, uint64_t op_site, int32_t layer, uint32_t op_kind, uint64_t flops,
@@ -156,7 +156,7 @@ int  tgp_model_trace(tgp_ctx *ctx, uint32_t S, uint32_t T, const uint32_t *exper
  * u32 n_acc, then n_acc x (u32 tensor, u32 mode, u64 touched). */
 int  tgp_trace_export(const tgp_ctx *ctx, void *buf, uint64_t *bytes);
 
-/* ---- policy (Section III-C, IV-C, IV-D) ------------------------------------------------------ */
+/* ---- policy (Section III-C, IV-D, IV-E) ------------------------------------------------------ */
 int  tgp_set_budget(tgp_ctx *ctx, uint64_t bytes);          /* device bytes for resident pool tensors     */
 int  tgp_set_variant(tgp_ctx *ctx, uint32_t variant, uint32_t policy_bits);
 /* Segment size of TGP_VAR_MANAGED_OBJECT: the prefetcher of the paper's motivation (Section III-B) sees the
@@ -165,7 +165,7 @@ int  tgp_set_variant(tgp_ctx *ctx, uint32_t variant, uint32_t policy_bits);
  * allocator; at least 64 KiB).  tgp_step_stats.h2d_bytes then counts the bytes it asked for, whether they were
  * already resident or not; nothing is advised and nothing is evicted explicitly. */
 int  tgp_set_object_bytes(tgp_ctx *ctx, uint64_t bytes);
-/* Runtime monitor (Section IV-D): measured kernel times, one per op of the finished trace, in integer nanoseconds
+/* Runtime monitor (Section IV-E): measured kernel times, one per op of the finished trace, in integer nanoseconds
  * (0 = not measured: that op keeps its analytic class).  With a time t the link test becomes mig / Bl > t, i.e. an
  * op is link-bound iff moving its pool bytes takes longer than the kernel ran; the next tgp_plan() uses it.
  * n_ops == 0 clears the log; a new trace clears it too.  Integers make the re-plan reproducible: the same log fed
@@ -190,14 +190,15 @@ int  tgp_model_bind(tgp_ctx *ctx, const tgp_model_cfg *cfg, const tgp_role_entry
 int  tgp_run_reset(tgp_ctx *ctx);
 /* Runs the next step of the plan: enqueues its copies on copy_stream and its kernels on compute_stream and
  * returns without waiting unless stats != NULL.  tokens_host [B, q_len] int32, or NULL in a decode step to
- * feed the previous step's argmax, which stays on the device.  logits_dev [B, V] fp32 of the last position;
+ * feed the previous step's argmax, which stays on the device.  A host token outside [0, V) is refused with TGP_E_INVAL
+ * before anything is enqueued.  logits_dev [B, V] fp32 of the last position;
  * argmax_dev [B] int32 or NULL.  With stats the step is waited for, and TGP_E_CUDA is returned if a tensor-core kernel
  * of this process has recorded a bounded wait that ran out (tgp_k_gemm_status / tgp_k_attn_status). */
 int  tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_host, uint32_t B, uint32_t q_len,
               float *logits_dev, int32_t *argmax_dev, void *compute_stream, void *copy_stream,
               tgp_step_stats *stats);
 
-/* MoE profile (Section IV-C: one profiling pass recovers which tensors the kernels really touch): the tokens
+/* MoE profile (Section IV-D: one profiling pass recovers which tensors the kernels really touch): the tokens
  * routed to each expert, per step and layer, in the run since the last tgp_run_reset(): uint32 [steps, L, E].
  * Two-call form: out == NULL returns the element count in *n.  Feed it to tgp_model_trace() to trace exactly the
  * experts in use.  At run time an expert the router picks but the trace does not list is fetched synchronously
@@ -227,7 +228,7 @@ int  tgp_managed_evict(void *ptr, uint64_t bytes);
 int  tgp_set_tap(tgp_ctx *ctx, void *tap_dev, uint64_t bytes);
 int  tgp_tap_index(tgp_ctx *ctx, uint64_t *out, uint64_t *n_words);
 
-/* Per-op timestamps (Section IV-D "Runtime Monitor": lightweight timestamping).  While enabled, tgp_step()
+/* Per-op timestamps (Section IV-E "Runtime Monitor": lightweight timestamping).  While enabled, tgp_step()
  * brackets every op with CUDA events on the compute stream (after the op's copies have been waited for, so
  * the figure is kernel time, not stall time).  tgp_op_times() waits for the last timed step and returns one
  * duration in ms per op of that step, ops [*first_op, *first_op + *n_ops) of the trace; ms == NULL asks
@@ -248,8 +249,16 @@ int  tgp_run_capture_end(tgp_ctx *ctx);
 int  tgp_run_graph_launch(tgp_ctx *ctx, void *stream);
 
 /* ---- single kernels (device pointers; used by the model step, exported for parity tests and timing) ---- */
-/* x[m, :] = fp32(table[tok[m], :]);  table bf16 [V, d] (device or mapped host), tok int32 [M]. */
-int  tgp_k_embed(const void *table, const int32_t *tok_dev, float *x_dev, uint32_t M, uint32_t d, void *stream);
+/* x[m, :] = fp32(table[tok[m], :]);  table bf16 [V, d] (device or mapped host), tok int32 [M].  A token id outside
+ * [0, V) never indexes the table: its row of x is written as zeros and the first such (row, id) is kept in an error
+ * word that tgp_k_embed_status() reads and that tgp_step() reports (TGP_E_CUDA) when called with statistics. */
+int  tgp_k_embed(const void *table, const int32_t *tok_dev, float *x_dev, uint32_t M, uint32_t d, uint32_t V, void *stream);
+/* *bad = 1 if an embedding gather of this process met a token id outside its vocabulary since the last
+ * tgp_k_status_clear(), with the row and the id of the first one (row, token may be NULL).  Synchronous. */
+int  tgp_k_embed_status(int *bad, uint32_t *row, int32_t *token);
+/* Clears the three device-side error words (tgp_k_gemm_status, tgp_k_attn_status, tgp_k_embed_status) of the
+ * current device after waiting for it to go idle. */
+int  tgp_k_status_clear(void);
 /* h = bf16(x * rsqrt(mean(x^2) + eps) * g);  x fp32 [M, d] with row stride ldx elements, g bf16 [d], h bf16 [M, d]. */
 int  tgp_k_rmsnorm(const float *x_dev, uint32_t ldx, const void *g_dev, void *h_dev, uint32_t M, uint32_t d,
                    float eps, void *stream);
@@ -277,6 +286,9 @@ int  tgp_k_gemm_group(const void *A_dev, uint32_t count, const void *const *W_de
  * key may share a launch.  Needs a current device (the rule depends on its SM count). */
 int  tgp_k_gemm_group_key(uint32_t M, uint32_t n, uint32_t K, uint32_t *key);
 int  tgp_k_gemm_group_select(int enable);
+/* Name of the kernel that the calling thread's last tgp_k_gemm() / tgp_k_gemm_group() launched (the choice depends on
+ * M, n, K and the GPU's SM count), as a NUL-terminated string of at most capacity - 1 characters; "" before the first. */
+int  tgp_k_gemm_last_kernel(char *name, uint32_t capacity);
 /* Which kernel serves M > 16: 0 (default) the tcgen05 tensor-core GEMM, 1 the CUDA-core tile kernel (an on-device
  * cross-check).  M <= 16 always takes the weight-streaming GEMV.  Process-wide. */
 int  tgp_k_gemm_select(int impl);

@@ -10,7 +10,7 @@ Parity status of each part:
 * forward.py  - pinned by brute-force double-precision loops, closed forms, and
                 library cross-checks on tiny shapes (tests/test_oracle_forward.py).
 * trace.py    - pinned by hand-computed op counts on a toy shape (tests/test_oracle_policy.py).
-* policy.py   - the paper gives prose only (Sections III-B, IV-C, IV-D); classification
+* policy.py   - the paper gives prose only (Sections III-B, IV-D, IV-E); classification
                 is pinned by hand-computed toy rooflines, the schedule by the invariants
                 in validate.py, closed forms and a brute-force pin-set search.  The
                 policy *constants* (hold window, zero-copy ratio, ring minimum, alignment,

@@ -6,11 +6,11 @@ TEST INFRASTRUCTURE - see oracle/__init__.py.
 The paper describes the policy in prose only.  What it fixes, and where:
 * three kernel classes - CGI(link)-bound, GPU-memory-bound, compute-bound - from a roofline
   with a compute roof, an HBM roof and a much lower CPU-GPU interconnect roof
-  (Section III-C; Section IV-C "UVM Analyzer");
+  (Section III-C; Section IV-D "UVM Analyzer");
 * prefetch exactly the tensors the upcoming kernel accesses, nothing else of the pool
-  (Section IV-B, IV-D "Prefetch Engine");
+  (Section IV-B, IV-E "Prefetch Engine");
 * link-bound kernels trigger proactive prefetch; tensors reused across consecutive kernels
-  are held resident during their reuse window (Section IV-C look-ahead affinity, IV-D).
+  are held resident during their reuse window (Section IV-D look-ahead affinity, IV-E).
 Everything numeric below is this build's reading: the exact inequality, ties, the hold
 window W_AFF, the zero-copy ratio ZC_DEN, the ring minimum, the 512-byte alignment.
 
@@ -94,7 +94,7 @@ def alignup(x: int) -> int:
 
 def classify(flops: int, hbm: int, mig: int, m: Machine, bit_p: bool = True, measured_ns: int = 0) -> int:
     """measured_ns > 0: the runtime monitor's kernel time replaces both analytic roofs in the link test
-    (Section IV-D "Runtime Monitor": classes are re-evaluated from measured kernel time): LINK iff moving the op's
+    (Section IV-E "Runtime Monitor": classes are re-evaluated from measured kernel time): LINK iff moving the op's
     pool bytes over the link takes longer than the kernel itself ran, mig / Bl > t  <=>  mig * 1e9 > t_ns * Bl."""
     if mig > 0 and not bit_p:
         return CLS_LINK

@@ -2,9 +2,9 @@
 
 TEST INFRASTRUCTURE - see oracle/__init__.py.
 
-The paper records kernel-tensor access pairs in one offline profiling pass (Section IV-C,
+The paper records kernel-tensor access pairs in one offline profiling pass (Section IV-D,
 "Kernel-Tensor Access Tracing") and counts FLOPs and loads per kernel by binary
-instrumentation (Section IV-F).  Here the counts are analytic functions of the shapes,
+instrumentation (Section IV-G).  Here the counts are analytic functions of the shapes,
 fixed in one table below; the trace is logical (one op per weight block, whatever the
 GPU fuses).  All quantities are Python integers.
 

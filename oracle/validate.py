@@ -4,7 +4,7 @@ TEST INFRASTRUCTURE - see oracle/__init__.py.
 
 It knows nothing of how a plan was made.  It parses the canonical blobs, replays the
 commands against a versioned model of host pool and device arena, and checks the
-properties any correct schedule for the paper's problem must have (Section IV-D: the
+properties any correct schedule for the paper's problem must have (Section IV-E: the
 tensors a kernel needs are on the device before it runs, inside a fixed capacity):
 
  I1 resident at use : every (op, tensor) access finds that tensor's bytes in the arena

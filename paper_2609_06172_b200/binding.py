@@ -93,12 +93,15 @@ _SIGS = {
     "tgp_tap_index": [_P, C.POINTER(_U64), C.POINTER(_U64)],
     "tgp_set_op_timing": [_P, C.c_int],
     "tgp_op_times": [_P, C.POINTER(C.c_float), _U32, C.POINTER(_U32), C.POINTER(_U32)],
-    "tgp_k_embed": [_P, _P, _P, _U32, _U32, _P],
+    "tgp_k_embed": [_P, _P, _P, _U32, _U32, _U32, _P],
+    "tgp_k_embed_status": [C.POINTER(C.c_int), C.POINTER(_U32), C.POINTER(C.c_int32)],
+    "tgp_k_status_clear": [],
     "tgp_k_rmsnorm": [_P, _U32, _P, _P, _U32, _U32, C.c_float, _P],
     "tgp_k_gemm": [_P, _P, _P, _U32, _U32, _U32, _U32, _U32, C.c_int, _P],
     "tgp_k_gemm_group": [_P, _U32, _P, _P, C.POINTER(_U32), C.POINTER(_U32), _U32, _U32, C.c_int, _P],
     "tgp_k_gemm_group_key": [_U32, _U32, _U32, C.POINTER(_U32)],
     "tgp_k_gemm_group_select": [C.c_int],
+    "tgp_k_gemm_last_kernel": [C.c_char_p, _U32],
     "tgp_k_gemm_select": [C.c_int],
     "tgp_k_attn_select": [C.c_int],
     "tgp_k_gemv_overlap": [C.c_int],
@@ -136,6 +139,22 @@ def lib():
 
 def exported_symbols():
     return sorted(list(_SIGS) + ["tgp_strerror", "tgp_last_error"])
+
+
+def parse_trace(blob):
+    """Decodes the blob of tgp_trace_export(): per op u32 step, u64 site, i32 layer, u32 kind, u64 flops, u64 hbm bytes,
+    u32 n_acc, then n_acc x (u32 tensor, u32 mode, u64 touched).  Returns a list of
+    (step, site, layer, kind, flops, hbm, [(tensor, mode, touched)])."""
+    import struct
+    ops, off = [], 0
+    head = struct.Struct("<IQiIQQI")
+    while off < len(blob):
+        step, site, layer, kind, flops, hbm, n = head.unpack_from(blob, off)
+        off += head.size
+        acc = [struct.unpack_from("<IIQ", blob, off + 16 * k) for k in range(n)]
+        off += 16 * n
+        ops.append((step, site, layer, kind, flops, hbm, acc))
+    return ops
 
 
 def _ptr(x):
@@ -227,6 +246,10 @@ class Ctx:
         buf = C.create_string_buffer(max(1, n.value))
         self._ck(lib().tgp_trace_export(self._h, buf, C.byref(n)), "tgp_trace_export")
         return buf.raw[:n.value]
+
+    def trace_ops(self):
+        """The recorded trace decoded: a list of (step, site, layer, kind, flops, hbm bytes, [(tensor, mode, touched)])."""
+        return parse_trace(self.trace_export())
 
     def set_budget(self, nbytes):
         self._ck(lib().tgp_set_budget(self._h, nbytes), "tgp_set_budget")
@@ -353,8 +376,19 @@ def _k(rc, where):
         raise TgpError(rc, where)
 
 
-def k_embed(table, tok, x, M, d, stream=None):
-    _k(lib().tgp_k_embed(_ptr(table), _ptr(tok), _ptr(x), M, d, _ptr(stream)), "tgp_k_embed")
+def k_embed(table, tok, x, M, d, V, stream=None):
+    _k(lib().tgp_k_embed(_ptr(table), _ptr(tok), _ptr(x), M, d, V, _ptr(stream)), "tgp_k_embed")
+
+
+def k_embed_status():
+    """(bad, row, token) of the first out-of-vocabulary token an embedding gather met, bad == 0 if none."""
+    b, r, t = C.c_int(), _U32(), C.c_int32()
+    _k(lib().tgp_k_embed_status(C.byref(b), C.byref(r), C.byref(t)), "tgp_k_embed_status")
+    return b.value, r.value, t.value
+
+
+def k_status_clear():
+    _k(lib().tgp_k_status_clear(), "tgp_k_status_clear")
 
 
 def k_rmsnorm(x, ldx, g, h, M, d, eps, stream=None):
@@ -401,6 +435,12 @@ def k_attn_select(impl):
 
 def k_gemm_tc_variant(v):
     _k(lib().tgp_k_gemm_tc_variant(v), "tgp_k_gemm_tc_variant")
+
+
+def k_gemm_last_kernel():
+    buf = C.create_string_buffer(96)
+    _k(lib().tgp_k_gemm_last_kernel(buf, 96), "tgp_k_gemm_last_kernel")
+    return buf.value.decode()
 
 
 def k_attn_status():

@@ -50,7 +50,7 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
 template <int DH> __device__ __forceinline__ uint32_t tile_off(uint32_t r, uint32_t c) { return r * (DH * 2) + ((c ^ (r & 7u)) << 4); }
 
 template <int DH>
-__global__ void __launch_bounds__(128) attn_prefill_mma_kernel(PArgs a) {
+__global__ void __launch_bounds__(128) tgp_attn_prefill_mma_kernel(PArgs a) {
     extern __shared__ __align__(128) uint8_t smem[];
     constexpr int CH = DH / 8;                              // 16-byte chunks per row
     constexpr int TILE = BN * DH * 2;
@@ -189,12 +189,12 @@ int tgpk_attn_prefill_tc(const void *qb, const TgpTilePtrs &tiles, void *ob, con
     static bool attr64 = false, attr128 = false;
     if (c->Dh == 64) {
         constexpr int SM = (BM + 4 * BN) * 64 * 2;
-        if (!attr64) { if (cudaFuncSetAttribute(attn_prefill_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM) != cudaSuccess) return TGP_E_CUDA; attr64 = true; }
-        attn_prefill_mma_kernel<64><<<grid, 128, SM, st>>>(a);
+        if (!attr64) { if (cudaFuncSetAttribute(tgp_attn_prefill_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM) != cudaSuccess) return TGP_E_CUDA; attr64 = true; }
+        tgp_attn_prefill_mma_kernel<64><<<grid, 128, SM, st>>>(a);
     } else if (c->Dh == 128) {
         constexpr int SM = (BM + 4 * BN) * 128 * 2;
-        if (!attr128) { if (cudaFuncSetAttribute(attn_prefill_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM) != cudaSuccess) return TGP_E_CUDA; attr128 = true; }
-        attn_prefill_mma_kernel<128><<<grid, 128, SM, st>>>(a);
+        if (!attr128) { if (cudaFuncSetAttribute(tgp_attn_prefill_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM) != cudaSuccess) return TGP_E_CUDA; attr128 = true; }
+        tgp_attn_prefill_mma_kernel<128><<<grid, 128, SM, st>>>(a);
     } else {
         return TGP_E_INVAL;
     }

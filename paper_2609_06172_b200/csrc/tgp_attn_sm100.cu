@@ -72,7 +72,7 @@ __device__ __forceinline__ uint64_t add2(uint64_t x, uint64_t y) { uint64_t d; a
 __device__ __forceinline__ float max3(float x, float y, float z) { float d; asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(x), "f"(y), "f"(z)); return d; }
 
 template <int DH>
-__global__ void __launch_bounds__(THREADS, 2) attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUtensorMap tmO, const TArgs a) {
+__global__ void __launch_bounds__(THREADS, 2) tgp_attn_prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV, const __grid_constant__ CUtensorMap tmO, const TArgs a) {
     extern __shared__ __align__(1024) uint8_t smem[];
     constexpr int KB = DH / 64;                          // 64-wide blocks of the head dimension
     constexpr uint32_t Q_BYTES = KB * BQ * 128, KV_BYTES = KB * BKV * 128;
@@ -382,23 +382,25 @@ int tgpk_attn_prefill_tc5(const void *qb, const TgpTilePtrs &tiles, void *ob, co
     static bool attr64 = false, attr128 = false;
     if (c->Dh == 64) {
         if (!attr64) {
-            if (cudaFuncSetAttribute(attn_prefill_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64>()) != cudaSuccess) return TGP_E_CUDA;
-            cudaFuncSetAttribute(attn_prefill_tc_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+            if (cudaFuncSetAttribute(tgp_attn_prefill_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<64>()) != cudaSuccess) return TGP_E_CUDA;
+            cudaFuncSetAttribute(tgp_attn_prefill_tc_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
             attr64 = true;
         }
-        attn_prefill_tc_kernel<64><<<grid, THREADS, smem_bytes<64>(), st>>>(mq, mkv, mo, a);
+        tgp_attn_prefill_tc_kernel<64><<<grid, THREADS, smem_bytes<64>(), st>>>(mq, mkv, mo, a);
     } else {
         if (!attr128) {
-            if (cudaFuncSetAttribute(attn_prefill_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128>()) != cudaSuccess) return TGP_E_CUDA;
-            cudaFuncSetAttribute(attn_prefill_tc_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+            if (cudaFuncSetAttribute(tgp_attn_prefill_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<128>()) != cudaSuccess) return TGP_E_CUDA;
+            cudaFuncSetAttribute(tgp_attn_prefill_tc_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
             attr128 = true;
         }
-        attn_prefill_tc_kernel<128><<<grid, THREADS, smem_bytes<128>(), st>>>(mq, mkv, mo, a);
+        tgp_attn_prefill_tc_kernel<128><<<grid, THREADS, smem_bytes<128>(), st>>>(mq, mkv, mo, a);
     }
     if (cudaGetLastError() != cudaSuccess) return TGP_E_CUDA;
     tgpk_launches += 1;
     return TGP_OK;
 }
+
+int tgpk_attn_status_clear() { const int z = 0; return cudaMemcpyToSymbol(g_attn_tc_error, &z, sizeof(z)) == cudaSuccess ? TGP_OK : TGP_E_CUDA; }
 
 extern "C" int tgp_k_attn_status(int *error_code) {
     if (!error_code) return TGP_E_INVAL;

@@ -60,7 +60,7 @@ struct TgpEngine {
     uint32_t next_step = 0, pos = 0;
     const int32_t *tok_src = nullptr;
     int device = -1;
-    // optional per-op timestamps (Section IV-D "Runtime Monitor": lightweight timestamping of kernels)
+    // optional per-op timestamps (Section IV-E "Runtime Monitor": lightweight timestamping of kernels)
     bool op_timing = false;
     std::vector<cudaEvent_t> ta, tb_;
     uint32_t timed_op0 = 0, timed_nops = 0;
@@ -335,7 +335,7 @@ static inline char *where(const tgp_ctx *ctx, const TgpOp &o, uint32_t k) {
     return w == UINT64_MAX ? ctx->pools[t.pool].dev_alias + t.off : (char *)ctx->arena + w;
 }
 
-// ---- managed-hints variant (the paper's mechanism, Section IV-D: cudaMemPrefetchAsync at tensor granularity and
+// ---- managed-hints variant (the paper's mechanism, Section IV-E: cudaMemPrefetchAsync at tensor granularity and
 // cudaMemAdvise for resident tensors) driven by the same plan as the ring --------------------------------------------
 // advice, once per run: pins prefer the device; in-place (zero-copy) tensors stay on the host, mapped into the GPU.
 // (Read-mostly duplication of the weights was measured slower here than plain migration with explicit eviction.)
@@ -472,7 +472,7 @@ static int run_expert_block(tgp_ctx *ctx, const TgpRole &r, const void *W, uint3
     }
 }
 
-// An expert the router chose but the trace does not list (Section IV-C: identity mismatch -> no prefetch for it):
+// An expert the router chose but the trace does not list (Section IV-D: identity mismatch -> no prefetch for it):
 // its blocks are fetched one at a time into the spill buffer on the compute stream and used at once.
 static int run_expert_fallback(tgp_ctx *ctx, int32_t layer, int32_t expert, cudaStream_t cs) {
     TgpEngine *e = ctx->eng;
@@ -493,6 +493,16 @@ static int run_expert_fallback(tgp_ctx *ctx, int32_t layer, int32_t expert, cuda
         }
     }
     return TGP_OK;
+}
+
+// Model role of access k of op o, or nullptr when the op has no such access or its tensor was never bound to a role
+// (a trace recorded by hand through tgp_trace_op(), a tensor registered after tgp_model_bind()).
+static inline const TgpRole *role_of(const tgp_ctx *ctx, const TgpOp &o, uint32_t k) {
+    if (k >= o.nacc) return nullptr;
+    const uint32_t t = ctx->acc[o.acc0 + k].tensor;
+    if (t >= ctx->role_of_tensor.size()) return nullptr;
+    const int32_t ri = ctx->role_of_tensor[t];
+    return ri < 0 ? nullptr : &ctx->roles[ri];
 }
 
 // What a dense weight block is multiplied with and where its product goes: activations, output (row stride ldc, the
@@ -528,6 +538,12 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
                         float *logits_dev, int32_t *argmax_dev, void *compute_stream, void *copy_stream, tgp_step_stats *stats) {
     if (!ctx || !logits_dev) return TGP_E_INVAL;
     if (!ctx->plan.valid) return TGP_E_NO_PLAN;
+    // host tokens are checked before anything is enqueued: an id outside the vocabulary would make the embedding gather
+    // read past its table (the device kernel zeroes such a row and records it, but a caller's mistake is reported here)
+    if (tokens_host && ctx->bound)
+        for (uint64_t i = 0, n = (uint64_t)B * q_len; i < n; ++i)
+            if (tokens_host[i] < 0 || (uint32_t)tokens_host[i] >= ctx->cfg.V)
+                return tgp_fail(ctx, TGP_E_INVAL, "token id outside the vocabulary at index " + std::to_string(i));
     TgpEngine *e = ctx->eng;
     if (!e || !ctx->bound) return tgp_fail(ctx, TGP_E_STATE, "no model bound with a workspace");
     const bool ring = ctx->variant == TGP_VAR_EXPLICIT_RING;
@@ -573,9 +589,9 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             for (uint32_t j = 0; j < TGP_GEMM_GROUP_MAX && i + j < st.op0 + st.nops; ++j) {
                 const TgpOp &f = ctx->ops[i + j];
                 if (f.kind != TGP_OP_GEMM || f.layer != o.layer || !f.nacc) break;
-                const int32_t ri = ctx->role_of_tensor[ctx->acc[f.acc0].tensor];
-                if (ri < 0) break;
-                const TgpRole &r = ctx->roles[ri];
+                const TgpRole *rp = role_of(ctx, f, 0);
+                if (!rp) break;
+                const TgpRole &r = *rp;
                 GemmTarget t;
                 if (!r.rows || !gemm_target(e, c, r, M, B, logits_dev, &t) || !t.Mrows || t.Mrows > 32) break;
                 const uint32_t Kj = (uint32_t)(ctx->tensors[ctx->acc[f.acc0].tensor].size / (2ull * r.rows));
@@ -594,7 +610,7 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
                 if (ctx->plan.op_is_wait_target[i + j] && ctx->tensors[ctx->acc[ctx->ops[i + j].acc0].tensor].size < (2u << 20)) cnt = 0;
             if (cnt >= 2) span = cnt;
             for (uint32_t j = 0; j < span && span > 1 && g_expert >= 0; ++j) {       // what run_expert_block does around an expert's products
-                const TgpRole &r = ctx->roles[ctx->role_of_tensor[ctx->acc[ctx->ops[i + j].acc0].tensor]];
+                const TgpRole &r = *role_of(ctx, ctx->ops[i + j], 0);
                 g_gather |= r.kind == TGP_K_WG && r.row0 == 0;
                 g_scatter |= r.kind == TGP_K_WD && r.row0 + r.rows == c.d;
             }
@@ -616,19 +632,22 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
         rc = TGP_OK;
         switch (o.kind) {
         case TGP_OP_EMBED:
-            rc = tgpk_embed(where(ctx, o, 0), tok, e->x, M, c.d, cs);
+            if (!o.nacc) return tgp_fail(ctx, TGP_E_MISMATCH, "embedding op without a table");
+            rc = tgpk_embed(where(ctx, o, 0), tok, e->x, M, c.d, c.V, cs);
             break;
         case TGP_OP_RMSNORM: {
-            const TgpRole &r = ctx->roles[ctx->role_of_tensor[ctx->acc[o.acc0].tensor]];
+            const TgpRole *rp = role_of(ctx, o, 0);
+            if (!rp || (rp->kind != TGP_K_G1 && rp->kind != TGP_K_G2 && rp->kind != TGP_K_GF)) return tgp_fail(ctx, TGP_E_MISMATCH, "norm op on a tensor that is not a bound gain");
+            const TgpRole &r = *rp;
             if (r.kind == TGP_K_GF) rc = tgpk_rmsnorm(e->x + (size_t)(q_len - 1) * c.d, q_len * c.d, where(ctx, o, 0), e->hf, B, c.d, c.eps, cs);
             else rc = tgpk_rmsnorm(e->x, c.d, where(ctx, o, 0), e->h, M, c.d, c.eps, cs);
             break;
         }
         case TGP_OP_GEMM: {
+            const TgpRole *rp = role_of(ctx, o, 0);
+            if (!rp || !rp->rows) return tgp_fail(ctx, TGP_E_MISMATCH, "GEMM op on a tensor with no model role");
             const tgp_access &a = ctx->acc[o.acc0];
-            const int32_t ri = ctx->role_of_tensor[a.tensor];
-            if (ri < 0) return tgp_fail(ctx, TGP_E_MISMATCH, "GEMM op on a tensor with no model role");
-            const TgpRole &r = ctx->roles[ri];
+            const TgpRole &r = *rp;
             const uint32_t K = (uint32_t)(ctx->tensors[a.tensor].size / (2ull * r.rows));
             const void *W = where(ctx, o, 0);
             if (span > 1) {
@@ -657,7 +676,7 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             break;
         }
         case TGP_OP_ROUTER: {
-            if (!c.E) return tgp_fail(ctx, TGP_E_MISMATCH, "router op in a dense model");
+            if (!c.E || !o.nacc) return tgp_fail(ctx, TGP_E_MISMATCH, "router op in a dense model or without its weight");
             rc = tgpk_router(e->h, where(ctx, o, 0), e->bias_dev + (size_t)o.layer * c.E, e->topk_idx, e->topk_gate, e->erow, e->egate, e->ecount,
                              M, e->max_tokens, c.d, c.E, c.topk, cs);
             if (rc) break;
@@ -668,8 +687,8 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             for (uint32_t j = i + 1; j < st.op0 + st.nops && ctx->ops[j].layer == o.layer; ++j) {
                 const TgpOp &f = ctx->ops[j];
                 if (f.kind != TGP_OP_GEMM) { if (f.kind == TGP_OP_SWIGLU) continue; break; }
-                const int32_t fr = ctx->role_of_tensor[ctx->acc[f.acc0].tensor];
-                if (fr >= 0 && ctx->roles[fr].expert >= 0) traced[ctx->roles[fr].expert] = 1;
+                const TgpRole *fr = role_of(ctx, f, 0);
+                if (fr && fr->expert >= 0 && (uint32_t)fr->expert < c.E) traced[fr->expert] = 1;
             }
             const size_t slot = ((size_t)e->next_step * c.L + o.layer) * c.E;
             if (ctx->run_counts.size() < slot + c.E) ctx->run_counts.resize(slot + c.E, 0);
@@ -689,10 +708,18 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             memset(&tp, 0, sizeof(tp));
             uint32_t nt = 0;
             for (uint32_t k = 0; k < o.nacc; ++k) {
-                const TgpRole &r = ctx->roles[ctx->role_of_tensor[ctx->acc[o.acc0 + k].tensor]];
+                const TgpRole *rp = role_of(ctx, o, k);
+                if (!rp || (rp->kind != TGP_K_KTILE && rp->kind != TGP_K_VTILE)) return tgp_fail(ctx, TGP_E_MISMATCH, "attention op on a tensor that is not a bound KV tile");
+                const TgpRole &r = *rp;
                 if (r.block >= TGP_MAX_TILES) return tgp_fail(ctx, TGP_E_TOO_LARGE, "KV tile index");
                 (r.kind == TGP_K_KTILE ? tp.k : tp.v)[r.block] = where(ctx, o, k);
                 nt = std::max(nt, r.block + 1);
+            }
+            {   // every tile the kernel will address must have been listed by the op (an append touches the tiles of the new
+                // positions, attention every tile below the cached length)
+                const uint32_t t_lo = o.kind == TGP_OP_ROPE_KV ? pos0 / c.TK : 0, t_hi = (pos0 + q_len - 1) / c.TK;
+                for (uint32_t j = t_lo; j <= t_hi; ++j)
+                    if (j >= TGP_MAX_TILES || !tp.k[j] || !tp.v[j]) return tgp_fail(ctx, TGP_E_MISMATCH, "the trace does not list a KV tile this step addresses");
             }
             if (o.kind == TGP_OP_ROPE_KV) rc = tgpk_rope_kv(e->q32, e->k32, e->v32, e->qb, tp, e->cos_t, e->sin_t, &c, B, q_len, pos0, cs);
             else rc = tgpk_attn(e->qb, tp, (c.max_len + c.TK - 1) / c.TK, e->ob, &c, B, q_len, pos0, e->scratch, cs);
@@ -722,12 +749,12 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             };
             int trc = TGP_OK;
             if (o.kind == TGP_OP_RMSNORM) {
-                const bool fin = ctx->roles[ctx->role_of_tensor[ctx->acc[o.acc0].tensor]].kind == TGP_K_GF;
+                const bool fin = role_of(ctx, o, 0)->kind == TGP_K_GF;
                 trc = fin ? tap_copy(TGP_TAP_HF, 0, e->hf, (uint64_t)B * c.d * 2) : tap_copy(TGP_TAP_H, 0, e->h, (uint64_t)M * c.d * 2);
             } else if (o.kind == TGP_OP_ROPE_KV) {
                 trc = tap_copy(TGP_TAP_Q, 0, e->qb, (uint64_t)M * qd * 2);
                 for (uint32_t k = 0; k < o.nacc && !trc; ++k) {
-                    const TgpRole &r = ctx->roles[ctx->role_of_tensor[ctx->acc[o.acc0 + k].tensor]];
+                    const TgpRole &r = *role_of(ctx, o, k);
                     trc = tap_copy(r.kind == TGP_K_KTILE ? TGP_TAP_KTILE : TGP_TAP_VTILE, r.block, where(ctx, o, k), ctx->tensors[ctx->acc[o.acc0 + k].tensor].size);
                 }
             } else if (o.kind == TGP_OP_ATTN) {
@@ -770,9 +797,12 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
         stats->n_cmds = n_cmds; stats->n_launches = (uint32_t)(tgpk_launches - launches0); stats->n_mismatch = n_mismatch;
         CU(ctx, cudaEventElapsedTime(&stats->step_ms, e->t0, e->t1));
         // the step has been waited for: a tensor-core kernel whose bounded wait ran out has left its mark
-        int gemm_err = 0, attn_err = 0;
+        int gemm_err = 0, attn_err = 0, bad_tok = 0;
+        uint32_t bad_row = 0; int32_t bad_id = 0;
         if (tgp_k_gemm_status(&gemm_err) == TGP_OK && tgp_k_attn_status(&attn_err) == TGP_OK && (gemm_err || attn_err))
             return tgp_fail(ctx, TGP_E_CUDA, "a tensor-core kernel gave up on a bounded wait (GEMM code " + std::to_string(gemm_err) + ", attention code " + std::to_string(attn_err) + "): results of this step are incomplete");
+        if (tgp_k_embed_status(&bad_tok, &bad_row, &bad_id) == TGP_OK && bad_tok)
+            return tgp_fail(ctx, TGP_E_CUDA, "the embedding gather met token id " + std::to_string(bad_id) + " (row " + std::to_string(bad_row) + "), outside the vocabulary: that row was computed from zeros");
     }
     return TGP_OK;
 }

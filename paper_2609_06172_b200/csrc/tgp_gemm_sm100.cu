@@ -38,7 +38,7 @@ struct Smem {
 // activation rows a CTA then streams 128 weight rows through its TMA ring instead of BN, which is what such a product
 // is bound by.
 template <int BN, int ST, int KH, bool SWAP>
-__global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+__global__ void __launch_bounds__(192) tgp_matmul_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                                                       float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     extern __shared__ uint8_t smem_raw[];
     using S = Smem<BN, ST, KH>;
@@ -170,7 +170,7 @@ __global__ void __launch_bounds__(192) gemm_tc_kernel(const __grid_constant__ CU
 // one (acc_full / acc_empty barriers per buffer).  Same bounded waits and error word as the kernel above.
 constexpr int P_BN = 256, P_STAGES = 4;
 
-__global__ void __launch_bounds__(192, 1) gemm_tc_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+__global__ void __launch_bounds__(192, 1) tgp_matmul_tc_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                                                                     float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     extern __shared__ uint8_t smem_raw[];
     constexpr int A_BYTES = BM * BK * 2, B_BYTES = P_BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
@@ -313,7 +313,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_persistent_kernel(const __grid
 // TMEM is freed keeps either CTA from leaving while its partner still works on its memory.
 constexpr int Q_HALVES = 2, Q_STAGES = 6 / Q_HALVES;   // a stage holds Q_HALVES 64-wide K blocks
 
-__global__ void __launch_bounds__(192, 1) gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+__global__ void __launch_bounds__(192, 1) tgp_matmul_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                                                               float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     extern __shared__ uint8_t smem_raw[];
     constexpr int A_BYTES = BM * BK * 2, B_BYTES = (P_BN / 2) * BK * 2, STAGE_BYTES = Q_HALVES * (A_BYTES + B_BYTES);
@@ -467,11 +467,11 @@ template <int BN, int ST, int KH, bool SWAP = false>
 static bool launch_tile(const CUtensorMap &ma, const CUtensorMap &mb, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(gemm_tc_kernel<BN, ST, KH, SWAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN, ST, KH>::TOTAL) != cudaSuccess) return false;
+        if (cudaFuncSetAttribute(tgp_matmul_tc_kernel<BN, ST, KH, SWAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN, ST, KH>::TOTAL) != cudaSuccess) return false;
         attr_set = true;
     }
     dim3 grid(((M + BM - 1) / BM) * ((n + BN - 1) / BN));
-    gemm_tc_kernel<BN, ST, KH, SWAP><<<grid, 192, Smem<BN, ST, KH>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
+    tgp_matmul_tc_kernel<BN, ST, KH, SWAP><<<grid, 192, Smem<BN, ST, KH>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
     return true;
 }
 
@@ -485,7 +485,7 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
     static int sms = 0;
     if (!sms) { int dev = 0; cudaGetDevice(&dev); if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148; }
     // Up to 64 activation rows on a block with 128-row tiles for a good part of the SMs: the weights become the 128-row
-    // operand (see gemm_tc_kernel), the activations the narrow one.  A CTA takes in about 100 GB/s through its TMA ring
+    // operand (see tgp_matmul_tc_kernel), the activations the narrow one.  A CTA takes in about 100 GB/s through its TMA ring
     // whatever the tile, so the form pays from 64 weight tiles on (n=8192, K=8192, M=64: 34 us against 47 us), for more
     // than 32 rows from 32 tiles on (n=4096, K=14336, M=64: 48 us against 70 us); with fewer tiles the weight-streaming
     // kernels and the narrow tiles below have more CTAs at work
@@ -499,6 +499,7 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
                                  : launch_tile<128, 2, 3, true>(mw, mx, C, n, M, K, ldc, col0, accumulate, st);
         if (!ok || cudaGetLastError() != cudaSuccess) return TGP_E_CUDA;
         tgpk_launches += 1;
+        tgpk_last_gemm_kernel = "tgp_matmul_tc_kernel (weights as the 128-row operand)";
         return TGP_OK;
     }
     const uint32_t tiles_p = ((M + BM - 1) / BM) * ((n + P_BN - 1) / P_BN);
@@ -520,7 +521,7 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
         constexpr int SMEM = Q_STAGES * Q_HALVES * (BM * BK * 2 + (P_BN / 2) * BK * 2) + 160 + 1024;
         static bool attr_q = false;
         if (!attr_q) {
-            if (cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess) return TGP_E_CUDA;
+            if (cudaFuncSetAttribute(tgp_matmul_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess) return TGP_E_CUDA;
             attr_q = true;
         }
         const uint32_t pairs_max = (uint32_t)sms / 2, npairs = tiles_q < pairs_max ? tiles_q : pairs_max;
@@ -534,15 +535,15 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
         attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, gemm_tc_pair_kernel, ma, mb, C, M, n, K, ldc, col0, accumulate) != cudaSuccess) return TGP_E_CUDA;
+        if (cudaLaunchKernelEx(&cfg, tgp_matmul_tc_pair_kernel, ma, mb, C, M, n, K, ldc, col0, accumulate) != cudaSuccess) return TGP_E_CUDA;
     } else if (persistent) {
         constexpr int SMEM = P_STAGES * (BM * BK * 2 + P_BN * BK * 2) + 128 + 1024;
         static bool attr_p = false;
         if (!attr_p) {
-            if (cudaFuncSetAttribute(gemm_tc_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess) return TGP_E_CUDA;
+            if (cudaFuncSetAttribute(tgp_matmul_tc_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess) return TGP_E_CUDA;
             attr_p = true;
         }
-        gemm_tc_persistent_kernel<<<tiles_p < (uint32_t)sms ? tiles_p : (uint32_t)sms, 192, SMEM, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
+        tgp_matmul_tc_persistent_kernel<<<tiles_p < (uint32_t)sms ? tiles_p : (uint32_t)sms, 192, SMEM, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
     } else if (bn == 128) {
         // fewer tiles than SMs: one CTA per SM, so the ring may take all of shared memory (a 3-stage ring leaves a lone
         // CTA waiting on L2 latency); otherwise two CTAs per SM with three stages each
@@ -555,6 +556,7 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
     }
     if (cudaGetLastError() != cudaSuccess) return TGP_E_CUDA;
     tgpk_launches += 1;
+    tgpk_last_gemm_kernel = paired ? "tgp_matmul_tc_pair_kernel" : persistent ? "tgp_matmul_tc_persistent_kernel" : "tgp_matmul_tc_kernel";
     return TGP_OK;
 }
 
@@ -563,6 +565,8 @@ extern "C" int tgp_k_gemm_tc_variant(int v) {
     g_tc_variant = v;
     return TGP_OK;
 }
+
+int tgpk_gemm_status_clear() { const int z = 0; return cudaMemcpyToSymbol(g_gemm_tc_error, &z, sizeof(z)) == cudaSuccess ? TGP_OK : TGP_E_CUDA; }
 
 extern "C" int tgp_k_gemm_status(int *error_code) {
     if (!error_code) return TGP_E_INVAL;

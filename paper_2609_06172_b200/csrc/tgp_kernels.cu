@@ -9,6 +9,7 @@
 #include "tgp_kernels.h"
 
 thread_local uint64_t tgpk_launches = 0;     // kernels launched by this thread (reported in the step statistics)
+thread_local const char *tgpk_last_gemm_kernel = "";   // name of the kernel the last weight-block product of this thread launched
 #define LAUNCH_CHECK(n) do { cudaError_t e_ = cudaGetLastError(); if (e_ != cudaSuccess) return TGP_E_CUDA; tgpk_launches += (n); } while (0)
 
 typedef __nv_bfloat16 bf16;
@@ -31,10 +32,20 @@ __device__ __forceinline__ float warp_max(float v) {
 }
 
 // ---- embedding gather ------------------------------------------------------------------------
-__global__ void embed_kernel(const bf16 *__restrict__ table, const int32_t *__restrict__ tok, float *__restrict__ x, uint32_t d) {
+// A token id outside [0, V) would index past the table (which may be mapped host memory): such a row is written as
+// zeros and the first offending (row, id) is recorded in g_embed_error for tgp_k_embed_status().
+__device__ unsigned long long g_embed_error = 0;      // 0, or 1 << 63 | row << 32 | (uint32_t)id of the first bad token
+
+__global__ void tgp_embed_kernel(const bf16 *__restrict__ table, const int32_t *__restrict__ tok, float *__restrict__ x, uint32_t d, uint32_t V) {
     const uint32_t m = blockIdx.x;
-    const uint4 *row = reinterpret_cast<const uint4 *>(table + (size_t)tok[m] * d);
+    const int32_t id = tok[m];
     float4 *out = reinterpret_cast<float4 *>(x + (size_t)m * d);
+    if (id < 0 || (uint32_t)id >= V) {
+        for (uint32_t i = threadIdx.x; i < d / 4; i += blockDim.x) out[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (threadIdx.x == 0) atomicCAS(&g_embed_error, 0ull, (1ull << 63) | ((unsigned long long)m << 32) | (uint32_t)id);
+        return;
+    }
+    const uint4 *row = reinterpret_cast<const uint4 *>(table + (size_t)id * d);
     for (uint32_t i = threadIdx.x; i < d / 8; i += blockDim.x) {
         float f[8];
         unpack8(row[i], f);
@@ -44,7 +55,7 @@ __global__ void embed_kernel(const bf16 *__restrict__ table, const int32_t *__re
 }
 
 // ---- RMSNorm -> bf16 -------------------------------------------------------------------------
-__global__ void rmsnorm_kernel(const float *__restrict__ x, uint32_t ldx, const bf16 *__restrict__ g, bf16 *__restrict__ h, uint32_t d, float eps) {
+__global__ void tgp_rmsnorm_kernel(const float *__restrict__ x, uint32_t ldx, const bf16 *__restrict__ g, bf16 *__restrict__ h, uint32_t d, float eps) {
     __shared__ float red[32];
     const float4 *row = reinterpret_cast<const float4 *>(x + (size_t)blockIdx.x * ldx);
     float ss = 0.f;
@@ -75,7 +86,7 @@ __global__ void rmsnorm_kernel(const float *__restrict__ x, uint32_t ldx, const 
 // No block barrier and no shared memory, so no SM idles while another warp reduces; the summation order
 // is fixed (lane-strided partials, butterfly), hence results are deterministic run to run.
 template <int MT, int R, int U>
-__global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+__global__ void __launch_bounds__(256) tgp_wstream_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                    uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarp = (gridDim.x * blockDim.x) >> 5;
@@ -135,13 +146,13 @@ __global__ void __launch_bounds__(256) gemv_kernel(const bf16 *__restrict__ A, c
 }
 
 // Several products that read the same activations (the q, k and v projections of a layer) in one launch: the output
-// rows of the parts are walked as one list, one warp per row, with exactly the arithmetic of gemv_kernel<MT, 1, U>, so
+// rows of the parts are walked as one list, one warp per row, with exactly the arithmetic of tgp_wstream_kernel<MT, 1, U>, so
 // the result is bit-identical to separate launches; what is saved is two launch floors of about a microsecond each.
 // (groups[s]: CTAs' worth of rows in part s, for the kernels that walk row groups instead of rows)
 struct GemvParts { const bf16 *W[TGP_GEMM_GROUP_MAX]; float *C[TGP_GEMM_GROUP_MAX]; uint32_t n[TGP_GEMM_GROUP_MAX], ldc[TGP_GEMM_GROUP_MAX], groups[TGP_GEMM_GROUP_MAX], count; };
 
 template <int MT, int U>
-__global__ void __launch_bounds__(256) gemv_group_kernel(const bf16 *__restrict__ A, const GemvParts p, uint32_t Mrows, uint32_t n_total, uint32_t K, int accumulate) {
+__global__ void __launch_bounds__(256) tgp_wstream_group_kernel(const bf16 *__restrict__ A, const GemvParts p, uint32_t Mrows, uint32_t n_total, uint32_t K, int accumulate) {
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarp = (gridDim.x * blockDim.x) >> 5;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -197,7 +208,7 @@ __global__ void __launch_bounds__(256) gemv_group_kernel(const bf16 *__restrict_
 // rows leave a quarter of them with half the work.  The 8 partial sums of a row meet in shared memory and are added in
 // warp order: deterministic.  Same dependent-launch protocol.
 template <int MT, int RB, int U>
-__global__ void __launch_bounds__(256) gemv_splitk_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+__global__ void __launch_bounds__(256) tgp_wstream_splitk_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                           uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     __shared__ float part[8][RB * MT];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -265,14 +276,14 @@ __global__ void __launch_bounds__(256) gemv_splitk_kernel(const bf16 *__restrict
 // instructions.  Which physical k lands in which logical k-slot of the instruction does not matter for a dot product
 // as long as both operands use the same assignment, and they do (same lane, same byte offsets), so no shuffle or
 // shared-memory staging is needed and every weight byte is loaded exactly once.  Persistent warps, 16 rows each,
-// NB groups of 8 activation rows re-use the weight registers.  Same dependent-launch protocol as gemv_kernel.
+// NB groups of 8 activation rows re-use the weight registers.  Same dependent-launch protocol as tgp_wstream_kernel.
 __device__ __forceinline__ void mma_bf16_16816(float *d, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 template <int NB, int U>
-__global__ void __launch_bounds__(256) gemv_mma_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+__global__ void __launch_bounds__(256) tgp_wstream_mma_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                        uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     const uint32_t lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
     const uint32_t gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarp = (gridDim.x * blockDim.x) >> 5;
@@ -321,7 +332,7 @@ __global__ void __launch_bounds__(256) gemv_mma_kernel(const bf16 *__restrict__ 
 }
 
 // ---- generic tiled GEMM on CUDA cores (any M, n; K % 8 == 0): 64x64 tile, 4x4 per thread ---------
-__global__ void __launch_bounds__(256) gemm_simt_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+__global__ void __launch_bounds__(256) tgp_matmul_simt_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                         uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     __shared__ float As[32][64 + 4];
     __shared__ float Ws[32][64 + 4];
@@ -366,7 +377,7 @@ struct RopeArgs {
     TgpTilePtrs tiles;
 };
 
-__global__ void rope_kv_kernel(RopeArgs a) {
+__global__ void tgp_rope_kv_kernel(RopeArgs a) {
     const uint32_t m = blockIdx.x, b = m / a.q_len, pos = a.pos0 + m % a.q_len;
     const uint32_t half = a.Dh / 2, qd = a.Hq * a.Dh, kd = a.Hkv * a.Dh;
     const float *cs = a.cos_t + (size_t)pos * half, *sn = a.sin_t + (size_t)pos * half;
@@ -406,7 +417,7 @@ struct AttnArgs {
 
 // One warp per query row, 32 keys per pass: lane = key for the scores, lane = output dims for P.V.
 template <int DH>
-__global__ void __launch_bounds__(128) attn_rows_kernel(AttnArgs a) {
+__global__ void __launch_bounds__(128) tgp_attn_rows_kernel(AttnArgs a) {
     __shared__ float qs[4][DH];
     const uint32_t w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t p = blockIdx.x * 4 + w, hq = blockIdx.y, b = blockIdx.z;
@@ -463,7 +474,7 @@ __global__ void __launch_bounds__(128) attn_rows_kernel(AttnArgs a) {
 // output dims for P.V, fully unrolled so a pass's V loads are in flight together); their partial (max, sum, o[Dh])
 // meet in shared memory and one unnormalised partial per (query head, tile) goes to scratch.
 template <int DH>
-__global__ void attn_decode_partial_kernel(AttnArgs a, uint32_t SPLIT) {
+__global__ void tgp_attn_decode_partial_kernel(AttnArgs a, uint32_t SPLIT) {
     extern __shared__ float dsm[];
     const uint32_t G = a.Hq / a.Hkv;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -549,9 +560,9 @@ __global__ void attn_decode_partial_kernel(AttnArgs a, uint32_t SPLIT) {
 // 16-byte loads, all in flight at once, and dots it with the G queries held in shared memory), then lane = DH/32
 // consecutive output dimensions for P V (each V row is one coalesced warp load; the G weights of a key come by
 // shuffle).  Per-warp online softmax; the SPLIT partials of a head are merged in warp order; output as in the
-// per-head kernel: (max, sum, unnormalised o[DH]) per (sequence, head, tile) for attn_decode_merge_kernel.
+// per-head kernel: (max, sum, unnormalised o[DH]) per (sequence, head, tile) for tgp_attn_decode_merge_kernel.
 template <int DH, int G>
-__global__ void __launch_bounds__(256, 2) attn_decode_group_kernel(AttnArgs a, uint32_t SPLIT) {
+__global__ void __launch_bounds__(256, 2) tgp_attn_decode_group_kernel(AttnArgs a, uint32_t SPLIT) {
     extern __shared__ float dsm[];
     constexpr int DPL = DH / 32;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -687,7 +698,7 @@ __global__ void __launch_bounds__(256, 2) attn_decode_group_kernel(AttnArgs a, u
 }
 
 template <int DH>
-__global__ void attn_decode_merge_kernel(AttnArgs a) {
+__global__ void tgp_attn_decode_merge_kernel(AttnArgs a) {
     const uint32_t hq = blockIdx.x, b = blockIdx.y, i = threadIdx.x;
     const uint32_t nt = (a.pos0 + 1 + a.TK - 1) / a.TK;
     const float *part = a.scratch + (size_t)(b * a.Hq + hq) * a.n_tiles * (DH + 2);
@@ -703,7 +714,7 @@ __global__ void attn_decode_merge_kernel(AttnArgs a) {
 }
 
 // ---- SwiGLU -----------------------------------------------------------------------------------------
-__global__ void swiglu_kernel(const float4 *__restrict__ g, const float4 *__restrict__ u, __nv_bfloat162 *__restrict__ out, uint64_t n4) {
+__global__ void tgp_swiglu_kernel(const float4 *__restrict__ g, const float4 *__restrict__ u, __nv_bfloat162 *__restrict__ out, uint64_t n4) {
     for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n4; i += (uint64_t)gridDim.x * blockDim.x) {
         float4 a = g[i], b = u[i];
         float r0 = a.x / (1.0f + expf(-a.x)) * b.x, r1 = a.y / (1.0f + expf(-a.y)) * b.y;
@@ -714,11 +725,12 @@ __global__ void swiglu_kernel(const float4 *__restrict__ g, const float4 *__rest
 }
 
 // ---- argmax, lowest index on ties -----------------------------------------------------------------
-__global__ void __launch_bounds__(1024) argmax_kernel(const float *__restrict__ logits, int32_t *__restrict__ out, uint32_t V) {
+__global__ void __launch_bounds__(1024) tgp_argmax_kernel(const float *__restrict__ logits, int32_t *__restrict__ out, uint32_t V) {
     __shared__ float bv[32];
     __shared__ uint32_t bi[32];
     const float *row = logits + (size_t)blockIdx.x * V;
-    float best = -INFINITY; uint32_t idx = 0xffffffffu;
+    // the index starts at 0, not at a sentinel: a row of NaNs (no comparison holds) must still give a legal token id
+    float best = -INFINITY; uint32_t idx = 0u;
     for (uint32_t j = threadIdx.x; j < V; j += blockDim.x) { float v = row[j]; if (v > best || (v == best && j < idx)) { best = v; idx = j; } }
     auto merge = [](float &v, uint32_t &i, float ov, uint32_t oi) { if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; } };
 #pragma unroll
@@ -727,7 +739,7 @@ __global__ void __launch_bounds__(1024) argmax_kernel(const float *__restrict__ 
     __syncthreads();
     if (threadIdx.x < 32) {
         best = threadIdx.x < (blockDim.x >> 5) ? bv[threadIdx.x] : -INFINITY;
-        idx = threadIdx.x < (blockDim.x >> 5) ? bi[threadIdx.x] : 0xffffffffu;
+        idx = threadIdx.x < (blockDim.x >> 5) ? bi[threadIdx.x] : 0u;
 #pragma unroll
         for (int o = 16; o; o >>= 1) merge(best, idx, __shfl_xor_sync(0xffffffffu, best, o), __shfl_xor_sync(0xffffffffu, idx, o));
         if (threadIdx.x == 0) out[blockIdx.x] = (int32_t)idx;
@@ -738,7 +750,7 @@ __global__ void __launch_bounds__(1024) argmax_kernel(const float *__restrict__ 
 // logits[e] = sum_k h[m,k] * Wr[e,k] + bias[e] in fp32; the two largest (ties: lower expert id); gates = softmax
 // over those two logits.
 template <int E>
-__global__ void __launch_bounds__(256) router_kernel(const bf16 *__restrict__ h, const bf16 *__restrict__ Wr, const float *__restrict__ bias,
+__global__ void __launch_bounds__(256) tgp_router_kernel(const bf16 *__restrict__ h, const bf16 *__restrict__ Wr, const float *__restrict__ bias,
                                                      int32_t *__restrict__ idx, float *__restrict__ gate, uint32_t M, uint32_t d, uint32_t topk) {
     const uint32_t m = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (m >= M) return;
@@ -779,7 +791,7 @@ __global__ void __launch_bounds__(256) router_kernel(const bf16 *__restrict__ h,
 // Tokens of expert e in ascending token order: rows[e*stride + pos] = m, gates[e*stride + pos] = that token's gate for e.
 // One block per expert walks the tokens in chunks; positions come from a block-wide exclusive scan, so the
 // grouping is deterministic.  topk = number of routed slots per token (1 or 2).
-__global__ void __launch_bounds__(1024) route_fill_kernel(const int32_t *__restrict__ idx, const float *__restrict__ gate, int32_t *__restrict__ rows,
+__global__ void __launch_bounds__(1024) tgp_route_fill_kernel(const int32_t *__restrict__ idx, const float *__restrict__ gate, int32_t *__restrict__ rows,
                                                           float *__restrict__ gates, int32_t *__restrict__ counts, uint32_t M, uint32_t stride, uint32_t topk) {
     __shared__ uint32_t warp_tot[32];
     __shared__ uint32_t base;
@@ -808,14 +820,14 @@ __global__ void __launch_bounds__(1024) route_fill_kernel(const int32_t *__restr
     if (threadIdx.x == 0) counts[e] = (int32_t)base;
 }
 
-__global__ void gather_rows_kernel(const bf16 *__restrict__ src, const int32_t *__restrict__ rows, bf16 *__restrict__ dst, uint32_t d) {
+__global__ void tgp_gather_rows_kernel(const bf16 *__restrict__ src, const int32_t *__restrict__ rows, bf16 *__restrict__ dst, uint32_t d) {
     const uint4 *s = reinterpret_cast<const uint4 *>(src + (size_t)rows[blockIdx.x] * d);
     uint4 *o = reinterpret_cast<uint4 *>(dst + (size_t)blockIdx.x * d);
     for (uint32_t i = threadIdx.x; i < d / 8; i += blockDim.x) o[i] = s[i];
 }
 
 // x[rows[i], :] += gates[i] * y[i, :]   (each token appears at most once per expert: no write conflicts)
-__global__ void scatter_add_kernel(float *__restrict__ x, const float *__restrict__ y, const int32_t *__restrict__ rows, const float *__restrict__ gates, uint32_t d) {
+__global__ void tgp_scatter_add_kernel(float *__restrict__ x, const float *__restrict__ y, const int32_t *__restrict__ rows, const float *__restrict__ gates, uint32_t d) {
     const float g = gates[blockIdx.x];
     float4 *o = reinterpret_cast<float4 *>(x + (size_t)rows[blockIdx.x] * d);
     const float4 *s = reinterpret_cast<const float4 *>(y + (size_t)blockIdx.x * d);
@@ -834,36 +846,36 @@ int tgpk_router(const void *h, const void *Wr, const float *bias, int32_t *idx, 
     if (d % 8 || topk < 1 || topk > 2) return TGP_E_INVAL;
     const uint32_t blocks = (M + 7) / 8;
     switch (E) {
-    case 1: router_kernel<1><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
-    case 2: router_kernel<2><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
-    case 4: router_kernel<4><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
-    case 8: router_kernel<8><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
-    case 16: router_kernel<16><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
+    case 1: tgp_router_kernel<1><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
+    case 2: tgp_router_kernel<2><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
+    case 4: tgp_router_kernel<4><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
+    case 8: tgp_router_kernel<8><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
+    case 16: tgp_router_kernel<16><<<blocks, 256, 0, st>>>((const bf16 *)h, (const bf16 *)Wr, bias, idx, gate, M, d, topk); break;
     default: return TGP_E_INVAL;
     }
-    route_fill_kernel<<<E, 1024, 0, st>>>(idx, gate, rows, gates, counts, M, stride, topk);
+    tgp_route_fill_kernel<<<E, 1024, 0, st>>>(idx, gate, rows, gates, counts, M, stride, topk);
     LAUNCH_CHECK(2);
     return TGP_OK;
 }
 
 int tgpk_gather_rows(const void *src, const int32_t *rows, void *dst, uint32_t m, uint32_t d, cudaStream_t st) {
     if (!m) return TGP_OK;
-    gather_rows_kernel<<<m, 128, 0, st>>>((const bf16 *)src, rows, (bf16 *)dst, d);
+    tgp_gather_rows_kernel<<<m, 128, 0, st>>>((const bf16 *)src, rows, (bf16 *)dst, d);
     LAUNCH_CHECK(1);
     return TGP_OK;
 }
 
 int tgpk_scatter_add(float *x, const float *y, const int32_t *rows, const float *gates, uint32_t m, uint32_t d, cudaStream_t st) {
     if (!m) return TGP_OK;
-    scatter_add_kernel<<<m, 256, 0, st>>>(x, y, rows, gates, d);
+    tgp_scatter_add_kernel<<<m, 256, 0, st>>>(x, y, rows, gates, d);
     LAUNCH_CHECK(1);
     return TGP_OK;
 }
 
-int tgpk_embed(const void *table, const int32_t *tok, float *x, uint32_t M, uint32_t d, cudaStream_t st) {
+int tgpk_embed(const void *table, const int32_t *tok, float *x, uint32_t M, uint32_t d, uint32_t V, cudaStream_t st) {
     if (!M) return TGP_OK;
-    if (d % 8) return TGP_E_INVAL;
-    embed_kernel<<<M, 128, 0, st>>>((const bf16 *)table, tok, x, d);
+    if (d % 8 || !V) return TGP_E_INVAL;
+    tgp_embed_kernel<<<M, 128, 0, st>>>((const bf16 *)table, tok, x, d, V);
     LAUNCH_CHECK(1);
     return TGP_OK;
 }
@@ -871,7 +883,7 @@ int tgpk_embed(const void *table, const int32_t *tok, float *x, uint32_t M, uint
 int tgpk_rmsnorm(const float *x, uint32_t ldx, const void *g, void *h, uint32_t M, uint32_t d, float eps, cudaStream_t st) {
     if (!M) return TGP_OK;
     if (d % 4 || ldx % 4) return TGP_E_INVAL;
-    rmsnorm_kernel<<<M, 256, 0, st>>>(x, ldx, (const bf16 *)g, (bf16 *)h, d, eps);
+    tgp_rmsnorm_kernel<<<M, 256, 0, st>>>(x, ldx, (const bf16 *)g, (bf16 *)h, d, eps);
     LAUNCH_CHECK(1);
     return TGP_OK;
 }
@@ -891,7 +903,7 @@ static void launch_gemv(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, 
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, gemv_kernel<MT, R, U>, 256, 0) != cudaSuccess || blocks_per_sm < 1) blocks_per_sm = 1;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, tgp_wstream_kernel<MT, R, U>, 256, 0) != cudaSuccess || blocks_per_sm < 1) blocks_per_sm = 1;
         if (sms < 1) sms = 148;
     }
     uint32_t need = (n + R * 8 - 1) / (R * 8), full = (uint32_t)(sms * blocks_per_sm);
@@ -904,7 +916,8 @@ static void launch_gemv(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, 
     attr[0].val.programmaticStreamSerializationAllowed = g_gemv_pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, gemv_kernel<MT, R, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
+    cudaLaunchKernelEx(&cfg, tgp_wstream_kernel<MT, R, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
+    tgpk_last_gemm_kernel = "tgp_wstream_kernel";
 }
 
 // Same product for blocks with few rows: one CTA owns ROWS (16, or 8 with the upper half of the MMA tile left empty)
@@ -913,7 +926,7 @@ static void launch_gemv(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, 
 // RPC <= ROWS: rows a CTA owns (the tile's remaining rows re-read its last row and are not stored; a row's sum does not
 // depend on its place in the tile).  14 of 16 turns the 256 CTAs of a 4096-row block into 293, two for every SM.
 template <int NB, int U, int NW, int ROWS, int RPC = ROWS>
-__global__ void __launch_bounds__(NW * 32) gemv_mma_splitk_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+__global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_splitk_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                               uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     constexpr int UL = ROWS == 8 ? 2 * U : U;             // half a tile per load step: twice the steps in flight
     __shared__ float part[NW][NB * 4][32];
@@ -974,10 +987,10 @@ __global__ void __launch_bounds__(NW * 32) gemv_mma_splitk_kernel(const bf16 *__
 // projections): their row groups are walked as one list and a CTA takes RG consecutive groups, whose MMAs share each
 // activation fragment - every CTA reads its K slices of all activation rows from L2, so at 8 or 16 rows per CTA that
 // traffic equals or exceeds the weights' and bounds the kernel; RG row groups divide it by RG.  A group's arithmetic
-// (which warp adds which k, in which order) is that of gemv_mma_splitk_kernel<NB, U, NW, ROWS> whatever RG and the list:
+// (which warp adds which k, in which order) is that of tgp_wstream_mma_splitk_kernel<NB, U, NW, ROWS> whatever RG and the list:
 // same bits as one launch per block.
 template <int NB, int U, int NW, int ROWS, int RG>
-__global__ void __launch_bounds__(NW * 32) gemv_mma_group_kernel(const bf16 *__restrict__ A, const GemvParts p, uint32_t Mrows, uint32_t groups_total,
+__global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_group_kernel(const bf16 *__restrict__ A, const GemvParts p, uint32_t Mrows, uint32_t groups_total,
                                                               uint32_t K, int accumulate, uint32_t rpc) {
     constexpr int UL = ROWS == 8 ? 2 * U : U;             // half a tile per load step: twice the steps in flight
     constexpr int G = RG, SUB = UL / G;                  // SUB load steps of G groups in flight at a time: as many loads as UL of one
@@ -1113,8 +1126,8 @@ static SkinnyPick pick_skinny(uint32_t M, uint32_t n, uint32_t K) {
 template <int NB, int U>
 static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint32_t Mrows, uint32_t K, int acc, cudaStream_t st) {
     static int blocks_per_sm = 0, blocks_per_sm_split = 0;
-    if (!blocks_per_sm && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, gemv_mma_kernel<NB, U>, 256, 0) != cudaSuccess || blocks_per_sm < 1)) blocks_per_sm = 1;
-    if (!blocks_per_sm_split && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm_split, gemv_mma_splitk_kernel<NB, U, 8, 16>, 256, 0) != cudaSuccess || blocks_per_sm_split < 1))
+    if (!blocks_per_sm && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, tgp_wstream_mma_kernel<NB, U>, 256, 0) != cudaSuccess || blocks_per_sm < 1)) blocks_per_sm = 1;
+    if (!blocks_per_sm_split && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm_split, tgp_wstream_mma_splitk_kernel<NB, U, 8, 16>, 256, 0) != cudaSuccess || blocks_per_sm_split < 1))
         blocks_per_sm_split = 1;
     const uint32_t sms = (uint32_t)device_sms();
     uint32_t need = 0, rows_total = 0, rpc = (uint32_t)k.rows;
@@ -1154,32 +1167,33 @@ static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint3
     cfg.numAttrs = 1;
     uint32_t total = 0;
     for (uint32_t s = 0; k.split && s < p.count; ++s) total += p.groups[s];
-    if (!k.split) cudaLaunchKernelEx(&cfg, gemv_mma_kernel<NB, U>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
+    tgpk_last_gemm_kernel = !k.split ? "tgp_wstream_mma_kernel" : p.count > 1 ? "tgp_wstream_mma_group_kernel" : "tgp_wstream_mma_splitk_kernel";
+    if (!k.split) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_kernel<NB, U>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
     else if (p.count > 1) {                               // only few-row blocks are ever grouped: 16 warps, doubled load steps
         if constexpr (NB <= 2 && U == 8) {
-            if (pairs && k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 8, 2>, A, p, Mrows, total, K, acc, rpc);
-            else if (pairs) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 16, 2>, A, p, Mrows, total, K, acc, rpc);
-            else if (k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 8, 1>, A, p, Mrows, total, K, acc, rpc);
-            else cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc, rpc);
+            if (pairs && k.rows == 8) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 8, 2>, A, p, Mrows, total, K, acc, rpc);
+            else if (pairs) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 2>, A, p, Mrows, total, K, acc, rpc);
+            else if (k.rows == 8) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 8, 1>, A, p, Mrows, total, K, acc, rpc);
+            else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc, rpc);
         } else if constexpr (NB == 4 && U == 4) {
-            if (k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 8, 1>, A, p, Mrows, total, K, acc, rpc);
-            else cudaLaunchKernelEx(&cfg, gemv_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc, rpc);
+            if (k.rows == 8) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 8, 1>, A, p, Mrows, total, K, acc, rpc);
+            else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc, rpc);
         }
     }
-    else if (k.nw == 16 && k.rows == 8) cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 8>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
+    else if (k.nw == 16 && k.rows == 8) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_splitk_kernel<NB, U, 16, 8>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
     else if (k.nw == 16) {
         if constexpr (NB == 1 && U == 4) {
             // 33.5 MB blocks at M <= 8, two CTAs per SM: 14 rows per CTA when that gives every SM two
             const uint32_t c14 = (p.n[0] + 13) / 14;
             if (g_gemv_balance && need > sms && c14 <= 2 * sms && c14 > need) {
                 cfg.gridDim = dim3(c14);
-                cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 16, 14>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
+                cudaLaunchKernelEx(&cfg, tgp_wstream_mma_splitk_kernel<NB, U, 16, 16, 14>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
                 return;
             }
         }
-        cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 16, 16>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
+        cudaLaunchKernelEx(&cfg, tgp_wstream_mma_splitk_kernel<NB, U, 16, 16>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
     }
-    else cudaLaunchKernelEx(&cfg, gemv_mma_splitk_kernel<NB, U, 8, 16>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
+    else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_splitk_kernel<NB, U, 8, 16>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
 }
 
 static void launch_skinny_pick(const bf16 *A, const GemvParts &p, const SkinnyPick &k, uint32_t Mrows, uint32_t K, int acc, cudaStream_t st) {
@@ -1195,7 +1209,7 @@ static void launch_gemv_splitk(const bf16 *A, const bf16 *W, float *C, uint32_t 
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, gemv_splitk_kernel<MT, RB, U>, 256, 0) != cudaSuccess || blocks_per_sm < 1) blocks_per_sm = 1;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, tgp_wstream_splitk_kernel<MT, RB, U>, 256, 0) != cudaSuccess || blocks_per_sm < 1) blocks_per_sm = 1;
         if (sms < 1) sms = 148;
     }
     uint32_t need = (n + RB - 1) / RB, full = (uint32_t)(sms * blocks_per_sm);
@@ -1208,7 +1222,8 @@ static void launch_gemv_splitk(const bf16 *A, const bf16 *W, float *C, uint32_t 
     attr[0].val.programmaticStreamSerializationAllowed = g_gemv_pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, gemv_splitk_kernel<MT, RB, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
+    cudaLaunchKernelEx(&cfg, tgp_wstream_splitk_kernel<MT, RB, U>, A, W, C, Mrows, n, K, ldc, col0, acc);
+    tgpk_last_gemm_kernel = "tgp_wstream_splitk_kernel";
 }
 
 // rows per warp: fewer when the block has few rows, so that every SM still gets warps
@@ -1234,7 +1249,7 @@ static void launch_gemv_group(const bf16 *A, const GemvParts &p, uint32_t Mrows,
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, gemv_group_kernel<MT, 8>, 256, 0) != cudaSuccess || blocks_per_sm < 1) blocks_per_sm = 1;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, tgp_wstream_group_kernel<MT, 8>, 256, 0) != cudaSuccess || blocks_per_sm < 1) blocks_per_sm = 1;
         if (sms < 1) sms = 148;
     }
     uint32_t need = (n_total + 7) / 8, full = (uint32_t)(sms * blocks_per_sm);
@@ -1247,11 +1262,12 @@ static void launch_gemv_group(const bf16 *A, const GemvParts &p, uint32_t Mrows,
     attr[0].val.programmaticStreamSerializationAllowed = g_gemv_pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, gemv_group_kernel<MT, 8>, A, p, Mrows, n_total, K, acc);
+    cudaLaunchKernelEx(&cfg, tgp_wstream_group_kernel<MT, 8>, A, p, Mrows, n_total, K, acc);
+    tgpk_last_gemm_kernel = "tgp_wstream_group_kernel";
 }
 
 // Which products may share a launch: those with the same non-zero key.  A key names the kernel a block takes on its own
-// (M <= 2: gemv_kernel<MT, 1, 8>; 3 <= M <= 32: one instance of the split-K skinny kernel); blocks of so many rows that
+// (M <= 2: tgp_wstream_kernel<MT, 1, 8>; 3 <= M <= 32: one instance of the split-K skinny kernel); blocks of so many rows that
 // they fill the machine alone, and the shapes served by other kernels, have key 0 and are launched alone.
 uint32_t tgpk_gemm_group_key(uint32_t M, uint32_t n, uint32_t K) {
     if (!g_gemm_group || !M || !n || !K || K % 8) return 0;
@@ -1332,7 +1348,8 @@ int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, ui
         return tgpk_gemm_tc(A, W, C, M, n, K, ldc, col0, accumulate, st);
     } else {
         dim3 grid((n + 63) / 64, (M + 63) / 64);
-        gemm_simt_kernel<<<grid, 256, 0, st>>>(a, w, C, M, n, K, ldc, col0, accumulate);
+        tgp_matmul_simt_kernel<<<grid, 256, 0, st>>>(a, w, C, M, n, K, ldc, col0, accumulate);
+        tgpk_last_gemm_kernel = "tgp_matmul_simt_kernel";
     }
     LAUNCH_CHECK(1);
     return TGP_OK;
@@ -1342,7 +1359,7 @@ int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb,
                  const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0, cudaStream_t st) {
     if (!B || !q_len) return TGP_OK;
     RopeArgs a{q32, k32, v32, (bf16 *)qb, cos_t, sin_t, c->Hq, c->Hkv, c->Dh, c->TK, q_len, pos0, tiles};
-    rope_kv_kernel<<<B * q_len, 256, 0, st>>>(a);
+    tgp_rope_kv_kernel<<<B * q_len, 256, 0, st>>>(a);
     LAUNCH_CHECK(1);
     return TGP_OK;
 }
@@ -1369,16 +1386,16 @@ int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *
         }
         const size_t sm = (size_t)(G * c->Dh + G * split * (c->Dh + 2)) * sizeof(float);
 #define TGP_DECODE_GROUP(DH_) do { \
-            if (G == 1) attn_decode_group_kernel<DH_, 1><<<grid, 32 * split, sm, st>>>(a, split); \
-            else if (G == 2) attn_decode_group_kernel<DH_, 2><<<grid, 32 * split, sm, st>>>(a, split); \
-            else if (G == 4) attn_decode_group_kernel<DH_, 4><<<grid, 32 * split, sm, st>>>(a, split); \
-            else attn_decode_group_kernel<DH_, 8><<<grid, 32 * split, sm, st>>>(a, split); } while (0)
+            if (G == 1) tgp_attn_decode_group_kernel<DH_, 1><<<grid, 32 * split, sm, st>>>(a, split); \
+            else if (G == 2) tgp_attn_decode_group_kernel<DH_, 2><<<grid, 32 * split, sm, st>>>(a, split); \
+            else if (G == 4) tgp_attn_decode_group_kernel<DH_, 4><<<grid, 32 * split, sm, st>>>(a, split); \
+            else tgp_attn_decode_group_kernel<DH_, 8><<<grid, 32 * split, sm, st>>>(a, split); } while (0)
         if (c->Dh == 64) {
-            if (grouped) TGP_DECODE_GROUP(64); else attn_decode_partial_kernel<64><<<grid, 32 * G * split, sm, st>>>(a, split);
-            attn_decode_merge_kernel<64><<<dim3(c->Hq, B), 64, 0, st>>>(a);
+            if (grouped) TGP_DECODE_GROUP(64); else tgp_attn_decode_partial_kernel<64><<<grid, 32 * G * split, sm, st>>>(a, split);
+            tgp_attn_decode_merge_kernel<64><<<dim3(c->Hq, B), 64, 0, st>>>(a);
         } else {
-            if (grouped) TGP_DECODE_GROUP(128); else attn_decode_partial_kernel<128><<<grid, 32 * G * split, sm, st>>>(a, split);
-            attn_decode_merge_kernel<128><<<dim3(c->Hq, B), 128, 0, st>>>(a);
+            if (grouped) TGP_DECODE_GROUP(128); else tgp_attn_decode_partial_kernel<128><<<grid, 32 * G * split, sm, st>>>(a, split);
+            tgp_attn_decode_merge_kernel<128><<<dim3(c->Hq, B), 128, 0, st>>>(a);
         }
 #undef TGP_DECODE_GROUP
         tgpk_launches += 1;
@@ -1389,8 +1406,8 @@ int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *
         return tgpk_attn_prefill_tc(qb, tiles, ob, c, B, q_len, pos0, st);
     } else {
         dim3 grid((q_len + 3) / 4, c->Hq, B);
-        if (c->Dh == 64) attn_rows_kernel<64><<<grid, 128, 0, st>>>(a);
-        else attn_rows_kernel<128><<<grid, 128, 0, st>>>(a);
+        if (c->Dh == 64) tgp_attn_rows_kernel<64><<<grid, 128, 0, st>>>(a);
+        else tgp_attn_rows_kernel<128><<<grid, 128, 0, st>>>(a);
     }
     LAUNCH_CHECK(1);
     return TGP_OK;
@@ -1401,14 +1418,14 @@ int tgpk_swiglu(const float *g, const float *u, void *ab, uint64_t n, cudaStream
     if (n % 4) return TGP_E_INVAL;
     uint64_t n4 = n / 4;
     uint32_t blocks = (uint32_t)((n4 + 255) / 256 < 148 * 16 ? (n4 + 255) / 256 : 148 * 16);
-    swiglu_kernel<<<blocks, 256, 0, st>>>((const float4 *)g, (const float4 *)u, (__nv_bfloat162 *)ab, n4);
+    tgp_swiglu_kernel<<<blocks, 256, 0, st>>>((const float4 *)g, (const float4 *)u, (__nv_bfloat162 *)ab, n4);
     LAUNCH_CHECK(1);
     return TGP_OK;
 }
 
 int tgpk_argmax(const float *logits, int32_t *out, uint32_t B, uint32_t V, cudaStream_t st) {
     if (!B) return TGP_OK;
-    argmax_kernel<<<B, 1024, 0, st>>>(logits, out, V);
+    tgp_argmax_kernel<<<B, 1024, 0, st>>>(logits, out, V);
     LAUNCH_CHECK(1);
     return TGP_OK;
 }
@@ -1423,9 +1440,27 @@ static int fill_tiles(TgpTilePtrs &t, void *const *k, void *const *v, uint32_t n
 
 extern "C" {
 
-int tgp_k_embed(const void *table, const int32_t *tok_dev, float *x_dev, uint32_t M, uint32_t d, void *stream) {
+int tgp_k_embed(const void *table, const int32_t *tok_dev, float *x_dev, uint32_t M, uint32_t d, uint32_t V, void *stream) {
     if (!table || !tok_dev || !x_dev) return TGP_E_INVAL;
-    return tgpk_embed(table, tok_dev, x_dev, M, d, (cudaStream_t)stream);
+    return tgpk_embed(table, tok_dev, x_dev, M, d, V, (cudaStream_t)stream);
+}
+
+int tgp_k_embed_status(int *bad, uint32_t *row, int32_t *token) {
+    if (!bad) return TGP_E_INVAL;
+    unsigned long long w = 0;
+    if (cudaMemcpyFromSymbol(&w, g_embed_error, sizeof(w)) != cudaSuccess) return TGP_E_CUDA;
+    *bad = (w >> 63) ? 1 : 0;
+    if (row) *row = (uint32_t)((w >> 32) & 0x7fffffffu);
+    if (token) *token = (int32_t)(uint32_t)w;
+    return TGP_OK;
+}
+
+int tgp_k_status_clear(void) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return TGP_E_CUDA;
+    const unsigned long long z = 0;
+    if (cudaMemcpyToSymbol(g_embed_error, &z, sizeof(z)) != cudaSuccess) return TGP_E_CUDA;
+    int rc = tgpk_gemm_status_clear();
+    return rc ? rc : tgpk_attn_status_clear();
 }
 
 int tgp_k_rmsnorm(const float *x_dev, uint32_t ldx, const void *g_dev, void *h_dev, uint32_t M, uint32_t d, float eps, void *stream) {
@@ -1449,6 +1484,15 @@ int tgp_k_gemm_group(const void *A_dev, uint32_t count, const void *const *W_dev
 int tgp_k_gemm_group_key(uint32_t M, uint32_t n, uint32_t K, uint32_t *key) {
     if (!key) return TGP_E_INVAL;
     *key = tgpk_gemm_group_key(M, n, K);
+    return TGP_OK;
+}
+
+int tgp_k_gemm_last_kernel(char *name, uint32_t capacity) {
+    if (!name || !capacity) return TGP_E_INVAL;
+    const char *k = tgpk_last_gemm_kernel;
+    uint32_t i = 0;
+    for (; k[i] && i + 1 < capacity; ++i) name[i] = k[i];
+    name[i] = 0;
     return TGP_OK;
 }
 

@@ -8,7 +8,8 @@
 
 struct TgpTilePtrs { void *k[TGP_MAX_TILES]; void *v[TGP_MAX_TILES]; };
 
-int tgpk_embed(const void *table, const int32_t *tok, float *x, uint32_t M, uint32_t d, cudaStream_t st);
+// rows of token ids outside [0, V) are written as zeros and recorded (tgp_k_embed_status)
+int tgpk_embed(const void *table, const int32_t *tok, float *x, uint32_t M, uint32_t d, uint32_t V, cudaStream_t st);
 int tgpk_rmsnorm(const float *x, uint32_t ldx, const void *g, void *h, uint32_t M, uint32_t d, float eps, cudaStream_t st);
 int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st);
 // products over the same activations A [M, K]: C[s][m, j] (=|+=) sum_k A[m, k] * W[s][j, k].  Blocks with the same non-zero
@@ -36,3 +37,8 @@ int tgpk_scatter_add(float *x, const float *y, const int32_t *rows, const float 
 int tgpk_argmax(const float *logits, int32_t *out, uint32_t B, uint32_t V, cudaStream_t st);
 // cos/sin tables [max_len, Dh/2] fp32 (angle = pos * base^(-2i/Dh), evaluated in double) written to device memory
 int tgp_rope_tables_upload(uint32_t Dh, uint32_t max_len, float base, float *cos_dev, float *sin_dev);
+// reset of the tensor-core kernels' error words (tgp_gemm_sm100.cu, tgp_attn_sm100.cu)
+int tgpk_gemm_status_clear();
+int tgpk_attn_status_clear();
+// name of the kernel the last tgpk_gemm / tgpk_gemm_group / tgpk_gemm_tc call of this thread launched
+extern thread_local const char *tgpk_last_gemm_kernel;

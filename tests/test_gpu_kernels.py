@@ -137,6 +137,48 @@ def test_tensor_core_gemm_with_the_weights_as_the_128_row_operand(M, n, K, acc):
     assert np.array_equal(got[:, :col0], c0[:, :col0]) and np.array_equal(got[:, col0 + n:], c0[:, col0 + n:])
 
 
+# (M, K, n, residual): the weight-block products of the prefill steps the benchmark times - M = B * S of the 8B shape (8 x 1024),
+# the MoE shape (32 x 512) and the 70B shape (16 x 2048); K = d or FFN; n = rows of one 32 MiB sub-range block of that matrix
+REAL_PREFILL = [(8192, 4096, 4096, 0), (8192, 14336, 1152, 1), (16384, 4096, 4096, 0), (32768, 8192, 2048, 0), (32768, 28672, 512, 1)]
+
+
+@pytest.mark.parametrize("M,K,n,acc", REAL_PREFILL)
+def test_gemm_at_the_real_prefill_shapes_sampled_rows_against_the_oracle(M, K, n, acc):
+    """Full-size prefill products in the launch configuration the benchmark times (automatic kernel choice: the paired
+    tcgen05 kernel).  A full CPU product would take minutes, and an output row depends on one activation row only, so
+    the oracle recomputes 64 sampled rows - first, last, the rows around every 128- and 256-row tile edge it can hit,
+    and seeded random ones - from the same bf16 inputs, in double.  The rows in between are covered by a checksum
+    property that holds at any size: the column sums of C equal (column sums of A) . W^T."""
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(M * 31 + K)
+    A = torch.randn((M, K), device=DEV, generator=gen).bfloat16()
+    W = (torch.randn((n, K), device=DEV, generator=gen) * 0.02).bfloat16()
+    c0 = (torch.randn((M, n), device=DEV, generator=gen) * 0.5).float() if acc else None
+    Cd = c0.clone() if acc else torch.empty((M, n), dtype=torch.float32, device=DEV)
+    tb.k_gemm(A, W, Cd, M, n, K, n, 0, acc)
+    torch.cuda.synchronize()
+    assert tb.k_gemm_status() == 0
+    rng = np.random.default_rng(M + K)
+    rows = sorted(set([0, 1, 127, 128, 255, 256, M // 2 - 1, M // 2, M - 257, M - 256, M - 129, M - 128, M - 2, M - 1] + rng.integers(0, M, 50).tolist()))[:64]
+    ridx = torch.tensor(rows, device=DEV)
+    a_rows = si.bf16_bits_to_f32(A[ridx].view(torch.int16).cpu().numpy().view(np.uint16))
+    w_bits = W.view(torch.int16).cpu().numpy().view(np.uint16)
+    want = oracle().linear(a_rows, si.bf16_bits_to_f32(w_bits).astype(np.float64)).astype(np.float64)
+    if acc:
+        want = want + c0[ridx].cpu().numpy().astype(np.float64)
+    got = Cd[ridx].cpu().numpy().astype(np.float64)
+    scale = np.abs(want).max()
+    assert np.abs(got - want).max() < 2e-5 * scale + 1e-7, (np.abs(got - want).max(), scale)
+    # every row, through a property: sum_m C[m, j] = (sum_m A[m, :]) . W[j, :]  (+ sum_m C0[m, j]), in double
+    colsum = Cd.double().sum(dim=0).cpu().numpy()
+    asum = A.double().sum(dim=0).cpu().numpy()
+    ref = si.bf16_bits_to_f32(w_bits).astype(np.float64) @ asum + (c0.double().sum(dim=0).cpu().numpy() if acc else 0.0)
+    # fp32 accumulation error of one output element is ~1e-6 of its scale; M of them add up at random
+    assert np.abs(colsum - ref).max() < 2e-5 * scale * np.sqrt(M) + 1e-6, (np.abs(colsum - ref).max(), scale)
+    # and no element is non-finite or left unwritten
+    assert bool(torch.isfinite(Cd).all())
+
+
 def test_gemm_rejects_bad_arguments_and_accepts_empty():
     A = torch.zeros(8, 16, dtype=torch.bfloat16, device=DEV)
     Cd = torch.zeros(8, 8, dtype=torch.float32, device=DEV)
@@ -154,9 +196,10 @@ def test_rmsnorm_and_embed(M, d):
     tab_bits = rnd_bits(3, V * d).reshape(V, d)
     tok = (np.arange(M, dtype=np.int32) * 37 + 5) % V
     x = torch.empty(M, d, dtype=torch.float32, device=DEV)
-    tb.k_embed(bf16_dev(tab_bits), torch.from_numpy(tok).to(DEV), x, M, d)
+    tb.k_embed(bf16_dev(tab_bits), torch.from_numpy(tok).to(DEV), x, M, d, V)
     torch.cuda.synchronize()
     assert np.array_equal(x.cpu().numpy(), si.bf16_bits_to_f32(tab_bits)[tok])
+    assert tb.k_embed_status()[0] == 0
     xin = (np.random.default_rng(d).standard_normal((M, d)) * 3).astype(np.float32)
     g_bits = si.f32_to_bf16_bits(1.0 + 0.1 * np.random.default_rng(1).standard_normal(d).astype(np.float32))
     h = torch.empty(M, d, dtype=torch.bfloat16, device=DEV)
@@ -165,6 +208,38 @@ def test_rmsnorm_and_embed(M, d):
     o = oracle()
     want = o.rmsnorm(xin, si.bf16_bits_to_f32(g_bits).astype(np.float64))
     bf16_close(h.float().cpu().numpy(), want)
+
+
+def test_embed_zeroes_rows_of_tokens_outside_the_vocabulary_and_records_the_first():
+    """A token id outside [0, V) must never index the table (in an oversubscribed run the table may be mapped host
+    memory): its row is zeros, the others are gathered as usual, and the error word names the row and the id."""
+    V, d, M = 50, 64, 6
+    tab_bits = rnd_bits(11, V * d).reshape(V, d)
+    tok = np.array([3, V, 7, -1, 49, 2 ** 31 - 1], dtype=np.int32)
+    x = torch.full((M, d), 7.0, dtype=torch.float32, device=DEV)
+    tb.k_status_clear()
+    tb.k_embed(bf16_dev(tab_bits), torch.from_numpy(tok).to(DEV), x, M, d, V)
+    torch.cuda.synchronize()
+    got = x.cpu().numpy()
+    ok = (tok >= 0) & (tok < V)
+    assert np.array_equal(got[ok], si.bf16_bits_to_f32(tab_bits)[tok[ok]])
+    assert not got[~ok].any()
+    bad, row, token = tb.k_embed_status()
+    assert bad == 1 and row in (1, 3, 5) and token == int(tok[row])
+    tb.k_status_clear()
+    assert tb.k_embed_status()[0] == 0
+
+
+def test_argmax_of_a_row_of_nans_is_a_legal_token():
+    V = 5000
+    lg = np.full((3, V), np.nan, dtype=np.float32)
+    lg[1] = -np.inf
+    lg[2, 4000] = 1.0
+    am = torch.full((3,), -7, dtype=torch.int32, device=DEV)
+    tb.k_argmax(torch.from_numpy(lg).to(DEV), am, 3, V)
+    torch.cuda.synchronize()
+    got = am.cpu().numpy()
+    assert got[0] == 0 and got[1] == 0 and 0 <= got[2] < V
 
 
 def make_tiles(cfg, B):
@@ -449,8 +524,8 @@ def test_grouped_products_equal_single_products_and_oracle(M, ns, K, grouped, ac
 
 @pytest.mark.parametrize("M,n,K", [(3, 100, 64), (8, 4096, 4096), (8, 1030, 512), (13, 77, 128), (16, 260, 1024), (17, 64, 96), (24, 2049, 2048),
                                    (32, 4100, 8192), (5, 16, 32),
-                                   # few rows and long K: K split over a thread-block cluster of 8, 4, 2 CTAs (ragged rows, K that leaves
-                                   # the last ranks without a chunk)
+                                   # few rows and long K: the split-K kernel (K divided among the warps of a CTA; ragged rows, K that
+                                   # leaves the last warps without a chunk)
                                    (8, 1152, 14336), (5, 650, 14368), (16, 1024, 4096), (9, 24, 2080), (8, 16, 16384)])
 @pytest.mark.parametrize("accumulate", [0, 1])
 def test_skinny_tensor_core_gemv_matches_oracle_and_cuda_core_path(M, n, K, accumulate):

@@ -203,6 +203,14 @@ def test_config_2_prefill_and_first_decode_steps_match_oracle():
     r = Runner(s, cfg.B * cfg.S)
     got, _ = r.generate(prompt, n_dec, forced=toks)
     fl_max, fl_rel = precision_floor(2)
+    worst_abs = max(float(np.abs(a - b).max()) for a, b in zip(got, ref))
+    worst_rel = max(float(np.abs(a - b).mean() / np.abs(b).mean()) for a, b in zip(got, ref))
+    print(f"config 2 free-running logits error: max abs {worst_abs:.3e} (oracle float32-vs-float64 floor {fl_max:.3e}, stated {MAX_ABS:.0e}), "
+          f"mean relative {worst_rel:.3e} (floor {fl_rel:.3e}, stated {MEAN_REL:.0e})")
+    import os
+    os.makedirs("gpurun_out", exist_ok=True)
+    with open(os.path.join("gpurun_out", "free_running_error_config2.txt"), "w") as f:
+        f.write(f"max_abs {worst_abs:.6e} floor_max_abs {fl_max:.6e} mean_rel {worst_rel:.6e} floor_mean_rel {fl_rel:.6e}\n")
     check_logits(got, ref, max(MAX_ABS, 2 * fl_max), max(MEAN_REL, 2 * fl_rel))
     assert all(np.argmax(a[0]) == np.argmax(b[0]) or abs(np.sort(b[0])[-1] - np.sort(b[0])[-2]) < 2 * fl_max for a, b in zip(got, ref))
     s.close()
@@ -238,8 +246,7 @@ def test_managed_variants_give_the_same_bits_as_the_explicit_ring():
                 # the prefetcher asks for whole 1 MiB segments: at least every touched byte, at most the pool per op
                 r.reset()
                 st = r.step(tb.PREFILL, np.ascontiguousarray(prompt, dtype=np.int32), cfg.S, want_stats=True)
-                from bench import parse_trace
-                acc = [a for o in parse_trace(sm.ctx.trace_export()) if o[0] == 0 for a in o[6]]
+                acc = [a for o in sm.ctx.trace_ops() if o[0] == 0 for a in o[6]]
                 whole = sum(t.size for t in lay.tensors if t.kind not in (si.K_EMBED, si.K_KT, si.K_VT))      # read whole by a prefill
                 assert st.zc_bytes == 0 and st.d2h_bytes == 0
                 assert 0.9 * whole <= st.h2d_bytes <= sum(lay.tensors[a[0]].size + (2 << 20) for a in acc)
@@ -387,32 +394,97 @@ def test_llama_8b_widths_at_two_layers_lockstep_parity():
 
 
 def test_mixtral_widths_at_one_layer_match_oracle_batch_of_eight():
-    """Full widths of the Mixtral shape (8 experts of 14336, top-2) at one layer, batch 8: the expert products run at
-    the handful of tokens each expert receives (skinny tensor-core GEMV on blocks of few rows), planned from a profile pass."""
+    """Full widths of the Mixtral shape (8 experts of 14336, top-2) at one layer, batch 8, free-running: the expert
+    products run at the handful of tokens each expert receives (skinny tensor-core GEMV on blocks of few rows), planned
+    from a profile pass.  Routing is an fp32 comparison of router logits whose inputs differ between the two sides by
+    bf16 rounding flips, so a token whose second and third logits are within FRAGILE of each other may route either
+    way: every difference in the routed-token counts must be explained by such tokens, and the logits of every
+    sequence whose deciding (last-position) token is not fragile are compared unconditionally - at one layer a token's
+    routing reaches no other position's logits."""
+    FRAGILE = 2e-2
     cfg = replace(si.CONFIGS[5], L=1, B=8, S=16, T=2, budget_rule="half_w")
     lay = si.build_layout(cfg)
     bias = si.router_bias(cfg)
     pool = pinned_pool(lay.pool_bytes)
     si.fill_pool_torch(lay, pool, device="cuda:0")
     om = forward.OracleModel(cfg, _weights_from_pool(lay, pool), bias, dtype=np.float32)
+    Wr = om.w[(si.K_ROUTER, 0, -1)].astype(np.float64)
+    fragile = []                                                  # per step: bool [B, q]
+
+    def hook(name, layer, pre, out):
+        if name == "h2":
+            rl = np.sort(out.reshape(-1, cfg.d).astype(np.float64) @ Wr.T + np.asarray(bias[layer], dtype=np.float64), axis=-1)
+            fragile.append(((rl[:, -2] - rl[:, -3]) < FRAGILE).reshape(out.shape[0], out.shape[1]))
+        return out
+
+    om.hook = hook
     prompt = si.prompt_tokens(cfg)
     ref, toks = om.generate(prompt, cfg.T)
+    om.hook = None
     want_counts = np.array([[c.tolist() for c in step] for step in om.expert_counts], dtype=np.uint32)
     s = Session(lay, MACHINE, pool_base=pool.data_ptr(), pool_flags=tb.POOL_PINNED, router_bias=bias)
     s.plan(expert_counts=np.ones_like(want_counts))
     r = Runner(s, cfg.B * cfg.S)
     got, mism = _run_steps(r, cfg, prompt, toks, cfg.T)
     counts = s.ctx.expert_counts(cfg.L, cfg.E)
-    # routing decisions are fp32 comparisons of router logits: a near-tie may fall the other way on a few tokens
-    assert np.abs(counts.astype(np.int64) - want_counts.astype(np.int64)).sum() <= 4
+    for k in range(1 + cfg.T):
+        moved = int(np.abs(counts[k].astype(np.int64) - want_counts[k].astype(np.int64)).sum())
+        assert moved <= 2 * int(fragile[k].sum()), (k, moved, int(fragile[k].sum()))
     s.plan(expert_counts=counts)
     got2, mism2 = _run_steps(r, cfg, prompt, toks, cfg.T)
     assert sum(mism2) == 0
     for a, b in zip(got, got2):
         assert np.array_equal(a, b)                                           # profile pass and planned run: same bits
-    if np.array_equal(counts, want_counts):
-        check_logits(got2, ref)
+    compared = 0
+    for k in range(1 + cfg.T):
+        keep = ~fragile[k][:, -1]                                             # sequences whose last position routes robustly
+        compared += int(keep.sum())
+        check_logits([got2[k][keep]], [ref[k][keep]])
+    assert compared >= (1 + cfg.T) * cfg.B * 3 // 4, compared
     s.close()
+
+
+def test_mixtral_widths_at_three_layers_lockstep_parity():
+    """Full widths of the Mixtral shape at three layers, batch 4, prefill of 4 x 24 tokens and two decode steps, half
+    the weights resident, in lockstep: routing counts equal to the oracle's at every step and layer, every rounding
+    point a legal rounding, logits within the stated tolerance."""
+    cfg = replace(si.CONFIGS[5], L=3, B=4, S=24, T=2, budget_rule="half_w")
+    lay = si.build_layout(cfg)
+    bias = si.router_bias(cfg)
+    pool = pinned_pool(lay.pool_bytes)
+    si.fill_pool_torch(lay, pool, device="cuda:0")
+    worst, flips = _lockstep(cfg, lay, pool, _weights_from_pool(lay, pool), cfg.T, np.float32, bias=bias)
+    assert worst < 5e-3
+    assert all(v < 0.02 for k, v in flips.items() if k != "o") and flips["o"] < 0.5
+    assert tb.k_attn_status() == 0 and tb.k_gemm_status() == 0
+
+
+def test_llama_70b_widths_at_two_layers_lockstep_parity():
+    """Full widths of the 70B shape (d 8192, 64 query / 8 KV heads, FFN 28672, vocabulary 128256) at two layers: prefill
+    of 2 x 136 tokens and two decode steps at batch 2, half the weights resident, in lockstep."""
+    cfg = replace(si.CONFIGS[4], L=2, B=2, S=136, T=2, budget_rule="half_w")
+    lay = si.build_layout(cfg)
+    pool = pinned_pool(lay.pool_bytes)
+    si.fill_pool_torch(lay, pool, device="cuda:0")
+    worst, flips = _lockstep(cfg, lay, pool, _weights_from_pool(lay, pool), cfg.T, np.float32)
+    assert worst < 5e-3
+    assert all(v < 0.02 for k, v in flips.items() if k != "o") and flips["o"] < 0.5
+    assert tb.k_attn_status() == 0 and tb.k_gemm_status() == 0
+
+
+def test_llama_8b_full_depth_lockstep_parity_reduced_tokens():
+    """The 8B configuration at its full depth (all 32 layers), full widths and its 8 GiB budget (2x oversubscribed), with
+    reduced tokens - one sequence, prompt of 16, four decode steps - because a full-size CPU forward pass would take
+    hours.  Lockstep: every rounding point of all 32 layers element by element, logits within the stated tolerance."""
+    cfg = replace(si.CONFIGS[3], B=1, S=16, T=4)
+    lay = si.build_layout(cfg)
+    assert lay.budget == 8 << 30 and cfg.L == 32 and lay.pool_bytes > 2 * lay.budget * 0.95
+    pool = pinned_pool(lay.pool_bytes)
+    si.fill_pool_torch(lay, pool, device="cuda:0")
+    worst, flips = _lockstep(cfg, lay, pool, _weights_from_pool(lay, pool), cfg.T, np.float32)
+    assert worst < 5e-3
+    assert all(v < 0.02 for k, v in flips.items() if k != "o") and flips["o"] < 0.5
+    assert tb.k_attn_status() == 0 and tb.k_gemm_status() == 0
 
 
 def test_layer_aliased_host_pool_runs_like_a_pool_with_repeated_layers():
@@ -482,20 +554,31 @@ def _bf16_ulp(x):
     return 2.0 ** (np.floor(np.log2(ax)) - 7)
 
 
-def _lockstep(cfg, lay, pool, W, n_dec, dtype):
+ROUTER_MARGIN = 1e-4      # a token whose second and third router logits are closer than this could route either way
+
+
+def _lockstep(cfg, lay, pool, W, n_dec, dtype, bias=None):
     """Runs GPU and oracle step by step.  At every bf16 rounding point the oracle is handed the GPU's tensor, checks
     that each element is a legal rounding of the oracle's own pre-rounding value (|gpu - pre| <= ulp/2 plus the
     summation-order slack of that op) and continues from the GPU's codes, so a flipped rounding cannot cascade.
+    Mixture of experts (bias given): both routers then see the same bf16 inputs, so the routed-token counts of every
+    step and layer must be equal - after checking, as a fact about the seeded inputs, that no token's second and third
+    router logits are within ROUTER_MARGIN of each other (fp32 summation order moves a logit by ~1e-6).
     Returns worst logit error and the fraction of roundings that differ from the oracle's, per kind."""
-    from bench import parse_trace
-    s = Session(lay, MACHINE, pool_base=pool.data_ptr(), pool_flags=tb.POOL_PINNED)
-    s.plan(T=n_dec)
-    ops = parse_trace(s.ctx.trace_export())
+    s = Session(lay, MACHINE, pool_base=pool.data_ptr(), pool_flags=tb.POOL_PINNED, router_bias=bias)
+    if cfg.E:
+        s.plan(T=n_dec, expert_counts=np.ones((1 + n_dec, cfg.L, cfg.E), dtype=np.uint32))     # every expert traced: nothing falls back
+    else:
+        s.plan(T=n_dec)
+    ops = s.ctx.trace_ops()
     r = Runner(s, cfg.B * cfg.S)
     qd, F, d = cfg.Hq * cfg.Dh, cfg.F, cfg.d
     per_layer = cfg.B * cfg.S * (2 * d + 2 * qd + F) * 2 + 2 * cfg.n_tiles * cfg.B * cfg.Hkv * cfg.TK * cfg.Dh * 2 + 16 * 256
     tap = torch.empty(per_layer * cfg.L + (1 << 20), dtype=torch.uint8, device="cuda:0")
-    om = forward.OracleModel(cfg, W, dtype=dtype)
+    om = forward.OracleModel(cfg, W, bias, dtype=dtype)
+    W = None                                               # the oracle holds its own converted copy
+    Wr = {l: om.w[(si.K_ROUTER, l, -1)].astype(np.float64) for l in range(cfg.L)} if cfg.E else {}
+    margins = []
     # slack per rounding point, relative to |pre| + mean|pre|: fp32 summation order and libm vs device exp.  The normed
     # states sit behind the residual stream, which sums tensor-core products of K up to 8192 per layer (their fp32
     # accumulation is not round-to-nearest: ~5e-5 typical, 3e-4 covers the tail of 1e6 elements); the attention output
@@ -549,11 +632,18 @@ def _lockstep(cfg, lay, pool, W, n_dec, dtype):
             assert not bad.any(), (name, layer, int(bad.sum()), float(np.abs(g - pre)[bad].max()))
             flips[name][0] += int((g != out).sum())
             flips[name][1] += g.size
+            if name == "h2" and cfg.E:                     # the router's input: how far is every token from a routing tie?
+                rl = np.sort(g.reshape(-1, cfg.d).astype(np.float64) @ Wr[layer].T + np.asarray(bias[layer], dtype=np.float64), axis=-1)
+                margins.append(float((rl[:, -cfg.topk] - rl[:, -cfg.topk - 1]).min()))
             return g
 
         om.hook = hook
         ref = om.step(tok, pos0)
         om.hook = None
+        if cfg.E:
+            assert min(margins) > ROUTER_MARGIN, ("seeded inputs put a token on a routing near-tie: pick another seed", min(margins))
+            want_counts = np.array([c.tolist() for c in om.expert_counts[-1]], dtype=np.uint32)
+            assert np.array_equal(s.ctx.expert_counts(cfg.L, cfg.E)[step], want_counts), step
         dev = r.logits.cpu().numpy()
         err = np.abs(dev - ref)
         assert err.max() < MAX_ABS and err.mean() / np.abs(ref).mean() < MEAN_REL, (step, err.max())

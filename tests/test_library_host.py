@@ -230,6 +230,28 @@ def test_model_bind_rejects_bad_shapes_and_roles():
     s.close()
 
 
+def test_step_refuses_host_tokens_outside_the_vocabulary_before_touching_a_device():
+    """A host token id outside [0, V) would send the embedding gather past its table; tgp_step() must refuse it at the
+    boundary (no GPU involved: the check comes before the engine is looked at), and an op whose tensor has no model role
+    must be a mismatch code, not a crash."""
+    lay = si.build_layout(si.CONFIGS[1])
+    s = Session(lay, MACHINE)
+    s.plan(T=1)
+    cfg = lay.cfg
+    dummy = np.zeros(16, dtype=np.float32)                      # stands for the logits pointer; never written without a workspace
+    for bad in (-1, cfg.V, 2 ** 31 - 1):
+        tok = np.zeros((cfg.B, cfg.S), dtype=np.int32)
+        tok[0, 5] = bad
+        with pytest.raises(tb.TgpError) as ei:
+            s.ctx.step(tb.PREFILL, tok, cfg.B, cfg.S, dummy, None, None, None)
+        assert ei.value.code == tb.E_INVAL and "vocabulary" in str(ei.value)
+    ok = np.full((cfg.B, cfg.S), cfg.V - 1, dtype=np.int32)
+    with pytest.raises(tb.TgpError) as ei:
+        s.ctx.step(tb.PREFILL, ok, cfg.B, cfg.S, dummy, None, None, None)
+    assert ei.value.code == tb.E_STATE                          # legal tokens get as far as "no workspace bound"
+    s.close()
+
+
 def test_replan_from_a_timing_log_is_bit_exact_and_changes_classes():
     """Runtime monitor: the same integer log of kernel times fed to both planners gives the same schedule; an op whose
     kernel ran longer than its bytes take on the link stops being link-bound, and its tensors lose their pin score."""

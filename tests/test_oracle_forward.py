@@ -35,8 +35,12 @@ def s_bf16(x):
     return struct.unpack("<f", struct.pack("<I", u))[0]
 
 
-def scalar_forward(cfg, W, tokens_b):
-    """One sequence, prefill of all its tokens; returns logits for every position (lists of python floats)."""
+def scalar_forward(cfg, W, tokens_b, bias=None, routed=None):
+    """One sequence, prefill of all its tokens; returns logits for every position (lists of python floats).
+    With cfg.E > 0 the FFN is the mixture of experts: router logits = h2 . Wr + bias in fp32, the two largest (tie ->
+    lower id), gates = softmax over those two logits only, each chosen expert's SwiGLU FFN scaled by its gate after the
+    down projection (fp32) and added to the residual stream in ascending expert id.  routed (a list) receives the
+    (layer, position, [(expert, gate)]) choices."""
     f = lambda k, l=-1, e=-1: si.bf16_bits_to_f32(W[(k, l, e)]).astype(np.float64).tolist()
     S = len(tokens_b)
     half = cfg.Dh // 2
@@ -79,10 +83,26 @@ def scalar_forward(cfg, W, tokens_b):
             att = lin(o, f(si.K_WO, l))
             x[p] = [s_f32(a + b) for a, b in zip(x[p], att)]
             h2 = rms(x[p], f(si.K_G2, l)[0])
-            gt, up = lin(h2, f(si.K_WG, l)), lin(h2, f(si.K_WU, l))
-            a = [s_bf16(s_f32(gv / (1.0 + math.exp(-gv)) * uv)) for gv, uv in zip(gt, up)]
-            dn = lin(a, f(si.K_WD, l))
-            x[p] = [s_f32(a_ + b_) for a_, b_ in zip(x[p], dn)]
+
+            def ffn(e):
+                gt, up = lin(h2, f(si.K_WG, l, e)), lin(h2, f(si.K_WU, l, e))
+                a = [s_bf16(s_f32(gv / (1.0 + math.exp(-gv)) * uv)) for gv, uv in zip(gt, up)]
+                return lin(a, f(si.K_WD, l, e))
+
+            if not cfg.E:
+                x[p] = [s_f32(a_ + b_) for a_, b_ in zip(x[p], ffn(-1))]
+                continue
+            rl = [s_f32(z + float(bias[l][e])) for e, z in enumerate(lin(h2, f(si.K_ROUTER, l)))]
+            first = max(range(cfg.E), key=lambda e: (rl[e], -e))                       # largest logit, lower id on a tie
+            second = max((e for e in range(cfg.E) if e != first), key=lambda e: (rl[e], -e))
+            mx = max(rl[first], rl[second])
+            w1, w2 = math.exp(rl[first] - mx), math.exp(rl[second] - mx)
+            gate = {first: s_f32(w1 / (w1 + w2)), second: s_f32(w2 / (w1 + w2))}
+            if routed is not None:
+                routed.append((l, p, sorted(gate.items())))
+            for e in sorted(gate):                                                     # ascending expert id
+                y = ffn(e)
+                x[p] = [s_f32(a_ + s_f32(gate[e] * b_)) for a_, b_ in zip(x[p], y)]
     return [lin(rms(x[p], f(si.K_GF)[0]), f(si.K_LM)) for p in range(S)]
 
 
@@ -216,6 +236,97 @@ def test_moe_top2_routing_counts_and_tie_break():
     m2 = OracleModel(cfg, W, bias2)
     m2.step(si.prompt_tokens(cfg), 0)
     assert m2.expert_counts[0][0].tolist() == [cfg.B * cfg.S, cfg.B * cfg.S, 0, 0]
+
+
+MOE_TOY = replace(TOY, L=2, E=4, topk=2, F=16)
+
+
+def test_moe_top2_matches_scalar_loops():
+    """The whole mixture-of-experts forward pass (router, top-2 with the tie rule, softmax over the two selected logits
+    only, gate <-> expert pairing, scaling after the down projection, summation in ascending expert id) against plain
+    Python loops in double.  A softmax over all E logits, gates swapped between the two slots, or the gate applied
+    before the down projection's fp32 rounding all move the logits by far more than the tolerance."""
+    cfg = MOE_TOY
+    m, W = toy_model(cfg)
+    bias = si.router_bias(cfg)
+    toks = si.prompt_tokens(cfg)
+    got = m.step(toks, 0, all_positions=True)
+    seen = np.zeros((cfg.L, cfg.E), dtype=np.int64)
+    for b in range(cfg.B):
+        routed = []
+        ref = np.array(scalar_forward(cfg, W, toks[b].tolist(), bias, routed))
+        assert np.abs(got[b] - ref).max() < 2e-3 * max(1.0, np.abs(ref).max())
+        assert np.mean(np.abs(got[b] - ref)) < 1e-4
+        for (l, p, choice) in routed:
+            assert len(choice) == 2 and abs(sum(g for _, g in choice) - 1.0) < 1e-6
+            for e, g in choice:
+                seen[l, e] += 1
+    assert [c.tolist() for c in m.expert_counts[0]] == seen.tolist()
+    assert (seen > 0).sum() >= 5                 # the toy routes to several experts, with unequal gates
+    # the same pass with the two gates of every token exchanged must NOT pass: the pin would catch a swapped pairing
+    class Swapped(OracleModel):
+        def ffn_moe(self, l, h2, x):
+            cfg_ = self.cfg
+            logits = (h2.astype(np.float64) @ self.w[(self.ROUTER, l, -1)].T + self.bias[l]).astype(np.float32)
+            order = np.argsort(-logits, axis=-1, kind="stable")[:, :2]
+            sel = np.take_along_axis(logits, order, axis=-1).astype(np.float64)
+            ex = np.exp(sel - sel.max(axis=-1, keepdims=True))
+            gates = (ex / ex.sum(axis=-1, keepdims=True)).astype(np.float32)[:, ::-1]
+            counts = np.zeros(cfg_.E, dtype=np.int64)
+            for e in range(cfg_.E):
+                rows, slot = np.nonzero(order == e)
+                counts[e] = len(rows)
+                if len(rows):
+                    x[rows] = (x[rows].astype(np.float64) + gates[rows, slot][:, None] * self.ffn_dense(l, h2[rows], e)).astype(np.float32)
+            return x, counts
+    lay = si.build_layout(cfg)
+    bad = Swapped(cfg, W, bias).step(toks, 0, all_positions=True)
+    ref0 = np.array(scalar_forward(cfg, W, toks[0].tolist(), bias))
+    assert np.abs(bad[0] - ref0).max() > 20 * 2e-3 * max(1.0, np.abs(ref0).max())
+
+
+def test_moe_gates_closed_forms():
+    """Router weights zero, so the logits are the bias.  (1) Two experts with equal logits and equal weights: gates
+    1/2, 1/2, and y/2 + y/2 is exactly the dense FFN's y.  (2) Bias (ln 3, 0, -1/2, -1/2) over four experts: the top
+    two are experts 0 and 1 with gates 3/4 and 1/4 - a softmax over all four logits would give 0.575 and 0.192 - and
+    with expert 1's down projection zeroed the layer adds exactly 3/4 of expert 0's output; with expert 0's zeroed,
+    1/4 of expert 1's: the gate goes with its own expert."""
+    dense = replace(TOY, L=1)
+    lay = si.build_layout(dense)
+    W = si.weights_as_bits(lay)
+    for k, v in W.items():
+        if k[0] not in (si.K_G1, si.K_G2, si.K_GF):
+            W[k] = si.f32_to_bf16_bits(si.bf16_bits_to_f32(v) * np.float32(8.0))
+    toks = si.prompt_tokens(dense)
+    base = {k: v for k, v in W.items() if k[0] not in (si.K_WG, si.K_WU, si.K_WD)}
+    base[(si.K_ROUTER, 0, -1)] = np.zeros((2, dense.d), dtype=np.uint16)
+    two = dict(base)
+    for e in range(2):
+        for k in (si.K_WG, si.K_WU, si.K_WD):
+            two[(k, 0, e)] = W[(k, 0, -1)]
+    a = OracleModel(dense, W).step(toks, 0)
+    b = OracleModel(replace(dense, E=2, topk=2), two, np.array([[0.3, 0.3]], np.float32)).step(toks, 0)
+    assert np.abs(a - b).max() < 1e-6
+    # (2) at the level of the layer function, on a zero residual stream
+    cfg4 = replace(dense, E=4, topk=2)
+    lay4 = si.build_layout(cfg4)
+    W4 = si.weights_as_bits(lay4)
+    for k, v in W4.items():
+        if k[0] not in (si.K_G1, si.K_G2, si.K_GF):
+            W4[k] = si.f32_to_bf16_bits(si.bf16_bits_to_f32(v) * np.float32(8.0))
+    W4[(si.K_ROUTER, 0, -1)][:] = 0
+    bias = np.array([[math.log(3.0), 0.0, -0.5, -0.5]], dtype=np.float32)
+    rng = np.random.default_rng(8)
+    h2 = bf16_round(rng.standard_normal((5, dense.d)).astype(np.float32)).astype(np.float64)
+    for keep, gate in ((0, 0.75), (1, 0.25)):
+        Wk = {k: v.copy() for k, v in W4.items()}
+        Wk[(si.K_WD, 0, 1 - keep)][:] = 0
+        m = OracleModel(cfg4, Wk, bias)
+        y, counts = m.ffn_moe(0, h2, np.zeros((5, dense.d), dtype=np.float32))
+        assert counts.tolist() == [5, 5, 0, 0]
+        want = gate * m.ffn_dense(0, h2, keep).astype(np.float64)
+        assert np.abs(y - want).max() < 1e-6 * max(1.0, np.abs(want).max())
+        assert np.abs(want).max() > 1e-3
 
 
 def test_fp32_and_fp64_oracles_agree_on_config_1_prefill():

@@ -4,7 +4,8 @@ Some users of this library run where they cannot allocate device memory: the dev
 spent on the arena and workspace, or an allocation's implicit synchronisation would stall their serving
 loop.  For them tgp_k_attn_decode_static() keeps its scratch in a fixed array inside the library.  Here it
 is called through the C ABI twice in a row (the array is shared and keeps the previous call's contents) and
-must give what tgp_k_attn() gives with caller scratch.  This file sorts last on purpose: a run that stops at
+must give what tgp_k_attn() gives with caller scratch, and what the CPU oracle's attention gives on the same
+queries and cache (the rule the kernel tests use: within one bf16 ulp of the largest output).  This file sorts last on purpose: a run that stops at
 the first failure has then already run everything else.
 """
 import numpy as np
@@ -15,6 +16,7 @@ import seeded_inputs as si
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
+from oracle.forward import OracleModel, bf16_round  # noqa: E402
 from paper_2609_06172_b200 import binding as tb  # noqa: E402
 from paper_2609_06172_b200.session import model_cfg  # noqa: E402
 
@@ -47,6 +49,13 @@ def test_static_scratch_variant_matches_caller_scratch_variant_twice_in_a_row(sh
         g, w = got.float().cpu().numpy(), want.float().cpu().numpy()
         assert (np.abs(g - w) <= np.abs(w) * 2.0 ** -7).all()
         assert np.array_equal(g, w)
+        # and against the oracle: softmax(q K^T / sqrt(Dh)) V over the pos0 + 1 cached keys, from the same bf16 inputs
+        om = OracleModel(cfg, {})
+        cache = lambda tiles: torch.stack([x.view(cfg.B, cfg.Hkv, cfg.TK, cfg.Dh) for x in tiles], dim=2).reshape(cfg.B, cfg.Hkv, -1, cfg.Dh).float().cpu().numpy()
+        om.K[0], om.V[0] = cache(kt)[:, :, :cfg.max_len], cache(vt)[:, :, :cfg.max_len]
+        att = om.attention(0, qb.float().cpu().numpy().reshape(cfg.B, 1, cfg.Hq, cfg.Dh), pos0).reshape(cfg.B, cfg.Hq * cfg.Dh)
+        assert np.abs(g - att).max() < 2.0 ** -7 * np.abs(att).max() + 1e-6
+        assert np.mean(np.abs(g - bf16_round(att))) < 3e-3 * np.abs(att).mean()
 
 
 def test_static_scratch_variant_rejects_sizes_beyond_its_fixed_array():
