@@ -215,7 +215,8 @@ int  tgp_managed_evict(void *ptr, uint64_t bytes);
 
 /* Activation tap, for parity checks at every rounding point.  While a tap buffer is set, tgp_step() copies each
  * bf16-rounded activation it produces into it (on the compute stream, 256-byte aligned, in op order): normed
- * hidden states, rotated q, the KV tiles an append touched, attention output, the SwiGLU output (dense FFN),
+ * hidden states, rotated q, the KV tiles an append touched, attention output, the SwiGLU output (dense FFN: all tokens,
+ * sub-index 0; mixture of experts: per expert the rows routed to it in ascending token order, sub-index = expert),
  * the final normed state.  tgp_tap_index() returns 5 uint64 per record: op index, tag, sub-index (tile), offset,
  * bytes (two-call form: out == NULL gives the word count).  tgp_set_tap() also rewinds the buffer; NULL disables. */
 #define TGP_TAP_H 0u
@@ -319,6 +320,14 @@ int  tgp_k_attn_status(int *error_code);
 /* Error word of the tensor-core GEMM: 0, or (role << 8 | stage) of the first bounded wait that ran out
  * (role 1 TMA producer, 2 MMA issuer, 3 epilogue).  Synchronous. */
 int  tgp_k_gemm_status(int *error_code);
+/* For tests of the give-up path of the tensor-core kernels (every wait on an mbarrier in them is bounded in time; a wait
+ * that runs out records an error word, the CTA drains its copies in flight, frees its tensor memory, stores nothing and
+ * returns).  Sets, for the current device and until changed back, the time limit of those waits (default 2 s; at least
+ * 100 us) and the index of one load step - a K block of the GEMM kernels, a V block of the attention kernel - that the
+ * TMA thread of the grid's first CTA (CTA pair) leaves out (-1: none), so that the wait for it runs out; nothing traps or
+ * faults, the other CTAs of the launch complete normally.  limit_ns == 0 restores the defaults.  Waits for the device to
+ * go idle first.  Process-wide. */
+int  tgp_k_wait_test(uint64_t limit_ns, int withhold_step);
 /* Fills caller-owned device tables cos/sin fp32 [max_len, Dh/2]: angle = pos * base^(-2i/Dh), evaluated in
  * double on the host.  Synchronous. */
 int  tgp_k_rope_tables(uint32_t Dh, uint32_t max_len, float base, float *cos_dev, float *sin_dev);

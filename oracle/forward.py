@@ -112,7 +112,7 @@ class OracleModel:
     def ffn_dense(self, l, h2, e=-1):
         g = self.linear(h2, self.w[(self.WG, l, e)]).astype(self.dt)
         u = self.linear(h2, self.w[(self.WU, l, e)]).astype(self.dt)
-        a = self._round("a", l, g / (1.0 + np.exp(-g)) * u) if e < 0 else bf16_round(to_f32(g / (1.0 + np.exp(-g)) * u))
+        a = self._round("a" if e < 0 else "a.e%d" % e, l, g / (1.0 + np.exp(-g)) * u)
         return self.linear(a, self.w[(self.WD, l, e)])
 
     def ffn_moe(self, l, h2, x):

@@ -96,6 +96,7 @@ _SIGS = {
     "tgp_k_embed": [_P, _P, _P, _U32, _U32, _U32, _P],
     "tgp_k_embed_status": [C.POINTER(C.c_int), C.POINTER(_U32), C.POINTER(C.c_int32)],
     "tgp_k_status_clear": [],
+    "tgp_k_wait_test": [_U64, C.c_int],
     "tgp_k_rmsnorm": [_P, _U32, _P, _P, _U32, _U32, C.c_float, _P],
     "tgp_k_gemm": [_P, _P, _P, _U32, _U32, _U32, _U32, _U32, C.c_int, _P],
     "tgp_k_gemm_group": [_P, _U32, _P, _P, C.POINTER(_U32), C.POINTER(_U32), _U32, _U32, C.c_int, _P],
@@ -385,6 +386,10 @@ def k_embed_status():
     b, r, t = C.c_int(), _U32(), C.c_int32()
     _k(lib().tgp_k_embed_status(C.byref(b), C.byref(r), C.byref(t)), "tgp_k_embed_status")
     return b.value, r.value, t.value
+
+
+def k_wait_test(limit_ns, withhold_step):
+    _k(lib().tgp_k_wait_test(limit_ns, withhold_step), "tgp_k_wait_test")
 
 
 def k_status_clear():

@@ -148,8 +148,11 @@ __global__ void __launch_bounds__(THREADS, 2) tgp_attn_prefill_tc_kernel(const _
         if (warp == 5) {
             // ======================= TMA warp: lane 0 requests the remaining K and V blocks =======================
             if (lane == 0) {
+                // test hook: the first CTA of the grid never loads this V block, so the wait for it runs out
+                const uint32_t withhold = (blockIdx.x | blockIdx.y | blockIdx.z) == 0 ? (uint32_t)g_withhold_step : 0xffffffffu;
                 for (uint32_t jb = 0; jb + 1 < nblk; ++jb) {
                     const uint32_t st = jb & 1;
+                    if (jb + 1 == withhold) break;
                     if (jb + 2 < nblk) {                                         // K_jb+2 goes where K_jb is, once S_jb is complete
                         if (!mbar_wait(bar_kfree + st, (jb >> 1) & 1, failed)) { give_up(1); break; }
                         next_k(0);
@@ -398,6 +401,11 @@ int tgpk_attn_prefill_tc5(const void *qb, const TgpTilePtrs &tiles, void *ob, co
     if (cudaGetLastError() != cudaSuccess) return TGP_E_CUDA;
     tgpk_launches += 1;
     return TGP_OK;
+}
+
+int tgpk_attn_wait_test(unsigned long long limit_ns, int withhold_step) {
+    if (cudaMemcpyToSymbol(g_wait_limit_ns, &limit_ns, sizeof(limit_ns)) != cudaSuccess) return TGP_E_CUDA;
+    return cudaMemcpyToSymbol(g_withhold_step, &withhold_step, sizeof(withhold_step)) == cudaSuccess ? TGP_OK : TGP_E_CUDA;
 }
 
 int tgpk_attn_status_clear() { const int z = 0; return cudaMemcpyToSymbol(g_attn_tc_error, &z, sizeof(z)) == cudaSuccess ? TGP_OK : TGP_E_CUDA; }

@@ -761,6 +761,9 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
                 trc = tap_copy(TGP_TAP_O, 0, e->ob, (uint64_t)M * qd * 2);
             } else if (o.kind == TGP_OP_SWIGLU && !c.E) {
                 trc = tap_copy(TGP_TAP_A, 0, e->ab, (uint64_t)M * c.F * 2);
+            } else if (o.kind == TGP_OP_SWIGLU && e->cur_expert >= 0 && e->cnt[e->cur_expert]) {
+                // mixture of experts: the rows routed to this expert, in ascending token order; the sub-index is the expert
+                trc = tap_copy(TGP_TAP_A, (uint64_t)e->cur_expert, e->ab, (uint64_t)e->cnt[e->cur_expert] * c.F * 2);
             }
             if (trc) return trc;
         }

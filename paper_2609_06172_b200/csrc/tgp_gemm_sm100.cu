@@ -78,8 +78,10 @@ __global__ void __launch_bounds__(192) tgp_matmul_tc_kernel(const __grid_constan
     if (warp == 0) {
         if (lane == 0) {
             uint32_t armed = 0;
+            const uint32_t withhold = blockIdx.x == 0 ? (uint32_t)g_withhold_step : 0xffffffffu;     // test hook: this stage is never loaded
             for (uint32_t kb = 0; kb < num_k; ++kb) {
                 const uint32_t s = kb % STAGES, ph = (kb / STAGES) & 1;
+                if (kb == withhold) break;
                 if (*failed || !mbar_wait(&empty[s], ph ^ 1, failed)) { if (!*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, (1 << 8) | (int)s); } break; }
                 mbar_expect_tx(&full[s], S::STAGE_BYTES);
 #pragma unroll
@@ -212,11 +214,13 @@ __global__ void __launch_bounds__(192, 1) tgp_matmul_tc_persistent_kernel(const 
         if (lane == 0) {
             uint32_t it = 0, armed = 0;
             bool ok = true;
+            const uint32_t withhold = blockIdx.x == 0 ? (uint32_t)g_withhold_step : 0xffffffffu;     // test hook: this stage is never loaded
             for (uint32_t tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
                 uint32_t m0, n0;
                 tile_origin(tile, m0, n0);
                 for (uint32_t kb = 0; kb < num_k; ++kb, ++it) {
                     const uint32_t s = it % P_STAGES, ph = (it / P_STAGES) & 1;
+                    if (it == withhold) { ok = false; break; }
                     if (*failed || !mbar_wait(&empty[s], ph ^ 1, failed)) { if (!*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, (1 << 8) | (int)s); } ok = false; break; }
                     mbar_expect_tx(&full[s], STAGE_BYTES);
                     tma_load_2d(smem + s * STAGE_BYTES, &tmA, (int)(kb * BK), (int)m0, &full[s]);
@@ -356,12 +360,14 @@ __global__ void __launch_bounds__(192, 1) tgp_matmul_tc_pair_kernel(const __grid
     if (warp == 0) {
         if (lane == 0) {                              // TMA thread of this CTA: its rows of A, its half of B
             uint32_t it = 0, armed = 0;
+            const uint32_t withhold = pair == 0 ? (uint32_t)g_withhold_step : 0xffffffffu;     // test hook: both CTAs of the first pair never load this stage
             for (uint32_t tile = pair; tile < tiles; tile += pairs) {
                 uint32_t m0, n0;
                 tile_origin(tile, m0, n0);
                 bool ok = true;
                 for (uint32_t kb = 0; kb < num_k; ++kb, ++it) {
                     const uint32_t s = it % Q_STAGES, ph = (it / Q_STAGES) & 1;
+                    if (it == withhold) { ok = false; break; }
                     if (*failed || !mbar_wait(&empty[s], ph ^ 1, failed)) { if (!*failed) { *failed = 1; atomicCAS(&g_gemm_tc_error, 0, (1 << 8) | (int)s); } ok = false; break; }
                     if (rank == 0) mbar_expect_tx(&full[s], 2 * STAGE_BYTES);
 #pragma unroll
@@ -564,6 +570,11 @@ extern "C" int tgp_k_gemm_tc_variant(int v) {
     if (v < 0 || v > 4) return TGP_E_INVAL;
     g_tc_variant = v;
     return TGP_OK;
+}
+
+int tgpk_gemm_wait_test(unsigned long long limit_ns, int withhold_step) {
+    if (cudaMemcpyToSymbol(g_wait_limit_ns, &limit_ns, sizeof(limit_ns)) != cudaSuccess) return TGP_E_CUDA;
+    return cudaMemcpyToSymbol(g_withhold_step, &withhold_step, sizeof(withhold_step)) == cudaSuccess ? TGP_OK : TGP_E_CUDA;
 }
 
 int tgpk_gemm_status_clear() { const int z = 0; return cudaMemcpyToSymbol(g_gemm_tc_error, &z, sizeof(z)) == cudaSuccess ? TGP_OK : TGP_E_CUDA; }

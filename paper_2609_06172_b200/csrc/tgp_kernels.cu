@@ -1455,6 +1455,14 @@ int tgp_k_embed_status(int *bad, uint32_t *row, int32_t *token) {
     return TGP_OK;
 }
 
+int tgp_k_wait_test(uint64_t limit_ns, int withhold_step) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return TGP_E_CUDA;
+    if (!limit_ns) { limit_ns = 2000000000ull; withhold_step = -1; }
+    if (limit_ns < 100000ull || withhold_step < -1) return TGP_E_INVAL;
+    int rc = tgpk_gemm_wait_test(limit_ns, withhold_step);
+    return rc ? rc : tgpk_attn_wait_test(limit_ns, withhold_step);
+}
+
 int tgp_k_status_clear(void) {
     if (cudaDeviceSynchronize() != cudaSuccess) return TGP_E_CUDA;
     const unsigned long long z = 0;

@@ -11,6 +11,12 @@ namespace tgp_sm100 {
 constexpr int BM = 128;                                // rows of every tcgen05 tile used here (TMEM lanes)
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;      // 2 s: far beyond any legitimate wait in these kernels
 
+// Hooks for testing the give-up path of the bounded waits (one copy per translation unit, set through
+// tgp_k_wait_test()): the time limit every mbarrier wait runs under, and the index of one load step that the TMA thread
+// of the grid's first CTA (or CTA pair) leaves out, so that the wait for it runs out; -1: nothing is left out.
+static __device__ unsigned long long g_wait_limit_ns = WAIT_LIMIT_NS;
+static __device__ int g_withhold_step = -1;
+
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ uint64_t now_ns() { uint64_t t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
@@ -36,7 +42,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
             if (*failed) return false;
             const uint64_t t = now_ns();
             if (!t0) t0 = t;
-            else if (t - t0 > WAIT_LIMIT_NS) return false;
+            else if (t - t0 > g_wait_limit_ns) return false;
         }
     }
 }

@@ -478,7 +478,7 @@ def test_llama_8b_full_depth_lockstep_parity_reduced_tokens():
     hours.  Lockstep: every rounding point of all 32 layers element by element, logits within the stated tolerance."""
     cfg = replace(si.CONFIGS[3], B=1, S=16, T=4)
     lay = si.build_layout(cfg)
-    assert lay.budget == 8 << 30 and cfg.L == 32 and lay.pool_bytes > 2 * lay.budget * 0.95
+    assert lay.budget == 8 << 30 and cfg.L == 32 and lay.pool_bytes > 1.8 * lay.budget          # weights alone: 1.87x the budget
     pool = pinned_pool(lay.pool_bytes)
     si.fill_pool_torch(lay, pool, device="cuda:0")
     worst, flips = _lockstep(cfg, lay, pool, _weights_from_pool(lay, pool), cfg.T, np.float32)
@@ -573,7 +573,7 @@ def _lockstep(cfg, lay, pool, W, n_dec, dtype, bias=None):
     ops = s.ctx.trace_ops()
     r = Runner(s, cfg.B * cfg.S)
     qd, F, d = cfg.Hq * cfg.Dh, cfg.F, cfg.d
-    per_layer = cfg.B * cfg.S * (2 * d + 2 * qd + F) * 2 + 2 * cfg.n_tiles * cfg.B * cfg.Hkv * cfg.TK * cfg.Dh * 2 + 16 * 256
+    per_layer = cfg.B * cfg.S * (2 * d + 2 * qd + F * max(1, cfg.topk)) * 2 + 2 * cfg.n_tiles * cfg.B * cfg.Hkv * cfg.TK * cfg.Dh * 2 + (16 + cfg.E) * 256
     tap = torch.empty(per_layer * cfg.L + (1 << 20), dtype=torch.uint8, device="cuda:0")
     om = forward.OracleModel(cfg, W, bias, dtype=dtype)
     W = None                                               # the oracle holds its own converted copy
@@ -583,7 +583,10 @@ def _lockstep(cfg, lay, pool, W, n_dec, dtype, bias=None):
     # states sit behind the residual stream, which sums tensor-core products of K up to 8192 per layer (their fp32
     # accumulation is not round-to-nearest: ~5e-5 typical, 3e-4 covers the tail of 1e6 elements); the attention output
     # also carries the tensor-core kernel's bf16 rounding of the softmax weights (not mirrored by the oracle)
-    rtol = {"h": 3e-4, "h2": 3e-4, "hf": 3e-4, "q": 1e-4, "k": 1e-4, "v": 1e-4, "a": 1e-4, "o": 4e-3}
+    # (the tensor cores' fp32 accumulation is not round-to-nearest: its error has a part linear in K, so the points fed
+    # directly by a product over K = d get a slack that grows with d beyond 4096)
+    kd = 1e-4 * max(1.0, cfg.d / 4096)
+    rtol = {"h": 3e-4, "h2": 3e-4, "hf": 3e-4, "q": kd, "k": kd, "v": kd, "a": kd, "o": 4e-3}
     flips = {k: [0, 0] for k in rtol}
     prompt = si.prompt_tokens(cfg)
     worst = 0.0
@@ -615,9 +618,14 @@ def _lockstep(cfg, lay, pool, W, n_dec, dtype, bias=None):
             elif tag == tb.TAP_O:
                 got[("o", layer)] = a.reshape(cfg.B, q, cfg.Hq, cfg.Dh)
             elif tag == tb.TAP_A:
-                got[("a", layer)] = a.reshape(cfg.B, q, F)
+                if cfg.E:
+                    got[("a.e%d" % sub, layer)] = a.reshape(-1, F)             # rows routed to expert `sub`, ascending token order
+                else:
+                    got[("a", layer)] = a.reshape(cfg.B, q, F)
 
         def hook(name, layer, pre, out, pos0=pos0, q=q):
+            if (name, layer) not in got:
+                raise AssertionError(("the GPU recorded no activation for this rounding point (routing differs?)", name, layer))
             g = got[(name, layer)]
             if name in ("k", "v"):                         # gather the new positions out of the tapped tiles
                 new = np.empty((cfg.B, q, cfg.Hkv, cfg.Dh), dtype=np.float32)
@@ -625,6 +633,7 @@ def _lockstep(cfg, lay, pool, W, n_dec, dtype, bias=None):
                     new[:, p - pos0] = g[p // cfg.TK][:, :, p % cfg.TK, :]
                 g = new
             g = g.reshape(pre.shape)
+            name = name.split(".")[0]                      # "a.e3" (expert 3's SwiGLU output) is checked like "a"
             # (the attention output averages rows of V, so its P-rounding error scales with |V| ~ max|o|, not with |o|)
             scale = np.abs(pre).max() if name == "o" else np.abs(pre).mean()
             bound = 0.5 * _bf16_ulp(pre) * (1 + 1e-6) + rtol[name] * (np.abs(pre) + scale)

@@ -42,7 +42,12 @@ def test_gemm_ridge_on_the_measured_machine():
 
 
 def test_trace_counts_by_hand_config_1():
+    # with the recipe's own 512 KiB blocks every FFN matrix is one block and the head four: 55 ops per decode step
     lay = si.build_layout(si.CONFIGS[1])
+    ops, steps = trace.run_trace(lay)
+    assert steps[1][2] == 1 + 4 * (1 + 3 + 1 + 1 + 1 + 1 + 1 + 1 + 1 + 1) + 1 + 4 + 1
+    # the hand computation below is for 128 KiB blocks (four blocks per FFN matrix, sixteen for the head)
+    lay = si.build_layout(si.CONFIGS[1], cap=128 << 10)
     ops, steps = trace.run_trace(lay)
     assert len(steps) == 17 and steps[0][0] == trace.STEP_PREFILL and steps[1][0] == trace.STEP_DECODE
     pre = ops[steps[0][1]: steps[0][1] + steps[0][2]]

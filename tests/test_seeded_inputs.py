@@ -29,7 +29,8 @@ def test_layout_sizes(c):
 
 
 def test_sub_range_cap_rule():
-    assert si.sub_range_cap(6_392_064) == 128 << 10
+    assert si.sub_range_cap(6_392_064) == 512 << 10
+    assert si.sub_range_cap(1 << 20) == 128 << 10
     assert si.sub_range_cap(1_104_218_112) == 32 << 20
     assert si.sub_range_cap(64 << 30) == 32 << 20
 
