@@ -449,15 +449,16 @@ def other_config_summaries(args, budget_s):
         if left < 60:
             out[str(c)] = {"skipped": "time budget of this run spent"}
             continue
-        cmd = [sys.executable, os.path.abspath(__file__), "--config", str(c), "--summary"]
-        t0 = time.monotonic()
-        try:
-            r = subprocess.run(cmd, capture_output=True, text=True, timeout=min(left, 600))
-            line = [l for l in r.stdout.splitlines() if l.startswith("{")]
-            out[str(c)] = json.loads(line[-1]) if r.returncode == 0 and line else {"failed": f"rc {r.returncode}", "stderr_tail": r.stderr[-400:]}
-        except subprocess.TimeoutExpired:
-            out[str(c)] = {"failed": "time limit"}
-        out[str(c)]["wall_s"] = round(time.monotonic() - t0, 1)
+        for key, extra in ((str(c), []),) + ((("1_graph", ["--graph"]),) if c == 1 else ()):      # the tiny configuration also as one CUDA graph per pass
+            cmd = [sys.executable, os.path.abspath(__file__), "--config", str(c), "--summary"] + extra
+            t0 = time.monotonic()
+            try:
+                r = subprocess.run(cmd, capture_output=True, text=True, timeout=min(left, 600))
+                line = [l for l in r.stdout.splitlines() if l.startswith("{")]
+                out[key] = json.loads(line[-1]) if r.returncode == 0 and line else {"failed": f"rc {r.returncode}", "stderr_tail": r.stderr[-400:]}
+            except subprocess.TimeoutExpired:
+                out[key] = {"failed": "time limit"}
+            out[key]["wall_s"] = round(time.monotonic() - t0, 1)
     return out
 
 
@@ -482,7 +483,7 @@ def main():
     ap.add_argument("--graph", action="store_true", help="replay the whole planned run as one CUDA graph (dense models; for host-bound tiny steps)")
     ap.add_argument("--layers", type=int, default=None, help="run the shape at reduced depth; a byte budget is scaled in proportion")
     ap.add_argument("--cap-mib", type=float, default=None, help="sub-range cap in MiB (default: the input recipe's rule)")
-    ap.add_argument("--bits", type=int, default=7, help="policy bits: 1 affinity/pins, 2 roofline selectivity, 4 zero-copy")
+    ap.add_argument("--bits", type=int, default=15, help="policy bits: 1 affinity/pins, 2 roofline selectivity, 4 zero-copy, 8 windowed pin reservation")
     ap.add_argument("--budget-frac", type=float, default=None, help="device budget as a fraction of the pool (oversubscription sweep)")
     args = ap.parse_args()
     cfg = si.CONFIGS[args.config]
@@ -494,7 +495,7 @@ def main():
     if args.alias_layers is None and args.config in ALIAS_LAYERS and args.layers is None and args.impl != "reference" and not args.kernel_loop:
         args.alias_layers = ALIAS_LAYERS[args.config]
     if args.summary:
-        args.steps, args.warmup, args.no_configs, args.no_cpu_baseline = 1, 1, True, True
+        args.steps, args.warmup, args.no_configs, args.no_cpu_baseline = (20, 5, True, True) if args.config == 1 else (1, 1, True, True)
         args.no_uvm = args.no_uvm or args.config != 2
     budget = None
     if args.layers is not None and args.layers != cfg.L:

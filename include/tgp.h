@@ -92,6 +92,8 @@ extern "C" {
 #define TGP_BIT_A  1u   /* look-ahead affinity: residency (pin) set              */
 #define TGP_BIT_P  2u   /* roofline selectivity; off = every op with pool traffic is link-bound */
 #define TGP_BIT_ZC 4u   /* sparse read-only accesses are served in place over the link          */
+#define TGP_BIT_W  8u   /* windowed pin reservation: the slot of a pinned tensor that is born on the device in a later
+                           step (a KV tile of positions not reached yet) houses unpinned read-only tensors until then */
 /* plan export selectors */
 #define TGP_X_CLASSES  0u   /* u8 per op: 0 LINK, 1 HBM, 2 COMPUTE                                   */
 #define TGP_X_TENSORS  1u   /* per tensor: u8 critical, u8 zero-copy, u64 score (link bytes residency saves) */
@@ -99,6 +101,7 @@ extern "C" {
 #define TGP_X_COMMANDS 3u   /* per command: u32 seq, u8 kind(0 H2D,1 ALLOC,2 D2H), u32 tensor, u64 bytes, u64 pool offset,
                                u64 arena offset, i32 wait_op, i32 first_use, i32 release_after      */
 #define TGP_X_TOTALS   4u   /* per step: u64 h2d bytes, u64 d2h bytes, u64 zero-copy bytes, u64 commands */
+#define TGP_X_TAIL 0x100u   /* or-ed into a selector: the tail plan that waits for tgp_replan_commit() (after tgp_replan_wait()) */
 
 typedef struct tgp_ctx tgp_ctx;
 
@@ -171,6 +174,18 @@ int  tgp_set_object_bytes(tgp_ctx *ctx, uint64_t bytes);
  * n_ops == 0 clears the log; a new trace clears it too.  Integers make the re-plan reproducible: the same log fed
  * to another planner gives the same schedule. */
 int  tgp_set_measured_times(tgp_ctx *ctx, const uint64_t *op_ns, uint64_t n_ops);
+/* Runtime monitor, while the run is under way (Section IV-E: classes are re-evaluated from measured kernel times and the
+ * engine adapts, in parallel with the kernels that follow).  tgp_replan_begin() takes the timing log so far - one entry
+ * per op of the whole trace in integer nanoseconds, 0 = not measured (n_ops == 0 keeps the stored log) - and plans the
+ * steps from first_step on as a trace of their own on a helper thread, while tgp_step() goes on executing the current
+ * plan.  The tail plan assumes an empty arena at the boundary and that tensors written in earlier steps hold data in
+ * the pool.  tgp_replan_wait() waits for the planner and reports its result.  tgp_replan_commit() must be called when
+ * the run stands exactly at the boundary (first_step steps done): it waits for the device, copies the pinned tensors
+ * that were written back to the pool, and switches; tgp_plan_export() then exports the tail plan (op indices of the whole
+ * trace; classes and totals cover the tail only).  tgp_run_reset() brings the whole-run plan back.  Explicit engine only. */
+int  tgp_replan_begin(tgp_ctx *ctx, uint32_t first_step, const uint64_t *op_ns, uint64_t n_ops);
+int  tgp_replan_wait(tgp_ctx *ctx);
+int  tgp_replan_commit(tgp_ctx *ctx);
 /* Classifies ops, selects critical / zero-copy / pinned tensors, sizes the ring and builds the ordered
  * command list.  Host only; no CUDA call. */
 int  tgp_plan(tgp_ctx *ctx);

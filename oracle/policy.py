@@ -34,6 +34,14 @@ Steps, in order (notation: P = peak flop/s, Bh = HBM bytes/s, Bl = host-link byt
    by a greedy fill with skip.  Spreading keeps the link demand of the streamed rest uniform over a
    step instead of leaving the copy engine idle while compute walks a pinned prefix of layers.
    Pins sit at [0, used) in the order they were chosen; the ring is [used, budget).
+5b. windowed reservation (W bit): a pinned tensor that is born on the device (MUTABLE, first access a write, no data
+   in the pool) in step s >= 2 - a KV tile of positions not yet reached - does not need its slot before that step.
+   Adjacent such slots with the same birth step form a vacancy region, free for steps [0, s).  Regions are taken by
+   longest vacancy first (tie: lower offset); the unpinned, non-ZC, READONLY candidates of step 5, in the same density
+   order, become tenants by first fit: a tenant accessed in at least two steps before s is loaded at its first access
+   into the region (bump allocation) and stays there until its last access before step s, after which it is streamed
+   through the ring like any unpinned tensor.  The landlord's own placement waits for the last use of every tenant
+   of its region.  Saves the tenant's size once per step of the vacancy but the first.
 6. schedule: walk ops in order, accesses in list order.
      pinned tensor, first access: LOAD (H2D into its slot), or ALLOC if MUTABLE and the access is W.
      ring tensor, episode start: FIFO bump allocation (wrap to the ring base when the tail does
@@ -54,7 +62,7 @@ W_AFF = 4
 ZC_DEN = 2
 CLS_LINK, CLS_HBM, CLS_COMPUTE = 0, 1, 2
 CMD_H2D, CMD_ALLOC, CMD_D2H = 0, 1, 2
-BIT_A, BIT_P, BIT_ZC = 1, 2, 4
+BIT_A, BIT_P, BIT_ZC, BIT_W = 1, 2, 4, 8
 MODE_R, MODE_W = 1, 2
 F_READONLY, F_MUTABLE = 1, 2
 
@@ -132,9 +140,12 @@ class Plan:
         }
 
 
-def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A | BIT_P | BIT_ZC, measured_ns=None) -> Plan:
+def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A | BIT_P | BIT_ZC | BIT_W, measured_ns=None,
+         written_before=()) -> Plan:
     """tensors: list of objects with .size .pool_off .flags; ops: list with .step .flops .hbm .acc;
-    steps: [(kind, first op, count)]; measured_ns: optional per-op kernel times in integer nanoseconds (0 = none)."""
+    steps: [(kind, first op, count)]; measured_ns: optional per-op kernel times in integer nanoseconds (0 = none);
+    written_before: tensors that already hold data in the pool when the trace starts (a tail re-plan), whose first
+    access therefore loads them even if it is a write."""
     T, N = len(tensors), len(ops)
     # 1-2: classes, criticality, score
     cls = []
@@ -234,13 +245,51 @@ def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A |
                     used += a
     ring_base, ring_size = used, budget - used
     pins = sorted(pinned_off.items())
+    # 5b: windowed reservation - tenants of the slots of pinned tensors that are born late
+    tenancy: Dict[int, Tuple[int, int]] = {}       # tenant -> (arena offset, last op it is used there)
+    landlord_wait: Dict[int, int] = {}             # late-born pinned tensor -> op its placement must wait for
+    if (bits & BIT_W) and pinned_off:
+        first_acc: Dict[int, Tuple[int, int]] = {}
+        for i, op in enumerate(ops):
+            for (t, mode, _) in op.acc:
+                first_acc.setdefault(t, (i, mode))
+        late = [t for t in pinned_off if tensors[t].flags == F_MUTABLE and t not in written_before
+                and first_acc[t][1] == MODE_W and step_of[first_acc[t][0]] >= 2]
+        regions = []                               # [start, end, birth step, landlords]
+        for t in sorted(late, key=lambda t: pinned_off[t]):
+            o, a, b = pinned_off[t], alignup(tensors[t].size), step_of[first_acc[t][0]]
+            if regions and regions[-1][1] == o and regions[-1][2] == b:
+                regions[-1][1] = o + a
+                regions[-1][3].append(t)
+            else:
+                regions.append([o, o + a, b, [t]])
+        regions.sort(key=lambda r: (-r[2], r[0]))
+        fill = [r[0] for r in regions]
+        region_wait = [-1] * len(regions)
+        for t in order:
+            if t in pinned_off or tensors[t].flags != F_READONLY:
+                continue
+            a = alignup(tensors[t].size)
+            for k, (start, end, b, _) in enumerate(regions):
+                if fill[k] + a > end:
+                    continue
+                before = [i for i in acc_ops[t] if step_of[i] < b]
+                if not before or step_of[before[0]] == step_of[before[-1]]:
+                    continue                       # used in fewer than two steps of the vacancy: nothing to save
+                tenancy[t] = (fill[k], before[-1])
+                fill[k] += a
+                region_wait[k] = max(region_wait[k], before[-1])
+                break
+        for k, r in enumerate(regions):
+            for t in r[3]:
+                landlord_wait[t] = region_wait[k]
     # 6: schedule
     cmds: List[Cmd] = []
     totals = [[0, 0, 0, 0] for _ in steps]
     ep_index = {t: 0 for t in episodes_of}
     open_stay: Dict[int, int] = {}            # ring tensor -> arena offset of its current stay
     pin_loaded = set()
-    written_ever = set()
+    written_ever = set(written_before)
     last_wb_op: Dict[int, int] = {}
     fifo: List[Tuple[int, int, int]] = []     # (start, end, last-use op) of ring stays, oldest first
     head = 0
@@ -269,8 +318,14 @@ def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A |
             if t in pinned_off:
                 if t not in pin_loaded:
                     pin_loaded.add(t)
-                    emit(CMD_ALLOC if fresh_write else CMD_H2D, t, pinned_off[t], -1, i, N - 1)
+                    emit(CMD_ALLOC if fresh_write else CMD_H2D, t, pinned_off[t], landlord_wait.get(t, -1), i, N - 1)
+            elif t in tenancy and i <= tenancy[t][1]:
+                if t not in pin_loaded:                        # a tenant: loaded once into the vacant slot, used there
+                    pin_loaded.add(t)
+                    emit(CMD_H2D, t, tenancy[t][0], -1, i, tenancy[t][1])
             elif t not in open_stay:
+                while episodes_of[t][ep_index[t]][0] < i:      # stays a tenancy made unnecessary
+                    ep_index[t] += 1
                 f, l = episodes_of[t][ep_index[t]]
                 assert f == i
                 a = alignup(tensors[t].size)
@@ -304,3 +359,37 @@ def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A |
                 last_wb_op[t] = i
             ep_index[t] += 1
     return Plan(cls, crit, score, zc, pins, ring_base, ring_size, cmds, [tuple(x) for x in totals], ep_list)
+
+
+def plan_tail(tensors, ops, steps, machine: Machine, budget: int, first_step: int, bits: int = BIT_A | BIT_P | BIT_ZC | BIT_W,
+              measured_ns=None) -> Plan:
+    """Re-plan at a step boundary, while the run is under way (Section IV-E "Runtime Monitor": classes are re-evaluated
+    from measured kernel times and the engine adapts; the paper does not say how the switch is made).  Reading: the
+    steps from first_step on are planned as a trace of their own, with the same policy.  At the boundary the engine has
+    drained - every stay has ended (stays never cross a step) and every written pinned tensor has been written back -
+    so nothing is resident and the pool is up to date: the tail plan starts from an empty arena, and a tensor written in
+    an earlier step holds data, so its first access loads it (H2D) even when that access is a write.
+    measured_ns: one entry per op of the WHOLE trace (0 = not measured).  Op indices in the returned commands are those
+    of the whole trace; classes and per-step totals cover the tail only."""
+    import copy
+    first_op = steps[first_step][1]
+    written = set()
+    for op in ops[:first_op]:
+        for (t, mode, _) in op.acc:
+            if mode & MODE_W:
+                written.add(t)
+    sub_ops = []
+    for op in ops[first_op:]:
+        o = copy.copy(op)
+        o.step = op.step - first_step
+        sub_ops.append(o)
+    sub_steps = [(k, o0 - first_op, n) for (k, o0, n) in steps[first_step:]]
+    pl = plan(tensors, sub_ops, sub_steps, machine, budget, bits,
+              None if measured_ns is None else list(measured_ns[first_op:]), written_before=written)
+    for c in pl.cmds:
+        if c.wait_op >= 0:
+            c.wait_op += first_op
+        c.first_use += first_op
+        c.release_after += first_op
+    pl.episodes = [(t, f + first_op, l + first_op) for (t, f, l) in pl.episodes]
+    return pl

@@ -12,7 +12,10 @@ tensors a kernel needs are on the device before it runs, inside a fixed capacity
                       before the op: wait_op < first_use), or the tensor is zero-copy.
  I2 budget          : every placement lies in [0, budget); a placement never overlaps a stay
                       still needed (its release_after must be <= the placement's wait_op);
-                      pins do not overlap the ring or each other.
+                      pins do not overlap the ring or each other.  A tensor that is not pinned may be
+                      placed inside the pin region only as a tenant: wholly inside slots of pinned
+                      tensors that have not been placed yet, disjoint from live tenants, and every
+                      pin placement waits for the last use of the tenants of its slot.
  I3 cover           : each (tensor, first_use) appears exactly once; placements are ordered by
                       (first_use, position in that op's access list); a write-back follows the
                       placements of its op and precedes those of the next op.
@@ -53,9 +56,26 @@ def parse(blobs, n_tensors):
                 ring_size=ring_size, totals=totals, classes=list(blobs["classes"]))
 
 
-def check(tensors, ops, steps, budget, blobs):
-    """Raises PlanInvalid with a reason; returns a small summary dict when everything holds."""
+def check(tensors, ops, steps, budget, blobs, first_step=0):
+    """Raises PlanInvalid with a reason; returns a small summary dict when everything holds.
+    first_step > 0: `blobs` is a tail plan made at that step boundary for the rest of the trace (op indices of the
+    whole trace); the replay then starts from an empty arena with every tensor written in an earlier step holding
+    data in the pool, so such a tensor may never be placed by ALLOC."""
     P = parse(blobs, len(tensors))
+    first_op = steps[first_step][1]
+    written_before = {t for op in ops[:first_op] for (t, mode, _) in op.acc if mode & 2}
+    if first_step:
+        import copy
+        tail = []
+        for op in ops[first_op:]:
+            o = copy.copy(op)
+            o.step = op.step - first_step
+            tail.append(o)
+        ops, steps = tail, [(k, o0 - first_op, n) for (k, o0, n) in steps[first_step:]]
+        P["cmds"] = [(q, kind, t, nb, po, ao, (w - first_op if w >= 0 else w), f - first_op, r - first_op)
+                     for (q, kind, t, nb, po, ao, w, f, r) in P["cmds"]]
+        if any(c[6] < -1 or c[7] < 0 for c in P["cmds"]):
+            raise PlanInvalid("a tail command refers to an op before the boundary")
     N = len(ops)
     if len(P["classes"]) != N:
         raise PlanInvalid("class count")
@@ -94,10 +114,11 @@ def check(tensors, ops, steps, budget, blobs):
         if c[0] != k:
             raise PlanInvalid("sequence numbers")
     # replay
-    host_ver = [0] * len(tensors)
-    newest = [0] * len(tensors)
+    host_ver = [1 if t in written_before else 0 for t in range(len(tensors))]
+    newest = list(host_ver)
     stays = {}                      # tensor -> [arena_off, release_after, version held, is_pin]
     placed = []                     # (start, end, release_after) of ring stays not yet overwritten
+    tenants = []                    # (start, end, release_after) of placements of unpinned tensors inside the pin region
     ring_wait = -1
     h2d = [0] * len(steps)
     d2h = [0] * len(steps)
@@ -122,9 +143,31 @@ def check(tensors, ops, steps, budget, blobs):
             if is_pin:
                 if arena_off != pin_off[t] or t in stays:
                     raise PlanInvalid("pin loaded twice or at the wrong slot")
+                s, e = arena_off, arena_off + up(nbytes)
+                for (a, b, r) in tenants:
+                    if a < e and b > s and r > wait:
+                        raise PlanInvalid(f"pin placed over a tenant still needed until op {r}")
+            elif arena_off < P["ring_base"]:
+                # a tenant of slots whose pinned tensors are not there yet
+                s, e = arena_off, arena_off + up(nbytes)
+                if e > P["ring_base"] or kind != CMD_H2D:
+                    raise PlanInvalid("tenant placement leaves the pin region or is not a load")
+                covered = 0
+                for (pt, po) in P["pins"]:
+                    a, b = po, po + up(tensors[pt].size)
+                    if a < e and b > s:
+                        if pt in stays:
+                            raise PlanInvalid("tenant placed over a pinned tensor that is resident")
+                        covered += min(b, e) - max(a, s)
+                if covered != e - s:
+                    raise PlanInvalid("tenant placement not wholly inside pin slots")
+                for (a, b, r) in tenants:
+                    if a < e and b > s and r >= first:
+                        raise PlanInvalid("two tenants overlap in place and time")
+                tenants.append((s, e, rel))
+                if t in stays and stays[t][1] >= first:
+                    raise PlanInvalid("tensor has two overlapping stays")
             else:
-                if arena_off < P["ring_base"]:
-                    raise PlanInvalid("ring placement inside the pin region")
                 if wait < ring_wait:
                     raise PlanInvalid("ring waits must be non-decreasing")
                 ring_wait = wait

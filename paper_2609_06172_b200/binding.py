@@ -20,8 +20,9 @@ T_READONLY, T_MUTABLE = 1, 2
 R, W = 1, 2
 PREFILL, DECODE = 0, 1
 VAR_EXPLICIT_RING, VAR_MANAGED_HINTS, VAR_MANAGED_DEMAND, VAR_MANAGED_OBJECT = 0, 1, 2, 3
-BIT_A, BIT_P, BIT_ZC = 1, 2, 4
+BIT_A, BIT_P, BIT_ZC, BIT_W = 1, 2, 4, 8
 X_CLASSES, X_TENSORS, X_PINS, X_COMMANDS, X_TOTALS = range(5)
+X_TAIL = 0x100
 # tensor kinds (TGP_K_*)
 (K_EMBED, K_G1, K_WQ, K_WK, K_WV, K_WO, K_G2, K_WG, K_WU, K_WD, K_GF, K_LM, K_ROUTER, K_KTILE, K_VTILE) = range(15)
 TAP_H, TAP_HF, TAP_Q, TAP_KTILE, TAP_VTILE, TAP_O, TAP_A = range(7)
@@ -76,6 +77,9 @@ _SIGS = {
     "tgp_set_object_bytes": [_P, _U64],
     "tgp_set_measured_times": [_P, C.POINTER(_U64), _U64],
     "tgp_plan": [_P],
+    "tgp_replan_begin": [_P, _U32, C.POINTER(_U64), _U64],
+    "tgp_replan_wait": [_P],
+    "tgp_replan_commit": [_P],
     "tgp_plan_export": [_P, _U32, _P, C.POINTER(_U64)],
     "tgp_set_arena": [_P, _P, _U64],
     "tgp_model_workspace_bytes": [C.POINTER(ModelCfg), _U32, C.POINTER(_U64)],
@@ -252,6 +256,20 @@ class Ctx:
         """The recorded trace decoded: a list of (step, site, layer, kind, flops, hbm bytes, [(tensor, mode, touched)])."""
         return parse_trace(self.trace_export())
 
+    def replan_begin(self, first_step, op_ns=None):
+        """Starts planning the steps from first_step on (helper thread); op_ns: uint64 per op of the whole trace, or None."""
+        if op_ns is None:
+            self._ck(lib().tgp_replan_begin(self._h, first_step, None, 0), "tgp_replan_begin")
+        else:
+            a = np.ascontiguousarray(op_ns, dtype=np.uint64)
+            self._ck(lib().tgp_replan_begin(self._h, first_step, a.ctypes.data_as(C.POINTER(_U64)), len(a)), "tgp_replan_begin")
+
+    def replan_wait(self):
+        self._ck(lib().tgp_replan_wait(self._h), "tgp_replan_wait")
+
+    def replan_commit(self):
+        self._ck(lib().tgp_replan_commit(self._h), "tgp_replan_commit")
+
     def set_budget(self, nbytes):
         self._ck(lib().tgp_set_budget(self._h, nbytes), "tgp_set_budget")
 
@@ -280,9 +298,11 @@ class Ctx:
         self._ck(lib().tgp_plan_export(self._h, what, buf, C.byref(n)), "tgp_plan_export")
         return buf.raw[:n.value]
 
-    def plan_blobs(self):
-        return {k: self.plan_export(w) for k, w in (("classes", X_CLASSES), ("tensors", X_TENSORS), ("pins", X_PINS),
-                                                    ("commands", X_COMMANDS), ("totals", X_TOTALS))}
+    def plan_blobs(self, tail=False):
+        """The plan in use as canonical blobs; tail=True: the tail plan that waits for replan_commit()."""
+        f = X_TAIL if tail else 0
+        return {k: self.plan_export(w | f) for k, w in (("classes", X_CLASSES), ("tensors", X_TENSORS), ("pins", X_PINS),
+                                                        ("commands", X_COMMANDS), ("totals", X_TOTALS))}
 
     def set_arena(self, arena, nbytes):
         self._ck(lib().tgp_set_arena(self._h, _ptr(arena), nbytes), "tgp_set_arena")

@@ -237,6 +237,10 @@ int tgp_run_reset(tgp_ctx *ctx) {
     if (!ctx || !ctx->eng) return TGP_E_STATE;
     CU(ctx, cudaDeviceSynchronize());
     TgpEngine *e = ctx->eng;
+    if (ctx->base_plan.valid) {                          // the run ended on a tail plan: the whole-run plan comes back
+        ctx->plan = std::move(ctx->base_plan);
+        ctx->base_plan = TgpPlan();
+    }
     e->next_cmd = 0; e->next_step = 0; e->pos = 0; e->wb_pending = false; e->copy_waited_op = -1; e->tok_src = nullptr;
     e->rr = 0;
     for (int i = 0; i < TgpEngine::NCOPY; ++i) { e->waited[i] = -1; e->wb_pend[i] = false; }
@@ -807,6 +811,39 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
         if (tgp_k_embed_status(&bad_tok, &bad_row, &bad_id) == TGP_OK && bad_tok)
             return tgp_fail(ctx, TGP_E_CUDA, "the embedding gather met token id " + std::to_string(bad_id) + " (row " + std::to_string(bad_row) + "), outside the vocabulary: that row was computed from zeros");
     }
+    return TGP_OK;
+}
+
+// Switches to the tail plan built by tgp_replan_begin() at its step boundary.  Stays never cross a step, so after the
+// device has drained the only data the arena alone holds are pinned tensors that were written: those go home, then the
+// tail plan starts from an empty arena.
+extern "C" int tgp_replan_commit(tgp_ctx *ctx) {
+    if (!ctx || !ctx->eng) return TGP_E_STATE;
+    TgpEngine *e = ctx->eng;
+    if (e->capturing) return tgp_fail(ctx, TGP_E_STATE, "a run being captured cannot switch plans");
+    int rc = tgp_replan_wait(ctx);
+    if (rc) return rc;
+    if (!ctx->tail_ready || !ctx->tail_plan.valid) return tgp_fail(ctx, TGP_E_STATE, "no re-plan to commit");
+    if (e->next_step != ctx->tail_plan.first_step) return tgp_fail(ctx, TGP_E_STATE, "the run is not at the boundary the re-plan was made for");
+    CU(ctx, cudaDeviceSynchronize());
+    std::vector<uint8_t> written(ctx->tensors.size(), 0);
+    for (uint32_t i = 0; i < ctx->tail_plan.first_op; ++i)
+        for (uint32_t k = 0; k < ctx->ops[i].nacc; ++k)
+            if (ctx->acc[ctx->ops[i].acc0 + k].mode & TGP_W) written[ctx->acc[ctx->ops[i].acc0 + k].tensor] = 1;
+    for (auto &pin : ctx->plan.pins) {
+        const TgpTensor &t = ctx->tensors[pin.first];
+        if (t.flags == TGP_T_MUTABLE && written[pin.first])
+            CU(ctx, cudaMemcpy(ctx->pools[t.pool].host_base + t.off, (char *)ctx->arena + pin.second, t.size, cudaMemcpyDeviceToHost));
+    }
+    if (!ctx->base_plan.valid) ctx->base_plan = std::move(ctx->plan);       // kept for the next tgp_run_reset()
+    ctx->plan = std::move(ctx->tail_plan);
+    ctx->tail_plan = TgpPlan();
+    ctx->tail_ready = false;
+    e->next_cmd = 0; e->wb_pending = false; e->copy_waited_op = -1; e->rr = 0;
+    for (int i = 0; i < TgpEngine::NCOPY; ++i) { e->waited[i] = -1; e->wb_pend[i] = false; }
+    uint64_t biggest = 0;
+    for (const TgpCmd &c : ctx->plan.cmds) if (c.kind == CMD_H2D && c.bytes > biggest) biggest = c.bytes;
+    e->n_copy = (biggest && biggest <= (512u << 10) && g_small_copy_streams) ? TgpEngine::NCOPY : 1;
     return TGP_OK;
 }
 

@@ -4,6 +4,7 @@
 #include <algorithm>
 #include <cstring>
 #include <deque>
+#include <thread>
 
 typedef unsigned __int128 u128;
 static const uint64_t ALIGN = 512;      // placement granularity in the arena
@@ -57,6 +58,7 @@ int tgp_create(tgp_ctx **out, const tgp_machine *m) {
 
 void tgp_destroy(tgp_ctx *ctx) {
     if (!ctx) return;
+    if (ctx->replan_thread.joinable()) ctx->replan_thread.join();
     tgp_engine_free(ctx);
     delete ctx;
 }
@@ -159,6 +161,8 @@ int tgp_tensor_identity(const tgp_ctx *ctx, uint32_t id, uint64_t *site_hash, ui
 // ---- trace ----------------------------------------------------------------------------------------
 int tgp_trace_begin(tgp_ctx *ctx) {
     if (!ctx) return TGP_E_INVAL;
+    if (ctx->replan_thread.joinable()) ctx->replan_thread.join();
+    ctx->tail_ready = false; ctx->base_plan = TgpPlan();
     ctx->ops.clear(); ctx->acc.clear(); ctx->steps.clear();
     ctx->measured_ns.clear();
     ctx->plan = TgpPlan();
@@ -216,12 +220,16 @@ int tgp_trace_export(const tgp_ctx *ctx, void *buf, uint64_t *bytes) {
 // ---- policy ---------------------------------------------------------------------------------------
 int tgp_set_budget(tgp_ctx *ctx, uint64_t bytes) {
     if (!ctx || !bytes) return TGP_E_INVAL;
+    if (ctx->replan_thread.joinable()) ctx->replan_thread.join();      // a re-plan under way reads these inputs
+    ctx->tail_ready = false;
     ctx->budget = bytes; ctx->plan.valid = false;
     return TGP_OK;
 }
 
 int tgp_set_measured_times(tgp_ctx *ctx, const uint64_t *op_ns, uint64_t n_ops) {
     if (!ctx) return TGP_E_INVAL;
+    if (ctx->replan_thread.joinable()) ctx->replan_thread.join();      // a re-plan under way reads these inputs
+    ctx->tail_ready = false;
     if (!n_ops) { ctx->measured_ns.clear(); ctx->plan.valid = false; return TGP_OK; }
     if (!op_ns) return TGP_E_INVAL;
     if (!ctx->traced || n_ops != ctx->ops.size()) return tgp_fail(ctx, TGP_E_STATE, "one time per op of the finished trace is required");
@@ -231,7 +239,9 @@ int tgp_set_measured_times(tgp_ctx *ctx, const uint64_t *op_ns, uint64_t n_ops) 
 }
 
 int tgp_set_variant(tgp_ctx *ctx, uint32_t variant, uint32_t bits) {
-    if (!ctx || variant > TGP_VAR_MANAGED_OBJECT || (bits & ~7u)) return TGP_E_INVAL;
+    if (!ctx || variant > TGP_VAR_MANAGED_OBJECT || (bits & ~15u)) return TGP_E_INVAL;
+    if (ctx->replan_thread.joinable()) ctx->replan_thread.join();      // a re-plan under way reads these inputs
+    ctx->tail_ready = false;
     ctx->variant = variant; ctx->bits = bits; ctx->plan.valid = false;
     return TGP_OK;
 }
@@ -255,16 +265,22 @@ static uint8_t classify(const tgp_machine &m, uint64_t flops, uint64_t hbm, uint
     return CLS_HBM;
 }
 
-int tgp_plan(tgp_ctx *ctx) {
-    if (!ctx) return TGP_E_INVAL;
-    if (!ctx->traced) return tgp_fail(ctx, TGP_E_STATE, "no finished trace");
-    if (!ctx->budget) return tgp_fail(ctx, TGP_E_STATE, "no budget set");
+}  // extern "C"
+
+// Builds the plan for the steps from first_step on (0: the whole run) into `out`; op indices are those of the whole
+// trace.  A tail plan starts from an empty arena with every tensor written in an earlier step holding data in the
+// pool (its first access loads it, write or not).  Touches nothing of ctx but `out` and `err`, so it may run on a
+// helper thread while tgp_step() executes the current plan.
+static int build_plan(const tgp_ctx *ctx, uint32_t first_step, TgpPlan &out, std::string &err) {
+    auto fail = [&](int code, const char *msg) { err = msg; return code; };
     const size_t T = ctx->tensors.size(), N = ctx->ops.size();
+    const size_t O0 = ctx->steps[first_step].op0;
     const std::vector<TgpTensor> &ten = ctx->tensors;
     TgpPlan pl;
+    pl.first_step = first_step; pl.first_op = (uint32_t)O0;
     pl.cls.resize(N); pl.crit.assign(T, 0); pl.zc.assign(T, 0); pl.score.assign(T, 0);
     // classes, criticality, score
-    for (size_t i = 0; i < N; ++i) {
+    for (size_t i = O0; i < N; ++i) {
         const TgpOp &o = ctx->ops[i];
         uint64_t mig = 0;
         for (uint32_t k = 0; k < o.nacc; ++k) mig += ctx->acc[o.acc0 + k].touched_bytes;
@@ -279,7 +295,8 @@ int tgp_plan(tgp_ctx *ctx) {
     // zero-copy: read-only, accessed, and every access sparse
     {
         std::vector<uint8_t> accessed(T, 0), sparse(T, 1);
-        for (const tgp_access &a : ctx->acc) {
+        for (size_t q = ctx->ops[O0].acc0; q < ctx->acc.size(); ++q) {
+            const tgp_access &a = ctx->acc[q];
             accessed[a.tensor] = 1;
             if ((u128)a.touched_bytes * ZC_DEN >= ten[a.tensor].size) sparse[a.tensor] = 0;
         }
@@ -291,7 +308,7 @@ int tgp_plan(tgp_ctx *ctx) {
     std::vector<std::vector<Stay>> stays(T);
     {
         std::vector<int32_t> last_op(T, -1);
-        for (size_t i = 0; i < N; ++i) {
+        for (size_t i = O0; i < N; ++i) {
             const TgpOp &o = ctx->ops[i];
             for (uint32_t k = 0; k < o.nacc; ++k) {
                 uint32_t t = ctx->acc[o.acc0 + k].tensor;
@@ -310,16 +327,17 @@ int tgp_plan(tgp_ctx *ctx) {
         for (size_t t = 0; t < T; ++t)
             for (const Stay &s : stays[t]) { delta[s.first] += (int64_t)alignup(ten[t].size); delta[s.last + 1] -= (int64_t)alignup(ten[t].size); }
         int64_t live = 0;
-        for (size_t i = 0; i < N; ++i) { live += delta[i]; wmax = std::max<uint64_t>(wmax, (uint64_t)live); }
+        for (size_t i = O0; i < N; ++i) { live += delta[i]; wmax = std::max<uint64_t>(wmax, (uint64_t)live); }
     }
     const uint64_t ring_min = 2 * wmax;
-    if (ring_min > ctx->budget) return tgp_fail(ctx, TGP_E_BUDGET_TOO_SMALL, "budget below twice the largest working set of one op");
+    if (ring_min > ctx->budget) return fail(TGP_E_BUDGET_TOO_SMALL, "budget below twice the largest working set of one op");
     const uint64_t pin_cap = ctx->budget - ring_min;
     // pins: greedy by density score/size, exact cross products, tie -> lower id, skip what does not fit
     std::vector<int64_t> pin_off(T, -1);
     uint64_t used = 0;
+    std::vector<uint32_t> cand_order;                    // pin candidates by falling density (kept for the tenants below)
     if (ctx->bits & TGP_BIT_A) {
-        std::vector<uint32_t> cand;
+        std::vector<uint32_t> &cand = cand_order;
         for (size_t t = 0; t < T; ++t) if (pl.score[t] > 0 && !pl.zc[t]) cand.push_back((uint32_t)t);
         std::sort(cand.begin(), cand.end(), [&](uint32_t a, uint32_t b) {
             u128 l = (u128)pl.score[a] * ten[b].size, r = (u128)pl.score[b] * ten[a].size;
@@ -351,6 +369,61 @@ int tgp_plan(tgp_ctx *ctx) {
     }
     for (size_t t = 0; t < T; ++t) if (pin_off[t] >= 0) pl.pins.push_back({(uint32_t)t, (uint64_t)pin_off[t]});
     pl.ring_base = used; pl.ring_size = ctx->budget - used;
+    // windowed reservation: the slot of a pinned tensor that is born on the device in a later step houses tenants until then
+    std::vector<int64_t> tenant_off(T, -1);
+    std::vector<int32_t> tenant_last(T, -1), landlord_wait(T, -1);
+    if ((ctx->bits & TGP_BIT_W) && !pl.pins.empty()) {
+        std::vector<uint8_t> written0(T, 0);
+        for (size_t i = 0; i < O0; ++i)
+            for (uint32_t k = 0; k < ctx->ops[i].nacc; ++k)
+                if (ctx->acc[ctx->ops[i].acc0 + k].mode & TGP_W) written0[ctx->acc[ctx->ops[i].acc0 + k].tensor] = 1;
+        std::vector<int32_t> first_op_of(T, -1);
+        std::vector<uint32_t> first_mode(T, 0);
+        for (size_t i = O0; i < N; ++i)
+            for (uint32_t k = 0; k < ctx->ops[i].nacc; ++k) {
+                const tgp_access &a = ctx->acc[ctx->ops[i].acc0 + k];
+                if (first_op_of[a.tensor] < 0) { first_op_of[a.tensor] = (int32_t)i; first_mode[a.tensor] = a.mode; }
+            }
+        struct Region { uint64_t start, end, fill; uint32_t birth; int32_t wait; std::vector<uint32_t> lords; };
+        std::vector<Region> regions;
+        std::vector<uint32_t> late;
+        for (auto &p : pl.pins) {
+            const uint32_t t = p.first;
+            if (ten[t].flags == TGP_T_MUTABLE && !written0[t] && first_mode[t] == TGP_W && ctx->ops[first_op_of[t]].step - first_step >= 2) late.push_back(t);
+        }
+        std::sort(late.begin(), late.end(), [&](uint32_t a, uint32_t b) { return pin_off[a] < pin_off[b]; });
+        for (uint32_t t : late) {
+            const uint64_t o = (uint64_t)pin_off[t], a = alignup(ten[t].size);
+            const uint32_t b = ctx->ops[first_op_of[t]].step;
+            if (!regions.empty() && regions.back().end == o && regions.back().birth == b) { regions.back().end = o + a; regions.back().lords.push_back(t); }
+            else regions.push_back({o, o + a, o, b, -1, {t}});
+        }
+        std::stable_sort(regions.begin(), regions.end(), [](const Region &x, const Region &y) { return x.birth != y.birth ? x.birth > y.birth : x.start < y.start; });
+        if (!regions.empty()) {
+            // accesses of each unpinned read-only candidate, in op order (only those are ever tenants)
+            std::vector<std::vector<int32_t>> acc_ops(T);
+            for (size_t i = O0; i < N; ++i)
+                for (uint32_t k = 0; k < ctx->ops[i].nacc; ++k) {
+                    const uint32_t t = ctx->acc[ctx->ops[i].acc0 + k].tensor;
+                    if (pin_off[t] < 0 && !pl.zc[t] && pl.score[t] > 0 && ten[t].flags == TGP_T_READONLY) acc_ops[t].push_back((int32_t)i);
+                }
+            for (uint32_t t : cand_order) {
+                if (pin_off[t] >= 0 || ten[t].flags != TGP_T_READONLY) continue;
+                const uint64_t a = alignup(ten[t].size);
+                for (Region &r : regions) {
+                    if (r.fill + a > r.end) continue;
+                    int32_t first = -1, last = -1;
+                    for (int32_t i : acc_ops[t]) { if (ctx->ops[i].step >= r.birth) break; if (first < 0) first = i; last = i; }
+                    if (first < 0 || ctx->ops[first].step == ctx->ops[last].step) continue;      // used in fewer than two steps of the vacancy
+                    tenant_off[t] = (int64_t)r.fill; tenant_last[t] = last;
+                    r.fill += a;
+                    r.wait = std::max(r.wait, last);
+                    break;
+                }
+            }
+            for (const Region &r : regions) for (uint32_t t : r.lords) landlord_wait[t] = r.wait;
+        }
+    }
     // schedule
     pl.totals.assign(ctx->steps.size() * 4, 0);
     pl.acc_where.assign(ctx->acc.size(), 0);
@@ -363,6 +436,9 @@ int tgp_plan(tgp_ctx *ctx) {
     std::vector<uint32_t> stay_idx(T, 0);
     std::vector<int64_t> open_at(T, -1);                 // arena offset of the open stay, -1 if none
     std::vector<uint8_t> pin_loaded(T, 0), written_ever(T, 0), dirty(T, 0);
+    for (size_t i = 0; i < O0; ++i)                      // a tail plan: what earlier steps wrote holds data in the pool
+        for (uint32_t k = 0; k < ctx->ops[i].nacc; ++k)
+            if (ctx->acc[ctx->ops[i].acc0 + k].mode & TGP_W) written_ever[ctx->acc[ctx->ops[i].acc0 + k].tensor] = 1;
     std::vector<int32_t> last_wb(T, -1);
     std::vector<std::vector<uint32_t>> ending(N);
     auto emit = [&](uint8_t kind, uint32_t t, uint64_t where, int32_t wait, int32_t first, int32_t rel) {
@@ -372,7 +448,7 @@ int tgp_plan(tgp_ctx *ctx) {
         if (kind == CMD_H2D) tot[0] += ten[t].size; else if (kind == CMD_D2H) tot[1] += ten[t].size;
         if (kind != CMD_D2H) pl.op_last_place[first] = (int32_t)pl.cmds.size() - 1;
     };
-    for (size_t i = 0; i < N; ++i) {
+    for (size_t i = O0; i < N; ++i) {
         const TgpOp &o = ctx->ops[i];
         for (uint32_t k = 0; k < o.nacc; ++k) {
             const tgp_access &a = ctx->acc[o.acc0 + k];
@@ -381,13 +457,22 @@ int tgp_plan(tgp_ctx *ctx) {
             bool mut = ten[t].flags == TGP_T_MUTABLE;
             bool fresh = mut && a.mode == TGP_W && !written_ever[t];
             if (pin_off[t] >= 0) {
-                if (!pin_loaded[t]) { pin_loaded[t] = 1; emit(fresh ? CMD_ALLOC : CMD_H2D, t, (uint64_t)pin_off[t], -1, (int32_t)i, (int32_t)N - 1); }
+                if (!pin_loaded[t]) {
+                    pin_loaded[t] = 1;
+                    emit(fresh ? CMD_ALLOC : CMD_H2D, t, (uint64_t)pin_off[t], landlord_wait[t], (int32_t)i, (int32_t)N - 1);
+                    if (landlord_wait[t] >= 0) pl.op_is_wait_target[landlord_wait[t]] = 1;
+                }
                 pl.acc_where[o.acc0 + k] = (uint64_t)pin_off[t];
+            } else if (tenant_off[t] >= 0 && (int32_t)i <= tenant_last[t]) {
+                // a tenant of a late-born pinned tensor's slot: loaded once, used there until its last access of the vacancy
+                if (!pin_loaded[t]) { pin_loaded[t] = 1; emit(CMD_H2D, t, (uint64_t)tenant_off[t], -1, (int32_t)i, tenant_last[t]); }
+                pl.acc_where[o.acc0 + k] = (uint64_t)tenant_off[t];
             } else {
                 if (open_at[t] < 0) {
+                    while (stays[t][stay_idx[t]].first < (int32_t)i) stay_idx[t]++;      // stays a tenancy made unnecessary
                     const Stay &s = stays[t][stay_idx[t]];
                     uint64_t sz = alignup(ten[t].size);
-                    if (sz > pl.ring_size) return tgp_fail(ctx, TGP_E_BUDGET_TOO_SMALL, "tensor larger than the ring");
+                    if (sz > pl.ring_size) return fail(TGP_E_BUDGET_TOO_SMALL, "tensor larger than the ring");
                     int32_t ev = -1;
                     if (head + sz > pl.ring_size) {                      // tail too short: skip it and wrap
                         while (!fifo.empty() && fifo.front().start >= head) { ev = std::max(ev, fifo.front().last_use); fifo.pop_front(); }
@@ -395,7 +480,7 @@ int tgp_plan(tgp_ctx *ctx) {
                     }
                     while (!fifo.empty() && fifo.front().start < head + sz && fifo.front().end > head) { ev = std::max(ev, fifo.front().last_use); fifo.pop_front(); }
                     run_wait = std::max(run_wait, std::max(ev, last_wb[t]));
-                    if (run_wait >= (int32_t)i) return tgp_fail(ctx, TGP_E_BUDGET_TOO_SMALL, "ring too small: a stay would wait on its own op");
+                    if (run_wait >= (int32_t)i) return fail(TGP_E_BUDGET_TOO_SMALL, "ring too small: a stay would wait on its own op");
                     fifo.push_back({head, head + sz, s.last});
                     open_at[t] = (int64_t)(pl.ring_base + head);
                     emit(fresh ? CMD_ALLOC : CMD_H2D, t, pl.ring_base + head, run_wait, (int32_t)i, s.last);
@@ -415,17 +500,62 @@ int tgp_plan(tgp_ctx *ctx) {
         }
     }
     pl.valid = true;
+    out = std::move(pl);
+    return TGP_OK;
+}
+
+extern "C" {
+
+int tgp_plan(tgp_ctx *ctx) {
+    if (!ctx) return TGP_E_INVAL;
+    if (!ctx->traced) return tgp_fail(ctx, TGP_E_STATE, "no finished trace");
+    if (!ctx->budget) return tgp_fail(ctx, TGP_E_STATE, "no budget set");
+    if (ctx->steps.empty() || ctx->ops.empty()) return tgp_fail(ctx, TGP_E_STATE, "empty trace");
+    if (ctx->replan_thread.joinable()) ctx->replan_thread.join();
+    ctx->tail_ready = false;
+    ctx->base_plan = TgpPlan();
+    TgpPlan pl;
+    std::string err;
+    const int rc = build_plan(ctx, 0, pl, err);
+    if (rc) return tgp_fail(ctx, rc, err);
     ctx->plan = std::move(pl);
+    return TGP_OK;
+}
+
+int tgp_replan_begin(tgp_ctx *ctx, uint32_t first_step, const uint64_t *op_ns, uint64_t n_ops) {
+    if (!ctx) return TGP_E_INVAL;
+    if (!ctx->plan.valid) return TGP_E_NO_PLAN;
+    if (ctx->variant != TGP_VAR_EXPLICIT_RING) return tgp_fail(ctx, TGP_E_STATE, "only the explicit engine re-plans in the middle of a run");
+    if (!first_step || first_step >= ctx->steps.size()) return tgp_fail(ctx, TGP_E_INVAL, "the boundary must lie between two steps of the trace");
+    if (first_step <= ctx->plan.first_step) return tgp_fail(ctx, TGP_E_INVAL, "the boundary must lie after the current plan's first step");
+    if (n_ops && (!op_ns || n_ops != ctx->ops.size())) return tgp_fail(ctx, TGP_E_INVAL, "one time per op of the whole trace is required");
+    if (ctx->replan_thread.joinable()) return tgp_fail(ctx, TGP_E_STATE, "a re-plan is already under way");
+    // the log is stored without touching the plan in use (tgp_set_measured_times() would invalidate it)
+    if (n_ops) ctx->measured_ns.assign(op_ns, op_ns + n_ops);
+    ctx->tail_ready = false; ctx->tail_rc = TGP_OK; ctx->tail_err.clear(); ctx->tail_step = first_step;
+    ctx->replan_thread = std::thread([ctx, first_step]() { ctx->tail_rc = build_plan(ctx, first_step, ctx->tail_plan, ctx->tail_err); });
+    return TGP_OK;
+}
+
+int tgp_replan_wait(tgp_ctx *ctx) {
+    if (!ctx) return TGP_E_INVAL;
+    if (!ctx->replan_thread.joinable()) return ctx->tail_ready ? TGP_OK : tgp_fail(ctx, TGP_E_STATE, "no re-plan under way");
+    ctx->replan_thread.join();
+    if (ctx->tail_rc) return tgp_fail(ctx, ctx->tail_rc, "re-plan: " + ctx->tail_err);
+    ctx->tail_ready = true;
     return TGP_OK;
 }
 
 int tgp_plan_export(const tgp_ctx *ctx, uint32_t what, void *buf, uint64_t *bytes) {
     if (!ctx) return TGP_E_INVAL;
-    if (!ctx->plan.valid) return TGP_E_NO_PLAN;
-    const TgpPlan &pl = ctx->plan;
+    const bool tail = what & TGP_X_TAIL;
+    what &= ~TGP_X_TAIL;
+    if (tail && (!ctx->tail_ready || !ctx->tail_plan.valid)) return TGP_E_NO_PLAN;
+    if (!tail && !ctx->plan.valid) return TGP_E_NO_PLAN;
+    const TgpPlan &pl = tail ? ctx->tail_plan : ctx->plan;
     std::vector<uint8_t> b;
     switch (what) {
-    case TGP_X_CLASSES: b = pl.cls; break;
+    case TGP_X_CLASSES: b.assign(pl.cls.begin() + pl.first_op, pl.cls.end()); break;
     case TGP_X_TENSORS:
         for (size_t t = 0; t < pl.crit.size(); ++t) { put<uint8_t>(b, pl.crit[t]); put<uint8_t>(b, pl.zc[t]); put<uint64_t>(b, pl.score[t]); }
         break;
@@ -442,7 +572,7 @@ int tgp_plan_export(const tgp_ctx *ctx, uint32_t what, void *buf, uint64_t *byte
         }
         break;
     case TGP_X_TOTALS:
-        for (uint64_t v : pl.totals) put<uint64_t>(b, v);
+        for (size_t k = (size_t)pl.first_step * 4; k < pl.totals.size(); ++k) put<uint64_t>(b, pl.totals[k]);
         break;
     default: return TGP_E_INVAL;
     }

@@ -5,6 +5,7 @@
 #include <vector>
 #include <map>
 #include <tuple>
+#include <thread>
 #include "tgp.h"
 
 struct TgpPool { char *host_base; uint64_t bytes; uint32_t flags; char *dev_alias; bool locked_by_us; };
@@ -29,6 +30,7 @@ enum { CLS_LINK = 0, CLS_HBM = 1, CLS_COMPUTE = 2 };
 
 struct TgpPlan {
     bool valid = false;
+    uint32_t first_step = 0, first_op = 0;   // > 0: a tail plan made at that step boundary; arrays below are still sized for the whole trace
     std::vector<uint8_t> cls, crit, zc;
     std::vector<uint64_t> score;
     std::vector<std::pair<uint32_t, uint64_t>> pins;
@@ -60,9 +62,16 @@ struct tgp_ctx {
     std::vector<TgpStep> steps;
     // policy inputs
     uint64_t budget = 0, object_bytes = 20ull << 20;
-    uint32_t variant = TGP_VAR_EXPLICIT_RING, bits = TGP_BIT_A | TGP_BIT_P | TGP_BIT_ZC;
+    uint32_t variant = TGP_VAR_EXPLICIT_RING, bits = TGP_BIT_A | TGP_BIT_P | TGP_BIT_ZC | TGP_BIT_W;
     std::vector<uint64_t> measured_ns;                   // runtime monitor: kernel time per op in ns (0 = not measured), or empty
     TgpPlan plan;
+    // re-plan of the remaining steps while the run is under way: built on a helper thread, swapped in at its boundary
+    TgpPlan tail_plan, base_plan;                        // base_plan: the whole-run plan set aside while a tail plan is in use
+    std::thread replan_thread;
+    bool tail_ready = false;
+    int tail_rc = 0;
+    uint32_t tail_step = 0;
+    std::string tail_err;
     // model
     bool bound = false;
     tgp_model_cfg cfg{};

@@ -37,7 +37,7 @@ class Session:
         self.ctx.model_bind(self.cfg, self.roles, router_bias)
         self.ctx.set_budget(layout.budget)
 
-    def plan(self, S=None, T=None, expert_counts=None, variant=tb.VAR_EXPLICIT_RING, bits=tb.BIT_A | tb.BIT_P | tb.BIT_ZC):
+    def plan(self, S=None, T=None, expert_counts=None, variant=tb.VAR_EXPLICIT_RING, bits=tb.BIT_A | tb.BIT_P | tb.BIT_ZC | tb.BIT_W):
         cfg = self.layout.cfg
         self.ctx.set_variant(variant, bits)
         self.ctx.model_trace(cfg.S if S is None else S, cfg.T if T is None else T, expert_counts)

@@ -30,7 +30,7 @@ def precision_floor(config):
     raise KeyError(config)
 
 
-def setup(cfg, budget=None, bits=7, n_dec=None, cap=None):
+def setup(cfg, budget=None, bits=15, n_dec=None, cap=None):
     lay = si.build_layout(cfg, budget=budget, cap=cap)
     pool = pinned_pool(lay.pool_bytes)
     si.fill_pool(lay, pool.numpy())
@@ -77,7 +77,7 @@ def test_oversubscribed_run_is_bitwise_equal_to_a_fully_resident_run(bits):
     prompt = si.prompt_tokens(cfg)
     forced = (np.arange(cfg.B * cfg.T, dtype=np.int32).reshape(cfg.B, cfg.T) * 911 + 3) % cfg.V
     outs = []
-    for budget, b in ((None, bits), (64 << 20, 7)):
+    for budget, b in ((None, bits), (64 << 20, 15)):
         lay, pool, s, blobs, T = setup(cfg, budget=budget, bits=b, cap=128 << 10)
         ops, steps = trace.run_trace(lay)
         validate.check(lay.tensors, ops, steps, lay.budget, blobs)
@@ -717,6 +717,86 @@ def test_runtime_monitor_replan_from_measured_kernel_times():
     for a, b in zip(before, after):
         assert np.array_equal(a, b)
     s.close()
+
+
+@pytest.mark.parametrize("budget", [None, 3 << 20])
+def test_replan_in_the_middle_of_a_run_switches_plans_at_a_step_boundary(budget):
+    """Runtime monitor while the run is under way: after decode step 3 the timing log so far is handed to the planner,
+    which plans steps 6.. on a helper thread while steps 4 and 5 still execute from the old plan; at the boundary the
+    engine drains, writes the written pinned KV tiles back and switches.  The tail schedule is bit for bit what the
+    oracle's tail planner gives for the same integer log and passes the validator; logits of every step equal those
+    of the un-switched run bit for bit; a reset brings the whole-run plan back."""
+    cfg = si.CONFIGS[1]
+    lay, pool, s, blobs, T = setup(cfg, budget=budget)
+    r = Runner(s, cfg.B * cfg.S)
+    prompt = si.prompt_tokens(cfg)
+    forced = (np.arange(cfg.B * T, dtype=np.int32).reshape(cfg.B, T) * 211 + 5) % cfg.V
+    plain, _ = r.generate(prompt, T, forced=forced)
+    ops, steps = trace.run_trace(lay)
+    boundary, measured_through = 6, 3
+    ns = np.zeros(len(ops), dtype=np.uint64)
+    got = []
+    r.reset()
+    s.ctx.set_op_timing(True)
+    for k in range(1 + T):
+        if k == measured_through + 1:
+            # the log so far; ops still to come take the time of the same op in the last measured decode step
+            s.ctx.set_op_timing(False)
+            o0, n = steps[measured_through][1], steps[measured_through][2]
+            for j in range(measured_through + 1, len(steps)):
+                assert steps[j][2] == n
+                ns[steps[j][1]: steps[j][1] + n] = ns[o0: o0 + n]
+            s.ctx.replan_begin(boundary, ns)                            # plans on a helper thread from here on
+        if k == boundary:
+            s.ctx.replan_commit()
+            tail = s.ctx.plan_blobs()
+        tok = prompt if k == 0 else np.ascontiguousarray(forced[:, k - 1:k], dtype=np.int32)
+        r.step(tb.PREFILL if k == 0 else tb.DECODE, tok, tok.shape[1], want_stats=True)
+        if k <= measured_through:
+            first, ms = s.ctx.op_times()
+            ns[first:first + len(ms)] = np.maximum(1, np.round(ms.astype(np.float64) * 1e6)).astype(np.uint64)
+        got.append(r.logits.cpu().numpy().copy())
+    r.sync()
+    want = policy.plan_tail(lay.tensors, ops, steps, policy.Machine(**MACHINE), lay.budget, boundary, measured_ns=ns.tolist()).blobs()
+    assert tail == want
+    validate.check(lay.tensors, ops, steps, lay.budget, tail, first_step=boundary)
+    assert tail["commands"] != blobs["commands"]
+    for a, b in zip(got, plain):
+        assert np.array_equal(a, b)
+    # the KV tiles the old plan had pinned were written back at the switch: the pool holds their data
+    old_pins = {t for t, _ in np.frombuffer(blobs["pins"][:-16], dtype=np.dtype([("t", "<u4"), ("o", "<u8")])).tolist()}
+    written = {t for o in ops[:steps[boundary][1]] for (t, m, _) in o.acc if m & 2}
+    host = pool.numpy()
+    assert old_pins & written
+    assert all(host[lay.tensors[t].pool_off: lay.tensors[t].pool_off + lay.tensors[t].size].any() for t in old_pins & written)
+    # after a reset the whole-run plan is in use again
+    again, _ = r.generate(prompt, T, forced=forced)
+    assert s.ctx.plan_blobs() == blobs
+    for a, b in zip(again, plain):
+        assert np.array_equal(a, b)
+    s.close()
+
+
+def test_windowed_pin_reservation_runs_bitwise_equal_to_a_resident_run():
+    """Slots of KV tiles that are born in later decode steps house weight blocks until then (tenants are loaded once,
+    used in place, and give the slot up before the tile's first write): the plan differs from the static one, moves
+    fewer bytes, equals the oracle's bit for bit, and the logits of all 41 steps equal those of a run with everything
+    resident."""
+    cfg = replace(si.CONFIGS[1], B=4, S=30, T=40, TK=16)
+    prompt = si.prompt_tokens(cfg)
+    forced = (np.arange(cfg.B * cfg.T, dtype=np.int32).reshape(cfg.B, cfg.T) * 733 + 1) % cfg.V
+    outs, moved = {}, {}
+    for name, budget, bits in (("windowed", None, 15), ("static", None, 7), ("resident", 64 << 20, 15)):
+        lay, pool, s, blobs, T = setup(cfg, budget=budget, bits=bits, cap=16 << 10)
+        ops, steps = trace.run_trace(lay)
+        assert blobs == policy.plan(lay.tensors, ops, steps, policy.Machine(**MACHINE), lay.budget, bits=bits).blobs()
+        validate.check(lay.tensors, ops, steps, lay.budget, blobs)
+        moved[name] = int(np.frombuffer(blobs["totals"], dtype="<u8").reshape(-1, 4)[:, 0].sum())
+        outs[name], _ = Runner(s, cfg.B * cfg.S).generate(prompt, T, forced=forced)
+        s.close()
+    assert moved["windowed"] < moved["static"]
+    for a, b, c in zip(outs["windowed"], outs["static"], outs["resident"]):
+        assert np.array_equal(a, c) and np.array_equal(b, c)
 
 
 def test_whole_run_cuda_graph_replays_bit_identically():

@@ -30,7 +30,7 @@ def pack_trace(ops):
     return b"".join(out)
 
 
-def oracle_blobs(lay, bits=7, expert_counts=None, budget=None):
+def oracle_blobs(lay, bits=15, expert_counts=None, budget=None):
     ops, steps = trace.run_trace(lay, expert_counts=expert_counts)
     pl = policy.plan(lay.tensors, ops, steps, policy.Machine(**MACHINE), budget or lay.budget, bits)
     return ops, steps, pl.blobs()
@@ -98,7 +98,7 @@ def test_plan_bit_exact_moe_reduced_and_full_shape():
     s.close()
 
 
-@pytest.mark.parametrize("bits", [0, tb.BIT_A, tb.BIT_P, tb.BIT_A | tb.BIT_P, tb.BIT_ZC, 7])
+@pytest.mark.parametrize("bits", [0, tb.BIT_A, tb.BIT_P, tb.BIT_A | tb.BIT_P, tb.BIT_ZC, 7, tb.BIT_W, 15])
 def test_plan_bit_exact_under_ablation_bits(bits):
     lay = si.build_layout(si.CONFIGS[1])
     s = Session(lay, MACHINE)
@@ -114,6 +114,37 @@ def test_plan_bit_exact_under_ablation_bits(bits):
         assert got[k] == want[k], (bits, k)
     validate.check(lay.tensors, ops, steps, lay.budget, got)
     s.close()
+
+
+@pytest.mark.parametrize("first_step", [0, 2, 20])
+def test_windowed_pin_reservation_is_bit_exact_and_moves_fewer_bytes(first_step):
+    """A long decode on a small model whose KV tiles (32 KiB) hold two 16 KiB weight blocks: the slots of the tiles born
+    in later decode steps house unpinned weight blocks until then.  Library and oracle agree bit for bit, with the bit
+    on and off, for the whole run and for a tail plan; the windowed plan passes the validator and moves fewer bytes."""
+    cfg = replace(si.CONFIGS[1], B=4, S=30, T=40, TK=16)
+    lay = si.build_layout(cfg, cap=16 << 10)
+    ops, steps = trace.run_trace(lay)
+    mach = policy.Machine(**MACHINE)
+    totals = {}
+    for bits in (7, 15):
+        s = Session(lay, MACHINE)
+        got = s.plan(bits=bits)
+        if first_step:
+            s.ctx.replan_begin(first_step)
+            s.ctx.replan_wait()
+            got = s.ctx.plan_blobs(tail=True)
+            want = policy.plan_tail(lay.tensors, ops, steps, mach, lay.budget, first_step, bits=bits).blobs()
+        else:
+            want = policy.plan(lay.tensors, ops, steps, mach, lay.budget, bits=bits).blobs()
+        for k in want:
+            assert got[k] == want[k], (bits, k)
+        validate.check(lay.tensors, ops, steps, lay.budget, got, first_step=first_step)
+        totals[bits] = int(np.frombuffer(got["totals"], dtype="<u8").reshape(-1, 4)[:, 0].sum())
+        s.close()
+    if first_step == 0:
+        assert totals[15] < totals[7]
+    else:
+        assert totals[15] <= totals[7]
 
 
 def test_library_plan_passes_the_validator_config_2():
@@ -283,6 +314,54 @@ def test_replan_from_a_timing_log_is_bit_exact_and_changes_classes():
     assert s.ctx.plan_blobs() == base
     with pytest.raises(tb.TgpError) as ei:
         s.ctx.set_measured_times(ns[:-1])
+    assert ei.value.code == tb.E_STATE
+    s.close()
+
+
+@pytest.mark.parametrize("c,first_step", [(1, 1), (1, 9), (2, 3)])
+def test_tail_replan_in_the_middle_of_a_run_is_bit_exact(c, first_step):
+    """Runtime monitor, second half: the steps from a boundary on are planned again, as a trace of their own, from the
+    timing log so far, on a helper thread.  The same integer log fed to the oracle's tail planner gives the same blobs;
+    the tail plan passes the validator started from an empty arena with the earlier steps' writes in the pool."""
+    cfg = si.CONFIGS[c] if c == 1 else replace(si.CONFIGS[c], T=6)
+    lay = si.build_layout(cfg)
+    ops, steps = trace.run_trace(lay)
+    first_op = steps[first_step][1]
+    rng = np.random.default_rng(first_step)
+    ns = np.zeros(len(ops), dtype=np.uint64)
+    ns[:first_op] = rng.integers(500, 40000, first_op)                    # measured so far
+    # ops still to come: the time of the same op in the last measured step of the same kind, where there is one
+    if first_step >= 2:
+        o0, n = steps[first_step - 1][1], steps[first_step - 1][2]
+        for k in range(first_step, len(steps)):
+            if steps[k][2] == n:
+                ns[steps[k][1]: steps[k][1] + n] = ns[o0: o0 + n]
+    s = Session(lay, MACHINE)
+    base = s.plan(T=cfg.T)
+    s.ctx.replan_begin(first_step, ns)
+    s.ctx.replan_wait()
+    got = s.ctx.plan_blobs(tail=True)
+    assert s.ctx.plan_blobs() == base                                     # the plan in use is untouched until the commit
+    want = policy.plan_tail(lay.tensors, ops, steps, policy.Machine(**MACHINE), lay.budget, first_step, measured_ns=ns.tolist()).blobs()
+    assert got == want
+    validate.check(lay.tensors, ops, steps, lay.budget, got, first_step=first_step)
+    assert len(got["classes"]) == len(ops) - first_op and len(got["totals"]) == 32 * (len(steps) - first_step)
+    # without a log the tail plan is the analytic one
+    s.ctx.set_measured_times(None)
+    s.ctx.plan()
+    s.ctx.replan_begin(first_step)
+    s.ctx.replan_wait()
+    assert s.ctx.plan_blobs(tail=True) == policy.plan_tail(lay.tensors, ops, steps, policy.Machine(**MACHINE), lay.budget, first_step).blobs()
+    # call-order and argument errors are codes
+    for bad in (0, len(steps)):
+        with pytest.raises(tb.TgpError) as ei:
+            s.ctx.replan_begin(bad)
+        assert ei.value.code == tb.E_INVAL
+    with pytest.raises(tb.TgpError) as ei:
+        s.ctx.replan_begin(first_step, ns[:-1])
+    assert ei.value.code == tb.E_INVAL
+    with pytest.raises(tb.TgpError) as ei:
+        s.ctx.replan_commit()                                             # no engine without a device
     assert ei.value.code == tb.E_STATE
     s.close()
 

@@ -240,3 +240,116 @@ def test_hold_window_keeps_short_reuse_in_place():
     assert kinds == [(policy.CMD_H2D, 0, 0, 2), (policy.CMD_H2D, 1, 1, 1), (policy.CMD_H2D, 0, 8, 8),
                      (policy.CMD_ALLOC, 2, 9, 10), (policy.CMD_D2H, 2, 10, 10)]
     validate.check(tensors, ops, [(0, 0, len(ops))], 6 * size, pl.blobs())
+
+
+def test_tail_plan_closed_forms_and_invariants():
+    """A plan made at a step boundary for the rest of the run: (1) it passes the validator started from an empty arena;
+    (2) a KV tile written before the boundary is loaded (H2D), never allocated, at its first access in the tail - a
+    tile first written after the boundary is still born on the device; (3) with nothing measured, classes of the tail
+    equal the whole-run plan's classes for those ops, and a steady decode step of the tail moves the same bytes as the
+    same step of the whole-run plan (same pin capacity, same per-step accesses); (4) a boundary at step 0 is the
+    whole-run plan itself."""
+    cfg = replace(si.CONFIGS[1], S=30, T=8)             # TK = 16: positions 30, 31 fill tile 1; tile 2 is born at decode step 3
+    lay = si.build_layout(cfg)
+    ops, steps = trace.run_trace(lay)
+    whole = policy.plan(lay.tensors, ops, steps, M, lay.budget)
+    assert policy.plan_tail(lay.tensors, ops, steps, M, lay.budget, 0).blobs() == whole.blobs()
+    for k in (1, 2, 3, 4, 8):
+        tail = policy.plan_tail(lay.tensors, ops, steps, M, lay.budget, k)
+        validate.check(lay.tensors, ops, steps, lay.budget, tail.blobs(), first_step=k)
+        first_op = steps[k][1]
+        assert tail.cls == whole.cls[first_op:]
+        written = {t for o in ops[:first_op] for (t, m, _) in o.acc if m & 2}
+        later = {t for o in ops[first_op:] for (t, m, _) in o.acc if m & 2} - written
+        kinds = {}
+        for c in tail.cmds:
+            if c.kind != policy.CMD_D2H:
+                kinds.setdefault(c.tensor, c.kind)
+        assert all(kinds[t] == policy.CMD_H2D for t in written if t in kinds)
+        assert all(kinds[t] == policy.CMD_ALLOC for t in later)
+        assert (k <= 3) == bool(later)                  # tile 2 of every layer is first written in decode step 3
+        assert min(c.first_use for c in tail.cmds) >= first_op and all(c.wait_op == -1 or c.wait_op >= first_op for c in tail.cmds)
+        if k <= 6:
+            assert tail.totals[-1][0] == whole.totals[-1][0]
+    # a tampered tail plan that allocates a tile holding data is caught
+    tail = policy.plan_tail(lay.tensors, ops, steps, M, lay.budget, 4)
+    blobs = tail.blobs()
+    kv = next(c.seq for c in tail.cmds if lay.tensors[c.tensor].flags == si.F_MUTABLE and c.kind == policy.CMD_H2D)
+    def to_alloc(cmds):
+        cmds[kv][1] = policy.CMD_ALLOC
+    with pytest.raises(validate.PlanInvalid):
+        validate.check(lay.tensors, ops, steps, lay.budget, _tamper(blobs, to_alloc), first_step=4)
+
+
+def _window_toy(n_w=5, born=3, n_steps=6, size=4096):
+    """n_w read-only tensors read once per step, and one mutable tensor of the same size first written in step `born`
+    and read and written in every step after it (a KV tile of later positions)."""
+    tensors = [_T(size, k * size) for k in range(n_w)] + [_T(size, n_w * size, flags=2)]
+    ops, steps = [], []
+    for st in range(n_steps):
+        o0 = len(ops)
+        for t in range(n_w):
+            ops.append(_O(st, 10, 10, [(t, 1, size)]))
+            ops += [_O(st, 10, 10, []) for _ in range(policy.W_AFF + 1)]
+        if st >= born:
+            ops.append(_O(st, 10, 10, [(n_w, 2, size)]))
+            ops.append(_O(st, 10, 10, [(n_w, 1, size)]))
+        steps.append((1 if st else 0, o0, len(ops) - o0))
+    return tensors, ops, steps
+
+
+def test_windowed_reservation_matches_brute_force_on_a_toy_run():
+    """The late-born tensor is the densest (a write costs its write-back too), so it is pinned; its slot is idle for the
+    first `born` steps.  Static reservation leaves it empty; windowed reservation lends it to the densest unpinned
+    tensor, which is then loaded once instead of once per step.  Brute force over every way to use the idle slot (any one
+    read-only tensor, or none) gives the same minimum."""
+    size = 4096
+    for born in (2, 3, 5):
+        tensors, ops, steps = _window_toy(born=born, n_steps=born + 4)
+        n_w = len(tensors) - 1
+        budget = 2 * size + 2 * size                       # ring of two tensors, room for two pins
+        static = policy.plan(tensors, ops, steps, M, budget, bits=7)
+        windowed = policy.plan(tensors, ops, steps, M, budget, bits=15)
+        validate.check(tensors, ops, steps, budget, static.blobs())
+        validate.check(tensors, ops, steps, budget, windowed.blobs())
+        assert [t for t, _ in static.pins] == [t for t, _ in windowed.pins] and n_w in dict(static.pins)
+        h_static = sum(t[0] for t in static.totals)
+        h_win = sum(t[0] for t in windowed.totals)
+        # by hand: one pinned weight is loaded once, the others every step; the tenant saves (born - 1) loads
+        n_steps = len(steps)
+        assert h_static == size * (1 + (n_w - 1) * n_steps)
+        assert h_win == h_static - size * (born - 1)
+        # brute force: the idle slot holds tensor x (or nothing) during steps [0, born)
+        pinned_w = [t for t, _ in static.pins if t != n_w][0]
+        best = min(h_static - (size * (born - 1) if x is not None else 0) for x in [None] + [t for t in range(n_w) if t != pinned_w])
+        assert h_win == best
+        # the tenant is the first unpinned tensor in density order (equal densities: lowest id), placed at the landlord's slot
+        ten = [c for c in windowed.cmds if c.tensor != n_w and c.tensor not in dict(windowed.pins) and c.arena_off < windowed.ring_base]
+        assert len(ten) == 1 and ten[0].arena_off == dict(windowed.pins)[n_w] and ten[0].tensor == min(t for t in range(n_w) if t != pinned_w)
+        # the landlord's placement waits for the tenant's last use
+        lord = [c for c in windowed.cmds if c.tensor == n_w and c.kind == policy.CMD_ALLOC][0]
+        assert lord.wait_op == ten[0].release_after and lord.wait_op < lord.first_use
+    # born in step 1: the vacancy is the cold first step only, nothing to save, plans are identical
+    tensors, ops, steps = _window_toy(born=1)
+    assert policy.plan(tensors, ops, steps, M, 4 * 4096, bits=7).blobs() == policy.plan(tensors, ops, steps, M, 4 * 4096, bits=15).blobs()
+
+
+def test_validator_rejects_broken_tenancies():
+    tensors, ops, steps = _window_toy(born=3)
+    budget = 4 * 4096
+    pl = policy.plan(tensors, ops, steps, M, budget, bits=15)
+    good = pl.blobs()
+    validate.check(tensors, ops, steps, budget, good)
+    n_w = len(tensors) - 1
+    lord = next(c.seq for c in pl.cmds if c.tensor == n_w and c.kind == policy.CMD_ALLOC)
+    ten = next(c.seq for c in pl.cmds if c.tensor not in dict(pl.pins) and c.arena_off < pl.ring_base)
+    other_pin = next(o for t, o in pl.pins if t != n_w)
+    def early_landlord(cmds):                 # the pinned tensor takes its slot while the tenant is still in use
+        cmds[lord][6] = -1
+    def on_a_resident_pin(cmds):              # a tenant placed over a pinned tensor that is there
+        cmds[ten][5] = other_pin
+    def overstays(cmds):                      # the tenant claims the slot beyond the landlord's birth
+        cmds[ten][8] = cmds[lord][7] + 1
+    for fn in (early_landlord, on_a_resident_pin, overstays):
+        with pytest.raises(validate.PlanInvalid):
+            validate.check(tensors, ops, steps, budget, _tamper(good, fn))
