@@ -312,9 +312,12 @@ int  tgp_k_gemm_select(int impl);
  * than 4096 rows): 0 (default) the weight-streaming tensor-core kernel, 1 the
  * CUDA-core GEMV (M <= 16) / GEMM paths (an on-device cross-check).  Process-wide. */
 int  tgp_k_skinny_select(int impl);
-/* Weight-streaming launches (M <= 32) use programmatic dependent launch so that a launch may begin reading its
- * weights while the previous kernel of the stream drains; 0 switches that off (each launch then starts after the
- * previous one has completed).  Results are identical either way.  Process-wide; default on. */
+/* Weight-streaming launches (M <= 32) and the small kernels of a step (embedding gather, RMSNorm, RoPE + KV append, decode
+ * attention and its merge, SwiGLU, argmax) use programmatic dependent launch: a launch lets its successor be scheduled
+ * at once; a weight-streaming kernel starts reading its weights while the previous kernel of the stream drains and
+ * waits for it only before it touches activations or output, a small kernel waits first thing, so that only its launch
+ * latency overlaps.  0 switches that off (each launch then starts after the previous one has completed).  Results are
+ * identical either way.  Process-wide; default on. */
 int  tgp_k_gemv_overlap(int enable);
 /* Tensor-core GEMM variant: 0 (default) picks by problem size, 1 forces the 128x128 one-tile-per-CTA kernel,
  * 2 the persistent 128x256 kernel with double-buffered accumulators, 3 the paired kernel (256x256 tiles on the two SMs

@@ -31,12 +31,44 @@ __device__ __forceinline__ float warp_max(float v) {
     return v;
 }
 
+// Activations are produced by the grid under which this one may already have been launched (programmatic dependent
+// launch), so they are read with an ordinary load after griddepcontrol.wait - never through the read-only path
+// (ld.global.nc, what __ldg and const __restrict__ pointers compile to), whose cached lines may predate the wait and
+// were seen to serve the previous layer's values.  The activation pointers of these kernels are therefore not
+// __restrict__, and the load is a plain one (an asm volatile load costs the M <= 2 kernel a tenth of its speed, an
+// L2-only load a third).
+__device__ __forceinline__ uint4 ld_act(const uint4 *p) { return *p; }
+
+// Programmatic dependent launch for the small kernels of a decode step: the grid lets its successor be scheduled at
+// once and then waits for its predecessor to complete and flush, before it reads anything - the dependency is the full
+// one, but the successor's launch latency (a microsecond or two, as long as these kernels run) overlaps this grid's
+// execution.  Every thread of every kernel launched through launch_pdl() executes this first.
+__device__ __forceinline__ void pdl_enter() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+static int g_small_pdl = 1;      // small kernels are launched as programmatic dependents of their predecessor (0: plain launches)
+
+template <typename... KArgs, typename... Args>
+static void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = g_small_pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- embedding gather ------------------------------------------------------------------------
 // A token id outside [0, V) would index past the table (which may be mapped host memory): such a row is written as
 // zeros and the first offending (row, id) is recorded in g_embed_error for tgp_k_embed_status().
 __device__ unsigned long long g_embed_error = 0;      // 0, or 1 << 63 | row << 32 | (uint32_t)id of the first bad token
 
-__global__ void tgp_embed_kernel(const bf16 *__restrict__ table, const int32_t *__restrict__ tok, float *__restrict__ x, uint32_t d, uint32_t V) {
+__global__ void tgp_embed_kernel(const bf16 *__restrict__ table, const int32_t *tok, float *x, uint32_t d, uint32_t V) {
+    pdl_enter();
     const uint32_t m = blockIdx.x;
     const int32_t id = tok[m];
     float4 *out = reinterpret_cast<float4 *>(x + (size_t)m * d);
@@ -55,7 +87,8 @@ __global__ void tgp_embed_kernel(const bf16 *__restrict__ table, const int32_t *
 }
 
 // ---- RMSNorm -> bf16 -------------------------------------------------------------------------
-__global__ void tgp_rmsnorm_kernel(const float *__restrict__ x, uint32_t ldx, const bf16 *__restrict__ g, bf16 *__restrict__ h, uint32_t d, float eps) {
+__global__ void tgp_rmsnorm_kernel(const float *x, uint32_t ldx, const bf16 *__restrict__ g, bf16 *h, uint32_t d, float eps) {
+    pdl_enter();
     __shared__ float red[32];
     const float4 *row = reinterpret_cast<const float4 *>(x + (size_t)blockIdx.x * ldx);
     float ss = 0.f;
@@ -86,7 +119,7 @@ __global__ void tgp_rmsnorm_kernel(const float *__restrict__ x, uint32_t ldx, co
 // No block barrier and no shared memory, so no SM idles while another warp reduces; the summation order
 // is fixed (lane-strided partials, butterfly), hence results are deterministic run to run.
 template <int MT, int R, int U>
-__global__ void __launch_bounds__(256) tgp_wstream_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+__global__ void __launch_bounds__(256) tgp_wstream_kernel(const bf16 *A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                    uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarp = (gridDim.x * blockDim.x) >> 5;
@@ -118,7 +151,7 @@ __global__ void __launch_bounds__(256) tgp_wstream_kernel(const bf16 *__restrict
 #pragma unroll
                 for (int m = 0; m < MT; ++m) {
                     float xf[8];
-                    unpack8((k < K && m < (int)Mrows) ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)) : make_uint4(0, 0, 0, 0), xf);
+                    unpack8((k < K && m < (int)Mrows) ? ld_act(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)) : make_uint4(0, 0, 0, 0), xf);
 #pragma unroll
                     for (int r = 0; r < R; ++r) {
                         float wf[8];
@@ -152,7 +185,7 @@ __global__ void __launch_bounds__(256) tgp_wstream_kernel(const bf16 *__restrict
 struct GemvParts { const bf16 *W[TGP_GEMM_GROUP_MAX]; float *C[TGP_GEMM_GROUP_MAX]; uint32_t n[TGP_GEMM_GROUP_MAX], ldc[TGP_GEMM_GROUP_MAX], groups[TGP_GEMM_GROUP_MAX], count; };
 
 template <int MT, int U>
-__global__ void __launch_bounds__(256) tgp_wstream_group_kernel(const bf16 *__restrict__ A, const GemvParts p, uint32_t Mrows, uint32_t n_total, uint32_t K, int accumulate) {
+__global__ void __launch_bounds__(256) tgp_wstream_group_kernel(const bf16 *A, const GemvParts p, uint32_t Mrows, uint32_t n_total, uint32_t K, int accumulate) {
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarp = (gridDim.x * blockDim.x) >> 5;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -185,7 +218,7 @@ __global__ void __launch_bounds__(256) tgp_wstream_group_kernel(const bf16 *__re
 #pragma unroll
                 for (int m = 0; m < MT; ++m) {
                     float xf[8];
-                    unpack8((k < K && m < (int)Mrows) ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)) : make_uint4(0, 0, 0, 0), xf);
+                    unpack8((k < K && m < (int)Mrows) ? ld_act(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)) : make_uint4(0, 0, 0, 0), xf);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) acc[m] = fmaf(wf[i], xf[i], acc[m]);
                 }
@@ -208,7 +241,7 @@ __global__ void __launch_bounds__(256) tgp_wstream_group_kernel(const bf16 *__re
 // rows leave a quarter of them with half the work.  The 8 partial sums of a row meet in shared memory and are added in
 // warp order: deterministic.  Same dependent-launch protocol.
 template <int MT, int RB, int U>
-__global__ void __launch_bounds__(256) tgp_wstream_splitk_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+__global__ void __launch_bounds__(256) tgp_wstream_splitk_kernel(const bf16 *A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                           uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     __shared__ float part[8][RB * MT];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -238,7 +271,7 @@ __global__ void __launch_bounds__(256) tgp_wstream_splitk_kernel(const bf16 *__r
 #pragma unroll
                 for (int m = 0; m < MT; ++m) {
                     float xf[8];
-                    unpack8((k < K && m < (int)Mrows) ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)) : make_uint4(0, 0, 0, 0), xf);
+                    unpack8((k < K && m < (int)Mrows) ? ld_act(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)) : make_uint4(0, 0, 0, 0), xf);
 #pragma unroll
                     for (int r = 0; r < RB; ++r) {
                         float wf[8];
@@ -283,7 +316,7 @@ __device__ __forceinline__ void mma_bf16_16816(float *d, uint32_t a0, uint32_t a
 }
 
 template <int NB, int U>
-__global__ void __launch_bounds__(256) tgp_wstream_mma_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+__global__ void __launch_bounds__(256) tgp_wstream_mma_kernel(const bf16 *A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                        uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     const uint32_t lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
     const uint32_t gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarp = (gridDim.x * blockDim.x) >> 5;
@@ -310,7 +343,7 @@ __global__ void __launch_bounds__(256) tgp_wstream_mma_kernel(const bf16 *__rest
 #pragma unroll
                 for (int b = 0; b < NB; ++b) {
                     const uint32_t m = b * 8 + g;
-                    const uint4 xv = (k < K && m < Mrows) ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k + c * 8)) : make_uint4(0, 0, 0, 0);
+                    const uint4 xv = (k < K && m < Mrows) ? ld_act(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k + c * 8)) : make_uint4(0, 0, 0, 0);
                     mma_bf16_16816(acc[b], lo[u].x, hi[u].x, lo[u].y, hi[u].y, xv.x, xv.y);
                     mma_bf16_16816(acc[b], lo[u].z, hi[u].z, lo[u].w, hi[u].w, xv.z, xv.w);
                 }
@@ -332,7 +365,7 @@ __global__ void __launch_bounds__(256) tgp_wstream_mma_kernel(const bf16 *__rest
 }
 
 // ---- generic tiled GEMM on CUDA cores (any M, n; K % 8 == 0): 64x64 tile, 4x4 per thread ---------
-__global__ void __launch_bounds__(256) tgp_matmul_simt_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+__global__ void __launch_bounds__(256) tgp_matmul_simt_kernel(const bf16 *A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                         uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     __shared__ float As[32][64 + 4];
     __shared__ float Ws[32][64 + 4];
@@ -378,6 +411,7 @@ struct RopeArgs {
 };
 
 __global__ void tgp_rope_kv_kernel(RopeArgs a) {
+    pdl_enter();
     const uint32_t m = blockIdx.x, b = m / a.q_len, pos = a.pos0 + m % a.q_len;
     const uint32_t half = a.Dh / 2, qd = a.Hq * a.Dh, kd = a.Hkv * a.Dh;
     const float *cs = a.cos_t + (size_t)pos * half, *sn = a.sin_t + (size_t)pos * half;
@@ -475,6 +509,7 @@ __global__ void __launch_bounds__(128) tgp_attn_rows_kernel(AttnArgs a) {
 // meet in shared memory and one unnormalised partial per (query head, tile) goes to scratch.
 template <int DH>
 __global__ void tgp_attn_decode_partial_kernel(AttnArgs a, uint32_t SPLIT) {
+    pdl_enter();
     extern __shared__ float dsm[];
     const uint32_t G = a.Hq / a.Hkv;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -563,6 +598,7 @@ __global__ void tgp_attn_decode_partial_kernel(AttnArgs a, uint32_t SPLIT) {
 // per-head kernel: (max, sum, unnormalised o[DH]) per (sequence, head, tile) for tgp_attn_decode_merge_kernel.
 template <int DH, int G>
 __global__ void __launch_bounds__(256, 2) tgp_attn_decode_group_kernel(AttnArgs a, uint32_t SPLIT) {
+    pdl_enter();
     extern __shared__ float dsm[];
     constexpr int DPL = DH / 32;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -699,6 +735,7 @@ __global__ void __launch_bounds__(256, 2) tgp_attn_decode_group_kernel(AttnArgs 
 
 template <int DH>
 __global__ void tgp_attn_decode_merge_kernel(AttnArgs a) {
+    pdl_enter();
     const uint32_t hq = blockIdx.x, b = blockIdx.y, i = threadIdx.x;
     const uint32_t nt = (a.pos0 + 1 + a.TK - 1) / a.TK;
     const float *part = a.scratch + (size_t)(b * a.Hq + hq) * a.n_tiles * (DH + 2);
@@ -714,7 +751,8 @@ __global__ void tgp_attn_decode_merge_kernel(AttnArgs a) {
 }
 
 // ---- SwiGLU -----------------------------------------------------------------------------------------
-__global__ void tgp_swiglu_kernel(const float4 *__restrict__ g, const float4 *__restrict__ u, __nv_bfloat162 *__restrict__ out, uint64_t n4) {
+__global__ void tgp_swiglu_kernel(const float4 *g, const float4 *u, __nv_bfloat162 *out, uint64_t n4) {
+    pdl_enter();
     for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n4; i += (uint64_t)gridDim.x * blockDim.x) {
         float4 a = g[i], b = u[i];
         float r0 = a.x / (1.0f + expf(-a.x)) * b.x, r1 = a.y / (1.0f + expf(-a.y)) * b.y;
@@ -725,7 +763,8 @@ __global__ void tgp_swiglu_kernel(const float4 *__restrict__ g, const float4 *__
 }
 
 // ---- argmax, lowest index on ties -----------------------------------------------------------------
-__global__ void __launch_bounds__(1024) tgp_argmax_kernel(const float *__restrict__ logits, int32_t *__restrict__ out, uint32_t V) {
+__global__ void __launch_bounds__(1024) tgp_argmax_kernel(const float *logits, int32_t *out, uint32_t V) {
+    pdl_enter();
     __shared__ float bv[32];
     __shared__ uint32_t bi[32];
     const float *row = logits + (size_t)blockIdx.x * V;
@@ -875,7 +914,7 @@ int tgpk_scatter_add(float *x, const float *y, const int32_t *rows, const float 
 int tgpk_embed(const void *table, const int32_t *tok, float *x, uint32_t M, uint32_t d, uint32_t V, cudaStream_t st) {
     if (!M) return TGP_OK;
     if (d % 8 || !V) return TGP_E_INVAL;
-    tgp_embed_kernel<<<M, 128, 0, st>>>((const bf16 *)table, tok, x, d, V);
+    launch_pdl(tgp_embed_kernel, dim3(M), dim3(128), 0, st, (const bf16 *)table, tok, x, d, V);
     LAUNCH_CHECK(1);
     return TGP_OK;
 }
@@ -883,7 +922,7 @@ int tgpk_embed(const void *table, const int32_t *tok, float *x, uint32_t M, uint
 int tgpk_rmsnorm(const float *x, uint32_t ldx, const void *g, void *h, uint32_t M, uint32_t d, float eps, cudaStream_t st) {
     if (!M) return TGP_OK;
     if (d % 4 || ldx % 4) return TGP_E_INVAL;
-    tgp_rmsnorm_kernel<<<M, 256, 0, st>>>(x, ldx, (const bf16 *)g, (bf16 *)h, d, eps);
+    launch_pdl(tgp_rmsnorm_kernel, dim3(M), dim3(256), 0, st, x, ldx, (const bf16 *)g, (bf16 *)h, d, eps);
     LAUNCH_CHECK(1);
     return TGP_OK;
 }
@@ -926,7 +965,7 @@ static void launch_gemv(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, 
 // RPC <= ROWS: rows a CTA owns (the tile's remaining rows re-read its last row and are not stored; a row's sum does not
 // depend on its place in the tile).  14 of 16 turns the 256 CTAs of a 4096-row block into 293, two for every SM.
 template <int NB, int U, int NW, int ROWS, int RPC = ROWS>
-__global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_splitk_kernel(const bf16 *__restrict__ A, const bf16 *__restrict__ W, float *__restrict__ C,
+__global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_splitk_kernel(const bf16 *A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                               uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
     constexpr int UL = ROWS == 8 ? 2 * U : U;             // half a tile per load step: twice the steps in flight
     __shared__ float part[NW][NB * 4][32];
@@ -955,7 +994,7 @@ __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_splitk_kernel(const b
 #pragma unroll
                 for (int b = 0; b < NB; ++b) {
                     const uint32_t m = b * 8 + g;
-                    const uint4 xv = (k < K && m < Mrows) ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k + c * 8)) : make_uint4(0, 0, 0, 0);
+                    const uint4 xv = (k < K && m < Mrows) ? ld_act(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k + c * 8)) : make_uint4(0, 0, 0, 0);
                     mma_bf16_16816(acc[b], lo[u].x, hi[u].x, lo[u].y, hi[u].y, xv.x, xv.y);
                     mma_bf16_16816(acc[b], lo[u].z, hi[u].z, lo[u].w, hi[u].w, xv.z, xv.w);
                 }
@@ -990,7 +1029,7 @@ __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_splitk_kernel(const b
 // (which warp adds which k, in which order) is that of tgp_wstream_mma_splitk_kernel<NB, U, NW, ROWS> whatever RG and the list:
 // same bits as one launch per block.
 template <int NB, int U, int NW, int ROWS, int RG>
-__global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_group_kernel(const bf16 *__restrict__ A, const GemvParts p, uint32_t Mrows, uint32_t groups_total,
+__global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_group_kernel(const bf16 *A, const GemvParts p, uint32_t Mrows, uint32_t groups_total,
                                                               uint32_t K, int accumulate, uint32_t rpc) {
     constexpr int UL = ROWS == 8 ? 2 * U : U;             // half a tile per load step: twice the steps in flight
     constexpr int G = RG, SUB = UL / G;                  // SUB load steps of G groups in flight at a time: as many loads as UL of one
@@ -1049,7 +1088,7 @@ __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_group_kernel(const bf
 #pragma unroll
                     for (int b = 0; b < NB; ++b) {
                         const uint32_t m = b * 8 + g;
-                        const uint4 xv = (k < K && m < Mrows) ? __ldg(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k + c * 8)) : make_uint4(0, 0, 0, 0);
+                        const uint4 xv = (k < K && m < Mrows) ? ld_act(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k + c * 8)) : make_uint4(0, 0, 0, 0);
 #pragma unroll
                         for (int r = 0; r < G; ++r) {
                             mma_bf16_16816(acc[r][b], lo[r][u].x, hi[r][u].x, lo[r][u].y, hi[r][u].y, xv.x, xv.y);
@@ -1359,7 +1398,7 @@ int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb,
                  const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0, cudaStream_t st) {
     if (!B || !q_len) return TGP_OK;
     RopeArgs a{q32, k32, v32, (bf16 *)qb, cos_t, sin_t, c->Hq, c->Hkv, c->Dh, c->TK, q_len, pos0, tiles};
-    tgp_rope_kv_kernel<<<B * q_len, 256, 0, st>>>(a);
+    launch_pdl(tgp_rope_kv_kernel, dim3(B * q_len), dim3(256), 0, st, a);
     LAUNCH_CHECK(1);
     return TGP_OK;
 }
@@ -1386,16 +1425,16 @@ int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *
         }
         const size_t sm = (size_t)(G * c->Dh + G * split * (c->Dh + 2)) * sizeof(float);
 #define TGP_DECODE_GROUP(DH_) do { \
-            if (G == 1) tgp_attn_decode_group_kernel<DH_, 1><<<grid, 32 * split, sm, st>>>(a, split); \
-            else if (G == 2) tgp_attn_decode_group_kernel<DH_, 2><<<grid, 32 * split, sm, st>>>(a, split); \
-            else if (G == 4) tgp_attn_decode_group_kernel<DH_, 4><<<grid, 32 * split, sm, st>>>(a, split); \
-            else tgp_attn_decode_group_kernel<DH_, 8><<<grid, 32 * split, sm, st>>>(a, split); } while (0)
+            if (G == 1) launch_pdl(tgp_attn_decode_group_kernel<DH_, 1>, grid, dim3(32 * split), sm, st, a, split); \
+            else if (G == 2) launch_pdl(tgp_attn_decode_group_kernel<DH_, 2>, grid, dim3(32 * split), sm, st, a, split); \
+            else if (G == 4) launch_pdl(tgp_attn_decode_group_kernel<DH_, 4>, grid, dim3(32 * split), sm, st, a, split); \
+            else launch_pdl(tgp_attn_decode_group_kernel<DH_, 8>, grid, dim3(32 * split), sm, st, a, split); } while (0)
         if (c->Dh == 64) {
-            if (grouped) TGP_DECODE_GROUP(64); else tgp_attn_decode_partial_kernel<64><<<grid, 32 * G * split, sm, st>>>(a, split);
-            tgp_attn_decode_merge_kernel<64><<<dim3(c->Hq, B), 64, 0, st>>>(a);
+            if (grouped) TGP_DECODE_GROUP(64); else launch_pdl(tgp_attn_decode_partial_kernel<64>, grid, dim3(32 * G * split), sm, st, a, split);
+            launch_pdl(tgp_attn_decode_merge_kernel<64>, dim3(c->Hq, B), dim3(64), 0, st, a);
         } else {
-            if (grouped) TGP_DECODE_GROUP(128); else tgp_attn_decode_partial_kernel<128><<<grid, 32 * G * split, sm, st>>>(a, split);
-            tgp_attn_decode_merge_kernel<128><<<dim3(c->Hq, B), 128, 0, st>>>(a);
+            if (grouped) TGP_DECODE_GROUP(128); else launch_pdl(tgp_attn_decode_partial_kernel<128>, grid, dim3(32 * G * split), sm, st, a, split);
+            launch_pdl(tgp_attn_decode_merge_kernel<128>, dim3(c->Hq, B), dim3(128), 0, st, a);
         }
 #undef TGP_DECODE_GROUP
         tgpk_launches += 1;
@@ -1418,14 +1457,14 @@ int tgpk_swiglu(const float *g, const float *u, void *ab, uint64_t n, cudaStream
     if (n % 4) return TGP_E_INVAL;
     uint64_t n4 = n / 4;
     uint32_t blocks = (uint32_t)((n4 + 255) / 256 < 148 * 16 ? (n4 + 255) / 256 : 148 * 16);
-    tgp_swiglu_kernel<<<blocks, 256, 0, st>>>((const float4 *)g, (const float4 *)u, (__nv_bfloat162 *)ab, n4);
+    launch_pdl(tgp_swiglu_kernel, dim3(blocks), dim3(256), 0, st, (const float4 *)g, (const float4 *)u, (__nv_bfloat162 *)ab, n4);
     LAUNCH_CHECK(1);
     return TGP_OK;
 }
 
 int tgpk_argmax(const float *logits, int32_t *out, uint32_t B, uint32_t V, cudaStream_t st) {
     if (!B) return TGP_OK;
-    tgp_argmax_kernel<<<B, 1024, 0, st>>>(logits, out, V);
+    launch_pdl(tgp_argmax_kernel, dim3(B), dim3(1024), 0, st, logits, out, V);
     LAUNCH_CHECK(1);
     return TGP_OK;
 }
@@ -1511,6 +1550,7 @@ int tgp_k_gemm_group_select(int enable) {
 
 int tgp_k_gemv_overlap(int enable) {
     g_gemv_pdl = enable ? 1 : 0;
+    g_small_pdl = enable ? 1 : 0;
     return TGP_OK;
 }
 
