@@ -295,25 +295,28 @@ def attention_loop(cfg, reps, device):
         out[name] = {"us": round(t * 1e6, 1), "TFLOPs": round(flops / t / 1e12, 1)}
     tb.k_attn_select(0)
     out["status"] = tb.k_attn_status()
-    # decode: one query per sequence over the same S keys (KV bytes read once: 2 * B * Hkv * S * Dh * 2)
+    # decode: one query per sequence over the same S keys (KV bytes read once: 2 * B * Hkv * S * Dh * 2), per kernel
     q1 = qb[:B].contiguous()
     o1 = torch.zeros(B, cfg.Hq * cfg.Dh, dtype=torch.bfloat16, device=device)
     scratch = torch.empty(tb.k_attn_scratch_bytes(mc) // 4, dtype=torch.float32, device=device)
-    for _ in range(3):
-        tb.k_attn(q1, kt, vt, o1, mc, B, 1, S - 1, scratch)
-    torch.cuda.synchronize()
-    ms = 0.0
-    for _ in range(reps):
-        flush.fill_(1)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        tb.k_attn(q1, kt, vt, o1, mc, B, 1, S - 1, scratch)
-        e1.record()
-        torch.cuda.synchronize()
-        ms += e0.elapsed_time(e1)
-    t = ms * 1e-3 / reps
     kv_bytes = 2 * B * cfg.Hkv * S * cfg.Dh * 2
-    out["decode"] = {"us": round(t * 1e6, 1), "GBps": round(kv_bytes / t / 1e9, 1), "kv_bytes": kv_bytes}
+    for name, impl in (("decode_mma", 2), ("decode_cuda_core", 1), ("decode", 0)):
+        tb.k_attn_decode_select(impl)
+        for _ in range(3):
+            tb.k_attn(q1, kt, vt, o1, mc, B, 1, S - 1, scratch)
+        torch.cuda.synchronize()
+        ms = 0.0
+        for _ in range(reps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            tb.k_attn(q1, kt, vt, o1, mc, B, 1, S - 1, scratch)
+            e1.record()
+            torch.cuda.synchronize()
+            ms += e0.elapsed_time(e1)
+        t = ms * 1e-3 / reps
+        out[name] = {"us": round(t * 1e6, 1), "GBps": round(kv_bytes / t / 1e9, 1), "kv_bytes": kv_bytes}
+    tb.k_attn_decode_select(0)
     return out, flops
 
 

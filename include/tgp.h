@@ -331,6 +331,12 @@ int  tgp_k_gemm_tc_variant(int variant);
  * kernel needs KV tiles of a multiple of 64 keys whose base addresses differ by whole rows of Dh elements (and
  * 16-byte aligned q); any other geometry is served by the mma.sync kernel even when 3 is forced.  Process-wide. */
 int  tgp_k_attn_select(int impl);
+/* Which kernel serves decode attention (q_len == 1 with scratch): 0 (default) by size - the tensor-core kernel (the G query
+ * heads of a KV head as rows of an mma.sync tile, K and V staged through shared memory with cp.async three chunks of 16
+ * keys deep, P rounded to bf16 for the second product) when KV tiles hold a multiple of 16 keys, G is 1, 2, 4 or 8 and
+ * the batch's context adds up to 256 chunks or more, else the CUDA-core kernels (one pass per KV tile and group of query
+ * heads); 1 forces the CUDA-core kernels, 2 the tensor-core kernel wherever its geometry allows.  Process-wide. */
+int  tgp_k_attn_decode_select(int impl);
 /* Error word of the tcgen05 attention kernel: 0, or which bounded wait ran out first (1 for S, 2 for P V, 3 for a K/V
  * load, 4 for the hand-over between the softmax warps and the MMA warp), or 5 if shared memory was not 1024-byte
  * aligned.  A CTA that gives up stores nothing.  Synchronous. */

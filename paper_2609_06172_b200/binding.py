@@ -109,6 +109,7 @@ _SIGS = {
     "tgp_k_gemm_last_kernel": [C.c_char_p, _U32],
     "tgp_k_gemm_select": [C.c_int],
     "tgp_k_attn_select": [C.c_int],
+    "tgp_k_attn_decode_select": [C.c_int],
     "tgp_k_gemv_overlap": [C.c_int],
     "tgp_k_skinny_select": [C.c_int],
     "tgp_k_gemm_tc_variant": [C.c_int],
@@ -466,6 +467,10 @@ def k_gemm_last_kernel():
     buf = C.create_string_buffer(96)
     _k(lib().tgp_k_gemm_last_kernel(buf, 96), "tgp_k_gemm_last_kernel")
     return buf.value.decode()
+
+
+def k_attn_decode_select(impl):
+    _k(lib().tgp_k_attn_decode_select(impl), "tgp_k_attn_decode_select")
 
 
 def k_attn_status():

@@ -87,12 +87,18 @@ __global__ void tgp_embed_kernel(const bf16 *__restrict__ table, const int32_t *
 }
 
 // ---- RMSNorm -> bf16 -------------------------------------------------------------------------
+// One step of a thread's sum of squares, written with explicit roundings so that the fused form below (a consumer that
+// normalises its activations itself) reproduces the kernel's statistics bit for bit.
+__device__ __forceinline__ float sumsq4(float ss, const float4 &v) {
+    return __fadd_rn(ss, __fmaf_rn(v.w, v.w, __fmaf_rn(v.z, v.z, __fmaf_rn(v.y, v.y, __fmul_rn(v.x, v.x)))));
+}
+
 __global__ void tgp_rmsnorm_kernel(const float *x, uint32_t ldx, const bf16 *__restrict__ g, bf16 *h, uint32_t d, float eps) {
     pdl_enter();
     __shared__ float red[32];
     const float4 *row = reinterpret_cast<const float4 *>(x + (size_t)blockIdx.x * ldx);
     float ss = 0.f;
-    for (uint32_t i = threadIdx.x; i < d / 4; i += blockDim.x) { float4 v = row[i]; ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w; }
+    for (uint32_t i = threadIdx.x; i < d / 4; i += blockDim.x) ss = sumsq4(ss, row[i]);
     ss = warp_sum(ss);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
     __syncthreads();
@@ -184,12 +190,58 @@ __global__ void __launch_bounds__(256) tgp_wstream_kernel(const bf16 *A, const b
 // (groups[s]: CTAs' worth of rows in part s, for the kernels that walk row groups instead of rows)
 struct GemvParts { const bf16 *W[TGP_GEMM_GROUP_MAX]; float *C[TGP_GEMM_GROUP_MAX]; uint32_t n[TGP_GEMM_GROUP_MAX], ldc[TGP_GEMM_GROUP_MAX], groups[TGP_GEMM_GROUP_MAX], count; };
 
+// Where the activations of a product come from.  mode 0: bf16 rows A[m, K].  mode 1: the RMSNorm of the fp32 rows x[m, :K]
+// (row stride ldx) with gain g - the warp computes the row statistics itself, exactly as tgp_rmsnorm_kernel's 256 threads
+// do (lane l plays threads l, 32 + l, ... of that kernel), and rounds each normalised value to bf16 as that kernel
+// stores it.  mode 2: SwiGLU of the fp32 rows g32, u32 [m, K], rounded to bf16 as tgp_swiglu_kernel stores it.  The fused
+// modes give bit for bit what the separate kernels followed by mode 0 give; they save a launch and a round trip for
+// the decode steps of small models, where every warp recomputing a row of a few hundred elements costs nothing.
+struct ASrc { int mode; const float *x; uint32_t ldx; const bf16 *gain; float eps; const float *g32, *u32; };
+
+__device__ __forceinline__ float rms_scale_as_kernel(const float *xrow, uint32_t d, float eps, uint32_t lane) {
+    const float4 *row = reinterpret_cast<const float4 *>(xrow);
+    float red[8];
+#pragma unroll
+    for (uint32_t w = 0; w < 8; ++w) {
+        float ss = 0.f;
+        for (uint32_t i = 32 * w + lane; i < d / 4; i += 256) ss = sumsq4(ss, row[i]);
+        red[w] = warp_sum(ss);
+    }
+    float t = 0.f;
+#pragma unroll
+    for (uint32_t w = 0; w < 8; ++w) if (lane == w) t = red[w];
+    t = warp_sum(t);
+    return 1.0f / sqrtf(t / (float)d + eps);
+}
+
+__device__ __forceinline__ void act8(const ASrc &s, const bf16 *A, uint32_t m, uint32_t K, uint32_t k, float r, float *xf) {
+    if (s.mode == 0) { unpack8(ld_act(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)), xf); return; }
+    if (s.mode == 1) {
+        const float4 *xr = reinterpret_cast<const float4 *>(s.x + (size_t)m * s.ldx + k);
+        const float4 v0 = xr[0], v1 = xr[1];
+        float g[8];
+        unpack8(*reinterpret_cast<const uint4 *>(s.gain + k), g);
+        const float v[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) xf[i] = __bfloat162float(__float2bfloat16_rn(v[i] * r * g[i]));
+        return;
+    }
+    const float4 *gr = reinterpret_cast<const float4 *>(s.g32 + (size_t)m * K + k), *ur = reinterpret_cast<const float4 *>(s.u32 + (size_t)m * K + k);
+    const float4 g0 = gr[0], g1 = gr[1], u0 = ur[0], u1 = ur[1];
+    const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w}, uv[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) xf[i] = __bfloat162float(__float2bfloat16_rn(gv[i] / (1.0f + expf(-gv[i])) * uv[i]));
+}
+
 template <int MT, int U>
-__global__ void __launch_bounds__(256) tgp_wstream_group_kernel(const bf16 *A, const GemvParts p, uint32_t Mrows, uint32_t n_total, uint32_t K, int accumulate) {
+__global__ void __launch_bounds__(256) tgp_wstream_group_kernel(const bf16 *A, const GemvParts p, uint32_t Mrows, uint32_t n_total, uint32_t K, int accumulate, const ASrc src) {
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t gwarp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarp = (gridDim.x * blockDim.x) >> 5;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     bool synced = false;
+    float rs[MT];
+#pragma unroll
+    for (int m = 0; m < MT; ++m) rs[m] = 0.f;
     for (uint32_t row = gwarp; row < n_total; row += nwarp) {
         const bf16 *W = p.W[0];
         float *C = p.C[0];
@@ -209,7 +261,14 @@ __global__ void __launch_bounds__(256) tgp_wstream_group_kernel(const bf16 *A, c
 #pragma unroll
             for (int u = 0; u < U; ++u)
                 wv[u] = (k0 + 256 * u < K) ? __ldcs(reinterpret_cast<const uint4 *>(wrow + k0 + 256 * u)) : make_uint4(0, 0, 0, 0);
-            if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
+            if (!synced) {
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                synced = true;
+                if (src.mode == 1) {
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) if (m < (int)Mrows) rs[m] = rms_scale_as_kernel(src.x + (size_t)m * src.ldx, K, src.eps, lane);
+                }
+            }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const uint32_t k = k0 + 256 * u;
@@ -218,7 +277,11 @@ __global__ void __launch_bounds__(256) tgp_wstream_group_kernel(const bf16 *A, c
 #pragma unroll
                 for (int m = 0; m < MT; ++m) {
                     float xf[8];
-                    unpack8((k < K && m < (int)Mrows) ? ld_act(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k)) : make_uint4(0, 0, 0, 0), xf);
+                    if (k < K && m < (int)Mrows) act8(src, A, m, K, k, rs[m], xf);
+                    else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) xf[i] = 0.f;
+                    }
 #pragma unroll
                     for (int i = 0; i < 8; ++i) acc[m] = fmaf(wf[i], xf[i], acc[m]);
                 }
@@ -447,6 +510,7 @@ struct AttnArgs {
     uint32_t Hq, Hkv, Dh, TK, q_len, pos0, n_tiles;
     float scale;
     TgpTilePtrs tiles;
+    uint32_t n_parts;                 // partials per head the merge kernel reads; 0: one per KV tile with valid keys
 };
 
 // One warp per query row, 32 keys per pass: lane = key for the scores, lane = output dims for P.V.
@@ -737,7 +801,7 @@ template <int DH>
 __global__ void tgp_attn_decode_merge_kernel(AttnArgs a) {
     pdl_enter();
     const uint32_t hq = blockIdx.x, b = blockIdx.y, i = threadIdx.x;
-    const uint32_t nt = (a.pos0 + 1 + a.TK - 1) / a.TK;
+    const uint32_t nt = a.n_parts ? a.n_parts : (a.pos0 + 1 + a.TK - 1) / a.TK;
     const float *part = a.scratch + (size_t)(b * a.Hq + hq) * a.n_tiles * (DH + 2);
     float mx = -INFINITY;
     for (uint32_t t = 0; t < nt; ++t) mx = fmaxf(mx, part[t * (DH + 2)]);
@@ -748,6 +812,184 @@ __global__ void tgp_attn_decode_merge_kernel(AttnArgs a) {
         o += w * part[t * (DH + 2) + 2 + i];
     }
     a.ob[(size_t)b * a.Hq * DH + hq * DH + i] = __float2bfloat16_rn(o / l);
+}
+
+// ---- decode attention on the tensor cores (mma.sync), K and V staged through shared memory ---------------------------------
+// The group kernel above is a latency chain: a warp's 32-key chunk is loads, 4*G*Dh FMAs per lane and shuffles, one after
+// the other, and a B200 needs ~35 KB in flight per SM to keep HBM busy.  Here the G query heads of a KV head are the rows
+// of a 16-row MMA tile (rows >= G are zero), a warp works on chunks of 16 keys, and the K and V rows of the next chunks are
+// already on their way: every warp owns DEC_STAGES private stages that it fills with cp.async (16 bytes per lane and
+// instruction, rows past the sequence zero-filled) - no block-wide barrier in the key loop.  Per chunk:
+//   S[16 x 16 keys] = Q K^T      2 x Dh/16 MMAs (m16n8k16, bf16 -> fp32), K fragments by ldmatrix from the swizzled stage;
+//   online softmax per row       (the running maximum moves rarely: O is rescaled only when a row's maximum grew);
+//   O[16 x Dh] += P V            Dh/8 MMAs, P straight from the S accumulators as the A fragment, V fragments by
+//                                ldmatrix.trans (V rows are keys: the transposed load makes keys the contraction index).
+// P is rounded to bf16 for the second product, as in the prefill kernels.  A CTA of four warps owns a contiguous range of
+// chunks of one (sequence, KV head); its warps take every fourth chunk, merge their four partials through shared memory
+// and write one (max, sum, unnormalised O) per query head and CTA to the scratch array tgp_attn_decode_merge_kernel reads.
+// Stage layout: row = key, 2*DH bytes, 16-byte chunk j of row r at chunk position j ^ (r & 7): conflict-free for the
+// ldmatrix reads (eight rows, same j) and for the cp.async writes.
+constexpr int DEC_STAGES = 3, DEC_WARPS = 4, DEC_KEYS = 16;
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float fast_ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+
+template <int DH, int G>
+__global__ void __launch_bounds__(DEC_WARPS * 32) tgp_attn_decode_mma_kernel(AttnArgs a, uint32_t chunks_per_cta) {
+    pdl_enter();
+    extern __shared__ __align__(128) uint8_t dec_sm[];
+    constexpr uint32_t ROW = DH * 2, CPR = ROW / 16;                  // bytes and 16-byte chunks per key row
+    constexpr uint32_t KV_BYTES = DEC_KEYS * ROW, STAGE = 2 * KV_BYTES;
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane >> 2, c = lane & 3;
+    const uint32_t part = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+    const uint32_t kvlen = a.pos0 + 1, nchunks = (kvlen + DEC_KEYS - 1) / DEC_KEYS;
+    const uint32_t q_lo = part * chunks_per_cta, q_hi = min(nchunks, q_lo + chunks_per_cta);
+    uint8_t *mine = dec_sm + (size_t)warp * DEC_STAGES * STAGE;
+    const uint32_t mine_u = (uint32_t)__cvta_generic_to_shared(mine);
+    const float sl2 = a.scale * 1.4426950408889634f;                  // scores are kept in units of log2
+
+    // Q fragments of this group: rows 0..G-1 real, the rest zero; held in registers for the whole kernel
+    uint32_t qf[DH / 16][2];
+    {
+        const bf16 *q = a.qb + ((size_t)b * a.Hq + hk * G) * DH + (size_t)r * DH;
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks) {
+            qf[ks][0] = r < G ? *reinterpret_cast<const uint32_t *>(q + ks * 16 + 2 * c) : 0u;
+            qf[ks][1] = r < G ? *reinterpret_cast<const uint32_t *>(q + ks * 16 + 2 * c + 8) : 0u;
+        }
+    }
+    // chunk q: its KV tile and offset; lane l copies 16-byte pieces idx = i * 32 + l of the chunk's K and V rows
+    auto issue = [&](uint32_t q, uint32_t stage) {
+        const uint32_t key0 = q * DEC_KEYS, tile = key0 / a.TK, off = key0 - tile * a.TK;
+        const uint8_t *kg = reinterpret_cast<const uint8_t *>(a.tiles.k[tile]) + ((size_t)(b * a.Hkv + hk) * a.TK + off) * ROW;
+        const uint8_t *vg = reinterpret_cast<const uint8_t *>(a.tiles.v[tile]) + ((size_t)(b * a.Hkv + hk) * a.TK + off) * ROW;
+        const uint32_t base = mine_u + stage * STAGE;
+#pragma unroll
+        for (uint32_t i = 0; i < DEC_KEYS * CPR / 32; ++i) {
+            const uint32_t idx = i * 32 + lane, row = idx / CPR, j = idx % CPR;
+            const uint32_t dst = row * ROW + ((j ^ (row & 7)) << 4);
+            const uint32_t nbytes = key0 + row < kvlen ? 16u : 0u;  // rows past the sequence are written as zeros, not read
+            cp_async16(base + dst, kg + (size_t)row * ROW + j * 16, nbytes);
+            cp_async16(base + KV_BYTES + dst, vg + (size_t)row * ROW + j * 16, nbytes);
+        }
+    };
+    // this warp's chunks: q_lo + warp, q_lo + warp + 4, ...
+    uint32_t issued = 0, total = 0;
+    for (uint32_t q = q_lo + warp; q < q_hi; q += DEC_WARPS) ++total;
+#pragma unroll
+    for (int s = 0; s < DEC_STAGES - 1; ++s) {
+        if (issued < total) { issue(q_lo + warp + issued * DEC_WARPS, issued % DEC_STAGES); ++issued; }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    float o[DH / 8][4];
+#pragma unroll
+    for (int j = 0; j < DH / 8; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+    float m_run = -INFINITY, l_run = 0.f;                             // of row r (replicated over the four lanes of the row)
+    for (uint32_t it = 0; it < total; ++it) {
+        if (issued < total) { issue(q_lo + warp + issued * DEC_WARPS, issued % DEC_STAGES); ++issued; }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group %0;" ::"n"(DEC_STAGES - 1) : "memory");
+        __syncwarp();
+        const uint32_t q = q_lo + warp + it * DEC_WARPS, key0 = q * DEC_KEYS;
+        const uint32_t kb = mine_u + (it % DEC_STAGES) * STAGE, vb = kb + KV_BYTES;
+        // ---- S = Q K^T: two n-tiles of 8 keys ----
+        float sacc[2][4];
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt) {
+            sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
+#pragma unroll
+            for (int kp = 0; kp < DH / 32; ++kp) {
+                const uint32_t row = nt * 8 + (lane & 7), j = kp * 4 + (lane >> 3);
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4(kb + row * ROW + ((j ^ (row & 7)) << 4), b0, b1, b2, b3);
+                mma_bf16(sacc[nt], qf[2 * kp][0], 0u, qf[2 * kp][1], 0u, b0, b1);
+                mma_bf16(sacc[nt], qf[2 * kp + 1][0], 0u, qf[2 * kp + 1][1], 0u, b2, b3);
+            }
+        }
+        // ---- online softmax of row r over the chunk's 16 keys (this lane: keys 2c, 2c+1, 8+2c, 9+2c) ----
+        float sv[4] = {sacc[0][0] * sl2, sacc[0][1] * sl2, sacc[1][0] * sl2, sacc[1][1] * sl2};
+        if (key0 + DEC_KEYS > kvlen) {
+            const uint32_t kk[4] = {2 * c, 2 * c + 1, 8 + 2 * c, 9 + 2 * c};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) if (key0 + kk[i] >= kvlen) sv[i] = -INFINITY;
+        }
+        float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(m_run, mx);                          // finite: every chunk holds a valid key
+        if (__any_sync(0xffffffffu, m_new > m_run)) {
+            const float alpha = fast_ex2(m_run - m_new);              // first chunk: ex2(-inf) = 0 on zeros
+            l_run *= alpha;
+#pragma unroll
+            for (int j = 0; j < DH / 8; ++j) { o[j][0] *= alpha; o[j][1] *= alpha; }
+            m_run = m_new;
+        }
+        float p[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) p[i] = fast_ex2(sv[i] - m_run);
+        float ls = (p[0] + p[1]) + (p[2] + p[3]);
+        ls += __shfl_xor_sync(0xffffffffu, ls, 1);
+        ls += __shfl_xor_sync(0xffffffffu, ls, 2);
+        l_run += ls;
+        __nv_bfloat162 plo = __floats2bfloat162_rn(p[0], p[1]), phi = __floats2bfloat162_rn(p[2], p[3]);
+        const uint32_t pa0 = *reinterpret_cast<uint32_t *>(&plo), pa2 = *reinterpret_cast<uint32_t *>(&phi);
+        // ---- O += P V: Dh/8 n-tiles, two per ldmatrix ----
+#pragma unroll
+        for (int jp = 0; jp < DH / 16; ++jp) {
+            const uint32_t row = ((lane >> 3) & 1) * 8 + (lane & 7), j = 2 * jp + (lane >> 4);
+            uint32_t v0, v1, v2, v3;
+            ldsm_x4_t(vb + row * ROW + ((j ^ (row & 7)) << 4), v0, v1, v2, v3);
+            mma_bf16(o[2 * jp], pa0, 0u, pa2, 0u, v0, v1);
+            mma_bf16(o[2 * jp + 1], pa0, 0u, pa2, 0u, v2, v3);
+        }
+        __syncwarp();                                                 // the stage may be refilled two iterations from now
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    // ---- merge the four warps' partials (rows < G), write one partial per head for this CTA ----
+    // (each warp's partial goes to the start of its own stages, which it no longer needs: [G][DH + 2] floats)
+    __syncwarp();
+    constexpr size_t WSTRIDE = (size_t)DEC_STAGES * STAGE / sizeof(float);
+    float *wp = reinterpret_cast<float *>(dec_sm);
+    if (r < G) {
+        float *dst = wp + (size_t)warp * WSTRIDE + (size_t)r * (DH + 2);
+        if (c == 0) { dst[0] = m_run; dst[1] = l_run; }
+#pragma unroll
+        for (int j = 0; j < DH / 8; ++j) { dst[2 + j * 8 + 2 * c] = o[j][0]; dst[2 + j * 8 + 2 * c + 1] = o[j][1]; }
+    }
+    __syncthreads();
+    for (uint32_t e = threadIdx.x; e < G * DH; e += blockDim.x) {
+        const uint32_t g = e / DH, d = e % DH;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, wp[(size_t)w * WSTRIDE + (size_t)g * (DH + 2)]);
+        float l = 0.f, acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < DEC_WARPS; ++w) {
+            const float *src = wp + (size_t)w * WSTRIDE + (size_t)g * (DH + 2);
+            const float wgt = src[0] == -INFINITY ? 0.f : fast_ex2(src[0] - M);       // a warp without a chunk: weight 0
+            l += wgt * src[1];
+            acc += wgt * src[2 + d];
+        }
+        if (a.n_parts == 1) {                                              // the CTA saw the whole context: this is the result
+            a.ob[((size_t)b * a.Hq + hk * G + g) * DH + d] = __float2bfloat16_rn(acc / l);
+            continue;
+        }
+        float *out = a.scratch + ((size_t)(b * a.Hq + hk * G + g) * a.n_tiles + part) * (DH + 2);
+        if (d == 0) { out[0] = M * 0.6931471805599453f; out[1] = l; }      // the merge kernel works in natural-log units
+        out[2 + d] = acc;
+    }
 }
 
 // ---- SwiGLU -----------------------------------------------------------------------------------------
@@ -1282,7 +1524,7 @@ static void launch_gemv_rows(const bf16 *A, const bf16 *W, float *C, uint32_t Mr
 }
 
 template <int MT>
-static void launch_gemv_group(const bf16 *A, const GemvParts &p, uint32_t Mrows, uint32_t n_total, uint32_t K, int acc, cudaStream_t st) {
+static void launch_gemv_group(const bf16 *A, const GemvParts &p, uint32_t Mrows, uint32_t n_total, uint32_t K, int acc, cudaStream_t st, const ASrc &src = ASrc{}) {
     static int blocks_per_sm = 0, sms = 0;
     if (!blocks_per_sm) {
         int dev = 0;
@@ -1301,7 +1543,7 @@ static void launch_gemv_group(const bf16 *A, const GemvParts &p, uint32_t Mrows,
     attr[0].val.programmaticStreamSerializationAllowed = g_gemv_pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, tgp_wstream_group_kernel<MT, 8>, A, p, Mrows, n_total, K, acc);
+    cudaLaunchKernelEx(&cfg, tgp_wstream_group_kernel<MT, 8>, A, p, Mrows, n_total, K, acc, src);
     tgpk_last_gemm_kernel = "tgp_wstream_group_kernel";
 }
 
@@ -1345,6 +1587,24 @@ int tgpk_gemm_group(const void *A, uint32_t count, const void *const *W, float *
     return TGP_OK;
 }
 
+
+// Products of M <= 2 activation rows whose activations are computed on the fly (see ASrc): the RMSNorm of x, or SwiGLU of
+// (g32, u32).  Every block must carry the M <= 2 group key (tgpk_gemm_group_key(M, n, K) == M); K % 8 == 0.
+int tgpk_gemm_group_fused(int mode, const float *x, uint32_t ldx, const void *gain, float eps, const float *g32, const float *u32, uint32_t count,
+                          const void *const *W, float *const *C, const uint32_t *n, const uint32_t *ldc, uint32_t M, uint32_t K, int accumulate, cudaStream_t st) {
+    if (!count || count > TGP_GEMM_GROUP_MAX || !M || M > 2 || K % 8 || (mode != 1 && mode != 2)) return TGP_E_INVAL;
+    for (uint32_t s = 0; s < count; ++s) if (tgpk_gemm_group_key(M, n[s], K) != M) return TGP_E_INVAL;
+    GemvParts p;
+    memset(&p, 0, sizeof(p));
+    uint32_t total = 0;
+    for (uint32_t s = 0; s < count; ++s) { p.W[s] = (const bf16 *)W[s]; p.C[s] = C[s]; p.n[s] = n[s]; p.ldc[s] = ldc[s]; total += n[s]; }
+    p.count = count;
+    const ASrc src{mode, x, ldx, (const bf16 *)gain, eps, g32, u32};
+    if (M == 1) launch_gemv_group<1>(nullptr, p, M, total, K, accumulate, st, src);
+    else launch_gemv_group<2>(nullptr, p, M, total, K, accumulate, st, src);
+    LAUNCH_CHECK(1);
+    return TGP_OK;
+}
 
 int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
     if (!M || !n) return TGP_OK;
@@ -1404,6 +1664,7 @@ int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb,
 }
 
 static int g_attn_decode_grouped = 1;   // decode: one pass over a KV tile serves all query heads of the group (0: one pass per head)
+static int g_attn_decode_impl = 0;      // decode: 0 by size, 1 the CUDA-core per-tile kernels only, 2 the tensor-core kernel wherever its geometry allows
 static int g_attn_impl = 0;      // q_len >= 16: 0 by problem size, 3 tcgen05 kernel, 2 mma.sync flash kernel, 1 warp-per-row CUDA-core kernel
 
 int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *ob, const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0,
@@ -1419,6 +1680,34 @@ int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *
         if (split < 1) split = 1;
         dim3 grid(nt, c->Hkv, B);
         const bool grouped = g_attn_decode_grouped && (G == 1 || G == 2 || G == 4 || G == 8) && c->Hq % c->Hkv == 0;
+        // tensor-core decode kernel: whole 16-key chunks inside a tile, 16-byte aligned rows; the context must be long enough
+        // to give its warps a few chunks each (below that the per-tile kernel's single pass is as fast)
+        const uint32_t nchunks = (pos0 + 1 + DEC_KEYS - 1) / DEC_KEYS;
+        bool aligned16 = (reinterpret_cast<uintptr_t>(qb) & 3u) == 0;
+        for (uint32_t t = 0; t < nt && aligned16; ++t) aligned16 = ((reinterpret_cast<uintptr_t>(tiles.k[t]) | reinterpret_cast<uintptr_t>(tiles.v[t])) & 15u) == 0;
+        if (grouped && g_attn_decode_impl != 1 && c->TK % DEC_KEYS == 0 && aligned16 && (g_attn_decode_impl == 2 || nchunks * B * c->Hkv >= 256)) {
+            static int sms = 0;
+            if (!sms) { int dev = 0; cudaGetDevice(&dev); if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) sms = 148; }
+            const uint32_t units = B * c->Hkv, per_sm = c->Dh == 64 ? 4 : 2;             // CTAs that fit an SM (96 / 48 KB of shared memory each)
+            uint32_t parts = (uint32_t)sms * per_sm / units;                              // CTAs per (sequence, KV head): one wave at most
+            parts = std::max(1u, std::min(parts, std::min(n_tiles, (nchunks + DEC_WARPS - 1) / DEC_WARPS)));
+            const uint32_t per_cta = (nchunks + parts - 1) / parts;
+            parts = (nchunks + per_cta - 1) / per_cta;                                    // no CTA without a chunk
+            a.n_parts = parts;
+            const size_t smem = (size_t)DEC_WARPS * DEC_STAGES * 2 * DEC_KEYS * c->Dh * 2;        // 96 KB at Dh = 128, 48 KB at 64
+            dim3 g2(parts, c->Hkv, B);
+#define TGP_DECODE_MMA(DH_, G_) do { \
+                static bool attr_set = false; \
+                if (!attr_set) { if (cudaFuncSetAttribute(tgp_attn_decode_mma_kernel<DH_, G_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return TGP_E_CUDA; attr_set = true; } \
+                launch_pdl(tgp_attn_decode_mma_kernel<DH_, G_>, g2, dim3(DEC_WARPS * 32), smem, st, a, per_cta); } while (0)
+#define TGP_DECODE_MMA_G(DH_) do { if (G == 1) TGP_DECODE_MMA(DH_, 1); else if (G == 2) TGP_DECODE_MMA(DH_, 2); else if (G == 4) TGP_DECODE_MMA(DH_, 4); else TGP_DECODE_MMA(DH_, 8); } while (0)
+            if (c->Dh == 64) { TGP_DECODE_MMA_G(64); if (parts > 1) launch_pdl(tgp_attn_decode_merge_kernel<64>, dim3(c->Hq, B), dim3(64), 0, st, a); }
+            else { TGP_DECODE_MMA_G(128); if (parts > 1) launch_pdl(tgp_attn_decode_merge_kernel<128>, dim3(c->Hq, B), dim3(128), 0, st, a); }
+#undef TGP_DECODE_MMA_G
+#undef TGP_DECODE_MMA
+            LAUNCH_CHECK(parts > 1 ? 2 : 1);
+            return TGP_OK;
+        }
         if (grouped) {                                      // K and V read once for the whole group of query heads
             split = (c->TK + 31) / 32;
             if (split > 8) split = 8;
@@ -1551,6 +1840,12 @@ int tgp_k_gemm_group_select(int enable) {
 int tgp_k_gemv_overlap(int enable) {
     g_gemv_pdl = enable ? 1 : 0;
     g_small_pdl = enable ? 1 : 0;
+    return TGP_OK;
+}
+
+int tgp_k_attn_decode_select(int impl) {
+    if (impl < 0 || impl > 2) return TGP_E_INVAL;
+    g_attn_decode_impl = impl;
     return TGP_OK;
 }
 

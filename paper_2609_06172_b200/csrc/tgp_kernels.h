@@ -45,3 +45,7 @@ extern thread_local const char *tgpk_last_gemm_kernel;
 // test hooks of the tensor-core kernels' bounded waits (see tgp_k_wait_test)
 int tgpk_gemm_wait_test(unsigned long long limit_ns, int withhold_step);
 int tgpk_attn_wait_test(unsigned long long limit_ns, int withhold_step);
+// products of M <= 2 rows with the activations computed on the fly: mode 1 the RMSNorm of x (row stride ldx, gain, eps),
+// mode 2 SwiGLU of (g32, u32); bit-identical to the separate kernels followed by tgpk_gemm_group()
+int tgpk_gemm_group_fused(int mode, const float *x, uint32_t ldx, const void *gain, float eps, const float *g32, const float *u32, uint32_t count,
+                          const void *const *W, float *const *C, const uint32_t *n, const uint32_t *ldc, uint32_t M, uint32_t K, int accumulate, cudaStream_t st);

@@ -490,6 +490,47 @@ def test_tensor_core_prefill_attention_of_a_later_chunk(Dh, TK):
     assert tb.k_attn_status() == 0
 
 
+@pytest.mark.parametrize("Dh,Hq,Hkv,TK,kvlen,B", [(128, 32, 8, 256, 1280, 2), (128, 32, 8, 256, 1037, 3), (128, 64, 8, 64, 2112, 2), (64, 32, 8, 128, 640, 1),
+                                                 (64, 4, 4, 16, 48, 1), (128, 8, 4, 32, 33, 2), (64, 8, 1, 16, 17, 4), (128, 4, 4, 48, 1, 2),
+                                                 (64, 16, 2, 80, 401, 5)])
+def test_tensor_core_decode_attention_matches_oracle_and_cuda_core_kernel(Dh, Hq, Hkv, TK, kvlen, B):
+    """Decode attention on the tensor cores (forced wherever the geometry allows) against the oracle's softmax(q K^T) V on
+    the same bf16 queries and cache, and against the CUDA-core kernel: contexts that end in the middle of a 16-key chunk,
+    span many KV tiles and several CTAs per (sequence, KV head), groups of 1, 2, 4 and 8 query heads, a single key, and
+    tiles whose bytes past the context are NaN (they must be neither read into the result nor multiplied by zero)."""
+    cfg = replace(KCFG, Dh=Dh, Hq=Hq, Hkv=Hkv, TK=TK, S=kvlen, T=0, B=B, d=Hq * Dh)
+    mc = model_cfg(cfg)
+    kt, vt = make_tiles(cfg, B)
+    assert len(kt) == (kvlen + TK - 1) // TK
+    for j, (k, v) in enumerate(zip(kt, vt)):
+        k.copy_(bf16_dev(rnd_bits(90 + j, k.numel())) * 40)
+        v.copy_(bf16_dev(rnd_bits(190 + j, v.numel())) * 40)
+    # everything past the context is poison
+    last = kt[-1].view(B, Hkv, TK, Dh), vt[-1].view(B, Hkv, TK, Dh)
+    used = kvlen - (len(kt) - 1) * TK
+    if used < TK:
+        last[0][:, :, used:, :] = float("nan")
+        last[1][:, :, used:, :] = float("nan")
+    qb = (bf16_dev(rnd_bits(7, B * Hq * Dh)) * 40).view(B, Hq * Dh)
+    scratch = torch.empty(tb.k_attn_scratch_bytes(mc) // 4, dtype=torch.float32, device=DEV)
+    outs = {}
+    for impl in (2, 1):
+        tb.k_attn_decode_select(impl)
+        ob = torch.full((B, Hq * Dh), float("nan"), dtype=torch.bfloat16, device=DEV)
+        tb.k_attn(qb, kt, vt, ob, mc, B, 1, kvlen - 1, scratch)
+        torch.cuda.synchronize()
+        outs[impl] = ob.float().cpu().numpy().reshape(B, 1, Hq, Dh)
+    tb.k_attn_decode_select(0)
+    o = OracleModel(cfg, {})
+    kc, vc = tiles_to_cache(kt, cfg, B)[:, :, :kvlen], tiles_to_cache(vt, cfg, B)[:, :, :kvlen]
+    o.K[0], o.V[0] = kc, vc
+    att = o.attention(0, qb.float().cpu().numpy().reshape(B, 1, Hq, Dh), kvlen - 1)
+    for impl, got in outs.items():
+        assert np.isfinite(got).all(), impl
+        assert np.abs(got - att).max() < 2.0 ** -7 * np.abs(att).max() + 1e-6, impl
+        assert np.mean(np.abs(got - bf16_round(att))) < 3e-3 * np.abs(att).mean(), impl
+
+
 def test_attention_single_key_returns_v():
     cfg = replace(KCFG, B=1, S=1, T=0)
     mc = model_cfg(cfg)
