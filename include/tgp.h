@@ -305,6 +305,12 @@ int  tgp_k_gemm_group_select(int enable);
 /* Name of the kernel that the calling thread's last tgp_k_gemm() / tgp_k_gemm_group() launched (the choice depends on
  * M, n, K and the GPU's SM count), as a NUL-terminated string of at most capacity - 1 characters; "" before the first. */
 int  tgp_k_gemm_last_kernel(char *name, uint32_t capacity);
+/* Decode steps of at most two sequences on models whose rows hold at most 1024 elements (d for the norms, F for SwiGLU):
+ * tgp_step() lets the products that consume a normalised state or a SwiGLU output compute it themselves (each warp of
+ * the weight-streaming kernel redoes the row, bit for bit as the separate kernel would), so those ops launch nothing.
+ * Results are identical either way.  Process-wide; default off: on the tiny configuration it takes a decode step from 50
+ * launches to 32, but a fused span waits for the copies of all its blocks, and the step got no faster (measured). */
+int  tgp_k_decode_fuse(int enable);
 /* Which kernel serves M > 16: 0 (default) the tcgen05 tensor-core GEMM, 1 the CUDA-core tile kernel (an on-device
  * cross-check).  M <= 16 always takes the weight-streaming GEMV.  Process-wide. */
 int  tgp_k_gemm_select(int impl);

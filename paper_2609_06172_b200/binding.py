@@ -108,6 +108,7 @@ _SIGS = {
     "tgp_k_gemm_group_select": [C.c_int],
     "tgp_k_gemm_last_kernel": [C.c_char_p, _U32],
     "tgp_k_gemm_select": [C.c_int],
+    "tgp_k_decode_fuse": [C.c_int],
     "tgp_k_attn_select": [C.c_int],
     "tgp_k_attn_decode_select": [C.c_int],
     "tgp_k_gemv_overlap": [C.c_int],
@@ -471,6 +472,10 @@ def k_gemm_last_kernel():
 
 def k_attn_decode_select(impl):
     _k(lib().tgp_k_attn_decode_select(impl), "tgp_k_attn_decode_select")
+
+
+def k_decode_fuse(enable):
+    _k(lib().tgp_k_decode_fuse(int(enable)), "tgp_k_decode_fuse")
 
 
 def k_attn_status():

@@ -26,6 +26,9 @@ extern thread_local uint64_t tgpk_launches;
 #define CU(ctx, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return tgp_fail(ctx, TGP_E_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } while (0)
 
 static int g_small_copy_streams = 1;     // plans of small copies use three copy streams (0: always one)
+static int g_fuse_small = 0;             // decode steps of small models: RMSNorm and SwiGLU are computed by the products that consume them (off:
+                                         // 32 instead of 50 launches per step of the tiny configuration, but a span waits for all its copies, and
+                                         // with a ring of two blocks copies and kernels already alternate more than they overlap: 0.56 against 0.58)
 
 struct TgpEngine {
     // workspace carve-up
@@ -588,11 +591,14 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
         GemmTarget g0 = {};
         int32_t g_expert = -1;
         bool g_gather = false, g_scatter = false;
-        if (ring && o.kind == TGP_OP_GEMM && !e->tap) {
+        uint32_t gbase = i;                                  // first product of the span (after a fused norm / SwiGLU op: i + 1)
+        int fuse = 0;                                        // 1: op i is an RMSNorm computed by its consumers; 2: a SwiGLU computed by its consumers
+        // products from op `base` on that may share a launch: same layer, activations, accumulation, K and group key
+        auto form_group = [&](uint32_t base, uint32_t *key_out) -> uint32_t {
             uint32_t cnt = 0, key0 = 0;
-            for (uint32_t j = 0; j < TGP_GEMM_GROUP_MAX && i + j < st.op0 + st.nops; ++j) {
-                const TgpOp &f = ctx->ops[i + j];
-                if (f.kind != TGP_OP_GEMM || f.layer != o.layer || !f.nacc) break;
+            for (uint32_t j = 0; j < TGP_GEMM_GROUP_MAX && base + j < st.op0 + st.nops; ++j) {
+                const TgpOp &f = ctx->ops[base + j];
+                if (f.kind != TGP_OP_GEMM || f.layer != ctx->ops[base].layer || !f.nacc) break;
                 const TgpRole *rp = role_of(ctx, f, 0);
                 if (!rp) break;
                 const TgpRole &r = *rp;
@@ -603,10 +609,15 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
                 if (!key) break;
                 if (j == 0) { g0 = t; gK = Kj; key0 = key; g_expert = r.expert; }
                 else if (t.A != g0.A || t.acc != g0.acc || t.Mrows != g0.Mrows || Kj != gK || key != key0 || r.expert != g_expert) break;
-                if (ctx->plan.op_last_place[i + j] >= 0 && (size_t)ctx->plan.op_last_place[i + j] >= e->next_cmd) break;   // its copy is not enqueued yet
+                if (ctx->plan.op_last_place[base + j] >= 0 && (size_t)ctx->plan.op_last_place[base + j] >= e->next_cmd) break;   // its copy is not enqueued yet
                 gC[j] = t.C + r.row0; gn[j] = r.rows; gld[j] = t.ldc;
                 cnt = j + 1;
             }
+            if (key_out) *key_out = key0;
+            return cnt;
+        };
+        if (ring && o.kind == TGP_OP_GEMM && !e->tap) {
+            uint32_t cnt = form_group(i, nullptr);
             // A grouped launch keeps the ring slots of its first blocks until its last block has arrived and the launch has
             // run.  Against copies of megabytes that wait is a percent of the copy time; against copies of a few
             // microseconds it is as long as the copies themselves, so small blocks whose slot a later copy waits for stay alone.
@@ -617,6 +628,31 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
                 const TgpRole &r = *role_of(ctx, ctx->ops[i + j], 0);
                 g_gather |= r.kind == TGP_K_WG && r.row0 == 0;
                 g_scatter |= r.kind == TGP_K_WD && r.row0 + r.rows == c.d;
+            }
+        } else if (ring && g_fuse_small && !e->tap && !c.E && q_len == 1 && M <= 2 && (o.kind == TGP_OP_RMSNORM || o.kind == TGP_OP_SWIGLU) &&
+                   i + 1 < st.op0 + st.nops && (ctx->plan.op_last_place[i] < 0 || (size_t)ctx->plan.op_last_place[i] < e->next_cmd)) {
+            // Launch-bound decode steps of small models (one or two sequences, rows of at most 1024 elements): the products
+            // that consume a normalised state or a SwiGLU output compute it themselves, bit for bit as the separate kernel
+            // would have (every warp redoes a row of a few hundred elements), and the op's own launch disappears.  The span
+            // is the op and the products after it that may share a launch; all wait for all placements, as a group does.
+            const TgpRole *np = o.kind == TGP_OP_RMSNORM ? role_of(ctx, o, 0) : nullptr;
+            uint32_t key = 0;
+            const uint32_t cnt = form_group(i + 1, &key);
+            const void *want_A = o.kind == TGP_OP_SWIGLU ? (const void *)e->ab : (np && np->kind == TGP_K_GF) ? (const void *)e->hf : (const void *)e->h;
+            const bool norm_ok = o.kind == TGP_OP_RMSNORM && np && gK == c.d && c.d <= 1024;
+            const bool glu_ok = o.kind == TGP_OP_SWIGLU && gK == c.F && c.F <= 1024;
+            if (cnt >= 1 && g0.A == want_A && g0.Mrows <= 2 && key == g0.Mrows && g_expert < 0 && (norm_ok || glu_ok)) {
+                // ... and nothing else reads the state the op would have written: the products after the span are another op's
+                bool later_reader = false;
+                for (uint32_t j = i + 1 + cnt; j < st.op0 + st.nops && !later_reader; ++j) {
+                    const TgpOp &f = ctx->ops[j];
+                    if (f.kind == o.kind) break;                                   // the state is rewritten here
+                    if (f.kind != TGP_OP_GEMM) continue;
+                    const TgpRole *rp = role_of(ctx, f, 0);
+                    GemmTarget t;
+                    if (rp && gemm_target(e, c, *rp, M, B, logits_dev, &t) && t.A == want_A) later_reader = true;
+                }
+                if (!later_reader) { fuse = o.kind == TGP_OP_RMSNORM ? 1 : 2; span = 1 + cnt; gbase = i + 1; }
             }
         }
         for (uint32_t j = i; j < i + span; ++j)
@@ -643,6 +679,14 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             const TgpRole *rp = role_of(ctx, o, 0);
             if (!rp || (rp->kind != TGP_K_G1 && rp->kind != TGP_K_G2 && rp->kind != TGP_K_GF)) return tgp_fail(ctx, TGP_E_MISMATCH, "norm op on a tensor that is not a bound gain");
             const TgpRole &r = *rp;
+            if (fuse == 1) {
+                const void *gW[TGP_GEMM_GROUP_MAX];
+                for (uint32_t j = 0; j + 1 < span; ++j) gW[j] = where(ctx, ctx->ops[gbase + j], 0);
+                const bool fin = r.kind == TGP_K_GF;
+                rc = tgpk_gemm_group_fused(1, fin ? e->x + (size_t)(q_len - 1) * c.d : e->x, fin ? q_len * c.d : c.d, where(ctx, o, 0), c.eps, nullptr, nullptr,
+                                           span - 1, gW, gC, gn, gld, g0.Mrows, gK, g0.acc, cs);
+                break;
+            }
             if (r.kind == TGP_K_GF) rc = tgpk_rmsnorm(e->x + (size_t)(q_len - 1) * c.d, q_len * c.d, where(ctx, o, 0), e->hf, B, c.d, c.eps, cs);
             else rc = tgpk_rmsnorm(e->x, c.d, where(ctx, o, 0), e->h, M, c.d, c.eps, cs);
             break;
@@ -730,6 +774,12 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             break;
         }
         case TGP_OP_SWIGLU:
+            if (fuse == 2) {
+                const void *gW[TGP_GEMM_GROUP_MAX];
+                for (uint32_t j = 0; j + 1 < span; ++j) gW[j] = where(ctx, ctx->ops[gbase + j], 0);
+                rc = tgpk_gemm_group_fused(2, nullptr, 0, nullptr, 0.f, e->g32, e->u32, span - 1, gW, gC, gn, gld, g0.Mrows, gK, g0.acc, cs);
+                break;
+            }
             if (c.E) { if (e->cur_expert >= 0 && e->cnt[e->cur_expert]) rc = tgpk_swiglu(e->g32, e->u32, e->ab, (uint64_t)e->cnt[e->cur_expert] * c.F, cs); }
             else rc = tgpk_swiglu(e->g32, e->u32, e->ab, (uint64_t)M * c.F, cs);
             break;
@@ -847,6 +897,11 @@ extern "C" int tgp_replan_commit(tgp_ctx *ctx) {
     return TGP_OK;
 }
 
+extern "C" int tgp_k_decode_fuse(int enable) {
+    g_fuse_small = enable ? 1 : 0;
+    return TGP_OK;
+}
+
 extern "C" int tgp_set_op_timing(tgp_ctx *ctx, int enable) {
     if (!ctx || !ctx->eng) return TGP_E_STATE;
     ctx->eng->op_timing = enable != 0;
@@ -937,12 +992,14 @@ extern "C" int tgp_run_capture_begin(tgp_ctx *ctx, void *compute_stream, void *c
         if (ctx->plan.op_last_place[i] >= 0 && (rc = get_event(ctx, e->copied_ev, i, &ev))) return rc;
     }
     e->cap_cs = (cudaStream_t)compute_stream; e->cap_cp = (cudaStream_t)copy_stream;
-    e->n_copy = 1;                                       // in a graph the joins of several copy branches cost more than they hide (measured)
+    e->n_copy = 1;                                       // in a graph the joins of several copy branches cost more than they hide (measured: the tiny
+                                                         // configuration at 512 KiB blocks replays at 0.56 / 0.52 / 0.51 of its roofline with 1 / 2 / 3 copy streams)
     CU(ctx, cudaStreamBeginCapture(e->cap_cs, cudaStreamCaptureModeRelaxed));
     // fork: the copy and write-back streams join the capture
     cudaError_t er = cudaEventRecord(e->fork_ev, e->cap_cs);
     if (er == cudaSuccess) er = cudaStreamWaitEvent(e->cap_cp, e->fork_ev, 0);
     if (er == cudaSuccess) er = cudaStreamWaitEvent(e->wb_stream, e->fork_ev, 0);
+    for (uint32_t k = 1; k < e->n_copy && er == cudaSuccess; ++k) er = cudaStreamWaitEvent(e->xcopy[k - 1], e->fork_ev, 0);
     if (er != cudaSuccess) {
         cudaGraph_t g = nullptr;
         cudaStreamEndCapture(e->cap_cs, &g);
@@ -962,6 +1019,10 @@ extern "C" int tgp_run_capture_end(tgp_ctx *ctx) {
     if (er == cudaSuccess) er = cudaEventRecord(e->join_wb, e->wb_stream);
     if (er == cudaSuccess) er = cudaStreamWaitEvent(e->cap_cs, e->join_cp, 0);
     if (er == cudaSuccess) er = cudaStreamWaitEvent(e->cap_cs, e->join_wb, 0);
+    for (uint32_t k = 1; k < e->n_copy && er == cudaSuccess; ++k) {      // the library's extra copy streams, when the captured run used them
+        er = cudaEventRecord(e->xmark[k], e->xcopy[k - 1]);
+        if (er == cudaSuccess) er = cudaStreamWaitEvent(e->cap_cs, e->xmark[k], 0);
+    }
     cudaGraph_t g = nullptr;
     cudaError_t ee = cudaStreamEndCapture(e->cap_cs, &g);
     if (er != cudaSuccess || ee != cudaSuccess || !g) {

@@ -169,6 +169,35 @@ def test_decode_step_groups_products_into_one_launch_with_the_same_bits(B, budge
     assert min(saved) >= (2 * cfg.L if budget else 1), saved
 
 
+@pytest.mark.parametrize("B", [1, 2])
+def test_decode_step_of_a_small_model_lets_products_compute_their_norm_and_swiglu_with_the_same_bits(B):
+    """Launch-bound decode steps: the q/k/v, gate/up and head products normalise the residual stream themselves and the
+    down projection computes SwiGLU itself, so those ops launch nothing - fewer launches per step, not a bit of
+    difference in any logit (the fused forms redo the separate kernels' arithmetic in the same order)."""
+    cfg = replace(si.CONFIGS[1], B=B, S=19, T=6, TK=8)
+    prompt = si.prompt_tokens(cfg)
+    forced = (np.arange(cfg.B * cfg.T, dtype=np.int32).reshape(cfg.B, cfg.T) * 577 + 11) % cfg.V
+    lay, pool, s, blobs, T = setup(cfg, budget=64 << 20)              # everything resident: every span forms
+    r = Runner(s, cfg.B * cfg.S)
+    runs = {}
+    for enable in (1, 0):
+        tb.k_decode_fuse(enable)
+        logits, launches = [], []
+        r.reset()
+        r.step(tb.PREFILL, prompt, cfg.S)
+        for t in range(T):
+            st = r.step(tb.DECODE, np.ascontiguousarray(forced[:, t:t + 1]), 1, want_stats=True)
+            launches.append(st.n_launches)
+            logits.append(r.logits.cpu().numpy().copy())
+        runs[enable] = (logits, launches)
+    tb.k_decode_fuse(0)
+    s.close()
+    for a, b in zip(runs[1][0], runs[0][0]):
+        assert np.array_equal(a, b)
+    # per layer two norms and one SwiGLU disappear, and the final norm
+    assert all(u - f >= 3 * cfg.L + 1 for f, u in zip(runs[1][1], runs[0][1])), (runs[1][1], runs[0][1])
+
+
 _CFG2 = {}
 
 
