@@ -213,6 +213,13 @@ int  tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_host, uint
               float *logits_dev, int32_t *argmax_dev, void *compute_stream, void *copy_stream,
               tgp_step_stats *stats);
 
+/* Copy coalescing: consecutive host-to-device commands of the plan whose pool ranges and arena slots continue one another
+ * (sub-ranges that were registered next to each other and placed next to each other), that need no further wait and
+ * together stay under 1 MiB, are carried by one cudaMemcpyAsync (a pinned copy of a few hundred KiB is mostly latency).
+ * The schedule itself does not change.  tgp_k_merge_copies(0) switches it off (process-wide; default on);
+ * tgp_copies_issued() returns the host-to-device copies issued since the last tgp_run_reset(). */
+int  tgp_k_merge_copies(int enable);
+int  tgp_copies_issued(tgp_ctx *ctx, uint64_t *n);
 /* MoE profile (Section IV-D: one profiling pass recovers which tensors the kernels really touch): the tokens
  * routed to each expert, per step and layer, in the run since the last tgp_run_reset(): uint32 [steps, L, E].
  * Two-call form: out == NULL returns the element count in *n.  Feed it to tgp_model_trace() to trace exactly the
@@ -305,6 +312,11 @@ int  tgp_k_gemm_group_select(int enable);
 /* Name of the kernel that the calling thread's last tgp_k_gemm() / tgp_k_gemm_group() launched (the choice depends on
  * M, n, K and the GPU's SM count), as a NUL-terminated string of at most capacity - 1 characters; "" before the first. */
 int  tgp_k_gemm_last_kernel(char *name, uint32_t capacity);
+/* Prefill (more than 128 activation rows, dense FFN): the tensor-core GEMM that computes the up projection applies SwiGLU in
+ * its epilogue - a = bf16(silu(g) * u) from the gate projection already in memory and the accumulator - so the up
+ * projection is never stored, the gate is read once and the step's SwiGLU op launches nothing (at the 70B shape that is
+ * 7.5 GB of HBM traffic per layer).  Bit-identical to the separate kernel; 0 switches it off.  Process-wide; default on. */
+int  tgp_k_swiglu_epilogue(int enable);
 /* Decode steps of at most two sequences on models whose rows hold at most 1024 elements (d for the norms, F for SwiGLU):
  * tgp_step() lets the products that consume a normalised state or a SwiGLU output compute it themselves (each warp of
  * the weight-streaming kernel redoes the row, bit for bit as the separate kernel would), so those ops launch nothing.

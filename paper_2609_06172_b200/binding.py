@@ -109,6 +109,9 @@ _SIGS = {
     "tgp_k_gemm_last_kernel": [C.c_char_p, _U32],
     "tgp_k_gemm_select": [C.c_int],
     "tgp_k_decode_fuse": [C.c_int],
+    "tgp_k_merge_copies": [C.c_int],
+    "tgp_copies_issued": [_P, C.POINTER(_U64)],
+    "tgp_k_swiglu_epilogue": [C.c_int],
     "tgp_k_attn_select": [C.c_int],
     "tgp_k_attn_decode_select": [C.c_int],
     "tgp_k_gemv_overlap": [C.c_int],
@@ -257,6 +260,11 @@ class Ctx:
     def trace_ops(self):
         """The recorded trace decoded: a list of (step, site, layer, kind, flops, hbm bytes, [(tensor, mode, touched)])."""
         return parse_trace(self.trace_export())
+
+    def copies_issued(self):
+        n = _U64()
+        self._ck(lib().tgp_copies_issued(self._h, C.byref(n)), "tgp_copies_issued")
+        return n.value
 
     def replan_begin(self, first_step, op_ns=None):
         """Starts planning the steps from first_step on (helper thread); op_ns: uint64 per op of the whole trace, or None."""
@@ -472,6 +480,14 @@ def k_gemm_last_kernel():
 
 def k_attn_decode_select(impl):
     _k(lib().tgp_k_attn_decode_select(impl), "tgp_k_attn_decode_select")
+
+
+def k_swiglu_epilogue(enable):
+    _k(lib().tgp_k_swiglu_epilogue(int(enable)), "tgp_k_swiglu_epilogue")
+
+
+def k_merge_copies(enable):
+    _k(lib().tgp_k_merge_copies(int(enable)), "tgp_k_merge_copies")
 
 
 def k_decode_fuse(enable):

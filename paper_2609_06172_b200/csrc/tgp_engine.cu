@@ -26,6 +26,8 @@ extern thread_local uint64_t tgpk_launches;
 #define CU(ctx, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return tgp_fail(ctx, TGP_E_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } while (0)
 
 static int g_small_copy_streams = 1;     // plans of small copies use three copy streams (0: always one)
+static int g_merge_copies = 1;           // adjacent small loads that need no further wait share one cudaMemcpyAsync
+static int g_fuse_swiglu_epilogue = 1;   // prefill: the up projection's tensor-core epilogue applies SwiGLU (0: separate kernel)
 static int g_fuse_small = 0;             // decode steps of small models: RMSNorm and SwiGLU are computed by the products that consume them (off:
                                          // 32 instead of 50 launches per step of the tiny configuration, but a span waits for all its copies, and
                                          // with a ring of two blocks copies and kernels already alternate more than they overlap: 0.56 against 0.58)
@@ -60,6 +62,7 @@ struct TgpEngine {
     int32_t waited[NCOPY] = {-1, -1, -1};
     bool wb_pend[NCOPY] = {false, false, false};
     size_t next_cmd = 0;
+    uint64_t n_dma = 0;                                   // host-to-device copies issued since the last reset (merged commands count once)
     uint32_t next_step = 0, pos = 0;
     const int32_t *tok_src = nullptr;
     int device = -1;
@@ -245,6 +248,7 @@ int tgp_run_reset(tgp_ctx *ctx) {
         ctx->base_plan = TgpPlan();
     }
     e->next_cmd = 0; e->next_step = 0; e->pos = 0; e->wb_pending = false; e->copy_waited_op = -1; e->tok_src = nullptr;
+    e->n_dma = 0;
     e->rr = 0;
     for (int i = 0; i < TgpEngine::NCOPY; ++i) { e->waited[i] = -1; e->wb_pend[i] = false; }
     {   // small-copy plans use all copy streams (decided per run: the plan may have changed)
@@ -286,46 +290,56 @@ static int pump(tgp_ctx *ctx, int32_t limit, cudaStream_t copy, uint32_t *n_cmds
             CU(ctx, cudaEventRecord(e->wb_ev, e->wb_stream));
             e->wb_pending = true;
             for (bool &b : e->wb_pend) b = true;
-        } else if (e->n_copy > 1) {
-            // small copies: this command goes to the next of the copy streams; each stream keeps its own record of what
-            // it has already waited for
-            const uint32_t si = e->rr++ % e->n_copy;
+        } else {
+            // Placement (H2D or ALLOC).  With several copy streams (plans of small copies) this command goes to the next
+            // of them, each stream keeping its own record of what it has already waited for.
+            const uint32_t si = e->n_copy > 1 ? e->rr++ % e->n_copy : 0;
             cudaStream_t mine = si ? e->xcopy[si - 1] : copy;
-            if (c.wait_op > e->waited[si]) {
+            int32_t &waited = e->n_copy > 1 ? e->waited[si] : e->copy_waited_op;
+            bool &wbp = e->n_copy > 1 ? e->wb_pend[si] : e->wb_pending;
+            if (c.wait_op > waited) {
                 int rc = get_event(ctx, e->done_ev, (size_t)c.wait_op, &ev);
                 if (rc) return rc;
                 CU(ctx, cudaStreamWaitEvent(mine, ev, 0));
-                e->waited[si] = c.wait_op;
+                waited = c.wait_op;
             }
-            if (e->wb_pend[si]) { CU(ctx, cudaStreamWaitEvent(mine, e->wb_ev, 0)); e->wb_pend[si] = false; }
-            if (c.kind == CMD_H2D) CU(ctx, cudaMemcpyAsync(dev, host, c.bytes, cudaMemcpyHostToDevice, mine));
-            if (pl.op_last_place[c.first_use] == (int32_t)e->next_cmd) {
-                // commands are in first-use order, so everything the other streams hold is wanted by this op or an
-                // earlier one: this stream waits for what they hold now, and its event covers all of it
-                for (uint32_t sj = 0; sj < e->n_copy; ++sj) {
-                    if (sj == si) continue;
-                    cudaStream_t other = sj ? e->xcopy[sj - 1] : copy;
-                    CU(ctx, cudaEventRecord(e->xmark[sj], other));
-                    CU(ctx, cudaStreamWaitEvent(mine, e->xmark[sj], 0));
+            if (wbp) { CU(ctx, cudaStreamWaitEvent(mine, e->wb_ev, 0)); wbp = false; }
+            // Coalescing: the commands that follow are carried by the same copy when they are loads that need no further
+            // wait, their pool ranges and arena slots continue this one's at the same distance (the alignment padding
+            // between two sub-ranges travels along: it lies inside the earlier tensor's slot), and the whole stays small -
+            // a copy of a few hundred KiB is mostly latency, while merging megabytes would only delay the first tensor.
+            size_t last = e->next_cmd;
+            uint64_t span_bytes = c.bytes;
+            if (c.kind == CMD_H2D && g_merge_copies)
+                while (last + 1 < pl.cmds.size()) {
+                    const TgpCmd &d = pl.cmds[last + 1], &p = pl.cmds[last];
+                    if (d.kind != CMD_H2D || d.wait_op > waited || d.wait_op > limit || ctx->tensors[d.tensor].pool != ctx->tensors[c.tensor].pool) break;
+                    if (d.pool_off < p.pool_off + p.bytes || d.pool_off - p.pool_off != d.arena_off - p.arena_off || d.pool_off - (p.pool_off + p.bytes) >= 512) break;
+                    if (d.pool_off + d.bytes - c.pool_off > (1u << 20)) break;
+                    span_bytes = d.pool_off + d.bytes - c.pool_off;
+                    ++last;
                 }
-                int rc = get_event(ctx, e->copied_ev, (size_t)c.first_use, &ev);
+            if (c.kind == CMD_H2D) CU(ctx, cudaMemcpyAsync(dev, host, span_bytes, cudaMemcpyHostToDevice, mine));
+            for (size_t k = e->next_cmd; k <= last; ++k) {
+                const TgpCmd &m = pl.cmds[k];
+                if (pl.op_last_place[m.first_use] != (int32_t)k) continue;
+                if (e->n_copy > 1) {
+                    // commands are in first-use order, so everything the other streams hold is wanted by this op or an
+                    // earlier one: this stream waits for what they hold now, and its event covers all of it
+                    for (uint32_t sj = 0; sj < e->n_copy; ++sj) {
+                        if (sj == si) continue;
+                        cudaStream_t other = sj ? e->xcopy[sj - 1] : copy;
+                        CU(ctx, cudaEventRecord(e->xmark[sj], other));
+                        CU(ctx, cudaStreamWaitEvent(mine, e->xmark[sj], 0));
+                    }
+                }
+                int rc = get_event(ctx, e->copied_ev, (size_t)m.first_use, &ev);
                 if (rc) return rc;
                 CU(ctx, cudaEventRecord(ev, mine));
             }
-        } else {
-            if (c.wait_op > e->copy_waited_op) {
-                int rc = get_event(ctx, e->done_ev, (size_t)c.wait_op, &ev);
-                if (rc) return rc;
-                CU(ctx, cudaStreamWaitEvent(copy, ev, 0));
-                e->copy_waited_op = c.wait_op;
-            }
-            if (e->wb_pending) { CU(ctx, cudaStreamWaitEvent(copy, e->wb_ev, 0)); e->wb_pending = false; }
-            if (c.kind == CMD_H2D) CU(ctx, cudaMemcpyAsync(dev, host, c.bytes, cudaMemcpyHostToDevice, copy));
-            if (pl.op_last_place[c.first_use] == (int32_t)e->next_cmd) {
-                int rc = get_event(ctx, e->copied_ev, (size_t)c.first_use, &ev);
-                if (rc) return rc;
-                CU(ctx, cudaEventRecord(ev, copy));
-            }
+            if (n_cmds) *n_cmds += (uint32_t)(last - e->next_cmd);
+            if (c.kind == CMD_H2D) e->n_dma += 1;
+            e->next_cmd = last;
         }
         if (n_cmds) ++*n_cmds;
         ++e->next_cmd;
@@ -580,7 +594,8 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
     if (objects && (rc = prefetch_objects(ctx, st.op0, cp, &object_bytes_asked))) return rc;
     if (ring && (rc = pump(ctx, (int32_t)st.op0 - 1, cp, &n_cmds))) return rc;
     if (hints && (rc = pump_managed(ctx, (int32_t)st.op0 - 1, cp, &n_cmds))) return rc;
-    const uint32_t qd = c.Hq * c.Dh, kd = c.Hkv * c.Dh;
+    const uint32_t qd = c.Hq * c.Dh;
+    int32_t glu_fused_layer = -1;                            // layer whose SwiGLU was applied by its up projection's epilogue
     for (uint32_t i = st.op0; i < st.op0 + st.nops; ++i) {
         const TgpOp &o = ctx->ops[i];
         // Consecutive weight-block products of a decode step that read the same activations (the q, k and v projections, gate
@@ -720,6 +735,13 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
             }
             GemmTarget t;
             if (!gemm_target(e, c, r, M, B, logits_dev, &t)) return tgp_fail(ctx, TGP_E_MISMATCH, "GEMM op on a tensor that is not a weight");
+            if (r.kind == TGP_K_WU && g_fuse_swiglu_epilogue && tgpk_swiglu_fusable(t.Mrows)) {
+                // prefill: the gate projection of these rows is complete (its blocks come first), so the up projection's
+                // epilogue applies SwiGLU itself and stores bf16 a; the step's SwiGLU op then has nothing left to do
+                rc = tgpk_gemm_tc(t.A, W, t.C, t.Mrows, r.rows, K, t.ldc, r.row0, 0, cs, e->g32, e->ab);
+                glu_fused_layer = o.layer;
+                break;
+            }
             rc = tgpk_gemm(t.A, W, t.C, t.Mrows, r.rows, K, t.ldc, r.row0, t.acc, cs);
             break;
         }
@@ -780,6 +802,7 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
                 rc = tgpk_gemm_group_fused(2, nullptr, 0, nullptr, 0.f, e->g32, e->u32, span - 1, gW, gC, gn, gld, g0.Mrows, gK, g0.acc, cs);
                 break;
             }
+            if (!c.E && glu_fused_layer == o.layer) break;                  // done in the up projection's epilogue
             if (c.E) { if (e->cur_expert >= 0 && e->cnt[e->cur_expert]) rc = tgpk_swiglu(e->g32, e->u32, e->ab, (uint64_t)e->cnt[e->cur_expert] * c.F, cs); }
             else rc = tgpk_swiglu(e->g32, e->u32, e->ab, (uint64_t)M * c.F, cs);
             break;
@@ -894,6 +917,22 @@ extern "C" int tgp_replan_commit(tgp_ctx *ctx) {
     uint64_t biggest = 0;
     for (const TgpCmd &c : ctx->plan.cmds) if (c.kind == CMD_H2D && c.bytes > biggest) biggest = c.bytes;
     e->n_copy = (biggest && biggest <= (512u << 10) && g_small_copy_streams) ? TgpEngine::NCOPY : 1;
+    return TGP_OK;
+}
+
+extern "C" int tgp_k_merge_copies(int enable) {
+    g_merge_copies = enable ? 1 : 0;
+    return TGP_OK;
+}
+
+extern "C" int tgp_copies_issued(tgp_ctx *ctx, uint64_t *n) {
+    if (!ctx || !ctx->eng || !n) return TGP_E_STATE;
+    *n = ctx->eng->n_dma;
+    return TGP_OK;
+}
+
+extern "C" int tgp_k_swiglu_epilogue(int enable) {
+    g_fuse_swiglu_epilogue = enable ? 1 : 0;
     return TGP_OK;
 }
 

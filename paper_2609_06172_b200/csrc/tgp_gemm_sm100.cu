@@ -12,6 +12,7 @@
 // and the CTA drains and returns instead of hanging the GPU.
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <cuda_bf16.h>
 #include <cudaTypedefs.h>
 #include <cstdint>
 #include "tgp.h"
@@ -24,6 +25,35 @@ using namespace tgp_sm100;
 constexpr int BK = 64, GROUP_M = 16;
 
 __device__ int g_gemm_tc_error = 0;                    // 0 ok; else (role << 8) | stage of the first wait that ran out
+
+// Optional epilogue: the accumulator is the up projection u of a SwiGLU FFN and the gate projection g of the same
+// elements is already in memory (fp32, same geometry as C).  Instead of storing u, the epilogue stores
+// a = bf16(g / (1 + exp(-g)) * u) - the arithmetic of the stand-alone SwiGLU kernel, on the very values it would have
+// read - so u never goes to memory, g is read once instead of twice and the SwiGLU launch disappears.
+struct Epi { const float *gate; __nv_bfloat16 *aout; };
+
+// 32 consecutive elements of one output row, element offset `off` in C's geometry, `cnt` of them inside the matrix
+__device__ __forceinline__ void swiglu_store32(const Epi &ep, size_t off, const float *v, uint32_t cnt) {
+    const float *g = ep.gate + off;
+    __nv_bfloat16 *a = ep.aout + off;
+    if (cnt == 32 && (off & 7) == 0 && ((reinterpret_cast<uintptr_t>(ep.gate) | reinterpret_cast<uintptr_t>(ep.aout)) & 15u) == 0) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+            const float4 g0 = *reinterpret_cast<const float4 *>(g + j), g1 = *reinterpret_cast<const float4 *>(g + j + 4);
+            const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                __nv_bfloat162 pk = __floats2bfloat162_rn(gv[2 * i] / (1.0f + expf(-gv[2 * i])) * v[j + 2 * i],
+                                                          gv[2 * i + 1] / (1.0f + expf(-gv[2 * i + 1])) * v[j + 2 * i + 1]);
+                w[i] = *reinterpret_cast<uint32_t *>(&pk);
+            }
+            *reinterpret_cast<uint4 *>(a + j) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    } else {
+        for (uint32_t j = 0; j < cnt; ++j) a[j] = __float2bfloat16_rn(g[j] / (1.0f + expf(-g[j])) * v[j]);
+    }
+}
 
 template <int BN, int ST, int KH>
 struct Smem {
@@ -39,7 +69,7 @@ struct Smem {
 // is bound by.
 template <int BN, int ST, int KH, bool SWAP>
 __global__ void __launch_bounds__(192) tgp_matmul_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                                                      float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
+                                                      float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, const Epi ep) {
     extern __shared__ uint8_t smem_raw[];
     using S = Smem<BN, ST, KH>;
     constexpr int STAGES = ST;                      // depth of this instantiation's TMA ring
@@ -142,7 +172,8 @@ __global__ void __launch_bounds__(192) tgp_matmul_tc_kernel(const __grid_constan
                 } else if (row < M) {
                     float *dst = C + (size_t)row * ldc + col0 + n0 + c * 32;
                     const uint32_t col = n0 + c * 32;
-                    if (vec && col + 32 <= n) {
+                    if (ep.aout) { if (col < n) swiglu_store32(ep, (size_t)row * ldc + col0 + col, v, min(32u, n - col)); }
+                    else if (vec && col + 32 <= n) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
                             float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
@@ -173,7 +204,7 @@ __global__ void __launch_bounds__(192) tgp_matmul_tc_kernel(const __grid_constan
 constexpr int P_BN = 256, P_STAGES = 4;
 
 __global__ void __launch_bounds__(192, 1) tgp_matmul_tc_persistent_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                                                                    float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
+                                                                    float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, const Epi ep) {
     extern __shared__ uint8_t smem_raw[];
     constexpr int A_BYTES = BM * BK * 2, B_BYTES = P_BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -277,7 +308,8 @@ __global__ void __launch_bounds__(192, 1) tgp_matmul_tc_persistent_kernel(const 
                 const uint32_t col = n0 + c * 32;
                 if (row < M && col < n) {
                     float *dst = C + (size_t)row * ldc + col0 + col;
-                    if (vec && col + 32 <= n) {
+                    if (ep.aout) swiglu_store32(ep, (size_t)row * ldc + col0 + col, v, min(32u, n - col));
+                    else if (vec && col + 32 <= n) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
                             float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
@@ -318,7 +350,7 @@ __global__ void __launch_bounds__(192, 1) tgp_matmul_tc_persistent_kernel(const 
 constexpr int Q_HALVES = 2, Q_STAGES = 6 / Q_HALVES;   // a stage holds Q_HALVES 64-wide K blocks
 
 __global__ void __launch_bounds__(192, 1) tgp_matmul_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                                                              float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
+                                                              float *__restrict__ C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, const Epi ep) {
     extern __shared__ uint8_t smem_raw[];
     constexpr int A_BYTES = BM * BK * 2, B_BYTES = (P_BN / 2) * BK * 2, STAGE_BYTES = Q_HALVES * (A_BYTES + B_BYTES);
     constexpr int QK = Q_HALVES * BK;
@@ -431,7 +463,8 @@ __global__ void __launch_bounds__(192, 1) tgp_matmul_tc_pair_kernel(const __grid
                 const uint32_t col = n0 + c * 32;
                 if (row < M && col < n) {
                     float *dst = C + (size_t)row * ldc + col0 + col;
-                    if (vec && col + 32 <= n) {
+                    if (ep.aout) swiglu_store32(ep, (size_t)row * ldc + col0 + col, v, min(32u, n - col));
+                    else if (vec && col + 32 <= n) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
                             float4 o = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
@@ -470,22 +503,25 @@ bool make_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t K, uin
 extern thread_local uint64_t tgpk_launches;
 
 template <int BN, int ST, int KH, bool SWAP = false>
-static bool launch_tile(const CUtensorMap &ma, const CUtensorMap &mb, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
+static bool launch_tile(const CUtensorMap &ma, const CUtensorMap &mb, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st, const Epi ep = Epi{nullptr, nullptr}) {
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(tgp_matmul_tc_kernel<BN, ST, KH, SWAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<BN, ST, KH>::TOTAL) != cudaSuccess) return false;
         attr_set = true;
     }
     dim3 grid(((M + BM - 1) / BM) * ((n + BN - 1) / BN));
-    tgp_matmul_tc_kernel<BN, ST, KH, SWAP><<<grid, 192, Smem<BN, ST, KH>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
+    tgp_matmul_tc_kernel<BN, ST, KH, SWAP><<<grid, 192, Smem<BN, ST, KH>::TOTAL, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate, ep);
     return true;
 }
 
 static int g_tc_variant = 0;     // 0 auto, 1 force the 128x128 per-tile kernel, 2 the persistent 128x256 kernel, 3 the paired 256x256 kernel,
                                  // 4 the per-tile kernel with the weights as the 128-row operand (M <= 128 only; else as 0)
 
-int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st) {
+int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st,
+                 const float *gate, void *aout) {
     constexpr int BN = 128;
+    const Epi ep{aout ? gate : nullptr, gate ? (__nv_bfloat16 *)aout : nullptr};
+    if (ep.aout && accumulate) return TGP_E_INVAL;
     if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(W)) & 15u) return TGP_E_INVAL;     // TMA needs 16-byte aligned bases
     if (K % 8) return TGP_E_INVAL;                                                                       // and 16-byte row strides
     static int sms = 0;
@@ -496,7 +532,7 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
     // than 32 rows from 32 tiles on (n=4096, K=14336, M=64: 48 us against 70 us); with fewer tiles the weight-streaming
     // kernels and the narrow tiles below have more CTAs at work
     const uint32_t w_tiles = (n + BM - 1) / BM;
-    if (M <= 128 && (g_tc_variant == 4 || (g_tc_variant == 0 && M <= 64 && (w_tiles >= 64 || (M > 32 && w_tiles >= 32))))) {
+    if (!ep.aout && M <= 128 && (g_tc_variant == 4 || (g_tc_variant == 0 && M <= 64 && (w_tiles >= 64 || (M > 32 && w_tiles >= 32))))) {
         CUtensorMap mw, mx;
         const uint32_t bx = M <= 32 ? 32 : M <= 64 ? 64 : 128;
         if (!make_map(&mw, W, n, K, BM) || !make_map(&mx, A, M, K, bx)) return TGP_E_CUDA;
@@ -541,7 +577,7 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
         attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, tgp_matmul_tc_pair_kernel, ma, mb, C, M, n, K, ldc, col0, accumulate) != cudaSuccess) return TGP_E_CUDA;
+        if (cudaLaunchKernelEx(&cfg, tgp_matmul_tc_pair_kernel, ma, mb, C, M, n, K, ldc, col0, accumulate, ep) != cudaSuccess) return TGP_E_CUDA;
     } else if (persistent) {
         constexpr int SMEM = P_STAGES * (BM * BK * 2 + P_BN * BK * 2) + 128 + 1024;
         static bool attr_p = false;
@@ -549,16 +585,16 @@ int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n,
             if (cudaFuncSetAttribute(tgp_matmul_tc_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess) return TGP_E_CUDA;
             attr_p = true;
         }
-        tgp_matmul_tc_persistent_kernel<<<tiles_p < (uint32_t)sms ? tiles_p : (uint32_t)sms, 192, SMEM, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate);
+        tgp_matmul_tc_persistent_kernel<<<tiles_p < (uint32_t)sms ? tiles_p : (uint32_t)sms, 192, SMEM, st>>>(ma, mb, C, M, n, K, ldc, col0, accumulate, ep);
     } else if (bn == 128) {
         // fewer tiles than SMs: one CTA per SM, so the ring may take all of shared memory (a 3-stage ring leaves a lone
         // CTA waiting on L2 latency); otherwise two CTAs per SM with three stages each
         const bool lone = tm * ((n + 127) / 128) <= (uint32_t)sms;
-        if (!(lone ? launch_tile<128, 2, 3>(ma, mb, C, M, n, K, ldc, col0, accumulate, st) : launch_tile<128, 3, 1>(ma, mb, C, M, n, K, ldc, col0, accumulate, st))) return TGP_E_CUDA;
+        if (!(lone ? launch_tile<128, 2, 3>(ma, mb, C, M, n, K, ldc, col0, accumulate, st, ep) : launch_tile<128, 3, 1>(ma, mb, C, M, n, K, ldc, col0, accumulate, st, ep))) return TGP_E_CUDA;
     } else if (bn == 64) {
-        if (!launch_tile<64, 3, 3>(ma, mb, C, M, n, K, ldc, col0, accumulate, st)) return TGP_E_CUDA;
+        if (!launch_tile<64, 3, 3>(ma, mb, C, M, n, K, ldc, col0, accumulate, st, ep)) return TGP_E_CUDA;
     } else {
-        if (!launch_tile<32, 3, 3>(ma, mb, C, M, n, K, ldc, col0, accumulate, st)) return TGP_E_CUDA;
+        if (!launch_tile<32, 3, 3>(ma, mb, C, M, n, K, ldc, col0, accumulate, st, ep)) return TGP_E_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return TGP_E_CUDA;
     tgpk_launches += 1;

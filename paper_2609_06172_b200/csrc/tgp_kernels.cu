@@ -1654,6 +1654,8 @@ int tgpk_gemm(const void *A, const void *W, float *C, uint32_t M, uint32_t n, ui
     return TGP_OK;
 }
 
+bool tgpk_swiglu_fusable(uint32_t M) { return M > 128 && g_gemm_impl == 0; }
+
 int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb, const TgpTilePtrs &tiles, const float *cos_t, const float *sin_t,
                  const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0, cudaStream_t st) {
     if (!B || !q_len) return TGP_OK;

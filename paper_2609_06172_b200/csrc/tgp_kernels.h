@@ -19,7 +19,12 @@ uint32_t tgpk_gemm_group_key(uint32_t M, uint32_t n, uint32_t K);
 int tgpk_gemm_group(const void *A, uint32_t count, const void *const *W, float *const *C, const uint32_t *n, const uint32_t *ldc, uint32_t M, uint32_t K,
                     int accumulate, cudaStream_t st);
 // tcgen05 path (tgp_gemm_sm100.cu): any M, n; K % 8 == 0; A and W 16-byte aligned
-int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st);
+// gate / aout (both or neither): the accumulator is the up projection of a SwiGLU FFN; instead of storing it to C the epilogue
+// stores aout[m, col0 + j] = bf16(silu(gate[m, col0 + j]) * acc) (gate fp32 and aout bf16 in C's geometry); not with accumulate
+int tgpk_gemm_tc(const void *A, const void *W, float *C, uint32_t M, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate, cudaStream_t st,
+                 const float *gate = nullptr, void *aout = nullptr);
+// true if a product of M activation rows takes the tensor-core GEMM, whose epilogue can apply SwiGLU (M > 128, tensor cores selected)
+bool tgpk_swiglu_fusable(uint32_t M);
 int tgpk_rope_kv(const float *q32, const float *k32, const float *v32, void *qb, const TgpTilePtrs &tiles, const float *cos_t, const float *sin_t,
                  const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0, cudaStream_t st);
 int tgpk_attn(const void *qb, const TgpTilePtrs &tiles, uint32_t n_tiles, void *ob, const tgp_model_cfg *c, uint32_t B, uint32_t q_len, uint32_t pos0,
