@@ -634,10 +634,10 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
         if (ring && o.kind == TGP_OP_GEMM && !e->tap) {
             uint32_t cnt = form_group(i, nullptr);
             // A grouped launch keeps the ring slots of its first blocks until its last block has arrived and the launch has
-            // run.  Against copies of megabytes that wait is a percent of the copy time; against copies of a few
-            // microseconds it is as long as the copies themselves, so small blocks whose slot a later copy waits for stay alone.
+            // run, and the copies that wait for those slots start that much later: the link idles.  So a block whose slot a
+            // later copy waits for ends its group (pinned blocks, which nothing waits for, group freely).
             for (uint32_t j = 0; j + 1 < cnt; ++j)
-                if (ctx->plan.op_is_wait_target[i + j] && ctx->tensors[ctx->acc[ctx->ops[i + j].acc0].tensor].size < (2u << 20)) cnt = 0;
+                if (ctx->plan.op_is_wait_target[i + j]) { cnt = j + 1; break; }
             if (cnt >= 2) span = cnt;
             for (uint32_t j = 0; j < span && span > 1 && g_expert >= 0; ++j) {       // what run_expert_block does around an expert's products
                 const TgpRole &r = *role_of(ctx, ctx->ops[i + j], 0);

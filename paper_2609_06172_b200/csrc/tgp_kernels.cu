@@ -1274,19 +1274,26 @@ template <int NB, int U, int NW, int ROWS, int RG>
 __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_group_kernel(const bf16 *A, const GemvParts p, uint32_t Mrows, uint32_t groups_total,
                                                               uint32_t K, int accumulate, uint32_t rpc) {
     constexpr int UL = ROWS == 8 ? 2 * U : U;             // half a tile per load step: twice the steps in flight
-    constexpr int G = RG, SUB = UL / G;                  // SUB load steps of G groups in flight at a time: as many loads as UL of one
-    static_assert(UL % G == 0, "row groups per CTA must divide the load steps");
+    constexpr int G = RG, SK = UL / (2 * G);              // a register set holds SK load steps of G groups: two sets are as many loads as UL steps of one group
+    static_assert(UL % (2 * G) == 0 && SK >= 1, "row groups per CTA must divide half the load steps");
     __shared__ float part[NW][G * NB * 4][32];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, c = lane & 3;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    bool synced = false;
-    for (uint32_t grp0 = blockIdx.x * G; grp0 < groups_total; grp0 += gridDim.x * G) {
-        // which block a group belongs to: looked up here for the weights and again after the K loop for the output, so
-        // that the output's pointer and stride do not occupy registers while the loads are in flight
-        const bf16 *wlo[G], *whi[G];
+    uint32_t grp0 = blockIdx.x * G;
+    if (grp0 >= groups_total) return;
+    const bf16 *wlo[G], *whi[G];
+    uint4 lo[2][G][SK], hi[2][G][SK];                     // two register sets of SK load steps of every group
+    // the activation fragments of a set are loaded with its weights (they come from L2 more often than from L1 -
+    // a long K does not fit there - and would otherwise be waited for inside the MMA sequence)
+    constexpr bool XPRE = !(NB == 1 && ROWS == 8 && G == 1) && !(NB == 2 && G == 1);     // (those instances have no registers left for them)
+    uint4 xs[2][XPRE ? SK : 1][XPRE ? NB : 1];
+    float acc[G][NB][4];
+    // which block a group belongs to: looked up here for the weights and again after the K loop for the output, so
+    // that the output's pointer and stride do not occupy registers while the loads are in flight
+    auto locate = [&](uint32_t first) {
 #pragma unroll
         for (int r = 0; r < G; ++r) {
-            const uint32_t grp = min(grp0 + r, groups_total - 1);          // a group past the end re-reads the last one, never stored
+            const uint32_t grp = min(first + r, groups_total - 1);         // a group past the end re-reads the last one, never stored
             const bf16 *W = p.W[0];
             uint32_t n = p.n[0], local = grp;
             {
@@ -1305,42 +1312,95 @@ __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_group_kernel(const bf
             wlo[r] = W + (size_t)min(local * rpc + g, rlast) * K + c * 8;
             whi[r] = W + (size_t)min(local * rpc + g + 8, rlast) * K + c * 8;
         }
-        float acc[G][NB][4];
+    };
+    auto issue = [&](auto set, uint32_t kb) {              // SK load steps of every group, from column kb on, into one register set
+        constexpr int S = decltype(set)::value;
+#pragma unroll
+        for (int u = 0; u < SK; ++u) {
+            const uint32_t k = kb + 32 * u;
+#pragma unroll
+            for (int r = 0; r < G; ++r) {
+                lo[S][r][u] = k < K ? __ldcs(reinterpret_cast<const uint4 *>(wlo[r] + k)) : make_uint4(0, 0, 0, 0);
+                hi[S][r][u] = (k < K && ROWS == 16) ? __ldcs(reinterpret_cast<const uint4 *>(whi[r] + k)) : make_uint4(0, 0, 0, 0);   // ROWS == 8: the upper half of the tile stays empty
+            }
+        }
+    };
+    auto issue_act = [&](auto set, uint32_t kb) {          // the activation fragments that go with a set; only after griddepcontrol.wait
+        constexpr int S = decltype(set)::value;
+        if constexpr (XPRE) {
+#pragma unroll
+            for (int u = 0; u < SK; ++u) {
+                const uint32_t k = kb + 32 * u;
+#pragma unroll
+                for (int b = 0; b < NB; ++b)
+                    xs[S][u][b] = (k < K && b * 8 + g < Mrows) ? ld_act(reinterpret_cast<const uint4 *>(A + (size_t)(b * 8 + g) * K + k + c * 8)) : make_uint4(0, 0, 0, 0);
+            }
+        }
+    };
+    auto consume = [&](auto set, uint32_t kb) {
+        constexpr int S = decltype(set)::value;
+#pragma unroll
+        for (int u = 0; u < SK; ++u) {
+            const uint32_t k = kb + 32 * u;
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                const uint32_t m = b * 8 + g;
+                uint4 xv;
+                if constexpr (XPRE) xv = xs[S][u][b];
+                else xv = (k < K && m < Mrows) ? ld_act(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k + c * 8)) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int r = 0; r < G; ++r) {
+                    mma_bf16_16816(acc[r][b], lo[S][r][u].x, hi[S][r][u].x, lo[S][r][u].y, hi[S][r][u].y, xv.x, xv.y);
+                    mma_bf16_16816(acc[r][b], lo[S][r][u].z, hi[S][r][u].z, lo[S][r][u].w, hi[S][r][u].w, xv.z, xv.w);
+                }
+            }
+        }
+    };
+    auto clear = [&]() {
 #pragma unroll
         for (int r = 0; r < G; ++r)
 #pragma unroll
             for (int b = 0; b < NB; ++b) { acc[r][b][0] = acc[r][b][1] = acc[r][b][2] = acc[r][b][3] = 0.f; }
-        for (uint32_t k0 = warp * 32 * UL; k0 < K; k0 += NW * 32 * UL) {
-#pragma unroll
-            for (int sub = 0; sub < G; ++sub) {
-                uint4 lo[G][SUB], hi[G][SUB];
-#pragma unroll
-                for (int u = 0; u < SUB; ++u) {
-                    const uint32_t k = k0 + 32 * (sub * SUB + u);
-#pragma unroll
-                    for (int r = 0; r < G; ++r) {
-                        lo[r][u] = k < K ? __ldcs(reinterpret_cast<const uint4 *>(wlo[r] + k)) : make_uint4(0, 0, 0, 0);
-                        hi[r][u] = (k < K && ROWS == 16) ? __ldcs(reinterpret_cast<const uint4 *>(whi[r] + k)) : make_uint4(0, 0, 0, 0);   // ROWS == 8: the upper half of the tile stays empty
-                    }
-                }
-                if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
-#pragma unroll
-                for (int u = 0; u < SUB; ++u) {
-                    const uint32_t k = k0 + 32 * (sub * SUB + u);
-#pragma unroll
-                    for (int b = 0; b < NB; ++b) {
-                        const uint32_t m = b * 8 + g;
-                        const uint4 xv = (k < K && m < Mrows) ? ld_act(reinterpret_cast<const uint4 *>(A + (size_t)m * K + k + c * 8)) : make_uint4(0, 0, 0, 0);
-#pragma unroll
-                        for (int r = 0; r < G; ++r) {
-                            mma_bf16_16816(acc[r][b], lo[r][u].x, hi[r][u].x, lo[r][u].y, hi[r][u].y, xv.x, xv.y);
-                            mma_bf16_16816(acc[r][b], lo[r][u].z, hi[r][u].z, lo[r][u].w, hi[r][u].w, xv.z, xv.w);
-                        }
-                    }
-                }
-            }
-        }
-        if (!synced) { asm volatile("griddepcontrol.wait;" ::: "memory"); synced = true; }
+    };
+    const std::integral_constant<int, 0> set0;
+    const std::integral_constant<int, 1> set1;
+    // One stream of loads over all the groups this CTA takes.  A warp's chunk of 32 * UL columns is G pairs of load steps;
+    // the two register sets alternate, a set is loaded again as soon as its MMAs are issued, so a warp always has one
+    // or two sets in flight - also across the end of a group: the next group's first pair is on its way while the CTA
+    // meets in shared memory to sum and store the group it has finished, and the memory pipe never drains.  Per group
+    // the k order of a warp's additions is that of its chunks, ascending: the bits do not depend on the pairing.  A warp
+    // whose first chunk lies beyond K runs one pair of zeros (the sums do not change).
+    uint32_t grp = grp0, k0 = warp * 32 * UL, pr = 0;       // the pair that is loaded next: group, chunk, pair within the chunk
+    auto advance = [&]() -> bool {                         // moves on by one pair; true: the pair just passed ended its group
+        if (++pr == (uint32_t)G) { pr = 0; k0 += NW * 32 * UL; }
+        if (k0 < K) return false;
+        grp += gridDim.x * G;
+        k0 = warp * 32 * UL;
+        pr = 0;
+        if (grp < groups_total) locate(grp);
+        return true;
+    };
+    locate(grp);
+    uint32_t kb_cur = k0;
+    issue(set0, kb_cur);
+    issue(set1, kb_cur + 32 * SK);
+    bool cur_last = advance();
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // weights are never written by a kernel: the activations are read from here on
+    issue_act(set0, kb_cur);
+    issue_act(set1, kb_cur + 32 * SK);
+    clear();
+    for (;;) {
+        const bool have_next = grp < groups_total;
+        const uint32_t kb_next = k0 + pr * 64 * SK;
+        consume(set0, kb_cur);
+        if (have_next) { issue(set0, kb_next); issue_act(set0, kb_next); }
+        consume(set1, kb_cur + 32 * SK);
+        if (have_next) { issue(set1, kb_next + 32 * SK); issue_act(set1, kb_next + 32 * SK); }
+        const bool next_last = have_next ? advance() : false;
+        kb_cur = kb_next;
+        if (!cur_last) { cur_last = next_last; continue; }
+        cur_last = next_last;
+        // this warp has finished the group(s) at grp0
 #pragma unroll
         for (int r = 0; r < G; ++r)
 #pragma unroll
@@ -1350,19 +1410,19 @@ __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_group_kernel(const bf
         __syncthreads();
         for (uint32_t v = threadIdx.x; v < G * NB * 4 * 32; v += NW * 32) {
             const uint32_t slot = v >> 5, ln = v & 31, r = slot / (NB * 4), b = (slot >> 2) % NB, i = slot & 3;
-            const uint32_t grp = grp0 + r;
-            if (grp >= groups_total) continue;
+            const uint32_t gi = grp0 + r;
+            if (gi >= groups_total) continue;
             float sum = 0.f;
 #pragma unroll
             for (int w = 0; w < NW; ++w) sum += part[w][slot][ln];
             float *C = p.C[0];
-            uint32_t ldc = p.ldc[0], n = p.n[0], row0 = grp * rpc;
+            uint32_t ldc = p.ldc[0], n = p.n[0], row0 = gi * rpc;
             {
                 uint32_t start = p.groups[0];
 #pragma unroll
                 for (int s = 1; s < (int)TGP_GEMM_GROUP_MAX; ++s)
                     if (s < (int)p.count) {
-                        if (grp >= start) { C = p.C[s]; ldc = p.ldc[s]; n = p.n[s]; row0 = (grp - start) * rpc; }
+                        if (gi >= start) { C = p.C[s]; ldc = p.ldc[s]; n = p.n[s]; row0 = (gi - start) * rpc; }
                         start += p.groups[s];
                     }
             }
@@ -1373,14 +1433,17 @@ __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_group_kernel(const bf
                 else *out = sum;
             }
         }
+        grp0 += gridDim.x * G;
+        if (grp0 >= groups_total) break;
         __syncthreads();
+        clear();
     }
 }
 
 // Which skinny kernel serves a block of n rows at M activation rows: NB groups of 8 activation rows, U load steps in
 // flight, and for blocks too small to give every SM eight 16-row warps the split-K kernel with NW warps per CTA over
 // ROWS rows.  The choice depends on the block alone, so a block computes the same bits alone or as part of a group.
-struct SkinnyPick { int nb, u, nw, rows; bool split; };
+struct SkinnyPick { int nb, u, nw, rows; bool split, persistent; };
 
 static int device_sms() {
     static int sms = 0;
@@ -1390,52 +1453,67 @@ static int device_sms() {
 
 static SkinnyPick pick_skinny(uint32_t M, uint32_t n, uint32_t K) {
     const uint32_t sms = (uint32_t)device_sms(), groups16 = (n + 15) / 16;
-    const bool few = groups16 < sms;                      // fewer 16-row groups than SMs: few CTAs, so each warp keeps twice the loads in flight
     SkinnyPick k;
     k.nb = M <= 8 ? 1 : M <= 16 ? 2 : 4;
-    k.u = M <= 16 ? (few ? 8 : 4) : (few ? 4 : 2);
     k.split = n < 16u * 8u * sms;                         // too few 16-row groups to give every SM eight warps
-    const bool wide = k.split && groups16 < 2u * sms;     // fewer than two 16-row groups per SM: 16 warps per CTA
-    // 16-row groups for at most half the SMs and a K long enough to keep all 16 warps loading: 8 rows per CTA, twice the
-    // CTAs (each CTA reads its slice of the activations whatever its rows, so fewer rows per CTA cost L2 traffic)
-    const bool half = wide && g_gemv_rows8 && 2 * groups16 <= sms && K >= 16u * 32u * 2u * (uint32_t)k.u;
-    k.nw = wide ? 16 : 8;
-    k.rows = half ? 8 : 16;
+    // fewer than two 16-row groups per SM: one persistent CTA per SM walks the row groups of the block, or of a list of such
+    // blocks (tgp_wstream_mma_group_kernel).  One choice per class of M for all of them, so that the pieces of a matrix share
+    // a launch whatever the rows of its last piece:
+    //   M <= 8   16 warps, 8 load steps per warp and chunk; blocks of few rows and a long K as 8-row groups (twice the CTAs)
+    //   M <= 16  8 warps of twice the registers, 16 load steps: room for the activation fragments of a register set
+    //   M <= 32  16 warps, 4 load steps
+    k.persistent = k.split && groups16 < 2u * sms;
+    if (k.persistent) {
+        k.nw = k.nb == 2 ? 8 : 16;
+        k.u = k.nb == 1 ? 8 : k.nb == 2 ? 16 : 4;
+        const bool half = k.nb == 1 && g_gemv_rows8 && 2 * groups16 <= sms && K >= 16u * 32u * 2u * (uint32_t)k.u;
+        k.rows = half ? 8 : 16;
+    } else {
+        k.nw = 8;
+        k.u = M <= 16 ? 4 : 2;
+        k.rows = 16;
+    }
     return k;
 }
 
 template <int NB, int U>
 static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint32_t Mrows, uint32_t K, int acc, cudaStream_t st) {
     static int blocks_per_sm = 0, blocks_per_sm_split = 0;
-    if (!blocks_per_sm && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, tgp_wstream_mma_kernel<NB, U>, 256, 0) != cudaSuccess || blocks_per_sm < 1)) blocks_per_sm = 1;
-    if (!blocks_per_sm_split && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm_split, tgp_wstream_mma_splitk_kernel<NB, U, 8, 16>, 256, 0) != cudaSuccess || blocks_per_sm_split < 1))
-        blocks_per_sm_split = 1;
+    constexpr bool STREAMS = U <= 4;                         // the load depths of the kernels that are not persistent
+    if constexpr (STREAMS) {
+        if (!blocks_per_sm && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm, tgp_wstream_mma_kernel<NB, U>, 256, 0) != cudaSuccess || blocks_per_sm < 1)) blocks_per_sm = 1;
+        if (!blocks_per_sm_split && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks_per_sm_split, tgp_wstream_mma_splitk_kernel<NB, U, 8, 16>, 256, 0) != cudaSuccess || blocks_per_sm_split < 1))
+            blocks_per_sm_split = 1;
+    }
     const uint32_t sms = (uint32_t)device_sms();
     uint32_t need = 0, rows_total = 0, rpc = (uint32_t)k.rows;
     if (k.split) for (uint32_t s = 0; s < p.count; ++s) { p.groups[s] = (p.n[s] + k.rows - 1) / k.rows; need += p.groups[s]; rows_total += p.n[s]; }
     else need = (p.n[0] + 16 * 8 - 1) / (16 * 8);           // whole blocks of many rows are launched alone
-    // several blocks in one launch: two row groups per CTA share each activation fragment when that still leaves a CTA per SM
-    // (four groups of activation rows would need twice the shared memory a CTA may declare)
-    const bool pairs = k.split && p.count > 1 && NB <= 2 && need >= 2 * sms;
-    if (pairs) need = (need + 1) / 2;
-    // (the grouped kernels are 16 warps of more than 64 registers each: one CTA per SM)
-    const uint32_t full = (k.split && p.count > 1) ? sms : sms * (uint32_t)(k.split ? blocks_per_sm_split : blocks_per_sm);
-    if (k.split && p.count > 1 && need > full && g_gemv_balance) {
-        // The grid is one persistent CTA per resident slot, each walking its share of the row groups: 256 pairs of groups
-        // on 148 CTAs give 108 of them two and 40 one.  Slightly smaller groups (14 rows instead of 16) make the count a
-        // multiple of the grid, so that no CTA waits for the others' second round; not below half a tile plus one row.
-        const uint32_t per_cta = pairs ? 2 : 1, rounds = (need + full - 1) / full, target = rounds * full;
-        uint32_t r = (rows_total + per_cta * target - 1) / (per_cta * target);
-        r = std::min<uint32_t>((uint32_t)k.rows, std::max<uint32_t>(r, (uint32_t)k.rows / 2 + 1));
-        for (;; ++r) {                                    // per-block rounding may push the count past the target: one more row then
-            uint32_t groups = 0;
-            for (uint32_t s = 0; s < p.count; ++s) groups += (p.n[s] + r - 1) / r;
-            if (r >= (uint32_t)k.rows || (groups + per_cta - 1) / per_cta <= target) break;
-        }
-        rpc = r;
-        uint32_t groups = 0;
-        for (uint32_t s = 0; s < p.count; ++s) { p.groups[s] = (p.n[s] + rpc - 1) / rpc; groups += p.groups[s]; }
-        need = (groups + per_cta - 1) / per_cta;
+    const bool persistent = k.persistent;                   // one block or several: the kernel that walks a list of row groups
+    // (the persistent kernels use the whole register file: one CTA per SM)
+    const uint32_t full = persistent ? sms : sms * (uint32_t)(k.split ? blocks_per_sm_split : blocks_per_sm);
+    uint32_t per_cta = 1;
+    if (persistent) {
+        // The grid is one persistent CTA per SM, each walking its share of the row groups, G groups at a time whose MMAs share
+        // each activation fragment (every CTA reads its K slices of all activation rows per round, so at one group per round
+        // that traffic equals the weights').  Rows per group r <= the tile's rows: fewer rows make more groups, so that a
+        // block of few rows reaches every SM and no CTA waits for the others' last round (4096 rows: 256 groups of 16 leave
+        // 40 SMs one round short, 293 of 14 do not) - but the rows a tile lacks are loaded all the same.  G and r are the
+        // pair with the least estimated time of the busiest CTA: rounds x (G x (r + tile rows) / 2 + 4 NB), in rows read.
+        const uint32_t tile = (uint32_t)k.rows, gmax = NB == 1 ? 2 : NB == 2 ? 4 : 1;
+        uint32_t best = 0xffffffffu, best_r = tile;
+        for (uint32_t G = gmax; G >= 1; G >>= 1)
+            for (uint32_t r = g_gemv_balance ? tile / 2 + 1 : tile; r <= tile; ++r) {
+                uint32_t groups = 0;
+                for (uint32_t s = 0; s < p.count; ++s) groups += (p.n[s] + r - 1) / r;
+                const uint32_t ctas = (groups + G - 1) / G, rounds = (ctas + full - 1) / full;
+                const uint32_t cost = rounds * (G * (r + tile) + 8 * NB);           // twice the estimate
+                if (cost < best) { best = cost; best_r = r; per_cta = G; }
+            }
+        rpc = best_r;
+        need = 0;
+        for (uint32_t s = 0; s < p.count; ++s) { p.groups[s] = (p.n[s] + rpc - 1) / rpc; need += p.groups[s]; }
+        need = (need + per_cta - 1) / per_cta;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(need < full ? need : full);
@@ -1448,38 +1526,29 @@ static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint3
     cfg.numAttrs = 1;
     uint32_t total = 0;
     for (uint32_t s = 0; k.split && s < p.count; ++s) total += p.groups[s];
-    tgpk_last_gemm_kernel = !k.split ? "tgp_wstream_mma_kernel" : p.count > 1 ? "tgp_wstream_mma_group_kernel" : "tgp_wstream_mma_splitk_kernel";
-    if (!k.split) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_kernel<NB, U>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
-    else if (p.count > 1) {                               // only few-row blocks are ever grouped: 16 warps, doubled load steps
-        if constexpr (NB <= 2 && U == 8) {
-            if (pairs && k.rows == 8) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 8, 2>, A, p, Mrows, total, K, acc, rpc);
-            else if (pairs) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 2>, A, p, Mrows, total, K, acc, rpc);
+    tgpk_last_gemm_kernel = !k.split ? "tgp_wstream_mma_kernel" : persistent ? "tgp_wstream_mma_group_kernel" : "tgp_wstream_mma_splitk_kernel";
+    if (persistent) {
+        if constexpr (NB == 1 && U == 8) {
+            if (per_cta == 2 && k.rows == 8) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 8, 2>, A, p, Mrows, total, K, acc, rpc);
+            else if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 2>, A, p, Mrows, total, K, acc, rpc);
             else if (k.rows == 8) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 8, 1>, A, p, Mrows, total, K, acc, rpc);
             else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc, rpc);
+        } else if constexpr (NB == 2 && U == 16) {
+            if (per_cta == 4) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 4>, A, p, Mrows, total, K, acc, rpc);
+            else if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 2>, A, p, Mrows, total, K, acc, rpc);
+            else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 1>, A, p, Mrows, total, K, acc, rpc);
         } else if constexpr (NB == 4 && U == 4) {
-            if (k.rows == 8) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 8, 1>, A, p, Mrows, total, K, acc, rpc);
-            else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc, rpc);
+            cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc, rpc);
         }
+    } else if constexpr (STREAMS) {
+        if (!k.split) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_kernel<NB, U>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
+        else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_splitk_kernel<NB, U, 8, 16>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
     }
-    else if (k.nw == 16 && k.rows == 8) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_splitk_kernel<NB, U, 16, 8>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
-    else if (k.nw == 16) {
-        if constexpr (NB == 1 && U == 4) {
-            // 33.5 MB blocks at M <= 8, two CTAs per SM: 14 rows per CTA when that gives every SM two
-            const uint32_t c14 = (p.n[0] + 13) / 14;
-            if (g_gemv_balance && need > sms && c14 <= 2 * sms && c14 > need) {
-                cfg.gridDim = dim3(c14);
-                cudaLaunchKernelEx(&cfg, tgp_wstream_mma_splitk_kernel<NB, U, 16, 16, 14>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
-                return;
-            }
-        }
-        cudaLaunchKernelEx(&cfg, tgp_wstream_mma_splitk_kernel<NB, U, 16, 16>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
-    }
-    else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_splitk_kernel<NB, U, 8, 16>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
 }
 
 static void launch_skinny_pick(const bf16 *A, const GemvParts &p, const SkinnyPick &k, uint32_t Mrows, uint32_t K, int acc, cudaStream_t st) {
     if (k.nb == 1) { if (k.u == 8) launch_skinny<1, 8>(A, p, k, Mrows, K, acc, st); else launch_skinny<1, 4>(A, p, k, Mrows, K, acc, st); }
-    else if (k.nb == 2) { if (k.u == 8) launch_skinny<2, 8>(A, p, k, Mrows, K, acc, st); else launch_skinny<2, 4>(A, p, k, Mrows, K, acc, st); }
+    else if (k.nb == 2) { if (k.u == 16) launch_skinny<2, 16>(A, p, k, Mrows, K, acc, st); else launch_skinny<2, 4>(A, p, k, Mrows, K, acc, st); }
     else { if (k.u == 4) launch_skinny<4, 4>(A, p, k, Mrows, K, acc, st); else launch_skinny<4, 2>(A, p, k, Mrows, K, acc, st); }
 }
 
@@ -1554,9 +1623,8 @@ uint32_t tgpk_gemm_group_key(uint32_t M, uint32_t n, uint32_t K) {
     if (!g_gemm_group || !M || !n || !K || K % 8) return 0;
     if (M >= 3 && M <= 32 && K % 32 == 0 && g_skinny_impl == 0) {
         const SkinnyPick k = pick_skinny(M, n, K);
-        // grouping pays where a block alone has fewer 16-row groups than the GPU has SMs (those take the 16-warp kernels)
-        const bool few = (n + 15) / 16 < (uint32_t)device_sms();
-        return (k.split && few && k.nw == 16) ? (0x1000000u | (uint32_t)k.nb | (uint32_t)k.u << 4 | (uint32_t)k.nw << 8 | (uint32_t)k.rows << 16) : 0;
+        // the blocks served by the persistent 16-warp kernel, which walks the row groups of any number of blocks
+        return k.persistent ? (0x1000000u | (uint32_t)k.nb | (uint32_t)k.u << 4 | (uint32_t)k.nw << 8 | (uint32_t)k.rows << 16) : 0;
     }
     if (M <= 2) return (n < 2 * 148 * 16 && !(g_gemv_splitk && K >= 8192)) ? M : 0;
     return 0;

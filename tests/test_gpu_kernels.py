@@ -602,7 +602,9 @@ def test_overlapping_gemv_launches_keep_their_dependencies():
     (8, (1152, 1152, 1152, 640), 14336, True),    # the pieces of an 8B down projection: 8-row CTAs, 16 warps
     (16, (512,) * 8, 28672, True),                # eight pieces of a 70B down projection
     (8, (1024, 1024), 4096, True),                # k and v of the 8B shape
-    (8, (4096, 1024), 4096, False),               # q and k pick different kernels: one launch each
+    (8, (4096, 1024, 1024), 4096, True),          # q, k and v of the 8B shape: all take the persistent 16-warp kernel
+    (8, (4096, 4096, 4096, 2048, 4096, 4096, 4096, 2048), 4096, True),   # gate and up of the 8B shape in 32 MiB pieces
+    (8, (8192, 1024), 2048, False),               # a piece of many rows takes the 8-warp kernel: one launch each
     (32, (500, 260, 33), 160, True),              # ragged row counts, four groups of activation rows
     (5, (24000, 64), 64, False),                  # a block that fills the machine alone
     (40, (256, 256), 512, False)])                # more activation rows than the skinny kernels take
@@ -671,4 +673,5 @@ def test_skinny_tensor_core_gemv_matches_oracle_and_cuda_core_path(M, n, K, accu
     scale = max(np.abs(prod).max(), 0.01)
     assert np.abs(outs[0] - want).max() < 2e-5 * scale + 1e-7
     assert np.abs(outs[0] - outs[1]).max() < 2e-5 * scale + 1e-7
-    assert np.array_equal(outs[0][:, :4], c0[:, :4]) and np.array_equal(outs[0][:, 4 + n:], c0[:, 4 + n:])
+    for out in outs:
+        assert np.array_equal(out[:, :4], c0[:, :4]) and np.array_equal(out[:, 4 + n:], c0[:, 4 + n:])
