@@ -1174,7 +1174,6 @@ static int g_gemm_impl = 0;      // 0: tensor cores for M > 16; 1: CUDA-core til
 static int g_gemv_splitk = 1;    // small-n blocks at M <= 2: CTA per RB rows with K split over its warps (0: one warp per row)
 static int g_gemm_group = 1;     // products over the same activations: one launch where the parts allow it (0: always one launch each)
 static int g_gemv_balance = 1;   // grouped skinny launches: rows per group chosen so that every persistent CTA gets the same number of groups
-static int g_gemv_rows8 = 1;     // skinny products of few rows and long K: 8-row CTAs (0: always 16)
 static int g_gemv_pdl = 1;       // consecutive weight-streaming launches may overlap (programmatic dependent launch)
 
 template <int MT, int R, int U>
@@ -1285,7 +1284,7 @@ __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_group_kernel(const bf
     uint4 lo[2][G][SK], hi[2][G][SK];                     // two register sets of SK load steps of every group
     // the activation fragments of a set are loaded with its weights (they come from L2 more often than from L1 -
     // a long K does not fit there - and would otherwise be waited for inside the MMA sequence)
-    constexpr bool XPRE = !(NB == 1 && ROWS == 8 && G == 1) && !(NB == 2 && G == 1);     // (those instances have no registers left for them)
+    constexpr bool XPRE = !(NB >= 2 && G == 1);           // (those instances have no registers left for them)
     uint4 xs[2][XPRE ? SK : 1][XPRE ? NB : 1];
     float acc[G][NB][4];
     // which block a group belongs to: looked up here for the weights and again after the K loop for the output, so
@@ -1459,15 +1458,14 @@ static SkinnyPick pick_skinny(uint32_t M, uint32_t n, uint32_t K) {
     // fewer than two 16-row groups per SM: one persistent CTA per SM walks the row groups of the block, or of a list of such
     // blocks (tgp_wstream_mma_group_kernel).  One choice per class of M for all of them, so that the pieces of a matrix share
     // a launch whatever the rows of its last piece:
-    //   M <= 8   16 warps, 8 load steps per warp and chunk; blocks of few rows and a long K as 8-row groups (twice the CTAs)
+    //   M <= 8   16 warps, 8 load steps per warp and chunk
     //   M <= 16  8 warps of twice the registers, 16 load steps: room for the activation fragments of a register set
-    //   M <= 32  16 warps, 4 load steps
+    //   M <= 32  the same with 8 load steps (four groups of activation rows take the registers)
     k.persistent = k.split && groups16 < 2u * sms;
     if (k.persistent) {
-        k.nw = k.nb == 2 ? 8 : 16;
-        k.u = k.nb == 1 ? 8 : k.nb == 2 ? 16 : 4;
-        const bool half = k.nb == 1 && g_gemv_rows8 && 2 * groups16 <= sms && K >= 16u * 32u * 2u * (uint32_t)k.u;
-        k.rows = half ? 8 : 16;
+        k.nw = k.nb == 1 ? 16 : 8;
+        k.u = k.nb == 1 ? 8 : k.nb == 2 ? 16 : 8;
+        k.rows = 16;
     } else {
         k.nw = 8;
         k.u = M <= 16 ? 4 : 2;
@@ -1500,7 +1498,7 @@ static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint3
         // block of few rows reaches every SM and no CTA waits for the others' last round (4096 rows: 256 groups of 16 leave
         // 40 SMs one round short, 293 of 14 do not) - but the rows a tile lacks are loaded all the same.  G and r are the
         // pair with the least estimated time of the busiest CTA: rounds x (G x (r + tile rows) / 2 + 4 NB), in rows read.
-        const uint32_t tile = (uint32_t)k.rows, gmax = NB == 1 ? 2 : NB == 2 ? 4 : 1;
+        const uint32_t tile = (uint32_t)k.rows, gmax = NB == 2 ? 4 : 2;       // (four groups of 32 activation rows would need more shared memory than a CTA may declare)
         uint32_t best = 0xffffffffu, best_r = tile;
         for (uint32_t G = gmax; G >= 1; G >>= 1)
             for (uint32_t r = g_gemv_balance ? tile / 2 + 1 : tile; r <= tile; ++r) {
@@ -1529,16 +1527,15 @@ static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint3
     tgpk_last_gemm_kernel = !k.split ? "tgp_wstream_mma_kernel" : persistent ? "tgp_wstream_mma_group_kernel" : "tgp_wstream_mma_splitk_kernel";
     if (persistent) {
         if constexpr (NB == 1 && U == 8) {
-            if (per_cta == 2 && k.rows == 8) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 8, 2>, A, p, Mrows, total, K, acc, rpc);
-            else if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 2>, A, p, Mrows, total, K, acc, rpc);
-            else if (k.rows == 8) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 8, 1>, A, p, Mrows, total, K, acc, rpc);
+            if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 2>, A, p, Mrows, total, K, acc, rpc);
             else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc, rpc);
         } else if constexpr (NB == 2 && U == 16) {
             if (per_cta == 4) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 4>, A, p, Mrows, total, K, acc, rpc);
             else if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 2>, A, p, Mrows, total, K, acc, rpc);
             else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 1>, A, p, Mrows, total, K, acc, rpc);
-        } else if constexpr (NB == 4 && U == 4) {
-            cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc, rpc);
+        } else if constexpr (NB == 4 && U == 8) {
+            if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 2>, A, p, Mrows, total, K, acc, rpc);
+            else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 1>, A, p, Mrows, total, K, acc, rpc);
         }
     } else if constexpr (STREAMS) {
         if (!k.split) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_kernel<NB, U>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
@@ -1549,7 +1546,7 @@ static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint3
 static void launch_skinny_pick(const bf16 *A, const GemvParts &p, const SkinnyPick &k, uint32_t Mrows, uint32_t K, int acc, cudaStream_t st) {
     if (k.nb == 1) { if (k.u == 8) launch_skinny<1, 8>(A, p, k, Mrows, K, acc, st); else launch_skinny<1, 4>(A, p, k, Mrows, K, acc, st); }
     else if (k.nb == 2) { if (k.u == 16) launch_skinny<2, 16>(A, p, k, Mrows, K, acc, st); else launch_skinny<2, 4>(A, p, k, Mrows, K, acc, st); }
-    else { if (k.u == 4) launch_skinny<4, 4>(A, p, k, Mrows, K, acc, st); else launch_skinny<4, 2>(A, p, k, Mrows, K, acc, st); }
+    else { if (k.u == 8) launch_skinny<4, 8>(A, p, k, Mrows, K, acc, st); else launch_skinny<4, 2>(A, p, k, Mrows, K, acc, st); }
 }
 
 template <int MT, int RB, int U>
