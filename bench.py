@@ -111,10 +111,12 @@ def time_oracle(lay, om, sample_S, sample_T):
     return cfg.B * (sample_S + sample_T) / dt, dt
 
 
-def gemm_shapes_of_step(lay, M):
+def gemm_shapes_of_step(lay, M, pinned=None):
     """(n, K, residual, M) of every weight-block launch of one step, in trace order (lm_head at M = B).  Consecutive dense
     blocks that read the same activations and carry the same non-zero tgp_k_gemm_group_key() share a launch, as in
-    tgp_step() once their copies are enqueued; n is then the tuple of their row counts."""
+    tgp_step(); n is then the tuple of their row counts.  pinned: ids of the tensors the plan keeps resident - a block
+    that is staged through the ring ends its launch, as in tgp_step() (a later copy waits for its slot); None: every
+    block resident."""
     from paper_2609_06172_b200 import binding as tb
     cfg = lay.cfg
     out = []
@@ -138,6 +140,8 @@ def gemm_shapes_of_step(lay, M):
             if not run:
                 run_key[0] = key
             run.append(t)
+            if pinned is not None and t.tid not in pinned:
+                flush()
         flush()
 
     run_key = [0]
@@ -159,7 +163,7 @@ def gemm_shapes_of_step(lay, M):
 GROUP_MAX = 8     # TGP_GEMM_GROUP_MAX
 
 
-def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30, min_seconds=1.5):
+def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30, min_seconds=1.5, pinned=None):
     """Times the weight-block products of one step back to back on one stream, every launch reading a different
     (cold) region of a buffer larger than L2, exactly as tgp_step launches them (same entry point, shapes, M).
     The whole-step loop is replayed for at least min_seconds (and at least `reps` replays when min_seconds is 0: the small
@@ -168,7 +172,7 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30, min_seconds=1.5):
     import torch
     from paper_2609_06172_b200 import binding as tb
     cfg = lay.cfg
-    shapes = gemm_shapes_of_step(lay, M)
+    shapes = gemm_shapes_of_step(lay, M, pinned)
     # random operands with the weights' distribution: constant data would toggle few wires, draw little power and let
     # a seconds-long tensor-core loop run at clocks the real step (random weights, power-capped) never sees
     gen = torch.Generator(device=device)
@@ -479,6 +483,9 @@ def main():
     ap.add_argument("--no-uvm", action="store_true", help="skip the demand-paged managed-memory baseline")
     ap.add_argument("--kernel-loop", choices=["decode", "prefill", "attention"], default=None,
                     help="only run the back-to-back weight-product loop of one step (small, for ncu captures)")
+    ap.add_argument("--planned-mix", action="store_true",
+                    help="with --kernel-loop decode/prefill: the launch list of the planned run at the configuration's budget (blocks staged "
+                         "through the ring end their launch) instead of every block resident")
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--alias-layers", type=int, default=None, help="host pool with this many physical layers: layers l and l + N share host pages (for pools larger than the host can page-lock)")
     ap.add_argument("--unseen-prompts", action="store_true", help="MoE: time prompts of another seed than the profile pass saw")
@@ -525,9 +532,18 @@ def main():
                               "TK": cfg.TK, "causal_flops": flops, "L2_flushed_between_launches": True, "kernels": table}))
             return
         M = cfg.B * (cfg.S if args.kernel_loop == "prefill" else 1)
-        sec, b, f, nl, table = kernel_loop(lay, M, args.reps, torch.device("cuda:0"), min_seconds=0.0)
+        pinned = None
+        if args.planned_mix and not cfg.E:
+            # the launch list of the planned, oversubscribed run: planned on the host (no pool needed), pins read from the plan
+            from paper_2609_06172_b200.session import Session
+            ps = Session(lay, MACHINE)
+            pb = ps.plan(bits=args.bits)["pins"]
+            pinned = {struct.unpack_from("<IQ", pb, 12 * k)[0] for k in range((len(pb) - 16) // 12)}
+            ps.close()
+        sec, b, f, nl, table = kernel_loop(lay, M, args.reps, torch.device("cuda:0"), min_seconds=0.0, pinned=pinned)
         print(json.dumps({"kernel_loop": args.kernel_loop, "M": M, "avg_us": sec * 1e6, "GBps": b / sec / 1e9, "TFLOPs": f / sec / 1e12,
-                          "launches_per_step": nl, "timed": kernel_loop.last, "shapes": table}))
+                          "launches_per_step": nl, "launch_list": "planned run" if pinned is not None else "every block resident",
+                          "timed": kernel_loop.last, "shapes": table}))
         return
 
     t_start = time.monotonic()
@@ -715,7 +731,14 @@ def main():
     dom = max(kind_ms, key=lambda k: kind_ms[k])
     if dom[1] == "gemm":
         Mk = cfg.B * (cfg.S if dom[0] == "prefill" else 1)
-        sec, bpl, fpl, nl, table = kernel_loop(lay, Mk, args.reps, dev)
+        pb = s.ctx.plan_blobs()["pins"]
+        pinned = {struct.unpack_from("<IQ", pb, 12 * k)[0] for k in range((len(pb) - 16) // 12)}
+        sec, bpl, fpl, nl, table = kernel_loop(lay, Mk, args.reps, dev, pinned=pinned)
+        timed_mix = dict(kernel_loop.last)
+        # the same products with every block resident (what tgp_step launches when the budget holds the pool: all pieces of
+        # a matrix in one launch), for comparison with the mix of the oversubscribed run
+        sec_res, bpl_res, _, nl_res, _ = kernel_loop(lay, Mk, args.reps, dev, min_seconds=0.5, pinned=None)
+        kernel_loop.last = timed_mix
         if dom[0] == "prefill" and fpl / MACHINE["peak_flops"] > bpl / MACHINE["hbm_Bps"]:
             ach = fpl / sec / 1e12
             # the loop below replays the step's launches for seconds under the power cap: the matching denominator is the
@@ -727,7 +750,10 @@ def main():
                     "frac_of_burst_peak": ach / peaks["bf16_tflops"]}
         else:
             ach = bpl / sec / 1e9
-            roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"]}
+            roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                    "all_blocks_resident": {"launches_per_step": nl_res, "avg_us": sec_res * 1e6, "achieved": bpl_res / sec_res / 1e9,
+                                            "frac": bpl_res / sec_res / 1e9 / peaks["hbm_gbs"],
+                                            "note": "the same products as tgp_step launches them when no block is staged through the ring (budget >= pool)"}}
         # the kernels that ran, as the library reports them per launch (its choice depends on M, n, K), heaviest first
         by_kernel = {}
         for v in table.values():
@@ -736,7 +762,7 @@ def main():
         roof.update({"kernel": f"weight-block product ({dom[0]}, M={Mk}): " + " + ".join(names),
                      "kernel_time_share": {k: round(by_kernel[k] / sum(by_kernel.values()), 3) for k in names},
                      "launches": nl * (T if dom[0] == "decode" else 1), "avg_us": sec * 1e6, "algorithmic_per_launch": fpl if roof["bound"] == "tensor" else bpl,
-                     "timing": f"CUDA-graph replay of the {nl} launches of one step, {kernel_loop.last['reps']} x {kernel_loop.last['passes']} passes back to back ({kernel_loop.last['seconds']:.2f} s), random operands, cold inputs cycling through 1 GiB, CUDA events on the launch stream",
+                     "timing": f"CUDA-graph replay of the {nl} weight-block launches of one step of the timed run (blocks the plan pins share launches, a block staged through the ring ends its launch), {kernel_loop.last['reps']} x {kernel_loop.last['passes']} passes back to back ({kernel_loop.last['seconds']:.2f} s), random operands, cold inputs cycling through 1 GiB, CUDA events on the launch stream",
                      "in_step_avg_us": kind_ms[dom] / (nl * (T if dom[0] == "decode" else 1)) * 1e3, "shapes": table})
     else:
         ach = kind_bytes[dom] / (kind_ms[dom] * 1e-3) / 1e9

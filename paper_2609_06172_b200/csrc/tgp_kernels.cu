@@ -1496,7 +1496,8 @@ static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint3
         // each activation fragment (every CTA reads its K slices of all activation rows per round, so at one group per round
         // that traffic equals the weights').  Rows per group r <= the tile's rows: fewer rows make more groups, so that a
         // block of few rows reaches every SM and no CTA waits for the others' last round (4096 rows: 256 groups of 16 leave
-        // 40 SMs one round short, 293 of 14 do not) - but the rows a tile lacks are loaded all the same.  G and r are the
+        // 40 SMs one round short, 293 of 14 do not) - but the rows a tile lacks still occupy its load slots (their lanes
+        // re-read the group's last row; fewer than 9 rows per group measured no faster for blocks of few rows).  G and r are the
         // pair with the least estimated time of the busiest CTA: rounds x (G x (r + tile rows) / 2 + 4 NB), in rows read.
         const uint32_t tile = (uint32_t)k.rows, gmax = NB == 2 ? 4 : 2;       // (four groups of 32 activation rows would need more shared memory than a CTA may declare)
         uint32_t best = 0xffffffffu, best_r = tile;
