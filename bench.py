@@ -122,8 +122,10 @@ def gemm_shapes_of_step(lay, M, pinned=None):
     out = []
 
     def emit(blocks, res, m):
-        """blocks: weight blocks in op order, all multiplied with the same activations."""
+        """blocks: weight blocks in op order, all multiplied with the same activations (new ones: another kernel wrote them
+        just before the first of these launches)."""
         run = []
+        first = len(out)
         def flush():
             if len(run) == 1:
                 out.append((run[0].rows, run[0].cols, res, m))
@@ -143,8 +145,12 @@ def gemm_shapes_of_step(lay, M, pinned=None):
             if pinned is not None and t.tid not in pinned:
                 flush()
         flush()
+        if len(out) > first:
+            new_acts.add(first)
 
     run_key = [0]
+    new_acts = set()          # indices of the launches that are the first over their activations
+    gemm_shapes_of_step.new_acts = new_acts
     for l in range(cfg.L):
         emit([t for kind in (si.K_WQ, si.K_WK, si.K_WV) for t in lay.blocks(kind, l)], 0, M)
         emit(lay.blocks(si.K_WO, l), 1, M)
@@ -186,7 +192,11 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30, min_seconds=1.5, pinne
     kmax = max(k for (_, k, _, _) in shapes)
     nmax = max(rows_of(n) for (n, _, _, _) in shapes)
     mmax = max(m for (_, _, _, m) in shapes)
-    A = torch.randn((mmax, kmax), device=device, generator=gen).bfloat16()
+    # two activation buffers: a launch that is the first over its activations (another kernel has just written them in a real
+    # step) takes the other one, so that only the launches that follow it may request their activations early (tgp_k_gemm_chain)
+    A2 = [torch.randn((mmax, kmax), device=device, generator=gen).bfloat16() for _ in range(2)]
+    new_acts = gemm_shapes_of_step.new_acts
+    tb.k_gemm_chain(True)
     Cbuf = torch.zeros((mmax, nmax), dtype=torch.float32, device=device)
     stream = torch.cuda.Stream(device=device)
     off = 0
@@ -195,7 +205,11 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30, min_seconds=1.5, pinne
 
     def run_all(st, only=None):
         nonlocal off
-        for (n, K, res, m) in shapes:
+        which = 0
+        for idx, (n, K, res, m) in enumerate(shapes):
+            if idx in new_acts:
+                which ^= 1
+            A = A2[which]
             if only is not None and (n, K, res, m) != only:
                 continue
             nb = (rows_of(n) * K * 2 + 511) // 512 * 512
@@ -258,6 +272,7 @@ def kernel_loop(lay, M, reps, device, cold_bytes=1 << 30, min_seconds=1.5, pinne
         name = "+".join(str(x) for x in n) if isinstance(n, tuple) else str(n)
         table[f"n={name} K={K} M={m} res={res}"] = {"kernel": kernel_of.get(sh, "?"), "launches_per_step": cnt, "us": round(t * 1e6, 2),
                                                       "GBps": round(b / t / 1e9, 1), "TFLOPs": round(2 * m * K * nr / t / 1e12, 2)}
+    tb.k_gemm_chain(False)
     return sec, bytes_per, flops_per, len(shapes), table
 
 

@@ -337,6 +337,13 @@ int  tgp_k_skinny_select(int impl);
  * latency overlaps.  0 switches that off (each launch then starts after the previous one has completed).  Results are
  * identical either way.  Process-wide; default on. */
 int  tgp_k_gemv_overlap(int enable);
+/* A promise by a caller of the kernel entry points, for the calling thread: between consecutive tgp_k_gemm() /
+ * tgp_k_gemm_group() calls on one stream nothing but this library's kernels (launched by this thread) is enqueued on that
+ * stream.  A product of 3 - 32 activation rows that directly follows another one over the same activation pointer then
+ * requests its activations together with its weights, before the previous launch has finished (they are older than that
+ * launch); results are identical.  tgp_step() works this way by itself.  Default off: a caller that rewrites the
+ * activations between two calls by other means must leave it off. */
+int  tgp_k_gemm_chain(int enable);
 /* Tensor-core GEMM variant: 0 (default) picks by problem size, 1 forces the 128x128 one-tile-per-CTA kernel,
  * 2 the persistent 128x256 kernel with double-buffered accumulators, 3 the paired kernel (256x256 tiles on the two SMs
  * of a CTA pair, each loading half of the weight tile), 4 the one-tile-per-CTA kernel with the operands swapped (the

@@ -115,6 +115,7 @@ _SIGS = {
     "tgp_k_attn_select": [C.c_int],
     "tgp_k_attn_decode_select": [C.c_int],
     "tgp_k_gemv_overlap": [C.c_int],
+    "tgp_k_gemm_chain": [C.c_int],
     "tgp_k_skinny_select": [C.c_int],
     "tgp_k_gemm_tc_variant": [C.c_int],
     "tgp_k_gemm_status": [C.POINTER(C.c_int)],
@@ -462,6 +463,10 @@ def k_skinny_select(impl):
 
 def k_gemv_overlap(enable):
     _k(lib().tgp_k_gemv_overlap(int(enable)), "tgp_k_gemv_overlap")
+
+
+def k_gemm_chain(enable):
+    _k(lib().tgp_k_gemm_chain(int(enable)), "tgp_k_gemm_chain")
 
 
 def k_attn_select(impl):

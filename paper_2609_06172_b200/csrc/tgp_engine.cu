@@ -582,6 +582,9 @@ extern "C" int tgp_step(tgp_ctx *ctx, uint32_t step_kind, const int32_t *tokens_
     cudaStream_t cs = (cudaStream_t)compute_stream, cp = (cudaStream_t)copy_stream;
     const uint32_t M = B * q_len, pos0 = e->pos;
     const uint64_t launches0 = tgpk_launches;
+    // every kernel of the step is launched from here on the compute stream: consecutive products over the same activations
+    // may read them before their predecessor has finished
+    struct ChainScope { bool was; ChainScope() : was(tgpk_chain_ok) { tgpk_chain_ok = true; } ~ChainScope() { tgpk_chain_ok = was; } } chain_scope;
     uint32_t n_cmds = 0, n_mismatch = 0;
     e->cur_expert = -1;
     if (stats) CU(ctx, cudaEventRecord(e->t0, cs));

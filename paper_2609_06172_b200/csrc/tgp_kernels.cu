@@ -9,6 +9,10 @@
 #include "tgp_kernels.h"
 
 thread_local uint64_t tgpk_launches = 0;     // kernels launched by this thread (reported in the step statistics)
+// true while the caller vouches that this thread's launches are all that is enqueued on their streams (tgp_step does; direct
+// callers say so through tgp_k_gemm_chain): consecutive weight products over the same activations may then read them early
+thread_local bool tgpk_chain_ok = false;
+namespace { struct ProductChain { const void *A; cudaStream_t st; uint64_t launches_before; }; thread_local ProductChain g_chain = {nullptr, nullptr, 0}; }
 thread_local const char *tgpk_last_gemm_kernel = "";   // name of the kernel the last weight-block product of this thread launched
 #define LAUNCH_CHECK(n) do { cudaError_t e_ = cudaGetLastError(); if (e_ != cudaSuccess) return TGP_E_CUDA; tgpk_launches += (n); } while (0)
 
@@ -1271,13 +1275,12 @@ __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_splitk_kernel(const b
 // same bits as one launch per block.
 template <int NB, int U, int NW, int ROWS, int RG>
 __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_group_kernel(const bf16 *A, const GemvParts p, uint32_t Mrows, uint32_t groups_total,
-                                                              uint32_t K, int accumulate, uint32_t rpc) {
+                                                              uint32_t K, int accumulate, uint32_t rpc, int acts_early) {
     constexpr int UL = ROWS == 8 ? 2 * U : U;             // half a tile per load step: twice the steps in flight
     constexpr int G = RG, SK = UL / (2 * G);              // a register set holds SK load steps of G groups: two sets are as many loads as UL steps of one group
     static_assert(UL % (2 * G) == 0 && SK >= 1, "row groups per CTA must divide half the load steps");
     __shared__ float part[NW][G * NB * 4][32];
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, c = lane & 3;
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     uint32_t grp0 = blockIdx.x * G;
     if (grp0 >= groups_total) return;
     const bf16 *wlo[G], *whi[G];
@@ -1384,9 +1387,14 @@ __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_group_kernel(const bf
     issue(set0, kb_cur);
     issue(set1, kb_cur + 32 * SK);
     bool cur_last = advance();
-    asm volatile("griddepcontrol.wait;" ::: "memory");      // weights are never written by a kernel: the activations are read from here on
-    issue_act(set0, kb_cur);
-    issue_act(set1, kb_cur + 32 * SK);
+    // Weights are never written by a kernel, so they are requested before the previous launch of the stream has finished.
+    // The activations are read after it has - unless the launcher knows that they are older than that launch (it read the
+    // same activations): then they are requested with the weights.  The next launch is released only here, after the wait:
+    // when it starts, everything before this launch is complete, which is what lets it read its activations early in turn.
+    if (acts_early) { issue_act(set0, kb_cur); issue_act(set1, kb_cur + 32 * SK); }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (!acts_early) { issue_act(set0, kb_cur); issue_act(set1, kb_cur + 32 * SK); }
     clear();
     for (;;) {
         const bool have_next = grp < groups_total;
@@ -1525,18 +1533,23 @@ static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint3
     cfg.numAttrs = 1;
     uint32_t total = 0;
     for (uint32_t s = 0; k.split && s < p.count; ++s) total += p.groups[s];
+    // the previous launch of this thread was a product of this family over the same activations on the same stream, and the
+    // caller vouches that nothing else was enqueued there in between: the activations are older than that launch
+    const int early = persistent && tgpk_chain_ok && g_gemv_pdl && g_chain.A == (const void *)A && g_chain.st == st && g_chain.launches_before + 1 == tgpk_launches;
+    if (persistent) { g_chain.A = A; g_chain.st = st; g_chain.launches_before = tgpk_launches; }
+    else g_chain.A = nullptr;
     tgpk_last_gemm_kernel = !k.split ? "tgp_wstream_mma_kernel" : persistent ? "tgp_wstream_mma_group_kernel" : "tgp_wstream_mma_splitk_kernel";
     if (persistent) {
         if constexpr (NB == 1 && U == 8) {
-            if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 2>, A, p, Mrows, total, K, acc, rpc);
-            else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc, rpc);
+            if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 2>, A, p, Mrows, total, K, acc, rpc, early);
+            else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 16, 16, 1>, A, p, Mrows, total, K, acc, rpc, early);
         } else if constexpr (NB == 2 && U == 16) {
-            if (per_cta == 4) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 4>, A, p, Mrows, total, K, acc, rpc);
-            else if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 2>, A, p, Mrows, total, K, acc, rpc);
-            else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 1>, A, p, Mrows, total, K, acc, rpc);
+            if (per_cta == 4) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 4>, A, p, Mrows, total, K, acc, rpc, early);
+            else if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 2>, A, p, Mrows, total, K, acc, rpc, early);
+            else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 1>, A, p, Mrows, total, K, acc, rpc, early);
         } else if constexpr (NB == 4 && U == 8) {
-            if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 2>, A, p, Mrows, total, K, acc, rpc);
-            else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 1>, A, p, Mrows, total, K, acc, rpc);
+            if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 2>, A, p, Mrows, total, K, acc, rpc, early);
+            else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 1>, A, p, Mrows, total, K, acc, rpc, early);
         }
     } else if constexpr (STREAMS) {
         if (!k.split) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_kernel<NB, U>, A, p.W[0], p.C[0], Mrows, p.n[0], K, p.ldc[0], 0u, acc);
@@ -1902,6 +1915,12 @@ int tgp_k_gemm_last_kernel(char *name, uint32_t capacity) {
 
 int tgp_k_gemm_group_select(int enable) {
     g_gemm_group = enable ? 1 : 0;
+    return TGP_OK;
+}
+
+int tgp_k_gemm_chain(int enable) {
+    tgpk_chain_ok = enable != 0;
+    g_chain.A = nullptr;
     return TGP_OK;
 }
 

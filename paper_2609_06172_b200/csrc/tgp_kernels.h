@@ -47,6 +47,8 @@ int tgpk_gemm_status_clear();
 int tgpk_attn_status_clear();
 // name of the kernel the last tgpk_gemm / tgpk_gemm_group / tgpk_gemm_tc call of this thread launched
 extern thread_local const char *tgpk_last_gemm_kernel;
+// set while the caller vouches that this thread's kernel launches are all that is enqueued on their streams (see tgp_k_gemm_chain)
+extern thread_local bool tgpk_chain_ok;
 // test hooks of the tensor-core kernels' bounded waits (see tgp_k_wait_test)
 int tgpk_gemm_wait_test(unsigned long long limit_ns, int withhold_step);
 int tgpk_attn_wait_test(unsigned long long limit_ns, int withhold_step);

@@ -594,6 +594,37 @@ def test_overlapping_gemv_launches_keep_their_dependencies():
     assert np.abs(outs[0] - want).max() < 1e-4 * np.abs(want).max()
 
 
+def test_chained_products_read_their_activations_early_with_the_same_bits():
+    """Under the caller's promise (tgp_k_gemm_chain) a product that directly follows another one over the same activations
+    requests them before its predecessor has finished.  The chain must give the bits of unchained launches; a product
+    that follows a kernel which rewrote the activations (an RMSNorm of this library) is not chained and sees the new values."""
+    M, n, K = 8, 1152, 4096
+    rng = np.random.default_rng(77)
+    x0 = torch.from_numpy(rng.standard_normal((M, K)).astype(np.float32)).to(DEV)
+    gain = bf16_dev(rnd_bits(78, K))
+    A = torch.empty(M, K, dtype=torch.bfloat16, device=DEV)
+    Ws = [bf16_dev(rnd_bits(80 + i, n * K).reshape(n, K)) for i in range(4)]
+    outs = []
+    for chain in (0, 1):
+        tb.k_gemm_chain(chain)
+        x = x0.clone()
+        res = []
+        for rep in range(3):
+            tb.k_rmsnorm(x, K, gain, A, M, K, 1e-5)               # rewrites A: the product after it waits for it
+            x.mul_(1.25)                                          # (another stream op between the repetitions; before the norm, not between products)
+            Cs = [torch.zeros(M, n, dtype=torch.float32, device=DEV) for _ in Ws]
+            for W, C in zip(Ws, Cs):
+                tb.k_gemm(A, W, C, M, n, K, n, 0, 0)
+            torch.cuda.synchronize()
+            res.append([c.cpu().numpy() for c in Cs])
+        outs.append(res)
+    tb.k_gemm_chain(0)
+    for rep in range(3):
+        for a, b in zip(outs[0][rep], outs[1][rep]):
+            assert np.array_equal(a, b)
+    assert not np.array_equal(outs[0][0][0], outs[0][1][0])          # the activations did change between repetitions
+
+
 @pytest.mark.parametrize("M,ns,K,grouped", [
     (1, (2048, 512, 512), 2048, True),            # the q, k, v projections of the 1B shape: one launch
     (2, (300, 7, 129, 1), 264, True),             # four ragged parts, K not a multiple of the chunk
