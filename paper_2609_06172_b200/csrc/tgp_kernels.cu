@@ -1204,11 +1204,11 @@ static void launch_gemv(const bf16 *A, const bf16 *W, float *C, uint32_t Mrows, 
     tgpk_last_gemm_kernel = "tgp_wstream_kernel";
 }
 
-// Same product for blocks with few rows: one CTA owns ROWS (16, or 8 with the upper half of the MMA tile left empty)
-// rows of W and its NW (8 or 16) warps split K (interleaved chunks of 32*U), so n/ROWS CTAs of NW warps fill the machine
-// where n/16 warps would not.  The partial tiles meet in shared memory and are summed in warp order: deterministic.
-// RPC <= ROWS: rows a CTA owns (the tile's remaining rows re-read its last row and are not stored; a row's sum does not
-// depend on its place in the tile).  14 of 16 turns the 256 CTAs of a 4096-row block into 293, two for every SM.
+// Same product for blocks with two to eight 16-row groups per SM: one CTA owns ROWS rows of W and its NW warps split K
+// (interleaved chunks of 32*U), so n/ROWS CTAs of NW warps fill the machine where n/16 warps would not.  The partial
+// tiles meet in shared memory and are summed in warp order: deterministic.  RPC <= ROWS: rows a CTA owns (the tile's
+// remaining rows re-read its last row and are not stored; a row's sum does not depend on its place in the tile).
+// (Blocks of fewer rows take tgp_wstream_mma_group_kernel.)
 template <int NB, int U, int NW, int ROWS, int RPC = ROWS>
 __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_splitk_kernel(const bf16 *A, const bf16 *__restrict__ W, float *__restrict__ C,
                                                               uint32_t Mrows, uint32_t n, uint32_t K, uint32_t ldc, uint32_t col0, int accumulate) {
@@ -1267,12 +1267,13 @@ __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_splitk_kernel(const b
     }
 }
 
-// The same kernel over several weight blocks that read the same activations (the pieces of one matrix; the q, k and v
-// projections): their row groups are walked as one list and a CTA takes RG consecutive groups, whose MMAs share each
-// activation fragment - every CTA reads its K slices of all activation rows from L2, so at 8 or 16 rows per CTA that
-// traffic equals or exceeds the weights' and bounds the kernel; RG row groups divide it by RG.  A group's arithmetic
-// (which warp adds which k, in which order) is that of tgp_wstream_mma_splitk_kernel<NB, U, NW, ROWS> whatever RG and the list:
-// same bits as one launch per block.
+// The product for blocks of fewer than two 16-row groups per SM, one block or a list of blocks that read the same
+// activations (the pieces of one matrix; the q, k and v projections): one persistent CTA per SM walks the row groups
+// as one list, RG consecutive groups at a time, whose MMAs share each activation fragment - every CTA reads its K
+// slices of all activation rows from L2, so at 16 rows per CTA that traffic equals the weights'; RG row groups divide
+// it by RG.  K is split over the CTA's NW warps in interleaved chunks of 32*U columns and the partial tiles are summed
+// in warp order.  A group's arithmetic (which warp adds which k, in which order) depends on NB, U, NW and K alone -
+// not on RG, the rows per group or the list: a block gives the same bits alone or in any list.
 template <int NB, int U, int NW, int ROWS, int RG>
 __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_group_kernel(const bf16 *A, const GemvParts p, uint32_t Mrows, uint32_t groups_total,
                                                               uint32_t K, int accumulate, uint32_t rpc, int acts_early) {
