@@ -1280,7 +1280,11 @@ __global__ void __launch_bounds__(NW * 32) tgp_wstream_mma_group_kernel(const bf
     constexpr int UL = ROWS == 8 ? 2 * U : U;             // half a tile per load step: twice the steps in flight
     constexpr int G = RG, SK = UL / (2 * G);              // a register set holds SK load steps of G groups: two sets are as many loads as UL steps of one group
     static_assert(UL % (2 * G) == 0 && SK >= 1, "row groups per CTA must divide half the load steps");
-    __shared__ float part[NW][G * NB * 4][32];
+    // the warps' partial tiles: static where they fit the 48 KB a kernel may declare, else the launch's dynamic shared memory
+    constexpr bool PART_DYNAMIC = (size_t)NW * G * NB * 4 * 32 * 4 > 48 * 1024;
+    __shared__ float part_static[PART_DYNAMIC ? 1 : NW * G * NB * 4 * 32];
+    extern __shared__ float part_dynamic[];
+    float (*part)[G * NB * 4][32] = reinterpret_cast<float (*)[G * NB * 4][32]>(PART_DYNAMIC ? part_dynamic : part_static);
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, c = lane & 3;
     uint32_t grp0 = blockIdx.x * G;
     if (grp0 >= groups_total) return;
@@ -1508,7 +1512,7 @@ static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint3
         // 40 SMs one round short, 293 of 14 do not) - but the rows a tile lacks still occupy its load slots (their lanes
         // re-read the group's last row; fewer than 9 rows per group measured no faster for blocks of few rows).  G and r are the
         // pair with the least estimated time of the busiest CTA: rounds x (G x (r + tile rows) / 2 + 4 NB), in rows read.
-        const uint32_t tile = (uint32_t)k.rows, gmax = NB == 2 ? 4 : 2;       // (four groups of 32 activation rows would need more shared memory than a CTA may declare)
+        const uint32_t tile = (uint32_t)k.rows, gmax = NB == 1 ? 2 : 4;
         uint32_t best = 0xffffffffu, best_r = tile;
         for (uint32_t G = gmax; G >= 1; G >>= 1)
             for (uint32_t r = g_gemv_balance ? tile / 2 + 1 : tile; r <= tile; ++r) {
@@ -1549,7 +1553,14 @@ static void launch_skinny(const bf16 *A, GemvParts p, const SkinnyPick &k, uint3
             else if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 2>, A, p, Mrows, total, K, acc, rpc, early);
             else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 1>, A, p, Mrows, total, K, acc, rpc, early);
         } else if constexpr (NB == 4 && U == 8) {
-            if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 2>, A, p, Mrows, total, K, acc, rpc, early);
+            if (per_cta == 4) {
+                // four groups of 32 activation rows: the warps' partial tiles take 64 KB of dynamic shared memory
+                constexpr size_t smem = (size_t)8 * 4 * NB * 4 * 32 * 4;
+                static bool attr_set = false;
+                if (!attr_set) { cudaFuncSetAttribute(tgp_wstream_mma_group_kernel<NB, U, 8, 16, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); attr_set = true; }
+                cfg.dynamicSmemBytes = smem;
+                cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 4>, A, p, Mrows, total, K, acc, rpc, early);
+            } else if (per_cta == 2) cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 2>, A, p, Mrows, total, K, acc, rpc, early);
             else cudaLaunchKernelEx(&cfg, tgp_wstream_mma_group_kernel<NB, U, 8, 16, 1>, A, p, Mrows, total, K, acc, rpc, early);
         }
     } else if constexpr (STREAMS) {
