@@ -679,17 +679,22 @@ def main():
     e2e_value = world * tokens_per_pass * args.steps / (ms_e2e * 1e-3) if ms_e2e else None
 
     # ---- per-phase timing, launches and the live per-kernel roofline: one extra pass with op timestamps -----------
+    # (step times from a pass without op timestamps: the event brackets around every op keep consecutive launches from
+    # overlapping, which a step of a few milliseconds would feel)
     r.reset()
-    s.ctx.set_op_timing(True)
-    kind_ms, kind_bytes, kind_flops, kind_n = {}, {}, {}, {}
     launches = mismatches = 0
     step_ms = []
     for k in range(1 + T):
         st = r.step(tb.PREFILL if k == 0 else tb.DECODE, prompt_pinned.numpy() if k == 0 else None, cfg.S if k == 0 else 1, want_stats=True)
-        first, tms = s.ctx.op_times()
         launches += st.n_launches
         mismatches += st.n_mismatch
         step_ms.append(st.step_ms)
+    r.reset()
+    s.ctx.set_op_timing(True)
+    kind_ms, kind_bytes, kind_flops, kind_n = {}, {}, {}, {}
+    for k in range(1 + T):
+        st = r.step(tb.PREFILL if k == 0 else tb.DECODE, prompt_pinned.numpy() if k == 0 else None, cfg.S if k == 0 else 1, want_stats=True)
+        first, tms = s.ctx.op_times()
         phase = "prefill" if k == 0 else "decode"
         for j, t in enumerate(tms):
             o = ops[first + j]
