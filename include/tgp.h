@@ -186,6 +186,12 @@ int  tgp_set_measured_times(tgp_ctx *ctx, const uint64_t *op_ns, uint64_t n_ops)
 int  tgp_replan_begin(tgp_ctx *ctx, uint32_t first_step, const uint64_t *op_ns, uint64_t n_ops);
 int  tgp_replan_wait(tgp_ctx *ctx);
 int  tgp_replan_commit(tgp_ctx *ctx);
+/* keep != 0: tail plans made from now on keep the pinned tensors of the plan in use that are on the device at the
+ * boundary.  A tensor the tail plan pins again stays where it is - with the newest data, so the commit writes back only
+ * the written pins that are given up - and is not loaded again; newly pinned tensors go into the first gap between the
+ * kept ones that holds them; the windowed reservation (TGP_BIT_W) is not applied to such a plan.  The switch then costs
+ * the link only what the new plan pins anew.  Default 0 (the tail plan starts from an empty arena). */
+int  tgp_set_replan_keep(tgp_ctx *ctx, int keep);
 /* Classifies ops, selects critical / zero-copy / pinned tensors, sizes the ring and builds the ordered
  * command list.  Host only; no CUDA call. */
 int  tgp_plan(tgp_ctx *ctx);

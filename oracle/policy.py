@@ -141,7 +141,7 @@ class Plan:
 
 
 def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A | BIT_P | BIT_ZC | BIT_W, measured_ns=None,
-         written_before=()) -> Plan:
+         written_before=(), resident=None) -> Plan:
     """tensors: list of objects with .size .pool_off .flags; ops: list with .step .flops .hbm .acc;
     steps: [(kind, first op, count)]; measured_ns: optional per-op kernel times in integer nanoseconds (0 = none);
     written_before: tensors that already hold data in the pool when the trace starts (a tail re-plan), whose first
@@ -243,12 +243,41 @@ def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A |
                 if t not in pinned_off and used + a <= pin_cap:
                     pinned_off[t] = used
                     used += a
+    # 5a: pins that are resident already (a plan made in the middle of a run, see plan_tail): a chosen tensor that is on the
+    # device keeps its place and is not loaded again; the others go, in the order they were chosen, into the first gap
+    # between the kept ones that holds them (none: not pinned after all).  The pin region ends where the longer of the
+    # two layouts ends.
+    kept: Dict[int, int] = {}
+    if resident is not None:
+        kept = {t: resident[t] for t in pinned_off if t in resident}
+        chosen = sorted(pinned_off, key=pinned_off.get)
+        region_end = max([used] + [o + alignup(tensors[t].size) for t, o in kept.items()])
+        holes, pos = [], 0
+        for (a0, a1) in sorted((o, o + alignup(tensors[t].size)) for t, o in kept.items()):
+            if a0 > pos:
+                holes.append([pos, a0])
+            pos = max(pos, a1)
+        if pos < region_end:
+            holes.append([pos, region_end])
+        placed = dict(kept)
+        for t in chosen:
+            if t in kept:
+                continue
+            a = alignup(tensors[t].size)
+            for h in holes:
+                if h[1] - h[0] >= a:
+                    placed[t] = h[0]
+                    h[0] += a
+                    break
+        pinned_off, used = placed, region_end
+        if budget - used < ring_min:
+            raise PlanError("kept pins leave less than the ring minimum")
     ring_base, ring_size = used, budget - used
     pins = sorted(pinned_off.items())
-    # 5b: windowed reservation - tenants of the slots of pinned tensors that are born late
+    # 5b: windowed reservation - tenants of the slots of pinned tensors that are born late (not in a plan that keeps pins)
     tenancy: Dict[int, Tuple[int, int]] = {}       # tenant -> (arena offset, last op it is used there)
     landlord_wait: Dict[int, int] = {}             # late-born pinned tensor -> op its placement must wait for
-    if (bits & BIT_W) and pinned_off:
+    if (bits & BIT_W) and pinned_off and resident is None:
         first_acc: Dict[int, Tuple[int, int]] = {}
         for i, op in enumerate(ops):
             for (t, mode, _) in op.acc:
@@ -288,7 +317,7 @@ def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A |
     totals = [[0, 0, 0, 0] for _ in steps]
     ep_index = {t: 0 for t in episodes_of}
     open_stay: Dict[int, int] = {}            # ring tensor -> arena offset of its current stay
-    pin_loaded = set()
+    pin_loaded = set(kept)
     written_ever = set(written_before)
     last_wb_op: Dict[int, int] = {}
     fifo: List[Tuple[int, int, int]] = []     # (start, end, last-use op) of ring stays, oldest first
@@ -362,7 +391,7 @@ def plan(tensors, ops, steps, machine: Machine, budget: int, bits: int = BIT_A |
 
 
 def plan_tail(tensors, ops, steps, machine: Machine, budget: int, first_step: int, bits: int = BIT_A | BIT_P | BIT_ZC | BIT_W,
-              measured_ns=None) -> Plan:
+              measured_ns=None, resident=None) -> Plan:
     """Re-plan at a step boundary, while the run is under way (Section IV-E "Runtime Monitor": classes are re-evaluated
     from measured kernel times and the engine adapts; the paper does not say how the switch is made).  Reading: the
     steps from first_step on are planned as a trace of their own, with the same policy.  At the boundary the engine has
@@ -370,7 +399,10 @@ def plan_tail(tensors, ops, steps, machine: Machine, budget: int, first_step: in
     so nothing is resident and the pool is up to date: the tail plan starts from an empty arena, and a tensor written in
     an earlier step holds data, so its first access loads it (H2D) even when that access is a write.
     measured_ns: one entry per op of the WHOLE trace (0 = not measured).  Op indices in the returned commands are those
-    of the whole trace; classes and per-step totals cover the tail only."""
+    of the whole trace; classes and per-step totals cover the tail only.
+    resident (tensor -> arena offset): the pinned tensors of the plan in use that are on the device at the boundary.  Given,
+    the switch keeps them: those the tail plan pins again stay where they are, hold the newest data (the engine then
+    writes back only the written pins it gives up) and are not loaded again; the windowed reservation is not applied."""
     import copy
     first_op = steps[first_step][1]
     written = set()
@@ -385,7 +417,7 @@ def plan_tail(tensors, ops, steps, machine: Machine, budget: int, first_step: in
         sub_ops.append(o)
     sub_steps = [(k, o0 - first_op, n) for (k, o0, n) in steps[first_step:]]
     pl = plan(tensors, sub_ops, sub_steps, machine, budget, bits,
-              None if measured_ns is None else list(measured_ns[first_op:]), written_before=written)
+              None if measured_ns is None else list(measured_ns[first_op:]), written_before=written, resident=resident)
     for c in pl.cmds:
         if c.wait_op >= 0:
             c.wait_op += first_op

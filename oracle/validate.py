@@ -56,11 +56,14 @@ def parse(blobs, n_tensors):
                 ring_size=ring_size, totals=totals, classes=list(blobs["classes"]))
 
 
-def check(tensors, ops, steps, budget, blobs, first_step=0):
+def check(tensors, ops, steps, budget, blobs, first_step=0, resident=None):
     """Raises PlanInvalid with a reason; returns a small summary dict when everything holds.
     first_step > 0: `blobs` is a tail plan made at that step boundary for the rest of the trace (op indices of the
     whole trace); the replay then starts from an empty arena with every tensor written in an earlier step holding
-    data in the pool, so such a tensor may never be placed by ALLOC."""
+    data in the pool, so such a tensor may never be placed by ALLOC.
+    resident (tensor -> arena offset): pinned tensors that are on the device at the boundary, with the newest data; a pin
+    of the tail plan at the same offset starts the replay resident (the pool's copy of one written earlier is stale: it
+    was not written back), and must not be placed again."""
     P = parse(blobs, len(tensors))
     first_op = steps[first_step][1]
     written_before = {t for op in ops[:first_op] for (t, mode, _) in op.acc if mode & 2}
@@ -117,6 +120,11 @@ def check(tensors, ops, steps, budget, blobs, first_step=0):
     host_ver = [1 if t in written_before else 0 for t in range(len(tensors))]
     newest = list(host_ver)
     stays = {}                      # tensor -> [arena_off, release_after, version held, is_pin]
+    for t, off in (resident or {}).items():
+        if pin_off.get(t) == off:
+            stays[t] = [off, N - 1, newest[t], True]
+            if newest[t]:
+                host_ver[t] = 0     # written on the device, not written back at the switch
     placed = []                     # (start, end, release_after) of ring stays not yet overwritten
     tenants = []                    # (start, end, release_after) of placements of unpinned tensors inside the pin region
     ring_wait = -1

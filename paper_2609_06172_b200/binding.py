@@ -80,6 +80,7 @@ _SIGS = {
     "tgp_replan_begin": [_P, _U32, C.POINTER(_U64), _U64],
     "tgp_replan_wait": [_P],
     "tgp_replan_commit": [_P],
+    "tgp_set_replan_keep": [C.c_void_p, C.c_int],
     "tgp_plan_export": [_P, _U32, _P, C.POINTER(_U64)],
     "tgp_set_arena": [_P, _P, _U64],
     "tgp_model_workspace_bytes": [C.POINTER(ModelCfg), _U32, C.POINTER(_U64)],
@@ -280,6 +281,9 @@ class Ctx:
 
     def replan_commit(self):
         self._ck(lib().tgp_replan_commit(self._h), "tgp_replan_commit")
+
+    def set_replan_keep(self, keep):
+        self._ck(lib().tgp_set_replan_keep(self._h, int(keep)), "tgp_set_replan_keep")
 
     def set_budget(self, nbytes):
         self._ck(lib().tgp_set_budget(self._h, nbytes), "tgp_set_budget")

@@ -906,9 +906,12 @@ extern "C" int tgp_replan_commit(tgp_ctx *ctx) {
     for (uint32_t i = 0; i < ctx->tail_plan.first_op; ++i)
         for (uint32_t k = 0; k < ctx->ops[i].nacc; ++k)
             if (ctx->acc[ctx->ops[i].acc0 + k].mode & TGP_W) written[ctx->acc[ctx->ops[i].acc0 + k].tensor] = 1;
+    // written pinned tensors go back to the pool - except those the tail plan keeps where they are (they hold the newest data)
+    std::vector<uint8_t> kept(ctx->tensors.size(), 0);
+    for (uint32_t t : ctx->tail_plan.kept) kept[t] = 1;
     for (auto &pin : ctx->plan.pins) {
         const TgpTensor &t = ctx->tensors[pin.first];
-        if (t.flags == TGP_T_MUTABLE && written[pin.first])
+        if (t.flags == TGP_T_MUTABLE && written[pin.first] && !kept[pin.first])
             CU(ctx, cudaMemcpy(ctx->pools[t.pool].host_base + t.off, (char *)ctx->arena + pin.second, t.size, cudaMemcpyDeviceToHost));
     }
     if (!ctx->base_plan.valid) ctx->base_plan = std::move(ctx->plan);       // kept for the next tgp_run_reset()

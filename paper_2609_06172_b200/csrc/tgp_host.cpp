@@ -226,6 +226,13 @@ int tgp_set_budget(tgp_ctx *ctx, uint64_t bytes) {
     return TGP_OK;
 }
 
+int tgp_set_replan_keep(tgp_ctx *ctx, int keep) {
+    if (!ctx) return TGP_E_INVAL;
+    if (ctx->replan_thread.joinable()) ctx->replan_thread.join();
+    ctx->replan_keep = keep != 0;
+    return TGP_OK;
+}
+
 int tgp_set_measured_times(tgp_ctx *ctx, const uint64_t *op_ns, uint64_t n_ops) {
     if (!ctx) return TGP_E_INVAL;
     if (ctx->replan_thread.joinable()) ctx->replan_thread.join();      // a re-plan under way reads these inputs
@@ -367,12 +374,48 @@ static int build_plan(const tgp_ctx *ctx, uint32_t first_step, TgpPlan &out, std
             g0 = g1;
         }
     }
-    for (size_t t = 0; t < T; ++t) if (pin_off[t] >= 0) pl.pins.push_back({(uint32_t)t, (uint64_t)pin_off[t]});
+    // Pins that are resident already (a plan made in the middle of a run that keeps them): a chosen tensor that is on the
+    // device keeps its place and is not loaded again; the others go, in the order they were chosen, into the first gap
+    // between the kept ones that holds them (none: not pinned after all).  The pin region ends where the longer of the two
+    // layouts ends.  Resident = a pin of the plan in use that was placed before the boundary, or that the plan itself kept.
+    std::vector<uint8_t> kept(T, 0);
+    const bool keep = first_step > 0 && ctx->replan_keep && ctx->plan.valid;
+    if (keep) {
+        std::vector<int64_t> res(T, -1), old_off(T, -1);
+        for (auto &pin : ctx->plan.pins) old_off[pin.first] = (int64_t)pin.second;
+        std::vector<int32_t> placed_at(T, -2);               // first use of the pin's own placement in the plan in use; -2: it has none
+        for (const TgpCmd &c : ctx->plan.cmds)
+            if (c.kind != CMD_D2H && old_off[c.tensor] >= 0 && (int64_t)c.arena_off == old_off[c.tensor] && placed_at[c.tensor] == -2) placed_at[c.tensor] = c.first_use;
+        for (auto &pin : ctx->plan.pins)
+            if (placed_at[pin.first] == -2 || placed_at[pin.first] < (int32_t)O0) res[pin.first] = (int64_t)pin.second;   // kept by that plan itself, or placed before the boundary
+        std::vector<uint32_t> chosen;
+        for (size_t t = 0; t < T; ++t) if (pin_off[t] >= 0) chosen.push_back((uint32_t)t);
+        std::sort(chosen.begin(), chosen.end(), [&](uint32_t a, uint32_t b) { return pin_off[a] < pin_off[b]; });
+        uint64_t region_end = used;
+        std::vector<std::pair<uint64_t, uint64_t>> iv;
+        for (uint32_t t : chosen)
+            if (res[t] >= 0) { kept[t] = 1; iv.push_back({(uint64_t)res[t], (uint64_t)res[t] + alignup(ten[t].size)}); region_end = std::max(region_end, iv.back().second); }
+        std::sort(iv.begin(), iv.end());
+        std::vector<std::pair<uint64_t, uint64_t>> holes;
+        uint64_t pos = 0;
+        for (auto &v : iv) { if (v.first > pos) holes.push_back({pos, v.first}); pos = std::max(pos, v.second); }
+        if (pos < region_end) holes.push_back({pos, region_end});
+        for (uint32_t t : chosen) {
+            if (kept[t]) { pin_off[t] = res[t]; continue; }
+            const uint64_t a = alignup(ten[t].size);
+            pin_off[t] = -1;
+            for (auto &h : holes)
+                if (h.second - h.first >= a) { pin_off[t] = (int64_t)h.first; h.first += a; break; }
+        }
+        used = region_end;
+        if (ctx->budget - used < ring_min) return fail(TGP_E_BUDGET_TOO_SMALL, "kept pins leave less than the ring minimum");
+    }
+    for (size_t t = 0; t < T; ++t) if (pin_off[t] >= 0) { pl.pins.push_back({(uint32_t)t, (uint64_t)pin_off[t]}); if (kept[t]) pl.kept.push_back((uint32_t)t); }
     pl.ring_base = used; pl.ring_size = ctx->budget - used;
     // windowed reservation: the slot of a pinned tensor that is born on the device in a later step houses tenants until then
     std::vector<int64_t> tenant_off(T, -1);
     std::vector<int32_t> tenant_last(T, -1), landlord_wait(T, -1);
-    if ((ctx->bits & TGP_BIT_W) && !pl.pins.empty()) {
+    if ((ctx->bits & TGP_BIT_W) && !pl.pins.empty() && !keep) {
         std::vector<uint8_t> written0(T, 0);
         for (size_t i = 0; i < O0; ++i)
             for (uint32_t k = 0; k < ctx->ops[i].nacc; ++k)
@@ -435,7 +478,7 @@ static int build_plan(const tgp_ctx *ctx, uint32_t first_step, TgpPlan &out, std
     int32_t run_wait = -1;
     std::vector<uint32_t> stay_idx(T, 0);
     std::vector<int64_t> open_at(T, -1);                 // arena offset of the open stay, -1 if none
-    std::vector<uint8_t> pin_loaded(T, 0), written_ever(T, 0), dirty(T, 0);
+    std::vector<uint8_t> pin_loaded(kept), written_ever(T, 0), dirty(T, 0);
     for (size_t i = 0; i < O0; ++i)                      // a tail plan: what earlier steps wrote holds data in the pool
         for (uint32_t k = 0; k < ctx->ops[i].nacc; ++k)
             if (ctx->acc[ctx->ops[i].acc0 + k].mode & TGP_W) written_ever[ctx->acc[ctx->ops[i].acc0 + k].tensor] = 1;

@@ -34,6 +34,7 @@ struct TgpPlan {
     std::vector<uint8_t> cls, crit, zc;
     std::vector<uint64_t> score;
     std::vector<std::pair<uint32_t, uint64_t>> pins;
+    std::vector<uint32_t> kept;          // pins that were resident when the plan began (a tail plan that keeps pins): never placed
     uint64_t ring_base = 0, ring_size = 0;
     std::vector<TgpCmd> cmds;
     std::vector<uint64_t> totals;        // 4 per step
@@ -69,6 +70,7 @@ struct tgp_ctx {
     TgpPlan tail_plan, base_plan;                        // base_plan: the whole-run plan set aside while a tail plan is in use
     std::thread replan_thread;
     bool tail_ready = false;
+    bool replan_keep = false;            // tail plans keep the resident pins of the plan in use (tgp_set_replan_keep)
     int tail_rc = 0;
     uint32_t tail_step = 0;
     std::string tail_err;

@@ -807,6 +807,69 @@ def test_runtime_monitor_replan_from_measured_kernel_times():
     s.close()
 
 
+def test_replan_that_keeps_the_pins_switches_twice_without_reloading_them():
+    """tgp_set_replan_keep: at a switch the pinned tensors that are on the device stay where they are.  Two switches in one
+    run (the second from a plan that itself kept pins): each tail schedule is bit for bit the oracle's for the resident set
+    read off the plan in use, passes the validator started with that set resident, and places none of the kept tensors;
+    the step after a switch copies far fewer bytes than the same step after a cold switch; the logits of every step -
+    KV tiles written before a switch are read after it from where they stayed - equal those of the run that never
+    switched, bit for bit."""
+    cfg = si.CONFIGS[1]
+    lay, pool, s, blobs, T = setup(cfg)
+    r = Runner(s, cfg.B * cfg.S)
+    prompt = si.prompt_tokens(cfg)
+    forced = (np.arange(cfg.B * T, dtype=np.int32).reshape(cfg.B, T) * 211 + 5) % cfg.V
+    plain, _ = r.generate(prompt, T, forced=forced)
+    ops, steps = trace.run_trace(lay)
+    mach = policy.Machine(**MACHINE)
+    nt = len(lay.tensors)
+
+    def resident_of(b, first_op):
+        P = validate.parse(b, nt)
+        placed = {}
+        for (seq, kind, t, nb, po, ao, w, f, rel) in P["cmds"]:
+            if kind != validate.CMD_D2H:
+                placed.setdefault((t, ao), f)
+        return {t: o for t, o in P["pins"] if placed.get((t, o), -1) < first_op}
+
+    def run(keep, boundaries):
+        r.reset()
+        s.ctx.set_replan_keep(keep)
+        out, h2d, tails = [], [], {}
+        for k in range(1 + T):
+            if k + 2 in boundaries:
+                s.ctx.replan_begin(k + 2)
+            if k in boundaries:
+                in_use = s.ctx.plan_blobs()
+                s.ctx.replan_commit()
+                tails[k] = (in_use, s.ctx.plan_blobs())
+            tok = prompt if k == 0 else np.ascontiguousarray(forced[:, k - 1:k], dtype=np.int32)
+            st = r.step(tb.PREFILL if k == 0 else tb.DECODE, tok, tok.shape[1], want_stats=True)
+            h2d.append(st.h2d_bytes)
+            out.append(r.logits.cpu().numpy().copy())
+        r.sync()
+        return out, h2d, tails
+
+    cold_out, cold_h2d, _ = run(False, (4, 9))
+    keep_out, keep_h2d, tails = run(True, (4, 9))
+    for k, (in_use, tail) in tails.items():
+        res = resident_of(in_use, steps[k][1])
+        assert tail == policy.plan_tail(lay.tensors, ops, steps, mach, lay.budget, k, resident=res).blobs()
+        validate.check(lay.tensors, ops, steps, lay.budget, tail, first_step=k, resident=res)
+        P = validate.parse(tail, nt)
+        kept = {t for t, o in res.items() if dict(P["pins"]).get(t) == o}
+        assert kept and not ({c[2] for c in P["cmds"] if c[1] != validate.CMD_D2H} & kept)
+        assert keep_h2d[k] < 0.6 * cold_h2d[k]                      # the cold switch reloads the pinned half of the pool in this step
+    for a, b, c in zip(keep_out, cold_out, plain):
+        assert np.array_equal(a, c) and np.array_equal(b, c)
+    s.ctx.set_replan_keep(False)
+    again, _ = r.generate(prompt, T, forced=forced)
+    assert s.ctx.plan_blobs() == blobs
+    for a, b in zip(again, plain):
+        assert np.array_equal(a, b)
+    s.close()
+
+
 @pytest.mark.parametrize("budget", [None, 3 << 20])
 def test_replan_in_the_middle_of_a_run_switches_plans_at_a_step_boundary(budget):
     """Runtime monitor while the run is under way: after decode step 3 the timing log so far is handed to the planner,

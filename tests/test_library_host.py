@@ -366,6 +366,56 @@ def test_tail_replan_in_the_middle_of_a_run_is_bit_exact(c, first_step):
     s.close()
 
 
+def _resident_of(blobs, n_tensors, first_op):
+    """tensor -> arena offset of the pins of a plan that are on the device when op first_op starts: placed before it, or
+    never placed at all (kept by that plan itself)."""
+    P = validate.parse(blobs, n_tensors)
+    placed = {}
+    for (seq, kind, t, nb, po, ao, w, f, r) in P["cmds"]:
+        if kind != validate.CMD_D2H:
+            placed.setdefault((t, ao), f)
+    return {t: o for t, o in P["pins"] if placed.get((t, o), -1) < first_op}
+
+
+@pytest.mark.parametrize("c,first_step", [(1, 2), (1, 9), (2, 3)])
+def test_tail_replan_that_keeps_the_resident_pins_is_bit_exact(c, first_step):
+    """With tgp_set_replan_keep the tail plan keeps the pinned tensors that are on the device at the boundary: same blobs as
+    the oracle's tail planner given that resident set, valid for a replay that starts with them resident, nothing of
+    them placed again, fewer bytes in the first tail step than a tail that starts cold; with the switch off again the
+    planner returns the cold tail."""
+    cfg = si.CONFIGS[c] if c == 1 else replace(si.CONFIGS[c], T=8)
+    lay = si.build_layout(cfg)
+    ops, steps = trace.run_trace(lay)
+    mach = policy.Machine(**MACHINE)
+    rng = np.random.default_rng(10 + first_step)
+    ns = np.zeros(len(ops), dtype=np.uint64)
+    ns[:steps[first_step][1]] = rng.integers(500, 40000, steps[first_step][1])
+    s = Session(lay, MACHINE)
+    base = s.plan(T=cfg.T)
+    s.ctx.replan_begin(first_step, ns)
+    s.ctx.replan_wait()
+    cold = s.ctx.plan_blobs(tail=True)
+    s.ctx.set_replan_keep(True)
+    s.ctx.replan_begin(first_step, ns)
+    s.ctx.replan_wait()
+    got = s.ctx.plan_blobs(tail=True)
+    res = _resident_of(base, len(lay.tensors), steps[first_step][1])
+    assert res
+    want = policy.plan_tail(lay.tensors, ops, steps, mach, lay.budget, first_step, measured_ns=ns.tolist(), resident=res).blobs()
+    assert got == want
+    validate.check(lay.tensors, ops, steps, lay.budget, got, first_step=first_step, resident=res)
+    P = validate.parse(got, len(lay.tensors))
+    off = dict(P["pins"])
+    kept = {t for t, o in res.items() if off.get(t) == o}
+    assert kept and not ({c[2] for c in P["cmds"] if c[1] != validate.CMD_D2H} & kept)
+    assert validate.parse(got, len(lay.tensors))["totals"][0][0] < validate.parse(cold, len(lay.tensors))["totals"][0][0]
+    s.ctx.set_replan_keep(False)
+    s.ctx.replan_begin(first_step, ns)
+    s.ctx.replan_wait()
+    assert s.ctx.plan_blobs(tail=True) == cold                              # the switch is per plan: off again, the cold tail again
+    s.close()
+
+
 def test_measured_time_link_test_by_hand():
     toy = policy.Machine(1000, 100, 10, 10)            # link 10 B/s
     # 100 bytes over the link take 10 s: a 9 s kernel is link-bound, a 10 s or 11 s kernel is not

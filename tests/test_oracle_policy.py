@@ -281,6 +281,100 @@ def test_tail_plan_closed_forms_and_invariants():
         validate.check(lay.tensors, ops, steps, lay.budget, _tamper(blobs, to_alloc), first_step=4)
 
 
+def _resident_at(plan, first_op):
+    """tensor -> arena offset of the pins of `plan` that are on the device when op `first_op` starts."""
+    off = dict(plan.pins)
+    return {c.tensor: c.arena_off for c in plan.cmds if c.kind != policy.CMD_D2H and c.first_use < first_op and off.get(c.tensor) == c.arena_off}
+
+
+def test_tail_plan_that_keeps_the_resident_pins():
+    """A switch of plans in the middle of a run that keeps what is pinned and loaded: (1) the tail plan passes the validator
+    started with those tensors resident (a second placement of one of them, or a kept tensor at another offset, is caught);
+    (2) with nothing measured the tail pins what the whole-run plan pinned (same densities per step) and every kept pin
+    stays at its offset, so the only loads of pinned tensors are those of pins the run had not reached yet; (3) the first
+    tail step moves fewer bytes than a tail that starts from an empty arena, by the bytes of the kept pins it touches, and a
+    later steady step moves the same; (4) a written KV tile that is kept is never copied from the pool (its copy there is
+    stale), one that is not kept is loaded."""
+    cfg = replace(si.CONFIGS[1], S=30, T=8)
+    lay = si.build_layout(cfg)
+    ops, steps = trace.run_trace(lay)
+    whole = policy.plan(lay.tensors, ops, steps, M, lay.budget)
+    for k in (1, 3, 5):
+        first_op = steps[k][1]
+        res = _resident_at(whole, first_op)
+        assert res
+        cold = policy.plan_tail(lay.tensors, ops, steps, M, lay.budget, k)
+        keep = policy.plan_tail(lay.tensors, ops, steps, M, lay.budget, k, resident=res)
+        validate.check(lay.tensors, ops, steps, lay.budget, keep.blobs(), first_step=k, resident=res)
+        with pytest.raises(validate.PlanInvalid):
+            validate.check(lay.tensors, ops, steps, lay.budget, keep.blobs(), first_step=k)          # nothing resident: kept pins are missing
+        off = dict(keep.pins)
+        kept = {t for t, o in res.items() if off.get(t) == o}
+        assert kept and all(off[t] == res[t] for t in res if t in off)                              # a resident tensor never moves
+        placed = {c.tensor for c in keep.cmds if c.kind != policy.CMD_D2H}
+        assert not (placed & kept)
+        # pins do not overlap and stay below the ring
+        spans = sorted((o, o + policy.alignup(lay.tensors[t].size)) for t, o in keep.pins)
+        assert all(b <= c for (a, b), (c, d) in zip(spans, spans[1:])) and spans[-1][1] <= keep.ring_base
+        assert keep.ring_base + keep.ring_size == lay.budget
+        # bytes: the first tail step saves the kept pins it touches; a steady step costs at most what a cold tail without the
+        # windowed reservation costs (the kept plan does not lend late-born pins' slots)
+        cold_now = policy.plan_tail(lay.tensors, ops, steps, M, lay.budget, k, bits=policy.BIT_A | policy.BIT_P | policy.BIT_ZC)
+        touched = {t for o in ops[first_op:first_op + steps[k][2]] for (t, _, _) in o.acc}
+        saved = sum(lay.tensors[t].size for t in kept & touched if t in dict(cold_now.pins))
+        assert keep.totals[0][0] <= cold_now.totals[0][0] - saved + sum(lay.tensors[t].size for t in touched if t in dict(cold_now.pins) and t not in off)
+        assert keep.totals[0][0] < cold.totals[0][0]
+        # written tiles
+        written = {t for o in ops[:first_op] for (t, m, _) in o.acc if m & 2}
+        assert written & kept
+        for c in keep.cmds:
+            assert not (c.tensor in kept and c.kind == policy.CMD_H2D)
+    # tampering: the same plan with a kept tensor's pin moved is rejected
+    k = 3
+    first_op = steps[k][1]
+    res = _resident_at(whole, first_op)
+    keep = policy.plan_tail(lay.tensors, ops, steps, M, lay.budget, k, resident=res)
+    moved = dict(res)
+    t0 = next(t for t in res if t in dict(keep.pins))
+    moved[t0] += 512
+    with pytest.raises(validate.PlanInvalid):
+        validate.check(lay.tensors, ops, steps, lay.budget, keep.blobs(), first_step=k, resident=moved)
+
+
+def test_kept_pins_fill_gaps_first_fit_on_a_toy():
+    """Hand-checked layout: four read-only tensors of 1, 2, 1 and 1 KiB units are pinned at 0, 1, 3, 4 by the first plan;
+    in the tail the second one is no longer used, so a hole of 2 units opens at offset 1.  A tensor of 2 units that the
+    tail pins anew goes into that hole (first fit), one of 3 units does not fit any gap below the old end and goes after
+    the last kept pin only if the region may grow: the region ends at max(compact size, end of the kept pins)."""
+    U = 1024
+    sizes = [1 * U, 2 * U, 1 * U, 1 * U, 2 * U, 3 * U]
+    tensors = [_T(sz, sum(sizes[:i])) for i, sz in enumerate(sizes)]
+    ops, steps = [], []
+    def step(st, used):
+        o0 = len(ops)
+        for t in used:
+            ops.append(_O(st, 10, 10, [(t, 1, sizes[t])]))
+            ops.extend(_O(st, 10, 10, []) for _ in range(policy.W_AFF + 1))
+        steps.append((1 if st else 0, o0, len(ops) - o0))
+    step(0, [0, 1, 2, 3]); step(1, [0, 1, 2, 3])
+    for st in range(2, 6):
+        step(st, [0, 2, 3, 4, 5])
+    budget = 2 * 3 * U + 8 * U                       # ring minimum (twice the largest tensor) + room for 8 units of pins
+    # (the plan in use was made when only the first two steps were known: it pins tensors 0 - 3, in id order)
+    first = policy.plan(tensors, ops[:steps[2][1]], steps[:2], M, budget, bits=policy.BIT_A | policy.BIT_P)
+    res = _resident_at(first, steps[2][1])
+    assert res == {0: 0, 1: 1 * U, 2: 3 * U, 3: 4 * U}
+    tail = policy.plan_tail(tensors, ops, steps, M, budget, 2, bits=policy.BIT_A | policy.BIT_P, resident=res)
+    validate.check(tensors, ops, steps, budget, tail.blobs(), first_step=2, resident=res)
+    off = dict(tail.pins)
+    assert 1 not in off and all(off[t] == res[t] for t in (0, 2, 3))
+    hole = res[1]
+    assert off[4] == hole                            # two units: exactly the hole the unused tensor left
+    end_kept = max(res[t] + sizes[t] for t in (0, 2, 3))
+    assert off[5] >= end_kept or 5 not in off        # three units fit no gap between kept pins
+    assert tail.ring_base == max(sum(sizes[t] for t in off), end_kept if 5 not in off else off[5] + sizes[5])
+
+
 def _window_toy(n_w=5, born=3, n_steps=6, size=4096):
     """n_w read-only tensors read once per step, and one mutable tensor of the same size first written in step `born`
     and read and written in every step after it (a KV tile of later positions)."""
